@@ -1,0 +1,65 @@
+"""Pipeline of Linear+activation stages with an MSE loss: the gradient function grad f_t(u_fwd, u_bkwd).
+
+TEST INFRASTRUCTURE (see package docstring).
+
+A stage holds its Linear layers' tensors in the order [W_0, b_0, W_1, b_1, ...].
+Forward runs stages 1..P with u_fwd; the loss is the mean squared error of the
+last stage's output against the target; backward runs stages P..1 and reads
+u_bkwd only in the input-gradient products (Section 2.1's two-argument
+gradient).  The first layer of the network has no input gradient, so its
+backward weights are never read.
+
+Parity of whole training trajectories is unpinned by the paper; this module is
+pinned through finite differences (u_fwd = u_bkwd) and through the special
+cases of the recurrence that use it.
+"""
+import numpy as np
+
+from . import layers as L
+from .bf16 import bf16_round
+
+
+def make_grad_fn(stage_acts, data_fn, compute="f32"):
+    """stage_acts: per stage, the list of activation names of its Linear layers.
+    data_fn: t -> (x [T,in], target [T,out]).  compute: 'f32' | 'bf16'."""
+    rnd = bf16_round if compute == "bf16" else L.identity
+
+    def grad_fn(t, u_fwd, u_bkwd):
+        x, target = data_fn(t)
+        h = rnd(np.asarray(x, dtype=np.float64))
+        stash = []
+        for acts, wf in zip(stage_acts, u_fwd):
+            for j, act in enumerate(acts):
+                W = np.asarray(wf[2 * j], dtype=np.float64)
+                b = np.asarray(wf[2 * j + 1], dtype=np.float64)
+                y, z = L.linear_fwd(h, W, b, act, rnd)
+                stash.append((h, z))
+                h = y
+        loss, dy = L.mse_loss(h, target, rnd)
+        grads = [[None] * len(wf) for wf in u_fwd]
+        flat = len(stash) - 1
+        for i in reversed(range(len(stage_acts))):
+            for j in reversed(range(len(stage_acts[i]))):
+                x_in, z = stash[flat]
+                Wb = np.asarray(u_bkwd[i][2 * j], dtype=np.float64)
+                dW, db, dy = L.linear_bwd(dy, x_in, z, Wb, stage_acts[i][j], rnd, need_dx=flat > 0)
+                grads[i][2 * j], grads[i][2 * j + 1] = dW, db
+                flat -= 1
+        return loss, grads
+
+    return grad_fn
+
+
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None):
+    """Run a pm_inputs.Workload-like description through the recurrence.
+
+    params0: per stage a list of (W, b) pairs.  Returns recurrence.Result.
+    """
+    from . import recurrence
+    stage_acts = [[spec.act for spec in stage] for stage in wl.stages]
+    flat0 = [[t for pair in stage for t in pair] for stage in params0]
+    hp = dict(optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+              t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
+    grad_fn = make_grad_fn(stage_acts, data_fn, wl.compute)
+    return recurrence.run(flat0, wl.tau_fwd, wl.tau_bkwd, grad_fn,
+                          wl.steps if n_steps is None else n_steps, hp, dtype=dtype, on_step=on_step)

@@ -1,0 +1,24 @@
+"""Gradient samples of the one-dimensional quadratic models (Sections 3, 3.1, 3.2).
+
+TEST INFRASTRUCTURE (see package docstring).
+
+    f(w) = lambda w^2 / 2
+    no discrepancy:   grad = lambda * u_fwd - eta_t                      (Section 3)
+    with discrepancy: grad = (lambda + Delta) u_fwd - Delta u_bkwd - eta_t   (Section 3.2)
+
+These plug into recurrence.run as a single stage holding one scalar, so the
+stability lemmas and characteristic polynomials of the paper test the very
+loop the network workloads go through.
+"""
+import numpy as np
+
+
+def quadratic_grad(lam, Delta=0.0, noise=None):
+    """Return grad_fn for recurrence.run; noise: optional callable t -> eta_t."""
+    def grad_fn(t, u_fwd, u_bkwd):
+        wf = u_fwd[0][0]
+        wb = u_bkwd[0][0]
+        eta = 0.0 if noise is None else noise(t)
+        g = (lam + Delta) * wf - Delta * wb - eta
+        return float(0.5 * lam * wf[0] ** 2), [[np.asarray(g)]]
+    return grad_fn

@@ -1,0 +1,86 @@
+"""The delayed-update recurrence of Section 2.1, microbatch-major, with a queue of weight versions.
+
+TEST INFRASTRUCTURE (see package docstring).
+
+    w_{t+1} = w_t - alpha * grad f_t(u_fwd,t , u_bkwd,t)
+    (u_fwd,t)_i  = (w_{t - tau_fwd,i})_i
+    (u_bkwd,t)_i = (w_{t - tau_bkwd,i})_i  [ - (tau_fwd,i - tau_bkwd,i) * delta_{t,i}  with T2 ]
+
+"(w_t)_i" is stage i's weights after t updates have been written to it.  The
+gradient function receives both weight sets and must use u_fwd wherever the
+forward pass reads a weight and u_bkwd wherever the backward pass reads one.
+
+Readings where the paper is silent:
+  * t < tau: the version index is clamped at 0 (the pipeline is still filling
+    and the initial weights are the only ones that exist).
+  * delta_0 = 0.
+  * All reads of version t (every stage's backward) happen before any stage
+    writes version t+1.
+  * One microbatch per update (N = 1): microbatch index = update index.
+
+Pins: with all tau = 0 the loop is synchronous SGD, bit for bit; with T2 off
+and tau_bkwd = tau_fwd it is plain delayed SGD; on the scalar quadratic its
+iterates follow the roots of the characteristic polynomials of Sections 3.1,
+3.2 and Appendix B.3 (tests/test_oracle_recurrence.py).
+"""
+from collections import deque
+
+import numpy as np
+
+from . import update as U
+
+
+class Result:
+    def __init__(self):
+        self.losses = []      # loss of microbatch t, computed from its (stale) forward weights
+        self.book = []        # (t, stage index (1-based), forward version, backward version)
+        self.params = None    # final per-stage lists of tensors
+        self.delta = None
+        self.opt = None
+
+
+def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None):
+    """Run n_steps microbatches.
+
+    params0:   per stage, a list of arrays (that stage's tensors).
+    grad_fn:   (t, u_fwd, u_bkwd) -> (loss, grads) with grads shaped like params0.
+    hp:        hyper-parameters (see update.pipemare_update).
+    on_step:   optional callback (t, params) after the update of step t.
+    """
+    P = len(params0)
+    w = [[np.array(a, dtype=dtype) for a in stage] for stage in params0]
+    opt = [[U.fresh_opt_state(a, hp["optimizer"]) for a in stage] for stage in w]
+    delta = [[np.zeros_like(a) for a in stage] for stage in w]
+    depth = [max(tau_fwd[i], tau_bkwd[i]) + 1 for i in range(P)]
+    # queue of versions per stage: hist[i][-1] is version t, hist[i][-1-d] is version t-d
+    hist = [deque([w[i]], maxlen=depth[i]) for i in range(P)]
+    res = Result()
+
+    def version(i, t, lag):
+        v = max(0, t - lag)
+        return v, hist[i][-1 - (t - v)]
+
+    for t in range(n_steps):
+        u_fwd, u_bkwd = [], []
+        for i in range(P):
+            vf, wf = version(i, t, tau_fwd[i])
+            vb, wb = version(i, t, tau_bkwd[i])
+            u_fwd.append(wf)
+            u_bkwd.append([U.corrected_backward_weights(a, d, tau_fwd[i], tau_bkwd[i], hp["t2"])
+                           for a, d in zip(wb, delta[i])])
+            res.book.append((t, i + 1, vf, vb))
+        loss, grads = grad_fn(t, u_fwd, u_bkwd)
+        res.losses.append(loss)
+        for i in range(P):
+            new_stage = []
+            for j, a in enumerate(w[i]):
+                g = np.asarray(grads[i][j], dtype=dtype)
+                a_new, opt[i][j], delta[i][j] = U.pipemare_update(
+                    a, opt[i][j], delta[i][j], g, k=t, tau_fwd=tau_fwd[i], tau_bkwd=tau_bkwd[i], hp=hp)
+                new_stage.append(a_new)
+            w[i] = new_stage
+            hist[i].append(new_stage)
+        if on_step is not None:
+            on_step(t, w)
+    res.params, res.delta, res.opt = w, delta, opt
+    return res

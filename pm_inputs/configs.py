@@ -1,0 +1,190 @@
+"""Workload descriptions and the recipes for their seeded synthetic data.
+
+A workload is plain data: the stage list (which Linear layers ride in which
+pipeline stage), the per-stage delays, the optimiser's hyper-parameters and
+the seeds.  The recipes below turn a workload and a step index into tensors.
+The teacher network that labels the MLP workloads is evaluated here, in
+float64, with its own few lines of numpy; it is part of the data, not of the
+training method.
+"""
+from dataclasses import dataclass, field
+from typing import List
+
+import numpy as np
+from scipy.special import erf as _erf
+
+from . import rng
+
+# stream ids (purpose of a random draw)
+_S_INIT, _S_TEACHER, _S_INPUT, _S_CALIB = 1, 2, 3, 500000
+_CALIB_ROWS = 256
+_S_UPD_W, _S_UPD_G, _S_UPD_M, _S_UPD_S, _S_UPD_D = 10, 11, 12, 13, 14
+
+
+@dataclass
+class LinearSpec:
+    n_in: int
+    n_out: int
+    act: str  # 'relu' | 'gelu' | 'none'
+
+
+@dataclass
+class Workload:
+    name: str
+    stages: List[List[LinearSpec]]
+    tau_fwd: List[int]
+    tau_bkwd: List[int]
+    microbatch: int
+    compute: str = "f32"        # 'f32' | 'bf16' (GEMM operand type; state is always fp32)
+    optimizer: str = "sgdm"     # 'sgdm' | 'adam'
+    alpha: float = 0.01
+    beta1: float = 0.9
+    beta2: float = 0.98
+    eps: float = 1e-8
+    t1: bool = True
+    K: int = 32
+    t2: bool = True
+    D: float = 0.5
+    steps: int = 64
+    seed: int = 191005124
+    notes: str = field(default="")
+
+    @property
+    def n_stages(self):
+        return len(self.stages)
+
+
+def pipemare_delays(P, n_micro=1):
+    """Forward delays ceil((2(P-i)+1)/N) for i=1..P and zero backward delays (PipeMare row of Table 1)."""
+    fwd = [-(-(2 * (P - i) + 1) // n_micro) for i in range(1, P + 1)]
+    return fwd, [0] * P
+
+
+def mlp_workload(name, P, width, linears_per_stage, act, microbatch, **kw):
+    stages = [[LinearSpec(width, width, act) for _ in range(linears_per_stage)] for _ in range(P)]
+    fwd, bkwd = pipemare_delays(P)
+    return Workload(name=name, stages=stages, tau_fwd=fwd, tau_bkwd=bkwd, microbatch=microbatch, **kw)
+
+
+def cfg1():
+    """4-stage MLP, one Linear(256,256)+ReLU per stage, fp32, microbatch 32, 64 steps."""
+    return mlp_workload("cfg1_mlp4_f32", 4, 256, 1, "relu", 32, compute="f32", optimizer="sgdm",
+                        alpha=0.01, beta1=0.9, K=32, D=0.5, steps=64, seed=191005124 + 1)
+
+
+def cfg3():
+    """32-stage MLP, two Linear(1024,1024)+GELU per stage, bf16 GEMMs, microbatch 128, 500 steps."""
+    return mlp_workload("cfg3_mlp32_bf16", 32, 1024, 2, "gelu", 128, compute="bf16", optimizer="sgdm",
+                        alpha=0.01, beta1=0.9, K=125, D=0.5, steps=500, seed=191005124 + 3)
+
+
+def cfg3_small(P=6, width=192, microbatch=40, steps=40, optimizer="sgdm"):
+    """Same structure as cfg3 at a size the oracle runs in seconds (several tiles, ragged tails)."""
+    return mlp_workload("cfg3_small", P, width, 2, "gelu", microbatch, compute="bf16", optimizer=optimizer,
+                        alpha=0.01 if optimizer == "sgdm" else 5e-4, beta1=0.9, K=max(steps // 4, 1), D=0.5,
+                        steps=steps, seed=191005124 + 33)
+
+
+def round_to_bf16(x):
+    """Round float values to the nearest bfloat16 (ties to even); returns float32 holding those values."""
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    u = (u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) & np.uint64(0xFFFF0000)
+    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+
+
+def _act(z, kind):
+    if kind == "relu":
+        return np.maximum(z, 0.0)
+    if kind == "gelu":
+        return 0.5 * z * (1.0 + _erf(z / np.sqrt(2.0)))
+    return z
+
+
+def _all_params(wl, stream):
+    """Draw every Linear as N(0, 1/fan_in), then rescale layer by layer so that each
+    pre-activation has unit root-mean-square on a fixed seeded calibration batch.
+
+    A plain 64-layer GELU stack has no stable signal scale under a fixed-variance
+    init (it vanishes or explodes with depth); calibrating on data keeps every
+    layer's activations O(1) so that no part of the workload is degenerate.
+    Biases start at zero.
+    """
+    n_in = wl.stages[0][0].n_in
+    h = rng.normal(wl.seed, _S_CALIB + stream, _CALIB_ROWS * n_in).reshape(_CALIB_ROWS, n_in)
+    out, index = [], 0
+    for stage in wl.stages:
+        tensors = []
+        for spec in stage:
+            w = rng.normal(wl.seed, stream + 1000 * (index + 1), spec.n_in * spec.n_out)
+            w = w.reshape(spec.n_out, spec.n_in) / np.sqrt(spec.n_in)
+            z = h @ w.T
+            scale = 1.0 / np.sqrt(np.mean(z * z))
+            w32 = (w * scale).astype(np.float32)
+            h = _act(h @ w32.astype(np.float64).T, spec.act)
+            tensors.append((w32, np.zeros(spec.n_out, dtype=np.float32)))
+            index += 1
+        out.append(tensors)
+    return out
+
+
+def init_stage_params(wl):
+    """Initial student weights: per stage a list of (W[out,in], b[out]) float32 pairs."""
+    return _all_params(wl, _S_INIT)
+
+
+def teacher_params(wl):
+    """Frozen teacher of the same architecture, drawn from a different stream."""
+    return _all_params(wl, _S_TEACHER)
+
+
+def batch(wl, t, teacher=None):
+    """Microbatch t: x ~ N(0,1) of shape [M, in] and its teacher output y*, both float32.
+
+    For bf16 workloads x is rounded to bfloat16-representable values first so
+    that every consumer starts from identical operand bits.
+    """
+    n_in = wl.stages[0][0].n_in
+    x = rng.normal(wl.seed, _S_INPUT + 16 * t, wl.microbatch * n_in).reshape(wl.microbatch, n_in)
+    x = x.astype(np.float32)
+    if wl.compute == "bf16":
+        x = round_to_bf16(x)
+    if teacher is None:
+        teacher = teacher_params(wl)
+    h = x.astype(np.float64)
+    for stage, tensors in zip(wl.stages, teacher):
+        for spec, (w, b) in zip(stage, tensors):
+            h = _act(h @ w.astype(np.float64).T + b.astype(np.float64), spec.act)
+    return x, h.astype(np.float32)
+
+
+def update_sweep_case(n_params, P, optimizer="sgdm", seed=191005124 + 2, align=64):
+    """Update-only workload: n_params split evenly over P stages, each slice padded to `align` elements.
+
+    Returns a dict with per-stage (offset, count) in the padded flat arena, the
+    delays, and float32 arrays w ~ N(0,1), g ~ N(0, sigma=1e-3), and small
+    non-zero optimiser state so that no lane works on zeros or denormals.
+    """
+    base, rem = divmod(n_params, P)
+    counts = [base + (1 if i < rem else 0) for i in range(P)]
+    offsets, cur = [], 0
+    for c in counts:
+        offsets.append(cur)
+        cur += -(-c // align) * align
+    total = cur
+    fwd, bkwd = pipemare_delays(P)
+
+    def fill(stream, scale, positive=False):
+        a = np.zeros(total, dtype=np.float32)
+        for i, (o, c) in enumerate(zip(offsets, counts)):
+            v = rng.normal(seed, stream + 100 * i, c) * scale
+            a[o:o + c] = (v * v if positive else v).astype(np.float32)
+        return a
+
+    case = dict(n_params=n_params, P=P, optimizer=optimizer, offsets=offsets, counts=counts, total=total,
+                tau_fwd=fwd, tau_bkwd=bkwd,
+                w=fill(_S_UPD_W, 1.0), g=fill(_S_UPD_G, 1e-3), m=fill(_S_UPD_M, 1e-3),
+                delta=fill(_S_UPD_D, 1e-4))
+    if optimizer == "adam":
+        case["s"] = fill(_S_UPD_S, 1e-3, positive=True)
+    return case

@@ -1,0 +1,267 @@
+"""Pins for oracle/recurrence.py (+ quadratic.py): special cases the paper fixes and its stability theory."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import recurrence, update as U
+from oracle.quadratic import quadratic_grad
+from oracle.mlp import make_grad_fn
+
+
+def hp_(**kw):
+    hp = dict(optimizer="sgdm", alpha=0.05, beta1=0.0, beta2=0.98, eps=1e-8, t1=False, K=1, t2=False, D=0.5)
+    hp.update(kw)
+    return hp
+
+
+def tiny_net(seed=0, P=3, d=5, T=4, act="relu"):
+    rng = np.random.default_rng(seed)
+    params = [[rng.normal(size=(d, d)) * 0.5, rng.normal(size=d) * 0.1] for _ in range(P)]
+    X = rng.normal(size=(64, T, d))
+    Y = rng.normal(size=(64, T, d))
+    grad_fn = make_grad_fn([[act]] * P, lambda t: (X[t], Y[t]), "f32")
+    return params, grad_fn
+
+
+# ---- tau = 0: synchronous SGD, bit for bit (Section 2.1: u_fwd = u_bkwd) --------------------
+
+@pytest.mark.parametrize("dtype", [np.float64, np.float32])
+@pytest.mark.parametrize("optimizer", ["sgdm", "adam"])
+def test_all_tau_zero_is_synchronous_sgd_bit_for_bit(dtype, optimizer):
+    params, grad_fn = tiny_net()
+    P = len(params)
+    hp = hp_(optimizer=optimizer, alpha=0.03, beta1=0.9, t1=True, K=8, t2=True, D=0.5)
+    res = recurrence.run(params, [0] * P, [0] * P, grad_fn, 12, hp, dtype=dtype)
+    # separately written plain loop: one weight copy, ordinary gradient, ordinary optimiser
+    w = [[np.array(a, dtype=dtype) for a in st] for st in params]
+    st1 = [[np.zeros_like(a) for a in st] for st in w]
+    st2 = [[np.zeros_like(a) for a in st] for st in w]
+    losses = []
+    one = dtype(1)
+    for t in range(12):
+        loss, g = grad_fn(t, w, w)
+        losses.append(loss)
+        for i in range(P):
+            for j in range(2):
+                gij = np.asarray(g[i][j], dtype=dtype)
+                if optimizer == "sgdm":
+                    st1[i][j] = dtype(0.9) * st1[i][j] - dtype(0.03) * gij
+                    w[i][j] = w[i][j] + st1[i][j]
+                else:
+                    b1, b2 = dtype(0.9), dtype(0.98)
+                    st1[i][j] = b1 * st1[i][j] + (one - b1) * gij
+                    st2[i][j] = b2 * st2[i][j] + (one - b2) * (gij * gij)
+                    mh = st1[i][j] / dtype(1.0 - float(b1) ** (t + 1))
+                    sh = st2[i][j] / dtype(1.0 - float(b2) ** (t + 1))
+                    w[i][j] = w[i][j] - (dtype(0.03) * mh) / (np.sqrt(sh) + dtype(1e-8))
+    assert res.losses == losses
+    for i in range(P):
+        for j in range(2):
+            np.testing.assert_array_equal(res.params[i][j], w[i][j])
+            np.testing.assert_array_equal(res.delta[i][j], np.zeros_like(w[i][j]))
+
+
+# ---- T2 off, tau_bkwd = tau_fwd: plain delayed SGD  w_{t+1} = w_t - alpha grad f_t(w_{t-tau}) ----
+
+def test_equal_delays_is_plain_delayed_sgd_bit_for_bit():
+    params, grad_fn = tiny_net(seed=3, P=3)
+    tau = [5, 3, 1]
+    res = recurrence.run(params, tau, tau, grad_fn, 20, hp_(alpha=0.04), dtype=np.float64)
+    hist = [[[np.array(a) for a in st]] for st in params]      # hist[i][v] = version v of stage i
+    for t in range(20):
+        u = [hist[i][max(0, t - tau[i])] for i in range(3)]
+        _, g = grad_fn(t, u, u)
+        for i in range(3):
+            hist[i].append([hist[i][t][j] - 0.04 * g[i][j] for j in range(2)])
+    for i in range(3):
+        for j in range(2):
+            np.testing.assert_array_equal(res.params[i][j], hist[i][20][j])
+
+
+def test_pipemare_delays_without_t2_reads_current_weights_in_backward():
+    # tau_bkwd = 0, T2 off: forward version t - tau, backward version t (Section 2.2, PipeMare)
+    params, grad_fn = tiny_net(seed=4, P=3)
+    tau = [5, 3, 1]
+    res = recurrence.run(params, tau, [0, 0, 0], grad_fn, 15, hp_(alpha=0.04), dtype=np.float64)
+    hist = [[[np.array(a) for a in st]] for st in params]
+    for t in range(15):
+        uf = [hist[i][max(0, t - tau[i])] for i in range(3)]
+        ub = [hist[i][t] for i in range(3)]
+        _, g = grad_fn(t, uf, ub)
+        for i in range(3):
+            hist[i].append([hist[i][t][j] - 0.04 * g[i][j] for j in range(2)])
+    for i in range(3):
+        np.testing.assert_array_equal(res.params[i][0], hist[i][15][0])
+    # and it differs from the equal-delay run (the discrepancy is real)
+    res_eq = recurrence.run(params, tau, tau, grad_fn, 15, hp_(alpha=0.04), dtype=np.float64)
+    assert np.abs(res_eq.params[0][0] - res.params[0][0]).max() > 1e-8
+
+
+def test_bookkeeping_versions():
+    params, grad_fn = tiny_net(P=3)
+    tau = [5, 3, 1]
+    res = recurrence.run(params, tau, [0, 0, 0], grad_fn, 9, hp_(), dtype=np.float64)
+    book = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    assert book[(0, 1)] == (0, 0)
+    assert book[(4, 1)] == (0, 4)
+    assert book[(5, 1)] == (0, 5)
+    assert book[(6, 1)] == (1, 6)
+    assert book[(8, 2)] == (5, 8)
+    assert book[(8, 3)] == (7, 8)
+
+
+# ---- scalar quadratic: Lemma 1 and the characteristic polynomial of Section 3.1 -----------------
+
+def scalar_run(tau_f, tau_b, grad_fn, n, hp, w0=1.0):
+    traj = []
+    recurrence.run([[np.array([w0])]], [tau_f], [tau_b], grad_fn, n, hp, dtype=np.float64,
+                   on_step=lambda t, w: traj.append(float(w[0][0][0])))
+    return np.array([w0] + traj)
+
+
+def growth_rate(traj, lo, hi):
+    """Asymptotic per-step growth factor from the envelope of |w_t| over two windows."""
+    a = np.abs(traj)
+    w = (hi - lo) // 2
+    e1, e2 = a[lo:lo + w].max(), a[hi - w:hi].max()
+    return (e2 / e1) ** (1.0 / (hi - w - lo))
+
+
+@pytest.mark.parametrize("tau", [0, 1, 3, 5, 10])
+def test_lemma1_threshold_is_sharp(tau):
+    lam = 1.0
+    a_star = (2.0 / lam) * math.sin(math.pi / (4 * tau + 2))
+    n = 4000
+    below = scalar_run(tau, tau, quadratic_grad(lam), n, hp_(alpha=0.97 * a_star))
+    above = scalar_run(tau, tau, quadratic_grad(lam), n, hp_(alpha=1.03 * a_star))
+    assert np.abs(below[-200:]).max() < 1e-3 * np.abs(below[:200]).max()
+    assert np.abs(above[-200:]).max() > 1e3 * np.abs(above[:200]).max()
+
+
+def test_lemma1_threshold_values():
+    # (2/lambda) sin(pi/(4 tau+2)) at lambda=1: the alpha = 0.2 of Figure 2(a) is above it for tau=10 only
+    vals = {t: 2.0 * math.sin(math.pi / (4 * t + 2)) for t in (0, 1, 5, 10)}
+    assert vals[0] == pytest.approx(2.0) and vals[1] == pytest.approx(1.0)
+    assert vals[5] > 0.2 > vals[10]
+
+
+@pytest.mark.parametrize("tau,alpha", [(10, 0.2), (5, 0.2), (10, 0.1), (3, 0.3)])
+def test_growth_rate_is_largest_root_of_char_poly(tau, alpha):
+    # p(w) = w^(tau+1) - w^tau + alpha*lambda   (Section 3.1)
+    lam = 1.0
+    coeffs = np.zeros(tau + 2)
+    coeffs[0], coeffs[1], coeffs[-1] = 1.0, -1.0, alpha * lam
+    radius = np.abs(np.roots(coeffs)).max()
+    traj = scalar_run(tau, tau, quadratic_grad(lam), 1200, hp_(alpha=alpha))
+    assert growth_rate(traj, 400, 1200) == pytest.approx(radius, rel=2e-3)
+
+
+def test_figure2a_setting_diverges_for_tau_10_not_for_tau_0():
+    rng = np.random.default_rng(5)
+    eta = rng.normal(size=600)
+    big = scalar_run(10, 10, quadratic_grad(1.0, noise=lambda t: eta[t]), 600, hp_(alpha=0.2), w0=0.0)
+    small = scalar_run(0, 0, quadratic_grad(1.0, noise=lambda t: eta[t]), 600, hp_(alpha=0.2), w0=0.0)
+    assert np.abs(big[-50:]).max() > 1e3
+    assert np.abs(small).max() < 5.0
+
+
+# ---- momentum (Appendix B.3): iterate = sum_j c_j w_j^t over the roots of the momentum polynomial ----
+
+@pytest.mark.parametrize("tau,alpha,beta", [(3, 0.02, 0.9), (7, 0.01, 0.9), (2, 0.1, 0.5)])
+def test_momentum_iterates_match_mode_sum(tau, alpha, beta):
+    lam, w0, n = 1.0, 1.0, 200
+    traj = scalar_run(tau, tau, quadratic_grad(lam), n, hp_(alpha=alpha, beta1=beta))
+    # p(w) = w^(tau+1) - (1+beta) w^tau + beta w^(tau-1) + alpha*lambda
+    coeffs = np.zeros(tau + 2)
+    coeffs[0], coeffs[1], coeffs[2], coeffs[-1] = 1.0, -(1 + beta), beta, coeffs[-1] + alpha * lam
+    if tau == 1:
+        coeffs = np.array([1.0, -(1 + beta), beta + alpha * lam])
+    roots = np.roots(coeffs).astype(complex)
+    # history: w_s = w0 for s = -tau..0 (zero initial velocity, clamped versions)
+    ts = np.arange(-tau, 1)
+    V = roots[None, :] ** ts[:, None]
+    c = np.linalg.solve(V, np.full(tau + 1, w0, dtype=complex))
+    pred = np.array([(c * roots ** t).sum().real for t in range(n + 1)])
+    np.testing.assert_allclose(traj, pred, atol=1e-9)
+    assert traj[1] == pytest.approx(w0 - alpha * lam * w0)
+
+
+def test_momentum_lemma3_bound_has_unstable_alpha():
+    # Lemma 3: some alpha <= (4/lambda) sin(pi/(4 tau+2)) is unstable: check the bound itself grows
+    tau, beta, lam = 6, 0.9, 1.0
+    a = (4.0 / lam) * math.sin(math.pi / (4 * tau + 2))
+    traj = scalar_run(tau, tau, quadratic_grad(lam), 800, hp_(alpha=a, beta1=beta))
+    assert np.abs(traj[-50:]).max() > 10 * np.abs(traj[:50]).max()
+
+
+# ---- delay discrepancy (Section 3.2) -------------------------------------------------------------
+
+def test_discrepancy_growth_rate_matches_its_char_poly():
+    # w_{t+1} = w_t - a(l+D) w_{t-tf} + a D w_{t-tb}:  w^(tf+1) - w^tf - a D w^(tf-tb) + a(l+D)
+    tf, tb, lam, Dl = 10, 6, 1.0, 5.0
+    for alpha in (0.05, 0.10):
+        coeffs = np.zeros(tf + 2)
+        coeffs[0], coeffs[1] = 1.0, -1.0
+        coeffs[(tf + 1) - (tf - tb)] += -alpha * Dl
+        coeffs[-1] += alpha * (lam + Dl)
+        radius = np.abs(np.roots(coeffs)).max()
+        assert radius > 1.0                                        # Figure 3(a): discrepancy diverges here
+        no_disc = np.zeros(tf + 2)
+        no_disc[0], no_disc[1], no_disc[-1] = 1.0, -1.0, alpha * lam
+        assert np.abs(np.roots(no_disc)).max() < 1.0               # ... where Delta = 0 converges
+        traj = scalar_run(tf, tb, quadratic_grad(lam, Dl), 900, hp_(alpha=alpha))
+        assert growth_rate(traj, 300, 900) == pytest.approx(radius, rel=2e-3)
+
+
+def t2_char_poly(tf, tb, alpha, lam, Dl, gamma):
+    """The T2 polynomial of the appendix, built term by term with numpy's polynomial algebra."""
+    P = np.polynomial.polynomial
+    w = np.array([0.0, 1.0])
+    wm1, wmg = np.array([-1.0, 1.0]), np.array([-gamma, 1.0])
+    wpow = lambda n: np.concatenate([np.zeros(n), [1.0]])
+    p = P.polymul(P.polymul(wm1, wmg), wpow(tf))
+    p = P.polyadd(p, alpha * (lam + Dl) * wmg)
+    p = P.polysub(p, alpha * Dl * P.polymul(wpow(tf - tb), wmg))
+    p = P.polyadd(p, alpha * Dl * (tf - tb) * (1 - gamma) * P.polymul(wpow(tf - tb), wm1))
+    return p  # ascending powers
+
+
+def test_t2_char_poly_construction_matches_printed_values_at_one():
+    P = np.polynomial.polynomial
+    tf, tb, alpha, lam, Dl, D = 10, 0, 0.05, 1.0, 5.0, 0.1
+    gamma = D ** (1.0 / (tf - tb))
+    p = t2_char_poly(tf, tb, alpha, lam, Dl, gamma)
+    assert P.polyval(1.0, p) == pytest.approx(alpha * lam * (1 - gamma), rel=1e-10)
+    assert P.polyval(1.0, P.polyder(p)) == pytest.approx(alpha * lam + 1 - gamma, rel=1e-10)
+
+
+@pytest.mark.parametrize("alpha", [0.05, 0.10])
+def test_t2_growth_rate_matches_t2_char_poly_for_pipemare_delays(alpha):
+    tf, tb, lam, Dl, D = 10, 0, 1.0, 5.0, 0.1
+    gamma = D ** (1.0 / (tf - tb))
+    radius = np.abs(np.roots(t2_char_poly(tf, tb, alpha, lam, Dl, gamma)[::-1])).max()
+    traj = scalar_run(tf, tb, quadratic_grad(lam, Dl), 900, hp_(alpha=alpha, t2=True, D=D))
+    assert growth_rate(traj, 300, 900) == pytest.approx(radius, rel=2e-3)
+    # T2 helps: without it the same setting grows faster
+    traj_off = scalar_run(tf, tb, quadratic_grad(lam, Dl), 900, hp_(alpha=alpha, t2=False))
+    assert growth_rate(traj_off, 300, 900) > growth_rate(traj, 300, 900)
+
+
+# ---- two-weight back-propagation on the scalar chain f = (w2 w1 x - y)^2 --------------------------
+
+def test_two_argument_gradient_on_scalar_chain():
+    x, y = 0.7, -0.3
+    grad_fn = make_grad_fn([["none"], ["none"]], lambda t: (np.array([[x]]), np.array([[y]])), "f32")
+    z = np.zeros(1)
+    uf = [[np.array([[1.5]]), z], [np.array([[-0.8]]), z]]
+    ub = [[np.array([[9.0]]), z], [np.array([[0.25]]), z]]
+    loss, g = grad_fn(0, uf, ub)
+    r = (-0.8) * 1.5 * x - y
+    assert loss == pytest.approx(r * r, rel=1e-14)
+    assert g[1][0][0, 0] == pytest.approx(2 * r * 1.5 * x, rel=1e-14)        # uses only forward values
+    assert g[0][0][0, 0] == pytest.approx(2 * r * 0.25 * x, rel=1e-14)       # backward value of w2
+    # stage 1's backward weights are never read; the last stage's gradient ignores every u_bkwd
+    ub2 = [[np.array([[-123.0]]), z], [np.array([[0.25]]), z]]
+    _, g2 = grad_fn(0, uf, ub2)
+    assert g2[0][0][0, 0] == g[0][0][0, 0] and g2[1][0][0, 0] == g[1][0][0, 0]
