@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the PipeMare hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one pipeline tick of the 32-stage bf16 MLP workload (32 stages x 2 Linear(1024,1024)+GELU,
+microbatch 128) in steady state: every stage runs one forward, one backward against the
+discrepancy-corrected weights, and the fused PipeMare update.  One microbatch (128 samples) leaves
+the pipeline per tick, so samples/s = 128 * K / time.  The second half of the metric, the fused
+update's GB/s against the HBM peak, is measured live inside the same steps (`roofline`) and, on its
+own, over a parameter-count sweep (`update_sweep`).
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the same
+pipeline on its own GPU: the path is not sharded in this build, no collective is on the data path,
+`value` is the sum over ranks divided by the slowest rank's time.
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "async-pipeline train samples/s on 1 B200; PipeMare update GB/s vs HBM peak"
+UNIT = "samples/s"
+BYTES_PER_PARAM = {"sgdm": 30, "adam": 38}     # fp32 g,w,m,delta read + w,m,delta write + bf16 copy (+ s r/w)
+# DRAM traffic of one fused-update launch on the benchmark workload, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
+UPDATE_TRAFFIC_BYTES = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if not dist.is_initialized():
+            dist.init_process_group(backend=backend)
+    return world, rank, local
+
+
+def reduce_over_ranks(elapsed_ms, units, world, device=None):
+    """Slowest rank's time and the total number of units processed by all ranks."""
+    if world == 1:
+        return elapsed_ms, units
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ---- the CUDA arm ---------------------------------------------------------------------------------
+
+def make_batches(wl, n, device):
+    import torch
+    import pm_inputs as I
+    teacher = I.teacher_params(wl)
+    xs, ys = [], []
+    for t in range(n):
+        x, y = I.batch(wl, t, teacher)
+        xs.append(torch.from_numpy(x))
+        ys.append(torch.from_numpy(y))
+    in_dtype = torch.bfloat16 if wl.compute == "bf16" else torch.float32
+    host = [(x.to(in_dtype).pin_memory(), y.pin_memory()) for x, y in zip(xs, ys)]
+    dev = [(x.to(device), y.to(device)) for x, y in host]
+    return host, dev
+
+
+def cpu_baseline(wl, n_steps):
+    """The oracle, as it stands, on this machine's host cores."""
+    import pm_inputs as I
+    from oracle.mlp import run_workload
+    params0 = I.init_stage_params(wl)
+    teacher = I.teacher_params(wl)
+    batches = [I.batch(wl, t, teacher) for t in range(n_steps)]
+    t0 = time.perf_counter()
+    run_workload(wl, params0, lambda t: batches[t], n_steps=n_steps)
+    dt = time.perf_counter() - t0
+    return {"value": wl.microbatch * n_steps / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{n_steps} microbatch steps of the {wl.name} workload (forward, backward, update of all "
+                      f"{wl.n_stages} stages), {dt:.1f} s"}
+
+
+def update_sweep(device, peak_gbs, quick=False):
+    """Stand-alone fused update over a parameter-count sweep; cold L2 by rotating arena sets."""
+    import torch
+    import paper_1910_05124_b200 as pm
+    import pm_inputs as I
+    out = []
+    sizes = [1_000_000, 10_000_000, 100_000_000] + ([] if quick else [1_000_000_000])
+    for opt in ("sgdm", "adam"):
+        for n in sizes:
+            for P in (8, 64, 512):
+                base, rem = divmod(n, P)
+                counts = [base + (1 if i < rem else 0) for i in range(P)]
+                offsets, cur = [], 0
+                for c in counts:
+                    offsets.append(cur)
+                    cur += -(-c // 64) * 64
+                total = cur
+                tau_f, tau_b = I.pipemare_delays(P)
+                bpp = BYTES_PER_PARAM[opt]
+                sets = max(1, min(16, -(-400_000_000 // (bpp * n))))      # > 2x L2 touched between reuses
+                arenas = []
+                g = torch.Generator(device=device)
+                g.manual_seed(1910 + P)
+                for _ in range(sets):
+                    w = torch.randn(total, device=device, generator=g)
+                    gr = torch.randn(total, device=device, generator=g) * 1e-3
+                    m = torch.randn(total, device=device, generator=g) * 1e-3
+                    dl = torch.randn(total, device=device, generator=g) * 1e-4
+                    s = (torch.randn(total, device=device, generator=g) * 1e-3) ** 2 if opt == "adam" else None
+                    lp = torch.empty(total, dtype=torch.bfloat16, device=device)
+                    arenas.append((w, m, s, dl, gr, lp))
+                fu = pm.FlatUpdate(offsets, counts, tau_f, tau_b, optimizer=opt, alpha=0.01 if opt == "sgdm" else 5e-4,
+                                   K=64, D=0.5, device=device)
+                iters = 20
+                for i in range(3):
+                    fu.pm_update_flat(*arenas[i % sets], 32)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(iters):
+                    fu.pm_update_flat(*arenas[i % sets], 32)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / iters
+                gbs = bpp * n / (ms * 1e-3) / 1e9
+                out.append({"n_params": n, "P": P, "optimizer": opt, "ms": round(ms, 5), "GB/s": round(gbs, 1),
+                            "frac_of_measured_peak": round(gbs / peak_gbs, 4), "arena_sets": sets})
+                del arenas, fu
+                torch.cuda.empty_cache()
+    return out
+
+
+def run_cuda(args):
+    import torch
+    import pm_inputs as I
+    import paper_1910_05124_b200 as pm
+    world, rank, local = dist_setup(args.gpus)
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    wl = I.cfg3()
+    P = wl.n_stages
+    params0 = I.init_stage_params(wl)
+    pipe = pm.Pipeline(wl, params0, device=str(device))
+    host_b, dev_b = make_batches(wl, 4, device)
+    n_params = sum(sp.n_in * sp.n_out + sp.n_out for st in wl.stages for sp in st)
+
+    # fill the pipeline (2P-1 ticks) and warm up
+    fill = 2 * P - 1
+    for s in range(fill + max(args.warmup, 3)):
+        pipe.pm_step(*dev_b[s % len(dev_b)])
+    torch.cuda.synchronize(device)
+
+    # ---- timed region 1: K steps, inputs resident in HBM --------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = pipe.pm_launch_count()
+    barrier(world)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(args.steps):
+        pipe.pm_step(*dev_b[s % len(dev_b)])
+    e1.record()
+    torch.cuda.synchronize(device)
+    barrier(world)
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = pipe.pm_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    t_ms, units = reduce_over_ranks(elapsed_ms, wl.microbatch * args.steps, world, device)
+    value = units / (t_ms * 1e-3)
+
+    # ---- timed region 2: the update kernel alone inside the step (CUDA events on the launch stream) --
+    upd_ms = []
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for s in range(args.steps):
+        x, y = dev_b[s % len(dev_b)]
+        pipe.pm_forward(x, y)
+        pipe.pm_backward()
+        ev[s][0].record()
+        pipe.pm_update()
+        ev[s][1].record()
+    torch.cuda.synchronize(device)
+    upd_ms = [a.elapsed_time(b) for a, b in ev]
+    upd_avg = sum(upd_ms) / len(upd_ms)
+    alg_bytes = BYTES_PER_PARAM[wl.optimizer] * n_params
+    achieved = alg_bytes / (upd_avg * 1e-3) / 1e9
+
+    # ---- timed region 3: end to end through the C ABI with host buffers -----------------------------
+    xin = torch.empty_like(dev_b[0][0])
+    yin = torch.empty_like(dev_b[0][1])
+    barrier(world)
+    torch.cuda.synchronize(device)
+    loss_sink = 0.0
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        hx, hy = host_b[s % len(host_b)]
+        xin.copy_(hx, non_blocking=True)
+        yin.copy_(hy, non_blocking=True)
+        pipe.pm_step(xin, yin)
+        # loss of the microbatch whose backward started this tick: device -> host, synchronises
+        mb_done = fill + max(args.warmup, 3) + 2 * args.steps + s - P
+        loss_sink += float(pipe.pm_get_losses(mb_done, 1)[0])
+    torch.cuda.synchronize(device)
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    barrier(world)
+    e2e_t, e2e_units = reduce_over_ranks(e2e_ms, wl.microbatch * args.steps, world, device)
+    h2d = host_b[0][0].numel() * host_b[0][0].element_size() + host_b[0][1].numel() * 4
+
+    if rank != 0:
+        return
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(t_ms / args.steps, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master "
+                               "weights, microbatch 128, SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
+                   "parallelism": "replicas only" if world > 1 else "single GPU, 32 emulated pipeline stages",
+                   "pipeline_fill_ticks": fill, "cache": "per-step working set ~3 GB > 126 MB L2 (no flush needed)",
+                   "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "params": n_params},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_units / (e2e_t * 1e-3), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": 4, "ms_per_step": round(e2e_t / args.steps, 5), "last_loss": loss_sink / args.steps},
+        "gpu_launches": launches,
+        "roofline": {"kernel": "update_kernel (fused PipeMare update)", "bound": "hbm", "achieved": round(achieved, 1),
+                     "peak": hbm_peak, "unit": "GB/s", "frac": round(achieved / hbm_peak, 4), "of": peak_kind,
+                     "traffic": UPDATE_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": alg_bytes,
+                     "avg_launch_ms": round(upd_avg, 5), "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
+                     "share_of_step": round(upd_avg / (t_ms / args.steps), 4)},
+    }
+    if world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, 2)
+        if not args.no_sweep:
+            line["update_sweep"] = update_sweep(device, hbm_peak)
+    print(json.dumps(line), flush=True)
+
+
+# ---- the reference arm: the CPU oracle -------------------------------------------------------------
+
+def run_reference(args):
+    """Times the oracle on the host cores.  Each step is one microbatch through a contiguous sample of
+    the workload's stages (as many as keep the whole run within a few minutes); throughput is scaled by
+    the fraction of stages sampled, since every stage costs the same."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import pm_inputs as I
+    from oracle.mlp import run_workload
+    full = I.cfg3()
+    budget_s = 150.0
+    total_steps = args.steps + args.warmup
+
+    def sub_workload(n_stages):
+        wl = I.mlp_workload(full.name, n_stages, 1024, 2, "gelu", full.microbatch, compute="bf16",
+                            optimizer=full.optimizer, alpha=full.alpha, beta1=full.beta1, K=full.K, D=full.D,
+                            steps=total_steps, seed=full.seed)
+        return wl
+
+    # pilot: one step of one stage
+    wl1 = sub_workload(1)
+    p1, t1 = I.init_stage_params(wl1), I.teacher_params(wl1)
+    b1 = I.batch(wl1, 0, t1)
+    t0 = time.perf_counter()
+    run_workload(wl1, p1, lambda t: b1, n_steps=2)
+    per_stage_step = (time.perf_counter() - t0) / 2
+    n_stages = int(max(1, min(full.n_stages, budget_s / (total_steps * per_stage_step))))
+    wl = sub_workload(n_stages)
+    params0, teacher = I.init_stage_params(wl), I.teacher_params(wl)
+    batches = [I.batch(wl, t, teacher) for t in range(min(total_steps, 4))]
+    marks = {}
+
+    def on_step(t, w):
+        if t == args.warmup - 1:
+            marks["t0"] = time.perf_counter()
+
+    if args.warmup == 0:
+        marks["t0"] = time.perf_counter()
+    run_workload(wl, params0, lambda t: batches[t % len(batches)], n_steps=total_steps, on_step=on_step)
+    dt = time.perf_counter() - marks["t0"]
+    scale = n_stages / full.n_stages
+    value = full.microbatch * args.steps / dt * scale
+    sample = (f"each step: one microbatch of 128 through {n_stages} of the {full.n_stages} stages "
+              f"(forward, backward, update); samples/s scaled by {n_stages}/{full.n_stages}")
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3 / scale, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, microbatch 128 "
+                                   "(CPU oracle, bf16-rounded operands, float64 accumulation)"},
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the stand-alone update sweep")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

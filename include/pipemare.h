@@ -1,0 +1,201 @@
+/*
+ * pipemare.h -- C ABI of the B200 (sm_100a) PipeMare hot path.
+ *
+ * One GPU emulates a P-stage asynchronous pipeline.  Each call of pm_step is one
+ * pipeline tick: every stage runs one forward with the weights it holds now, one
+ * backward for the microbatch that entered it tau_fwd updates ago (against the
+ * discrepancy-corrected weights of T2), and one weight update with the
+ * rescheduled step size of T1.  All arithmetic runs in CUDA kernels; this
+ * interface only carries pointers and sizes.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory owned by the caller.  The library
+ *     never allocates or frees device memory; it borrows the pointers for the
+ *     lifetime of the context.  "host" pointers are ordinary host memory, read
+ *     during the call unless stated otherwise.
+ *   - Work is enqueued on the CUDA stream given at initialisation and returns
+ *     before it completes, except pm_get_losses and pm_get_bookkeeping, which
+ *     synchronise that stream.
+ *   - Every function returns a pm_status; nothing throws or aborts.  After an
+ *     error pm_last_error(ctx) gives a readable message.
+ *   - Stages are numbered 1..P in the paper and 0..P-1 in array arguments here.
+ *   - One microbatch per update (N = 1 in the notation of Section 2.1).
+ */
+#ifndef PIPEMARE_H
+#define PIPEMARE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pm_ctx pm_ctx;
+
+typedef enum {
+  PM_OK = 0,
+  PM_ERR_INVALID_ARG = 1,   /* null pointer, negative size, unknown enum value            */
+  PM_ERR_SHAPE = 2,         /* dimensions the kernels cannot take (see pm_init_stages)    */
+  PM_ERR_STATE = 3,         /* phase calls out of order                                   */
+  PM_ERR_NOMEM = 4,         /* ring or workspace too small; message states the need       */
+  PM_ERR_UNSUPPORTED = 5,   /* valid request that is not built                            */
+  PM_ERR_CUDA = 6,          /* a CUDA runtime call failed; message carries its text       */
+  PM_ERR_TIMEOUT = 7        /* a bounded device-side wait expired                         */
+} pm_status;
+
+enum { PM_F32 = 0, PM_BF16 = 1 };                 /* GEMM operand type; state is always fp32 */
+enum { PM_SGDM = 0, PM_ADAM = 1 };
+enum { PM_ACT_NONE = 0, PM_ACT_RELU = 1, PM_ACT_GELU = 2 };   /* GELU = exact erf form      */
+enum { PM_OP_LINEAR = 0 };
+enum { PM_LOSS_MSE = 0 };
+
+/* Alignment, in elements, of every stage slice and of every tensor inside it. */
+#define PM_ALIGN_ELEMS 64
+#define PM_MAX_LINEARS 4       /* Linear ops per stage                                    */
+#define PM_MAX_STAGES 1024
+
+/* One operator of a stage.  LINEAR: y = act(x W^T + b), W is [n_out, n_in] row-major. */
+typedef struct {
+  int32_t kind;            /* PM_OP_LINEAR */
+  int32_t n_in, n_out;
+  int32_t act;             /* PM_ACT_* */
+} pm_op_desc;
+
+/* One pipeline stage (Section 2.1).  Copied during pm_init_stages.
+ * tau_fwd / tau_bkwd: number of updates between the forward / backward read of this
+ * stage's weights and the update that uses the resulting gradient.  PipeMare
+ * (Table 1) has tau_fwd = 2(P-i)+1 and tau_bkwd = 0, which is the only delay
+ * pattern the tick schedule realises; other values are PM_ERR_UNSUPPORTED.
+ * param_offset / param_count: this stage's slice of the flat arenas, in elements;
+ * both multiples of PM_ALIGN_ELEMS.  Inside the slice each op's W and then b start
+ * at the next multiple of PM_ALIGN_ELEMS (pm_op_param_offsets gives the numbers). */
+typedef struct {
+  int32_t tau_fwd, tau_bkwd;
+  int32_t n_ops;
+  const pm_op_desc* ops;   /* host */
+  uint64_t param_offset, param_count;
+} pm_stage_desc;
+
+/* Hyper-parameters.
+ * T1 (Section 3.1, Eq. 2): step size of stage i at its update k is
+ *   alpha_base(k) / tau_fwd,i ^ p_k,  p_k = 1 - min(k / t1_K, 1).
+ * T2 (Section 3.2): backward reads w - (tau_fwd - tau_bkwd) * delta, and
+ *   delta <- gamma delta + (1 - gamma)(w_new - w_old), gamma = t2_D ^ (1/(tau_fwd - tau_bkwd)).
+ * Optimiser: momentum SGD in the form of Appendix B.3 (v <- beta1 v - alpha g; w <- w + v)
+ * or bias-corrected Adam without weight decay.
+ * alpha_base(k) = alpha_by_step[min(k, alpha_len-1)] if alpha_by_step != NULL (host array,
+ * copied at initialisation), else alpha_const. */
+typedef struct {
+  int32_t n_stages;        /* P */
+  int32_t microbatch;      /* rows T of every activation matrix */
+  int32_t compute_dtype;   /* PM_F32 | PM_BF16 */
+  int32_t optimizer;       /* PM_SGDM | PM_ADAM */
+  int32_t loss;            /* PM_LOSS_MSE: mean over all T*out entries of (y - target)^2 */
+  float beta1, beta2, eps;
+  int32_t t1_enable;
+  int64_t t1_K;
+  int32_t t2_enable;
+  double t2_D;
+  double alpha_const;
+  const double* alpha_by_step;   /* host, may be NULL */
+  int64_t alpha_len;
+  int64_t loss_log_capacity;     /* losses kept on the device (a ring); 0 = default 4096 */
+} pm_config;
+
+/* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /
+ * Adam first moment; s: Adam second moment (may be NULL for SGD); delta: T2
+ * accumulator; grad: gradient of the current tick (written by the backward phase);
+ * w_lp: bfloat16 copy of w kept by the update kernel (may be NULL when
+ * compute_dtype is PM_F32).  All 256-byte aligned. */
+typedef struct {
+  float* w;
+  float* m;
+  float* s;
+  float* delta;
+  float* grad;
+  uint16_t* w_lp;
+  uint64_t count;
+} pm_arenas;
+
+/* ---- parameter layout (host arithmetic only) ------------------------------------------ */
+
+/* Number of elements a stage with these ops occupies in the arenas (padded). */
+pm_status pm_stage_param_count(const pm_op_desc* ops, int32_t n_ops, uint64_t* count);
+/* Offsets of op `op`'s weight matrix and bias vector relative to the stage's param_offset. */
+pm_status pm_op_param_offsets(const pm_op_desc* ops, int32_t n_ops, int32_t op,
+                              uint64_t* w_off, uint64_t* b_off);
+
+/* ---- pipeline context ------------------------------------------------------------------ */
+
+/* Bytes the caller must provide: state_bytes = all arenas together (fp32 w, m, [s,] delta,
+ * grad [+ bf16 copy]); ring_bytes = the per-stage delay rings of in-flight activations
+ * (Section 2 / Appendix A: depth grows with 2(P-i)+1); workspace_bytes = gradient
+ * mailboxes, per-stage scratch, target ring, loss log and tables. */
+pm_status pm_query_bytes(const pm_config* cfg, const pm_stage_desc* stages,
+                         uint64_t* state_bytes, uint64_t* ring_bytes, uint64_t* workspace_bytes);
+
+/* Build a context.  The arenas must already hold the initial weights (w, and w_lp = bf16(w)
+ * for PM_BF16), zero m/s/delta.  ring and workspace are device buffers of at least the
+ * queried sizes, 256-byte aligned; the library zero-fills neither (contents are written
+ * before they are read).  `stream` is a cudaStream_t passed as void*.
+ * PM_ERR_SHAPE: stage i's first n_in differs from stage i-1's last n_out; for PM_BF16 a
+ * dimension that is not a multiple of 8. */
+pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc* stages,
+                         const pm_arenas* arenas, void* ring, uint64_t ring_bytes,
+                         void* workspace, uint64_t workspace_bytes, void* stream);
+
+/* One tick = pm_forward, pm_backward, pm_update in this order (pm_step does all three).
+ * inputs/targets (device) belong to the microbatch that enters the pipeline at this tick:
+ * inputs is [T, n_in of stage 1] (float for PM_F32, bfloat16 for PM_BF16), targets is
+ * [T, n_out of stage P] float.  Both are copied before the call returns control to the
+ * stream order, so the caller may overwrite them after any later call on the same stream.
+ * Pass NULL for both to drain: N microbatches need N + 2P - 1 ticks.
+ *
+ * Tick s (0-based): stage i (1-based) runs the forward of microbatch s-(i-1) and the
+ * backward and update of microbatch s-(2P-i).  Hence its forward for microbatch a reads
+ * weight version max(0, a - tau_fwd,i) and its backward reads version a (Section 2.1 with
+ * PipeMare's delays). */
+pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets);
+pm_status pm_backward(pm_ctx* ctx);
+pm_status pm_update(pm_ctx* ctx);
+pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets);
+
+/* Per-stage record of the last completed tick, written by the device kernels, for the
+ * delay-bookkeeping check.  out[0..7] = forward microbatch (-1 if idle), weight version
+ * the forward read, backward microbatch (-1 if idle), weight version the backward read,
+ * updates applied so far, forward ring slot, backward ring slot, tick.  Synchronises. */
+pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8);
+
+/* Copy losses of microbatches first_mb .. first_mb+n-1 to host_out.  The loss of microbatch
+ * t is the one computed from its (stale) forward weights.  Synchronises.  PM_ERR_INVALID_ARG
+ * if a requested microbatch has not finished or has left the device log. */
+pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t n);
+
+/* Number of CUDA kernels this context has enqueued since pm_init_stages (for launch accounting). */
+uint64_t pm_launch_count(pm_ctx* ctx);
+
+const char* pm_last_error(pm_ctx* ctx);   /* never NULL; ctx may be NULL (global message) */
+void pm_destroy(pm_ctx* ctx);
+
+/* ---- the fused update on its own ---------------------------------------------------------- */
+
+/* One fused PipeMare update (T1 step size, momentum or Adam, T2 accumulator refresh,
+ * bf16 copy) over the flat arenas of n_stages stages, every stage at update index k.
+ * stage_offsets / stage_counts (host, elements, offsets multiples of PM_ALIGN_ELEMS)
+ * delimit the slices; elements between a slice's end and the next offset are padding
+ * and must hold zeros.  tau_fwd / tau_bkwd: host arrays.  From cfg the optimiser,
+ * betas, eps, T1/T2 settings and alpha are read.  `workspace` is a device buffer of at
+ * least pm_update_flat_workspace_bytes(n_stages) bytes that receives the stage table.
+ * Asynchronous on `stream`. */
+uint64_t pm_update_flat_workspace_bytes(int32_t n_stages);
+pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
+                         const uint64_t* stage_counts, const int32_t* tau_fwd,
+                         const int32_t* tau_bkwd, int32_t n_stages, const pm_config* cfg,
+                         int64_t k, void* workspace, uint64_t workspace_bytes, void* stream);
+
+const char* pm_status_string(pm_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIPEMARE_H */

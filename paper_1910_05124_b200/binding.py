@@ -1,0 +1,285 @@
+"""ctypes binding of libpipemare.so: the same entry points as include/pipemare.h, argument marshalling only.
+
+`Pipeline` and `FlatUpdate` are conveniences that allocate the caller-owned device
+buffers as torch tensors, pack parameters into the flat arenas with the layout the
+library reports, and pass raw pointers through.  No arithmetic of the method happens
+here.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+PM_F32, PM_BF16 = 0, 1
+PM_SGDM, PM_ADAM = 0, 1
+PM_ACT_NONE, PM_ACT_RELU, PM_ACT_GELU = 0, 1, 2
+PM_OP_LINEAR = 0
+PM_LOSS_MSE = 0
+PM_ALIGN_ELEMS = 64
+
+_ACT = {"none": PM_ACT_NONE, "relu": PM_ACT_RELU, "gelu": PM_ACT_GELU}
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpipemare.so")
+
+
+class pm_op_desc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("n_in", C.c_int32), ("n_out", C.c_int32), ("act", C.c_int32)]
+
+
+class pm_stage_desc(C.Structure):
+    _fields_ = [("tau_fwd", C.c_int32), ("tau_bkwd", C.c_int32), ("n_ops", C.c_int32),
+                ("ops", C.POINTER(pm_op_desc)), ("param_offset", C.c_uint64), ("param_count", C.c_uint64)]
+
+
+class pm_config(C.Structure):
+    _fields_ = [("n_stages", C.c_int32), ("microbatch", C.c_int32), ("compute_dtype", C.c_int32),
+                ("optimizer", C.c_int32), ("loss", C.c_int32),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("t1_enable", C.c_int32), ("t1_K", C.c_int64), ("t2_enable", C.c_int32), ("t2_D", C.c_double),
+                ("alpha_const", C.c_double), ("alpha_by_step", C.POINTER(C.c_double)), ("alpha_len", C.c_int64),
+                ("loss_log_capacity", C.c_int64)]
+
+
+class pm_arenas(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("m", C.c_void_p), ("s", C.c_void_p), ("delta", C.c_void_p),
+                ("grad", C.c_void_p), ("w_lp", C.c_void_p), ("count", C.c_uint64)]
+
+
+class PipeMareError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"{status}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Load libpipemare.so (once).  Raises if it has not been built: there is no fallback path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise PipeMareError("PM_ERR_NOLIB", f"{LIB_PATH} is missing; run paper_1910_05124_b200/build.py "
+                                            "(or __graft_entry__.build()) first")
+    L = C.CDLL(LIB_PATH)
+    vp, u64p = C.c_void_p, C.POINTER(C.c_uint64)
+    L.pm_status_string.restype = C.c_char_p
+    L.pm_status_string.argtypes = [C.c_int]
+    L.pm_last_error.restype = C.c_char_p
+    L.pm_last_error.argtypes = [vp]
+    L.pm_stage_param_count.argtypes = [C.POINTER(pm_op_desc), C.c_int32, u64p]
+    L.pm_op_param_offsets.argtypes = [C.POINTER(pm_op_desc), C.c_int32, C.c_int32, u64p, u64p]
+    L.pm_query_bytes.argtypes = [C.POINTER(pm_config), C.POINTER(pm_stage_desc), u64p, u64p, u64p]
+    L.pm_init_stages.argtypes = [C.POINTER(vp), C.POINTER(pm_config), C.POINTER(pm_stage_desc), C.POINTER(pm_arenas),
+                                 vp, C.c_uint64, vp, C.c_uint64, vp]
+    L.pm_forward.argtypes = [vp, vp, vp]
+    L.pm_backward.argtypes = [vp]
+    L.pm_update.argtypes = [vp]
+    L.pm_step.argtypes = [vp, vp, vp]
+    L.pm_get_bookkeeping.argtypes = [vp, C.c_int32, C.POINTER(C.c_int64)]
+    L.pm_get_losses.argtypes = [vp, C.POINTER(C.c_float), C.c_int64, C.c_int64]
+    L.pm_launch_count.argtypes = [vp]
+    L.pm_launch_count.restype = C.c_uint64
+    L.pm_destroy.argtypes = [vp]
+    L.pm_destroy.restype = None
+    L.pm_update_flat_workspace_bytes.argtypes = [C.c_int32]
+    L.pm_update_flat_workspace_bytes.restype = C.c_uint64
+    L.pm_update_flat.argtypes = [C.POINTER(pm_arenas), u64p, u64p, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                 C.c_int32, C.POINTER(pm_config), C.c_int64, vp, C.c_uint64, vp]
+    _lib = L
+    return L
+
+
+def _check(status, ctx=None):
+    if status != 0:
+        L = lib()
+        raise PipeMareError(L.pm_status_string(status).decode(), L.pm_last_error(ctx).decode())
+
+
+def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, beta2=0.98, eps=1e-8,
+                t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0):
+    cfg = pm_config()
+    cfg.n_stages, cfg.microbatch = n_stages, microbatch
+    cfg.compute_dtype = PM_BF16 if compute in ("bf16", PM_BF16) and compute != 0 else PM_F32
+    cfg.optimizer = PM_ADAM if optimizer in ("adam", PM_ADAM) and optimizer != 0 else PM_SGDM
+    cfg.loss = PM_LOSS_MSE
+    cfg.beta1, cfg.beta2, cfg.eps = beta1, beta2, eps
+    cfg.t1_enable, cfg.t1_K = int(bool(t1)), int(K)
+    cfg.t2_enable, cfg.t2_D = int(bool(t2)), float(D)
+    cfg.alpha_const = float(alpha)
+    keep = None
+    if alpha_by_step is not None:
+        keep = (C.c_double * len(alpha_by_step))(*alpha_by_step)
+        cfg.alpha_by_step = C.cast(keep, C.POINTER(C.c_double))
+        cfg.alpha_len = len(alpha_by_step)
+    cfg.loss_log_capacity = loss_log_capacity
+    return cfg, keep
+
+
+def _ops_array(specs):
+    arr = (pm_op_desc * len(specs))()
+    for j, sp in enumerate(specs):
+        arr[j].kind, arr[j].n_in, arr[j].n_out, arr[j].act = PM_OP_LINEAR, sp.n_in, sp.n_out, _ACT[sp.act]
+    return arr
+
+
+def stage_layout(specs):
+    """(padded element count, [(w_off, b_off) per op]) of a stage, as the library lays it out."""
+    L = lib()
+    arr = _ops_array(specs)
+    cnt = C.c_uint64()
+    _check(L.pm_stage_param_count(arr, len(specs), C.byref(cnt)))
+    offs = []
+    for j in range(len(specs)):
+        wo, bo = C.c_uint64(), C.c_uint64()
+        _check(L.pm_op_param_offsets(arr, len(specs), j, C.byref(wo), C.byref(bo)))
+        offs.append((wo.value, bo.value))
+    return cnt.value, offs
+
+
+class Pipeline:
+    """Owns the device buffers of one pipeline context and forwards calls to the C ABI.
+
+    wl: a workload description with fields stages (lists of objects with n_in, n_out, act),
+    tau_fwd, tau_bkwd, microbatch, compute, optimizer, alpha, beta1, beta2, eps, t1, K, t2, D.
+    params0: per stage a list of (W[out,in], b[out]) float32 numpy arrays.
+    """
+
+    def __init__(self, wl, params0, device="cuda:0", stream=None, loss_log_capacity=0):
+        import torch
+        self.torch = torch
+        self.wl = wl
+        self.L = lib()
+        self.device = torch.device(device)
+        P = len(wl.stages)
+        self._ops = [_ops_array(st) for st in wl.stages]
+        self.layout = [stage_layout(st) for st in wl.stages]
+        self.stage_desc = (pm_stage_desc * P)()
+        off = 0
+        for p in range(P):
+            d = self.stage_desc[p]
+            d.tau_fwd, d.tau_bkwd, d.n_ops = wl.tau_fwd[p], wl.tau_bkwd[p], len(wl.stages[p])
+            d.ops = C.cast(self._ops[p], C.POINTER(pm_op_desc))
+            d.param_offset, d.param_count = off, self.layout[p][0]
+            off += self.layout[p][0]
+        self.total = off
+        self.cfg, self._alpha_keep = make_config(
+            n_stages=P, microbatch=wl.microbatch, compute=wl.compute, optimizer=wl.optimizer, alpha=wl.alpha,
+            beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D,
+            loss_log_capacity=loss_log_capacity)
+        sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+        _check(self.L.pm_query_bytes(C.byref(self.cfg), self.stage_desc, C.byref(sb), C.byref(rb), C.byref(wb)))
+        self.state_bytes, self.ring_bytes, self.workspace_bytes = sb.value, rb.value, wb.value
+        dev = self.device
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.w = torch.zeros(self.total, **f32)
+        self.m = torch.zeros(self.total, **f32)
+        self.delta = torch.zeros(self.total, **f32)
+        self.grad = torch.zeros(self.total, **f32)
+        self.s = torch.zeros(self.total, **f32) if wl.optimizer == "adam" else None
+        flat = np.zeros(self.total, dtype=np.float32)
+        for p in range(P):
+            base = self.stage_desc[p].param_offset
+            for j, (W, b) in enumerate(params0[p]):
+                wo, bo = self.layout[p][1][j]
+                flat[base + wo: base + wo + W.size] = np.asarray(W, dtype=np.float32).ravel()
+                flat[base + bo: base + bo + b.size] = np.asarray(b, dtype=np.float32).ravel()
+        self.w.copy_(torch.from_numpy(flat))
+        self.w_lp = self.w.to(torch.bfloat16) if wl.compute == "bf16" else None
+        self.ring = torch.empty(max(self.ring_bytes, 256), dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=dev)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
+        self.arenas = pm_arenas(self.w.data_ptr(), self.m.data_ptr(), self.s.data_ptr() if self.s is not None else None,
+                                self.delta.data_ptr(), self.grad.data_ptr(),
+                                self.w_lp.data_ptr() if self.w_lp is not None else None, self.total)
+        self.ctx = C.c_void_p()
+        torch.cuda.synchronize(dev)
+        _check(self.L.pm_init_stages(C.byref(self.ctx), C.byref(self.cfg), self.stage_desc, C.byref(self.arenas),
+                                     self.ring.data_ptr(), self.ring.numel(), self.workspace.data_ptr(),
+                                     self.workspace.numel(), C.c_void_p(self.stream.cuda_stream)))
+
+    # -- the C entry points, same names -------------------------------------------------------
+    def _ptr(self, t):
+        return None if t is None else C.c_void_p(t.data_ptr())
+
+    def pm_forward(self, inputs=None, targets=None):
+        _check(self.L.pm_forward(self.ctx, self._ptr(inputs), self._ptr(targets)), self.ctx)
+
+    def pm_backward(self):
+        _check(self.L.pm_backward(self.ctx), self.ctx)
+
+    def pm_update(self):
+        _check(self.L.pm_update(self.ctx), self.ctx)
+
+    def pm_step(self, inputs=None, targets=None):
+        _check(self.L.pm_step(self.ctx, self._ptr(inputs), self._ptr(targets)), self.ctx)
+
+    def pm_get_bookkeeping(self, stage):
+        out = (C.c_int64 * 8)()
+        _check(self.L.pm_get_bookkeeping(self.ctx, stage, out), self.ctx)
+        return list(out)
+
+    def pm_get_losses(self, first_mb, n):
+        out = (C.c_float * n)()
+        _check(self.L.pm_get_losses(self.ctx, out, first_mb, n), self.ctx)
+        return np.array(out[:], dtype=np.float32)
+
+    def pm_launch_count(self):
+        return int(self.L.pm_launch_count(self.ctx))
+
+    # -- marshalling helpers --------------------------------------------------------------------
+    def unpack(self, flat_tensor):
+        """Split a flat arena (device tensor) into per-stage lists of (W, b) numpy arrays."""
+        flat = flat_tensor.detach().float().cpu().numpy()
+        out = []
+        for p, st in enumerate(self.wl.stages):
+            base = self.stage_desc[p].param_offset
+            tensors = []
+            for j, sp in enumerate(st):
+                wo, bo = self.layout[p][1][j]
+                W = flat[base + wo: base + wo + sp.n_in * sp.n_out].reshape(sp.n_out, sp.n_in).copy()
+                b = flat[base + bo: base + bo + sp.n_out].copy()
+                tensors.append((W, b))
+            out.append(tensors)
+        return out
+
+    def close(self):
+        if self.ctx:
+            self.L.pm_destroy(self.ctx)
+            self.ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class FlatUpdate:
+    """Marshals pm_update_flat: holds the host tables and the device workspace for one stage split."""
+
+    def __init__(self, offsets, counts, tau_fwd, tau_bkwd, *, optimizer, alpha, beta1=0.9, beta2=0.98, eps=1e-8,
+                 t1=True, K=1, t2=True, D=0.5, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.L = lib()
+        P = len(offsets)
+        self.P = P
+        self.offsets = (C.c_uint64 * P)(*offsets)
+        self.counts = (C.c_uint64 * P)(*counts)
+        self.tau_fwd = (C.c_int32 * P)(*tau_fwd)
+        self.tau_bkwd = (C.c_int32 * P)(*tau_bkwd)
+        self.cfg, self._keep = make_config(n_stages=P, microbatch=1, compute="f32", optimizer=optimizer, alpha=alpha,
+                                           beta1=beta1, beta2=beta2, eps=eps, t1=t1, K=K, t2=t2, D=D)
+        self.ws_bytes = self.L.pm_update_flat_workspace_bytes(P)
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
+
+    def pm_update_flat(self, w, m, s, delta, grad, w_lp, k, stream=None):
+        torch = self.torch
+        st = stream if stream is not None else torch.cuda.current_stream(w.device)
+        ar = pm_arenas(w.data_ptr(), m.data_ptr(), s.data_ptr() if s is not None else None, delta.data_ptr(),
+                       grad.data_ptr(), w_lp.data_ptr() if w_lp is not None else None, w.numel())
+        _check(self.L.pm_update_flat(C.byref(ar), self.offsets, self.counts, self.tau_fwd, self.tau_bkwd, self.P,
+                                     C.byref(self.cfg), k, self.workspace.data_ptr(), self.ws_bytes,
+                                     C.c_void_p(st.cuda_stream)))

@@ -1,0 +1,275 @@
+// Element-wise tick kernels (ingest, loss, activation backward) and the fp32 SIMT grouped GEMMs.
+//
+// Every kernel is "grouped": blockIdx.z (or .y) selects the stage, the per-tick table says
+// whether that stage is active and which ring slots it touches.  Within a tick the stages
+// only read what earlier ticks left in their rings and mailboxes, so one launch covers all.
+#include "pm_tick.cuh"
+
+namespace pm {
+
+template <typename AT> __device__ __forceinline__ AT* ring_ptr(const TickArgs& t, uint64_t off, int slot, uint64_t slot_elems) {
+  return reinterpret_cast<AT*>(t.ring + off) + (uint64_t)slot * slot_elems;
+}
+template <typename AT> __device__ __forceinline__ AT* ws_ptr(const TickArgs& t, uint64_t off) {
+  return reinterpret_cast<AT*>(t.ws + off);
+}
+
+// ---- ingest -----------------------------------------------------------------------------------
+template <typename AT>
+__global__ void ingest_kernel(TickArgs t, const AT* __restrict__ inputs, const float* __restrict__ targets, int64_t mb) {
+  const StageDev& s0 = t.st[0];
+  const uint64_t n_x = (uint64_t)t.T * t.n_in_first, n_t = (uint64_t)t.T * t.n_out_last;
+  AT* xdst = ring_ptr<AT>(t, s0.x_ring, (int)(mb % s0.xdepth), n_x);
+  float* tdst = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(mb % (t.P + 1)) * n_t;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_x + n_t; i += (uint64_t)gridDim.x * blockDim.x) {
+    if (i < n_x) xdst[i] = inputs[i];
+    else tdst[i - n_x] = targets[i - n_x];
+  }
+}
+
+cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, const float* targets, int64_t mb, cudaStream_t stream) {
+  uint64_t n = (uint64_t)t.T * (t.n_in_first + t.n_out_last);
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 1184) blocks = 1184;
+  if (dtype == PM_F32) ingest_kernel<float><<<blocks, 256, 0, stream>>>(t, (const float*)inputs, targets, mb);
+  else ingest_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(t, (const __nv_bfloat16*)inputs, targets, mb);
+  return cudaGetLastError();
+}
+
+// ---- MSE loss at the last stage ------------------------------------------------------------------
+// loss = mean over T*out of (y - y*)^2 ;  dy = 2 (y - y*) / (T*out), stored in the activation type.
+// One block; fixed summation order (strided per-thread partials, then a fixed tree).
+template <typename AT>
+__global__ void __launch_bounds__(1024) mse_loss_kernel(TickArgs t) {
+  const StageDyn& d = t.dyn[t.P - 1];
+  if (d.b_mb < 0) return;
+  const StageDev& sl = t.st[t.P - 1];
+  const uint64_t n = (uint64_t)t.T * t.n_out_last;
+  const int par = (int)((d.tick + 1) & 1);            // written during the previous tick
+  const AT* y = ws_ptr<AT>(t, t.yout_off) + (uint64_t)par * n;
+  const float* tg = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(d.b_mb % (t.P + 1)) * n;
+  AT* dy = ws_ptr<AT>(t, sl.gin) + (uint64_t)par * n;
+  const float scale = (float)(2.0 / (double)n);
+  float part = 0.f;
+  for (uint64_t i = threadIdx.x; i < n; i += blockDim.x) {
+    float r = __fsub_rn(to_f<AT>(y[i]), tg[i]);
+    part = __fadd_rn(part, __fmul_rn(r, r));
+    dy[i] = from_f<AT>(__fmul_rn(scale, r));
+  }
+  __shared__ float red[1024];
+  red[threadIdx.x] = part;
+  __syncthreads();
+  for (int off = 512; off > 0; off >>= 1) {
+    if ((int)threadIdx.x < off) red[threadIdx.x] = __fadd_rn(red[threadIdx.x], red[threadIdx.x + off]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) ws_ptr<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = red[0] / (float)n;
+}
+
+cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream) {
+  if (dtype == PM_F32) mse_loss_kernel<float><<<1, 1024, 0, stream>>>(t);
+  else mse_loss_kernel<__nv_bfloat16><<<1, 1024, 0, stream>>>(t);
+  return cudaGetLastError();
+}
+
+// ---- activation backward + bias gradient ---------------------------------------------------------
+// dz = dy * act'(z) (stored in the activation type); db[c] = sum over rows of the stored dz, rows ascending.
+template <typename AT>
+__global__ void __launch_bounds__(128) actbwd_kernel(TickArgs t, int lvl) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || lvl >= s.n_lin) return;
+  const LinDev& L = s.lin[lvl];
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= L.n_out) return;
+  const uint64_t n = (uint64_t)t.T * L.n_out;
+  const AT* dy = (lvl == s.n_lin - 1) ? ws_ptr<AT>(t, s.gin) + (uint64_t)((d.tick + 1) & 1) * n : ws_ptr<AT>(t, s.dh);
+  const AT* z = ring_ptr<AT>(t, L.z_ring, d.b_slot, n);
+  AT* dz = ws_ptr<AT>(t, s.dz);
+  float sum = 0.f;
+  for (int r = 0; r < t.T; ++r) {
+    uint64_t i = (uint64_t)r * L.n_out + c;
+    AT v = from_f<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act)));
+    dz[i] = v;
+    sum = __fadd_rn(sum, to_f<AT>(v));
+  }
+  t.a.grad[L.b_off + c] = sum;
+}
+
+cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
+  dim3 grid((t.max_dim + 127) / 128, t.P);
+  if (dtype == PM_F32) actbwd_kernel<float><<<grid, 128, 0, stream>>>(t, lvl);
+  else actbwd_kernel<__nv_bfloat16><<<grid, 128, 0, stream>>>(t, lvl);
+  return cudaGetLastError();
+}
+
+// ---- fp32 SIMT grouped GEMM ------------------------------------------------------------------------
+// C[M,N] = sum_k A(m,k) B(k,n), 64x64 tile per block, 16-deep k steps, 4x4 outputs per thread,
+// k ascending with fused multiply-add in fp32.
+//   mode 0 forward:  A = x [T,in],        B(k,n) = W[n,k]            -> z = C + b, y = act(z)
+//   mode 1 dgrad:    A = dz [T,out],      B(k,n) = W[k,n]-gap*delta  -> dx = C
+//   mode 2 wgrad:    A(m,k) = dz[k,m],    B(k,n) = x[k,n]            -> dW = C
+constexpr int BM = 64, BN = 64, BK = 16;
+
+template <typename AT, typename WT, int MODE>
+__global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
+  const int p = blockIdx.z;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (lvl >= s.n_lin) return;
+  if (MODE == 0 ? d.f_mb < 0 : d.b_mb < 0) return;
+  if (MODE == 1 && p == 0 && lvl == 0) return;        // the network input needs no gradient
+  const LinDev& L = s.lin[lvl];
+  const int T = t.T;
+  int M, N, K;
+  if (MODE == 0) { M = T; N = L.n_out; K = L.n_in; }
+  else if (MODE == 1) { M = T; N = L.n_in; K = L.n_out; }
+  else { M = L.n_out; N = L.n_in; K = T; }
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  if (m0 >= M || n0 >= N) return;
+
+  const uint64_t n_xin = (uint64_t)T * L.n_in, n_xout = (uint64_t)T * L.n_out;
+  // operand sources
+  const AT* xin;      // this Linear's input activation (forward slot or backward slot)
+  {
+    const int slot = MODE == 0 ? d.f_slot : d.b_slot;
+    const int xslot = MODE == 0 ? d.f_xslot : d.b_xslot;
+    xin = (lvl == 0) ? ring_ptr<AT>(t, s.x_ring, xslot, n_xin) : ring_ptr<AT>(t, s.lin[lvl - 1].h_ring, slot, n_xin);
+  }
+  const AT* dz = ws_ptr<AT>(t, s.dz);
+  const WT* wf;
+  if (sizeof(WT) == 4) wf = reinterpret_cast<const WT*>(t.a.w) + L.w_off;
+  else wf = reinterpret_cast<const WT*>(t.a.w_lp) + L.w_off;
+  const float* wm = t.a.w + L.w_off;
+  const float* dl = t.a.delta + L.w_off;
+  const float gapf = (float)s.gap;
+  const bool corr = d.use_delta != 0;
+
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Bs[BK][BN + 1];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    // A tile
+    if (MODE == 2) {            // m contiguous: A(m,k) = dz[k*out + m]
+      int kk = tid >> 4, mm = (tid & 15) * 4;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = m0 + mm + j, k = k0 + kk;
+        As[kk][mm + j] = (m < M && k < K) ? to_f<AT>(dz[(uint64_t)k * L.n_out + m]) : 0.f;
+      }
+    } else {                    // k contiguous
+      int mm = tid >> 2, kk = (tid & 3) * 4;
+      const AT* src = MODE == 0 ? xin : dz;
+      const int ld = MODE == 0 ? L.n_in : L.n_out;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = m0 + mm, k = k0 + kk + j;
+        As[kk + j][mm] = (m < M && k < K) ? to_f<AT>(src[(uint64_t)m * ld + k]) : 0.f;
+      }
+    }
+    // B tile
+    if (MODE == 0) {            // k contiguous: B(k,n) = W[n*in + k]
+      int nn = tid >> 2, kk = (tid & 3) * 4;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int n = n0 + nn, k = k0 + kk + j;
+        Bs[kk + j][nn] = (n < N && k < K) ? to_f<WT>(wf[(uint64_t)n * L.n_in + k]) : 0.f;
+      }
+    } else {                    // n contiguous
+      int kk = tid >> 4, nn = (tid & 15) * 4;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int n = n0 + nn + j, k = k0 + kk;
+        float v = 0.f;
+        if (n < N && k < K) {
+          uint64_t idx = (uint64_t)k * L.n_in + n;
+          if (MODE == 1) {      // T2: w - (tau_fwd - tau_bkwd) * delta, then rounded as the operand type holds it
+            float wv = wm[idx];
+            if (corr) wv = __fsub_rn(wv, __fmul_rn(gapf, dl[idx]));
+            v = round_as<WT>(wv);
+          } else {
+            v = to_f<AT>(xin[idx]);
+          }
+        }
+        Bs[kk][nn + j] = v;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  // epilogue
+  if (MODE == 0) {
+    AT* zout = ring_ptr<AT>(t, L.z_ring, d.f_slot, n_xout);
+    AT* yout;
+    if (lvl < s.n_lin - 1) yout = ring_ptr<AT>(t, L.h_ring, d.f_slot, n_xout);
+    else if (p < t.P - 1) yout = ring_ptr<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n_xout);
+    else yout = ws_ptr<AT>(t, t.yout_off) + (uint64_t)(d.tick & 1) * n_xout;
+    const float* bias = t.a.w + L.b_off;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+        if (m < M && n < N) {
+          AT zv = from_f<AT>(__fadd_rn(acc[i][j], bias[n]));
+          zout[(uint64_t)m * N + n] = zv;
+          yout[(uint64_t)m * N + n] = from_f<AT>(act_fwd(to_f<AT>(zv), L.act));
+        }
+      }
+  } else if (MODE == 1) {
+    AT* dx = (lvl == 0) ? ws_ptr<AT>(t, t.st[p - 1].gin) + (uint64_t)(d.tick & 1) * n_xin : ws_ptr<AT>(t, s.dh);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+        if (m < M && n < N) dx[(uint64_t)m * N + n] = from_f<AT>(acc[i][j]);
+      }
+  } else {
+    float* dW = t.a.grad + L.w_off;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+        if (m < M && n < N) dW[(uint64_t)m * N + n] = acc[i][j];
+      }
+  }
+}
+
+template <typename AT, typename WT>
+static cudaError_t launch_simt_t(const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
+  const int mt = mode == 2 ? t.max_dim : t.T;
+  dim3 grid((t.max_dim + BN - 1) / BN, (mt + BM - 1) / BM, t.P);
+  if (mode == 0) simt_gemm_kernel<AT, WT, 0><<<grid, 256, 0, stream>>>(t, lvl);
+  else if (mode == 1) simt_gemm_kernel<AT, WT, 1><<<grid, 256, 0, stream>>>(t, lvl);
+  else simt_gemm_kernel<AT, WT, 2><<<grid, 256, 0, stream>>>(t, lvl);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_simt_gemm(const TickArgs& t, int dtype, int mode, int lvl, cudaStream_t stream) {
+  if (dtype == PM_F32) return launch_simt_t<float, float>(t, mode, lvl, stream);
+  return launch_simt_t<__nv_bfloat16, __nv_bfloat16>(t, mode, lvl, stream);
+}
+
+}  // namespace pm

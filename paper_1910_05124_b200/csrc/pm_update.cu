@@ -1,0 +1,210 @@
+// Tick scheduler and the fused multi-tensor PipeMare update.
+//
+// The update is a pure HBM stream: per parameter it reads g, w, m, delta (and s for
+// Adam) and writes w, m, delta (and s) in fp32 plus a bfloat16 copy of w: 30 bytes per
+// parameter for momentum SGD, 38 for Adam.  One launch covers every stage; the stage
+// that owns a 64-element group is found by binary search in shared memory, and that
+// stage's scalars (T1 step size, T2 decay, Adam bias corrections) come from the table
+// the scheduler wrote for this tick.
+//
+// Arithmetic order (each operation rounded once in fp32, no fused multiply-add, so that
+// results can be reproduced bit for bit by any IEEE implementation):
+//   SGD-m (Appendix B.3):  v' = beta*v - alpha*g ;  w' = w + v'
+//   Adam:  m' = b1*m + (1-b1)*g ;  s' = b2*s + (1-b2)*(g*g) ;
+//          w' = w - (alpha*(m'/bc1)) / (sqrt(s'/bc2) + eps)
+//   T2 (Section 3.2):      delta' = gamma*delta + (1-gamma)*(w' - w)
+#include "pm_update.cuh"
+
+namespace pm {
+
+// ---- scheduler -------------------------------------------------------------------------------
+//
+// Tick s, stage i (1-based): forward of microbatch a = s-(i-1); backward and update of
+// microbatch b = s-(2P-i).  T1 (Eq. 2): alpha_i = alpha_base(k) / tau_i^p, p = 1 - min(k/K, 1).
+// T2: gamma_i = D^(1/(tau_fwd,i - tau_bkwd,i)).  Scalars are evaluated in double and rounded to
+// float once.
+__global__ void schedule_kernel(const StageSched* __restrict__ sched, const int64_t* __restrict__ nupd,
+                                StageDyn* __restrict__ dyn, HyperDev hp, int64_t tick, int64_t n_fed,
+                                int64_t flat_k) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= hp.n_stages) return;
+  StageSched s = sched[i];
+  StageDyn d;
+  const int P = hp.n_stages;
+  d.tick = tick;
+  int64_t ver = nupd[i];
+  if (flat_k >= 0) {
+    d.f_mb = -1; d.b_mb = -1; d.k = flat_k;
+    d.f_slot = d.f_xslot = d.f_next_xslot = d.b_slot = d.b_xslot = 0;
+  } else {
+    int64_t a = tick - i;
+    int64_t b = tick - (2 * (int64_t)P - (i + 1));
+    bool fa = a >= 0 && a < n_fed;
+    bool ba = b >= 0 && b < n_fed;
+    d.f_mb = fa ? a : -1;
+    d.b_mb = ba ? b : -1;
+    d.k = ba ? b : -1;
+    d.f_slot = fa ? (int32_t)(a % s.depth) : 0;
+    d.f_xslot = fa ? (int32_t)(a % s.xdepth) : 0;
+    d.f_next_xslot = (fa && s.next_xdepth > 0) ? (int32_t)(a % s.next_xdepth) : 0;
+    d.b_slot = ba ? (int32_t)(b % s.depth) : 0;
+    d.b_xslot = ba ? (int32_t)(b % s.xdepth) : 0;
+  }
+  d.f_ver = ver;
+  d.b_ver = ver;
+  d.active_update = d.k >= 0 ? 1 : 0;
+  d.alpha = 0.f; d.gamma = 0.f; d.one_minus_gamma = 1.f; d.bc1 = 1.f; d.bc2 = 1.f; d.use_delta = 0;
+  if (d.k >= 0) {
+    int64_t k = d.k;
+    double base = hp.alpha_const;
+    if (hp.alpha_tab != nullptr) base = hp.alpha_tab[k < hp.alpha_len ? k : hp.alpha_len - 1];
+    double alpha = base;
+    if (hp.t1) {
+      double r = (double)k / (double)hp.K;
+      double p = 1.0 - (r < 1.0 ? r : 1.0);
+      int tau = s.tau_f > 1 ? s.tau_f : 1;
+      alpha = base / pow((double)tau, p);
+    }
+    d.alpha = (float)alpha;
+    if (hp.t2 && s.gap > 0) {
+      d.gamma = (float)pow(hp.D, 1.0 / (double)s.gap);
+      d.one_minus_gamma = 1.0f - d.gamma;
+      d.use_delta = 1;
+    }
+    if (hp.optimizer == PM_ADAM) {
+      d.bc1 = (float)(1.0 - pow((double)hp.beta1, (double)(k + 1)));
+      d.bc2 = (float)(1.0 - pow((double)hp.beta2, (double)(k + 1)));
+    }
+  }
+  dyn[i] = d;
+}
+
+cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageDyn* dyn, HyperDev hp,
+                            int64_t tick, int64_t n_fed, int64_t flat_k, cudaStream_t stream) {
+  int threads = 128;
+  int blocks = (hp.n_stages + threads - 1) / threads;
+  schedule_kernel<<<blocks, threads, 0, stream>>>(sched, nupd, dyn, hp, tick, n_fed, flat_k);
+  return cudaGetLastError();
+}
+
+// ---- fused update ------------------------------------------------------------------------------
+
+struct UpdScalars {
+  float alpha, gamma, omg, bc1, bc2;
+  int use_delta;
+};
+
+__device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void st_stream(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+template <int OPT>
+__device__ __forceinline__ float upd_one(float g, float w, float& m, float& s, float& dl, const UpdScalars& c,
+                                         float beta1, float beta2, float omb1, float omb2, float eps) {
+  float wn;
+  if (OPT == PM_SGDM) {
+    m = __fsub_rn(__fmul_rn(beta1, m), __fmul_rn(c.alpha, g));
+    wn = __fadd_rn(w, m);
+  } else {
+    m = __fadd_rn(__fmul_rn(beta1, m), __fmul_rn(omb1, g));
+    s = __fadd_rn(__fmul_rn(beta2, s), __fmul_rn(omb2, __fmul_rn(g, g)));
+    float mh = __fdiv_rn(m, c.bc1);
+    float sh = __fdiv_rn(s, c.bc2);
+    wn = __fsub_rn(w, __fdiv_rn(__fmul_rn(c.alpha, mh), __fadd_rn(__fsqrt_rn(sh), eps)));
+  }
+  if (c.use_delta) dl = __fadd_rn(__fmul_rn(c.gamma, dl), __fmul_rn(c.omg, __fsub_rn(wn, w)));
+  return wn;
+}
+
+constexpr int kUpdThreads = 256;
+constexpr int kUpdUnroll = 2;      // float4 groups per thread per array in flight
+
+template <int OPT, bool HAS_LP>
+__global__ void __launch_bounds__(kUpdThreads)
+update_kernel(ArenasDev a, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
+              const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
+              float beta1, float beta2, float eps) {
+  extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends
+  uint32_t* sb = sm_bounds;
+  uint32_t* se = sm_bounds + n_stages;
+  for (int i = threadIdx.x; i < n_stages; i += blockDim.x) { sb[i] = begin64[i]; se[i] = end64[i]; }
+  __syncthreads();
+  const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
+  const uint64_t stride = (uint64_t)gridDim.x * kUpdThreads * kUpdUnroll;
+  for (uint64_t base = (uint64_t)blockIdx.x * kUpdThreads * kUpdUnroll; base < total_vec4; base += stride) {
+    uint64_t v[kUpdUnroll];
+    int stage[kUpdUnroll];
+    UpdScalars sc[kUpdUnroll];
+    float4 g[kUpdUnroll], w[kUpdUnroll], m[kUpdUnroll], dl[kUpdUnroll], s[kUpdUnroll];
+#pragma unroll
+    for (int u = 0; u < kUpdUnroll; ++u) {
+      v[u] = base + (uint64_t)u * kUpdThreads + threadIdx.x;
+      stage[u] = -1;
+      if (v[u] < total_vec4) {
+        uint32_t e64 = (uint32_t)(v[u] >> 4);
+        int lo = 0, hi = n_stages - 1;               // largest i with sb[i] <= e64
+        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (sb[mid] <= e64) lo = mid; else hi = mid - 1; }
+        if (sb[lo] <= e64 && e64 < se[lo] && dyn[lo].active_update) stage[u] = lo;
+      }
+      if (stage[u] >= 0) {
+        const uint64_t e = v[u] * 4;
+        g[u] = ld_stream(a.grad + e);
+        w[u] = ld_stream(a.w + e);
+        m[u] = ld_stream(a.m + e);
+        const StageDyn& d = dyn[stage[u]];
+        sc[u].alpha = d.alpha; sc[u].gamma = d.gamma; sc[u].omg = d.one_minus_gamma;
+        sc[u].bc1 = d.bc1; sc[u].bc2 = d.bc2; sc[u].use_delta = d.use_delta;
+        if (sc[u].use_delta) dl[u] = ld_stream(a.delta + e);
+        if (OPT == PM_ADAM) s[u] = ld_stream(a.s + e);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUpdUnroll; ++u) {
+      if (stage[u] < 0) continue;
+      const uint64_t e = v[u] * 4;
+      float4 wn;
+      wn.x = upd_one<OPT>(g[u].x, w[u].x, m[u].x, s[u].x, dl[u].x, sc[u], beta1, beta2, omb1, omb2, eps);
+      wn.y = upd_one<OPT>(g[u].y, w[u].y, m[u].y, s[u].y, dl[u].y, sc[u], beta1, beta2, omb1, omb2, eps);
+      wn.z = upd_one<OPT>(g[u].z, w[u].z, m[u].z, s[u].z, dl[u].z, sc[u], beta1, beta2, omb1, omb2, eps);
+      wn.w = upd_one<OPT>(g[u].w, w[u].w, m[u].w, s[u].w, dl[u].w, sc[u], beta1, beta2, omb1, omb2, eps);
+      st_stream(a.w + e, wn);
+      st_stream(a.m + e, m[u]);
+      if (OPT == PM_ADAM) st_stream(a.s + e, s[u]);
+      if (sc[u].use_delta) st_stream(a.delta + e, dl[u]);
+      if (HAS_LP) {
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(wn.x, wn.y);
+        __nv_bfloat162 hi2 = __floats2bfloat162_rn(wn.z, wn.w);
+        uint2 packed;
+        packed.x = *reinterpret_cast<uint32_t*>(&lo2);
+        packed.y = *reinterpret_cast<uint32_t*>(&hi2);
+        *reinterpret_cast<uint2*>(a.w_lp + e) = packed;   // re-read by the next forward: default caching
+      }
+      if ((uint32_t)(v[u] >> 4) == sb[stage[u]] && (v[u] & 15) == 0) nupd[stage[u]] += 1;
+    }
+  }
+}
+
+cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
+                          int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
+                          float eps, cudaStream_t stream) {
+  if (total64 == 0 || n_stages == 0) return cudaSuccess;
+  uint64_t total_vec4 = total64 * 16;
+  uint64_t per_block = (uint64_t)kUpdThreads * kUpdUnroll;
+  uint64_t need = (total_vec4 + per_block - 1) / per_block;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  uint64_t cap = (uint64_t)sms * 8;                 // whole waves of resident blocks
+  int blocks = (int)(need < cap ? need : cap);
+  size_t smem = sizeof(uint32_t) * 2 * (size_t)n_stages;
+  bool lp = a.w_lp != nullptr;
+  if (optimizer == PM_SGDM) {
+    if (lp) update_kernel<PM_SGDM, true><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
+    else    update_kernel<PM_SGDM, false><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
+  } else {
+    if (lp) update_kernel<PM_ADAM, true><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
+    else    update_kernel<PM_ADAM, false><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace pm

@@ -1,0 +1,104 @@
+"""The C-ABI library loads on a machine without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def built_lib():
+    from paper_1910_05124_b200 import build
+    path = build.build()
+    return ctypes.CDLL(path)
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "pipemare.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pm_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_required_entry_points():
+    syms = declared_symbols()
+    for name in ("pm_init_stages", "pm_forward", "pm_backward", "pm_update", "pm_step", "pm_update_flat",
+                 "pm_query_bytes", "pm_get_bookkeeping", "pm_get_losses", "pm_destroy"):
+        assert name in syms
+
+
+def test_library_exports_every_declared_symbol(built_lib):
+    for name in declared_symbols():
+        assert hasattr(built_lib, name), name
+
+
+def test_layout_arithmetic_needs_no_gpu(built_lib):
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding
+    cnt, offs = binding.stage_layout(I.cfg3().stages[0])
+    assert cnt == 2 * (1024 * 1024 + 1024)
+    assert offs == [(0, 1024 * 1024), (1024 * 1024 + 1024, 2 * 1024 * 1024 + 1024)]
+    cnt, offs = binding.stage_layout([I.LinearSpec(40, 24, "relu")])
+    assert offs == [(0, 960)] and cnt == 960 + 64          # W padded to 960 (=15*64), b padded to 64
+
+
+def test_query_bytes_and_state_copies_ratio(built_lib):
+    # PipeMare adds one weight-sized accumulator: 4/3 of the SGD-momentum state, 5/4 of Adam's
+    # (weight + optimiser memory relative to the synchronous baseline, Table 2 / Section 4.2)
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    wl = I.cfg1()
+    for opt, ratio in (("sgdm", 4 / 3), ("adam", 5 / 4)):
+        wl.optimizer = opt
+        P = len(wl.stages)
+        ops = [B._ops_array(st) for st in wl.stages]
+        sd = (B.pm_stage_desc * P)()
+        off = 0
+        for p in range(P):
+            cnt, _ = B.stage_layout(wl.stages[p])
+            sd[p].tau_fwd, sd[p].tau_bkwd, sd[p].n_ops = wl.tau_fwd[p], 0, len(wl.stages[p])
+            sd[p].ops = C.cast(ops[p], C.POINTER(B.pm_op_desc))
+            sd[p].param_offset, sd[p].param_count = off, cnt
+            off += cnt
+        cfg, _ = B.make_config(n_stages=P, microbatch=32, compute="f32", optimizer=opt, alpha=0.01, K=32)
+        sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+        assert B.lib().pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+        # state copies: weight, gradient, optimiser state (the synchronous baseline) plus delta
+        copies = sb.value / (off * 4)
+        baseline = 3 if opt == "sgdm" else 4            # w, g, v   |   w, g, m, s
+        assert copies == baseline + 1
+        assert copies / baseline == pytest.approx(ratio, rel=1e-12)
+        # ring: sum over stages of (tau+2) input slots + (tau+1) pre-activation slots, 32x256 fp32 each
+        slots = sum((t + 2) + (t + 1) for t in wl.tau_fwd)
+        assert rb.value == slots * 32 * 256 * 4
+
+
+def test_bad_arguments_are_rejected_without_a_gpu(built_lib):
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    wl = I.cfg1()
+    P = len(wl.stages)
+    ops = [B._ops_array(st) for st in wl.stages]
+    sd = (B.pm_stage_desc * P)()
+    off = 0
+    for p in range(P):
+        cnt, _ = B.stage_layout(wl.stages[p])
+        sd[p].tau_fwd, sd[p].tau_bkwd, sd[p].n_ops = wl.tau_fwd[p], 0, 1
+        sd[p].ops = C.cast(ops[p], C.POINTER(B.pm_op_desc))
+        sd[p].param_offset, sd[p].param_count = off, cnt
+        off += cnt
+    cfg, _ = B.make_config(n_stages=P, microbatch=32, compute="f32", optimizer="sgdm", alpha=0.01, K=32)
+    sb = C.c_uint64()
+    sd[1].tau_fwd = 4                                    # not 2(P-i)+1
+    st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), None, None)
+    assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED"
+    assert b"tau_fwd" in L.pm_last_error(None)
+    sd[1].tau_fwd = 5
+    ops[2][0].n_in = 128                                 # breaks the chain 256 -> 128
+    st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), None, None)
+    assert L.pm_status_string(st) == b"PM_ERR_SHAPE"
+    assert L.pm_status_string(L.pm_forward(None, None, None)) == b"PM_ERR_INVALID_ARG"

@@ -1,0 +1,110 @@
+"""GPU parity of the tick-major pipeline (pm_step) against the microbatch-major oracle."""
+import numpy as np
+import pytest
+
+import pm_inputs as I
+from parity_util import run_gpu_pipeline, run_oracle, compare_params, max_rel_err
+
+pytestmark = pytest.mark.gpu
+
+F32_TOL = 1e-5          # max |dw| / max |w| per tensor, fp32 path
+BF16_W_TOL = 2e-2       # bf16 GEMM path, weights
+BF16_LOSS_TOL = 1e-3    # bf16 GEMM path, loss trajectory (relative)
+
+
+def check_book(book, res, n_steps, P):
+    ref = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    assert len(book) == n_steps * P
+    for key, (vf, vb) in book.items():
+        assert (vf, vb) == ref[key], f"microbatch/stage {key}: device ({vf},{vb}) oracle {ref[key]}"
+
+
+def test_cfg1_fp32_full_run(cuda_device):
+    wl = I.cfg1()
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-5)
+    worst = compare_params(pipe, res, F32_TOL)
+    print("cfg1 worst relative weight error", worst)
+
+
+@pytest.mark.parametrize("P,width,T,per_stage,act,opt", [
+    (1, 64, 8, 1, "relu", "sgdm"),          # single stage: tau = 1
+    (3, 40, 7, 2, "gelu", "sgdm"),          # ragged everything
+    (5, 130, 33, 1, "relu", "adam"),        # spans several 64-wide tiles with a tail
+    (2, 72, 65, 3, "none", "adam"),
+])
+def test_fp32_shapes(cuda_device, P, width, T, per_stage, act, opt):
+    wl = I.mlp_workload("t", P, width, per_stage, act, T, compute="f32", optimizer=opt,
+                        alpha=0.01 if opt == "sgdm" else 1e-3, K=6, D=0.5, steps=14, seed=77 + P)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, P)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
+    compare_params(pipe, res, 2e-5 if opt == "adam" else F32_TOL)
+
+
+@pytest.mark.parametrize("t1,t2", [(False, False), (True, False), (False, True)])
+def test_fp32_technique_switches(cuda_device, t1, t2):
+    wl = I.mlp_workload("t", 3, 64, 1, "relu", 16, compute="f32", optimizer="sgdm", alpha=0.02, K=5, D=0.3,
+                        steps=12, seed=5, t1=t1, t2=t2)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-5)
+    compare_params(pipe, res, F32_TOL)
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam"])
+def test_bf16_small(cuda_device, opt):
+    wl = I.cfg3_small(optimizer=opt)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_LOSS_TOL)
+    worst = compare_params(pipe, res, BF16_W_TOL)
+    print("bf16 small worst relative weight error", worst)
+    # the bf16 shadow the forward reads is exactly the rounded master copy
+    import torch
+    assert torch.equal(pipe.w_lp, pipe.w.to(torch.bfloat16))
+
+
+def test_phase_order_and_drain_rules(cuda_device):
+    import torch
+    import paper_1910_05124_b200 as pm
+    wl = I.mlp_workload("t", 2, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
+    pipe = pm.Pipeline(wl, I.init_stage_params(wl))
+    x, y = I.batch(wl, 0)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_STATE"):
+        pipe.pm_backward()
+    pipe.pm_forward(xd, yd)
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_STATE"):
+        pipe.pm_forward(xd, yd)
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_STATE"):
+        pipe.pm_update()
+    pipe.pm_backward()
+    pipe.pm_update()
+    pipe.pm_step(None, None)
+    with pytest.raises(pm.PipeMareError, match="draining"):
+        pipe.pm_step(xd, yd)
+    with pytest.raises(pm.PipeMareError, match="not finished"):
+        pipe.pm_get_losses(0, 1)
+
+
+def test_too_small_buffers_are_reported(cuda_device):
+    import ctypes as C
+    import torch
+    import paper_1910_05124_b200 as pm
+    wl = I.mlp_workload("t", 2, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
+    pipe = pm.Pipeline(wl, I.init_stage_params(wl))
+    ctx = C.c_void_p()
+    st = pipe.L.pm_init_stages(C.byref(ctx), C.byref(pipe.cfg), pipe.stage_desc, C.byref(pipe.arenas),
+                               pipe.ring.data_ptr(), 256, pipe.workspace.data_ptr(), pipe.workspace.numel(),
+                               C.c_void_p(pipe.stream.cuda_stream))
+    assert pipe.L.pm_status_string(st) == b"PM_ERR_NOMEM"
+    assert str(pipe.ring_bytes).encode() in pipe.L.pm_last_error(None)
