@@ -193,6 +193,30 @@ pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
                          const int32_t* tau_bkwd, int32_t n_stages, const pm_config* cfg,
                          int64_t k, void* workspace, uint64_t workspace_bytes, void* stream);
 
+/* The same update for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience).  Who needs it: code running under a framework whose caching
+ * allocator already owns the device, real-time loops that must not allocate after start-up, and
+ * plug-ins that receive tensors but no allocator -- none of them can produce the `workspace`
+ * pm_update_flat asks for.  Here the stage table lives in a fixed array inside the library
+ * (about 35 KB on every GPU that loads the library, held until the process exits), so the call
+ * takes only the arenas.  Arguments and results are those of pm_update_flat.
+ *   - At most pm_update_flat_static_max_stages() (= 256) stages; more is PM_ERR_NOMEM with a
+ *     message that says so.  pm_update_flat_static_last_error() returns the message (per thread).
+ *   - Neither this call nor anything it uses calls cudaMalloc, cudaFree or an allocating library
+ *     routine; host staging is a fixed per-thread buffer.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any CUDA stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; each
+ *     call rewrites the whole table, counters included, before its kernels read it.  Two calls
+ *     whose GPU work overlaps (different streams, or threads racing on one device) would
+ *     overwrite each other's table: issue them on one stream or serialise them. */
+int32_t pm_update_flat_static_max_stages(void);
+const char* pm_update_flat_static_last_error(void);
+pm_status pm_update_flat_static(const pm_arenas* arenas, const uint64_t* stage_offsets,
+                                const uint64_t* stage_counts, const int32_t* tau_fwd,
+                                const int32_t* tau_bkwd, int32_t n_stages, const pm_config* cfg,
+                                int64_t k, void* stream);
+
 const char* pm_status_string(pm_status s);
 
 #ifdef __cplusplus

@@ -87,6 +87,10 @@ def lib():
     L.pm_update_flat_workspace_bytes.restype = C.c_uint64
     L.pm_update_flat.argtypes = [C.POINTER(pm_arenas), u64p, u64p, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
                                  C.c_int32, C.POINTER(pm_config), C.c_int64, vp, C.c_uint64, vp]
+    L.pm_update_flat_static.argtypes = [C.POINTER(pm_arenas), u64p, u64p, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                        C.c_int32, C.POINTER(pm_config), C.c_int64, vp]
+    L.pm_update_flat_static_max_stages.restype = C.c_int32
+    L.pm_update_flat_static_last_error.restype = C.c_char_p
     _lib = L
     return L
 
@@ -283,3 +287,16 @@ class FlatUpdate:
         _check(self.L.pm_update_flat(C.byref(ar), self.offsets, self.counts, self.tau_fwd, self.tau_bkwd, self.P,
                                      C.byref(self.cfg), k, self.workspace.data_ptr(), self.ws_bytes,
                                      C.c_void_p(st.cuda_stream)))
+
+    def pm_update_flat_static(self, w, m, s, delta, grad, w_lp, k, stream=None):
+        """Same update through the entry point that needs no device workspace: for callers that are not
+        allowed to allocate on the device (the stage table sits in a fixed array inside the library)."""
+        torch = self.torch
+        st = stream if stream is not None else torch.cuda.current_stream(w.device)
+        ar = pm_arenas(w.data_ptr(), m.data_ptr(), s.data_ptr() if s is not None else None, delta.data_ptr(),
+                       grad.data_ptr(), w_lp.data_ptr() if w_lp is not None else None, w.numel())
+        status = self.L.pm_update_flat_static(C.byref(ar), self.offsets, self.counts, self.tau_fwd, self.tau_bkwd,
+                                              self.P, C.byref(self.cfg), k, C.c_void_p(st.cuda_stream))
+        if status != 0:
+            raise PipeMareError(self.L.pm_status_string(status).decode(),
+                                self.L.pm_update_flat_static_last_error().decode())
