@@ -31,7 +31,7 @@ def build(force=False, verbose=False):
         return LIB
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc"),
-           "-o", LIB] + [os.path.join(HERE, "csrc", s) for s in SOURCES] + ["-lcuda"]
+           "-o", LIB] + [os.path.join(HERE, "csrc", s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

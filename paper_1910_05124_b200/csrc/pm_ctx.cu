@@ -23,7 +23,7 @@ struct Layout {
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
-  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0;
+  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0;
   int64_t loss_cap = 0;
   int32_t max_lin = 0, max_dim = 0, n_in_first = 0, n_out_last = 0;
 };
@@ -110,6 +110,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
   L.off_tgt = w; w = align_up(w + sizeof(float) * (uint64_t)(P + 1) * T * L.n_out_last, 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * esz, 256);
+  L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes(P) : 0), 256);
   for (int p = 0; p < P; ++p) {
     StageDev& s = L.st[p];
     const int n_out_last = s.lin[s.n_lin - 1].n_out;
@@ -268,7 +269,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
 
   if (cfg->compute_dtype == PM_BF16) {
     std::string uerr;
-    pm_status us = umma_plan_create(&c->umma, t, c->L.st, uerr);
+    pm_status us = umma_plan_create(&c->umma, t, c->L.st, c->ws + L.off_umma, c->stream, uerr);
     if (us != PM_OK) { delete c; return fail(nullptr, us, uerr); }
   }
   *out = c;
@@ -356,6 +357,17 @@ pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets) {
   return pm_update(ctx);
 }
 
+// After a synchronisation: did any CTA give up on a bounded wait?
+static pm_status check_device_status(pm_ctx* ctx) {
+  int* w = umma_status_word(ctx->umma);
+  if (!w) return PM_OK;
+  int code = 0;
+  cudaError_t e = cudaMemcpy(&code, w, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "status read-back");
+  if (code != 0) return fail(ctx, PM_ERR_TIMEOUT, "a bounded device-side wait expired in a GEMM kernel (role code " + std::to_string(code) + ")");
+  return PM_OK;
+}
+
 pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
   if (!ctx || !out8) return fail(ctx, PM_ERR_INVALID_ARG, "null argument");
   if (stage < 0 || stage >= ctx->cfg.n_stages) return fail(ctx, PM_ERR_INVALID_ARG, "stage out of range");
@@ -365,6 +377,7 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
   if (e == cudaSuccess) e = cudaMemcpy(&d, ctx->ws + ctx->L.off_dyn + sizeof(StageDyn) * stage, sizeof(StageDyn), cudaMemcpyDeviceToHost);
   if (e == cudaSuccess) e = cudaMemcpy(&n, ctx->ws + ctx->L.off_nupd + sizeof(int64_t) * stage, sizeof(int64_t), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "bookkeeping read-back");
+  if (pm_status ds = check_device_status(ctx)) return ds;
   out8[0] = d.f_mb; out8[1] = d.f_ver; out8[2] = d.b_mb; out8[3] = d.b_ver; out8[4] = n;
   out8[5] = d.f_slot; out8[6] = d.b_slot; out8[7] = d.tick;
   return PM_OK;
@@ -381,6 +394,7 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
   for (int64_t i = 0; i < n && e == cudaSuccess; ++i)
     e = cudaMemcpy(host_out + i, ctx->ws + ctx->L.off_loss + sizeof(float) * ((first_mb + i) % ctx->L.loss_cap), sizeof(float), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "loss read-back");
+  if (pm_status ds = check_device_status(ctx)) return ds;
   return PM_OK;
 }
 

@@ -1,14 +1,473 @@
-// bf16 grouped GEMMs.  Scaffold: routes to the SIMT kernels until the tcgen05 path lands.
+// bf16 grouped GEMMs of the pipeline on the 5th-generation tensor cores.
+//
+// One CTA computes one 128x128 output tile of one stage; blockIdx.z selects the stage, so a single
+// launch covers every stage that is active in this tick.  Operands are staged in shared memory in the
+// 128-byte-swizzled canonical layouts (TMA writes them; for dgrad a transform step writes B), the
+// accumulator lives in tensor memory (128 lanes x 128 fp32 columns), one elected thread issues
+// tcgen05.mma, and four warps drain the accumulator with tcgen05.ld for the epilogue.
+//
+//   mode 0 forward  D[T,out]  = x[T,in] * W[out,in]^T      A K-major (TMA), B K-major (TMA, bf16 shadow)
+//                   z = bf16(D + b) -> ring,  y = bf16(act(z)) -> next consumer
+//   mode 1 dgrad    D[T,in]   = dz[T,out] * Wc[out,in]     A K-major (TMA), B MN-major, written by the
+//                   transform warps as bf16(w - gap*delta) from the fp32 master arenas (T2 of
+//                   Section 3.2): the corrected weights exist only in shared memory
+//   mode 2 wgrad    D[out,in] = dz[T,out]^T * x[T,in]      A MN-major (TMA), B MN-major (TMA), fp32 out
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
+// warps 2..5 = (mode 1: operand transform, then) epilogue.
+// Every wait on an mbarrier is bounded; on expiry the CTA records a code in a status word, stops
+// issuing work, waits (bounded) for its copies in flight, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "pm_umma.cuh"
 
 namespace pm {
-struct UmmaPlan { int dummy; };
-pm_status umma_plan_create(UmmaPlan** out, const TickArgs&, const std::vector<StageDev>&, std::string&) {
-  *out = new UmmaPlan{0};
+
+constexpr int TILE_M = 128, TILE_N = 128, TILE_K = 64;     // bf16: 64 elements = one 128-byte swizzle row
+constexpr int N_STAGES = 3;
+constexpr int A_BYTES = TILE_M * TILE_K * 2;               // 16 KB
+constexpr int B_BYTES = TILE_N * TILE_K * 2;               // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TMEM_COLS = 128;
+constexpr int SMEM_BYTES = N_STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int N_THREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;      // about one second
+
+enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAPS_PER_LINEAR = 5 };
+
+// ---- PTX wrappers -----------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag and the global status word) when the
+// barrier did not flip within the cycle limit or another role of this CTA has already given up.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, code);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Offsets are in bytes.
+//   K-major : rows of 64 elements (128 B); 8-row groups 1024 B apart (stride offset); leading offset unused.
+//   MN-major: 64-element runs along M/N (128 B) x 8 k-rows = 1024 B atoms; next 8 k-rows `stride` bytes on,
+//             next 64-element run along M/N `leading` bytes on.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t leading_bytes, uint32_t stride_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((leading_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((stride_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;          // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;          // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, operand majors as given.
+__device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---- the kernel --------------------------------------------------------------------------------------
+template <int MODE>
+__global__ void __launch_bounds__(N_THREADS) umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int lvl, int* status) {
+  const int p = blockIdx.z;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (lvl >= s.n_lin) return;
+  if (MODE == 0 ? d.f_mb < 0 : d.b_mb < 0) return;
+  if (MODE == 1 && p == 0 && lvl == 0) return;          // the network input needs no gradient
+  const LinDev& L = s.lin[lvl];
+  int M, N, K;
+  if (MODE == 0) { M = t.T; N = L.n_out; K = L.n_in; }
+  else if (MODE == 1) { M = t.T; N = L.n_in; K = L.n_out; }
+  else { M = L.n_out; N = L.n_in; K = t.T; }
+  const int m0 = blockIdx.y * TILE_M, n0 = blockIdx.x * TILE_N;
+  if (m0 >= M || n0 >= N) return;
+  const int n_kb = (K + TILE_K - 1) / TILE_K;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  const uint32_t bars = tiles + N_STAGES * STAGE_BYTES;
+  // barrier block: full[N_STAGES], empty[N_STAGES], tmem_full, then tmem base word and abort flag
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * N_STAGES, bar_tmem = bars + 16 * N_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + N_STAGES * STAGE_BYTES + 16 * N_STAGES + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const CUtensorMap* lm = maps + ((size_t)p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+
+  if (threadIdx.x == 0) {
+    const uint32_t full_count = MODE == 1 ? 1 + 4 : 1;               // TMA thread (+ one arrival per transform warp)
+    for (int i = 0; i < N_STAGES; ++i) { mbar_init(bar_full + 8 * i, full_count); mbar_init(bar_empty + 8 * i, 1); }
+    mbar_init(bar_tmem, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      for (int kb = 0; kb < n_kb; ++kb) {
+        const int st = kb % N_STAGES;
+        const uint32_t ph = (kb / N_STAGES) & 1;
+        if (*abort_flag || !mbar_wait(bar_empty + 8 * st, ph ^ 1, abort_flag, status, 1)) break;
+        const uint32_t sa = tiles + st * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * st;
+        const int k0 = kb * TILE_K;
+        if (MODE == 0) {
+          mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+          tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, m0, lvl == 0 ? d.f_xslot : d.f_slot);
+          tma_load_2d(sb, lm + MAP_W_K, fb, k0, n0);
+        } else if (MODE == 1) {
+          mbar_arrive_expect_tx(fb, A_BYTES);
+          tma_load_2d(sa, lm + MAP_DZ_K, fb, k0, m0);
+        } else {
+          mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+          const int slot = lvl == 0 ? d.b_xslot : d.b_slot;
+          tma_load_2d(sa, lm + MAP_DZ_MN, fb, m0, k0);
+          tma_load_2d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, m0 + 64, k0);
+          tma_load_3d(sb, lm + MAP_ACT_MN, fb, n0, k0, slot);
+          tma_load_3d(sb + B_BYTES / 2, lm + MAP_ACT_MN, fb, n0 + 64, k0, slot);
+        }
+        issued = kb + 1;
+      }
+      if (*abort_flag) {
+        // copies already issued still land in this CTA's shared memory: wait for them (bounded) before leaving
+        for (int kb = issued > N_STAGES ? issued - N_STAGES : 0; kb < issued; ++kb) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_full + 8 * (kb % N_STAGES), (kb / N_STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(MODE == 2, MODE != 0);
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int st = kb % N_STAGES;
+        const uint32_t ph = (kb / N_STAGES) & 1;
+        if (*abort_flag || !mbar_wait(bar_full + 8 * st, ph, abort_flag, status, 2)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = tiles + st * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+        for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
+          // K-major: 16 elements = 32 bytes along the swizzled row.  MN-major: 16 k-rows of 128 bytes.
+          const uint64_t da = MODE == 2 ? make_desc(sa + k16 * 2048, A_BYTES / 2, 1024) : make_desc(sa + k16 * 32, 16, 1024);
+          const uint64_t db = MODE == 0 ? make_desc(sb + k16 * 32, 16, 1024) : make_desc(sb + k16 * 2048, B_BYTES / 2, 1024);
+          tc_mma_bf16(tmem_base, da, db, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+        }
+        tc_commit(bar_empty + 8 * st);        // frees the stage once these MMAs have read it
+      }
+      if (ok) tc_commit(bar_tmem);            // accumulator complete
+    }
+  } else {
+    // ---------------- warps 2..5: transform (dgrad) then epilogue ----------------
+    const int q = warp & 3;                                           // TMEM lane group this warp may read
+    if (MODE == 1) {
+      const int tt = threadIdx.x - 64;                                // 0..127
+      const int c = tt & 15, rb = tt >> 4;                            // 16-byte chunk (8 columns) and row within 8-row group
+      const int n = n0 + c * 8;
+      const float gapf = (float)s.gap;
+      const bool corr = d.use_delta != 0;
+      const float* wm = t.a.w + L.w_off;
+      const float* dl = t.a.delta + L.w_off;
+      const uint32_t dst_in_tile = (uint32_t)(c >> 3) * (B_BYTES / 2) + (uint32_t)rb * 128 + (uint32_t)(((c & 7) ^ rb) << 4);
+      for (int kb = 0; kb < n_kb; ++kb) {
+        const int st = kb % N_STAGES;
+        const uint32_t ph = (kb / N_STAGES) & 1;
+        bool go = !*abort_flag && mbar_wait(bar_empty + 8 * st, ph ^ 1, abort_flag, status, 3);
+        go = __all_sync(0xffffffffu, go);                             // leave the loop as a whole warp
+        if (!go) break;
+        float4 w0[8], w1[8], d0[8], d1[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int k = kb * TILE_K + rb + 8 * j;
+          if (k < K && n < N) {
+            const size_t idx = (size_t)k * L.n_in + n;
+            w0[j] = *reinterpret_cast<const float4*>(wm + idx);
+            w1[j] = *reinterpret_cast<const float4*>(wm + idx + 4);
+            if (corr) {
+              d0[j] = *reinterpret_cast<const float4*>(dl + idx);
+              d1[j] = *reinterpret_cast<const float4*>(dl + idx + 4);
+            } else {
+              d0[j] = make_float4(0.f, 0.f, 0.f, 0.f); d1[j] = d0[j];
+            }
+          } else {
+            w0[j] = make_float4(0.f, 0.f, 0.f, 0.f); w1[j] = w0[j]; d0[j] = w0[j]; d1[j] = w0[j];
+          }
+        }
+        uint8_t* sb = tiles_ptr + st * STAGE_BYTES + A_BYTES;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float v[8] = {w0[j].x, w0[j].y, w0[j].z, w0[j].w, w1[j].x, w1[j].y, w1[j].z, w1[j].w};
+          if (corr) {
+            const float dd[8] = {d0[j].x, d0[j].y, d0[j].z, d0[j].w, d1[j].x, d1[j].y, d1[j].z, d1[j].w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = __fsub_rn(v[e], __fmul_rn(gapf, dd[e]));   // w - (tau_fwd - tau_bkwd) * delta
+          }
+          uint4 pk = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+          *reinterpret_cast<uint4*>(sb + dst_in_tile + j * 1024) = pk;
+        }
+        fence_async_smem();                                           // make the generic-proxy stores visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_full + 8 * st);
+      }
+    }
+    // epilogue
+    bool acc_ready = !*abort_flag && mbar_wait(bar_tmem, 0, abort_flag, status, 4);
+    acc_ready = __all_sync(0xffffffffu, acc_ready);                   // tcgen05.ld needs the whole warp
+    if (acc_ready) {
+      tc_fence_after();
+      const int m = m0 + q * 32 + lane;
+#pragma unroll 1
+      for (int cc = 0; cc < TILE_N / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r);
+        tmem_ld_wait();
+        const int nb = n0 + cc * 32;
+        if (m < M) {
+          if (MODE == 0) {
+            const size_t n_out_elems = (size_t)t.T * L.n_out;
+            __nv_bfloat16* zout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.z_ring) + (size_t)d.f_slot * n_out_elems;
+            __nv_bfloat16* yout;
+            if (lvl < s.n_lin - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.h_ring) + (size_t)d.f_slot * n_out_elems;
+            else if (p < t.P - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[p + 1].x_ring) + (size_t)d.f_next_xslot * n_out_elems;
+            else yout = reinterpret_cast<__nv_bfloat16*>(t.ws + t.yout_off) + (size_t)(d.tick & 1) * n_out_elems;
+            const float* bias = t.a.w + L.b_off;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int n = nb + g * 8;
+              if (n < N) {
+                const float4 b0 = *reinterpret_cast<const float4*>(bias + n), b1 = *reinterpret_cast<const float4*>(bias + n + 4);
+                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                float zf[8], yf[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(r[g * 8 + e]), bb[e])));
+                  yf[e] = act_fwd(zf[e], L.act);
+                }
+                const size_t o = (size_t)m * N + n;
+                *reinterpret_cast<uint4*>(zout + o) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
+                *reinterpret_cast<uint4*>(yout + o) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
+              }
+            }
+          } else if (MODE == 1) {
+            const size_t n_in_elems = (size_t)t.T * L.n_in;
+            __nv_bfloat16* dx = (lvl == 0) ? reinterpret_cast<__nv_bfloat16*>(t.ws + t.st[p - 1].gin) + (size_t)(d.tick & 1) * n_in_elems
+                                           : reinterpret_cast<__nv_bfloat16*>(t.ws + s.dh);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int n = nb + g * 8;
+              if (n < N) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[g * 8 + e]);
+                *reinterpret_cast<uint4*>(dx + (size_t)m * N + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+              }
+            }
+          } else {
+            float* dW = t.a.grad + L.w_off;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              const int n = nb + g * 4;
+              if (n < N)
+                *reinterpret_cast<float4*>(dW + (size_t)m * N + n) =
+                    make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct UmmaPlan {
+  const CUtensorMap* d_maps = nullptr;
+  int* d_status = nullptr;
+};
+
+uint64_t umma_workspace_bytes(int n_stages) {
+  return (uint64_t)n_stages * PM_MAX_LINEARS * MAPS_PER_LINEAR * sizeof(CUtensorMap) + 256;
+}
+
+static bool encode(EncodeTiledFn fn, CUtensorMap* m, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                   const uint32_t* box, std::string& err) {
+  cuuint64_t gd[3]; cuuint64_t gs[2]; cuuint32_t bx[3]; cuuint32_t es[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return false; }
+  return true;
+}
+
+pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region, cudaStream_t stream, std::string& err) {
+  *out = nullptr;
+  void* fnp = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t ce = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres);
+  if (ce != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fnp) { err = "cuTensorMapEncodeTiled is not available from this driver"; return PM_ERR_CUDA; }
+  EncodeTiledFn fn = (EncodeTiledFn)fnp;
+  const int P = t.P;
+  std::vector<CUtensorMap> maps((size_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR);
+  memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+  const uint64_t T = (uint64_t)t.T;
+  for (int p = 0; p < P; ++p) {
+    const StageDev& s = st[p];
+    for (int l = 0; l < s.n_lin; ++l) {
+      const LinDev& L = s.lin[l];
+      CUtensorMap* m = maps.data() + ((size_t)p * PM_MAX_LINEARS + l) * MAPS_PER_LINEAR;
+      // input activation of this Linear: ring [slots][T][n_in]
+      char* act_base = t.ring + (l == 0 ? s.x_ring : s.lin[l - 1].h_ring);
+      const uint64_t slots = l == 0 ? (uint64_t)s.xdepth : (uint64_t)s.depth;
+      const uint64_t n_in = (uint64_t)L.n_in, n_out = (uint64_t)L.n_out;
+      {
+        uint64_t dims[3] = {n_in, T, slots}, strides[2] = {n_in * 2, T * n_in * 2};
+        uint32_t box_k[3] = {TILE_K, TILE_M, 1}, box_mn[3] = {64, TILE_K, 1};
+        if (!encode(fn, m + MAP_ACT_K, act_base, 3, dims, strides, box_k, err)) return PM_ERR_CUDA;
+        if (!encode(fn, m + MAP_ACT_MN, act_base, 3, dims, strides, box_mn, err)) return PM_ERR_CUDA;
+      }
+      {
+        uint64_t dims[2] = {n_in, n_out}, strides[1] = {n_in * 2};
+        uint32_t box[2] = {TILE_K, TILE_N};
+        if (!encode(fn, m + MAP_W_K, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err)) return PM_ERR_CUDA;
+      }
+      {
+        uint64_t dims[2] = {n_out, T}, strides[1] = {n_out * 2};
+        uint32_t box_k[2] = {TILE_K, TILE_M}, box_mn[2] = {64, TILE_K};
+        if (!encode(fn, m + MAP_DZ_K, t.ws + s.dz, 2, dims, strides, box_k, err)) return PM_ERR_CUDA;
+        if (!encode(fn, m + MAP_DZ_MN, t.ws + s.dz, 2, dims, strides, box_mn, err)) return PM_ERR_CUDA;
+      }
+    }
+  }
+  char* region = (char*)ws_region;
+  cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); return PM_ERR_CUDA; }
+  for (int mode = 0; mode < 3; ++mode) {
+    const void* f = mode == 0 ? (const void*)umma_gemm_kernel<0> : mode == 1 ? (const void*)umma_gemm_kernel<1> : (const void*)umma_gemm_kernel<2>;
+    e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return PM_ERR_CUDA; }
+  }
+  UmmaPlan* plan = new UmmaPlan();
+  plan->d_status = (int*)region;
+  plan->d_maps = (const CUtensorMap*)(region + 256);
+  *out = plan;
   return PM_OK;
 }
+
 void umma_plan_destroy(UmmaPlan* plan) { delete plan; }
-cudaError_t umma_launch(UmmaPlan*, const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
-  return launch_simt_gemm(t, PM_BF16, mode, lvl, stream);
+
+int* umma_status_word(UmmaPlan* plan) { return plan ? plan->d_status : nullptr; }
+
+cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
+  const int max_m = mode == 2 ? t.max_dim : t.T;
+  dim3 grid((t.max_dim + TILE_N - 1) / TILE_N, (max_m + TILE_M - 1) / TILE_M, t.P);
+  if (mode == 0) umma_gemm_kernel<0><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
+  else if (mode == 1) umma_gemm_kernel<1><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
+  else umma_gemm_kernel<2><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
+  return cudaGetLastError();
 }
+
 }  // namespace pm

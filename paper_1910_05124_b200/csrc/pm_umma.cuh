@@ -8,8 +8,14 @@ namespace pm {
 
 struct UmmaPlan;   // tensor maps and launch geometry, built once per context
 
-pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<StageDev>& st, std::string& err);
+// Bytes of caller workspace the plan needs (status word + tensor maps).
+uint64_t umma_workspace_bytes(int n_stages);
+// ws_region: device memory of at least umma_workspace_bytes(P), 256-byte aligned.  Synchronises `stream`.
+pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region,
+                           cudaStream_t stream, std::string& err);
 void umma_plan_destroy(UmmaPlan* plan);
+// Device word that a CTA sets when one of its bounded waits expired (0 = none).
+int* umma_status_word(UmmaPlan* plan);
 // mode: 0 forward, 1 dgrad (corrected weights formed in the operand-load path), 2 wgrad.
 cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream);
 
