@@ -33,7 +33,7 @@ UNIT = "samples/s"
 BYTES_PER_PARAM = {"sgdm": 30, "adam": 38}     # fp32 g,w,m,delta read + w,m,delta write + bf16 copy (+ s r/w)
 # DRAM traffic of one fused-update launch on the benchmark workload, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-UPDATE_TRAFFIC_BYTES = None
+UPDATE_TRAFFIC_BYTES = 1_976_000_000   # 2.941 GB at 100 M parameters, scaled by 67,174,400 / 100 M
 
 
 def measured_peaks():
@@ -51,7 +51,7 @@ class ClockSampler:
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.first = index, [], None, 0
 
     def start(self):
         try:
@@ -66,6 +66,15 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
+    def wait_first(self, timeout=3.0):
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < timeout:
+            time.sleep(0.02)
+
+    def mark(self):
+        """Samples taken before this point (start-up, pipeline fill) are not reported."""
+        self.first = max(len(self.rows) - 1, 0)
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -76,7 +85,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[self.first:]:
             if len(r) < 6:
                 continue
             try:
@@ -208,6 +217,41 @@ def update_sweep(device, peak_gbs, quick=False):
     return out
 
 
+def run_update_only(args):
+    """A few launches of the stand-alone fused update on one arena set (for profiler captures)."""
+    import torch
+    import paper_1910_05124_b200 as pm
+    import pm_inputs as I
+    device = torch.device("cuda:0")
+    n, P = args.update_only, 64
+    base, rem = divmod(n, P)
+    counts = [base + (1 if i < rem else 0) for i in range(P)]
+    offsets, cur = [], 0
+    for c in counts:
+        offsets.append(cur)
+        cur += -(-c // 64) * 64
+    tau_f, tau_b = I.pipemare_delays(P)
+    g = torch.Generator(device=device)
+    g.manual_seed(1910)
+    w = torch.randn(cur, device=device, generator=g)
+    gr = torch.randn(cur, device=device, generator=g) * 1e-3
+    m = torch.randn(cur, device=device, generator=g) * 1e-3
+    dl = torch.randn(cur, device=device, generator=g) * 1e-4
+    lp = torch.empty(cur, dtype=torch.bfloat16, device=device)
+    fu = pm.FlatUpdate(offsets, counts, tau_f, tau_b, optimizer="sgdm", alpha=0.01, K=64, D=0.5, device=device)
+    for _ in range(3):
+        fu.pm_update_flat(w, m, None, dl, gr, lp, 32)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(max(args.steps, 1)):
+        fu.pm_update_flat(w, m, None, dl, gr, lp, 32)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / max(args.steps, 1)
+    print(json.dumps({"update_only": {"n_params": n, "P": P, "ms": ms, "GB/s": 30 * n / (ms * 1e-3) / 1e9}}), flush=True)
+
+
 def run_cuda(args):
     import torch
     import pm_inputs as I
@@ -217,12 +261,19 @@ def run_cuda(args):
     torch.cuda.set_device(device)
     hbm_peak, tf_peak, peak_kind = measured_peaks()
     wl = I.cfg3()
+    if args.stages:                      # profiler captures only: fewer stages of the same shape, not a bench result
+        wl = I.mlp_workload(wl.name + f"_first{args.stages}", args.stages, 1024, 2, "gelu", wl.microbatch, compute="bf16",
+                            optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, K=wl.K, D=wl.D, steps=wl.steps,
+                            seed=wl.seed)
     P = wl.n_stages
     params0 = I.init_stage_params(wl)
     pipe = pm.Pipeline(wl, params0, device=str(device))
     host_b, dev_b = make_batches(wl, 4, device)
     n_params = sum(sp.n_in * sp.n_out + sp.n_out for st in wl.stages for sp in st)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     # fill the pipeline (2P-1 ticks) and warm up
     fill = 2 * P - 1
     for s in range(fill + max(args.warmup, 3)):
@@ -230,9 +281,9 @@ def run_cuda(args):
     torch.cuda.synchronize(device)
 
     # ---- timed region 1: K steps, inputs resident in HBM --------------------------------------------
-    sampler = ClockSampler(local)
     if rank == 0:
-        sampler.start()
+        sampler.wait_first()
+        sampler.mark()
     launches0 = pipe.pm_launch_count()
     barrier(world)
     torch.cuda.synchronize(device)
@@ -245,7 +296,6 @@ def run_cuda(args):
     barrier(world)
     elapsed_ms = e0.elapsed_time(e1)
     launches = pipe.pm_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
     t_ms, units = reduce_over_ranks(elapsed_ms, wl.microbatch * args.steps, world, device)
     value = units / (t_ms * 1e-3)
 
@@ -260,6 +310,7 @@ def run_cuda(args):
         pipe.pm_update()
         ev[s][1].record()
     torch.cuda.synchronize(device)
+    clocks = sampler.stop() if rank == 0 else None
     upd_ms = [a.elapsed_time(b) for a, b in ev]
     upd_avg = sum(upd_ms) / len(upd_ms)
     alg_bytes = BYTES_PER_PARAM[wl.optimizer] * n_params
@@ -308,7 +359,8 @@ def run_cuda(args):
                      "share_of_step": round(upd_avg / (t_ms / args.steps), 4)},
     }
     if world == 1:
-        line["cpu_baseline"] = cpu_baseline(wl, 2)
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(wl, 2)
         if not args.no_sweep:
             line["update_sweep"] = update_sweep(device, hbm_peak)
     print(json.dumps(line), flush=True)
@@ -378,8 +430,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the stand-alone update sweep")
+    ap.add_argument("--stages", type=int, default=0, help="profiling runs: same workload cut to this many stages")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
+    ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",
+                    help="run only the stand-alone fused update on N_PARAMS parameters (profiling runs)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.update_only:
+        run_update_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

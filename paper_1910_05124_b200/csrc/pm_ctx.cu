@@ -23,7 +23,7 @@ struct Layout {
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
-  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0;
+  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0;
   int64_t loss_cap = 0;
   int32_t max_lin = 0, max_dim = 0, n_in_first = 0, n_out_last = 0;
 };
@@ -108,6 +108,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_e64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_alpha = w; w = align_up(w + sizeof(double) * (cfg->alpha_by_step ? (uint64_t)cfg->alpha_len : 0), 256);
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
+  L.off_lossred = w; w = align_up(w + 512, 256);
   L.off_tgt = w; w = align_up(w + sizeof(float) * (uint64_t)(P + 1) * T * L.n_out_last, 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * esz, 256);
   L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes(P) : 0), 256);
@@ -249,6 +250,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   }
   e = cudaMemsetAsync(c->ws + L.off_nupd, 0, sizeof(int64_t) * P, c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_dyn, 0, sizeof(StageDyn) * P, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_lossred, 0, 512, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // host tables may go out of scope after this
   if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "context set-up"); delete c; return r; }
 
@@ -264,7 +266,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.dyn = (const StageDyn*)(c->ws + L.off_dyn);
   t.a = c->a; t.ring = (char*)ring; t.ws = c->ws; t.T = cfg->microbatch; t.P = P;
   t.n_in_first = L.n_in_first; t.n_out_last = L.n_out_last;
-  t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap;
+  t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
 
   if (cfg->compute_dtype == PM_BF16) {

@@ -38,9 +38,12 @@ cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, cons
 
 // ---- MSE loss at the last stage ------------------------------------------------------------------
 // loss = mean over T*out of (y - y*)^2 ;  dy = 2 (y - y*) / (T*out), stored in the activation type.
-// One block; fixed summation order (strided per-thread partials, then a fixed tree).
+// Fixed summation order: each block sums a contiguous chunk (strided per-thread partials, fixed tree),
+// the last block to finish adds the per-block partials in block order.
+constexpr int kLossBlocks = 64, kLossThreads = 256;
+
 template <typename AT>
-__global__ void __launch_bounds__(1024) mse_loss_kernel(TickArgs t) {
+__global__ void __launch_bounds__(kLossThreads) mse_loss_kernel(TickArgs t) {
   const StageDyn& d = t.dyn[t.P - 1];
   if (d.b_mb < 0) return;
   const StageDev& sl = t.st[t.P - 1];
@@ -49,58 +52,113 @@ __global__ void __launch_bounds__(1024) mse_loss_kernel(TickArgs t) {
   const AT* y = ws_ptr<AT>(t, t.yout_off) + (uint64_t)par * n;
   const float* tg = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(d.b_mb % (t.P + 1)) * n;
   AT* dy = ws_ptr<AT>(t, sl.gin) + (uint64_t)par * n;
+  float* partial = ws_ptr<float>(t, t.lossred_off);
+  unsigned int* counter = reinterpret_cast<unsigned int*>(partial + kLossBlocks);
   const float scale = (float)(2.0 / (double)n);
+  const uint64_t chunk = (n + gridDim.x - 1) / gridDim.x;
+  const uint64_t lo = (uint64_t)blockIdx.x * chunk, hi = lo + chunk < n ? lo + chunk : n;
   float part = 0.f;
-  for (uint64_t i = threadIdx.x; i < n; i += blockDim.x) {
+  for (uint64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) {
     float r = __fsub_rn(to_f<AT>(y[i]), tg[i]);
     part = __fadd_rn(part, __fmul_rn(r, r));
     dy[i] = from_f<AT>(__fmul_rn(scale, r));
   }
-  __shared__ float red[1024];
+  __shared__ float red[kLossThreads];
+  __shared__ bool last;
   red[threadIdx.x] = part;
   __syncthreads();
-  for (int off = 512; off > 0; off >>= 1) {
+  for (int off = kLossThreads / 2; off > 0; off >>= 1) {
     if ((int)threadIdx.x < off) red[threadIdx.x] = __fadd_rn(red[threadIdx.x], red[threadIdx.x + off]);
     __syncthreads();
   }
-  if (threadIdx.x == 0) ws_ptr<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = red[0] / (float)n;
+  if (threadIdx.x == 0) {
+    partial[blockIdx.x] = red[0];
+    __threadfence();
+    last = atomicAdd(counter, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (last && threadIdx.x == 0) {
+    __threadfence();
+    float sum = 0.f;
+    for (int b = 0; b < (int)gridDim.x; ++b) sum = __fadd_rn(sum, reinterpret_cast<volatile float*>(partial)[b]);
+    ws_ptr<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = sum / (float)n;
+    *counter = 0;                                     // ready for the next tick
+  }
 }
 
 cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream) {
-  if (dtype == PM_F32) mse_loss_kernel<float><<<1, 1024, 0, stream>>>(t);
-  else mse_loss_kernel<__nv_bfloat16><<<1, 1024, 0, stream>>>(t);
+  if (dtype == PM_F32) mse_loss_kernel<float><<<kLossBlocks, kLossThreads, 0, stream>>>(t);
+  else mse_loss_kernel<__nv_bfloat16><<<kLossBlocks, kLossThreads, 0, stream>>>(t);
   return cudaGetLastError();
 }
 
 // ---- activation backward + bias gradient ---------------------------------------------------------
-// dz = dy * act'(z) (stored in the activation type); db[c] = sum over rows of the stored dz, rows ascending.
+// dz = dy * act'(z) (stored in the activation type); db[c] = sum over rows of the stored dz.
+// A block owns 64 columns; warp w takes rows w, w+8, ... (ascending), two columns per thread; the eight
+// per-warp partial sums of a column are added in warp order.
+constexpr int kActCols = 64, kActWarps = 8;
+
+template <typename AT> struct Pair;
+template <> struct Pair<float> {
+  static __device__ __forceinline__ float2 ld(const float* p) { return *reinterpret_cast<const float2*>(p); }
+  static __device__ __forceinline__ void st(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
+};
+template <> struct Pair<__nv_bfloat16> {
+  static __device__ __forceinline__ float2 ld(const __nv_bfloat16* p) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p)); }
+  static __device__ __forceinline__ void st(__nv_bfloat16* p, float2 v) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v.x, v.y); }
+};
+
 template <typename AT>
-__global__ void __launch_bounds__(128) actbwd_kernel(TickArgs t, int lvl) {
+__global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
   const int p = blockIdx.y;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= L.n_out) return;
+  const int c0 = blockIdx.x * kActCols;
+  if (c0 >= L.n_out) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c = c0 + 2 * lane;                        // n_out is even whenever a pair straddles nothing: see guard
   const uint64_t n = (uint64_t)t.T * L.n_out;
   const AT* dy = (lvl == s.n_lin - 1) ? ws_ptr<AT>(t, s.gin) + (uint64_t)((d.tick + 1) & 1) * n : ws_ptr<AT>(t, s.dh);
   const AT* z = ring_ptr<AT>(t, L.z_ring, d.b_slot, n);
   AT* dz = ws_ptr<AT>(t, s.dz);
-  float sum = 0.f;
-  for (int r = 0; r < t.T; ++r) {
-    uint64_t i = (uint64_t)r * L.n_out + c;
-    AT v = from_f<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act)));
-    dz[i] = v;
-    sum = __fadd_rn(sum, to_f<AT>(v));
+  const bool pair_ok = (L.n_out & 1) == 0;            // vector path needs even row length for alignment
+  float s0 = 0.f, s1 = 0.f;
+  for (int r = warp; r < t.T; r += kActWarps) {
+    const uint64_t i = (uint64_t)r * L.n_out + c;
+    if (pair_ok && c + 1 < L.n_out) {
+      float2 g = Pair<AT>::ld(dy + i), zz = Pair<AT>::ld(z + i);
+      float2 v = make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act))));
+      Pair<AT>::st(dz + i, v);
+      s0 = __fadd_rn(s0, v.x); s1 = __fadd_rn(s1, v.y);
+    } else {
+      if (c < L.n_out) {
+        float v = round_as<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act)));
+        dz[i] = from_f<AT>(v); s0 = __fadd_rn(s0, v);
+      }
+      if (c + 1 < L.n_out) {
+        float v = round_as<AT>(__fmul_rn(to_f<AT>(dy[i + 1]), act_grad(to_f<AT>(z[i + 1]), L.act)));
+        dz[i + 1] = from_f<AT>(v); s1 = __fadd_rn(s1, v);
+      }
+    }
   }
-  t.a.grad[L.b_off + c] = sum;
+  __shared__ float red[kActWarps][kActCols];
+  red[warp][2 * lane] = s0;
+  red[warp][2 * lane + 1] = s1;
+  __syncthreads();
+  if (threadIdx.x < kActCols && c0 + (int)threadIdx.x < L.n_out) {
+    float sum = 0.f;
+#pragma unroll
+    for (int w = 0; w < kActWarps; ++w) sum = __fadd_rn(sum, red[w][threadIdx.x]);
+    t.a.grad[L.b_off + c0 + threadIdx.x] = sum;
+  }
 }
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
-  dim3 grid((t.max_dim + 127) / 128, t.P);
-  if (dtype == PM_F32) actbwd_kernel<float><<<grid, 128, 0, stream>>>(t, lvl);
-  else actbwd_kernel<__nv_bfloat16><<<grid, 128, 0, stream>>>(t, lvl);
+  dim3 grid((t.max_dim + kActCols - 1) / kActCols, t.P);
+  if (dtype == PM_F32) actbwd_kernel<float><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
+  else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   return cudaGetLastError();
 }
 

@@ -16,6 +16,7 @@ struct TickArgs {
   uint64_t yout_off;      // ws: last stage's output [2][T*n_out_last] (activation type)
   uint64_t tgt_off;       // ws: target ring [P+1][T*n_out_last] float
   uint64_t loss_off;      // ws: loss log [loss_cap] float
+  uint64_t lossred_off;   // ws: per-block loss partials [64] float + completion counter
   int64_t loss_cap;
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages
