@@ -1,20 +1,22 @@
 // bf16 grouped GEMMs of the pipeline on the 5th-generation tensor cores.
 //
-// One CTA computes one 128x128 output tile of one stage; blockIdx.z selects the stage, so a single
-// launch covers every stage that is active in this tick.  Operands are staged in shared memory in the
-// 128-byte-swizzled canonical layouts (TMA writes them; for dgrad a transform step writes B), the
-// accumulator lives in tensor memory (128 lanes x 128 fp32 columns), one elected thread issues
-// tcgen05.mma, and four warps drain the accumulator with tcgen05.ld for the epilogue.
+// One launch covers every stage that is active in this tick.  The kernel is persistent: one CTA per SM
+// walks a flattened list of 128x128 output tiles (stage, row tile, column tile).  Operands are staged in
+// shared memory in the 128-byte-swizzled canonical layouts, the accumulators live in tensor memory
+// (two buffers of 128 lanes x 128 fp32 columns, so the epilogue of one tile overlaps the main loop of
+// the next), one elected thread issues tcgen05.mma, and eight warps drain the accumulators with
+// tcgen05.ld.
 //
 //   mode 0 forward  D[T,out]  = x[T,in] * W[out,in]^T      A K-major (TMA), B K-major (TMA, bf16 shadow)
 //                   z = bf16(D + b) -> ring,  y = bf16(act(z)) -> next consumer
-//   mode 1 dgrad    D[T,in]   = dz[T,out] * Wc[out,in]     A K-major (TMA), B MN-major, written by the
-//                   transform warps as bf16(w - gap*delta) from the fp32 master arenas (T2 of
-//                   Section 3.2): the corrected weights exist only in shared memory
+//   mode 1 dgrad    D[T,in]   = dz[T,out] * Wc[out,in]     A K-major (TMA); the fp32 master weights and the
+//                   T2 accumulator delta arrive by TMA in a staging ring, four transform warps turn them
+//                   into the MN-major bf16 operand bf16(w - gap*delta) (Section 3.2): the corrected
+//                   weights exist only in shared memory
 //   mode 2 wgrad    D[out,in] = dz[T,out]^T * x[T,in]      A MN-major (TMA), B MN-major (TMA), fp32 out
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
-// warps 2..5 = (mode 1: operand transform, then) epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, (mode 1: warps 2..5 = operand
+// transform,) last eight warps = epilogue (two per TMEM lane group, each taking 64 of the 128 columns).
 // Every wait on an mbarrier is bounded; on expiry the CTA records a code in a status word, stops
 // issuing work, waits (bounded) for its copies in flight, frees its tensor memory and returns.
 #include <cuda.h>
@@ -24,16 +26,25 @@
 namespace pm {
 
 constexpr int TILE_M = 128, TILE_N = 128, TILE_K = 64;     // bf16: 64 elements = one 128-byte swizzle row
-constexpr int N_STAGES = 3;
 constexpr int A_BYTES = TILE_M * TILE_K * 2;               // 16 KB
 constexpr int B_BYTES = TILE_N * TILE_K * 2;               // 16 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int TMEM_COLS = 128;
-constexpr int SMEM_BYTES = N_STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int N_THREADS = 192;
+constexpr int STG_HALF_BYTES = TILE_K * TILE_N * 4;        // one fp32 [64 x 128] tile: 32 KB
+constexpr int STG_BYTES = 2 * STG_HALF_BYTES;              // w tile + delta tile
+constexpr int ACC_COLS = 128, TMEM_COLS = 2 * ACC_COLS;
+constexpr int N_EPI_WARPS = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;      // about one second
 
-enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAPS_PER_LINEAR = 5 };
+template <int MODE> struct Cfg {
+  static constexpr int kTransformWarps = MODE == 1 ? 4 : 0;
+  static constexpr int kStages = MODE == 1 ? 2 : 6;        // operand ring depth
+  static constexpr int kStaging = MODE == 1 ? 2 : 0;       // fp32 staging ring depth (dgrad only)
+  static constexpr int kThreads = 32 * (2 + kTransformWarps + N_EPI_WARPS);
+  static constexpr int kTileBytes = kStages * STAGE_BYTES + kStaging * STG_BYTES;
+  static constexpr int kSmemBytes = kTileBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+};
+
+enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6, MAPS_PER_LINEAR = 7 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -142,41 +153,61 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// ---- tile walk ---------------------------------------------------------------------------------------
+// tile_start[p] .. tile_start[p+1] are the flattened tile ids of stage p for this (mode, level).
+struct Tile { int p, m0, n0, M, N, K, n_kb; bool valid; };
+
+template <int MODE>
+__device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
+  Tile r;
+  int lo = 0, hi = t.P - 1;                                            // largest p with tile_start[p] <= tile
+  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  r.p = lo;
+  const StageDyn& d = t.dyn[lo];
+  const StageDev& s = t.st[lo];
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0);
+  const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
+  if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
+  else if (MODE == 1) { r.M = t.T; r.N = L.n_in; r.K = L.n_out; }
+  else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
+  const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
+  const int local = tile - tile_start[lo];
+  r.m0 = (local / tiles_n) * TILE_M;
+  r.n0 = (local % tiles_n) * TILE_N;
+  r.n_kb = (r.K + TILE_K - 1) / TILE_K;
+  return r;
+}
+
+struct Ring {                       // position in a ring of mbarrier-guarded slots
+  int idx; uint32_t phase;
+  __device__ __forceinline__ void advance(int n) { if (++idx == n) { idx = 0; phase ^= 1u; } }
+};
+
 // ---- the kernel --------------------------------------------------------------------------------------
 template <int MODE>
-__global__ void __launch_bounds__(N_THREADS) umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int lvl, int* status) {
-  const int p = blockIdx.z;
-  const StageDyn& d = t.dyn[p];
-  const StageDev& s = t.st[p];
-  if (lvl >= s.n_lin) return;
-  if (MODE == 0 ? d.f_mb < 0 : d.b_mb < 0) return;
-  if (MODE == 1 && p == 0 && lvl == 0) return;          // the network input needs no gradient
-  const LinDev& L = s.lin[lvl];
-  int M, N, K;
-  if (MODE == 0) { M = t.T; N = L.n_out; K = L.n_in; }
-  else if (MODE == 1) { M = t.T; N = L.n_in; K = L.n_out; }
-  else { M = L.n_out; N = L.n_in; K = t.T; }
-  const int m0 = blockIdx.y * TILE_M, n0 = blockIdx.x * TILE_N;
-  if (m0 >= M || n0 >= N) return;
-  const int n_kb = (K + TILE_K - 1) / TILE_K;
-
+__global__ void __launch_bounds__(Cfg<MODE>::kThreads, 1)
+umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, int n_tiles, int lvl, int* status) {
+  using C = Cfg<MODE>;
+  constexpr int NS = C::kStages, NG = C::kStaging, NT = C::kTransformWarps;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
   uint8_t* tiles_ptr = smem_raw + (tiles - raw);
-  const uint32_t bars = tiles + N_STAGES * STAGE_BYTES;
-  // barrier block: full[N_STAGES], empty[N_STAGES], tmem_full, then tmem base word and abort flag
-  const uint32_t bar_full = bars, bar_empty = bars + 8 * N_STAGES, bar_tmem = bars + 16 * N_STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + N_STAGES * STAGE_BYTES + 16 * N_STAGES + 8);
+  const uint32_t stg = tiles + NS * STAGE_BYTES;                      // fp32 staging ring (dgrad)
+  uint8_t* stg_ptr = tiles_ptr + NS * STAGE_BYTES;
+  const uint32_t bars = tiles + C::kTileBytes;
+  // barrier block: full[NS] empty[NS] sfull[NG] sempty[NG] tfull[2] tempty[2], then tmem base word and abort flag
+  const uint32_t bar_full = bars, bar_empty = bar_full + 8 * NS, bar_sfull = bar_empty + 8 * NS,
+                 bar_sempty = bar_sfull + 8 * NG, bar_tfull = bar_sempty + 8 * NG, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + C::kTileBytes + 8 * (2 * NS + 2 * NG + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const CUtensorMap* lm = maps + ((size_t)p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
 
   if (threadIdx.x == 0) {
-    const uint32_t full_count = MODE == 1 ? 1 + 4 : 1;               // TMA thread (+ one arrival per transform warp)
-    for (int i = 0; i < N_STAGES; ++i) { mbar_init(bar_full + 8 * i, full_count); mbar_init(bar_empty + 8 * i, 1); }
-    mbar_init(bar_tmem, 1);
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, MODE == 1 ? 1 + NT : 1); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, NT); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, N_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -193,35 +224,56 @@ __global__ void __launch_bounds__(N_THREADS) umma_gemm_kernel(TickArgs t, const 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < n_kb; ++kb) {
-        const int st = kb % N_STAGES;
-        const uint32_t ph = (kb / N_STAGES) & 1;
-        if (*abort_flag || !mbar_wait(bar_empty + 8 * st, ph ^ 1, abort_flag, status, 1)) break;
-        const uint32_t sa = tiles + st * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * st;
-        const int k0 = kb * TILE_K;
-        if (MODE == 0) {
-          mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-          tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, m0, lvl == 0 ? d.f_xslot : d.f_slot);
-          tma_load_2d(sb, lm + MAP_W_K, fb, k0, n0);
-        } else if (MODE == 1) {
-          mbar_arrive_expect_tx(fb, A_BYTES);
-          tma_load_2d(sa, lm + MAP_DZ_K, fb, k0, m0);
-        } else {
-          mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-          const int slot = lvl == 0 ? d.b_xslot : d.b_slot;
-          tma_load_2d(sa, lm + MAP_DZ_MN, fb, m0, k0);
-          tma_load_2d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, m0 + 64, k0);
-          tma_load_3d(sb, lm + MAP_ACT_MN, fb, n0, k0, slot);
-          tma_load_3d(sb + B_BYTES / 2, lm + MAP_ACT_MN, fb, n0 + 64, k0, slot);
+      Ring op{0, 0}, sg{0, 0};
+      int issued_op = 0, issued_sg = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        const StageDyn& d = t.dyn[tl.p];
+        const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        for (int kb = 0; kb < tl.n_kb; ++kb) {
+          const int k0 = kb * TILE_K;
+          if (MODE == 1) {
+            if (*abort_flag || !mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 5)) { ok = false; break; }
+            const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+            const bool corr = d.use_delta != 0;
+            mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
+            tma_load_2d(sw, lm + MAP_W_F32, fb, tl.n0, k0);
+            if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, tl.n0, k0);
+            sg.advance(NG); ++issued_sg;
+          }
+          if (*abort_flag || !mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 1)) { ok = false; break; }
+          const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * op.idx;
+          if (MODE == 0) {
+            mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+            tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, lvl == 0 ? d.f_xslot : d.f_slot);
+            tma_load_2d(sb, lm + MAP_W_K, fb, k0, tl.n0);
+          } else if (MODE == 1) {
+            mbar_arrive_expect_tx(fb, A_BYTES);
+            tma_load_2d(sa, lm + MAP_DZ_K, fb, k0, tl.m0);
+          } else {
+            mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+            const int slot = lvl == 0 ? d.b_xslot : d.b_slot;
+            tma_load_2d(sa, lm + MAP_DZ_MN, fb, tl.m0, k0);
+            tma_load_2d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, tl.m0 + 64, k0);
+            tma_load_3d(sb, lm + MAP_ACT_MN, fb, tl.n0, k0, slot);
+            tma_load_3d(sb + B_BYTES / 2, lm + MAP_ACT_MN, fb, tl.n0 + 64, k0, slot);
+          }
+          op.advance(NS); ++issued_op;
         }
-        issued = kb + 1;
       }
       if (*abort_flag) {
         // copies already issued still land in this CTA's shared memory: wait for them (bounded) before leaving
-        for (int kb = issued > N_STAGES ? issued - N_STAGES : 0; kb < issued; ++kb) {
+        for (int back = 1; back <= NS && back <= issued_op; ++back) {
+          const int it = issued_op - back;
           const long long t0 = clock64();
-          while (!mbar_try_wait(bar_full + 8 * (kb % N_STAGES), (kb / N_STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+          while (!mbar_try_wait(bar_full + 8 * (it % NS), (uint32_t)(it / NS) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+        for (int back = 1; back <= NG && back <= issued_sg; ++back) {
+          const int it = issued_sg - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_sfull + 8 * (it % (NG > 0 ? NG : 1)), (uint32_t)(it / (NG > 0 ? NG : 1)) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
       }
     }
@@ -229,138 +281,153 @@ __global__ void __launch_bounds__(N_THREADS) umma_gemm_kernel(TickArgs t, const 
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = make_idesc(MODE == 2, MODE != 0);
+      Ring op{0, 0}, acc{0, 0};
       bool ok = true;
-      for (int kb = 0; kb < n_kb && ok; ++kb) {
-        const int st = kb % N_STAGES;
-        const uint32_t ph = (kb / N_STAGES) & 1;
-        if (*abort_flag || !mbar_wait(bar_full + 8 * st, ph, abort_flag, status, 2)) { ok = false; break; }
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        if (*abort_flag || !mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 6)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = tiles + st * STAGE_BYTES, sb = sa + A_BYTES;
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * ACC_COLS);
+        for (int kb = 0; kb < tl.n_kb; ++kb) {
+          if (*abort_flag || !mbar_wait(bar_full + 8 * op.idx, op.phase, abort_flag, status, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
-        for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
-          // K-major: 16 elements = 32 bytes along the swizzled row.  MN-major: 16 k-rows of 128 bytes.
-          const uint64_t da = MODE == 2 ? make_desc(sa + k16 * 2048, A_BYTES / 2, 1024) : make_desc(sa + k16 * 32, 16, 1024);
-          const uint64_t db = MODE == 0 ? make_desc(sb + k16 * 32, 16, 1024) : make_desc(sb + k16 * 2048, B_BYTES / 2, 1024);
-          tc_mma_bf16(tmem_base, da, db, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
+            // K-major: 16 elements = 32 bytes along the swizzled row.  MN-major: 16 k-rows of 128 bytes.
+            const uint64_t da = MODE == 2 ? make_desc(sa + k16 * 2048, A_BYTES / 2, 1024) : make_desc(sa + k16 * 32, 16, 1024);
+            const uint64_t db = MODE == 0 ? make_desc(sb + k16 * 32, 16, 1024) : make_desc(sb + k16 * 2048, B_BYTES / 2, 1024);
+            tc_mma_bf16(tmem_acc, da, db, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          }
+          tc_commit(bar_empty + 8 * op.idx);      // frees the operand slot once these MMAs have read it
+          op.advance(NS);
         }
-        tc_commit(bar_empty + 8 * st);        // frees the stage once these MMAs have read it
+        if (ok) tc_commit(bar_tfull + 8 * acc.idx);   // accumulator complete
+        acc.advance(2);
       }
-      if (ok) tc_commit(bar_tmem);            // accumulator complete
     }
-  } else {
-    // ---------------- warps 2..5: transform (dgrad) then epilogue ----------------
-    const int q = warp & 3;                                           // TMEM lane group this warp may read
+  } else if (warp < 2 + NT) {
+    // ---------------- operand transform (dgrad): fp32 w, delta in staging -> bf16(w - gap*delta), MN-major ----------------
     if (MODE == 1) {
       const int tt = threadIdx.x - 64;                                // 0..127
-      const int c = tt & 15, rb = tt >> 4;                            // 16-byte chunk (8 columns) and row within 8-row group
-      const int n = n0 + c * 8;
-      const float gapf = (float)s.gap;
-      const bool corr = d.use_delta != 0;
-      const float* wm = t.a.w + L.w_off;
-      const float* dl = t.a.delta + L.w_off;
+      const int c = tt & 15, rb = tt >> 4;                            // 8-column chunk and row within each 8-row group
       const uint32_t dst_in_tile = (uint32_t)(c >> 3) * (B_BYTES / 2) + (uint32_t)rb * 128 + (uint32_t)(((c & 7) ^ rb) << 4);
-      for (int kb = 0; kb < n_kb; ++kb) {
-        const int st = kb % N_STAGES;
-        const uint32_t ph = (kb / N_STAGES) & 1;
-        bool go = !*abort_flag && mbar_wait(bar_empty + 8 * st, ph ^ 1, abort_flag, status, 3);
-        go = __all_sync(0xffffffffu, go);                             // leave the loop as a whole warp
-        if (!go) break;
-        float4 w0[8], w1[8], d0[8], d1[8];
+      const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
+      Ring op{0, 0}, sg{0, 0};
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        const float gapf = (float)t.st[tl.p].gap;
+        const bool corr = t.dyn[tl.p].use_delta != 0;
+        for (int kb = 0; kb < tl.n_kb; ++kb) {
+          bool go = !*abort_flag && mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 7);
+          go = go && mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 3);
+          go = __all_sync(0xffffffffu, go);                           // leave the loops as a whole warp
+          if (!go) { ok = false; break; }
+          const uint8_t* src = stg_ptr + sg.idx * STG_BYTES + src_in_tile;
+          uint8_t* dst = tiles_ptr + op.idx * STAGE_BYTES + A_BYTES + dst_in_tile;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int k = kb * TILE_K + rb + 8 * j;
-          if (k < K && n < N) {
-            const size_t idx = (size_t)k * L.n_in + n;
-            w0[j] = *reinterpret_cast<const float4*>(wm + idx);
-            w1[j] = *reinterpret_cast<const float4*>(wm + idx + 4);
+          for (int j = 0; j < 8; ++j) {
+            const float4 w0 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4);
+            const float4 w1 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4 + 16);
+            float v[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
             if (corr) {
-              d0[j] = *reinterpret_cast<const float4*>(dl + idx);
-              d1[j] = *reinterpret_cast<const float4*>(dl + idx + 4);
-            } else {
-              d0[j] = make_float4(0.f, 0.f, 0.f, 0.f); d1[j] = d0[j];
+              const float4 d0 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4);
+              const float4 d1 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4 + 16);
+              const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = __fsub_rn(v[e], __fmul_rn(gapf, dd[e]));   // w - (tau_fwd - tau_bkwd) * delta
             }
-          } else {
-            w0[j] = make_float4(0.f, 0.f, 0.f, 0.f); w1[j] = w0[j]; d0[j] = w0[j]; d1[j] = w0[j];
+            *reinterpret_cast<uint4*>(dst + j * 1024) =
+                make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
           }
+          fence_async_smem();                                         // generic-proxy stores -> visible to the tensor core
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(bar_full + 8 * op.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
+          op.advance(NS); sg.advance(NG > 0 ? NG : 1);
         }
-        uint8_t* sb = tiles_ptr + st * STAGE_BYTES + A_BYTES;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          float v[8] = {w0[j].x, w0[j].y, w0[j].z, w0[j].w, w1[j].x, w1[j].y, w1[j].z, w1[j].w};
-          if (corr) {
-            const float dd[8] = {d0[j].x, d0[j].y, d0[j].z, d0[j].w, d1[j].x, d1[j].y, d1[j].z, d1[j].w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = __fsub_rn(v[e], __fmul_rn(gapf, dd[e]));   // w - (tau_fwd - tau_bkwd) * delta
-          }
-          uint4 pk = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-          *reinterpret_cast<uint4*>(sb + dst_in_tile + j * 1024) = pk;
-        }
-        fence_async_smem();                                           // make the generic-proxy stores visible to the tensor core
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_full + 8 * st);
       }
     }
-    // epilogue
-    bool acc_ready = !*abort_flag && mbar_wait(bar_tmem, 0, abort_flag, status, 4);
-    acc_ready = __all_sync(0xffffffffu, acc_ready);                   // tcgen05.ld needs the whole warp
-    if (acc_ready) {
+  } else {
+    // ---------------- epilogue: 8 warps, warp%4 = TMEM lane group, two warps per group split the columns ----------------
+    const int q = warp & 3;
+    const int half = (warp - 2 - NT) >> 2;                            // 0: columns 0..63, 1: columns 64..127
+    Ring acc{0, 0};
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const StageDyn& d = t.dyn[tl.p];
+      const StageDev& s = t.st[tl.p];
+      const LinDev& L = s.lin[lvl];
+      const int m = tl.m0 + q * 32 + lane;
+      const int nb = tl.n0 + half * 64;
+      bool ready = !*abort_flag && mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
+      ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
+      if (!ready) { ok = false; break; }
       tc_fence_after();
-      const int m = m0 + q * 32 + lane;
-#pragma unroll 1
-      for (int cc = 0; cc < TILE_N / 32; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r);
-        tmem_ld_wait();
-        const int nb = n0 + cc * 32;
-        if (m < M) {
-          if (MODE == 0) {
-            const size_t n_out_elems = (size_t)t.T * L.n_out;
-            __nv_bfloat16* zout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.z_ring) + (size_t)d.f_slot * n_out_elems;
-            __nv_bfloat16* yout;
-            if (lvl < s.n_lin - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.h_ring) + (size_t)d.f_slot * n_out_elems;
-            else if (p < t.P - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[p + 1].x_ring) + (size_t)d.f_next_xslot * n_out_elems;
-            else yout = reinterpret_cast<__nv_bfloat16*>(t.ws + t.yout_off) + (size_t)(d.tick & 1) * n_out_elems;
-            const float* bias = t.a.w + L.b_off;
+      uint32_t r0[32], r1[32];
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * ACC_COLS + half * 64);
+      tmem_ld32(taddr, r0);
+      tmem_ld32(taddr + 32, r1);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc.idx);           // the accumulator buffer may be overwritten now
+      acc.advance(2);
+      if (m >= tl.M) continue;
+      const int N = tl.N;
+      if (MODE == 0) {
+        const size_t n_out_elems = (size_t)t.T * L.n_out;
+        __nv_bfloat16* zout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.z_ring) + (size_t)d.f_slot * n_out_elems;
+        __nv_bfloat16* yout;
+        if (lvl < s.n_lin - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.h_ring) + (size_t)d.f_slot * n_out_elems;
+        else if (tl.p < t.P - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[tl.p + 1].x_ring) + (size_t)d.f_next_xslot * n_out_elems;
+        else yout = reinterpret_cast<__nv_bfloat16*>(t.ws + t.yout_off) + (size_t)(d.tick & 1) * n_out_elems;
+        const float* bias = t.a.w + L.b_off;
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const int n = nb + g * 8;
-              if (n < N) {
-                const float4 b0 = *reinterpret_cast<const float4*>(bias + n), b1 = *reinterpret_cast<const float4*>(bias + n + 4);
-                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                float zf[8], yf[8];
+        for (int g = 0; g < 8; ++g) {
+          const int n = nb + g * 8;
+          if (n < N) {
+            const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
+            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+            float zf[8], yf[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(r[g * 8 + e]), bb[e])));
-                  yf[e] = act_fwd(zf[e], L.act);
-                }
-                const size_t o = (size_t)m * N + n;
-                *reinterpret_cast<uint4*>(zout + o) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
-                *reinterpret_cast<uint4*>(yout + o) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
-              }
+            for (int e = 0; e < 8; ++e) {
+              const uint32_t a = g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e];
+              zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(a), bb[e])));
+              yf[e] = act_fwd(zf[e], L.act);
             }
-          } else if (MODE == 1) {
-            const size_t n_in_elems = (size_t)t.T * L.n_in;
-            __nv_bfloat16* dx = (lvl == 0) ? reinterpret_cast<__nv_bfloat16*>(t.ws + t.st[p - 1].gin) + (size_t)(d.tick & 1) * n_in_elems
-                                           : reinterpret_cast<__nv_bfloat16*>(t.ws + s.dh);
+            const size_t o = (size_t)m * N + n;
+            *reinterpret_cast<uint4*>(zout + o) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
+            *reinterpret_cast<uint4*>(yout + o) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
+          }
+        }
+      } else if (MODE == 1) {
+        const size_t n_in_elems = (size_t)t.T * L.n_in;
+        __nv_bfloat16* dx = (lvl == 0) ? reinterpret_cast<__nv_bfloat16*>(t.ws + t.st[tl.p - 1].gin) + (size_t)(d.tick & 1) * n_in_elems
+                                       : reinterpret_cast<__nv_bfloat16*>(t.ws + s.dh);
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const int n = nb + g * 8;
-              if (n < N) {
-                float f[8];
+        for (int g = 0; g < 8; ++g) {
+          const int n = nb + g * 8;
+          if (n < N) {
+            float f[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[g * 8 + e]);
-                *reinterpret_cast<uint4*>(dx + (size_t)m * N + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-              }
-            }
-          } else {
-            float* dW = t.a.grad + L.w_off;
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+            *reinterpret_cast<uint4*>(dx + (size_t)m * N + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+          }
+        }
+      } else {
+        float* dW = t.a.grad + L.w_off;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              const int n = nb + g * 4;
-              if (n < N)
-                *reinterpret_cast<float4*>(dW + (size_t)m * N + n) =
-                    make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
-            }
+        for (int g = 0; g < 16; ++g) {
+          const int n = nb + g * 4;
+          if (n < N) {
+            const uint32_t* rr = g < 8 ? r0 + (g & 7) * 4 : r1 + (g & 7) * 4;
+            *reinterpret_cast<float4*>(dW + (size_t)m * N + n) =
+                make_float4(__uint_as_float(rr[0]), __uint_as_float(rr[1]), __uint_as_float(rr[2]), __uint_as_float(rr[3]));
           }
         }
       }
@@ -383,20 +450,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct UmmaPlan {
   const CUtensorMap* d_maps = nullptr;
+  const int* d_tile_start = nullptr;     // [3 modes][PM_MAX_LINEARS][P+1]
   int* d_status = nullptr;
+  int n_tiles[3][PM_MAX_LINEARS] = {};
+  int P = 0, sms = 148;
 };
 
-uint64_t umma_workspace_bytes(int n_stages) {
-  return (uint64_t)n_stages * PM_MAX_LINEARS * MAPS_PER_LINEAR * sizeof(CUtensorMap) + 256;
-}
+static uint64_t maps_bytes(int P) { return (uint64_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR * sizeof(CUtensorMap); }
+static uint64_t tiles_bytes(int P) { return ((uint64_t)3 * PM_MAX_LINEARS * (P + 1) * sizeof(int) + 255) / 256 * 256; }
 
-static bool encode(EncodeTiledFn fn, CUtensorMap* m, void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                   const uint32_t* box, std::string& err) {
+uint64_t umma_workspace_bytes(int n_stages) { return 256 + maps_bytes(n_stages) + tiles_bytes(n_stages); }
+
+static bool encode(EncodeTiledFn fn, CUtensorMap* m, bool f32, void* base, int rank, const uint64_t* dims,
+                   const uint64_t* strides_bytes, const uint32_t* box, std::string& err) {
   cuuint64_t gd[3]; cuuint64_t gs[2]; cuuint32_t bx[3]; cuuint32_t es[3] = {1, 1, 1};
   for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return false; }
   return true;
 }
@@ -411,6 +483,9 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   const int P = t.P;
   std::vector<CUtensorMap> maps((size_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR);
   memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+  std::vector<int> tile_start((size_t)3 * PM_MAX_LINEARS * (P + 1), 0);
+  UmmaPlan* plan = new UmmaPlan();
+  plan->P = P;
   const uint64_t T = (uint64_t)t.T;
   for (int p = 0; p < P; ++p) {
     const StageDev& s = st[p];
@@ -421,38 +496,61 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       char* act_base = t.ring + (l == 0 ? s.x_ring : s.lin[l - 1].h_ring);
       const uint64_t slots = l == 0 ? (uint64_t)s.xdepth : (uint64_t)s.depth;
       const uint64_t n_in = (uint64_t)L.n_in, n_out = (uint64_t)L.n_out;
+      bool okm = true;
       {
         uint64_t dims[3] = {n_in, T, slots}, strides[2] = {n_in * 2, T * n_in * 2};
         uint32_t box_k[3] = {TILE_K, TILE_M, 1}, box_mn[3] = {64, TILE_K, 1};
-        if (!encode(fn, m + MAP_ACT_K, act_base, 3, dims, strides, box_k, err)) return PM_ERR_CUDA;
-        if (!encode(fn, m + MAP_ACT_MN, act_base, 3, dims, strides, box_mn, err)) return PM_ERR_CUDA;
+        okm = okm && encode(fn, m + MAP_ACT_K, false, act_base, 3, dims, strides, box_k, err);
+        okm = okm && encode(fn, m + MAP_ACT_MN, false, act_base, 3, dims, strides, box_mn, err);
       }
       {
-        uint64_t dims[2] = {n_in, n_out}, strides[1] = {n_in * 2};
-        uint32_t box[2] = {TILE_K, TILE_N};
-        if (!encode(fn, m + MAP_W_K, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err)) return PM_ERR_CUDA;
+        uint64_t dims[2] = {n_in, n_out}, strides[1] = {n_in * 2}, strides4[1] = {n_in * 4};
+        uint32_t box[2] = {TILE_K, TILE_N}, box4[2] = {TILE_N, TILE_K};
+        okm = okm && encode(fn, m + MAP_W_K, false, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err);
+        okm = okm && encode(fn, m + MAP_W_F32, true, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
+        okm = okm && encode(fn, m + MAP_D_F32, true, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
       }
       {
         uint64_t dims[2] = {n_out, T}, strides[1] = {n_out * 2};
         uint32_t box_k[2] = {TILE_K, TILE_M}, box_mn[2] = {64, TILE_K};
-        if (!encode(fn, m + MAP_DZ_K, t.ws + s.dz, 2, dims, strides, box_k, err)) return PM_ERR_CUDA;
-        if (!encode(fn, m + MAP_DZ_MN, t.ws + s.dz, 2, dims, strides, box_mn, err)) return PM_ERR_CUDA;
+        okm = okm && encode(fn, m + MAP_DZ_K, false, t.ws + s.dz, 2, dims, strides, box_k, err);
+        okm = okm && encode(fn, m + MAP_DZ_MN, false, t.ws + s.dz, 2, dims, strides, box_mn, err);
       }
+      if (!okm) { delete plan; return PM_ERR_CUDA; }
     }
   }
+  auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
+  for (int mode = 0; mode < 3; ++mode)
+    for (int l = 0; l < PM_MAX_LINEARS; ++l) {
+      int* ts = tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
+      int acc = 0;
+      for (int p = 0; p < P; ++p) {
+        ts[p] = acc;
+        if (l < st[p].n_lin) {
+          const LinDev& L = st[p].lin[l];
+          const int M = mode == 2 ? L.n_out : t.T, N = mode == 0 ? L.n_out : L.n_in;
+          acc += cdiv(M, TILE_M) * cdiv(N, TILE_N);
+        }
+      }
+      ts[P] = acc;
+      plan->n_tiles[mode][l] = acc;
+    }
   char* region = (char*)ws_region;
-  cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream);
+  cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps_bytes(P), cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(region + 256 + maps_bytes(P), tile_start.data(), tile_start.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-  if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); return PM_ERR_CUDA; }
-  for (int mode = 0; mode < 3; ++mode) {
-    const void* f = mode == 0 ? (const void*)umma_gemm_kernel<0> : mode == 1 ? (const void*)umma_gemm_kernel<1> : (const void*)umma_gemm_kernel<2>;
-    e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return PM_ERR_CUDA; }
-  }
-  UmmaPlan* plan = new UmmaPlan();
+  if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
+  e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<0>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
+  if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&plan->sms, cudaDevAttrMultiProcessorCount, dev);
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
+  plan->d_tile_start = (const int*)(region + 256 + maps_bytes(P));
   *out = plan;
   return PM_OK;
 }
@@ -462,11 +560,13 @@ void umma_plan_destroy(UmmaPlan* plan) { delete plan; }
 int* umma_status_word(UmmaPlan* plan) { return plan ? plan->d_status : nullptr; }
 
 cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
-  const int max_m = mode == 2 ? t.max_dim : t.T;
-  dim3 grid((t.max_dim + TILE_N - 1) / TILE_N, (max_m + TILE_M - 1) / TILE_M, t.P);
-  if (mode == 0) umma_gemm_kernel<0><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
-  else if (mode == 1) umma_gemm_kernel<1><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
-  else umma_gemm_kernel<2><<<grid, N_THREADS, SMEM_BYTES, stream>>>(t, plan->d_maps, lvl, plan->d_status);
+  const int n_tiles = plan->n_tiles[mode][lvl];
+  if (n_tiles == 0) return cudaSuccess;
+  const int grid = n_tiles < plan->sms ? n_tiles : plan->sms;      // one persistent CTA per SM
+  const int* ts = plan->d_tile_start + ((size_t)mode * PM_MAX_LINEARS + lvl) * (plan->P + 1);
+  if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
+  else if (mode == 1) umma_gemm_kernel<1><<<grid, Cfg<1>::kThreads, Cfg<1>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
+  else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
   return cudaGetLastError();
 }
 
