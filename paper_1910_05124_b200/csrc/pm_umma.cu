@@ -37,14 +37,17 @@ constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;      // about one second
 
 template <int MODE> struct Cfg {
   static constexpr int kTransformWarps = MODE == 1 ? 4 : 0;
-  static constexpr int kStages = MODE == 1 ? 2 : 6;        // operand ring depth
+  static constexpr int kStages = MODE == 1 ? 2 : 4;        // operand ring depth
   static constexpr int kStaging = MODE == 1 ? 2 : 0;       // fp32 staging ring depth (dgrad only)
   static constexpr int kThreads = 32 * (2 + kTransformWarps + N_EPI_WARPS);
-  static constexpr int kTileBytes = kStages * STAGE_BYTES + kStaging * STG_BYTES;
+  static constexpr int kOutWarpBytes = MODE == 1 ? 4096 : 8192;   // per epilogue warp: 32 rows x 128 B per output box
+  static constexpr int kOutBytes = N_EPI_WARPS * kOutWarpBytes;
+  static constexpr int kTileBytes = kStages * STAGE_BYTES + kStaging * STG_BYTES + kOutBytes;
   static constexpr int kSmemBytes = kTileBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
-enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6, MAPS_PER_LINEAR = 7 };
+enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6,
+       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAPS_PER_LINEAR = 11 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -93,6 +96,23 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// TMA stores (shared -> global, bulk-group completion).  Rows and columns outside the tensor are clipped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -195,6 +215,8 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
   uint8_t* tiles_ptr = smem_raw + (tiles - raw);
   const uint32_t stg = tiles + NS * STAGE_BYTES;                      // fp32 staging ring (dgrad)
   uint8_t* stg_ptr = tiles_ptr + NS * STAGE_BYTES;
+  const uint32_t outs = stg + NG * STG_BYTES;                         // epilogue staging for TMA stores
+  uint8_t* outs_ptr = stg_ptr + NG * STG_BYTES;
   const uint32_t bars = tiles + C::kTileBytes;
   // barrier block: full[NS] empty[NS] sfull[NG] sempty[NG] tfull[2] tempty[2], then tmem base word and abort flag
   const uint32_t bar_full = bars, bar_empty = bar_full + 8 * NS, bar_sfull = bar_empty + 8 * NS,
@@ -232,6 +254,9 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         if (!tl.valid) continue;
         const StageDyn& d = t.dyn[tl.p];
         const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
+        else if (MODE == 1) { tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_F32); tma_prefetch_desc(lm + MAP_D_F32); }
+        else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         for (int kb = 0; kb < tl.n_kb; ++kb) {
           const int k0 = kb * TILE_K;
           if (MODE == 1) {
@@ -352,17 +377,26 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     }
   } else {
     // ---------------- epilogue: 8 warps, warp%4 = TMEM lane group, two warps per group split the columns ----------------
+    // Each warp drains a 32-row x 64-column block, writes it into its own swizzled staging buffer and lets
+    // the TMA engine store it (full 128-byte rows; rows and columns beyond the tensor are clipped).
     const int q = warp & 3;
-    const int half = (warp - 2 - NT) >> 2;                            // 0: columns 0..63, 1: columns 64..127
+    const int ew = warp - 2 - NT;                                     // 0..7
+    const int half = ew >> 2;                                         // 0: columns 0..63, 1: columns 64..127
+    uint8_t* obuf = outs_ptr + ew * C::kOutWarpBytes;
+    const uint32_t obuf_s = outs + ew * C::kOutWarpBytes;
+    const uint32_t row_off = (uint32_t)lane * 128;
+    const uint32_t sw = (uint32_t)(lane & 7);
     Ring acc{0, 0};
     bool ok = true;
+    bool stored = false;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
       const StageDyn& d = t.dyn[tl.p];
       const StageDev& s = t.st[tl.p];
       const LinDev& L = s.lin[lvl];
-      const int m = tl.m0 + q * 32 + lane;
+      const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+      const int mrow = tl.m0 + q * 32;                                // first row of this warp's block
       const int nb = tl.n0 + half * 64;
       bool ready = !*abort_flag && mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
@@ -375,63 +409,68 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc.idx);           // the accumulator buffer may be overwritten now
+      if (lane == 0) {
+        mbar_arrive(bar_tempty + 8 * acc.idx);                        // the accumulator buffer may be overwritten now
+        if (stored) tma_store_wait_read();                            // previous stores have finished reading the staging buffer
+      }
+      __syncwarp();
       acc.advance(2);
-      if (m >= tl.M) continue;
-      const int N = tl.N;
+      if (mrow >= tl.M || nb >= tl.N) continue;                       // nothing of this block is inside the tensor
       if (MODE == 0) {
-        const size_t n_out_elems = (size_t)t.T * L.n_out;
-        __nv_bfloat16* zout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.z_ring) + (size_t)d.f_slot * n_out_elems;
-        __nv_bfloat16* yout;
-        if (lvl < s.n_lin - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + L.h_ring) + (size_t)d.f_slot * n_out_elems;
-        else if (tl.p < t.P - 1) yout = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[tl.p + 1].x_ring) + (size_t)d.f_next_xslot * n_out_elems;
-        else yout = reinterpret_cast<__nv_bfloat16*>(t.ws + t.yout_off) + (size_t)(d.tick & 1) * n_out_elems;
         const float* bias = t.a.w + L.b_off;
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const int n = nb + g * 8;
-          if (n < N) {
+          float bb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          if (n < tl.N) {
             const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
-            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-            float zf[8], yf[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const uint32_t a = g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e];
-              zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(a), bb[e])));
-              yf[e] = act_fwd(zf[e], L.act);
-            }
-            const size_t o = (size_t)m * N + n;
-            *reinterpret_cast<uint4*>(zout + o) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
-            *reinterpret_cast<uint4*>(yout + o) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
+            bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
           }
+          float zf[8], yf[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t a = g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e];
+            zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(a), bb[e])));
+            yf[e] = act_fwd(zf[e], L.act);
+          }
+          const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
+          *reinterpret_cast<uint4*>(obuf + off) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
+          *reinterpret_cast<uint4*>(obuf + 4096 + off) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
         }
       } else if (MODE == 1) {
-        const size_t n_in_elems = (size_t)t.T * L.n_in;
-        __nv_bfloat16* dx = (lvl == 0) ? reinterpret_cast<__nv_bfloat16*>(t.ws + t.st[tl.p - 1].gin) + (size_t)(d.tick & 1) * n_in_elems
-                                       : reinterpret_cast<__nv_bfloat16*>(t.ws + s.dh);
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
-          const int n = nb + g * 8;
-          if (n < N) {
-            float f[8];
+          float f[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
-            *reinterpret_cast<uint4*>(dx + (size_t)m * N + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-          }
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+          *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
+              make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
         }
       } else {
-        float* dW = t.a.grad + L.w_off;
 #pragma unroll
-        for (int g = 0; g < 16; ++g) {
-          const int n = nb + g * 4;
-          if (n < N) {
-            const uint32_t* rr = g < 8 ? r0 + (g & 7) * 4 : r1 + (g & 7) * 4;
-            *reinterpret_cast<float4*>(dW + (size_t)m * N + n) =
-                make_float4(__uint_as_float(rr[0]), __uint_as_float(rr[1]), __uint_as_float(rr[2]), __uint_as_float(rr[3]));
-          }
+        for (int g = 0; g < 8; ++g) {                                 // two boxes of 32 fp32 columns
+          *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r0[g * 4], r0[g * 4 + 1], r0[g * 4 + 2], r0[g * 4 + 3]);
+          *reinterpret_cast<uint4*>(obuf + 4096 + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r1[g * 4], r1[g * 4 + 1], r1[g * 4 + 2], r1[g * 4 + 3]);
         }
       }
+      fence_async_smem();                                             // staging writes -> visible to the TMA engine
+      __syncwarp();
+      if (lane == 0) {
+        if (MODE == 0) {
+          tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
+          const int yslot = lvl < s.n_lin - 1 ? d.f_slot : (tl.p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1));
+          tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
+        } else if (MODE == 1) {
+          tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, lvl == 0 ? (int)(d.tick & 1) : 0);
+        } else {
+          tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
+          if (nb + 32 < tl.N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
+        }
+        tma_store_commit();
+      }
+      stored = true;
     }
+    if (lane == 0 && stored) tma_store_wait_all();                    // global writes complete before the CTA retires
   }
   tc_fence_before();
   __syncthreads();
@@ -461,13 +500,14 @@ static uint64_t tiles_bytes(int P) { return ((uint64_t)3 * PM_MAX_LINEARS * (P +
 
 uint64_t umma_workspace_bytes(int n_stages) { return 256 + maps_bytes(n_stages) + tiles_bytes(n_stages); }
 
-static bool encode(EncodeTiledFn fn, CUtensorMap* m, bool f32, void* base, int rank, const uint64_t* dims,
+// kind: 0/1 bf16 with 128-byte swizzle, 2 fp32 with 128-byte swizzle, 3 fp32 without swizzle
+static bool encode(EncodeTiledFn fn, CUtensorMap* m, int kind, void* base, int rank, const uint64_t* dims,
                    const uint64_t* strides_bytes, const uint32_t* box, std::string& err) {
   cuuint64_t gd[3]; cuuint64_t gs[2]; cuuint32_t bx[3]; cuuint32_t es[3] = {1, 1, 1};
   for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
-  CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+  CUresult r = fn(m, kind >= 2 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gd, gs, bx, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, kind == 3 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return false; }
   return true;
@@ -500,21 +540,40 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       {
         uint64_t dims[3] = {n_in, T, slots}, strides[2] = {n_in * 2, T * n_in * 2};
         uint32_t box_k[3] = {TILE_K, TILE_M, 1}, box_mn[3] = {64, TILE_K, 1};
-        okm = okm && encode(fn, m + MAP_ACT_K, false, act_base, 3, dims, strides, box_k, err);
-        okm = okm && encode(fn, m + MAP_ACT_MN, false, act_base, 3, dims, strides, box_mn, err);
+        okm = okm && encode(fn, m + MAP_ACT_K, 0, act_base, 3, dims, strides, box_k, err);
+        okm = okm && encode(fn, m + MAP_ACT_MN, 0, act_base, 3, dims, strides, box_mn, err);
       }
       {
         uint64_t dims[2] = {n_in, n_out}, strides[1] = {n_in * 2}, strides4[1] = {n_in * 4};
         uint32_t box[2] = {TILE_K, TILE_N}, box4[2] = {TILE_N, TILE_K};
-        okm = okm && encode(fn, m + MAP_W_K, false, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err);
-        okm = okm && encode(fn, m + MAP_W_F32, true, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
-        okm = okm && encode(fn, m + MAP_D_F32, true, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
+        okm = okm && encode(fn, m + MAP_W_K, 0, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err);
+        okm = okm && encode(fn, m + MAP_W_F32, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
+        okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
       }
       {
         uint64_t dims[2] = {n_out, T}, strides[1] = {n_out * 2};
         uint32_t box_k[2] = {TILE_K, TILE_M}, box_mn[2] = {64, TILE_K};
-        okm = okm && encode(fn, m + MAP_DZ_K, false, t.ws + s.dz, 2, dims, strides, box_k, err);
-        okm = okm && encode(fn, m + MAP_DZ_MN, false, t.ws + s.dz, 2, dims, strides, box_mn, err);
+        okm = okm && encode(fn, m + MAP_DZ_K, 0, t.ws + s.dz, 2, dims, strides, box_k, err);
+        okm = okm && encode(fn, m + MAP_DZ_MN, 0, t.ws + s.dz, 2, dims, strides, box_mn, err);
+      }
+      {
+        // outputs: 32-row boxes of one 128-byte swizzle row (64 bf16 or 32 fp32 columns)
+        uint32_t box_bf[3] = {64, 32, 1}, box_f32[2] = {32, 32};
+        uint64_t zd[3] = {n_out, T, (uint64_t)s.depth}, zs[2] = {n_out * 2, T * n_out * 2};
+        okm = okm && encode(fn, m + MAP_Z_OUT, 1, t.ring + L.z_ring, 3, zd, zs, box_bf, err);
+        char* ybase; uint64_t yslots;
+        if (l < s.n_lin - 1) { ybase = t.ring + L.h_ring; yslots = (uint64_t)s.depth; }
+        else if (p < P - 1) { ybase = t.ring + st[p + 1].x_ring; yslots = (uint64_t)st[p + 1].xdepth; }
+        else { ybase = t.ws + t.yout_off; yslots = 2; }
+        uint64_t yd[3] = {n_out, T, yslots};
+        okm = okm && encode(fn, m + MAP_Y_OUT, 1, ybase, 3, yd, zs, box_bf, err);
+        if (!(p == 0 && l == 0)) {
+          char* xbase = l == 0 ? t.ws + st[p - 1].gin : t.ws + s.dh;
+          uint64_t xd[3] = {n_in, T, (uint64_t)(l == 0 ? 2 : 1)}, xs[2] = {n_in * 2, T * n_in * 2};
+          okm = okm && encode(fn, m + MAP_DX_OUT, 1, xbase, 3, xd, xs, box_bf, err);
+        }
+        uint64_t wd[2] = {n_in, n_out}, wst[1] = {n_in * 4};
+        okm = okm && encode(fn, m + MAP_DW_OUT, 2, (void*)(t.a.grad + L.w_off), 2, wd, wst, box_f32, err);
       }
       if (!okm) { delete plan; return PM_ERR_CUDA; }
     }
