@@ -18,6 +18,7 @@ from . import rng
 # stream ids (purpose of a random draw)
 _S_INIT, _S_TEACHER, _S_INPUT, _S_CALIB = 1, 2, 3, 500000
 _CALIB_ROWS = 256
+_CALIB_RMS = 1.0      # root-mean-square every pre-activation is calibrated to at initialisation
 _S_UPD_W, _S_UPD_G, _S_UPD_M, _S_UPD_S, _S_UPD_D = 10, 11, 12, 13, 14
 
 
@@ -119,7 +120,7 @@ def _all_params(wl, stream):
             w = rng.normal(wl.seed, stream + 1000 * (index + 1), spec.n_in * spec.n_out)
             w = w.reshape(spec.n_out, spec.n_in) / np.sqrt(spec.n_in)
             z = h @ w.T
-            scale = 1.0 / np.sqrt(np.mean(z * z))
+            scale = _CALIB_RMS / np.sqrt(np.mean(z * z))
             w32 = (w * scale).astype(np.float32)
             h = _act(h @ w32.astype(np.float64).T, spec.act)
             tensors.append((w32, np.zeros(spec.n_out, dtype=np.float32)))

@@ -9,7 +9,13 @@ pytestmark = pytest.mark.gpu
 
 F32_TOL = 1e-5          # max |dw| / max |w| per tensor, fp32 path
 BF16_W_TOL = 2e-2       # bf16 GEMM path, weights
-BF16_LOSS_TOL = 1e-3    # bf16 GEMM path, loss trajectory (relative)
+BF16_LOSS_TOL = 1e-3    # bf16 GEMM path, loss trajectory (relative), networks up to a dozen layers deep
+# At 64 bf16 layers the loss cannot agree to 1e-3 between ANY two summation orders: every layer re-quantises
+# to bfloat16, which turns a relative perturbation eps into one of about sqrt(eps * 2^-8), so two correct
+# implementations drift to a one-ulp (0.4 %) activation difference within a few layers.  Swapping only the
+# oracle's float64 matmul for a float32 one moves the first loss of this workload by 1.4e-3
+# (tests/test_tolerance_evidence.py).  The deep configurations therefore use:
+BF16_DEEP_LOSS_TOL = 1e-2
 
 
 def check_book(book, res, n_steps, P):
@@ -108,3 +114,33 @@ def test_too_small_buffers_are_reported(cuda_device):
                                C.c_void_p(pipe.stream.cuda_stream))
     assert pipe.L.pm_status_string(st) == b"PM_ERR_NOMEM"
     assert str(pipe.ring_bytes).encode() in pipe.L.pm_last_error(None)
+
+
+def test_cfg3_full_size_first_microbatches(cuda_device):
+    """The benchmark's own configuration (32 stages x 2 Linear(1024,1024)+GELU, microbatch 128, bf16):
+    four microbatches fed, pipeline drained, so every stage has applied four updates."""
+    wl = I.cfg3()
+    n = 4
+    params0 = I.init_stage_params(wl)
+    teacher = I.teacher_params(wl)
+    res = run_oracle(wl, params0, n, teacher)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, n, teacher)
+    check_book(book, res, n, wl.n_stages)
+    print("cfg3 full size loss relative errors", np.abs(losses / np.array(res.losses) - 1))
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_DEEP_LOSS_TOL)
+    worst = compare_params(pipe, res, BF16_W_TOL)
+    print("cfg3 full size worst relative weight error", worst)
+
+
+def test_cfg3_shape_many_steps(cuda_device):
+    """cfg3's structure (32 stages, two GELU Linears per stage, tau up to 63) at width 128 for 200 steps:
+    crosses the T1 annealing window (K=50) and runs every stage far past its pipeline fill."""
+    wl = I.mlp_workload("cfg3_narrow", 32, 128, 2, "gelu", 64, compute="bf16", optimizer="sgdm", alpha=0.01, beta1=0.9,
+                        K=50, D=0.5, steps=200, seed=191005124 + 34)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, collect_book=False)
+    print("cfg3 narrow max loss relative error", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_DEEP_LOSS_TOL)
+    worst = compare_params(pipe, res, BF16_W_TOL)
+    print("cfg3 narrow 200 steps worst relative weight error", worst)
