@@ -1,0 +1,131 @@
+"""Pipeline of Transformer-encoder stages with a cross-entropy loss: grad f_t(u_fwd, u_bkwd).
+
+TEST INFRASTRUCTURE (see package docstring).
+
+Every stage holds exactly one weight matrix ("one stage per weight GEMM") and has the shape
+
+    pre   : 'embed' (token embedding * sqrt(d) + sinusoidal positions) | 'ln' (LayerNorm) | 'none'
+    linear: z = u W^T + b ;  y = act(z)
+    post  : 'attention' (split y into q, k, v; multi-head self-attention; also hands u on as a skip tensor)
+            'skip_out'  (hands u on as a skip tensor next to y)
+            'residual'  (adds the skip tensor received from the previous stage to y)
+            'none'
+
+A post-LN encoder layer is four stages: [ln|embed, W_qkv, attention] [W_o, residual] [ln, W_1 + ReLU, skip_out]
+[W_2, residual]; the last stage is [ln, W_vocab] followed by the loss.  Parameters of a stage in order:
+[table] (embed), [gain, bias] (ln), W, b.
+
+The backward pass reads u_bkwd in exactly two places (Section 2.1: the weights "used in the backward pass"):
+the Linear matrix of the input-gradient product and the LayerNorm gain of dx_hat = dy * gain.
+
+Parity of whole training trajectories is unpinned by the paper; this module is pinned through finite
+differences of the complete model (u_fwd = u_bkwd) and the layer-level library cross-checks.
+"""
+import numpy as np
+
+from . import layers as L
+from .bf16 import bf16_round
+
+
+def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
+    """stage_specs: per stage an object with fields pre, post, act (strings).
+    data_fn: t -> (ids [T] int, targets [T] int)."""
+    rnd = bf16_round if compute == "bf16" else L.identity
+    f64 = lambda a: np.asarray(a, dtype=np.float64)
+
+    def unpack(spec, tensors):
+        i = 0
+        out = {}
+        if spec.pre == "embed":
+            out["table"] = f64(tensors[i]); i += 1
+        if spec.pre == "ln":
+            out["gain"], out["beta"] = f64(tensors[i]), f64(tensors[i + 1]); i += 2
+        out["W"], out["b"] = f64(tensors[i]), f64(tensors[i + 1])
+        return out
+
+    def grad_fn(t, u_fwd, u_bkwd):
+        ids, targets = data_fn(t)
+        P = len(stage_specs)
+        main, skip = None, None
+        stash = []
+        logits = None
+        for i, spec in enumerate(stage_specs):
+            pf = unpack(spec, u_fwd[i])
+            st = {}
+            if spec.pre == "embed":
+                u = L.embed_fwd(ids, pf["table"], seq_len, rnd)
+            elif spec.pre == "ln":
+                u, st["xhat"], st["rstd"] = L.layernorm_fwd(main, pf["gain"], pf["beta"], rnd)
+            else:
+                u = main
+            st["u"] = u
+            acc = u @ rnd(pf["W"]).T + pf["b"]
+            if i == P - 1:
+                logits = acc                                   # fp32 on the device, not rounded
+                stash.append(st)
+                break
+            z = rnd(acc)
+            y = rnd(L.act_fwd(z, spec.act))
+            st["z"] = z
+            if spec.post == "attention":
+                d = y.shape[1] // 3
+                st["q"], st["k"], st["v"] = y[:, :d], y[:, d:2 * d], y[:, 2 * d:]
+                main, skip = L.attention_fwd(st["q"], st["k"], st["v"], n_heads, seq_len, False, rnd), u
+            elif spec.post == "skip_out":
+                main, skip = y, u
+            elif spec.post == "residual":
+                main, skip = rnd(skip + y), None
+            else:
+                main, skip = y, None
+            stash.append(st)
+
+        loss, d_main = L.cross_entropy(logits, targets, rnd)
+        d_skip = None
+        grads = [[None] * len(u_fwd[i]) for i in range(P)]
+        for i in reversed(range(P)):
+            spec, st = stage_specs[i], stash[i]
+            pb = unpack(spec, u_bkwd[i])
+            du_extra, d_in_skip = None, None
+            if i == P - 1:
+                dz = d_main                                     # dlogits, already in operand precision
+            else:
+                if spec.post == "attention":
+                    dq, dk, dv = L.attention_bwd(d_main, st["q"], st["k"], st["v"], n_heads, seq_len, False, rnd)
+                    dy, du_extra = np.concatenate([dq, dk, dv], axis=1), d_skip
+                elif spec.post == "skip_out":
+                    dy, du_extra = d_main, d_skip
+                elif spec.post == "residual":
+                    dy, d_in_skip = d_main, d_main
+                else:
+                    dy = d_main
+                dz = rnd(dy * L.act_grad(st["z"], spec.act))
+            dW = dz.T @ st["u"]
+            db = dz.sum(axis=0)
+            du = rnd(dz @ rnd(pb["W"]))
+            if du_extra is not None:
+                du = du + du_extra
+            g = []
+            if spec.pre == "embed":
+                g.append(L.embed_bwd(du, ids, vocab))
+                d_in = None
+            elif spec.pre == "ln":
+                d_in, dgain, dbeta = L.layernorm_bwd(du, st["xhat"], st["rstd"], pb["gain"], rnd)
+                g += [dgain, dbeta]
+            else:
+                d_in = du
+            g += [dW, db]
+            grads[i] = g
+            d_main, d_skip = d_in, d_in_skip
+        return loss, grads
+
+    return grad_fn
+
+
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None):
+    """params0: per stage the list of tensors in the order [table] [gain, bias] W b."""
+    from . import recurrence
+    hp = dict(optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+              t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
+    grad_fn = make_grad_fn(wl.stage_specs, data_fn, wl.n_heads, wl.seq_len, wl.vocab, wl.compute)
+    return recurrence.run(params0, wl.tau_fwd, wl.tau_bkwd, grad_fn, wl.steps if n_steps is None else n_steps,
+                          hp, dtype=dtype, on_step=on_step)

@@ -30,6 +30,16 @@ class LinearSpec:
 
 
 @dataclass
+class StageSpec:
+    """One Transformer stage: pre-op, one Linear, post-op (see the encoder workload below)."""
+    pre: str        # 'embed' | 'ln' | 'none'
+    n_in: int
+    n_out: int
+    act: str        # 'relu' | 'gelu' | 'none'
+    post: str       # 'attention' | 'skip_out' | 'residual' | 'none'
+
+
+@dataclass
 class Workload:
     name: str
     stages: List[List[LinearSpec]]
@@ -49,10 +59,16 @@ class Workload:
     steps: int = 64
     seed: int = 191005124
     notes: str = field(default="")
+    kind: str = "mlp"           # 'mlp' | 'encoder'
+    stage_specs: List[StageSpec] = field(default_factory=list)   # encoder workloads
+    n_heads: int = 0
+    seq_len: int = 0
+    vocab: int = 0
+    d_model: int = 0
 
     @property
     def n_stages(self):
-        return len(self.stages)
+        return len(self.stage_specs) if self.kind == "encoder" else len(self.stages)
 
 
 def pipemare_delays(P, n_micro=1):
@@ -189,3 +205,63 @@ def update_sweep_case(n_params, P, optimizer="sgdm", seed=191005124 + 2, align=6
     if optimizer == "adam":
         case["s"] = fill(_S_UPD_S, 1e-3, positive=True)
     return case
+
+
+# ---- Transformer encoder workloads -------------------------------------------------------------------------
+
+_S_TOKENS, _S_ENC_INIT = 40, 50
+
+
+def encoder_workload(name, n_layers, d_model, n_heads, d_ff, seq_len, batch, vocab, **kw):
+    """Post-LN encoder, one stage per weight matrix: per layer [W_qkv + attention] [W_o + residual]
+    [LN, W_1 + ReLU] [W_2 + residual]; the embedding rides with stage 1, each LayerNorm with the stage
+    that follows it, and the vocabulary projection (with the final LayerNorm) is the last stage."""
+    specs = []
+    for layer in range(n_layers):
+        specs.append(StageSpec("embed" if layer == 0 else "ln", d_model, 3 * d_model, "none", "attention"))
+        specs.append(StageSpec("none", d_model, d_model, "none", "residual"))
+        specs.append(StageSpec("ln", d_model, d_ff, "relu", "skip_out"))
+        specs.append(StageSpec("none", d_ff, d_model, "none", "residual"))
+    specs.append(StageSpec("ln", d_model, vocab, "none", "none"))
+    P = len(specs)
+    fwd, bkwd = pipemare_delays(P)
+    return Workload(name=name, stages=[], tau_fwd=fwd, tau_bkwd=bkwd, microbatch=batch * seq_len, kind="encoder",
+                    stage_specs=specs, n_heads=n_heads, seq_len=seq_len, vocab=vocab, d_model=d_model, **kw)
+
+
+def cfg4():
+    """Encoder, 6 layers, d_model 512, 8 heads, FFN 2048, sequence 128, microbatch 32 sequences, vocabulary 8192,
+    bf16 GEMMs; target = input sequence reversed; Adam(0.9, 0.98), alpha 5e-4, K = 100, D = 0.1; 300 steps."""
+    return encoder_workload("cfg4_encoder6_bf16", 6, 512, 8, 2048, 128, 32, 8192, compute="bf16", optimizer="adam",
+                            alpha=5e-4, beta1=0.9, beta2=0.98, eps=1e-8, K=100, D=0.1, steps=300, seed=191005124 + 4)
+
+
+def cfg4_small(compute="bf16", n_layers=2, d_model=64, n_heads=2, d_ff=128, seq_len=16, batch=3, vocab=96, steps=24):
+    """Same structure as cfg4 at a size the oracle runs in seconds."""
+    return encoder_workload("cfg4_small", n_layers, d_model, n_heads, d_ff, seq_len, batch, vocab, compute=compute,
+                            optimizer="adam", alpha=5e-4, beta1=0.9, beta2=0.98, eps=1e-8, K=max(steps // 3, 1), D=0.1,
+                            steps=steps, seed=191005124 + 44)
+
+
+def init_encoder_params(wl):
+    """Per stage the tensors [table] [gain, bias] W b (float32): W ~ N(0, 1/fan_in), table ~ N(0, 1/d_model),
+    biases 0, LayerNorm gain 1 and bias 0."""
+    out = []
+    for i, sp in enumerate(wl.stage_specs):
+        tensors = []
+        if sp.pre == "embed":
+            e = rng.normal(wl.seed, _S_ENC_INIT + 7, wl.vocab * wl.d_model) / np.sqrt(wl.d_model)
+            tensors.append(e.reshape(wl.vocab, wl.d_model).astype(np.float32))
+        if sp.pre == "ln":
+            tensors += [np.ones(sp.n_in, dtype=np.float32), np.zeros(sp.n_in, dtype=np.float32)]
+        w = rng.normal(wl.seed, _S_ENC_INIT + 1000 * (i + 1), sp.n_in * sp.n_out) / np.sqrt(sp.n_in)
+        tensors += [w.reshape(sp.n_out, sp.n_in).astype(np.float32), np.zeros(sp.n_out, dtype=np.float32)]
+        out.append(tensors)
+    return out
+
+
+def token_batch(wl, t):
+    """Microbatch t: ids uniform on [0, vocab) of shape [batch*seq_len]; target = each sequence reversed."""
+    n_seq = wl.microbatch // wl.seq_len
+    ids = rng.randint(wl.seed, _S_TOKENS + 16 * t, wl.microbatch, wl.vocab).reshape(n_seq, wl.seq_len)
+    return ids.reshape(-1).astype(np.int64), ids[:, ::-1].reshape(-1).astype(np.int64)
