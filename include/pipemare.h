@@ -46,19 +46,34 @@ typedef enum {
 enum { PM_F32 = 0, PM_BF16 = 1 };                 /* GEMM operand type; state is always fp32 */
 enum { PM_SGDM = 0, PM_ADAM = 1 };
 enum { PM_ACT_NONE = 0, PM_ACT_RELU = 1, PM_ACT_GELU = 2 };   /* GELU = exact erf form      */
-enum { PM_OP_LINEAR = 0 };
-enum { PM_LOSS_MSE = 0 };
+enum { PM_OP_LINEAR = 0, PM_OP_EMBED = 1, PM_OP_LAYERNORM = 2, PM_OP_ATTENTION = 3, PM_OP_SKIP_OUT = 4,
+       PM_OP_RESIDUAL = 5 };
+enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
 
 /* Alignment, in elements, of every stage slice and of every tensor inside it. */
 #define PM_ALIGN_ELEMS 64
 #define PM_MAX_LINEARS 4       /* Linear ops per stage                                    */
 #define PM_MAX_STAGES 1024
 
-/* One operator of a stage.  LINEAR: y = act(x W^T + b), W is [n_out, n_in] row-major. */
+/* One operator of a stage.  A stage is  [EMBED | LAYERNORM]  LINEAR{1..PM_MAX_LINEARS}  [ATTENTION | SKIP_OUT |
+ * RESIDUAL]  (with a pre- or post-op exactly one LINEAR).
+ *   LINEAR     y = act(x W^T + b), W is [n_out, n_in] row-major, b is [n_out].
+ *   EMBED      x = table[id] * sqrt(n_out) + sinusoidal position; table is [n_in = vocabulary, n_out = width];
+ *              first stage only; the stage's input is then int32 token ids.  seq_len gives the position period.
+ *   LAYERNORM  over the last dimension (n_in = n_out = width), eps 1e-5, biased variance; parameters gain, bias.
+ *   ATTENTION  splits the Linear's output [T, 3d] into q, k, v; softmax(q k^T / sqrt(d / n_heads)) v per head and
+ *              per sequence of seq_len rows (T a multiple of seq_len, seq_len <= 128); the stage hands o [T, d]
+ *              and, as a skip tensor, the Linear's input to the next stage, which must end in RESIDUAL.
+ *   SKIP_OUT   hands the Linear's input on as a skip tensor next to its output; next stage must end in RESIDUAL.
+ *   RESIDUAL   adds the skip tensor received from the previous stage to the Linear's output.
+ * Where the backward pass reads a parameter value it reads the T2-corrected one (Section 3.2): the Linear
+ * matrix in the input-gradient product and the LayerNorm gain.  Nothing else is read in the backward pass. */
 typedef struct {
-  int32_t kind;            /* PM_OP_LINEAR */
+  int32_t kind;            /* PM_OP_* */
   int32_t n_in, n_out;
-  int32_t act;             /* PM_ACT_* */
+  int32_t act;             /* PM_ACT_* (LINEAR) */
+  int32_t n_heads;         /* ATTENTION */
+  int32_t seq_len;         /* ATTENTION, EMBED */
 } pm_op_desc;
 
 /* One pipeline stage (Section 2.1).  Copied during pm_init_stages.
@@ -90,7 +105,9 @@ typedef struct {
   int32_t microbatch;      /* rows T of every activation matrix */
   int32_t compute_dtype;   /* PM_F32 | PM_BF16 */
   int32_t optimizer;       /* PM_SGDM | PM_ADAM */
-  int32_t loss;            /* PM_LOSS_MSE: mean over all T*out entries of (y - target)^2 */
+  int32_t loss;            /* PM_LOSS_MSE: mean over all T*out entries of (y - target)^2;
+                              PM_LOSS_CE: mean over the T rows of logsumexp(logits) - logits[target], logits =
+                              the last Linear's fp32 output (last stage: one Linear, activation none, no post-op) */
   float beta1, beta2, eps;
   int32_t t1_enable;
   int64_t t1_K;
@@ -121,7 +138,8 @@ typedef struct {
 
 /* Number of elements a stage with these ops occupies in the arenas (padded). */
 pm_status pm_stage_param_count(const pm_op_desc* ops, int32_t n_ops, uint64_t* count);
-/* Offsets of op `op`'s weight matrix and bias vector relative to the stage's param_offset. */
+/* Offsets of op `op`'s two parameter tensors relative to the stage's param_offset: LINEAR (W, b);
+ * LAYERNORM (gain, bias); EMBED (table, unused).  Ops without parameters give PM_ERR_INVALID_ARG. */
 pm_status pm_op_param_offsets(const pm_op_desc* ops, int32_t n_ops, int32_t op,
                               uint64_t* w_off, uint64_t* b_off);
 
@@ -146,8 +164,9 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
 
 /* One tick = pm_forward, pm_backward, pm_update in this order (pm_step does all three).
  * inputs/targets (device) belong to the microbatch that enters the pipeline at this tick:
- * inputs is [T, n_in of stage 1] (float for PM_F32, bfloat16 for PM_BF16), targets is
- * [T, n_out of stage P] float.  Both are copied before the call returns control to the
+ * inputs is [T, n_in of stage 1] (float for PM_F32, bfloat16 for PM_BF16), or [T] int32 token ids when
+ * stage 1 starts with EMBED; targets is [T, n_out of stage P] float (PM_LOSS_MSE) or [T] int32 class ids
+ * (PM_LOSS_CE).  Both are copied before the call returns control to the
  * stream order, so the caller may overwrite them after any later call on the same stream.
  * Pass NULL for both to drain: N microbatches need N + 2P - 1 ticks.
  *

@@ -13,8 +13,8 @@ import numpy as np
 PM_F32, PM_BF16 = 0, 1
 PM_SGDM, PM_ADAM = 0, 1
 PM_ACT_NONE, PM_ACT_RELU, PM_ACT_GELU = 0, 1, 2
-PM_OP_LINEAR = 0
-PM_LOSS_MSE = 0
+PM_OP_LINEAR, PM_OP_EMBED, PM_OP_LAYERNORM, PM_OP_ATTENTION, PM_OP_SKIP_OUT, PM_OP_RESIDUAL = 0, 1, 2, 3, 4, 5
+PM_LOSS_MSE, PM_LOSS_CE = 0, 1
 PM_ALIGN_ELEMS = 64
 
 _ACT = {"none": PM_ACT_NONE, "relu": PM_ACT_RELU, "gelu": PM_ACT_GELU}
@@ -23,7 +23,8 @@ LIB_PATH = os.path.join(_HERE, "libpipemare.so")
 
 
 class pm_op_desc(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("n_in", C.c_int32), ("n_out", C.c_int32), ("act", C.c_int32)]
+    _fields_ = [("kind", C.c_int32), ("n_in", C.c_int32), ("n_out", C.c_int32), ("act", C.c_int32),
+                ("n_heads", C.c_int32), ("seq_len", C.c_int32)]
 
 
 class pm_stage_desc(C.Structure):
@@ -102,12 +103,12 @@ def _check(status, ctx=None):
 
 
 def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, beta2=0.98, eps=1e-8,
-                t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0):
+                t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0, loss=PM_LOSS_MSE):
     cfg = pm_config()
     cfg.n_stages, cfg.microbatch = n_stages, microbatch
     cfg.compute_dtype = PM_BF16 if compute in ("bf16", PM_BF16) and compute != 0 else PM_F32
     cfg.optimizer = PM_ADAM if optimizer in ("adam", PM_ADAM) and optimizer != 0 else PM_SGDM
-    cfg.loss = PM_LOSS_MSE
+    cfg.loss = loss
     cfg.beta1, cfg.beta2, cfg.eps = beta1, beta2, eps
     cfg.t1_enable, cfg.t1_K = int(bool(t1)), int(K)
     cfg.t2_enable, cfg.t2_D = int(bool(t2)), float(D)
@@ -122,24 +123,65 @@ def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, b
 
 
 def _ops_array(specs):
-    arr = (pm_op_desc * len(specs))()
-    for j, sp in enumerate(specs):
-        arr[j].kind, arr[j].n_in, arr[j].n_out, arr[j].act = PM_OP_LINEAR, sp.n_in, sp.n_out, _ACT[sp.act]
+    """ctypes op array of an MLP stage (a list of Linear specs)."""
+    return _ops_from_dicts([dict(kind=PM_OP_LINEAR, n_in=sp.n_in, n_out=sp.n_out, act=_ACT[sp.act]) for sp in specs])
+
+
+def _ops_from_dicts(ops):
+    arr = (pm_op_desc * len(ops))()
+    for j, o in enumerate(ops):
+        arr[j].kind, arr[j].n_in, arr[j].n_out = o["kind"], o.get("n_in", 0), o.get("n_out", 0)
+        arr[j].act, arr[j].n_heads, arr[j].seq_len = o.get("act", 0), o.get("n_heads", 0), o.get("seq_len", 0)
     return arr
 
 
-def stage_layout(specs):
-    """(padded element count, [(w_off, b_off) per op]) of a stage, as the library lays it out."""
+def stage_ops(wl, p):
+    """Op list of stage p and, per parameter tensor in the workload's order, (op index, slot, shape)."""
+    if getattr(wl, "kind", "mlp") == "encoder":
+        sp = wl.stage_specs[p]
+        ops, tensors = [], []
+        if sp.pre == "embed":
+            ops.append(dict(kind=PM_OP_EMBED, n_in=wl.vocab, n_out=wl.d_model, seq_len=wl.seq_len))
+            tensors.append((0, 0, (wl.vocab, wl.d_model)))
+        elif sp.pre == "ln":
+            ops.append(dict(kind=PM_OP_LAYERNORM, n_in=sp.n_in, n_out=sp.n_in))
+            tensors += [(0, 0, (sp.n_in,)), (0, 1, (sp.n_in,))]
+        li = len(ops)
+        ops.append(dict(kind=PM_OP_LINEAR, n_in=sp.n_in, n_out=sp.n_out, act=_ACT[sp.act]))
+        tensors += [(li, 0, (sp.n_out, sp.n_in)), (li, 1, (sp.n_out,))]
+        if sp.post == "attention":
+            ops.append(dict(kind=PM_OP_ATTENTION, n_in=sp.n_out, n_out=sp.n_out // 3, n_heads=wl.n_heads, seq_len=wl.seq_len))
+        elif sp.post == "skip_out":
+            ops.append(dict(kind=PM_OP_SKIP_OUT))
+        elif sp.post == "residual":
+            ops.append(dict(kind=PM_OP_RESIDUAL))
+        return ops, tensors
+    ops, tensors = [], []
+    for j, sp in enumerate(wl.stages[p]):
+        ops.append(dict(kind=PM_OP_LINEAR, n_in=sp.n_in, n_out=sp.n_out, act=_ACT[sp.act]))
+        tensors += [(j, 0, (sp.n_out, sp.n_in)), (j, 1, (sp.n_out,))]
+    return ops, tensors
+
+
+def ops_layout(arr, n_ops, tensors):
+    """(padded element count of the stage, offset of each parameter tensor), as the library lays it out."""
     L = lib()
-    arr = _ops_array(specs)
     cnt = C.c_uint64()
-    _check(L.pm_stage_param_count(arr, len(specs), C.byref(cnt)))
+    _check(L.pm_stage_param_count(arr, n_ops, C.byref(cnt)))
     offs = []
-    for j in range(len(specs)):
-        wo, bo = C.c_uint64(), C.c_uint64()
-        _check(L.pm_op_param_offsets(arr, len(specs), j, C.byref(wo), C.byref(bo)))
-        offs.append((wo.value, bo.value))
+    for (op, slot, shape) in tensors:
+        a, b = C.c_uint64(), C.c_uint64()
+        _check(L.pm_op_param_offsets(arr, n_ops, op, C.byref(a), C.byref(b)))
+        offs.append(a.value if slot == 0 else b.value)
     return cnt.value, offs
+
+
+def stage_layout(specs):
+    """(padded element count, [(w_off, b_off) per op]) of an MLP stage, as the library lays it out."""
+    arr = _ops_array(specs)
+    tensors = [t for j, sp in enumerate(specs) for t in ((j, 0, None), (j, 1, None))]
+    cnt, offs = ops_layout(arr, len(specs), tensors)
+    return cnt, [(offs[2 * j], offs[2 * j + 1]) for j in range(len(specs))]
 
 
 class Pipeline:
@@ -156,14 +198,22 @@ class Pipeline:
         self.wl = wl
         self.L = lib()
         self.device = torch.device(device)
-        P = len(wl.stages)
-        self._ops = [_ops_array(st) for st in wl.stages]
-        self.layout = [stage_layout(st) for st in wl.stages]
+        P = wl.n_stages
+        self.P = P
+        self.is_encoder = getattr(wl, "kind", "mlp") == "encoder"
+        self._op_dicts, self._tensors, self._ops, self.layout = [], [], [], []
+        for p in range(P):
+            ops, tensors = stage_ops(wl, p)
+            arr = _ops_from_dicts(ops)
+            self._op_dicts.append(ops)
+            self._tensors.append(tensors)
+            self._ops.append(arr)
+            self.layout.append(ops_layout(arr, len(ops), tensors))
         self.stage_desc = (pm_stage_desc * P)()
         off = 0
         for p in range(P):
             d = self.stage_desc[p]
-            d.tau_fwd, d.tau_bkwd, d.n_ops = wl.tau_fwd[p], wl.tau_bkwd[p], len(wl.stages[p])
+            d.tau_fwd, d.tau_bkwd, d.n_ops = wl.tau_fwd[p], wl.tau_bkwd[p], len(self._op_dicts[p])
             d.ops = C.cast(self._ops[p], C.POINTER(pm_op_desc))
             d.param_offset, d.param_count = off, self.layout[p][0]
             off += self.layout[p][0]
@@ -171,7 +221,7 @@ class Pipeline:
         self.cfg, self._alpha_keep = make_config(
             n_stages=P, microbatch=wl.microbatch, compute=wl.compute, optimizer=wl.optimizer, alpha=wl.alpha,
             beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D,
-            loss_log_capacity=loss_log_capacity)
+            loss_log_capacity=loss_log_capacity, loss=PM_LOSS_CE if self.is_encoder else PM_LOSS_MSE)
         sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
         _check(self.L.pm_query_bytes(C.byref(self.cfg), self.stage_desc, C.byref(sb), C.byref(rb), C.byref(wb)))
         self.state_bytes, self.ring_bytes, self.workspace_bytes = sb.value, rb.value, wb.value
@@ -185,10 +235,12 @@ class Pipeline:
         flat = np.zeros(self.total, dtype=np.float32)
         for p in range(P):
             base = self.stage_desc[p].param_offset
-            for j, (W, b) in enumerate(params0[p]):
-                wo, bo = self.layout[p][1][j]
-                flat[base + wo: base + wo + W.size] = np.asarray(W, dtype=np.float32).ravel()
-                flat[base + bo: base + bo + b.size] = np.asarray(b, dtype=np.float32).ravel()
+            tensors = params0[p]
+            if not self.is_encoder:                       # MLP stages come as (W, b) pairs
+                tensors = [a for pair in tensors for a in pair]
+            for a, o in zip(tensors, self.layout[p][1]):
+                a = np.asarray(a, dtype=np.float32)
+                flat[base + o: base + o + a.size] = a.ravel()
         self.w.copy_(torch.from_numpy(flat))
         self.w_lp = self.w.to(torch.bfloat16) if wl.compute == "bf16" else None
         self.ring = torch.empty(max(self.ring_bytes, 256), dtype=torch.uint8, device=dev)
@@ -234,17 +286,18 @@ class Pipeline:
 
     # -- marshalling helpers --------------------------------------------------------------------
     def unpack(self, flat_tensor):
-        """Split a flat arena (device tensor) into per-stage lists of (W, b) numpy arrays."""
+        """Split a flat arena (device tensor) into per-stage parameter tensors (numpy): (W, b) pairs for MLP
+        stages, the list [table] [gain, bias] W b for encoder stages."""
         flat = flat_tensor.detach().float().cpu().numpy()
         out = []
-        for p, st in enumerate(self.wl.stages):
+        for p in range(self.P):
             base = self.stage_desc[p].param_offset
             tensors = []
-            for j, sp in enumerate(st):
-                wo, bo = self.layout[p][1][j]
-                W = flat[base + wo: base + wo + sp.n_in * sp.n_out].reshape(sp.n_out, sp.n_in).copy()
-                b = flat[base + bo: base + bo + sp.n_out].copy()
-                tensors.append((W, b))
+            for (op, slot, shape), o in zip(self._tensors[p], self.layout[p][1]):
+                n = int(np.prod(shape))
+                tensors.append(flat[base + o: base + o + n].reshape(shape).copy())
+            if not self.is_encoder:
+                tensors = [(tensors[2 * j], tensors[2 * j + 1]) for j in range(len(tensors) // 2)]
             out.append(tensors)
         return out
 

@@ -7,26 +7,44 @@
 
 namespace pm {
 
+enum { PRE_NONE = 0, PRE_EMBED = 1, PRE_LN = 2 };
+enum { POST_NONE = 0, POST_ATTENTION = 1, POST_SKIP_OUT = 2, POST_RESIDUAL = 3 };
+enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4 };
+
 // Static description of one Linear inside a stage (device copy).
 struct LinDev {
-  int32_t n_in, n_out, act, _pad;
+  int32_t n_in, n_out, act;
+  int32_t flags;              // LF_*: which of z (pre-activation stash), y (activation) the forward writes; fp32 logits
   uint64_t w_off, b_off;      // element offsets into the flat arenas
-  uint64_t z_ring;            // byte offset in the ring arena of z[depth][T*n_out] (pre-activation stash)
+  uint64_t z_ring;            // byte offset in the ring arena of z[depth][T*n_out] (pre-activation / q,k,v stash)
   uint64_t h_ring;            // byte offset of this Linear's output stash h[depth][T*n_out] (unused for the last Linear)
 };
 
-// Static description of one stage (device copy).
+// Static description of one stage (device copy).  A stage is [pre-op] Linear{1..4} [post-op]:
+//   pre : embedding (+ positions) | LayerNorm | none        post: attention | skip_out | residual | none
 struct StageDev {
   int32_t tau_f, gap;         // tau_fwd, tau_fwd - tau_bkwd
   int32_t n_lin;
-  int32_t depth;              // slots of z / h rings  = tau_f + 1
-  int32_t xdepth;             // slots of the input ring = tau_f + 2 (it doubles as the forward mailbox)
+  int32_t depth;              // slots of the stash rings = tau_f + 1
+  int32_t xdepth;             // slots of the main-input ring = tau_f + 2 (it doubles as the forward mailbox)
   int32_t max_dim;
+  int32_t pre, post;
+  int32_t n_heads, seq_len, vocab;
+  int32_t d_in;               // width of the main input (= width of u, the first Linear's input)
+  int32_t d_out_main;         // width of the main output handed to the next stage
+  int32_t _pad;
   uint64_t begin, end;        // padded element range of the stage's parameters in the arenas
-  uint64_t x_ring;            // byte offset of x[xdepth][T*n_in0]
-  uint64_t gin;               // workspace byte offset: incoming gradient mailbox [2][T*n_out_last]
-  uint64_t dz;                // workspace byte offset: dz scratch [T*max_dim]
-  uint64_t dh;                // workspace byte offset: dh scratch [T*max_dim]
+  uint64_t tab_off, g_off, beta_off;   // arena offsets: embedding table / LayerNorm gain / LayerNorm bias
+  uint64_t x_ring;            // ring: x[xdepth][T*d_in] main input (not used by an embedding stage)
+  uint64_t u_ring;            // ring: u[depth][T*d_in] first Linear's input when a pre-op produces it
+  uint64_t stat_ring;         // ring: LayerNorm mean, rstd [depth][T*2] float
+  uint64_t ids_ring;          // ring: token ids [depth][T] int32 (embedding stage)
+  uint64_t skip_in;           // ws: incoming skip tensor [2][T*n_out] (residual stage), slot = tick parity of its writer
+  uint64_t ytmp;              // ws: Linear output awaiting the residual add [T*n_out]
+  uint64_t gin;               // ws: incoming gradient w.r.t. the main output [3][T*d_out_main], slot = writer's tick % 3
+  uint64_t dy;                // ws: gradient w.r.t. the Linear output when a post-op produces it [T*n_out] (attention)
+  uint64_t dz;                // ws: dz scratch [T*max_dim]
+  uint64_t dh;                // ws: dgrad output scratch [T*max_dim] (du of the first Linear, dh between Linears)
   LinDev lin[PM_MAX_LINEARS];
 };
 

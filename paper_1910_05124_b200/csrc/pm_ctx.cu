@@ -1,4 +1,5 @@
 // Host side of the C ABI: layout arithmetic, context set-up, and the launch sequence of a tick.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <string>
@@ -23,12 +24,24 @@ struct Layout {
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
-  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0;
+  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0;
+  int32_t any_pre = 0, any_ln = 0, any_embed = 0, any_residual = 0, att_S = 0, att_dk = 0, att_blocks = 0, max_vocab = 0;
+  int32_t pe_seq = 0, pe_d = 0;
   int64_t loss_cap = 0;
   int32_t max_lin = 0, max_dim = 0, n_in_first = 0, n_out_last = 0;
 };
 
 pm_status fail(pm_ctx* ctx, pm_status s, const std::string& msg);
+
+// Parameter tensors of an op: count (0, 1 or 2) and their sizes.
+static int op_params(const pm_op_desc& op, uint64_t* n0, uint64_t* n1) {
+  switch (op.kind) {
+    case PM_OP_LINEAR: *n0 = (uint64_t)op.n_in * op.n_out; *n1 = (uint64_t)op.n_out; return 2;
+    case PM_OP_LAYERNORM: *n0 = (uint64_t)op.n_in; *n1 = (uint64_t)op.n_in; return 2;
+    case PM_OP_EMBED: *n0 = (uint64_t)op.n_in * op.n_out; *n1 = 0; return 1;
+    default: *n0 = *n1 = 0; return 0;
+  }
+}
 
 pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout& L, std::string& err) {
   if (!cfg || !stages) { err = "null config or stage list"; return PM_ERR_INVALID_ARG; }
@@ -37,65 +50,138 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   if (cfg->microbatch < 1) { err = "microbatch must be positive"; return PM_ERR_INVALID_ARG; }
   if (cfg->compute_dtype != PM_F32 && cfg->compute_dtype != PM_BF16) { err = "unknown compute_dtype"; return PM_ERR_INVALID_ARG; }
   if (cfg->optimizer != PM_SGDM && cfg->optimizer != PM_ADAM) { err = "unknown optimizer"; return PM_ERR_INVALID_ARG; }
-  if (cfg->loss != PM_LOSS_MSE) { err = "only PM_LOSS_MSE is built"; return PM_ERR_UNSUPPORTED; }
+  if (cfg->loss != PM_LOSS_MSE && cfg->loss != PM_LOSS_CE) { err = "unknown loss"; return PM_ERR_INVALID_ARG; }
   if (cfg->t1_enable && cfg->t1_K < 1) { err = "t1_K must be >= 1"; return PM_ERR_INVALID_ARG; }
   const uint64_t esz = cfg->compute_dtype == PM_F32 ? 4 : 2;
   const uint64_t T = (uint64_t)cfg->microbatch;
+  const bool ce = cfg->loss == PM_LOSS_CE;
   L.st.assign(P, StageDev{});
   L.sched.assign(P, StageSched{});
   L.begin64.assign(P, 0);
   L.end64.assign(P, 0);
   uint64_t ring = 0;
-  int prev_out = -1;
   uint64_t prev_end = 0;
+  auto stage_err = [&](int p, const std::string& m) { err = "stage " + std::to_string(p) + ": " + m; };
   for (int p = 0; p < P; ++p) {
     const pm_stage_desc& sd = stages[p];
     StageDev& s = L.st[p];
-    if (sd.n_ops < 1 || sd.n_ops > PM_MAX_LINEARS || !sd.ops) { err = "stage " + std::to_string(p) + ": n_ops must be in [1, " + std::to_string(PM_MAX_LINEARS) + "]"; return PM_ERR_INVALID_ARG; }
+    if (sd.n_ops < 1 || sd.n_ops > PM_MAX_LINEARS + 2 || !sd.ops) { stage_err(p, "bad op count"); return PM_ERR_INVALID_ARG; }
     if (sd.tau_bkwd != 0 || sd.tau_fwd != 2 * (P - (p + 1)) + 1) {
-      err = "stage " + std::to_string(p) + ": the tick schedule realises tau_fwd = 2(P-i)+1, tau_bkwd = 0 only";
+      stage_err(p, "the tick schedule realises tau_fwd = 2(P-i)+1, tau_bkwd = 0 only");
       return PM_ERR_UNSUPPORTED;
     }
-    if (sd.param_offset % PM_ALIGN_ELEMS || sd.param_count % PM_ALIGN_ELEMS) { err = "stage " + std::to_string(p) + ": param_offset/param_count must be multiples of 64"; return PM_ERR_INVALID_ARG; }
+    if (sd.param_offset % PM_ALIGN_ELEMS || sd.param_count % PM_ALIGN_ELEMS) { stage_err(p, "param_offset/param_count must be multiples of 64"); return PM_ERR_INVALID_ARG; }
     if (sd.param_offset < prev_end) { err = "stage slices must ascend without overlap"; return PM_ERR_INVALID_ARG; }
     uint64_t need = 0;
     pm_status ps = pm_stage_param_count(sd.ops, sd.n_ops, &need);
-    if (ps != PM_OK) { err = "stage " + std::to_string(p) + ": bad op list"; return ps; }
-    if (sd.param_count < need) { err = "stage " + std::to_string(p) + ": param_count smaller than its ops need"; return PM_ERR_INVALID_ARG; }
-    s.tau_f = sd.tau_fwd; s.gap = sd.tau_fwd - sd.tau_bkwd; s.n_lin = sd.n_ops;
+    if (ps != PM_OK) { stage_err(p, "bad op list"); return ps; }
+    if (sd.param_count < need) { stage_err(p, "param_count smaller than its ops need"); return PM_ERR_INVALID_ARG; }
+    s.tau_f = sd.tau_fwd; s.gap = sd.tau_fwd - sd.tau_bkwd;
     s.depth = s.tau_f + 1; s.xdepth = s.tau_f + 2;
     s.begin = sd.param_offset; s.end = sd.param_offset + sd.param_count;
     prev_end = s.end;
     L.begin64[p] = (uint32_t)(s.begin / 64); L.end64[p] = (uint32_t)(s.end / 64);
-    s.max_dim = 0;
-    for (int l = 0; l < sd.n_ops; ++l) {
-      const pm_op_desc& op = sd.ops[l];
-      if (op.kind != PM_OP_LINEAR) { err = "only PM_OP_LINEAR is built"; return PM_ERR_UNSUPPORTED; }
-      if (op.n_in < 1 || op.n_out < 1 || op.act < PM_ACT_NONE || op.act > PM_ACT_GELU) { err = "bad Linear description"; return PM_ERR_INVALID_ARG; }
-      if (cfg->compute_dtype == PM_BF16 && (op.n_in % 8 || op.n_out % 8)) { err = "PM_BF16 needs Linear dimensions that are multiples of 8"; return PM_ERR_SHAPE; }
-      if (prev_out >= 0 && op.n_in != prev_out) { err = "stage " + std::to_string(p) + " op " + std::to_string(l) + ": n_in does not match the previous n_out"; return PM_ERR_SHAPE; }
-      prev_out = op.n_out;
-      LinDev& ld = s.lin[l];
-      ld.n_in = op.n_in; ld.n_out = op.n_out; ld.act = op.act;
-      uint64_t wo, bo;
-      pm_op_param_offsets(sd.ops, sd.n_ops, l, &wo, &bo);
-      ld.w_off = s.begin + wo; ld.b_off = s.begin + bo;
-      s.max_dim = std::max(s.max_dim, std::max(op.n_in, op.n_out));
+    // ---- parse [pre] LINEAR+ [post]
+    int idx = 0;
+    s.pre = PRE_NONE; s.post = POST_NONE; s.n_lin = 0;
+    auto offsets = [&](int op, uint64_t* a, uint64_t* b) { pm_op_param_offsets(sd.ops, sd.n_ops, op, a, b); *a += s.begin; *b += s.begin; };
+    if (sd.ops[0].kind == PM_OP_EMBED) {
+      if (p != 0) { stage_err(p, "EMBED belongs to the first stage"); return PM_ERR_UNSUPPORTED; }
+      const pm_op_desc& op = sd.ops[0];
+      if (op.n_in < 1 || op.n_out < 2 || (op.n_out & 1) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (even width, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
+      s.pre = PRE_EMBED; s.vocab = op.n_in; s.seq_len = op.seq_len;
+      uint64_t dummy; offsets(0, &s.tab_off, &dummy);
+      L.pe_seq = op.seq_len; L.pe_d = op.n_out;
+      idx = 1;
+    } else if (sd.ops[0].kind == PM_OP_LAYERNORM) {
+      if (sd.ops[0].n_in < 1 || sd.ops[0].n_in != sd.ops[0].n_out) { stage_err(p, "LAYERNORM needs n_in = n_out"); return PM_ERR_INVALID_ARG; }
+      s.pre = PRE_LN;
+      offsets(0, &s.g_off, &s.beta_off);
+      idx = 1;
     }
-    // rings
-    s.x_ring = ring; ring = align_up(ring + (uint64_t)s.xdepth * T * s.lin[0].n_in * esz, 256);
+    const int pre_width = idx == 1 ? sd.ops[0].n_out : -1;
+    s.max_dim = 0;
+    int max_out = 0, max_in = 0;
+    while (idx < sd.n_ops && sd.ops[idx].kind == PM_OP_LINEAR) {
+      if (s.n_lin == PM_MAX_LINEARS) { stage_err(p, "too many Linear ops"); return PM_ERR_INVALID_ARG; }
+      const pm_op_desc& op = sd.ops[idx];
+      if (op.n_in < 1 || op.n_out < 1 || op.act < PM_ACT_NONE || op.act > PM_ACT_GELU) { stage_err(p, "bad Linear description"); return PM_ERR_INVALID_ARG; }
+      if (cfg->compute_dtype == PM_BF16 && (op.n_in % 8 || op.n_out % 8)) { err = "PM_BF16 needs Linear dimensions that are multiples of 8"; return PM_ERR_SHAPE; }
+      LinDev& ld = s.lin[s.n_lin];
+      ld.n_in = op.n_in; ld.n_out = op.n_out; ld.act = op.act;
+      offsets(idx, &ld.w_off, &ld.b_off);
+      if (s.n_lin > 0 && op.n_in != s.lin[s.n_lin - 1].n_out) { stage_err(p, "Linear n_in does not match the previous n_out"); return PM_ERR_SHAPE; }
+      max_out = std::max(max_out, op.n_out); max_in = std::max(max_in, op.n_in);
+      ++s.n_lin; ++idx;
+    }
+    if (s.n_lin < 1) { stage_err(p, "a stage needs at least one LINEAR"); return PM_ERR_INVALID_ARG; }
+    if (pre_width >= 0 && pre_width != s.lin[0].n_in) { stage_err(p, "pre-op width does not match the Linear's n_in"); return PM_ERR_SHAPE; }
+    if (idx < sd.n_ops) {
+      const pm_op_desc& op = sd.ops[idx];
+      if (op.kind == PM_OP_ATTENTION) {
+        const int n_out = s.lin[s.n_lin - 1].n_out;
+        if (n_out % 3 || op.n_heads < 1 || (n_out / 3) % op.n_heads || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad ATTENTION description"); return PM_ERR_INVALID_ARG; }
+        if (op.seq_len > 128) { stage_err(p, "ATTENTION is built for seq_len <= 128"); return PM_ERR_UNSUPPORTED; }
+        s.post = POST_ATTENTION; s.n_heads = op.n_heads; s.seq_len = op.seq_len;
+      } else if (op.kind == PM_OP_SKIP_OUT) s.post = POST_SKIP_OUT;
+      else if (op.kind == PM_OP_RESIDUAL) s.post = POST_RESIDUAL;
+      else { stage_err(p, "unexpected op after the Linear ops"); return PM_ERR_INVALID_ARG; }
+      ++idx;
+    }
+    if (idx != sd.n_ops) { stage_err(p, "ops must follow [EMBED|LAYERNORM] LINEAR+ [ATTENTION|SKIP_OUT|RESIDUAL]"); return PM_ERR_INVALID_ARG; }
+    if ((s.pre != PRE_NONE || s.post != POST_NONE) && s.n_lin != 1) { stage_err(p, "a stage with a pre- or post-op holds exactly one LINEAR"); return PM_ERR_UNSUPPORTED; }
+    s.d_in = s.lin[0].n_in;
+    const int n_out_last = s.lin[s.n_lin - 1].n_out;
+    s.d_out_main = s.post == POST_ATTENTION ? n_out_last / 3 : n_out_last;
+    s.max_dim = std::max(std::max(max_in, max_out), s.d_in);
+    // ---- chaining
+    if (p > 0) {
+      const StageDev& q = L.st[p - 1];
+      if (s.pre == PRE_EMBED) { stage_err(p, "EMBED belongs to the first stage"); return PM_ERR_UNSUPPORTED; }
+      if (s.d_in != q.d_out_main) { stage_err(p, "input width does not match the previous stage's output"); return PM_ERR_SHAPE; }
+      const bool emits = q.post == POST_ATTENTION || q.post == POST_SKIP_OUT;
+      if (emits != (s.post == POST_RESIDUAL)) { stage_err(p, "RESIDUAL must directly follow a stage ending in ATTENTION or SKIP_OUT, and only then"); return PM_ERR_UNSUPPORTED; }
+      if (s.post == POST_RESIDUAL && q.d_in != n_out_last) { stage_err(p, "skip tensor width does not match the Linear's output"); return PM_ERR_SHAPE; }
+    } else if (s.post == POST_RESIDUAL) { stage_err(p, "the first stage has no skip tensor to add"); return PM_ERR_UNSUPPORTED; }
+    if (p == P - 1 && (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT)) { stage_err(p, "the last stage cannot emit a skip tensor"); return PM_ERR_UNSUPPORTED; }
+    if (p == P - 1 && ce && (s.n_lin != 1 || s.post != POST_NONE || s.lin[0].act != PM_ACT_NONE)) { stage_err(p, "PM_LOSS_CE needs a last stage of one Linear without activation or post-op"); return PM_ERR_UNSUPPORTED; }
+    // ---- what each Linear's forward writes
     for (int l = 0; l < s.n_lin; ++l) {
-      s.lin[l].z_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256);
+      LinDev& ld = s.lin[l];
+      const bool last = l == s.n_lin - 1;
+      const bool logits = last && p == P - 1 && ce;
+      ld.flags = 0;
+      if (ld.act != PM_ACT_NONE || (last && s.post == POST_ATTENTION)) ld.flags |= LF_WRITE_Z;
+      if (!(last && s.post == POST_ATTENTION) && !logits) ld.flags |= LF_WRITE_Y;
+      if (logits) ld.flags |= LF_OUT_F32;
+    }
+    // ---- rings
+    if (s.pre != PRE_EMBED) { s.x_ring = ring; ring = align_up(ring + (uint64_t)s.xdepth * T * s.d_in * esz, 256); }
+    if (s.pre != PRE_NONE) { s.u_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.d_in * esz, 256); }
+    if (s.pre == PRE_LN) { s.stat_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * 2 * 4, 256); }
+    if (s.pre == PRE_EMBED) { s.ids_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * 4, 256); }
+    for (int l = 0; l < s.n_lin; ++l) {
+      if (s.lin[l].flags & LF_WRITE_Z) { s.lin[l].z_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
       if (l < s.n_lin - 1) { s.lin[l].h_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
     }
     L.max_lin = std::max(L.max_lin, s.n_lin);
     L.max_dim = std::max(L.max_dim, s.max_dim);
+    if (s.pre != PRE_NONE) L.any_pre = 1;
+    if (s.pre == PRE_LN) L.any_ln = 1;
+    if (s.pre == PRE_EMBED) { L.any_embed = 1; L.max_vocab = std::max(L.max_vocab, s.vocab); }
+    if (s.post == POST_RESIDUAL) L.any_residual = 1;
+    if (s.post == POST_ATTENTION) {
+      const int dk = s.d_out_main / s.n_heads;
+      L.att_S = std::max(L.att_S, s.seq_len); L.att_dk = std::max(L.att_dk, dk);
+      L.att_blocks = std::max(L.att_blocks, (int)(T / s.seq_len) * s.n_heads);
+    }
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
   }
   for (int p = 0; p < P; ++p) L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
+  if (L.att_blocks > 0 && attention_smem_bytes(L.att_S, L.att_dk) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
   L.ring_bytes = ring;
   L.total = L.st[P - 1].end;
-  L.n_in_first = L.st[0].lin[0].n_in;
+  L.n_in_first = L.st[0].pre == PRE_EMBED ? 0 : L.st[0].lin[0].n_in;
   L.n_out_last = L.st[P - 1].lin[L.st[P - 1].n_lin - 1].n_out;
   L.loss_cap = cfg->loss_log_capacity > 0 ? cfg->loss_log_capacity : 4096;
   // workspace
@@ -109,15 +195,24 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_alpha = w; w = align_up(w + sizeof(double) * (cfg->alpha_by_step ? (uint64_t)cfg->alpha_len : 0), 256);
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
   L.off_lossred = w; w = align_up(w + 512, 256);
-  L.off_tgt = w; w = align_up(w + sizeof(float) * (uint64_t)(P + 1) * T * L.n_out_last, 256);
-  L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * esz, 256);
+  L.off_rowloss = w; w = align_up(w + (ce ? T * 4 : 0), 256);
+  L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
+  L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
+  L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
   L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes(P) : 0), 256);
   for (int p = 0; p < P; ++p) {
     StageDev& s = L.st[p];
-    const int n_out_last = s.lin[s.n_lin - 1].n_out;
-    s.gin = w; w = align_up(w + 2 * T * n_out_last * esz, 256);
-    s.dz = w; w = align_up(w + T * s.max_dim * esz, 256);
-    s.dh = w; w = align_up(w + T * s.max_dim * esz, 256);
+    const uint64_t n_out_last = s.lin[s.n_lin - 1].n_out;
+    uint64_t mo = 0, mi = 0;
+    for (int l = 0; l < s.n_lin; ++l) { mo = std::max<uint64_t>(mo, s.lin[l].n_out); mi = std::max<uint64_t>(mi, s.lin[l].n_in); }
+    s.gin = w; w = align_up(w + 3 * T * s.d_out_main * esz, 256);
+    if (s.post == POST_RESIDUAL) {
+      s.skip_in = w; w = align_up(w + 2 * T * n_out_last * esz, 256);
+      s.ytmp = w; w = align_up(w + T * n_out_last * esz, 256);
+    }
+    if (s.post == POST_ATTENTION) { s.dy = w; w = align_up(w + T * n_out_last * esz, 256); }
+    s.dz = w; w = align_up(w + T * mo * esz, 256);
+    s.dh = w; w = align_up(w + T * mi * esz, 256);
   }
   L.ws_bytes = w;
   return PM_OK;
@@ -172,9 +267,12 @@ pm_status pm_stage_param_count(const pm_op_desc* ops, int32_t n_ops, uint64_t* c
   if (!ops || !count || n_ops < 1) return PM_ERR_INVALID_ARG;
   uint64_t c = 0;
   for (int l = 0; l < n_ops; ++l) {
-    if (ops[l].n_in < 1 || ops[l].n_out < 1) return PM_ERR_INVALID_ARG;
-    c = align_up(c + (uint64_t)ops[l].n_in * ops[l].n_out, PM_ALIGN_ELEMS);
-    c = align_up(c + (uint64_t)ops[l].n_out, PM_ALIGN_ELEMS);
+    if (ops[l].kind < PM_OP_LINEAR || ops[l].kind > PM_OP_RESIDUAL) return PM_ERR_INVALID_ARG;
+    if (ops[l].kind <= PM_OP_LAYERNORM && (ops[l].n_in < 1 || ops[l].n_out < 1)) return PM_ERR_INVALID_ARG;
+    uint64_t n0, n1;
+    const int k = op_params(ops[l], &n0, &n1);
+    if (k >= 1) c = align_up(c + n0, PM_ALIGN_ELEMS);
+    if (k >= 2) c = align_up(c + n1, PM_ALIGN_ELEMS);
   }
   *count = c;
   return PM_OK;
@@ -184,11 +282,17 @@ pm_status pm_op_param_offsets(const pm_op_desc* ops, int32_t n_ops, int32_t op, 
   if (!ops || op < 0 || op >= n_ops) return PM_ERR_INVALID_ARG;
   uint64_t c = 0;
   for (int l = 0; l <= op; ++l) {
-    uint64_t wo = c;
-    c = align_up(c + (uint64_t)ops[l].n_in * ops[l].n_out, PM_ALIGN_ELEMS);
-    uint64_t bo = c;
-    c = align_up(c + (uint64_t)ops[l].n_out, PM_ALIGN_ELEMS);
-    if (l == op) { if (w_off) *w_off = wo; if (b_off) *b_off = bo; }
+    uint64_t n0, n1;
+    const int k = op_params(ops[l], &n0, &n1);
+    const uint64_t o0 = c;
+    if (k >= 1) c = align_up(c + n0, PM_ALIGN_ELEMS);
+    const uint64_t o1 = c;
+    if (k >= 2) c = align_up(c + n1, PM_ALIGN_ELEMS);
+    if (l == op) {
+      if (k == 0) return PM_ERR_INVALID_ARG;
+      if (w_off) *w_off = o0;
+      if (b_off) *b_off = o1;
+    }
   }
   return PM_OK;
 }
@@ -268,6 +372,26 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.n_in_first = L.n_in_first; t.n_out_last = L.n_out_last;
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
+  t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
+  t.any_pre = L.any_pre; t.any_ln = L.any_ln; t.any_embed = L.any_embed; t.any_residual = L.any_residual;
+  t.att_S = L.att_S; t.att_dk = L.att_dk; t.att_blocks = L.att_blocks; t.max_vocab = L.max_vocab;
+  if (L.pe_seq > 0) {
+    // sinusoidal positions: PE[pos, 2i] = sin(pos / 10000^(2i/d)), PE[pos, 2i+1] = cos(same); double, rounded once to float
+    std::vector<float> pe((size_t)L.pe_seq * L.pe_d);
+    for (int pos = 0; pos < L.pe_seq; ++pos)
+      for (int i = 0; i < L.pe_d / 2; ++i) {
+        const double ang = (double)pos / std::pow(10000.0, 2.0 * i / (double)L.pe_d);
+        pe[(size_t)pos * L.pe_d + 2 * i] = (float)std::sin(ang);
+        pe[(size_t)pos * L.pe_d + 2 * i + 1] = (float)std::cos(ang);
+      }
+    e = cudaMemcpyAsync(c->ws + L.off_pe, pe.data(), pe.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "position table upload"); delete c; return r; }
+  }
+  if (L.att_blocks > 0) {
+    e = attention_set_smem_limits(L.att_S, L.att_dk);
+    if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "attention shared-memory limit"); delete c; return r; }
+  }
 
   if (cfg->compute_dtype == PM_BF16) {
     std::string uerr;
@@ -278,9 +402,9 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   return PM_OK;
 }
 
-// every call checked here enqueued exactly one kernel
-static pm_status check(pm_ctx* ctx, cudaError_t e, const char* what) {
-  ctx->launches += 1;
+// every call checked here enqueued `kernels` kernels
+static pm_status check(pm_ctx* ctx, cudaError_t e, const char* what, int kernels = 1) {
+  ctx->launches += kernels;
   return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, what);
 }
 
@@ -301,11 +425,14 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   }
   // forward of every stage whose microbatch exists: s - (i-1) in [0, n_fed)
   if (ctx->tick - (ctx->cfg.n_stages - 1) < ctx->n_fed) {
+    if (ctx->L.any_pre && (s = check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->stream), "embedding / LayerNorm forward")) != PM_OK) return s;
     for (int l = 0; l < ctx->L.max_lin; ++l) {
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 0, l, ctx->stream)
                                    : umma_launch(ctx->umma, ctx->ta, 0, l, ctx->stream);
       if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
     }
+    const int n_post = (ctx->L.att_blocks > 0 ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
+    if (n_post && (s = check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream), "attention / residual forward", n_post)) != PM_OK) return s;
   }
   ctx->phase = 1;
   return PM_OK;
@@ -321,6 +448,7 @@ pm_status pm_backward(pm_ctx* ctx) {
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
     if ((s = check(ctx, launch_loss(ctx->ta, dt, ctx->stream), "loss")) != PM_OK) return s;
+    if (ctx->L.att_blocks > 0 && (s = check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward")) != PM_OK) return s;
     for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
       if ((s = check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward")) != PM_OK) return s;
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->stream)
@@ -330,6 +458,8 @@ pm_status pm_backward(pm_ctx* ctx) {
                        : umma_launch(ctx->umma, ctx->ta, 1, l, ctx->stream);
       if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
     }
+    const int n_pre = pre_bwd_launches(ctx->ta);
+    if (n_pre && (s = check(ctx, launch_pre_bwd(ctx->ta, dt, ctx->stream), "LayerNorm / embedding backward", n_pre)) != PM_OK) return s;
   }
   ctx->phase = 2;
   return PM_OK;

@@ -8,31 +8,41 @@
 namespace pm {
 
 template <typename AT> __device__ __forceinline__ AT* ring_ptr(const TickArgs& t, uint64_t off, int slot, uint64_t slot_elems) {
-  return reinterpret_cast<AT*>(t.ring + off) + (uint64_t)slot * slot_elems;
+  return ring_at<AT>(t, off, slot, slot_elems);
 }
-template <typename AT> __device__ __forceinline__ AT* ws_ptr(const TickArgs& t, uint64_t off) {
-  return reinterpret_cast<AT*>(t.ws + off);
-}
+template <typename AT> __device__ __forceinline__ AT* ws_ptr(const TickArgs& t, uint64_t off) { return ws_at<AT>(t, off); }
 
 // ---- ingest -----------------------------------------------------------------------------------
+// MLP: inputs [T, n_in] (activation type) -> stage 1's input ring slot; targets [T, n_out] float -> target ring.
+// Encoder: token ids [T] int32 -> stage 1's id ring slot; target ids [T] int32 -> target ring.
 template <typename AT>
-__global__ void ingest_kernel(TickArgs t, const AT* __restrict__ inputs, const float* __restrict__ targets, int64_t mb) {
+__global__ void ingest_kernel(TickArgs t, const void* __restrict__ inputs, const void* __restrict__ targets, int64_t mb) {
   const StageDev& s0 = t.st[0];
-  const uint64_t n_x = (uint64_t)t.T * t.n_in_first, n_t = (uint64_t)t.T * t.n_out_last;
-  AT* xdst = ring_ptr<AT>(t, s0.x_ring, (int)(mb % s0.xdepth), n_x);
-  float* tdst = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(mb % (t.P + 1)) * n_t;
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_x + n_t; i += (uint64_t)gridDim.x * blockDim.x) {
-    if (i < n_x) xdst[i] = inputs[i];
-    else tdst[i - n_x] = targets[i - n_x];
+  const uint64_t gid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (uint64_t)gridDim.x * blockDim.x;
+  if (s0.pre == PRE_EMBED) {
+    int32_t* idst = ring_ptr<int32_t>(t, s0.ids_ring, (int)(mb % s0.depth), (uint64_t)t.T);
+    for (uint64_t i = gid; i < (uint64_t)t.T; i += stride) idst[i] = reinterpret_cast<const int32_t*>(inputs)[i];
+  } else {
+    const uint64_t n_x = (uint64_t)t.T * t.n_in_first;
+    AT* xdst = ring_ptr<AT>(t, s0.x_ring, (int)(mb % s0.xdepth), n_x);
+    for (uint64_t i = gid; i < n_x; i += stride) xdst[i] = reinterpret_cast<const AT*>(inputs)[i];
+  }
+  if (t.loss_kind == PM_LOSS_CE) {
+    int32_t* tdst = ws_ptr<int32_t>(t, t.tgt_off) + (uint64_t)(mb % (t.P + 1)) * t.T;
+    for (uint64_t i = gid; i < (uint64_t)t.T; i += stride) tdst[i] = reinterpret_cast<const int32_t*>(targets)[i];
+  } else {
+    const uint64_t n_t = (uint64_t)t.T * t.n_out_last;
+    float* tdst = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(mb % (t.P + 1)) * n_t;
+    for (uint64_t i = gid; i < n_t; i += stride) tdst[i] = reinterpret_cast<const float*>(targets)[i];
   }
 }
 
 cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, const float* targets, int64_t mb, cudaStream_t stream) {
-  uint64_t n = (uint64_t)t.T * (t.n_in_first + t.n_out_last);
+  uint64_t n = (uint64_t)t.T * (t.n_in_first > t.n_out_last ? t.n_in_first : t.n_out_last);
   int blocks = (int)((n + 255) / 256);
   if (blocks > 1184) blocks = 1184;
-  if (dtype == PM_F32) ingest_kernel<float><<<blocks, 256, 0, stream>>>(t, (const float*)inputs, targets, mb);
-  else ingest_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(t, (const __nv_bfloat16*)inputs, targets, mb);
+  if (dtype == PM_F32) ingest_kernel<float><<<blocks, 256, 0, stream>>>(t, inputs, targets, mb);
+  else ingest_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(t, inputs, targets, mb);
   return cudaGetLastError();
 }
 
@@ -51,7 +61,7 @@ __global__ void __launch_bounds__(kLossThreads) mse_loss_kernel(TickArgs t) {
   const int par = (int)((d.tick + 1) & 1);            // written during the previous tick
   const AT* y = ws_ptr<AT>(t, t.yout_off) + (uint64_t)par * n;
   const float* tg = ws_ptr<float>(t, t.tgt_off) + (uint64_t)(d.b_mb % (t.P + 1)) * n;
-  AT* dy = ws_ptr<AT>(t, sl.gin) + (uint64_t)par * n;
+  AT* dy = gin_read<AT>(t, sl, d);
   float* partial = ws_ptr<float>(t, t.lossred_off);
   unsigned int* counter = reinterpret_cast<unsigned int*>(partial + kLossBlocks);
   const float scale = (float)(2.0 / (double)n);
@@ -86,7 +96,10 @@ __global__ void __launch_bounds__(kLossThreads) mse_loss_kernel(TickArgs t) {
   }
 }
 
+cudaError_t launch_ce_loss(const TickArgs& t, int dtype, cudaStream_t stream);   // pm_xfmr.cu
+
 cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream) {
+  if (t.loss_kind == PM_LOSS_CE) return launch_ce_loss(t, dtype, stream);
   if (dtype == PM_F32) mse_loss_kernel<float><<<kLossBlocks, kLossThreads, 0, stream>>>(t);
   else mse_loss_kernel<__nv_bfloat16><<<kLossBlocks, kLossThreads, 0, stream>>>(t);
   return cudaGetLastError();
@@ -120,8 +133,10 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = c0 + 2 * lane;                        // n_out is even whenever a pair straddles nothing: see guard
   const uint64_t n = (uint64_t)t.T * L.n_out;
-  const AT* dy = (lvl == s.n_lin - 1) ? ws_ptr<AT>(t, s.gin) + (uint64_t)((d.tick + 1) & 1) * n : ws_ptr<AT>(t, s.dh);
-  const AT* z = ring_ptr<AT>(t, L.z_ring, d.b_slot, n);
+  const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
+                 : (s.post == POST_ATTENTION ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
+  const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy and no stash is read
+  const AT* z = has_act ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n) : dy;
   AT* dz = ws_ptr<AT>(t, s.dz);
   const bool pair_ok = (L.n_out & 1) == 0;            // vector path needs even row length for alignment
   float s0 = 0.f, s1 = 0.f;
@@ -129,16 +144,16 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
     const uint64_t i = (uint64_t)r * L.n_out + c;
     if (pair_ok && c + 1 < L.n_out) {
       float2 g = Pair<AT>::ld(dy + i), zz = Pair<AT>::ld(z + i);
-      float2 v = make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act))));
+      float2 v = has_act ? make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act)))) : g;
       Pair<AT>::st(dz + i, v);
       s0 = __fadd_rn(s0, v.x); s1 = __fadd_rn(s1, v.y);
     } else {
       if (c < L.n_out) {
-        float v = round_as<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act)));
+        float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act))) : to_f<AT>(dy[i]);
         dz[i] = from_f<AT>(v); s0 = __fadd_rn(s0, v);
       }
       if (c + 1 < L.n_out) {
-        float v = round_as<AT>(__fmul_rn(to_f<AT>(dy[i + 1]), act_grad(to_f<AT>(z[i + 1]), L.act)));
+        float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i + 1]), act_grad(to_f<AT>(z[i + 1]), L.act))) : to_f<AT>(dy[i + 1]);
         dz[i + 1] = from_f<AT>(v); s1 = __fadd_rn(s1, v);
       }
     }
@@ -177,7 +192,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
   const StageDev& s = t.st[p];
   if (lvl >= s.n_lin) return;
   if (MODE == 0 ? d.f_mb < 0 : d.b_mb < 0) return;
-  if (MODE == 1 && p == 0 && lvl == 0) return;        // the network input needs no gradient
+  if (MODE == 1 && p == 0 && lvl == 0 && s.pre != PRE_EMBED) return;   // raw network inputs need no gradient
   const LinDev& L = s.lin[lvl];
   const int T = t.T;
   int M, N, K;
@@ -189,12 +204,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
 
   const uint64_t n_xin = (uint64_t)T * L.n_in, n_xout = (uint64_t)T * L.n_out;
   // operand sources
-  const AT* xin;      // this Linear's input activation (forward slot or backward slot)
-  {
-    const int slot = MODE == 0 ? d.f_slot : d.b_slot;
-    const int xslot = MODE == 0 ? d.f_xslot : d.b_xslot;
-    xin = (lvl == 0) ? ring_ptr<AT>(t, s.x_ring, xslot, n_xin) : ring_ptr<AT>(t, s.lin[lvl - 1].h_ring, slot, n_xin);
-  }
+  const AT* xin = lin_input<AT>(t, s, d, lvl, MODE == 0);   // this Linear's input activation (forward or backward slot)
   const AT* dz = ws_ptr<AT>(t, s.dz);
   const WT* wf;
   if (sizeof(WT) == 4) wf = reinterpret_cast<const WT*>(t.a.w) + L.w_off;
@@ -277,11 +287,9 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
 
   // epilogue
   if (MODE == 0) {
-    AT* zout = ring_ptr<AT>(t, L.z_ring, d.f_slot, n_xout);
-    AT* yout;
-    if (lvl < s.n_lin - 1) yout = ring_ptr<AT>(t, L.h_ring, d.f_slot, n_xout);
-    else if (p < t.P - 1) yout = ring_ptr<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n_xout);
-    else yout = ws_ptr<AT>(t, t.yout_off) + (uint64_t)(d.tick & 1) * n_xout;
+    AT* zout = (L.flags & LF_WRITE_Z) ? ring_ptr<AT>(t, L.z_ring, d.f_slot, n_xout) : nullptr;
+    AT* yout = y_dest<AT>(t, p, s, d, lvl);
+    float* lout = (L.flags & LF_OUT_F32) ? ws_ptr<float>(t, t.yout_off) + (uint64_t)(d.tick & 1) * n_xout : nullptr;
     const float* bias = t.a.w + L.b_off;
 #pragma unroll
     for (int i = 0; i < 4; ++i)
@@ -289,13 +297,15 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
       for (int j = 0; j < 4; ++j) {
         int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
         if (m < M && n < N) {
-          AT zv = from_f<AT>(__fadd_rn(acc[i][j], bias[n]));
-          zout[(uint64_t)m * N + n] = zv;
-          yout[(uint64_t)m * N + n] = from_f<AT>(act_fwd(to_f<AT>(zv), L.act));
+          const float pre_act = __fadd_rn(acc[i][j], bias[n]);
+          if (lout) lout[(uint64_t)m * N + n] = pre_act;          // logits stay fp32
+          AT zv = from_f<AT>(pre_act);
+          if (zout) zout[(uint64_t)m * N + n] = zv;
+          if (yout) yout[(uint64_t)m * N + n] = from_f<AT>(act_fwd(to_f<AT>(zv), L.act));
         }
       }
   } else if (MODE == 1) {
-    AT* dx = (lvl == 0) ? ws_ptr<AT>(t, t.st[p - 1].gin) + (uint64_t)(d.tick & 1) * n_xin : ws_ptr<AT>(t, s.dh);
+    AT* dx = (lvl == 0 && s.pre == PRE_NONE) ? gin_write_prev<AT>(t, p, d) : ws_ptr<AT>(t, s.dh);
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll

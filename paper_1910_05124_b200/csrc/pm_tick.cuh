@@ -13,14 +13,60 @@ struct TickArgs {
   char* ws;
   int32_t T, P;
   int32_t n_in_first, n_out_last;
-  uint64_t yout_off;      // ws: last stage's output [2][T*n_out_last] (activation type)
-  uint64_t tgt_off;       // ws: target ring [P+1][T*n_out_last] float
+  uint64_t yout_off;      // ws: last stage's output [2][T*n_out_last]: activation type (MSE) or fp32 logits (CE)
+  uint64_t tgt_off;       // ws: target ring [P+1]: [T*n_out_last] float (MSE) or [T] int32 (CE)
+  uint64_t pe_off;        // ws: sinusoidal positions [seq_len][d] float (0 if no embedding stage)
+  uint64_t rowloss_off;   // ws: per-token losses [T] float (cross-entropy)
+  int32_t loss_kind;      // PM_LOSS_*
+  int32_t any_pre, any_ln, any_embed, any_residual;   // which grouped launches this pipeline needs
+  int32_t att_S, att_dk, att_blocks;                   // attention: sequence length, head width, (sequences x heads); 0 = none
+  int32_t max_vocab;
   uint64_t loss_off;      // ws: loss log [loss_cap] float
   uint64_t lossred_off;   // ws: per-block loss partials [64] float + completion counter
   int64_t loss_cap;
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages
 };
+
+// ---- where things live (shared by every tick kernel) -----------------------------------------------------
+template <typename AT> __device__ __forceinline__ AT* ring_at(const TickArgs& t, uint64_t off, int slot, uint64_t slot_elems) {
+  return reinterpret_cast<AT*>(t.ring + off) + (uint64_t)slot * slot_elems;
+}
+template <typename AT> __device__ __forceinline__ AT* ws_at(const TickArgs& t, uint64_t off) {
+  return reinterpret_cast<AT*>(t.ws + off);
+}
+// input activation of Linear `lvl` (forward A operand, wgrad B operand); fwd selects this tick's forward or backward slot
+template <typename AT> __device__ __forceinline__ const AT* lin_input(const TickArgs& t, const StageDev& s, const StageDyn& d, int lvl, bool fwd) {
+  const uint64_t n = (uint64_t)t.T * s.lin[lvl].n_in;
+  if (lvl > 0) return ring_at<AT>(t, s.lin[lvl - 1].h_ring, fwd ? d.f_slot : d.b_slot, n);
+  if (s.pre != PRE_NONE) return ring_at<AT>(t, s.u_ring, fwd ? d.f_slot : d.b_slot, n);
+  return ring_at<AT>(t, s.x_ring, fwd ? d.f_xslot : d.b_xslot, n);
+}
+// gradient w.r.t. this stage's main output: written by the next stage during the previous tick
+template <typename AT> __device__ __forceinline__ AT* gin_read(const TickArgs& t, const StageDev& s, const StageDyn& d) {
+  return ws_at<AT>(t, s.gin) + (uint64_t)((d.tick + 2) % 3) * ((uint64_t)t.T * s.d_out_main);
+}
+// where stage p writes the gradient w.r.t. its main input (= stage p-1's main output)
+template <typename AT> __device__ __forceinline__ AT* gin_write_prev(const TickArgs& t, int p, const StageDyn& d) {
+  const StageDev& sp = t.st[p - 1];
+  return ws_at<AT>(t, sp.gin) + (uint64_t)(d.tick % 3) * ((uint64_t)t.T * sp.d_out_main);
+}
+// gradient w.r.t. the skip tensor stage p emitted: it equals the gradient the next (residual) stage received
+// one tick ago for the same microbatch, i.e. what the stage after it wrote two ticks ago
+template <typename AT> __device__ __forceinline__ const AT* gskip_read(const TickArgs& t, int p, const StageDyn& d) {
+  const StageDev& sn = t.st[p + 1];
+  return ws_at<AT>(t, sn.gin) + (uint64_t)((d.tick + 1) % 3) * ((uint64_t)t.T * sn.d_out_main);
+}
+// destination of Linear lvl's activation y in the forward pass (nullptr: not written)
+template <typename AT> __device__ __forceinline__ AT* y_dest(const TickArgs& t, int p, const StageDev& s, const StageDyn& d, int lvl) {
+  const LinDev& L = s.lin[lvl];
+  if (!(L.flags & LF_WRITE_Y)) return nullptr;
+  const uint64_t n = (uint64_t)t.T * L.n_out;
+  if (lvl < s.n_lin - 1) return ring_at<AT>(t, L.h_ring, d.f_slot, n);
+  if (s.post == POST_RESIDUAL) return ws_at<AT>(t, s.ytmp);
+  if (p < t.P - 1) return ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
+  return ws_at<AT>(t, t.yout_off) + (uint64_t)(d.tick & 1) * n;
+}
 
 // inputs/targets -> stage 1's input ring slot and the target ring (activation type AT = float | bf16).
 cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, const float* targets, int64_t mb,
@@ -29,6 +75,15 @@ cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, cons
 cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream);
 // dz = dy * act'(z) and db = column sums, level `lvl` of every stage that runs backward this tick.
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream);
+
+// Transformer pieces (all grouped over the stages that carry the op this tick).
+cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream);        // embedding / LayerNorm forward (+ skip hand-over)
+cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream);       // attention forward, residual add
+cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream);       // attention backward
+cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream);        // LayerNorm / embedding backward
+int pre_bwd_launches(const TickArgs& t);
+size_t attention_smem_bytes(int S, int dk);
+cudaError_t attention_set_smem_limits(int S, int dk);
 
 // fp32 SIMT grouped GEMMs (PM_F32 path).  mode: 0 forward, 1 dgrad (corrected weights), 2 wgrad.
 cudaError_t launch_simt_gemm(const TickArgs& t, int dtype, int mode, int lvl, cudaStream_t stream);

@@ -185,7 +185,7 @@ __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __rest
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
-  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0);
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
   const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
   else if (MODE == 1) { r.M = t.T; r.N = L.n_in; r.K = L.n_out; }
@@ -272,14 +272,14 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * op.idx;
           if (MODE == 0) {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-            tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, lvl == 0 ? d.f_xslot : d.f_slot);
+            tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.f_xslot : d.f_slot);
             tma_load_2d(sb, lm + MAP_W_K, fb, k0, tl.n0);
           } else if (MODE == 1) {
             mbar_arrive_expect_tx(fb, A_BYTES);
             tma_load_2d(sa, lm + MAP_DZ_K, fb, k0, tl.m0);
           } else {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-            const int slot = lvl == 0 ? d.b_xslot : d.b_slot;
+            const int slot = (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.b_xslot : d.b_slot;
             tma_load_2d(sa, lm + MAP_DZ_MN, fb, tl.m0, k0);
             tma_load_2d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, tl.m0 + 64, k0);
             tma_load_3d(sb, lm + MAP_ACT_MN, fb, tl.n0, k0, slot);
@@ -418,6 +418,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       if (mrow >= tl.M || nb >= tl.N) continue;                       // nothing of this block is inside the tensor
       if (MODE == 0) {
         const float* bias = t.a.w + L.b_off;
+        const bool f32out = (L.flags & LF_OUT_F32) != 0;
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const int n = nb + g * 8;
@@ -426,16 +427,25 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
             const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
             bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
           }
-          float zf[8], yf[8];
+          float pf[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const uint32_t a = g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e];
-            zf[e] = __bfloat162float(__float2bfloat16_rn(__fadd_rn(__uint_as_float(a), bb[e])));
-            yf[e] = act_fwd(zf[e], L.act);
+          for (int e = 0; e < 8; ++e) pf[e] = __fadd_rn(__uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]), bb[e]);
+          if (f32out) {
+            // fp32 logits: two 32-column boxes per warp, eight 16-byte chunks per row each
+            uint8_t* box = obuf + (g >> 2) * 4096;
+            *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2) ^ sw) << 4)) = make_float4(pf[0], pf[1], pf[2], pf[3]);
+            *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
+          } else {
+            float zf[8], yf[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              zf[e] = __bfloat162float(__float2bfloat16_rn(pf[e]));
+              yf[e] = act_fwd(zf[e], L.act);
+            }
+            const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
+            *reinterpret_cast<uint4*>(obuf + off) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
+            *reinterpret_cast<uint4*>(obuf + 4096 + off) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
           }
-          const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
-          *reinterpret_cast<uint4*>(obuf + off) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
-          *reinterpret_cast<uint4*>(obuf + 4096 + off) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
         }
       } else if (MODE == 1) {
 #pragma unroll
@@ -457,11 +467,19 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       __syncwarp();
       if (lane == 0) {
         if (MODE == 0) {
-          tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
-          const int yslot = lvl < s.n_lin - 1 ? d.f_slot : (tl.p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1));
-          tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
+          if (L.flags & LF_OUT_F32) {
+            tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
+            if (nb + 32 < tl.N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
+          } else {
+            if (L.flags & LF_WRITE_Z) tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
+            if (L.flags & LF_WRITE_Y) {
+              const int yslot = lvl < s.n_lin - 1 ? d.f_slot
+                                : (s.post == POST_RESIDUAL ? 0 : (tl.p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
+              tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
+            }
+          }
         } else if (MODE == 1) {
-          tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, lvl == 0 ? (int)(d.tick & 1) : 0);
+          tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0);
         } else {
           tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
           if (nb + 32 < tl.N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
@@ -533,8 +551,9 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       const LinDev& L = s.lin[l];
       CUtensorMap* m = maps.data() + ((size_t)p * PM_MAX_LINEARS + l) * MAPS_PER_LINEAR;
       // input activation of this Linear: ring [slots][T][n_in]
-      char* act_base = t.ring + (l == 0 ? s.x_ring : s.lin[l - 1].h_ring);
-      const uint64_t slots = l == 0 ? (uint64_t)s.xdepth : (uint64_t)s.depth;
+      const bool in_is_x = l == 0 && s.pre == PRE_NONE;
+      char* act_base = t.ring + (l > 0 ? s.lin[l - 1].h_ring : (in_is_x ? s.x_ring : s.u_ring));
+      const uint64_t slots = in_is_x ? (uint64_t)s.xdepth : (uint64_t)s.depth;
       const uint64_t n_in = (uint64_t)L.n_in, n_out = (uint64_t)L.n_out;
       bool okm = true;
       {
@@ -560,16 +579,24 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         // outputs: 32-row boxes of one 128-byte swizzle row (64 bf16 or 32 fp32 columns)
         uint32_t box_bf[3] = {64, 32, 1}, box_f32[2] = {32, 32};
         uint64_t zd[3] = {n_out, T, (uint64_t)s.depth}, zs[2] = {n_out * 2, T * n_out * 2};
-        okm = okm && encode(fn, m + MAP_Z_OUT, 1, t.ring + L.z_ring, 3, zd, zs, box_bf, err);
-        char* ybase; uint64_t yslots;
-        if (l < s.n_lin - 1) { ybase = t.ring + L.h_ring; yslots = (uint64_t)s.depth; }
-        else if (p < P - 1) { ybase = t.ring + st[p + 1].x_ring; yslots = (uint64_t)st[p + 1].xdepth; }
-        else { ybase = t.ws + t.yout_off; yslots = 2; }
-        uint64_t yd[3] = {n_out, T, yslots};
-        okm = okm && encode(fn, m + MAP_Y_OUT, 1, ybase, 3, yd, zs, box_bf, err);
-        if (!(p == 0 && l == 0)) {
-          char* xbase = l == 0 ? t.ws + st[p - 1].gin : t.ws + s.dh;
-          uint64_t xd[3] = {n_in, T, (uint64_t)(l == 0 ? 2 : 1)}, xs[2] = {n_in * 2, T * n_in * 2};
+        if (L.flags & LF_WRITE_Z) okm = okm && encode(fn, m + MAP_Z_OUT, 1, t.ring + L.z_ring, 3, zd, zs, box_bf, err);
+        if (L.flags & LF_OUT_F32) {
+          uint64_t ld[3] = {n_out, T, 2}, ls[2] = {n_out * 4, T * n_out * 4};
+          uint32_t box3[3] = {32, 32, 1};
+          okm = okm && encode(fn, m + MAP_Y_OUT, 2, t.ws + t.yout_off, 3, ld, ls, box3, err);
+        } else if (L.flags & LF_WRITE_Y) {
+          char* ybase; uint64_t yslots;
+          if (l < s.n_lin - 1) { ybase = t.ring + L.h_ring; yslots = (uint64_t)s.depth; }
+          else if (s.post == POST_RESIDUAL) { ybase = t.ws + s.ytmp; yslots = 1; }
+          else if (p < P - 1) { ybase = t.ring + st[p + 1].x_ring; yslots = (uint64_t)st[p + 1].xdepth; }
+          else { ybase = t.ws + t.yout_off; yslots = 2; }
+          uint64_t yd[3] = {n_out, T, yslots};
+          okm = okm && encode(fn, m + MAP_Y_OUT, 1, ybase, 3, yd, zs, box_bf, err);
+        }
+        if (!(p == 0 && l == 0 && s.pre != PRE_EMBED)) {
+          const bool to_prev = l == 0 && s.pre == PRE_NONE;
+          char* xbase = to_prev ? t.ws + st[p - 1].gin : t.ws + s.dh;
+          uint64_t xd[3] = {n_in, T, (uint64_t)(to_prev ? 3 : 1)}, xs[2] = {n_in * 2, T * n_in * 2};
           okm = okm && encode(fn, m + MAP_DX_OUT, 1, xbase, 3, xd, xs, box_bf, err);
         }
         uint64_t wd[2] = {n_in, n_out}, wst[1] = {n_in * 4};

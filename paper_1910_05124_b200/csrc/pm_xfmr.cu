@@ -1,0 +1,502 @@
+// Transformer pieces of a pipeline tick: embedding, LayerNorm, multi-head attention, residual add and
+// cross-entropy, forward and backward.  Every kernel is grouped over the stages (blockIdx.y) and acts only
+// on stages that carry the op and are active this tick.
+//
+// Which weight value is read where (Section 2.1: forward pass reads the forward weights, backward pass the
+// backward weights): the embedding table and the LayerNorm gain/bias are read in the forward pass; the
+// backward pass reads only the LayerNorm gain, in dx_hat = dy * gain, and takes it T2-corrected
+// (gain - gap * delta).  Parameter gradients use stashed forward quantities only.
+#include "pm_tick.cuh"
+
+namespace pm {
+
+constexpr float LN_EPS = 1e-5f;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+template <typename AT> __device__ __forceinline__ const AT* table_ptr(const TickArgs& t);
+template <> __device__ __forceinline__ const float* table_ptr<float>(const TickArgs& t) { return t.a.w; }
+template <> __device__ __forceinline__ const __nv_bfloat16* table_ptr<__nv_bfloat16>(const TickArgs& t) { return t.a.w_lp; }
+
+// ---- pre-op forward: embedding or LayerNorm, one warp per row ------------------------------------------------
+//   embedding: u = table[id] * sqrt(d) + PE[position]     (table in the GEMM operand type)
+//   LayerNorm: mean, biased variance, rstd = 1/sqrt(var + eps) in fp32; u = xhat * gain + bias (fp32 master values)
+// If the stage emits a skip tensor (attention / skip_out) u is also written to the next stage's skip buffer.
+template <typename AT>
+__global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.f_mb < 0 || s.pre == PRE_NONE) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= t.T) return;
+  const int dm = s.d_in;
+  const uint64_t n = (uint64_t)t.T * dm;
+  AT* u = ring_at<AT>(t, s.u_ring, d.f_slot, n) + (uint64_t)row * dm;
+  AT* skip = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT)
+                 ? ws_at<AT>(t, t.st[p + 1].skip_in) + (uint64_t)(d.tick & 1) * n + (uint64_t)row * dm : nullptr;
+  if (s.pre == PRE_EMBED) {
+    const int32_t id = ring_at<int32_t>(t, s.ids_ring, d.f_slot, (uint64_t)t.T)[row];
+    const AT* e = table_ptr<AT>(t) + s.tab_off + (uint64_t)id * dm;
+    const float* pe = ws_at<float>(t, t.pe_off) + (uint64_t)(row % s.seq_len) * dm;
+    const float sc = sqrtf((float)dm);
+    for (int c = lane; c < dm; c += 32) {
+      AT v = from_f<AT>(__fadd_rn(__fmul_rn(to_f<AT>(e[c]), sc), pe[c]));
+      u[c] = v;
+      if (skip) skip[c] = v;
+    }
+    return;
+  }
+  const AT* x = ring_at<AT>(t, s.x_ring, d.f_xslot, n) + (uint64_t)row * dm;
+  float sum = 0.f;
+  for (int c = lane; c < dm; c += 32) sum += to_f<AT>(x[c]);
+  const float mu = warp_sum(sum) / (float)dm;
+  float sq = 0.f;
+  for (int c = lane; c < dm; c += 32) { float v = to_f<AT>(x[c]) - mu; sq += v * v; }
+  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)dm + LN_EPS);
+  const float* g = t.a.w + s.g_off;
+  const float* b = t.a.w + s.beta_off;
+  for (int c = lane; c < dm; c += 32) {
+    AT v = from_f<AT>(__fadd_rn(__fmul_rn(__fmul_rn(to_f<AT>(x[c]) - mu, rstd), g[c]), b[c]));
+    u[c] = v;
+    if (skip) skip[c] = v;
+  }
+  if (lane == 0) {
+    float* st = ring_at<float>(t, s.stat_ring, d.f_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
+    st[0] = mu; st[1] = rstd;
+  }
+}
+
+cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
+  dim3 grid((t.T + 7) / 8, t.P);
+  if (dtype == PM_F32) pre_fwd_kernel<float><<<grid, 256, 0, stream>>>(t);
+  else pre_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
+  return cudaGetLastError();
+}
+
+// ---- residual add: next stage's input = skip + y --------------------------------------------------------------
+template <typename AT>
+__global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.f_mb < 0 || s.post != POST_RESIDUAL) return;
+  const uint64_t n = (uint64_t)t.T * s.d_out_main;
+  const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)((d.tick + 1) & 1) * n;     // written by the previous stage last tick
+  const AT* y = ws_at<AT>(t, s.ytmp);
+  AT* out = ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
+    out[i] = from_f<AT>(__fadd_rn(to_f<AT>(skip[i]), to_f<AT>(y[i])));
+}
+
+// ---- multi-head self-attention, one block per (sequence, head) -----------------------------------------------
+// s = q k^T / sqrt(d_k); p~ = exp(s - rowmax); l = sum p~ (unrounded); O = (round(p~) V) / l.
+// Whole score matrix in shared memory (S <= 128): the softmax is exact over the full row.
+struct AttnShape { int S, dk, d; };
+
+template <typename AT>
+__global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t, int causal) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.f_mb < 0 || s.post != POST_ATTENTION) return;
+  const int S = s.seq_len, H = s.n_heads, dm = s.d_out_main, dk = dm / H;
+  const int n_seq = t.T / S;
+  if ((int)blockIdx.x >= n_seq * H) return;
+  const int b = blockIdx.x / H, h = blockIdx.x % H;
+  extern __shared__ float sm[];
+  float* Q = sm;                       // [S][dk+1]
+  float* K = Q + S * (dk + 1);
+  float* V = K + S * (dk + 1);
+  float* Pm = V + S * (dk + 1);        // [S][S+1]
+  float* Ls = Pm + S * (S + 1);        // [S]
+  const int ld = dk + 1, lp = S + 1;
+  const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
+  const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.f_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
+  for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
+    const int r = i / dk, c = i % dk;
+    const AT* row = qkv + (uint64_t)r * 3 * dm;
+    Q[r * ld + c] = to_f<AT>(row[c]);
+    K[r * ld + c] = to_f<AT>(row[dm + c]);
+    V[r * ld + c] = to_f<AT>(row[2 * dm + c]);
+  }
+  __syncthreads();
+  const float scale = 1.0f / sqrtf((float)dk);
+  for (int i = threadIdx.x; i < S * S; i += blockDim.x) {
+    const int r = i / S, c = i % S;
+    float acc = 0.f;
+    for (int k = 0; k < dk; ++k) acc = fmaf(Q[r * ld + k], K[c * ld + k], acc);
+    Pm[r * lp + c] = (causal && c > r) ? -INFINITY : acc * scale;
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = warp; r < S; r += 8) {
+    float mx = -INFINITY;
+    for (int c = lane; c < S; c += 32) mx = fmaxf(mx, Pm[r * lp + c]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int c = lane; c < S; c += 32) {
+      float e = expf(Pm[r * lp + c] - mx);
+      sum += e;
+      Pm[r * lp + c] = round_as<AT>(e);
+    }
+    sum = warp_sum(sum);
+    if (lane == 0) Ls[r] = sum;
+  }
+  __syncthreads();
+  const uint64_t no = (uint64_t)t.T * dm;
+  AT* out = ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, no) + (uint64_t)b * S * dm + h * dk;
+  for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
+    const int r = i / dk, c = i % dk;
+    float acc = 0.f;
+    for (int j = 0; j < S; ++j) acc = fmaf(Pm[r * lp + j], V[j * ld + c], acc);
+    out[(uint64_t)r * dm + c] = from_f<AT>(acc / Ls[r]);
+  }
+}
+
+static size_t attn_fwd_smem(int S, int dk) { return sizeof(float) * (3 * (size_t)S * (dk + 1) + (size_t)S * (S + 1) + S); }
+static size_t attn_bwd_smem(int S, int dk) { return sizeof(float) * (4 * (size_t)S * (dk + 1) + 2 * (size_t)S * (S + 1) + S); }
+
+size_t attention_smem_bytes(int S, int dk) { return attn_bwd_smem(S, dk); }
+
+cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
+  int S = 0, dk = 0, nblk = 0;
+  bool any_res = false, any_att = false;
+  // the shapes are uniform over stages in the supported workloads; the host keeps the maxima in TickArgs
+  S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0; any_res = t.any_residual != 0;
+  cudaError_t e = cudaSuccess;
+  if (any_att) {
+    dim3 grid(nblk, t.P);
+    size_t smem = attn_fwd_smem(S, dk);
+    if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, smem, stream>>>(t, 0);
+    else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(t, 0);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  if (any_res) {
+    dim3 grid(296, t.P);
+    if (dtype == PM_F32) residual_kernel<float><<<grid, 256, 0, stream>>>(t);
+    else residual_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+// ---- attention backward ------------------------------------------------------------------------------------------
+// P recomputed as in the forward pass.  dV = round(P)^T dO; dP = dO V^T; dS = round(P * (dP - rowsum(dP * P)));
+// dQ = dS K / sqrt(d_k); dK = dS^T Q / sqrt(d_k).  Results go to the stage's dy buffer as [dq | dk | dv].
+template <typename AT>
+__global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int causal) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.post != POST_ATTENTION) return;
+  const int S = s.seq_len, H = s.n_heads, dm = s.d_out_main, dk = dm / H;
+  const int n_seq = t.T / S;
+  if ((int)blockIdx.x >= n_seq * H) return;
+  const int b = blockIdx.x / H, h = blockIdx.x % H;
+  extern __shared__ float sm[];
+  const int ld = dk + 1, lp = S + 1;
+  float* Q = sm;
+  float* K = Q + S * ld;
+  float* V = K + S * ld;
+  float* dO = V + S * ld;
+  float* Pm = dO + S * ld;             // [S][S+1] softmax probabilities (fp32)
+  float* Dm = Pm + S * lp;             // [S][S+1] dP, then dS
+  float* Ls = Dm + S * lp;
+  const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
+  const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.b_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
+  const AT* go = gin_read<AT>(t, s, d) + (uint64_t)b * S * dm + h * dk;
+  for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
+    const int r = i / dk, c = i % dk;
+    const AT* row = qkv + (uint64_t)r * 3 * dm;
+    Q[r * ld + c] = to_f<AT>(row[c]);
+    K[r * ld + c] = to_f<AT>(row[dm + c]);
+    V[r * ld + c] = to_f<AT>(row[2 * dm + c]);
+    dO[r * ld + c] = to_f<AT>(go[(uint64_t)r * dm + c]);
+  }
+  __syncthreads();
+  const float scale = 1.0f / sqrtf((float)dk);
+  for (int i = threadIdx.x; i < S * S; i += blockDim.x) {
+    const int r = i / S, c = i % S;
+    float acc = 0.f, accd = 0.f;
+    for (int k = 0; k < dk; ++k) {
+      acc = fmaf(Q[r * ld + k], K[c * ld + k], acc);
+      accd = fmaf(dO[r * ld + k], V[c * ld + k], accd);
+    }
+    Pm[r * lp + c] = (causal && c > r) ? -INFINITY : acc * scale;
+    Dm[r * lp + c] = accd;                                     // dP
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = warp; r < S; r += 8) {
+    float mx = -INFINITY;
+    for (int c = lane; c < S; c += 32) mx = fmaxf(mx, Pm[r * lp + c]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int c = lane; c < S; c += 32) { float e = expf(Pm[r * lp + c] - mx); sum += e; Pm[r * lp + c] = e; }
+    sum = warp_sum(sum);
+    float dsum = 0.f;
+    for (int c = lane; c < S; c += 32) { float pr = Pm[r * lp + c] / sum; Pm[r * lp + c] = pr; dsum += Dm[r * lp + c] * pr; }
+    dsum = warp_sum(dsum);
+    for (int c = lane; c < S; c += 32) Dm[r * lp + c] = round_as<AT>(Pm[r * lp + c] * (Dm[r * lp + c] - dsum));   // dS
+  }
+  __syncthreads();
+  AT* dy = ws_at<AT>(t, s.dy) + (uint64_t)b * S * 3 * dm + h * dk;
+  for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
+    const int r = i / dk, c = i % dk;
+    float aq = 0.f, ak = 0.f, av = 0.f;
+    for (int j = 0; j < S; ++j) {
+      aq = fmaf(Dm[r * lp + j], K[j * ld + c], aq);            // dQ[r] = sum_j dS[r][j] K[j]
+      ak = fmaf(Dm[j * lp + r], Q[j * ld + c], ak);            // dK[r] = sum_j dS[j][r] Q[j]
+      av = fmaf(round_as<AT>(Pm[j * lp + r]), dO[j * ld + c], av);   // dV[r] = sum_j P[j][r] dO[j]
+    }
+    AT* row = dy + (uint64_t)r * 3 * dm;
+    row[c] = from_f<AT>(aq * scale);
+    row[dm + c] = from_f<AT>(ak * scale);
+    row[2 * dm + c] = from_f<AT>(av);
+  }
+}
+
+cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
+  if (t.att_blocks <= 0) return cudaSuccess;
+  dim3 grid(t.att_blocks, t.P);
+  size_t smem = attn_bwd_smem(t.att_S, t.att_dk);
+  if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, smem, stream>>>(t, 0);
+  else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(t, 0);
+  return cudaGetLastError();
+}
+
+cudaError_t attention_set_smem_limits(int S, int dk) {
+  cudaError_t e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk));
+  return e;
+}
+
+// ---- cross-entropy at the last stage -------------------------------------------------------------------------------
+// One block per token: lse = max + log(sum exp(logit - max)); loss_t = lse - logit[target];
+// dlogits = (softmax - onehot) / T in the activation type, written where the last stage reads its incoming
+// gradient.  The last block to finish adds the per-token losses in token order.
+template <typename AT>
+__global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
+  const StageDyn& d = t.dyn[t.P - 1];
+  if (d.b_mb < 0) return;
+  const StageDev& sl = t.st[t.P - 1];
+  const int V = t.n_out_last, row = blockIdx.x;
+  const uint64_t n = (uint64_t)t.T * V;
+  const float* lg = ws_at<float>(t, t.yout_off) + (uint64_t)((d.tick + 1) & 1) * n + (uint64_t)row * V;
+  const int32_t tgt = (ws_at<int32_t>(t, t.tgt_off) + (uint64_t)(d.b_mb % (t.P + 1)) * t.T)[row];
+  AT* dl = gin_read<AT>(t, sl, d) + (uint64_t)row * V;
+  __shared__ float red[8];
+  __shared__ float bc;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, lg[c]);
+  mx = warp_max(mx);
+  if (lane == 0) red[warp] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) { float m = red[0]; for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i]); bc = m; }
+  __syncthreads();
+  mx = bc;
+  float sum = 0.f;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) sum += expf(lg[c] - mx);
+  sum = warp_sum(sum);
+  __syncthreads();
+  if (lane == 0) red[warp] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) { float a = 0.f; for (int i = 0; i < 8; ++i) a += red[i]; bc = a; }
+  __syncthreads();
+  sum = bc;
+  const float invT = 1.0f / (float)t.T;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) {
+    float pr = expf(lg[c] - mx) / sum;
+    if (c == tgt) pr -= 1.0f;
+    dl[c] = from_f<AT>(pr * invT);
+  }
+  float* rowloss = ws_at<float>(t, t.rowloss_off);
+  unsigned int* counter = reinterpret_cast<unsigned int*>(ws_at<float>(t, t.lossred_off) + 64);
+  __shared__ bool last;
+  if (threadIdx.x == 0) {
+    rowloss[row] = (mx + logf(sum)) - lg[tgt];
+    __threadfence();
+    last = atomicAdd(counter, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (last && threadIdx.x == 0) {
+    __threadfence();
+    float a = 0.f;
+    for (int r = 0; r < t.T; ++r) a += reinterpret_cast<volatile float*>(rowloss)[r];
+    ws_at<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = a / (float)t.T;
+    *counter = 0;
+  }
+}
+
+cudaError_t launch_ce_loss(const TickArgs& t, int dtype, cudaStream_t stream) {
+  if (dtype == PM_F32) ce_loss_kernel<float><<<t.T, 256, 0, stream>>>(t);
+  else ce_loss_kernel<__nv_bfloat16><<<t.T, 256, 0, stream>>>(t);
+  return cudaGetLastError();
+}
+
+// ---- pre-op backward --------------------------------------------------------------------------------------------
+// du_total = du (dgrad output of the first Linear) + gradient of the skip tensor the stage emitted, if any.
+template <typename AT>
+__device__ __forceinline__ float du_total(const AT* du, const AT* gs, uint64_t i) {
+  float v = to_f<AT>(du[i]);
+  if (gs) v = __fadd_rn(v, to_f<AT>(gs[i]));
+  return v;
+}
+
+// LayerNorm input gradient, one warp per row:
+//   dxhat = du_total * gain_b (gain_b = gain - gap*delta: T2);  dx = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat*xhat))
+template <typename AT>
+__global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.pre != PRE_LN || p == 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= t.T) return;
+  const int dm = s.d_in;
+  const uint64_t n = (uint64_t)t.T * dm, ro = (uint64_t)row * dm;
+  const AT* du = ws_at<AT>(t, s.dh);
+  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n) + ro;
+  const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
+  const float mu = st[0], rstd = st[1];
+  const float* g = t.a.w + s.g_off;
+  const float* dl = t.a.delta + s.g_off;
+  const float gapf = (float)s.gap;
+  const bool corr = d.use_delta != 0;
+  float s1 = 0.f, s2 = 0.f;
+  for (int c = lane; c < dm; c += 32) {
+    float gb = g[c];
+    if (corr) gb = __fsub_rn(gb, __fmul_rn(gapf, dl[c]));
+    const float xh = (to_f<AT>(x[c]) - mu) * rstd;
+    const float dxh = du_total<AT>(du, gs, ro + c) * gb;
+    s1 += dxh; s2 += dxh * xh;
+  }
+  s1 = warp_sum(s1) / (float)dm;
+  s2 = warp_sum(s2) / (float)dm;
+  AT* out = gin_write_prev<AT>(t, p, d) + ro;
+  for (int c = lane; c < dm; c += 32) {
+    float gb = g[c];
+    if (corr) gb = __fsub_rn(gb, __fmul_rn(gapf, dl[c]));
+    const float xh = (to_f<AT>(x[c]) - mu) * rstd;
+    const float dxh = du_total<AT>(du, gs, ro + c) * gb;
+    out[c] = from_f<AT>(rstd * (dxh - s1 - xh * s2));
+  }
+}
+
+// LayerNorm parameter gradients: dgain[c] = sum_rows du_total * xhat, dbias[c] = sum_rows du_total.
+// A block owns 32 columns; warp w takes rows w, w+8, ... ascending; per-warp partials are added in warp order.
+template <typename AT>
+__global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.pre != PRE_LN) return;
+  const int dm = s.d_in;
+  const int c = blockIdx.x * 32 + (threadIdx.x & 31);
+  if (blockIdx.x * 32 >= dm) return;
+  const int warp = threadIdx.x >> 5;
+  const uint64_t n = (uint64_t)t.T * dm;
+  const AT* du = ws_at<AT>(t, s.dh);
+  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n);
+  const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
+  float ag = 0.f, ab = 0.f;
+  if (c < dm)
+    for (int r = warp; r < t.T; r += 8) {
+      const uint64_t i = (uint64_t)r * dm + c;
+      const float v = du_total<AT>(du, gs, i);
+      const float xh = (to_f<AT>(x[i]) - st[2 * r]) * st[2 * r + 1];
+      ag = __fadd_rn(ag, __fmul_rn(v, xh));
+      ab = __fadd_rn(ab, v);
+    }
+  __shared__ float rg[8][32], rb[8][32];
+  rg[warp][threadIdx.x & 31] = ag;
+  rb[warp][threadIdx.x & 31] = ab;
+  __syncthreads();
+  if (threadIdx.x < 32 && c < dm) {
+    float a = 0.f, b2 = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, rg[w][threadIdx.x]); b2 = __fadd_rn(b2, rb[w][threadIdx.x]); }
+    t.a.grad[s.g_off + c] = a;
+    t.a.grad[s.beta_off + c] = b2;
+  }
+}
+
+// Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
+// One warp per vocabulary row, so the order of the additions is fixed and every row is written (zeros included).
+template <typename AT>
+__global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.pre != PRE_EMBED) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int v = blockIdx.x * 8 + warp;
+  if (v >= s.vocab) return;
+  const int dm = s.d_in;
+  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
+  const AT* du = ws_at<AT>(t, s.dh);
+  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
+  const float sc = sqrtf((float)dm);
+  for (int c0 = 0; c0 < dm; c0 += 32 * 8) {                 // up to 8 columns per lane per pass
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int tb = 0; tb < t.T; tb += 32) {
+      const int tok = tb + lane;
+      unsigned hit = __ballot_sync(0xffffffffu, tok < t.T && ids[tok] == v);
+      while (hit) {
+        const int j = __ffs(hit) - 1;
+        hit &= hit - 1;
+        const uint64_t ro = (uint64_t)(tb + j) * dm;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int c = c0 + e * 32 + lane;
+          if (c < dm) acc[e] = __fadd_rn(acc[e], __fmul_rn(du_total<AT>(du, gs, ro + c), sc));
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int c = c0 + e * 32 + lane;
+      if (c < dm) out[c] = acc[e];
+    }
+  }
+}
+
+int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? 2 : 0) + (t.any_embed ? 1 : 0); }
+
+cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
+  cudaError_t e = cudaSuccess;
+  if (t.any_ln) {
+    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + 31) / 32, t.P);
+    if (dtype == PM_F32) { ln_bwd_dx_kernel<float><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<float><<<g2, 256, 0, stream>>>(t); }
+    else { ln_bwd_dx_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(t); }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  if (t.any_embed) {
+    dim3 g((t.max_vocab + 7) / 8, t.P);
+    if (dtype == PM_F32) embed_bwd_kernel<float><<<g, 256, 0, stream>>>(t);
+    else embed_bwd_kernel<__nv_bfloat16><<<g, 256, 0, stream>>>(t);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+}  // namespace pm

@@ -12,15 +12,22 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
     import torch
     import paper_1910_05124_b200 as pm
     pipe = pm.Pipeline(wl, params0)
-    P = len(wl.stages)
-    teacher = I.teacher_params(wl) if teacher is None else teacher
+    P = wl.n_stages
+    encoder = wl.kind == "encoder"
+    if not encoder:
+        teacher = I.teacher_params(wl) if teacher is None else teacher
     book = {}
     in_dtype = torch.bfloat16 if wl.compute == "bf16" else torch.float32
     for s in range(n_steps + 2 * P - 1):
         if s < n_steps:
-            x, y = I.batch(wl, s, teacher)
-            xd = torch.from_numpy(x).to(pipe.device).to(in_dtype)
-            yd = torch.from_numpy(y).to(pipe.device)
+            if encoder:
+                ids, tg = I.token_batch(wl, s)
+                xd = torch.from_numpy(ids.astype(np.int32)).to(pipe.device)
+                yd = torch.from_numpy(tg.astype(np.int32)).to(pipe.device)
+            else:
+                x, y = I.batch(wl, s, teacher)
+                xd = torch.from_numpy(x).to(pipe.device).to(in_dtype)
+                yd = torch.from_numpy(y).to(pipe.device)
             pipe.pm_step(xd, yd)
         else:
             pipe.pm_step(None, None)
@@ -38,6 +45,9 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
 
 
 def run_oracle(wl, params0, n_steps, teacher=None):
+    if wl.kind == "encoder":
+        from oracle import transformer
+        return transformer.run_workload(wl, params0, lambda t: I.token_batch(wl, t), n_steps=n_steps)
     from oracle.mlp import run_workload
     teacher = I.teacher_params(wl) if teacher is None else teacher
     return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps)
@@ -50,9 +60,34 @@ def max_rel_err(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
 
 
-def compare_params(pipe, res, tol):
+def compare_params(pipe, res, tol, per_stage=False):
+    """per_stage: measure max |dw| against the largest weight of the whole stage vector (w_t)_i instead of the
+    tensor's own largest entry.  Used for bf16 + Adam, where the step of an element is about alpha whatever the
+    size of its gradient: an element whose gradient sign is decided by bf16 rounding noise moves by +-alpha per
+    step on either side, which is large against a bias vector that is itself only a few alpha in size."""
     worst = 0.0
     got = pipe.unpack(pipe.w)
+    if pipe.is_encoder:
+        wl = pipe.wl
+        for p, stage in enumerate(got):
+            sp = wl.stage_specs[p]
+            for j, a in enumerate(stage):
+                ref = np.asarray(res.params[p][j], dtype=np.float64)
+                a = np.asarray(a, dtype=np.float64)
+                if sp.post == "attention" and j == len(stage) - 1:
+                    # The key bias is a gauge direction: softmax(q k^T) does not depend on it, its exact
+                    # gradient is zero, and what reaches the optimiser is rounding noise (which Adam turns into
+                    # steps of up to alpha).  It is checked against that bound instead of element by element.
+                    d = sp.n_out // 3
+                    bound = wl.alpha * len(res.losses) * 1.01 + 1e-12
+                    assert np.abs(a[d:2 * d]).max() <= bound and np.abs(ref[d:2 * d]).max() <= bound
+                    keep = np.r_[0:d, 2 * d:3 * d]
+                    a, ref = a[keep], ref[keep]
+                scale = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p]) if per_stage else None
+                e = max_rel_err(a, ref) if scale is None else float(np.abs(a - ref).max() / scale)
+                worst = max(worst, e)
+                assert e <= tol, f"stage {p} tensor {j}: {e}"
+        return worst
     for p, stage in enumerate(got):
         for j, (W, b) in enumerate(stage):
             eW = max_rel_err(W, res.params[p][2 * j])

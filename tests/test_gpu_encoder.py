@@ -1,0 +1,42 @@
+"""GPU parity of the Transformer-encoder pipeline (embedding, LayerNorm, attention, residuals, cross-entropy)."""
+import numpy as np
+import pytest
+
+import pm_inputs as I
+from parity_util import run_gpu_pipeline, run_oracle, compare_params
+
+pytestmark = pytest.mark.gpu
+
+
+def check_book(book, res, n_steps, P):
+    ref = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    assert len(book) == n_steps * P
+    for key, (vf, vb) in book.items():
+        assert (vf, vb) == ref[key]
+
+
+@pytest.mark.parametrize("kw", [
+    dict(n_layers=1, d_model=32, n_heads=2, d_ff=64, seq_len=8, batch=2, vocab=40, steps=12),
+    dict(n_layers=2, d_model=64, n_heads=4, d_ff=136, seq_len=16, batch=3, vocab=96, steps=24),
+])
+def test_encoder_fp32(cuda_device, kw):
+    wl = I.cfg4_small(compute="f32", **kw)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
+    worst = compare_params(pipe, res, 2e-5)
+    print("encoder fp32 worst relative weight error", worst)
+
+
+def test_encoder_bf16_small(cuda_device):
+    wl = I.cfg4_small(compute="bf16")
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("encoder bf16 loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("encoder bf16 worst relative weight error (per stage vector)", worst)
