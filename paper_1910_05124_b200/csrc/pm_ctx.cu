@@ -178,7 +178,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
   }
   for (int p = 0; p < P; ++p) L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
-  if (L.att_blocks > 0 && attention_smem_bytes(L.att_S, L.att_dk) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
+  if (L.att_blocks > 0 && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
   L.ring_bytes = ring;
   L.total = L.st[P - 1].end;
   L.n_in_first = L.st[0].pre == PRE_EMBED ? 0 : L.st[0].lin[0].n_in;
@@ -389,7 +389,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "position table upload"); delete c; return r; }
   }
   if (L.att_blocks > 0) {
-    e = attention_set_smem_limits(L.att_S, L.att_dk);
+    e = attention_set_smem_limits(L.att_S, L.att_dk, cfg->compute_dtype);
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "attention shared-memory limit"); delete c; return r; }
   }
 

@@ -82,8 +82,8 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream); 
 cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream);       // attention backward
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream);        // LayerNorm / embedding backward
 int pre_bwd_launches(const TickArgs& t);
-size_t attention_smem_bytes(int S, int dk);
-cudaError_t attention_set_smem_limits(int S, int dk);
+size_t attention_smem_bytes(int S, int dk, int dtype);
+cudaError_t attention_set_smem_limits(int S, int dk, int dtype);
 
 // fp32 SIMT grouped GEMMs (PM_F32 path).  mode: 0 forward, 1 dgrad (corrected weights), 2 wgrad.
 cudaError_t launch_simt_gemm(const TickArgs& t, int dtype, int mode, int lvl, cudaStream_t stream);

@@ -114,27 +114,27 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t, int caus
   if ((int)blockIdx.x >= n_seq * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
   extern __shared__ float sm[];
-  float* Q = sm;                       // [S][dk+1]
-  float* K = Q + S * (dk + 1);
-  float* V = K + S * (dk + 1);
-  float* Pm = V + S * (dk + 1);        // [S][S+1]
-  float* Ls = Pm + S * (S + 1);        // [S]
-  const int ld = dk + 1, lp = S + 1;
+  const int ld = dk + 2, lp = S + 1;   // operands are kept in the activation type, scores in fp32
+  float* Pm = sm;                      // [S][S+1]
+  float* Ls = Pm + S * lp;             // [S]
+  AT* Q = reinterpret_cast<AT*>(Ls + S);   // [S][dk+2]
+  AT* K = Q + S * ld;
+  AT* V = K + S * ld;
   const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
   const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.f_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
     const AT* row = qkv + (uint64_t)r * 3 * dm;
-    Q[r * ld + c] = to_f<AT>(row[c]);
-    K[r * ld + c] = to_f<AT>(row[dm + c]);
-    V[r * ld + c] = to_f<AT>(row[2 * dm + c]);
+    Q[r * ld + c] = row[c];
+    K[r * ld + c] = row[dm + c];
+    V[r * ld + c] = row[2 * dm + c];
   }
   __syncthreads();
   const float scale = 1.0f / sqrtf((float)dk);
   for (int i = threadIdx.x; i < S * S; i += blockDim.x) {
     const int r = i / S, c = i % S;
     float acc = 0.f;
-    for (int k = 0; k < dk; ++k) acc = fmaf(Q[r * ld + k], K[c * ld + k], acc);
+    for (int k = 0; k < dk; ++k) acc = fmaf(to_f<AT>(Q[r * ld + k]), to_f<AT>(K[c * ld + k]), acc);
     Pm[r * lp + c] = (causal && c > r) ? -INFINITY : acc * scale;
   }
   __syncthreads();
@@ -158,15 +158,15 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t, int caus
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
     float acc = 0.f;
-    for (int j = 0; j < S; ++j) acc = fmaf(Pm[r * lp + j], V[j * ld + c], acc);
+    for (int j = 0; j < S; ++j) acc = fmaf(Pm[r * lp + j], to_f<AT>(V[j * ld + c]), acc);
     out[(uint64_t)r * dm + c] = from_f<AT>(acc / Ls[r]);
   }
 }
 
-static size_t attn_fwd_smem(int S, int dk) { return sizeof(float) * (3 * (size_t)S * (dk + 1) + (size_t)S * (S + 1) + S); }
-static size_t attn_bwd_smem(int S, int dk) { return sizeof(float) * (4 * (size_t)S * (dk + 1) + 2 * (size_t)S * (S + 1) + S); }
+static size_t attn_fwd_smem(int S, int dk, size_t esz) { return sizeof(float) * ((size_t)S * (S + 1) + S) + esz * 3 * (size_t)S * (dk + 2); }
+static size_t attn_bwd_smem(int S, int dk, size_t esz) { return sizeof(float) * (2 * (size_t)S * (S + 1) + S) + esz * 4 * (size_t)S * (dk + 2); }
 
-size_t attention_smem_bytes(int S, int dk) { return attn_bwd_smem(S, dk); }
+size_t attention_smem_bytes(int S, int dk, int dtype) { return attn_bwd_smem(S, dk, dtype == PM_F32 ? 4 : 2); }
 
 cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   int S = 0, dk = 0, nblk = 0;
@@ -176,9 +176,8 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
   if (any_att) {
     dim3 grid(nblk, t.P);
-    size_t smem = attn_fwd_smem(S, dk);
-    if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, smem, stream>>>(t, 0);
-    else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(t, 0);
+    if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, attn_fwd_smem(S, dk, 4), stream>>>(t, 0);
+    else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, attn_fwd_smem(S, dk, 2), stream>>>(t, 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -205,24 +204,24 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
   if ((int)blockIdx.x >= n_seq * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
   extern __shared__ float sm[];
-  const int ld = dk + 1, lp = S + 1;
-  float* Q = sm;
-  float* K = Q + S * ld;
-  float* V = K + S * ld;
-  float* dO = V + S * ld;
-  float* Pm = dO + S * ld;             // [S][S+1] softmax probabilities (fp32)
+  const int ld = dk + 2, lp = S + 1;
+  float* Pm = sm;                      // [S][S+1] softmax probabilities (fp32)
   float* Dm = Pm + S * lp;             // [S][S+1] dP, then dS
   float* Ls = Dm + S * lp;
+  AT* Q = reinterpret_cast<AT*>(Ls + S);   // operands in the activation type, [S][dk+2]
+  AT* K = Q + S * ld;
+  AT* V = K + S * ld;
+  AT* dO = V + S * ld;
   const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
   const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.b_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
   const AT* go = gin_read<AT>(t, s, d) + (uint64_t)b * S * dm + h * dk;
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
     const AT* row = qkv + (uint64_t)r * 3 * dm;
-    Q[r * ld + c] = to_f<AT>(row[c]);
-    K[r * ld + c] = to_f<AT>(row[dm + c]);
-    V[r * ld + c] = to_f<AT>(row[2 * dm + c]);
-    dO[r * ld + c] = to_f<AT>(go[(uint64_t)r * dm + c]);
+    Q[r * ld + c] = row[c];
+    K[r * ld + c] = row[dm + c];
+    V[r * ld + c] = row[2 * dm + c];
+    dO[r * ld + c] = go[(uint64_t)r * dm + c];
   }
   __syncthreads();
   const float scale = 1.0f / sqrtf((float)dk);
@@ -230,8 +229,8 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
     const int r = i / S, c = i % S;
     float acc = 0.f, accd = 0.f;
     for (int k = 0; k < dk; ++k) {
-      acc = fmaf(Q[r * ld + k], K[c * ld + k], acc);
-      accd = fmaf(dO[r * ld + k], V[c * ld + k], accd);
+      acc = fmaf(to_f<AT>(Q[r * ld + k]), to_f<AT>(K[c * ld + k]), acc);
+      accd = fmaf(to_f<AT>(dO[r * ld + k]), to_f<AT>(V[c * ld + k]), accd);
     }
     Pm[r * lp + c] = (causal && c > r) ? -INFINITY : acc * scale;
     Dm[r * lp + c] = accd;                                     // dP
@@ -256,9 +255,9 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
     const int r = i / dk, c = i % dk;
     float aq = 0.f, ak = 0.f, av = 0.f;
     for (int j = 0; j < S; ++j) {
-      aq = fmaf(Dm[r * lp + j], K[j * ld + c], aq);            // dQ[r] = sum_j dS[r][j] K[j]
-      ak = fmaf(Dm[j * lp + r], Q[j * ld + c], ak);            // dK[r] = sum_j dS[j][r] Q[j]
-      av = fmaf(round_as<AT>(Pm[j * lp + r]), dO[j * ld + c], av);   // dV[r] = sum_j P[j][r] dO[j]
+      aq = fmaf(Dm[r * lp + j], to_f<AT>(K[j * ld + c]), aq);            // dQ[r] = sum_j dS[r][j] K[j]
+      ak = fmaf(Dm[j * lp + r], to_f<AT>(Q[j * ld + c]), ak);            // dK[r] = sum_j dS[j][r] Q[j]
+      av = fmaf(round_as<AT>(Pm[j * lp + r]), to_f<AT>(dO[j * ld + c]), av);   // dV[r] = sum_j P[j][r] dO[j]
     }
     AT* row = dy + (uint64_t)r * 3 * dm;
     row[c] = from_f<AT>(aq * scale);
@@ -270,17 +269,20 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
 cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   if (t.att_blocks <= 0) return cudaSuccess;
   dim3 grid(t.att_blocks, t.P);
-  size_t smem = attn_bwd_smem(t.att_S, t.att_dk);
-  if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, smem, stream>>>(t, 0);
-  else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(t, 0);
+  if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 4), stream>>>(t, 0);
+  else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 2), stream>>>(t, 0);
   return cudaGetLastError();
 }
 
-cudaError_t attention_set_smem_limits(int S, int dk) {
-  cudaError_t e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk));
+cudaError_t attention_set_smem_limits(int S, int dk, int dtype) {
+  cudaError_t e;
+  if (dtype == PM_F32) {
+    e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk, 4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk, 4));
+  } else {
+    e = cudaFuncSetAttribute((const void*)attention_fwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_fwd_smem(S, dk, 2));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attention_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_bwd_smem(S, dk, 2));
+  }
   return e;
 }
 

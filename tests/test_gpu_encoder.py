@@ -40,3 +40,18 @@ def test_encoder_bf16_small(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("encoder bf16 worst relative weight error (per stage vector)", worst)
+
+
+def test_cfg4_full_size_first_microbatches(cuda_device):
+    """Config 4 at its full size (6 layers, d_model 512, 8 heads, FFN 2048, 32 sequences of 128 tokens,
+    vocabulary 8192, 25 stages): two microbatches fed and drained, so every stage has applied two updates."""
+    wl = I.cfg4()
+    n = 2
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, n)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, n)
+    check_book(book, res, n, wl.n_stages)
+    print("cfg4 loss relative errors", np.abs(losses / np.array(res.losses) - 1))
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("cfg4 full size worst relative weight error (per stage vector)", worst)
