@@ -135,9 +135,47 @@ def barrier(world):
 
 # ---- the CUDA arm ---------------------------------------------------------------------------------
 
+WORKLOADS = {
+    "cfg3": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master weights, microbatch 128, "
+            "SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
+    "cfg4": "cfg4: Transformer encoder, 6 layers, d_model 512, 8 heads, FFN 2048, 32 sequences x 128 tokens per "
+            "microbatch, vocabulary 8192, bf16 GEMMs, fp32 master weights, one stage per weight GEMM (25 stages), "
+            "Adam(0.9, 0.98), T1 (K=100) + T2 (D=0.1), tau_i=2(25-i)+1",
+}
+
+
+def build_workload(args):
+    """Workload description, initial parameters, samples per step and parameter count."""
+    import pm_inputs as I
+    if args.workload == "cfg4":
+        wl = I.cfg4()
+        if args.stages:      # profiler captures only: fewer layers of the same shape, not a bench result
+            wl = I.encoder_workload(wl.name + f"_{args.stages}layers", args.stages, 512, 8, 2048, 128, 32, 8192, compute="bf16",
+                                    optimizer="adam", alpha=wl.alpha, beta1=0.9, beta2=0.98, eps=1e-8, K=wl.K, D=wl.D,
+                                    steps=wl.steps, seed=wl.seed)
+        params0 = I.init_encoder_params(wl)
+        n_params = sum(int(a.size) for st in params0 for a in st)
+        return wl, params0, wl.microbatch // wl.seq_len, n_params
+    wl = I.cfg3()
+    if args.stages:          # profiler captures only: fewer stages of the same shape, not a bench result
+        wl = I.mlp_workload(wl.name + f"_first{args.stages}", args.stages, 1024, 2, "gelu", wl.microbatch, compute="bf16",
+                            optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, K=wl.K, D=wl.D, steps=wl.steps,
+                            seed=wl.seed)
+    params0 = I.init_stage_params(wl)
+    n_params = sum(sp.n_in * sp.n_out + sp.n_out for st in wl.stages for sp in st)
+    return wl, params0, wl.microbatch, n_params
+
+
 def make_batches(wl, n, device):
     import torch
     import pm_inputs as I
+    if wl.kind == "encoder":
+        import numpy as np
+        host = []
+        for t in range(n):
+            ids, tg = I.token_batch(wl, t)
+            host.append((torch.from_numpy(ids.astype(np.int32)).pin_memory(), torch.from_numpy(tg.astype(np.int32)).pin_memory()))
+        return host, [(x.to(device), y.to(device)) for x, y in host]
     teacher = I.teacher_params(wl)
     xs, ys = [], []
     for t in range(n):
@@ -150,17 +188,22 @@ def make_batches(wl, n, device):
     return host, dev
 
 
-def cpu_baseline(wl, n_steps):
+def cpu_baseline(wl, n_steps, samples_per_step):
     """The oracle, as it stands, on this machine's host cores."""
     import pm_inputs as I
-    from oracle.mlp import run_workload
-    params0 = I.init_stage_params(wl)
-    teacher = I.teacher_params(wl)
-    batches = [I.batch(wl, t, teacher) for t in range(n_steps)]
+    if wl.kind == "encoder":
+        from oracle.transformer import run_workload
+        params0 = I.init_encoder_params(wl)
+        batches = [I.token_batch(wl, t) for t in range(n_steps)]
+    else:
+        from oracle.mlp import run_workload
+        params0 = I.init_stage_params(wl)
+        teacher = I.teacher_params(wl)
+        batches = [I.batch(wl, t, teacher) for t in range(n_steps)]
     t0 = time.perf_counter()
     run_workload(wl, params0, lambda t: batches[t], n_steps=n_steps)
     dt = time.perf_counter() - t0
-    return {"value": wl.microbatch * n_steps / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+    return {"value": samples_per_step * n_steps / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
             "sample": f"{n_steps} microbatch steps of the {wl.name} workload (forward, backward, update of all "
                       f"{wl.n_stages} stages), {dt:.1f} s"}
 
@@ -260,16 +303,10 @@ def run_cuda(args):
     device = torch.device(f"cuda:{local}")
     torch.cuda.set_device(device)
     hbm_peak, tf_peak, peak_kind = measured_peaks()
-    wl = I.cfg3()
-    if args.stages:                      # profiler captures only: fewer stages of the same shape, not a bench result
-        wl = I.mlp_workload(wl.name + f"_first{args.stages}", args.stages, 1024, 2, "gelu", wl.microbatch, compute="bf16",
-                            optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, K=wl.K, D=wl.D, steps=wl.steps,
-                            seed=wl.seed)
+    wl, params0, samples_per_step, n_params = build_workload(args)
     P = wl.n_stages
-    params0 = I.init_stage_params(wl)
     pipe = pm.Pipeline(wl, params0, device=str(device))
     host_b, dev_b = make_batches(wl, 4, device)
-    n_params = sum(sp.n_in * sp.n_out + sp.n_out for st in wl.stages for sp in st)
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -296,7 +333,7 @@ def run_cuda(args):
     barrier(world)
     elapsed_ms = e0.elapsed_time(e1)
     launches = pipe.pm_launch_count() - launches0
-    t_ms, units = reduce_over_ranks(elapsed_ms, wl.microbatch * args.steps, world, device)
+    t_ms, units = reduce_over_ranks(elapsed_ms, samples_per_step * args.steps, world, device)
     value = units / (t_ms * 1e-3)
 
     # ---- timed region 2: the update kernel alone inside the step (CUDA events on the launch stream) --
@@ -334,8 +371,8 @@ def run_cuda(args):
     torch.cuda.synchronize(device)
     e2e_ms = (time.perf_counter() - t0) * 1e3
     barrier(world)
-    e2e_t, e2e_units = reduce_over_ranks(e2e_ms, wl.microbatch * args.steps, world, device)
-    h2d = host_b[0][0].numel() * host_b[0][0].element_size() + host_b[0][1].numel() * 4
+    e2e_t, e2e_units = reduce_over_ranks(e2e_ms, samples_per_step * args.steps, world, device)
+    h2d = sum(x.numel() * x.element_size() for x in host_b[0])
 
     if rank != 0:
         return
@@ -343,10 +380,10 @@ def run_cuda(args):
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(t_ms / args.steps, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master "
-                               "weights, microbatch 128, SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
-                   "parallelism": "replicas only" if world > 1 else "single GPU, 32 emulated pipeline stages",
-                   "pipeline_fill_ticks": fill, "cache": "per-step working set ~3 GB > 126 MB L2 (no flush needed)",
+        "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
+                   "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
+                   "samples_per_step": samples_per_step,
+                   "pipeline_fill_ticks": fill, "cache": "per-step working set (state + rings, see state_bytes) far exceeds the 126 MB L2: no flush needed",
                    "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "params": n_params},
         "clocks": clocks,
         "e2e": {"value": round(e2e_units / (e2e_t * 1e-3), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -360,7 +397,7 @@ def run_cuda(args):
     }
     if world == 1:
         if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(wl, 2)
+            line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, samples_per_step)
         if not args.no_sweep:
             line["update_sweep"] = update_sweep(device, hbm_peak)
     print(json.dumps(line), flush=True)
@@ -430,6 +467,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the stand-alone update sweep")
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
     ap.add_argument("--stages", type=int, default=0, help="profiling runs: same workload cut to this many stages")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
     ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",

@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["pm_ctx.cu", "pm_update.cu", "pm_update_static.cu", "pm_simt.cu", "pm_xfmr.cu", "pm_umma.cu"]
+SOURCES = ["pm_ctx.cu", "pm_update.cu", "pm_update_static.cu", "pm_simt.cu", "pm_xfmr.cu", "pm_attn.cu", "pm_umma.cu"]
 LIB = os.path.join(HERE, "libpipemare.so")
 
 

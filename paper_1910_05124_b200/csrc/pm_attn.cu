@@ -1,0 +1,376 @@
+// Multi-head self-attention on the tensor cores (tcgen05 + TMEM + TMA), forward and backward, for
+// sequences of 128 tokens and heads of width 64 (bf16).  One CTA of 128 threads handles one (sequence, head):
+// thread r owns query row r = TMEM lane r, so the softmax needs no cross-thread traffic.
+//
+// forward :  S = Q K^T (128x128x64)  ->  p~ = exp(S/8 - rowmax), l = sum p~  ->  O = (bf16(p~) V) / l  (128x64x128)
+// backward:  S = Q K^T, dP = dO V^T  ->  P = softmax, D = rowsum(dP*P), dS = bf16(P*(dP - D)), Pb = bf16(P)
+//            dV = Pb^T dO,  dQ = dS K / 8,  dK = dS^T Q / 8   (each 128x64x128)
+// Q, K, V, dO arrive by TMA as 128-byte-swizzled [128 rows x 64] tiles; the same tile serves as a K-major
+// operand (rows x d_k) or as an MN-major operand (k-rows x 64) depending on the product.  P and dS are
+// written by the threads as two [128 x 64-key] swizzled tiles, read K-major (P V, dS K) or MN-major (P^T dO,
+// dS^T Q).  Every mbarrier wait is bounded.
+#include <string>
+#include <vector>
+
+#include "pm_ptx.cuh"
+#include "pm_tick.cuh"
+
+namespace pm {
+
+constexpr int AT_S = 128, AT_DK = 64;
+constexpr int AT_TILE = AT_S * AT_DK * 2;          // 16 KB: one [128 x 64] bf16 tile
+constexpr int AT_FWD_SMEM = 3 * AT_TILE + 2 * AT_TILE + 1024 + 128;
+constexpr int AT_BWD_SMEM = 4 * AT_TILE + 4 * AT_TILE + 1024 + 128;
+constexpr int AT_TMEM_COLS = 256;
+
+enum { AMAP_QKV = 0, AMAP_DO = 1, AMAPS_PER_STAGE = 2 };
+
+__device__ __forceinline__ void issue_k64(uint32_t tmem_d, uint32_t a, uint32_t b, uint32_t idesc, bool a_kmajor, bool b_kmajor,
+                                          uint32_t a_lbo, uint32_t b_lbo, bool acc_first) {
+  // one 64-deep k slab: four MMAs of depth 16
+#pragma unroll
+  for (int k16 = 0; k16 < 4; ++k16) {
+    const uint64_t da = a_kmajor ? make_desc(a + k16 * 32, 16, 1024) : make_desc(a + k16 * 2048, a_lbo, 1024);
+    const uint64_t db = b_kmajor ? make_desc(b + k16 * 32, 16, 1024) : make_desc(b + k16 * 2048, b_lbo, 1024);
+    tc_mma_bf16(tmem_d, da, db, idesc, (acc_first || k16 > 0) ? 1u : 0u);
+  }
+}
+
+// write 8 consecutive bf16 (16 bytes) of row r, column chunk j (0..15) into a pair of [128 x 64] swizzled tiles
+__device__ __forceinline__ void put_chunk(uint8_t* tiles, int r, int j, uint4 v) {
+  *reinterpret_cast<uint4*>(tiles + (j >> 3) * AT_TILE + r * 128 + (((j & 7) ^ (r & 7)) << 4)) = v;
+}
+
+struct AttnCommon {
+  uint32_t sbase; uint8_t* sptr; uint32_t bar_load, bar_mma; uint32_t* tmem_slot; volatile int* abort_flag;
+};
+
+__device__ __forceinline__ AttnCommon attn_setup(uint8_t* smem_raw, int tile_bytes) {
+  AttnCommon c;
+  const uint32_t raw = smem_u32(smem_raw);
+  c.sbase = (raw + 1023u) & ~1023u;
+  c.sptr = smem_raw + (c.sbase - raw);
+  c.bar_load = c.sbase + tile_bytes;
+  c.bar_mma = c.bar_load + 8;
+  c.tmem_slot = reinterpret_cast<uint32_t*>(c.sptr + tile_bytes + 16);
+  c.abort_flag = reinterpret_cast<volatile int*>(c.tmem_slot + 1);
+  if (threadIdx.x == 0) {
+    mbar_init(c.bar_load, 1);
+    mbar_init(c.bar_mma, 1);
+    *c.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if ((threadIdx.x >> 5) == 0) {
+    __syncwarp();
+    tmem_alloc(smem_u32(c.tmem_slot), AT_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  return c;
+}
+
+__device__ __forceinline__ void attn_teardown(const AttnCommon& c, uint32_t tmem_base) {
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 0) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, AT_TMEM_COLS);
+  }
+}
+
+// all threads: wait for an MMA batch; returns false (uniformly) if any thread gave up
+__device__ __forceinline__ bool wait_mma(const AttnCommon& c, uint32_t parity, int* status, int code) {
+  bool ok = !*c.abort_flag && mbar_wait(c.bar_mma, parity, c.abort_flag, status, code);
+  ok = __syncthreads_and(ok);
+  tc_fence_after();
+  return ok;
+}
+
+__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int causal, int* status) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.f_mb < 0 || s.post != POST_ATTENTION) return;
+  const int H = s.n_heads, dm = s.d_out_main;
+  if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
+  const int b = blockIdx.x / H, h = blockIdx.x % H;
+  extern __shared__ uint8_t smem_raw[];
+  const AttnCommon c = attn_setup(smem_raw, 5 * AT_TILE);
+  const uint32_t tmem_base = *c.tmem_slot;
+  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sV = sK + AT_TILE, sP = sV + AT_TILE;
+  uint8_t* pP = c.sptr + 3 * AT_TILE;
+  const CUtensorMap* lm = maps + (size_t)p * AMAPS_PER_STAGE;
+  const int r = threadIdx.x;                                 // query row = TMEM lane
+  const int warp = r >> 5;
+
+  if (r == 0) {
+    mbar_arrive_expect_tx(c.bar_load, 3 * AT_TILE);
+    tma_load_3d(sQ, lm + AMAP_QKV, c.bar_load, h * AT_DK, b * AT_S, d.f_slot);
+    tma_load_3d(sK, lm + AMAP_QKV, c.bar_load, dm + h * AT_DK, b * AT_S, d.f_slot);
+    tma_load_3d(sV, lm + AMAP_QKV, c.bar_load, 2 * dm + h * AT_DK, b * AT_S, d.f_slot);
+    if (mbar_wait(c.bar_load, 0, c.abort_flag, status, 11)) {
+      tc_fence_after();
+      issue_k64(tmem_base, sQ, sK, make_idesc_mn(128, 128, 0, 0), true, true, 0, 0, false);   // S = Q K^T
+      tc_commit(c.bar_mma);
+    }
+  }
+  if (wait_mma(c, 0, status, 12)) {
+    const float scale = 0.125f;                              // 1 / sqrt(64)
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (!causal || cc * 32 + j <= r) mx = fmaxf(mx, __uint_as_float(v[j]) * scale);
+    }
+    float l = 0.f;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld_wait();
+      float e[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        e[j] = (!causal || cc * 32 + j <= r) ? expf(__uint_as_float(v[j]) * scale - mx) : 0.f;
+        l += e[j];
+      }
+#pragma unroll
+      for (int g = 0; g < 4; ++g)
+        put_chunk(pP, r, cc * 4 + g, make_uint4(pack_bf16(e[g * 8], e[g * 8 + 1]), pack_bf16(e[g * 8 + 2], e[g * 8 + 3]),
+                                                 pack_bf16(e[g * 8 + 4], e[g * 8 + 5]), pack_bf16(e[g * 8 + 6], e[g * 8 + 7])));
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (r == 0) {
+      tc_fence_after();
+      const uint32_t idesc = make_idesc_mn(128, 64, 0, 1);   // O = P V : A = P K-major, B = V MN-major (k = key rows)
+      issue_k64(tmem_base + 128, sP, sV, idesc, true, false, 0, 8192, false);
+      issue_k64(tmem_base + 128, sP + AT_TILE, sV + 4 * 2048, idesc, true, false, 0, 8192, true);
+      tc_commit(c.bar_mma);
+    }
+    if (wait_mma(c, 1, status, 13)) {
+      uint32_t o0[32], o1[32];
+      tmem_ld32(lane_addr + 128, o0);
+      tmem_ld32(lane_addr + 160, o1);
+      tmem_ld_wait();
+      const float inv = 1.0f / l;
+      __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[p + 1].x_ring) + (size_t)d.f_next_xslot * ((size_t)t.T * dm) +
+                           (size_t)(b * AT_S + r) * dm + h * AT_DK;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        const uint32_t* src = g < 4 ? o0 + (g & 3) * 8 : o1 + (g & 3) * 8;
+        float f[8];
+#pragma unroll
+        for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(src[e2]) * inv;
+        *reinterpret_cast<uint4*>(out + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+      }
+    }
+  }
+  attn_teardown(c, tmem_base);
+}
+
+__global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int causal, int* status) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.post != POST_ATTENTION) return;
+  const int H = s.n_heads, dm = s.d_out_main;
+  if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
+  const int b = blockIdx.x / H, h = blockIdx.x % H;
+  extern __shared__ uint8_t smem_raw[];
+  const AttnCommon c = attn_setup(smem_raw, 8 * AT_TILE);
+  const uint32_t tmem_base = *c.tmem_slot;
+  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sV = sK + AT_TILE, sdO = sV + AT_TILE, sP = sdO + AT_TILE, sdS = sP + 2 * AT_TILE;
+  uint8_t* pP = c.sptr + 4 * AT_TILE;
+  uint8_t* pdS = c.sptr + 6 * AT_TILE;
+  const CUtensorMap* lm = maps + (size_t)p * AMAPS_PER_STAGE;
+  const int r = threadIdx.x;
+  const int warp = r >> 5;
+
+  if (r == 0) {
+    mbar_arrive_expect_tx(c.bar_load, 4 * AT_TILE);
+    tma_load_3d(sQ, lm + AMAP_QKV, c.bar_load, h * AT_DK, b * AT_S, d.b_slot);
+    tma_load_3d(sK, lm + AMAP_QKV, c.bar_load, dm + h * AT_DK, b * AT_S, d.b_slot);
+    tma_load_3d(sV, lm + AMAP_QKV, c.bar_load, 2 * dm + h * AT_DK, b * AT_S, d.b_slot);
+    tma_load_3d(sdO, lm + AMAP_DO, c.bar_load, h * AT_DK, b * AT_S, (int)((d.tick + 2) % 3));
+    if (mbar_wait(c.bar_load, 0, c.abort_flag, status, 14)) {
+      tc_fence_after();
+      const uint32_t idesc = make_idesc_mn(128, 128, 0, 0);
+      issue_k64(tmem_base, sQ, sK, idesc, true, true, 0, 0, false);          // S  = Q K^T
+      issue_k64(tmem_base + 128, sdO, sV, idesc, true, true, 0, 0, false);   // dP = dO V^T
+      tc_commit(c.bar_mma);
+    }
+  }
+  if (wait_mma(c, 0, status, 15)) {
+    const float scale = 0.125f;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (!causal || cc * 32 + j <= r) mx = fmaxf(mx, __uint_as_float(v[j]) * scale);
+    }
+    float l = 0.f;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (!causal || cc * 32 + j <= r) l += expf(__uint_as_float(v[j]) * scale - mx);
+    }
+    const float inv = 1.0f / l;
+    float D = 0.f;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32], g[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld32(lane_addr + 128 + cc * 32, g);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (!causal || cc * 32 + j <= r) D += __uint_as_float(g[j]) * (expf(__uint_as_float(v[j]) * scale - mx) * inv);
+    }
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      uint32_t v[32], g[32];
+      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld32(lane_addr + 128 + cc * 32, g);
+      tmem_ld_wait();
+      float pr[32], ds[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        pr[j] = (!causal || cc * 32 + j <= r) ? expf(__uint_as_float(v[j]) * scale - mx) * inv : 0.f;
+        ds[j] = pr[j] * (__uint_as_float(g[j]) - D);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        put_chunk(pP, r, cc * 4 + q, make_uint4(pack_bf16(pr[q * 8], pr[q * 8 + 1]), pack_bf16(pr[q * 8 + 2], pr[q * 8 + 3]),
+                                                 pack_bf16(pr[q * 8 + 4], pr[q * 8 + 5]), pack_bf16(pr[q * 8 + 6], pr[q * 8 + 7])));
+        put_chunk(pdS, r, cc * 4 + q, make_uint4(pack_bf16(ds[q * 8], ds[q * 8 + 1]), pack_bf16(ds[q * 8 + 2], ds[q * 8 + 3]),
+                                                  pack_bf16(ds[q * 8 + 4], ds[q * 8 + 5]), pack_bf16(ds[q * 8 + 6], ds[q * 8 + 7])));
+      }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (r == 0) {
+      tc_fence_after();
+      // dV = P^T dO : A = P read MN-major (m = key, k = query row; the second 64-key group one tile on), B = dO MN-major
+      const uint32_t i_mm = make_idesc_mn(128, 64, 1, 1), i_km = make_idesc_mn(128, 64, 0, 1);
+      issue_k64(tmem_base, sP, sdO, i_mm, false, false, AT_TILE, 8192, false);
+      issue_k64(tmem_base, sP + 4 * 2048, sdO + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
+      // dQ = dS K : A = dS K-major (k = key), B = K MN-major (k = key rows)
+      issue_k64(tmem_base + 64, sdS, sK, i_km, true, false, 0, 8192, false);
+      issue_k64(tmem_base + 64, sdS + AT_TILE, sK + 4 * 2048, i_km, true, false, 0, 8192, true);
+      // dK = dS^T Q : A = dS read MN-major (m = key, k = query row), B = Q MN-major
+      issue_k64(tmem_base + 128, sdS, sQ, i_mm, false, false, AT_TILE, 8192, false);
+      issue_k64(tmem_base + 128, sdS + 4 * 2048, sQ + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
+      tc_commit(c.bar_mma);
+    }
+    if (wait_mma(c, 1, status, 16)) {
+      __nv_bfloat16* dy = reinterpret_cast<__nv_bfloat16*>(t.ws + s.dy) + (size_t)(b * AT_S + r) * 3 * dm + h * AT_DK;
+#pragma unroll 1
+      for (int which = 0; which < 3; ++which) {              // TMEM columns: dV at 0, dQ at 64, dK at 128
+        uint32_t o0[32], o1[32];
+        tmem_ld32(lane_addr + which * 64, o0);
+        tmem_ld32(lane_addr + which * 64 + 32, o1);
+        tmem_ld_wait();
+        const float sc = which == 0 ? 1.0f : scale;
+        __nv_bfloat16* dst = dy + (which == 0 ? 2 * dm : (which == 1 ? 0 : dm));
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t* src = g < 4 ? o0 + (g & 3) * 8 : o1 + (g & 3) * 8;
+          float f[8];
+#pragma unroll
+          for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(src[e2]) * sc;
+          *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+        }
+      }
+    }
+  }
+  attn_teardown(c, tmem_base);
+}
+
+// ---- host side --------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct AttnPlan {
+  const CUtensorMap* d_maps = nullptr;
+  int* d_status = nullptr;
+};
+
+uint64_t attn_workspace_bytes(int n_stages) { return 256 + (uint64_t)n_stages * AMAPS_PER_STAGE * sizeof(CUtensorMap); }
+
+bool attn_tc_supported(int dtype, int S, int dk) { return dtype == PM_BF16 && S == AT_S && dk == AT_DK; }
+
+pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region, cudaStream_t stream, std::string& err) {
+  *out = nullptr;
+  void* fnp = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t ce = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres);
+  if (ce != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fnp) { err = "cuTensorMapEncodeTiled is not available from this driver"; return PM_ERR_CUDA; }
+  EncodeTiledFn fn = (EncodeTiledFn)fnp;
+  std::vector<CUtensorMap> maps((size_t)t.P * AMAPS_PER_STAGE);
+  memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+  const cuuint64_t T = (cuuint64_t)t.T;
+  for (int p = 0; p < t.P; ++p) {
+    const StageDev& s = st[p];
+    if (s.post != POST_ATTENTION) continue;
+    const cuuint64_t d3 = (cuuint64_t)s.lin[0].n_out, dm = (cuuint64_t)s.d_out_main;
+    cuuint32_t box[3] = {AT_DK, AT_S, 1}, es[3] = {1, 1, 1};
+    {
+      cuuint64_t dims[3] = {d3, T, (cuuint64_t)s.depth}, strides[2] = {d3 * 2, T * d3 * 2};
+      CUresult r = fn(&maps[(size_t)p * AMAPS_PER_STAGE + AMAP_QKV], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, t.ring + s.lin[0].z_ring, dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled (attention qkv) failed with code " + std::to_string((int)r); return PM_ERR_CUDA; }
+    }
+    {
+      cuuint64_t dims[3] = {dm, T, 3}, strides[2] = {dm * 2, T * dm * 2};
+      CUresult r = fn(&maps[(size_t)p * AMAPS_PER_STAGE + AMAP_DO], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, t.ws + s.gin, dims, strides,
+                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled (attention dO) failed with code " + std::to_string((int)r); return PM_ERR_CUDA; }
+    }
+  }
+  char* region = (char*)ws_region;
+  cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_FWD_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_BWD_SMEM);
+  if (e != cudaSuccess) { err = std::string("attention plan: ") + cudaGetErrorString(e); return PM_ERR_CUDA; }
+  AttnPlan* plan = new AttnPlan();
+  plan->d_status = (int*)region;
+  plan->d_maps = (const CUtensorMap*)(region + 256);
+  *out = plan;
+  return PM_OK;
+}
+
+void attn_plan_destroy(AttnPlan* plan) { delete plan; }
+int* attn_status_word(AttnPlan* plan) { return plan ? plan->d_status : nullptr; }
+
+cudaError_t attn_tc_launch(AttnPlan* plan, const TickArgs& t, bool forward, cudaStream_t stream) {
+  dim3 grid(t.att_blocks, t.P);
+  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, 0, plan->d_status);
+  else attn_bwd_tc_kernel<<<grid, 128, AT_BWD_SMEM, stream>>>(t, plan->d_maps, 0, plan->d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace pm

@@ -9,6 +9,10 @@
 #include "pm_update.cuh"
 #include "pm_umma.cuh"
 
+namespace pm {
+pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region, cudaStream_t stream, std::string& err);
+}
+
 using namespace pm;
 
 namespace {
@@ -24,7 +28,8 @@ struct Layout {
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
-  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0;
+  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0;
+  bool att_tc = false;
   int32_t any_pre = 0, any_ln = 0, any_embed = 0, any_residual = 0, att_S = 0, att_dk = 0, att_blocks = 0, max_vocab = 0;
   int32_t pe_seq = 0, pe_d = 0;
   int64_t loss_cap = 0;
@@ -178,7 +183,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
   }
   for (int p = 0; p < P; ++p) L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
-  if (L.att_blocks > 0 && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
+  L.att_tc = L.att_blocks > 0;
+  for (int p = 0; p < P; ++p)
+    if (L.st[p].post == POST_ATTENTION && !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads)) L.att_tc = false;
+  if (L.att_blocks > 0 && !L.att_tc && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
   L.ring_bytes = ring;
   L.total = L.st[P - 1].end;
   L.n_in_first = L.st[0].pre == PRE_EMBED ? 0 : L.st[0].lin[0].n_in;
@@ -200,6 +208,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
   L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes(P) : 0), 256);
+  L.off_attn = w; w = align_up(w + (L.att_tc ? attn_workspace_bytes(P) : 0), 256);
   for (int p = 0; p < P; ++p) {
     StageDev& s = L.st[p];
     const uint64_t n_out_last = s.lin[s.n_lin - 1].n_out;
@@ -233,6 +242,7 @@ struct pm_ctx {
   bool draining = false;
   std::string err;
   UmmaPlan* umma = nullptr;
+  AttnPlan* attn = nullptr;
   uint64_t launches = 0;   // kernels enqueued by this context so far
 };
 
@@ -388,7 +398,11 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "position table upload"); delete c; return r; }
   }
-  if (L.att_blocks > 0) {
+  if (L.att_tc) {
+    std::string aerr;
+    pm_status as = attn_plan_create(&c->attn, t, c->L.st, c->ws + L.off_attn, c->stream, aerr);
+    if (as != PM_OK) { delete c; return fail(nullptr, as, aerr); }
+  } else if (L.att_blocks > 0) {
     e = attention_set_smem_limits(L.att_S, L.att_dk, cfg->compute_dtype);
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "attention shared-memory limit"); delete c; return r; }
   }
@@ -431,8 +445,9 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
                                    : umma_launch(ctx->umma, ctx->ta, 0, l, ctx->stream);
       if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
     }
-    const int n_post = (ctx->L.att_blocks > 0 ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
-    if (n_post && (s = check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream), "attention / residual forward", n_post)) != PM_OK) return s;
+    if (ctx->attn && (s = check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->stream), "attention forward")) != PM_OK) return s;
+    const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
+    if (n_post && (s = check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream, ctx->attn != nullptr), "attention / residual forward", n_post)) != PM_OK) return s;
   }
   ctx->phase = 1;
   return PM_OK;
@@ -448,7 +463,8 @@ pm_status pm_backward(pm_ctx* ctx) {
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
     if ((s = check(ctx, launch_loss(ctx->ta, dt, ctx->stream), "loss")) != PM_OK) return s;
-    if (ctx->L.att_blocks > 0 && (s = check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward")) != PM_OK) return s;
+    if (ctx->attn) { if ((s = check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->stream), "attention backward")) != PM_OK) return s; }
+    else if (ctx->L.att_blocks > 0 && (s = check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward")) != PM_OK) return s;
     for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
       if ((s = check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward")) != PM_OK) return s;
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->stream)
@@ -491,12 +507,14 @@ pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets) {
 
 // After a synchronisation: did any CTA give up on a bounded wait?
 static pm_status check_device_status(pm_ctx* ctx) {
-  int* w = umma_status_word(ctx->umma);
-  if (!w) return PM_OK;
-  int code = 0;
-  cudaError_t e = cudaMemcpy(&code, w, sizeof(int), cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "status read-back");
-  if (code != 0) return fail(ctx, PM_ERR_TIMEOUT, "a bounded device-side wait expired in a GEMM kernel (role code " + std::to_string(code) + ")");
+  int* words[2] = {umma_status_word(ctx->umma), attn_status_word(ctx->attn)};
+  for (int* w : words) {
+    if (!w) continue;
+    int code = 0;
+    cudaError_t e = cudaMemcpy(&code, w, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "status read-back");
+    if (code != 0) return fail(ctx, PM_ERR_TIMEOUT, "a bounded device-side wait expired in a tensor-core kernel (role code " + std::to_string(code) + ")");
+  }
   return PM_OK;
 }
 
@@ -537,6 +555,7 @@ const char* pm_last_error(pm_ctx* ctx) { return ctx ? ctx->err.c_str() : g_error
 void pm_destroy(pm_ctx* ctx) {
   if (!ctx) return;
   umma_plan_destroy(ctx->umma);
+  attn_plan_destroy(ctx->attn);
   delete ctx;
 }
 

@@ -78,8 +78,15 @@ cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t st
 
 // Transformer pieces (all grouped over the stages that carry the op this tick).
 cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream);        // embedding / LayerNorm forward (+ skip hand-over)
-cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream);       // attention forward, residual add
+cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, bool skip_attention);   // attention forward (SIMT), residual add
 cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream);       // attention backward
+// tensor-core attention (bf16, sequences of 128, heads of 64)
+struct AttnPlan;
+uint64_t attn_workspace_bytes(int n_stages);
+bool attn_tc_supported(int dtype, int S, int dk);
+cudaError_t attn_tc_launch(AttnPlan* plan, const TickArgs& t, bool forward, cudaStream_t stream);
+void attn_plan_destroy(AttnPlan* plan);
+int* attn_status_word(AttnPlan* plan);
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream);        // LayerNorm / embedding backward
 int pre_bwd_launches(const TickArgs& t);
 size_t attention_smem_bytes(int S, int dk, int dtype);

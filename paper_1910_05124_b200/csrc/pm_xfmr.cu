@@ -168,11 +168,11 @@ static size_t attn_bwd_smem(int S, int dk, size_t esz) { return sizeof(float) * 
 
 size_t attention_smem_bytes(int S, int dk, int dtype) { return attn_bwd_smem(S, dk, dtype == PM_F32 ? 4 : 2); }
 
-cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
+cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, bool skip_attention) {
   int S = 0, dk = 0, nblk = 0;
   bool any_res = false, any_att = false;
   // the shapes are uniform over stages in the supported workloads; the host keeps the maxima in TickArgs
-  S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0; any_res = t.any_residual != 0;
+  S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0 && !skip_attention; any_res = t.any_residual != 0;
   cudaError_t e = cudaSuccess;
   if (any_att) {
     dim3 grid(nblk, t.P);

@@ -55,3 +55,17 @@ def test_cfg4_full_size_first_microbatches(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("cfg4 full size worst relative weight error (per stage vector)", worst)
+
+
+def test_encoder_tensor_core_attention_shape(cuda_device):
+    """Sequences of 128 tokens and heads of width 64 take the tensor-core attention kernels; everything else in
+    this workload is small, so the oracle finishes quickly."""
+    wl = I.cfg4_small(compute="bf16", n_layers=2, d_model=128, n_heads=2, d_ff=256, seq_len=128, batch=2, vocab=200, steps=12)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("tc attention loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("tc attention worst relative weight error (per stage vector)", worst)
