@@ -28,7 +28,8 @@ struct Layout {
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
-  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0;
+  uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0, off_colred = 0;
+  int32_t row_chunks = 1;
   bool att_tc = false;
   int32_t any_pre = 0, any_ln = 0, any_embed = 0, any_residual = 0, att_S = 0, att_dk = 0, att_blocks = 0, max_vocab = 0;
   int32_t pe_seq = 0, pe_d = 0;
@@ -204,6 +205,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
   L.off_lossred = w; w = align_up(w + 512, 256);
   L.off_rowloss = w; w = align_up(w + (ce ? T * 4 : 0), 256);
+  L.row_chunks = (int32_t)((T + 255) / 256);
+  L.off_colred = w; w = align_up(w + (L.row_chunks > 1 ? (uint64_t)P * L.row_chunks * 2 * L.max_dim * 4 : 0), 256);
   L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
@@ -383,6 +386,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
+  t.colred_off = L.off_colred; t.row_chunks = L.row_chunks;
   t.any_pre = L.any_pre; t.any_ln = L.any_ln; t.any_embed = L.any_embed; t.any_residual = L.any_residual;
   t.att_S = L.att_S; t.att_dk = L.att_dk; t.att_blocks = L.att_blocks; t.max_vocab = L.max_vocab;
   if (L.pe_seq > 0) {
@@ -466,7 +470,7 @@ pm_status pm_backward(pm_ctx* ctx) {
     if (ctx->attn) { if ((s = check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->stream), "attention backward")) != PM_OK) return s; }
     else if (ctx->L.att_blocks > 0 && (s = check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward")) != PM_OK) return s;
     for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
-      if ((s = check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward")) != PM_OK) return s;
+      if ((s = check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward", actbwd_launches(ctx->ta))) != PM_OK) return s;
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->stream)
                                    : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->stream);
       if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;

@@ -121,40 +121,51 @@ template <> struct Pair<__nv_bfloat16> {
   static __device__ __forceinline__ void st(__nv_bfloat16* p, float2 v) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v.x, v.y); }
 };
 
+constexpr int kRowChunk = 256;                        // rows per block: 8 warps x 32 rows
+
 template <typename AT>
 __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
-  const int p = blockIdx.y;
+  const int p = blockIdx.z;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
   const int c0 = blockIdx.x * kActCols;
   if (c0 >= L.n_out) return;
+  const int chunk = blockIdx.y;
+  const int r0 = chunk * kRowChunk, r1 = min(t.T, r0 + kRowChunk);
+  if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c = c0 + 2 * lane;                        // n_out is even whenever a pair straddles nothing: see guard
+  const int c = c0 + 2 * lane;
   const uint64_t n = (uint64_t)t.T * L.n_out;
   const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
                  : (s.post == POST_ATTENTION ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
-  const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy and no stash is read
+  const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy: nothing is stored
   const AT* z = has_act ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n) : dy;
   AT* dz = ws_ptr<AT>(t, s.dz);
   const bool pair_ok = (L.n_out & 1) == 0;            // vector path needs even row length for alignment
   float s0 = 0.f, s1 = 0.f;
-  for (int r = warp; r < t.T; r += kActWarps) {
+  for (int r = r0 + warp; r < r1; r += kActWarps) {
     const uint64_t i = (uint64_t)r * L.n_out + c;
     if (pair_ok && c + 1 < L.n_out) {
-      float2 g = Pair<AT>::ld(dy + i), zz = Pair<AT>::ld(z + i);
-      float2 v = has_act ? make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act)))) : g;
-      Pair<AT>::st(dz + i, v);
+      float2 g = Pair<AT>::ld(dy + i);
+      float2 v = g;
+      if (has_act) {
+        float2 zz = Pair<AT>::ld(z + i);
+        v = make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act))));
+        Pair<AT>::st(dz + i, v);
+      }
       s0 = __fadd_rn(s0, v.x); s1 = __fadd_rn(s1, v.y);
     } else {
       if (c < L.n_out) {
         float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act))) : to_f<AT>(dy[i]);
-        dz[i] = from_f<AT>(v); s0 = __fadd_rn(s0, v);
+        if (has_act) dz[i] = from_f<AT>(v);
+        s0 = __fadd_rn(s0, v);
       }
       if (c + 1 < L.n_out) {
         float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i + 1]), act_grad(to_f<AT>(z[i + 1]), L.act))) : to_f<AT>(dy[i + 1]);
-        dz[i + 1] = from_f<AT>(v); s1 = __fadd_rn(s1, v);
+        if (has_act) dz[i + 1] = from_f<AT>(v);
+        s1 = __fadd_rn(s1, v);
       }
     }
   }
@@ -166,14 +177,36 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
     float sum = 0.f;
 #pragma unroll
     for (int w = 0; w < kActWarps; ++w) sum = __fadd_rn(sum, red[w][threadIdx.x]);
-    t.a.grad[L.b_off + c0 + threadIdx.x] = sum;
+    if (t.row_chunks == 1) t.a.grad[L.b_off + c0 + threadIdx.x] = sum;
+    else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + c0 + threadIdx.x] = sum;
   }
 }
 
+// adds the per-row-chunk partial column sums in chunk order: db of Linear lvl
+__global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || lvl >= s.n_lin) return;
+  const LinDev& L = s.lin[lvl];
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= L.n_out) return;
+  const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * (2 * (uint64_t)t.max_dim) + c;
+  float sum = 0.f;
+  for (int k = 0; k < t.row_chunks; ++k) sum = __fadd_rn(sum, part[(uint64_t)k * 2 * t.max_dim]);
+  t.a.grad[L.b_off + c] = sum;
+}
+
+int actbwd_launches(const TickArgs& t) { return t.row_chunks == 1 ? 1 : 2; }
+
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
-  dim3 grid((t.max_dim + kActCols - 1) / kActCols, t.P);
+  dim3 grid((t.max_dim + kActCols - 1) / kActCols, t.row_chunks, t.P);
   if (dtype == PM_F32) actbwd_kernel<float><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || t.row_chunks == 1) return e;
+  dim3 g2((t.max_dim + 255) / 256, t.P);
+  bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
   return cudaGetLastError();
 }
 
@@ -205,7 +238,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
   const uint64_t n_xin = (uint64_t)T * L.n_in, n_xout = (uint64_t)T * L.n_out;
   // operand sources
   const AT* xin = lin_input<AT>(t, s, d, lvl, MODE == 0);   // this Linear's input activation (forward or backward slot)
-  const AT* dz = ws_ptr<AT>(t, s.dz);
+  const AT* dz = dz_src<AT>(t, s, d, lvl);
   const WT* wf;
   if (sizeof(WT) == 4) wf = reinterpret_cast<const WT*>(t.a.w) + L.w_off;
   else wf = reinterpret_cast<const WT*>(t.a.w_lp) + L.w_off;

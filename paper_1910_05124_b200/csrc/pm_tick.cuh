@@ -17,6 +17,8 @@ struct TickArgs {
   uint64_t tgt_off;       // ws: target ring [P+1]: [T*n_out_last] float (MSE) or [T] int32 (CE)
   uint64_t pe_off;        // ws: sinusoidal positions [seq_len][d] float (0 if no embedding stage)
   uint64_t rowloss_off;   // ws: per-token losses [T] float (cross-entropy)
+  uint64_t colred_off;    // ws: per-row-chunk partial column sums [P][row_chunks][2*max_dim] float
+  int32_t row_chunks;     // ceil(T / 256)
   int32_t loss_kind;      // PM_LOSS_*
   int32_t any_pre, any_ln, any_embed, any_residual;   // which grouped launches this pipeline needs
   int32_t att_S, att_dk, att_blocks;                   // attention: sequence length, head width, (sequences x heads); 0 = none
@@ -57,6 +59,13 @@ template <typename AT> __device__ __forceinline__ const AT* gskip_read(const Tic
   const StageDev& sn = t.st[p + 1];
   return ws_at<AT>(t, sn.gin) + (uint64_t)((d.tick + 1) % 3) * ((uint64_t)t.T * sn.d_out_main);
 }
+// dz = dy * act'(z) of Linear lvl as the wgrad / dgrad operand: without an activation it IS the incoming gradient
+template <typename AT> __device__ __forceinline__ const AT* dz_src(const TickArgs& t, const StageDev& s, const StageDyn& d, int lvl) {
+  if (s.lin[lvl].act != PM_ACT_NONE) return ws_at<AT>(t, s.dz);
+  if (lvl < s.n_lin - 1) return ws_at<AT>(t, s.dh);
+  if (s.post == POST_ATTENTION) return ws_at<AT>(t, s.dy);
+  return gin_read<AT>(t, s, d);
+}
 // destination of Linear lvl's activation y in the forward pass (nullptr: not written)
 template <typename AT> __device__ __forceinline__ AT* y_dest(const TickArgs& t, int p, const StageDev& s, const StageDyn& d, int lvl) {
   const LinDev& L = s.lin[lvl];
@@ -75,6 +84,7 @@ cudaError_t launch_ingest(const TickArgs& t, int dtype, const void* inputs, cons
 cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream);
 // dz = dy * act'(z) and db = column sums, level `lvl` of every stage that runs backward this tick.
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream);
+int actbwd_launches(const TickArgs& t);
 
 // Transformer pieces (all grouped over the stages that carry the op this tick).
 cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream);        // embedding / LayerNorm forward (+ skip hand-over)

@@ -136,6 +136,10 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         if (!tl.valid) continue;
         const StageDyn& d = t.dyn[tl.p];
         const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        // dz operand: the dz scratch, or (no activation) the incoming gradient itself, which for the last Linear of a
+        // stage without attention is the rotating mailbox slot written during the previous tick
+        const StageDev& sd_ = t.st[tl.p];
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else if (MODE == 1) { tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_F32); tma_prefetch_desc(lm + MAP_D_F32); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
@@ -158,12 +162,12 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
             tma_load_2d(sb, lm + MAP_W_K, fb, k0, tl.n0);
           } else if (MODE == 1) {
             mbar_arrive_expect_tx(fb, A_BYTES);
-            tma_load_2d(sa, lm + MAP_DZ_K, fb, k0, tl.m0);
+            tma_load_3d(sa, lm + MAP_DZ_K, fb, k0, tl.m0, dz_slot);
           } else {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             const int slot = (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.b_xslot : d.b_slot;
-            tma_load_2d(sa, lm + MAP_DZ_MN, fb, tl.m0, k0);
-            tma_load_2d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, tl.m0 + 64, k0);
+            tma_load_3d(sa, lm + MAP_DZ_MN, fb, tl.m0, k0, dz_slot);
+            tma_load_3d(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, tl.m0 + 64, k0, dz_slot);
             tma_load_3d(sb, lm + MAP_ACT_MN, fb, tl.n0, k0, slot);
             tma_load_3d(sb + B_BYTES / 2, lm + MAP_ACT_MN, fb, tl.n0 + 64, k0, slot);
           }
@@ -452,10 +456,16 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
       }
       {
-        uint64_t dims[2] = {n_out, T}, strides[1] = {n_out * 2};
-        uint32_t box_k[2] = {TILE_K, TILE_M}, box_mn[2] = {64, TILE_K};
-        okm = okm && encode(fn, m + MAP_DZ_K, 0, t.ws + s.dz, 2, dims, strides, box_k, err);
-        okm = okm && encode(fn, m + MAP_DZ_MN, 0, t.ws + s.dz, 2, dims, strides, box_mn, err);
+        // dz operand (same rule as dz_src): dz scratch | dh scratch | attention's dy | rotating incoming-gradient mailbox
+        char* dzb; uint64_t dz_slots = 1;
+        if (L.act != PM_ACT_NONE) dzb = t.ws + s.dz;
+        else if (l < s.n_lin - 1) dzb = t.ws + s.dh;
+        else if (s.post == POST_ATTENTION) dzb = t.ws + s.dy;
+        else { dzb = t.ws + s.gin; dz_slots = 3; }
+        uint64_t dims[3] = {n_out, T, dz_slots}, strides[2] = {n_out * 2, T * n_out * 2};
+        uint32_t box_k[3] = {TILE_K, TILE_M, 1}, box_mn[3] = {64, TILE_K, 1};
+        okm = okm && encode(fn, m + MAP_DZ_K, 0, dzb, 3, dims, strides, box_k, err);
+        okm = okm && encode(fn, m + MAP_DZ_MN, 0, dzb, 3, dims, strides, box_mn, err);
       }
       {
         // outputs: 32-row boxes of one 128-byte swizzle row (64 bf16 or 32 fp32 columns)

@@ -402,16 +402,20 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
 }
 
 // LayerNorm parameter gradients: dgain[c] = sum_rows du_total * xhat, dbias[c] = sum_rows du_total.
-// A block owns 32 columns; warp w takes rows w, w+8, ... ascending; per-warp partials are added in warp order.
+// A block owns 32 columns and 256 rows; warp w takes rows w, w+8, ... ascending; per-warp partials are added in
+// warp order, per-block partials in block order by ln_param_finish_kernel.
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = blockIdx.z;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
   const int dm = s.d_in;
   const int c = blockIdx.x * 32 + (threadIdx.x & 31);
   if (blockIdx.x * 32 >= dm) return;
+  const int chunk = blockIdx.y;
+  const int r0 = chunk * 256, r1 = min(t.T, r0 + 256);
+  if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5;
   const uint64_t n = (uint64_t)t.T * dm;
   const AT* du = ws_at<AT>(t, s.dh);
@@ -420,7 +424,7 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
   float ag = 0.f, ab = 0.f;
   if (c < dm)
-    for (int r = warp; r < t.T; r += 8) {
+    for (int r = r0 + warp; r < r1; r += 8) {
       const uint64_t i = (uint64_t)r * dm + c;
       const float v = du_total<AT>(du, gs, i);
       const float xh = (to_f<AT>(x[i]) - st[2 * r]) * st[2 * r + 1];
@@ -435,9 +439,32 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
     float a = 0.f, b2 = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, rg[w][threadIdx.x]); b2 = __fadd_rn(b2, rb[w][threadIdx.x]); }
-    t.a.grad[s.g_off + c] = a;
-    t.a.grad[s.beta_off + c] = b2;
+    if (t.row_chunks == 1) {
+      t.a.grad[s.g_off + c] = a;
+      t.a.grad[s.beta_off + c] = b2;
+    } else {
+      float* part = ws_at<float>(t, t.colred_off) + ((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim);
+      part[c] = a;
+      part[t.max_dim + c] = b2;
+    }
   }
+}
+
+__global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
+  const int p = blockIdx.y;
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0 || s.pre != PRE_LN) return;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= s.d_in) return;
+  const float* part = ws_at<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * (2 * (uint64_t)t.max_dim);
+  float a = 0.f, b2 = 0.f;
+  for (int k = 0; k < t.row_chunks; ++k) {
+    a = __fadd_rn(a, part[(uint64_t)k * 2 * t.max_dim + c]);
+    b2 = __fadd_rn(b2, part[(uint64_t)k * 2 * t.max_dim + t.max_dim + c]);
+  }
+  t.a.grad[s.g_off + c] = a;
+  t.a.grad[s.beta_off + c] = b2;
 }
 
 // Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
@@ -481,16 +508,22 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   }
 }
 
-int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? 2 : 0) + (t.any_embed ? 1 : 0); }
+int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.row_chunks == 1 ? 2 : 3) : 0) + (t.any_embed ? 1 : 0); }
 
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
   if (t.any_ln) {
-    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + 31) / 32, t.P);
+    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + 31) / 32, t.row_chunks, t.P);
     if (dtype == PM_F32) { ln_bwd_dx_kernel<float><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<float><<<g2, 256, 0, stream>>>(t); }
     else { ln_bwd_dx_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(t); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (t.row_chunks > 1) {
+      dim3 g3((t.max_dim + 255) / 256, t.P);
+      ln_param_finish_kernel<<<g3, 256, 0, stream>>>(t);
+      e = cudaGetLastError();
+      if (e != cudaSuccess) return e;
+    }
   }
   if (t.any_embed) {
     dim3 g((t.max_vocab + 7) / 8, t.P);
