@@ -385,6 +385,264 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
   }
 }
 
+// ---- dgrad with reuse of the corrected operand -----------------------------------------------------------
+// D[T,in] = dz[T,out] * Wc[out,in].  With thousands of rows the fp32 w and delta tiles (64 KB per k-block) and
+// their conversion would be repeated for every 128-row tile; here one CTA computes up to four 128-row tiles
+// against the SAME converted tile: per k-block the staging ring receives w and delta once, the transform warps
+// write bf16(w - gap*delta) once, and the MMA warp issues one product per row tile into its own accumulator
+// (4 x 128 TMEM columns).  Traffic per 128x128x64 product drops from 80 KB to 32 KB.
+constexpr int DG_MG = 4;                                   // row tiles per B tile
+constexpr int DG_NA = 3, DG_NB = 2, DG_NG = 2;             // A ring, B (converted) ring, fp32 staging ring
+constexpr int DG_EPI_WARPS = 4;
+constexpr int DG_THREADS = 32 * (2 + 4 + DG_EPI_WARPS);
+constexpr int DG_TILE_BYTES = DG_NG * STG_BYTES + DG_NB * B_BYTES + DG_NA * A_BYTES + DG_EPI_WARPS * 4096;
+constexpr int DG_SMEM_BYTES = DG_TILE_BYTES + 1024 + 512;
+
+struct DgTile { int p, m0, n0, n_m, M, N, K, n_kb; bool valid; };
+
+__device__ __forceinline__ DgTile decode_dgrad(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
+  DgTile r;
+  int lo = 0, hi = t.P - 1;
+  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  r.p = lo;
+  const StageDyn& d = t.dyn[lo];
+  const StageDev& s = t.st[lo];
+  r.valid = lvl < s.n_lin && d.b_mb >= 0 && !(lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
+  const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
+  r.M = t.T; r.N = L.n_in; r.K = L.n_out;
+  const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
+  const int tiles_m = (r.M + TILE_M - 1) / TILE_M;
+  const int local = tile - tile_start[lo];
+  const int mg = local / tiles_n;
+  r.m0 = mg * DG_MG * TILE_M;
+  r.n0 = (local % tiles_n) * TILE_N;
+  r.n_m = min(DG_MG, tiles_m - mg * DG_MG);
+  r.n_kb = (r.K + TILE_K - 1) / TILE_K;
+  return r;
+}
+
+__global__ void __launch_bounds__(DG_THREADS, 1)
+umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, int n_tiles, int lvl, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t stg = base;                                          // [DG_NG][w 32 KB | delta 32 KB]
+  const uint32_t sB = stg + DG_NG * STG_BYTES;                        // [DG_NB][16 KB] converted operand
+  const uint32_t sA = sB + DG_NB * B_BYTES;                           // [DG_NA][16 KB] dz tiles
+  const uint32_t sO = sA + DG_NA * A_BYTES;                           // [4][4 KB] epilogue staging
+  uint8_t* stg_ptr = base_ptr;
+  uint8_t* sB_ptr = base_ptr + DG_NG * STG_BYTES;
+  uint8_t* sO_ptr = sB_ptr + DG_NB * B_BYTES + DG_NA * A_BYTES;
+  const uint32_t bars = base + DG_TILE_BYTES;
+  const uint32_t bar_sfull = bars, bar_sempty = bar_sfull + 8 * DG_NG, bar_bfull = bar_sempty + 8 * DG_NG,
+                 bar_bempty = bar_bfull + 8 * DG_NB, bar_afull = bar_bempty + 8 * DG_NB, bar_aempty = bar_afull + 8 * DG_NA,
+                 bar_tfull = bar_aempty + 8 * DG_NA, bar_tempty = bar_tfull + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + DG_TILE_BYTES + 8 * (2 * DG_NG + 2 * DG_NB + 2 * DG_NA + 2));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < DG_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, 4); }
+    for (int i = 0; i < DG_NB; ++i) { mbar_init(bar_bfull + 8 * i, 4); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < DG_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
+    mbar_init(bar_tfull, 1);
+    mbar_init(bar_tempty, DG_EPI_WARPS);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      Ring sg{0, 0}, ar{0, 0};
+      int issued_sg = 0, issued_a = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        const StageDyn& d = t.dyn[tl.p];
+        const StageDev& sd_ = t.st[tl.p];
+        const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        const bool corr = d.use_delta != 0;
+        tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_F32); tma_prefetch_desc(lm + MAP_D_F32);
+        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+          const int k0 = kb * TILE_K;
+          if (*abort_flag || !mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 21)) { ok = false; break; }
+          const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+          mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
+          tma_load_2d(sw, lm + MAP_W_F32, fb, tl.n0, k0);
+          if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, tl.n0, k0);
+          sg.advance(DG_NG); ++issued_sg;
+          for (int mi = 0; mi < tl.n_m; ++mi) {
+            if (*abort_flag || !mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 22)) { ok = false; break; }
+            const uint32_t fa = bar_afull + 8 * ar.idx;
+            mbar_arrive_expect_tx(fa, A_BYTES);
+            tma_load_3d(sA + ar.idx * A_BYTES, lm + MAP_DZ_K, fa, k0, tl.m0 + mi * TILE_M, dz_slot);
+            ar.advance(DG_NA); ++issued_a;
+          }
+        }
+      }
+      if (*abort_flag) {
+        for (int back = 1; back <= DG_NG && back <= issued_sg; ++back) {
+          const int it = issued_sg - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_sfull + 8 * (it % DG_NG), (uint32_t)(it / DG_NG) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+        for (int back = 1; back <= DG_NA && back <= issued_a; ++back) {
+          const int it = issued_a - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_afull + 8 * (it % DG_NA), (uint32_t)(it / DG_NA) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(0, 1);
+      Ring br{0, 0}, ar{0, 0};
+      uint32_t tphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        if (*abort_flag || !mbar_wait(bar_tempty, tphase ^ 1, abort_flag, status, 23)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+          if (*abort_flag || !mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 24)) { ok = false; break; }
+          const uint32_t sb = sB + br.idx * B_BYTES;
+          for (int mi = 0; mi < tl.n_m; ++mi) {
+            if (*abort_flag || !mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 25)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = sA + ar.idx * A_BYTES;
+#pragma unroll
+            for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+              tc_mma_bf16(tmem_base + (uint32_t)(mi * ACC_COLS), make_desc(sa + k16 * 32, 16, 1024), make_desc(sb + k16 * 2048, B_BYTES / 2, 1024),
+                          idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            tc_commit(bar_aempty + 8 * ar.idx);
+            ar.advance(DG_NA);
+          }
+          if (ok) tc_commit(bar_bempty + 8 * br.idx);
+          br.advance(DG_NB);
+        }
+        if (ok) tc_commit(bar_tfull);
+        tphase ^= 1;
+      }
+    }
+  } else if (warp < 6) {
+    // ---------------- operand transform: fp32 w, delta in staging -> bf16(w - gap*delta), MN-major ----------------
+    const int tt = threadIdx.x - 64;
+    const int c = tt & 15, rb = tt >> 4;
+    const uint32_t dst_in_tile = (uint32_t)(c >> 3) * (B_BYTES / 2) + (uint32_t)rb * 128 + (uint32_t)(((c & 7) ^ rb) << 4);
+    const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
+    Ring br{0, 0}, sg{0, 0};
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const float gapf = (float)t.st[tl.p].gap;
+      const bool corr = t.dyn[tl.p].use_delta != 0;
+      for (int kb = 0; kb < tl.n_kb; ++kb) {
+        bool go = !*abort_flag && mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 26);
+        go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 27);
+        go = __all_sync(0xffffffffu, go);
+        if (!go) { ok = false; break; }
+        const uint8_t* src = stg_ptr + sg.idx * STG_BYTES + src_in_tile;
+        uint8_t* dst = sB_ptr + br.idx * B_BYTES + dst_in_tile;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float4 w0 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4);
+          const float4 w1 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4 + 16);
+          float v[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+          if (corr) {
+            const float4 d0 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4);
+            const float4 d1 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4 + 16);
+            const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = __fsub_rn(v[e], __fmul_rn(gapf, dd[e]));   // w - (tau_fwd - tau_bkwd) * delta
+          }
+          *reinterpret_cast<uint4*>(dst + j * 1024) =
+              make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(bar_bfull + 8 * br.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
+        br.advance(DG_NB); sg.advance(DG_NG);
+      }
+    }
+  } else {
+    // ---------------- epilogue: one warp per TMEM lane group, 64 columns at a time through a swizzled staging buffer ----------------
+    const int q = warp & 3;
+    const int ew = warp - 6;
+    uint8_t* obuf = sO_ptr + ew * 4096;
+    const uint32_t obuf_s = sO + ew * 4096;
+    const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
+    uint32_t tphase = 0;
+    bool ok = true, stored = false;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const StageDyn& d = t.dyn[tl.p];
+      const StageDev& s = t.st[tl.p];
+      const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+      bool ready = !*abort_flag && mbar_wait(bar_tfull, tphase, abort_flag, status, 28);
+      ready = __all_sync(0xffffffffu, ready);
+      if (!ready) { ok = false; break; }
+      tc_fence_after();
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0;
+      for (int mi = 0; mi < tl.n_m; ++mi) {
+        const int mrow = tl.m0 + mi * TILE_M + q * 32;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          const int nb = tl.n0 + half * 64;
+          uint32_t r0[32], r1[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mi * ACC_COLS + half * 64);
+          tmem_ld32(taddr, r0);
+          tmem_ld32(taddr + 32, r1);
+          tmem_ld_wait();
+          if (mrow >= tl.M || nb >= tl.N) continue;
+          if (lane == 0 && stored) tma_store_wait_read();
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+            *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
+                make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) { tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, dslot); tma_store_commit(); }
+          stored = true;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty);                         // all four accumulators have been read
+      tphase ^= 1;
+    }
+    if (lane == 0 && stored) tma_store_wait_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
 // ---- host side -----------------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -507,7 +765,8 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         if (l < st[p].n_lin) {
           const LinDev& L = st[p].lin[l];
           const int M = mode == 2 ? L.n_out : t.T, N = mode == 0 ? L.n_out : L.n_in;
-          acc += cdiv(M, TILE_M) * cdiv(N, TILE_N);
+          const int tm = cdiv(M, TILE_M);
+          acc += (mode == 1 ? cdiv(tm, DG_MG) : tm) * cdiv(N, TILE_N);
         }
       }
       ts[P] = acc;
@@ -520,7 +779,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
   e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<0>::kSmemBytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
   if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
   int dev = 0;
@@ -543,7 +802,7 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   const int grid = n_tiles < plan->sms ? n_tiles : plan->sms;      // one persistent CTA per SM
   const int* ts = plan->d_tile_start + ((size_t)mode * PM_MAX_LINEARS + lvl) * (plan->P + 1);
   if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
-  else if (mode == 1) umma_gemm_kernel<1><<<grid, Cfg<1>::kThreads, Cfg<1>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
+  else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
   else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
   return cudaGetLastError();
 }
