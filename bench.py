@@ -1,18 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the PipeMare hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg3]
 
-A step is one pipeline tick of the 32-stage bf16 MLP workload (32 stages x 2 Linear(1024,1024)+GELU,
-microbatch 128) in steady state: every stage runs one forward, one backward against the
-discrepancy-corrected weights, and the fused PipeMare update.  One microbatch (128 samples) leaves
-the pipeline per tick, so samples/s = 128 * K / time.  The second half of the metric, the fused
-update's GB/s against the HBM peak, is measured live inside the same steps (`roofline`) and, on its
-own, over a parameter-count sweep (`update_sweep`).
+A step is one pipeline tick in steady state: every stage runs one forward with the weights it holds, one
+backward against the discrepancy-corrected weights for the microbatch that entered it tau_i updates ago, and
+the fused PipeMare update; one microbatch leaves the pipeline per tick.  The default workload is the largest
+one built: the 6-layer Transformer encoder (config 4; 25 stages; a sample is one sequence of 128 tokens, 32 per
+tick), which exercises every kind of stage.  The 32-stage bf16 MLP (config 3; a sample is one row, 128 per
+tick) is measured briefly in the same run and reported under `other_workload`.
 
-With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the same
-pipeline on its own GPU: the path is not sharded in this build, no collective is on the data path,
-`value` is the sum over ranks divided by the slowest rank's time.
+`roofline` describes the kernel class with the largest share of the step, timed live with CUDA events on
+the launch stream; `roofline_update` is the fused PipeMare update against the HBM peak (the second half of the
+metric), also live inside the step; `update_sweep` times that kernel alone over a parameter-count sweep.
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the same pipeline on
+its own GPU: the path is not sharded in this build, no collective is on the data path, `value` is the sum
+over ranks divided by the slowest rank's time.
 
 `--impl reference` times the CPU oracle, as it stands, on the host cores.
 """
@@ -31,9 +35,6 @@ if ROOT not in sys.path:
 METRIC = "async-pipeline train samples/s on 1 B200; PipeMare update GB/s vs HBM peak"
 UNIT = "samples/s"
 BYTES_PER_PARAM = {"sgdm": 30, "adam": 38}     # fp32 g,w,m,delta read + w,m,delta write + bf16 copy (+ s r/w)
-# DRAM traffic of one fused-update launch on the benchmark workload, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-UPDATE_TRAFFIC_BYTES = 1_976_000_000   # 2.941 GB at 100 M parameters, scaled by 67,174,400 / 100 M
 
 
 def measured_peaks():
@@ -295,30 +296,49 @@ def run_update_only(args):
     print(json.dumps({"update_only": {"n_params": n, "P": P, "ms": ms, "GB/s": 30 * n / (ms * 1e-3) / 1e9}}), flush=True)
 
 
-def run_cuda(args):
+def gemm_flops(wl):
+    """Algorithmic FLOPs of one tick per GEMM class: 2*T*in*out per Linear; the first Linear of a network fed raw
+    inputs has no input gradient."""
+    T = wl.microbatch
+    if wl.kind == "encoder":
+        lin = [(sp.n_in, sp.n_out) for sp in wl.stage_specs]
+        first_needs_dgrad = True            # the embedding needs the gradient of its output
+    else:
+        lin = [(sp.n_in, sp.n_out) for st in wl.stages for sp in st]
+        first_needs_dgrad = False
+    full = sum(2.0 * T * a * b for a, b in lin)
+    dgrad = full if first_needs_dgrad else full - 2.0 * T * lin[0][0] * lin[0][1]
+    return {"gemm_fwd": full, "wgrad": full, "dgrad": dgrad}
+
+
+# DRAM traffic per launch from ncu captures summarised under profiles/ (bytes); scaled to the benchmark workload by
+# the stated unit counts because the full-size workloads hold more device memory than a multi-pass capture may.
+NCU_TRAFFIC = {
+    # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
+    # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
+    "update_bytes_per_param": 29.41,
+}
+
+
+def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=True):
+    """Runs one workload: K timed steps with inputs resident in HBM, K profiled steps (per-class CUDA events), and
+    K end-to-end steps from pinned host buffers.  Returns a dict of results (rank 0 consumes it)."""
     import torch
-    import pm_inputs as I
     import paper_1910_05124_b200 as pm
-    world, rank, local = dist_setup(args.gpus)
-    device = torch.device(f"cuda:{local}")
-    torch.cuda.set_device(device)
-    hbm_peak, tf_peak, peak_kind = measured_peaks()
-    wl, params0, samples_per_step, n_params = build_workload(args)
+    a2 = argparse.Namespace(**vars(args))
+    a2.workload = workload
+    wl, params0, samples_per_step, n_params = build_workload(a2)
     P = wl.n_stages
     pipe = pm.Pipeline(wl, params0, device=str(device))
     host_b, dev_b = make_batches(wl, 4, device)
-
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    # fill the pipeline (2P-1 ticks) and warm up
+    warm = max(args.warmup, 3)
     fill = 2 * P - 1
-    for s in range(fill + max(args.warmup, 3)):
+    for s in range(fill + warm):
         pipe.pm_step(*dev_b[s % len(dev_b)])
     torch.cuda.synchronize(device)
 
-    # ---- timed region 1: K steps, inputs resident in HBM --------------------------------------------
-    if rank == 0:
+    # ---- timed region 1: K steps, inputs resident in HBM
+    if sampler is not None:
         sampler.wait_first()
         sampler.mark()
     launches0 = pipe.pm_launch_count()
@@ -334,70 +354,131 @@ def run_cuda(args):
     elapsed_ms = e0.elapsed_time(e1)
     launches = pipe.pm_launch_count() - launches0
     t_ms, units = reduce_over_ranks(elapsed_ms, samples_per_step * args.steps, world, device)
-    value = units / (t_ms * 1e-3)
 
-    # ---- timed region 2: the update kernel alone inside the step (CUDA events on the launch stream) --
-    upd_ms = []
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    # ---- timed region 2: the same K steps with CUDA events around every launch (on the launch stream)
+    pipe.pm_profile_enable(True)
     for s in range(args.steps):
-        x, y = dev_b[s % len(dev_b)]
-        pipe.pm_forward(x, y)
-        pipe.pm_backward()
-        ev[s][0].record()
-        pipe.pm_update()
-        ev[s][1].record()
-    torch.cuda.synchronize(device)
-    clocks = sampler.stop() if rank == 0 else None
-    upd_ms = [a.elapsed_time(b) for a, b in ev]
-    upd_avg = sum(upd_ms) / len(upd_ms)
-    alg_bytes = BYTES_PER_PARAM[wl.optimizer] * n_params
-    achieved = alg_bytes / (upd_avg * 1e-3) / 1e9
+        pipe.pm_step(*dev_b[s % len(dev_b)])
+    prof = pipe.pm_profile_read()
+    pipe.pm_profile_enable(False)
+    clocks = sampler.stop() if sampler is not None else None
+    per_tick = {k: v[0] / args.steps for k, v in prof.items() if v[1] > 0}
+    total_prof = sum(per_tick.values())
 
-    # ---- timed region 3: end to end through the C ABI with host buffers -----------------------------
-    xin = torch.empty_like(dev_b[0][0])
-    yin = torch.empty_like(dev_b[0][1])
-    barrier(world)
-    torch.cuda.synchronize(device)
-    loss_sink = 0.0
-    t0 = time.perf_counter()
-    for s in range(args.steps):
-        hx, hy = host_b[s % len(host_b)]
-        xin.copy_(hx, non_blocking=True)
-        yin.copy_(hy, non_blocking=True)
-        pipe.pm_step(xin, yin)
-        # loss of the microbatch whose backward started this tick: device -> host, synchronises
-        mb_done = fill + max(args.warmup, 3) + 2 * args.steps + s - P
-        loss_sink += float(pipe.pm_get_losses(mb_done, 1)[0])
-    torch.cuda.synchronize(device)
-    e2e_ms = (time.perf_counter() - t0) * 1e3
-    barrier(world)
-    e2e_t, e2e_units = reduce_over_ranks(e2e_ms, samples_per_step * args.steps, world, device)
-    h2d = sum(x.numel() * x.element_size() for x in host_b[0])
+    res = {"wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params,
+           "t_ms": t_ms, "units": units, "launches": launches, "clocks": clocks, "per_tick_ms": per_tick,
+           "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "prof": prof, "total_prof": total_prof}
 
+    # ---- timed region 3: end to end through the C ABI with host buffers
+    if with_e2e:
+        xin = torch.empty_like(dev_b[0][0])
+        yin = torch.empty_like(dev_b[0][1])
+        barrier(world)
+        torch.cuda.synchronize(device)
+        loss_sink = 0.0
+        t0 = time.perf_counter()
+        for s in range(args.steps):
+            hx, hy = host_b[s % len(host_b)]
+            xin.copy_(hx, non_blocking=True)
+            yin.copy_(hy, non_blocking=True)
+            pipe.pm_step(xin, yin)
+            # loss of the microbatch whose backward started this tick: device -> host, synchronises
+            mb_done = fill + warm + 2 * args.steps + s - P
+            loss_sink += float(pipe.pm_get_losses(mb_done, 1)[0])
+        torch.cuda.synchronize(device)
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+        barrier(world)
+        e2e_t, e2e_units = reduce_over_ranks(e2e_ms, samples_per_step * args.steps, world, device)
+        res.update(e2e_t=e2e_t, e2e_units=e2e_units, h2d=sum(x.numel() * x.element_size() for x in host_b[0]),
+                   last_loss=loss_sink / args.steps)
+    pipe.close()
+    del pipe
+    torch.cuda.empty_cache()
+    return res
+
+
+def rooflines(res, hbm_peak, tf_peak, peak_kind, steps):
+    """Roofline objects: the dominant kernel class of the step, and the fused update against HBM."""
+    wl, per_tick = res["wl"], res["per_tick_ms"]
+    step_ms = res["t_ms"] / steps
+    upd_ms = per_tick.get("update", 0.0)
+    alg_bytes = BYTES_PER_PARAM[wl.optimizer] * res["n_params"]
+    upd_gbs = alg_bytes / (upd_ms * 1e-3) / 1e9 if upd_ms > 0 else 0.0
+    update = {"kernel": "update_kernel (fused PipeMare update)", "bound": "hbm", "achieved": round(upd_gbs, 1),
+              "peak": hbm_peak, "unit": "GB/s", "frac": round(upd_gbs / hbm_peak, 4), "of": peak_kind,
+              "traffic": int(NCU_TRAFFIC["update_bytes_per_param"] * alg_bytes / 30.0),
+              "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": round(upd_ms, 5),
+              "frac_of_nominal_8TBs": round(upd_gbs / 8000.0, 4), "share_of_step": round(upd_ms / res["total_prof"], 4)}
+    dominant = max(per_tick, key=per_tick.get)
+    if dominant == "update":
+        return update, update
+    flops = gemm_flops(wl)
+    if dominant in flops:
+        launches = res["prof"][dominant][1] / steps
+        tfs = flops[dominant] / (per_tick[dominant] * 1e-3) / 1e12
+        names = {"gemm_fwd": "umma_gemm_kernel<0> (forward GEMMs)", "wgrad": "umma_gemm_kernel<2> (wgrad GEMMs)",
+                 "dgrad": "umma_dgrad_kernel (dgrad GEMMs, weights corrected while loading)"}
+        dom = {"kernel": names[dominant], "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
+               "frac": round(tfs / tf_peak, 4), "of": peak_kind + " (sustained bf16 matmul)", "traffic": None,
+               "algorithmic_flops_per_step": flops[dominant], "launches_per_step": launches,
+               "avg_ms_per_step": round(per_tick[dominant], 5), "frac_of_nominal_2250TFs": round(tfs / 2250.0, 4),
+               "share_of_step": round(per_tick[dominant] / res["total_prof"], 4)}
+        return dom, update
+    dom = {"kernel": dominant, "bound": "alu", "achieved": None, "peak": None, "unit": None, "frac": None, "traffic": None,
+           "avg_ms_per_step": round(per_tick[dominant], 5), "share_of_step": round(per_tick[dominant] / res["total_prof"], 4)}
+    return dom, update
+
+
+def run_cuda(args):
+    import torch
+    world, rank, local = dist_setup(args.gpus)
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler is not None:
+        sampler.start()
+    res = measure(args, args.workload, world, rank, local, device, sampler)
+    other = None
+    if world == 1 and not args.no_other and not args.stages:
+        other_name = "cfg3" if args.workload == "cfg4" else "cfg4"
+        other = measure(args, other_name, world, rank, local, device, None, with_e2e=False)
     if rank != 0:
         return
+    wl, P = res["wl"], res["P"]
+    value = res["units"] / (res["t_ms"] * 1e-3)
+    dom, upd = rooflines(res, hbm_peak, tf_peak, peak_kind, args.steps)
+    flops = gemm_flops(wl)
+    gemm_ms = sum(res["per_tick_ms"].get(k, 0.0) for k in flops)
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": round(t_ms / args.steps, 5), "higher_is_better": True,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(res["t_ms"] / args.steps, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
                    "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
-                   "samples_per_step": samples_per_step,
-                   "pipeline_fill_ticks": fill, "cache": "per-step working set (state + rings, see state_bytes) far exceeds the 126 MB L2: no flush needed",
-                   "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "params": n_params},
-        "clocks": clocks,
-        "e2e": {"value": round(e2e_units / (e2e_t * 1e-3), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": 4, "ms_per_step": round(e2e_t / args.steps, 5), "last_loss": loss_sink / args.steps},
-        "gpu_launches": launches,
-        "roofline": {"kernel": "update_kernel (fused PipeMare update)", "bound": "hbm", "achieved": round(achieved, 1),
-                     "peak": hbm_peak, "unit": "GB/s", "frac": round(achieved / hbm_peak, 4), "of": peak_kind,
-                     "traffic": UPDATE_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": alg_bytes,
-                     "avg_launch_ms": round(upd_avg, 5), "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
-                     "share_of_step": round(upd_avg / (t_ms / args.steps), 4)},
+                   "samples_per_step": res["samples_per_step"], "pipeline_fill_ticks": res["fill"],
+                   "cache": "per-step working set (state + rings, see state_bytes) far exceeds the 126 MB L2: no flush needed",
+                   "ring_bytes": res["ring_bytes"], "state_bytes": res["state_bytes"], "params": res["n_params"]},
+        "clocks": res["clocks"],
+        "e2e": {"value": round(res["e2e_units"] / (res["e2e_t"] * 1e-3), 2), "unit": UNIT, "h2d_bytes_per_step": res["h2d"],
+                "d2h_bytes_per_step": 4, "ms_per_step": round(res["e2e_t"] / args.steps, 5), "last_loss": res["last_loss"]},
+        "gpu_launches": res["launches"],
+        "roofline": dom,
+        "roofline_update": upd,
+        "gemm_all": {"TFLOP/s": round(sum(flops.values()) / (gemm_ms * 1e-3) / 1e12, 1) if gemm_ms > 0 else None,
+                     "frac_of_measured_sustained": round(sum(flops.values()) / (gemm_ms * 1e-3) / 1e12 / tf_peak, 4) if gemm_ms > 0 else None,
+                     "ms_per_step": round(gemm_ms, 5)},
+        "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(res["per_tick_ms"].items(), key=lambda kv: -kv[1])},
     }
+    if other is not None:
+        od, ou = rooflines(other, hbm_peak, tf_peak, peak_kind, args.steps)
+        line["other_workload"] = {"workload": WORKLOADS["cfg3" if args.workload == "cfg4" else "cfg4"],
+                                  "value": round(other["units"] / (other["t_ms"] * 1e-3), 2), "unit": UNIT,
+                                  "ms_per_step": round(other["t_ms"] / args.steps, 5), "roofline": od, "roofline_update": ou,
+                                  "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(other["per_tick_ms"].items(), key=lambda kv: -kv[1])}}
     if world == 1:
         if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, samples_per_step)
+            line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, res["samples_per_step"])
         if not args.no_sweep:
             line["update_sweep"] = update_sweep(device, hbm_peak)
     print(json.dumps(line), flush=True)
@@ -406,54 +487,86 @@ def run_cuda(args):
 # ---- the reference arm: the CPU oracle -------------------------------------------------------------
 
 def run_reference(args):
-    """Times the oracle on the host cores.  Each step is one microbatch through a contiguous sample of
-    the workload's stages (as many as keep the whole run within a few minutes); throughput is scaled by
-    the fraction of stages sampled, since every stage costs the same."""
+    """Times the oracle on the host cores on a bounded sample of the same workload, sized after a pilot step so
+    that the whole run stays within a few minutes.  cfg3: each step sends one microbatch through the first n of
+    the 32 (identical) stages.  cfg4: each step sends b of the 32 sequences through l of the 6 layers plus the
+    embedding and vocabulary stages.  Throughput is scaled to the full workload by the sampled fraction of its
+    matrix-product FLOPs."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import pm_inputs as I
-    from oracle.mlp import run_workload
-    full = I.cfg3()
     budget_s = 150.0
     total_steps = args.steps + args.warmup
-
-    def sub_workload(n_stages):
-        wl = I.mlp_workload(full.name, n_stages, 1024, 2, "gelu", full.microbatch, compute="bf16",
-                            optimizer=full.optimizer, alpha=full.alpha, beta1=full.beta1, K=full.K, D=full.D,
-                            steps=total_steps, seed=full.seed)
-        return wl
-
-    # pilot: one step of one stage
-    wl1 = sub_workload(1)
-    p1, t1 = I.init_stage_params(wl1), I.teacher_params(wl1)
-    b1 = I.batch(wl1, 0, t1)
-    t0 = time.perf_counter()
-    run_workload(wl1, p1, lambda t: b1, n_steps=2)
-    per_stage_step = (time.perf_counter() - t0) / 2
-    n_stages = int(max(1, min(full.n_stages, budget_s / (total_steps * per_stage_step))))
-    wl = sub_workload(n_stages)
-    params0, teacher = I.init_stage_params(wl), I.teacher_params(wl)
-    batches = [I.batch(wl, t, teacher) for t in range(min(total_steps, 4))]
     marks = {}
 
     def on_step(t, w):
         if t == args.warmup - 1:
             marks["t0"] = time.perf_counter()
 
+    if args.workload == "cfg3":
+        from oracle.mlp import run_workload
+        full = I.cfg3()
+
+        def sub(n_stages):
+            return I.mlp_workload(full.name, n_stages, 1024, 2, "gelu", full.microbatch, compute="bf16",
+                                  optimizer=full.optimizer, alpha=full.alpha, beta1=full.beta1, K=full.K, D=full.D,
+                                  steps=total_steps, seed=full.seed)
+        wl1 = sub(1)
+        p1, t1 = I.init_stage_params(wl1), I.teacher_params(wl1)
+        b1 = I.batch(wl1, 0, t1)
+        t0 = time.perf_counter()
+        run_workload(wl1, p1, lambda t: b1, n_steps=2)
+        per_stage_step = (time.perf_counter() - t0) / 2
+        n_stages = int(max(1, min(full.n_stages, budget_s / (total_steps * per_stage_step))))
+        wl = sub(n_stages)
+        params0, teacher = I.init_stage_params(wl), I.teacher_params(wl)
+        batches = [I.batch(wl, t, teacher) for t in range(min(total_steps, 4))]
+        scale = n_stages / full.n_stages
+        samples_per_step = full.microbatch
+        sample = (f"each step: one microbatch of 128 through {n_stages} of the {full.n_stages} stages "
+                  f"(forward, backward, update); samples/s scaled by {n_stages}/{full.n_stages}")
+    else:
+        from oracle.transformer import run_workload
+        full = I.cfg4()
+
+        def sub(layers, seqs):
+            return I.encoder_workload(full.name, layers, 512, 8, 2048, 128, seqs, 8192, compute="bf16", optimizer="adam",
+                                      alpha=full.alpha, beta1=0.9, beta2=0.98, eps=1e-8, K=full.K, D=full.D,
+                                      steps=total_steps, seed=full.seed)
+
+        def mm_flops(layers, seqs):
+            per_layer = 512 * (1536 + 512 + 2048 + 2048)
+            return 6.0 * seqs * 128 * (layers * per_layer + 512 * 8192)
+        wl1 = sub(1, 4)
+        p1 = I.init_encoder_params(wl1)
+        b1 = I.token_batch(wl1, 0)
+        t0 = time.perf_counter()
+        run_workload(wl1, p1, lambda t: b1, n_steps=1)
+        pilot = time.perf_counter() - t0
+        per_flop = pilot / mm_flops(1, 4)
+        layers, seqs = 6, 32
+        while layers > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
+            layers -= 1
+        while seqs > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
+            seqs //= 2
+        wl = sub(layers, seqs)
+        params0 = I.init_encoder_params(wl)
+        batches = [I.token_batch(wl, t) for t in range(min(total_steps, 4))]
+        scale = mm_flops(layers, seqs) / mm_flops(6, 32)
+        samples_per_step = 32
+        sample = (f"each step: {seqs} of the 32 sequences through {layers} of the 6 layers plus embedding and "
+                  f"vocabulary stages (forward, backward, update); samples/s scaled by the sampled fraction "
+                  f"{scale:.4f} of the workload's matrix-product FLOPs")
     if args.warmup == 0:
         marks["t0"] = time.perf_counter()
     run_workload(wl, params0, lambda t: batches[t % len(batches)], n_steps=total_steps, on_step=on_step)
     dt = time.perf_counter() - marks["t0"]
-    scale = n_stages / full.n_stages
-    value = full.microbatch * args.steps / dt * scale
-    sample = (f"each step: one microbatch of 128 through {n_stages} of the {full.n_stages} stages "
-              f"(forward, backward, update); samples/s scaled by {n_stages}/{full.n_stages}")
+    value = samples_per_step * args.steps / dt * scale
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3 / scale, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, microbatch 128 "
-                                   "(CPU oracle, bf16-rounded operands, float64 accumulation)"},
+            "config": {"workload": WORKLOADS[args.workload] + " (CPU oracle, bf16-rounded operands, float64 accumulation)"},
             "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -467,7 +580,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the stand-alone update sweep")
-    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-other", action="store_true", help="skip the short run of the other built workload")
     ap.add_argument("--stages", type=int, default=0, help="profiling runs: same workload cut to this many stages")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
     ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",

@@ -193,6 +193,16 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
 /* Number of CUDA kernels this context has enqueued since pm_init_stages (for launch accounting). */
 uint64_t pm_launch_count(pm_ctx* ctx);
 
+/* Optional timing of the tick's kernels by class, with CUDA events recorded on the context's stream around each
+ * launch (up to 8192 launches between reads; later ones are not recorded).  pm_profile_read synchronises the
+ * stream, writes the summed milliseconds and the number of timed launches per class (arrays of PM_PROF_CLASSES
+ * entries) and clears the record. */
+enum { PM_PROF_SCHEDULE = 0, PM_PROF_INGEST, PM_PROF_PRE_FWD, PM_PROF_GEMM_FWD, PM_PROF_ATTN_FWD, PM_PROF_POST_FWD,
+       PM_PROF_LOSS, PM_PROF_ATTN_BWD, PM_PROF_ACT_BWD, PM_PROF_WGRAD, PM_PROF_DGRAD, PM_PROF_PRE_BWD, PM_PROF_UPDATE,
+       PM_PROF_CLASSES };
+pm_status pm_profile_enable(pm_ctx* ctx, int32_t on);
+pm_status pm_profile_read(pm_ctx* ctx, float* ms_by_class, int64_t* launches_by_class);
+
 const char* pm_last_error(pm_ctx* ctx);   /* never NULL; ctx may be NULL (global message) */
 void pm_destroy(pm_ctx* ctx);
 

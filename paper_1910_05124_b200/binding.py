@@ -82,6 +82,8 @@ def lib():
     L.pm_get_losses.argtypes = [vp, C.POINTER(C.c_float), C.c_int64, C.c_int64]
     L.pm_launch_count.argtypes = [vp]
     L.pm_launch_count.restype = C.c_uint64
+    L.pm_profile_enable.argtypes = [vp, C.c_int32]
+    L.pm_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.pm_destroy.argtypes = [vp]
     L.pm_destroy.restype = None
     L.pm_update_flat_workspace_bytes.argtypes = [C.c_int32]
@@ -283,6 +285,19 @@ class Pipeline:
 
     def pm_launch_count(self):
         return int(self.L.pm_launch_count(self.ctx))
+
+    PROF_CLASSES = ["schedule", "ingest", "pre_fwd", "gemm_fwd", "attn_fwd", "post_fwd", "loss", "attn_bwd", "act_bwd",
+                    "wgrad", "dgrad", "pre_bwd", "update"]
+
+    def pm_profile_enable(self, on=True):
+        _check(self.L.pm_profile_enable(self.ctx, int(bool(on))), self.ctx)
+
+    def pm_profile_read(self):
+        """{class name: (milliseconds, launches)} since the last read."""
+        n = len(self.PROF_CLASSES)
+        ms, cnt = (C.c_float * n)(), (C.c_int64 * n)()
+        _check(self.L.pm_profile_read(self.ctx, ms, cnt), self.ctx)
+        return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(self.PROF_CLASSES)}
 
     # -- marshalling helpers --------------------------------------------------------------------
     def unpack(self, flat_tensor):

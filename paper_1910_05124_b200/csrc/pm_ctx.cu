@@ -246,7 +246,13 @@ struct pm_ctx {
   std::string err;
   UmmaPlan* umma = nullptr;
   AttnPlan* attn = nullptr;
-  uint64_t launches = 0;   // kernels enqueued by this context so far
+  uint64_t launches = 0;
+  // optional per-kernel-class timing with CUDA events on the context's stream
+  bool prof_on = false;
+  int prof_cls = 0;
+  std::vector<cudaEvent_t> prof_ev;          // pairs: start, stop
+  std::vector<int> prof_pair_cls;
+  size_t prof_used = 0;   // kernels enqueued by this context so far
 };
 
 namespace {
@@ -423,8 +429,21 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
 // every call checked here enqueued `kernels` kernels
 static pm_status check(pm_ctx* ctx, cudaError_t e, const char* what, int kernels = 1) {
   ctx->launches += kernels;
+  if (ctx->prof_on && ctx->prof_cls >= 0 && ctx->prof_used < ctx->prof_pair_cls.size()) {
+    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream);
+    ctx->prof_pair_cls[ctx->prof_used] = ctx->prof_cls;
+    ctx->prof_used += 1;
+    ctx->prof_cls = -1;
+  }
   return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, what);
 }
+// marks the start of a timed launch of class `cls`; the matching stop is recorded by check()
+static inline void prof_begin(pm_ctx* ctx, int cls) {
+  if (!ctx->prof_on || ctx->prof_used >= ctx->prof_pair_cls.size()) { ctx->prof_cls = -1; return; }
+  ctx->prof_cls = cls;
+  cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream);
+}
+#define TIMED(cls, call) (prof_begin(ctx, cls), call)
 
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
@@ -434,24 +453,25 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   const int dt = ctx->cfg.compute_dtype;
   pm_status s;
   if (inputs) ctx->n_fed = ctx->tick + 1; else ctx->draining = true;
-  s = check(ctx, launch_schedule((const StageSched*)(ctx->ws + ctx->L.off_sched), (const int64_t*)(ctx->ws + ctx->L.off_nupd),
-                                 (StageDyn*)(ctx->ws + ctx->L.off_dyn), ctx->hp, ctx->tick, ctx->n_fed, -1, ctx->stream), "schedule");
+  s = TIMED(PM_PROF_SCHEDULE, check(ctx, launch_schedule((const StageSched*)(ctx->ws + ctx->L.off_sched), (const int64_t*)(ctx->ws + ctx->L.off_nupd),
+                                 (StageDyn*)(ctx->ws + ctx->L.off_dyn), ctx->hp, ctx->tick, ctx->n_fed, -1, ctx->stream), "schedule"));
   if (s != PM_OK) return s;
   if (inputs) {
-    s = check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, ctx->tick, ctx->stream), "ingest");
+    s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, ctx->tick, ctx->stream), "ingest"));
     if (s != PM_OK) return s;
   }
   // forward of every stage whose microbatch exists: s - (i-1) in [0, n_fed)
   if (ctx->tick - (ctx->cfg.n_stages - 1) < ctx->n_fed) {
-    if (ctx->L.any_pre && (s = check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->stream), "embedding / LayerNorm forward")) != PM_OK) return s;
+    if (ctx->L.any_pre && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->stream), "embedding / LayerNorm forward"))) != PM_OK) return s;
     for (int l = 0; l < ctx->L.max_lin; ++l) {
+      prof_begin(ctx, PM_PROF_GEMM_FWD);
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 0, l, ctx->stream)
                                    : umma_launch(ctx->umma, ctx->ta, 0, l, ctx->stream);
       if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
     }
-    if (ctx->attn && (s = check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->stream), "attention forward")) != PM_OK) return s;
+    if (ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->stream), "attention forward"))) != PM_OK) return s;
     const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
-    if (n_post && (s = check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream, ctx->attn != nullptr), "attention / residual forward", n_post)) != PM_OK) return s;
+    if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
   }
   ctx->phase = 1;
   return PM_OK;
@@ -466,20 +486,22 @@ pm_status pm_backward(pm_ctx* ctx) {
   // any backward this tick?  stage P runs microbatch tick-P, stage 1 runs tick-(2P-1)
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
-    if ((s = check(ctx, launch_loss(ctx->ta, dt, ctx->stream), "loss")) != PM_OK) return s;
-    if (ctx->attn) { if ((s = check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->stream), "attention backward")) != PM_OK) return s; }
-    else if (ctx->L.att_blocks > 0 && (s = check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward")) != PM_OK) return s;
+    if ((s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ctx->ta, dt, ctx->stream), "loss"))) != PM_OK) return s;
+    if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->stream), "attention backward"))) != PM_OK) return s; }
+    else if (ctx->L.att_blocks > 0 && (s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward"))) != PM_OK) return s;
     for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
-      if ((s = check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward", actbwd_launches(ctx->ta))) != PM_OK) return s;
+      if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward", actbwd_launches(ctx->ta)))) != PM_OK) return s;
+      prof_begin(ctx, PM_PROF_WGRAD);
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->stream)
                                    : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->stream);
       if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+      prof_begin(ctx, PM_PROF_DGRAD);
       e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 1, l, ctx->stream)
                        : umma_launch(ctx->umma, ctx->ta, 1, l, ctx->stream);
       if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
     }
     const int n_pre = pre_bwd_launches(ctx->ta);
-    if (n_pre && (s = check(ctx, launch_pre_bwd(ctx->ta, dt, ctx->stream), "LayerNorm / embedding backward", n_pre)) != PM_OK) return s;
+    if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ctx->ta, dt, ctx->stream), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
   }
   ctx->phase = 2;
   return PM_OK;
@@ -491,6 +513,7 @@ pm_status pm_update(pm_ctx* ctx) {
   const int P = ctx->cfg.n_stages;
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
+    prof_begin(ctx, PM_PROF_UPDATE);
     cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
                                   (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
                                   ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->stream);
@@ -554,12 +577,44 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
 
 uint64_t pm_launch_count(pm_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+pm_status pm_profile_enable(pm_ctx* ctx, int32_t on) {
+  if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
+  if (on && ctx->prof_ev.empty()) {
+    const size_t pairs = 8192;
+    ctx->prof_ev.resize(2 * pairs);
+    for (auto& ev : ctx->prof_ev)
+      if (cudaEventCreate(&ev) != cudaSuccess) { ctx->prof_ev.clear(); return fail(ctx, PM_ERR_CUDA, "cudaEventCreate failed"); }
+    ctx->prof_pair_cls.assign(pairs, 0);
+  }
+  ctx->prof_on = on != 0;
+  ctx->prof_used = 0;
+  ctx->prof_cls = -1;
+  return PM_OK;
+}
+
+pm_status pm_profile_read(pm_ctx* ctx, float* ms_by_class, int64_t* launches_by_class) {
+  if (!ctx || !ms_by_class || !launches_by_class) return fail(ctx, PM_ERR_INVALID_ARG, "null argument");
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "profile read");
+  for (int i = 0; i < PM_PROF_CLASSES; ++i) { ms_by_class[i] = 0.f; launches_by_class[i] = 0; }
+  for (size_t i = 0; i < ctx->prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]) == cudaSuccess) {
+      ms_by_class[ctx->prof_pair_cls[i]] += ms;
+      launches_by_class[ctx->prof_pair_cls[i]] += 1;
+    }
+  }
+  ctx->prof_used = 0;
+  return PM_OK;
+}
+
 const char* pm_last_error(pm_ctx* ctx) { return ctx ? ctx->err.c_str() : g_error.c_str(); }
 
 void pm_destroy(pm_ctx* ctx) {
   if (!ctx) return;
   umma_plan_destroy(ctx->umma);
   attn_plan_destroy(ctx->attn);
+  for (auto& ev : ctx->prof_ev) cudaEventDestroy(ev);
   delete ctx;
 }
 

@@ -55,6 +55,20 @@ __device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
          ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 }
 
+// forward epilogue for 8 columns: z = bf16(acc + bias), y = bf16(act(z)); the activation is a template parameter so
+// that Linears without GELU never pay for erff
+template <int ACT>
+__device__ __forceinline__ void epi_zy8(const float (&pf)[8], uint8_t* zdst, uint8_t* ydst) {
+  float zf[8], yf[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    zf[e] = __bfloat162float(__float2bfloat16_rn(pf[e]));
+    yf[e] = ACT == PM_ACT_RELU ? fmaxf(zf[e], 0.0f) : (ACT == PM_ACT_GELU ? act_fwd(zf[e], PM_ACT_GELU) : zf[e]);
+  }
+  *reinterpret_cast<uint4*>(zdst) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
+  *reinterpret_cast<uint4*>(ydst) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
+}
+
 // ---- tile walk ---------------------------------------------------------------------------------------
 // tile_start[p] .. tile_start[p+1] are the flattened tile ids of stage p for this (mode, level).
 struct Tile { int p, m0, n0, M, N, K, n_kb; bool valid; };
@@ -305,6 +319,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       if (MODE == 0) {
         const float* bias = t.a.w + L.b_off;
         const bool f32out = (L.flags & LF_OUT_F32) != 0;
+        const int act = L.act;
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const int n = nb + g * 8;
@@ -322,15 +337,10 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
             *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2) ^ sw) << 4)) = make_float4(pf[0], pf[1], pf[2], pf[3]);
             *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
           } else {
-            float zf[8], yf[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              zf[e] = __bfloat162float(__float2bfloat16_rn(pf[e]));
-              yf[e] = act_fwd(zf[e], L.act);
-            }
             const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
-            *reinterpret_cast<uint4*>(obuf + off) = make_uint4(pack_bf16(zf[0], zf[1]), pack_bf16(zf[2], zf[3]), pack_bf16(zf[4], zf[5]), pack_bf16(zf[6], zf[7]));
-            *reinterpret_cast<uint4*>(obuf + 4096 + off) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
+            if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
+            else if (act == PM_ACT_RELU) epi_zy8<PM_ACT_RELU>(pf, obuf + off, obuf + 4096 + off);
+            else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);
           }
         }
       } else if (MODE == 1) {
