@@ -83,7 +83,7 @@ __device__ __forceinline__ void attn_teardown(const AttnCommon& c, uint32_t tmem
 
 // all threads: wait for an MMA batch; returns false (uniformly) if any thread gave up
 __device__ __forceinline__ bool wait_mma(const AttnCommon& c, uint32_t parity, int* status, int code) {
-  bool ok = !*c.abort_flag && mbar_wait(c.bar_mma, parity, c.abort_flag, status, code);
+  bool ok = mbar_wait(c.bar_mma, parity, c.abort_flag, status, code);
   ok = __syncthreads_and(ok);
   tc_fence_after();
   return ok;

@@ -31,8 +31,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag and the global status word) when the
 // barrier did not flip within the cycle limit or another role of this CTA has already given up.
-static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
+// The first poll is inlined: on the hot path a ready barrier costs one try_wait.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
@@ -45,6 +45,10 @@ static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, vol
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -126,6 +130,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+
+// The same descriptor split into its address-independent part and the start address, so that issuing loops add
+// only the address: desc = desc_base(leading, stride) + (saddr >> 4)   (valid while saddr < 256 KB).
+__device__ __forceinline__ uint64_t desc_base(uint32_t leading_bytes, uint32_t stride_bytes) {
+  return make_desc(0, leading_bytes, stride_bytes);
+}
+__device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t saddr) { return base + (uint64_t)(saddr >> 4); }
 
 // Instruction descriptor: bf16 x bf16 -> fp32 accumulate, M x N tile, operand majors as given (0 = K-major, 1 = MN-major).
 __device__ __forceinline__ uint32_t make_idesc_mn(int M, int N, int a_mn_major, int b_mn_major) {

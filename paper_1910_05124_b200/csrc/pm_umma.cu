@@ -160,7 +160,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         for (int kb = 0; kb < tl.n_kb; ++kb) {
           const int k0 = kb * TILE_K;
           if (MODE == 1) {
-            if (*abort_flag || !mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 5)) { ok = false; break; }
+            if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 5)) { ok = false; break; }
             const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
             const bool corr = d.use_delta != 0;
             mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
@@ -168,7 +168,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
             if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, tl.n0, k0);
             sg.advance(NG); ++issued_sg;
           }
-          if (*abort_flag || !mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 1)) { ok = false; break; }
+          if (!mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 1)) { ok = false; break; }
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * op.idx;
           if (MODE == 0) {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
@@ -206,25 +206,25 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = make_idesc(MODE == 2, MODE != 0);
+      // K-major: 16 elements = 32 bytes along the swizzled row.  MN-major: 16 k-rows of 128 bytes.
+      const uint64_t dba = MODE == 2 ? desc_base(A_BYTES / 2, 1024) : desc_base(16, 1024);
+      const uint64_t dbb = MODE == 0 ? desc_base(16, 1024) : desc_base(B_BYTES / 2, 1024);
+      const uint32_t ka = MODE == 2 ? 2048 : 32, kb_ = MODE == 0 ? 32 : 2048;
       Ring op{0, 0}, acc{0, 0};
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
-        if (*abort_flag || !mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 6)) { ok = false; break; }
+        if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 6)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * ACC_COLS);
         for (int kb = 0; kb < tl.n_kb; ++kb) {
-          if (*abort_flag || !mbar_wait(bar_full + 8 * op.idx, op.phase, abort_flag, status, 2)) { ok = false; break; }
+          if (!mbar_wait(bar_full + 8 * op.idx, op.phase, abort_flag, status, 2)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
-          for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
-            // K-major: 16 elements = 32 bytes along the swizzled row.  MN-major: 16 k-rows of 128 bytes.
-            const uint64_t da = MODE == 2 ? make_desc(sa + k16 * 2048, A_BYTES / 2, 1024) : make_desc(sa + k16 * 32, 16, 1024);
-            const uint64_t db = MODE == 0 ? make_desc(sb + k16 * 32, 16, 1024) : make_desc(sb + k16 * 2048, B_BYTES / 2, 1024);
-            tc_mma_bf16(tmem_acc, da, db, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
-          }
+          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+            tc_mma_bf16(tmem_acc, desc_at(dba, sa + k16 * ka), desc_at(dbb, sb + k16 * kb_), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
           tc_commit(bar_empty + 8 * op.idx);      // frees the operand slot once these MMAs have read it
           op.advance(NS);
         }
@@ -247,7 +247,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         const float gapf = (float)t.st[tl.p].gap;
         const bool corr = t.dyn[tl.p].use_delta != 0;
         for (int kb = 0; kb < tl.n_kb; ++kb) {
-          bool go = !*abort_flag && mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 7);
+          bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 7);
           go = go && mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 3);
           go = __all_sync(0xffffffffu, go);                           // leave the loops as a whole warp
           if (!go) { ok = false; break; }
@@ -298,7 +298,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
       const int mrow = tl.m0 + q * 32;                                // first row of this warp's block
       const int nb = tl.n0 + half * 64;
-      bool ready = !*abort_flag && mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
+      bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
       tc_fence_after();
@@ -404,7 +404,8 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
 constexpr int DG_MG = 4;                                   // row tiles per B tile
 constexpr int DG_NA = 3, DG_NB = 2, DG_NG = 2;             // A ring, B (converted) ring, fp32 staging ring
 constexpr int DG_EPI_WARPS = 4;
-constexpr int DG_THREADS = 32 * (2 + 4 + DG_EPI_WARPS);
+constexpr int DG_XF_WARPS = 8;                             // transform warps: 32 of the 64 k-rows per half
+constexpr int DG_THREADS = 32 * (2 + DG_XF_WARPS + DG_EPI_WARPS);
 constexpr int DG_TILE_BYTES = DG_NG * STG_BYTES + DG_NB * B_BYTES + DG_NA * A_BYTES + DG_EPI_WARPS * 4096;
 constexpr int DG_SMEM_BYTES = DG_TILE_BYTES + 1024 + 512;
 
@@ -453,8 +454,8 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < DG_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, 4); }
-    for (int i = 0; i < DG_NB; ++i) { mbar_init(bar_bfull + 8 * i, 4); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < DG_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, DG_XF_WARPS); }
+    for (int i = 0; i < DG_NB; ++i) { mbar_init(bar_bfull + 8 * i, DG_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }
     for (int i = 0; i < DG_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
     mbar_init(bar_tfull, 1);
     mbar_init(bar_tempty, DG_EPI_WARPS);
@@ -473,35 +474,49 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
+    // Two cursors walk the same (tile, k-block) sequence: the fp32 staging loads run one k-block ahead of the dz
+    // loads, so that the load + conversion of the next weight tile overlaps the products of the current one.
     if (lane == 0) {
+      struct Cursor { int tile, kb; DgTile tl; bool done; };
+      auto seek = [&](Cursor& c) {                                    // move to the next valid tile at or after c.tile
+        for (; c.tile < n_tiles; c.tile += gridDim.x) {
+          c.tl = decode_dgrad(t, tile_start, lvl, c.tile);
+          if (c.tl.valid) { c.kb = 0; c.done = false; return; }
+        }
+        c.done = true;
+      };
+      auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += gridDim.x; seek(c); } };
+      Cursor cs{(int)blockIdx.x, 0, DgTile{}, false}, ca{(int)blockIdx.x, 0, DgTile{}, false};
+      seek(cs); seek(ca);
       Ring sg{0, 0}, ar{0, 0};
       int issued_sg = 0, issued_a = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
-        if (!tl.valid) continue;
-        const StageDyn& d = t.dyn[tl.p];
-        const StageDev& sd_ = t.st[tl.p];
-        const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+      auto issue_staging = [&](const Cursor& c) {
+        const StageDyn& d = t.dyn[c.tl.p];
+        const CUtensorMap* lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 21)) { ok = false; return; }
+        const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
         const bool corr = d.use_delta != 0;
-        tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_F32); tma_prefetch_desc(lm + MAP_D_F32);
-        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
-          const int k0 = kb * TILE_K;
-          if (*abort_flag || !mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 21)) { ok = false; break; }
-          const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
-          mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
-          tma_load_2d(sw, lm + MAP_W_F32, fb, tl.n0, k0);
-          if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, tl.n0, k0);
-          sg.advance(DG_NG); ++issued_sg;
-          for (int mi = 0; mi < tl.n_m; ++mi) {
-            if (*abort_flag || !mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 22)) { ok = false; break; }
-            const uint32_t fa = bar_afull + 8 * ar.idx;
-            mbar_arrive_expect_tx(fa, A_BYTES);
-            tma_load_3d(sA + ar.idx * A_BYTES, lm + MAP_DZ_K, fa, k0, tl.m0 + mi * TILE_M, dz_slot);
-            ar.advance(DG_NA); ++issued_a;
-          }
+        mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
+        tma_load_2d(sw, lm + MAP_W_F32, fb, c.tl.n0, c.kb * TILE_K);
+        if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, c.tl.n0, c.kb * TILE_K);
+        sg.advance(DG_NG); ++issued_sg;
+      };
+      if (!cs.done) { issue_staging(cs); step(cs); }
+      while (!ca.done && ok) {
+        if (!cs.done) { issue_staging(cs); step(cs); if (!ok) break; }
+        const StageDyn& d = t.dyn[ca.tl.p];
+        const StageDev& sd_ = t.st[ca.tl.p];
+        const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        for (int mi = 0; mi < ca.tl.n_m; ++mi) {
+          if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 22)) { ok = false; break; }
+          const uint32_t fa = bar_afull + 8 * ar.idx;
+          mbar_arrive_expect_tx(fa, A_BYTES);
+          tma_load_3d(sA + ar.idx * A_BYTES, lm + MAP_DZ_K, fa, ca.kb * TILE_K, ca.tl.m0 + mi * TILE_M, dz_slot);
+          ar.advance(DG_NA); ++issued_a;
         }
+        step(ca);
       }
       if (*abort_flag) {
         for (int back = 1; back <= DG_NG && back <= issued_sg; ++back) {
@@ -520,24 +535,25 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = make_idesc(0, 1);
+      const uint64_t dba = desc_base(16, 1024), dbb = desc_base(B_BYTES / 2, 1024);
       Ring br{0, 0}, ar{0, 0};
       uint32_t tphase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
-        if (*abort_flag || !mbar_wait(bar_tempty, tphase ^ 1, abort_flag, status, 23)) { ok = false; break; }
+        if (!mbar_wait(bar_tempty, tphase ^ 1, abort_flag, status, 23)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
-          if (*abort_flag || !mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 24)) { ok = false; break; }
+          if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 24)) { ok = false; break; }
           const uint32_t sb = sB + br.idx * B_BYTES;
           for (int mi = 0; mi < tl.n_m; ++mi) {
-            if (*abort_flag || !mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 25)) { ok = false; break; }
+            if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 25)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = sA + ar.idx * A_BYTES;
 #pragma unroll
             for (int k16 = 0; k16 < TILE_K / 16; ++k16)
-              tc_mma_bf16(tmem_base + (uint32_t)(mi * ACC_COLS), make_desc(sa + k16 * 32, 16, 1024), make_desc(sb + k16 * 2048, B_BYTES / 2, 1024),
+              tc_mma_bf16(tmem_base + (uint32_t)(mi * ACC_COLS), desc_at(dba, sa + k16 * 32), desc_at(dbb, sb + k16 * 2048),
                           idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
             tc_commit(bar_aempty + 8 * ar.idx);
             ar.advance(DG_NA);
@@ -549,9 +565,10 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
         tphase ^= 1;
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 + DG_XF_WARPS) {
     // ---------------- operand transform: fp32 w, delta in staging -> bf16(w - gap*delta), MN-major ----------------
-    const int tt = threadIdx.x - 64;
+    const int tt = (threadIdx.x - 64) & 127;                          // position within a group of four warps
+    const int hsel = (threadIdx.x - 64) >> 7;                         // which half of the 64 k-rows this group converts
     const int c = tt & 15, rb = tt >> 4;
     const uint32_t dst_in_tile = (uint32_t)(c >> 3) * (B_BYTES / 2) + (uint32_t)rb * 128 + (uint32_t)(((c & 7) ^ rb) << 4);
     const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
@@ -563,14 +580,15 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       const float gapf = (float)t.st[tl.p].gap;
       const bool corr = t.dyn[tl.p].use_delta != 0;
       for (int kb = 0; kb < tl.n_kb; ++kb) {
-        bool go = !*abort_flag && mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 26);
+        bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 26);
         go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 27);
         go = __all_sync(0xffffffffu, go);
         if (!go) { ok = false; break; }
         const uint8_t* src = stg_ptr + sg.idx * STG_BYTES + src_in_tile;
         uint8_t* dst = sB_ptr + br.idx * B_BYTES + dst_in_tile;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int jj = 0; jj < 4; ++jj) {
+          const int j = hsel * 4 + jj;
           const float4 w0 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4);
           const float4 w1 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4 + 16);
           float v[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
@@ -593,7 +611,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
   } else {
     // ---------------- epilogue: one warp per TMEM lane group, 64 columns at a time through a swizzled staging buffer ----------------
     const int q = warp & 3;
-    const int ew = warp - 6;
+    const int ew = warp - 2 - DG_XF_WARPS;
     uint8_t* obuf = sO_ptr + ew * 4096;
     const uint32_t obuf_s = sO + ew * 4096;
     const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
@@ -605,7 +623,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       const StageDyn& d = t.dyn[tl.p];
       const StageDev& s = t.st[tl.p];
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-      bool ready = !*abort_flag && mbar_wait(bar_tfull, tphase, abort_flag, status, 28);
+      bool ready = mbar_wait(bar_tfull, tphase, abort_flag, status, 28);
       ready = __all_sync(0xffffffffu, ready);
       if (!ready) { ok = false; break; }
       tc_fence_after();
