@@ -210,7 +210,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
-  L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes(P) : 0), 256);
+  L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes((int)T, L.st) : 0), 256);
   L.off_attn = w; w = align_up(w + (L.att_tc ? attn_workspace_bytes(P) : 0), 256);
   for (int p = 0; p < P; ++p) {
     StageDev& s = L.st[p];

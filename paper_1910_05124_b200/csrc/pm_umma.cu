@@ -21,6 +21,8 @@
 // issuing work, waits (bounded) for its copies in flight, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "pm_ptx.cuh"
 #include "pm_umma.cuh"
 
@@ -102,7 +104,7 @@ struct Ring {                       // position in a ring of mbarrier-guarded sl
 // ---- the kernel --------------------------------------------------------------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(Cfg<MODE>::kThreads, 1)
-umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, int n_tiles, int lvl, int* status) {
+umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
   using C = Cfg<MODE>;
   constexpr int NS = C::kStages, NG = C::kStaging, NT = C::kTransformWarps;
   extern __shared__ uint8_t smem_raw[];
@@ -145,7 +147,9 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       Ring op{0, 0}, sg{0, 0};
       int issued_op = 0, issued_sg = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
         const StageDyn& d = t.dyn[tl.p];
@@ -212,7 +216,9 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const uint32_t ka = MODE == 2 ? 2048 : 32, kb_ = MODE == 0 ? 32 : 2048;
       Ring op{0, 0}, acc{0, 0};
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
         if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 6)) { ok = false; break; }
@@ -241,7 +247,9 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
       Ring op{0, 0}, sg{0, 0};
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
         const float gapf = (float)t.st[tl.p].gap;
@@ -289,7 +297,9 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     Ring acc{0, 0};
     bool ok = true;
     bool stored = false;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
       const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
       const StageDyn& d = t.dyn[tl.p];
@@ -433,7 +443,7 @@ __device__ __forceinline__ DgTile decode_dgrad(const TickArgs& t, const int* __r
 }
 
 __global__ void __launch_bounds__(DG_THREADS, 1)
-umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, int n_tiles, int lvl, int* status) {
+umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -479,8 +489,10 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     if (lane == 0) {
       struct Cursor { int tile, kb; DgTile tl; bool done; };
       auto seek = [&](Cursor& c) {                                    // move to the next valid tile at or after c.tile
-        for (; c.tile < n_tiles; c.tile += gridDim.x) {
-          c.tl = decode_dgrad(t, tile_start, lvl, c.tile);
+        for (; c.tile < n_slots; c.tile += gridDim.x) {              // c.tile walks the slots of the order array
+          const int tile = order[c.tile];
+          if (tile < 0) continue;
+          c.tl = decode_dgrad(t, tile_start, lvl, tile);
           if (c.tl.valid) { c.kb = 0; c.done = false; return; }
         }
         c.done = true;
@@ -539,7 +551,9 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       Ring br{0, 0}, ar{0, 0};
       uint32_t tphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
         const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
         if (!mbar_wait(bar_tempty, tphase ^ 1, abort_flag, status, 23)) { ok = false; break; }
@@ -574,7 +588,9 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
     Ring br{0, 0}, sg{0, 0};
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
       const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
       const float gapf = (float)t.st[tl.p].gap;
@@ -617,7 +633,9 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
     uint32_t tphase = 0;
     bool ok = true, stored = false;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
       const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
       const StageDyn& d = t.dyn[tl.p];
@@ -680,17 +698,92 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct UmmaPlan {
   const CUtensorMap* d_maps = nullptr;
   const int* d_tile_start = nullptr;     // [3 modes][PM_MAX_LINEARS][P+1]
+  const int* d_orders = nullptr;         // concatenated order arrays
   int* d_status = nullptr;
-  int n_tiles[3][PM_MAX_LINEARS] = {};
-  int P = 0, sms = 148;
+  int n_slots[3][PM_MAX_LINEARS] = {};
+  int grid[3][PM_MAX_LINEARS] = {};
+  size_t order_off[3][PM_MAX_LINEARS] = {};
+  int P = 0;
 };
 
+// Tile tables of every (mode, level): the flattened tile ids per stage, and the order in which the persistent
+// CTAs walk them.  CTA b takes order[b], order[b + G], ...: the lists are a longest-processing-time-first
+// assignment (weight = k-blocks x row tiles + a constant per tile), so that one very deep GEMM (a vocabulary
+// projection next to d_model-sized layers) does not leave most SMs idle.  Unused slots hold -1.
+struct TileTables {
+  std::vector<int> tile_start;           // [3][PM_MAX_LINEARS][P+1]
+  std::vector<int> orders;
+  int n_slots[3][PM_MAX_LINEARS] = {};
+  int grid[3][PM_MAX_LINEARS] = {};
+  size_t order_off[3][PM_MAX_LINEARS] = {};
+};
+
+static int device_sms() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+    cudaGetLastError();
+    return 148;
+  }
+  return sms;
+}
+
+static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int sms) {
+  const int P = (int)st.size();
+  TileTables tt;
+  tt.tile_start.assign((size_t)3 * PM_MAX_LINEARS * (P + 1), 0);
+  auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
+  for (int mode = 0; mode < 3; ++mode)
+    for (int l = 0; l < PM_MAX_LINEARS; ++l) {
+      int* ts = tt.tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
+      std::vector<std::pair<long long, int>> work;          // (weight, tile id)
+      int acc = 0;
+      for (int p = 0; p < P; ++p) {
+        ts[p] = acc;
+        if (l < st[p].n_lin) {
+          const LinDev& L = st[p].lin[l];
+          const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (mode == 1 ? L.n_out : T);
+          const int tm = cdiv(M, TILE_M), tn = cdiv(N, TILE_N), n_kb = cdiv(K, TILE_K);
+          const int groups = mode == 1 ? cdiv(tm, DG_MG) : tm;
+          for (int g = 0; g < groups; ++g) {
+            const int n_m = mode == 1 ? std::min(DG_MG, tm - g * DG_MG) : 1;
+            for (int n = 0; n < tn; ++n) work.push_back({(long long)n_kb * n_m + 3 * n_m, acc + g * tn + n});
+          }
+          acc += groups * tn;
+        }
+      }
+      ts[P] = acc;
+      const int G = std::max(1, std::min(acc, sms));
+      tt.grid[mode][l] = G;
+      tt.order_off[mode][l] = tt.orders.size();
+      if (acc == 0) { tt.n_slots[mode][l] = 0; continue; }
+      std::stable_sort(work.begin(), work.end(), [](const std::pair<long long, int>& a, const std::pair<long long, int>& b) { return a.first > b.first; });
+      std::vector<std::vector<int>> lists(G);
+      std::vector<long long> load(G, 0);
+      for (const auto& w : work) {
+        int best = 0;
+        for (int b = 1; b < G; ++b) if (load[b] < load[best]) best = b;
+        lists[best].push_back(w.second);
+        load[best] += w.first;
+      }
+      size_t max_len = 0;
+      for (const auto& li : lists) max_len = std::max(max_len, li.size());
+      tt.n_slots[mode][l] = (int)(max_len * G);
+      tt.orders.resize(tt.orders.size() + max_len * G, -1);
+      int* ord = tt.orders.data() + tt.order_off[mode][l];
+      for (int b = 0; b < G; ++b)
+        for (size_t k = 0; k < lists[b].size(); ++k) ord[k * G + b] = lists[b][k];
+    }
+  return tt;
+}
+
 static uint64_t maps_bytes(int P) { return (uint64_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR * sizeof(CUtensorMap); }
-static uint64_t tiles_bytes(int P) { return ((uint64_t)3 * PM_MAX_LINEARS * (P + 1) * sizeof(int) + 255) / 256 * 256; }
+static uint64_t ints_bytes(size_t n) { return ((uint64_t)n * sizeof(int) + 255) / 256 * 256; }
 
-uint64_t umma_workspace_bytes(int n_stages) { return 256 + maps_bytes(n_stages) + tiles_bytes(n_stages); }
+uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st) {
+  const TileTables tt = build_tile_tables(T, st, device_sms());
+  return 256 + maps_bytes((int)st.size()) + ints_bytes(tt.tile_start.size()) + ints_bytes(tt.orders.size());
+}
 
-// kind: 0/1 bf16 with 128-byte swizzle, 2 fp32 with 128-byte swizzle, 3 fp32 without swizzle
 static bool encode(EncodeTiledFn fn, CUtensorMap* m, int kind, void* base, int rank, const uint64_t* dims,
                    const uint64_t* strides_bytes, const uint32_t* box, std::string& err) {
   cuuint64_t gd[3]; cuuint64_t gs[2]; cuuint32_t bx[3]; cuuint32_t es[3] = {1, 1, 1};
@@ -713,7 +806,6 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   const int P = t.P;
   std::vector<CUtensorMap> maps((size_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR);
   memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
-  std::vector<int> tile_start((size_t)3 * PM_MAX_LINEARS * (P + 1), 0);
   UmmaPlan* plan = new UmmaPlan();
   plan->P = P;
   const uint64_t T = (uint64_t)t.T;
@@ -783,26 +875,19 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       if (!okm) { delete plan; return PM_ERR_CUDA; }
     }
   }
-  auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
+  const TileTables tt = build_tile_tables(t.T, st, device_sms());
   for (int mode = 0; mode < 3; ++mode)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
-      int* ts = tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
-      int acc = 0;
-      for (int p = 0; p < P; ++p) {
-        ts[p] = acc;
-        if (l < st[p].n_lin) {
-          const LinDev& L = st[p].lin[l];
-          const int M = mode == 2 ? L.n_out : t.T, N = mode == 0 ? L.n_out : L.n_in;
-          const int tm = cdiv(M, TILE_M);
-          acc += (mode == 1 ? cdiv(tm, DG_MG) : tm) * cdiv(N, TILE_N);
-        }
-      }
-      ts[P] = acc;
-      plan->n_tiles[mode][l] = acc;
+      plan->n_slots[mode][l] = tt.n_slots[mode][l];
+      plan->grid[mode][l] = tt.grid[mode][l];
+      plan->order_off[mode][l] = tt.order_off[mode][l];
     }
   char* region = (char*)ws_region;
   cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps_bytes(P), cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(region + 256 + maps_bytes(P), tile_start.data(), tile_start.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
+  char* ts_dev = region + 256 + maps_bytes(P);
+  char* ord_dev = ts_dev + ints_bytes(tt.tile_start.size());
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ts_dev, tt.tile_start.data(), tt.tile_start.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess && !tt.orders.empty()) e = cudaMemcpyAsync(ord_dev, tt.orders.data(), tt.orders.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
@@ -810,12 +895,10 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
   if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
-  int dev = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&plan->sms, cudaDevAttrMultiProcessorCount, dev);
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
-  plan->d_tile_start = (const int*)(region + 256 + maps_bytes(P));
+  plan->d_tile_start = (const int*)ts_dev;
+  plan->d_orders = (const int*)ord_dev;
   *out = plan;
   return PM_OK;
 }
@@ -825,13 +908,14 @@ void umma_plan_destroy(UmmaPlan* plan) { delete plan; }
 int* umma_status_word(UmmaPlan* plan) { return plan ? plan->d_status : nullptr; }
 
 cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
-  const int n_tiles = plan->n_tiles[mode][lvl];
-  if (n_tiles == 0) return cudaSuccess;
-  const int grid = n_tiles < plan->sms ? n_tiles : plan->sms;      // one persistent CTA per SM
+  const int n_slots = plan->n_slots[mode][lvl];
+  if (n_slots == 0) return cudaSuccess;
+  const int grid = plan->grid[mode][lvl];                             // one persistent CTA per SM
   const int* ts = plan->d_tile_start + ((size_t)mode * PM_MAX_LINEARS + lvl) * (plan->P + 1);
-  if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
-  else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
-  else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, n_tiles, lvl, plan->d_status);
+  const int* ord = plan->d_orders + plan->order_off[mode][lvl];
+  if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   return cudaGetLastError();
 }
 

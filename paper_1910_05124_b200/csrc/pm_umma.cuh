@@ -9,8 +9,8 @@ namespace pm {
 struct UmmaPlan;   // tensor maps and launch geometry, built once per context
 
 // Bytes of caller workspace the plan needs (status word + tensor maps).
-uint64_t umma_workspace_bytes(int n_stages);
-// ws_region: device memory of at least umma_workspace_bytes(P), 256-byte aligned.  Synchronises `stream`.
+uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st);
+// ws_region: device memory of at least umma_workspace_bytes(T, stages), 256-byte aligned.  Synchronises `stream`.
 pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region,
                            cudaStream_t stream, std::string& err);
 void umma_plan_destroy(UmmaPlan* plan);
