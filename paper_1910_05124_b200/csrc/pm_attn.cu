@@ -8,7 +8,8 @@
 // Q, K, V, dO arrive by TMA as 128-byte-swizzled [128 rows x 64] tiles; the same tile serves as a K-major
 // operand (rows x d_k) or as an MN-major operand (k-rows x 64) depending on the product.  P and dS are
 // written by the threads as two [128 x 64-key] swizzled tiles, read K-major (P V, dS K) or MN-major (P^T dO,
-// dS^T Q).  Every mbarrier wait is bounded.
+// dS^T Q).  exp is the fast ex2-based intrinsic (relative error ~1e-7, far below the bf16 rounding of P).
+// Every mbarrier wait is bounded.
 #include <string>
 #include <vector>
 
@@ -20,7 +21,7 @@ namespace pm {
 constexpr int AT_S = 128, AT_DK = 64;
 constexpr int AT_TILE = AT_S * AT_DK * 2;          // 16 KB: one [128 x 64] bf16 tile
 constexpr int AT_FWD_SMEM = 3 * AT_TILE + 2 * AT_TILE + 1024 + 128;
-constexpr int AT_BWD_SMEM = 4 * AT_TILE + 4 * AT_TILE + 1024 + 128;
+constexpr int AT_BWD_SMEM = 7 * AT_TILE + 1024 + 128;   // Q, K, dO, V|P0, P1, dS0, dS1: two CTAs fit on one SM
 constexpr int AT_TMEM_COLS = 256;
 
 enum { AMAP_QKV = 0, AMAP_DO = 1, AMAPS_PER_STAGE = 2 };
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
       float e[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        e[j] = (!causal || cc * 32 + j <= r) ? expf(__uint_as_float(v[j]) * scale - mx) : 0.f;
+        e[j] = (!causal || cc * 32 + j <= r) ? __expf(__uint_as_float(v[j]) * scale - mx) : 0.f;
         l += e[j];
       }
 #pragma unroll
@@ -187,11 +188,12 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
   if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
   extern __shared__ uint8_t smem_raw[];
-  const AttnCommon c = attn_setup(smem_raw, 8 * AT_TILE);
+  const AttnCommon c = attn_setup(smem_raw, 7 * AT_TILE);
   const uint32_t tmem_base = *c.tmem_slot;
-  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sV = sK + AT_TILE, sdO = sV + AT_TILE, sP = sdO + AT_TILE, sdS = sP + 2 * AT_TILE;
-  uint8_t* pP = c.sptr + 4 * AT_TILE;
-  uint8_t* pdS = c.sptr + 6 * AT_TILE;
+  // V is dead once dP = dO V^T has completed, so the P tiles take its place (plus one more tile)
+  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sdO = sK + AT_TILE, sV = sdO + AT_TILE, sP = sV, sdS = sP + 2 * AT_TILE;
+  uint8_t* pP = c.sptr + 3 * AT_TILE;
+  uint8_t* pdS = c.sptr + 5 * AT_TILE;
   const CUtensorMap* lm = maps + (size_t)p * AMAPS_PER_STAGE;
   const int r = threadIdx.x;
   const int warp = r >> 5;
@@ -231,7 +233,7 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
       tmem_ld_wait();
 #pragma unroll
       for (int j = 0; j < 32; ++j)
-        if (!causal || cc * 32 + j <= r) l += expf(__uint_as_float(v[j]) * scale - mx);
+        if (!causal || cc * 32 + j <= r) l += __expf(__uint_as_float(v[j]) * scale - mx);
     }
     const float inv = 1.0f / l;
     float D = 0.f;
@@ -243,7 +245,7 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
       tmem_ld_wait();
 #pragma unroll
       for (int j = 0; j < 32; ++j)
-        if (!causal || cc * 32 + j <= r) D += __uint_as_float(g[j]) * (expf(__uint_as_float(v[j]) * scale - mx) * inv);
+        if (!causal || cc * 32 + j <= r) D += __uint_as_float(g[j]) * (__expf(__uint_as_float(v[j]) * scale - mx) * inv);
     }
 #pragma unroll 1
     for (int cc = 0; cc < 4; ++cc) {
@@ -254,7 +256,7 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
       float pr[32], ds[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        pr[j] = (!causal || cc * 32 + j <= r) ? expf(__uint_as_float(v[j]) * scale - mx) * inv : 0.f;
+        pr[j] = (!causal || cc * 32 + j <= r) ? __expf(__uint_as_float(v[j]) * scale - mx) * inv : 0.f;
         ds[j] = pr[j] * (__uint_as_float(g[j]) - D);
       }
 #pragma unroll

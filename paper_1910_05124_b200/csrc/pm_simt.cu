@@ -122,6 +122,7 @@ template <> struct Pair<__nv_bfloat16> {
 };
 
 constexpr int kRowChunk = 256;                        // rows per block: 8 warps x 32 rows
+constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 
 template <typename AT>
 __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
@@ -130,55 +131,58 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
-  const int c0 = blockIdx.x * kActCols;
+  const int c0 = blockIdx.x * kActColsV;
   if (c0 >= L.n_out) return;
   const int chunk = blockIdx.y;
   const int r0 = chunk * kRowChunk, r1 = min(t.T, r0 + kRowChunk);
   if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c = c0 + 2 * lane;
+  const int c = c0 + 8 * lane;
   const uint64_t n = (uint64_t)t.T * L.n_out;
   const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
                  : (s.post == POST_ATTENTION ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
   const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy: nothing is stored
   const AT* z = has_act ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n) : dy;
   AT* dz = ws_ptr<AT>(t, s.dz);
-  const bool pair_ok = (L.n_out & 1) == 0;            // vector path needs even row length for alignment
-  float s0 = 0.f, s1 = 0.f;
+  const bool vec = (L.n_out & 7) == 0;                      // vector path needs 8-element alignment of every row
+  float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   for (int r = r0 + warp; r < r1; r += kActWarps) {
     const uint64_t i = (uint64_t)r * L.n_out + c;
-    if (pair_ok && c + 1 < L.n_out) {
-      float2 g = Pair<AT>::ld(dy + i);
-      float2 v = g;
-      if (has_act) {
-        float2 zz = Pair<AT>::ld(z + i);
-        v = make_float2(round_as<AT>(__fmul_rn(g.x, act_grad(zz.x, L.act))), round_as<AT>(__fmul_rn(g.y, act_grad(zz.y, L.act))));
-        Pair<AT>::st(dz + i, v);
-      }
-      s0 = __fadd_rn(s0, v.x); s1 = __fadd_rn(s1, v.y);
-    } else {
+    if (vec) {
       if (c < L.n_out) {
-        float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i]), act_grad(to_f<AT>(z[i]), L.act))) : to_f<AT>(dy[i]);
-        if (has_act) dz[i] = from_f<AT>(v);
-        s0 = __fadd_rn(s0, v);
+        float g[8];
+        load8<AT>(dy + i, g);
+        if (has_act) {
+          float zz[8];
+          load8<AT>(z + i, zz);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) g[k] = round_as<AT>(__fmul_rn(g[k], act_grad(zz[k], L.act)));
+          store8<AT>(dz + i, g);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) sum[k] = __fadd_rn(sum[k], g[k]);
       }
-      if (c + 1 < L.n_out) {
-        float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i + 1]), act_grad(to_f<AT>(z[i + 1]), L.act))) : to_f<AT>(dy[i + 1]);
-        if (has_act) dz[i + 1] = from_f<AT>(v);
-        s1 = __fadd_rn(s1, v);
-      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (c + k < L.n_out) {
+          float v = has_act ? round_as<AT>(__fmul_rn(to_f<AT>(dy[i + k]), act_grad(to_f<AT>(z[i + k]), L.act))) : to_f<AT>(dy[i + k]);
+          if (has_act) dz[i + k] = from_f<AT>(v);
+          sum[k] = __fadd_rn(sum[k], v);
+        }
     }
   }
-  __shared__ float red[kActWarps][kActCols];
-  red[warp][2 * lane] = s0;
-  red[warp][2 * lane + 1] = s1;
-  __syncthreads();
-  if (threadIdx.x < kActCols && c0 + (int)threadIdx.x < L.n_out) {
-    float sum = 0.f;
+  __shared__ float red[kActWarps][kActColsV];
 #pragma unroll
-    for (int w = 0; w < kActWarps; ++w) sum = __fadd_rn(sum, red[w][threadIdx.x]);
-    if (t.row_chunks == 1) t.a.grad[L.b_off + c0 + threadIdx.x] = sum;
-    else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + c0 + threadIdx.x] = sum;
+  for (int k = 0; k < 8; ++k) red[warp][8 * lane + k] = sum[k];
+  __syncthreads();
+  const int cc = c0 + threadIdx.x;
+  if (cc < L.n_out) {
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < kActWarps; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
+    if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = a;
+    else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc] = a;
   }
 }
 
@@ -200,7 +204,7 @@ __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
 int actbwd_launches(const TickArgs& t) { return t.row_chunks == 1 ? 1 : 2; }
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
-  dim3 grid((t.max_dim + kActCols - 1) / kActCols, t.row_chunks, t.P);
+  dim3 grid((t.max_dim + kActColsV - 1) / kActColsV, t.row_chunks, t.P);
   if (dtype == PM_F32) actbwd_kernel<float><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   cudaError_t e = cudaGetLastError();

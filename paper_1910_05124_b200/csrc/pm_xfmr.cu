@@ -44,27 +44,70 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   AT* u = ring_at<AT>(t, s.u_ring, d.f_slot, n) + (uint64_t)row * dm;
   AT* skip = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT)
                  ? ws_at<AT>(t, t.st[p + 1].skip_in) + (uint64_t)(d.tick & 1) * n + (uint64_t)row * dm : nullptr;
+  const bool vec = (dm & 7) == 0;                            // 8 consecutive columns per lane, 256 per pass
   if (s.pre == PRE_EMBED) {
     const int32_t id = ring_at<int32_t>(t, s.ids_ring, d.f_slot, (uint64_t)t.T)[row];
     const AT* e = table_ptr<AT>(t) + s.tab_off + (uint64_t)id * dm;
     const float* pe = ws_at<float>(t, t.pe_off) + (uint64_t)(row % s.seq_len) * dm;
     const float sc = sqrtf((float)dm);
-    for (int c = lane; c < dm; c += 32) {
-      AT v = from_f<AT>(__fadd_rn(__fmul_rn(to_f<AT>(e[c]), sc), pe[c]));
-      u[c] = v;
-      if (skip) skip[c] = v;
+    if (vec) {
+      for (int c = lane * 8; c < dm; c += 256) {
+        float ev[8], pv[8], o[8];
+        load8<AT>(e + c, ev);
+        load8<float>(pe + c, pv);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = __fadd_rn(__fmul_rn(ev[k], sc), pv[k]);
+        store8<AT>(u + c, o);
+        if (skip) store8<AT>(skip + c, o);
+      }
+    } else {
+      for (int c = lane; c < dm; c += 32) {
+        AT v = from_f<AT>(__fadd_rn(__fmul_rn(to_f<AT>(e[c]), sc), pe[c]));
+        u[c] = v;
+        if (skip) skip[c] = v;
+      }
     }
     return;
   }
   const AT* x = ring_at<AT>(t, s.x_ring, d.f_xslot, n) + (uint64_t)row * dm;
-  float sum = 0.f;
-  for (int c = lane; c < dm; c += 32) sum += to_f<AT>(x[c]);
-  const float mu = warp_sum(sum) / (float)dm;
-  float sq = 0.f;
-  for (int c = lane; c < dm; c += 32) { float v = to_f<AT>(x[c]) - mu; sq += v * v; }
-  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)dm + LN_EPS);
   const float* g = t.a.w + s.g_off;
   const float* b = t.a.w + s.beta_off;
+  float sum = 0.f, sq = 0.f;
+  if (vec) {
+    for (int c = lane * 8; c < dm; c += 256) {
+      float xv[8];
+      load8<AT>(x + c, xv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) sum += xv[k];
+    }
+    const float mu = warp_sum(sum) / (float)dm;
+    for (int c = lane * 8; c < dm; c += 256) {
+      float xv[8];
+      load8<AT>(x + c, xv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { const float v = xv[k] - mu; sq += v * v; }
+    }
+    const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)dm + LN_EPS);
+    for (int c = lane * 8; c < dm; c += 256) {
+      float xv[8], gv[8], bv[8], o[8];
+      load8<AT>(x + c, xv);
+      load8<float>(g + c, gv);
+      load8<float>(b + c, bv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) o[k] = __fadd_rn(__fmul_rn(__fmul_rn(xv[k] - mu, rstd), gv[k]), bv[k]);
+      store8<AT>(u + c, o);
+      if (skip) store8<AT>(skip + c, o);
+    }
+    if (lane == 0) {
+      float* st = ring_at<float>(t, s.stat_ring, d.f_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
+      st[0] = mu; st[1] = rstd;
+    }
+    return;
+  }
+  for (int c = lane; c < dm; c += 32) sum += to_f<AT>(x[c]);
+  const float mu = warp_sum(sum) / (float)dm;
+  for (int c = lane; c < dm; c += 32) { float v = to_f<AT>(x[c]) - mu; sq += v * v; }
+  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)dm + LN_EPS);
   for (int c = lane; c < dm; c += 32) {
     AT v = from_f<AT>(__fadd_rn(__fmul_rn(__fmul_rn(to_f<AT>(x[c]) - mu, rstd), g[c]), b[c]));
     u[c] = v;
@@ -289,7 +332,7 @@ cudaError_t attention_set_smem_limits(int S, int dk, int dtype) {
 // ---- cross-entropy at the last stage -------------------------------------------------------------------------------
 // One block per token: lse = max + log(sum exp(logit - max)); loss_t = lse - logit[target];
 // dlogits = (softmax - onehot) / T in the activation type, written where the last stage reads its incoming
-// gradient.  The last block to finish adds the per-token losses in token order.
+// gradient.  The last block to finish adds the per-token losses in a fixed order.
 template <typename AT>
 __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   const StageDyn& d = t.dyn[t.P - 1];
@@ -303,8 +346,22 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   __shared__ float red[8];
   __shared__ float bc;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool in_regs = V <= 8192 && (V & 7) == 0;            // the whole row fits: 4 x 8 values per thread, one read of the logits
+  float v[4][8];
   float mx = -INFINITY;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, lg[c]);
+  if (in_regs) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = (k * 256 + threadIdx.x) * 8;
+      if (c < V) {
+        load8<float>(lg + c, v[k]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mx = fmaxf(mx, v[k][e]);
+      }
+    }
+  } else {
+    for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, lg[c]);
+  }
   mx = warp_max(mx);
   if (lane == 0) red[warp] = mx;
   __syncthreads();
@@ -312,7 +369,16 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   __syncthreads();
   mx = bc;
   float sum = 0.f;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) sum += expf(lg[c] - mx);
+  if (in_regs) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if ((k * 256 + (int)threadIdx.x) * 8 < V) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { v[k][e] = expf(v[k][e] - mx); sum += v[k][e]; }
+      }
+  } else {
+    for (int c = threadIdx.x; c < V; c += blockDim.x) sum += expf(lg[c] - mx);
+  }
   sum = warp_sum(sum);
   __syncthreads();
   if (lane == 0) red[warp] = sum;
@@ -321,10 +387,27 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   __syncthreads();
   sum = bc;
   const float invT = 1.0f / (float)t.T;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) {
-    float pr = expf(lg[c] - mx) / sum;
-    if (c == tgt) pr -= 1.0f;
-    dl[c] = from_f<AT>(pr * invT);
+  if (in_regs) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = (k * 256 + threadIdx.x) * 8;
+      if (c < V) {
+        float o[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float pr = v[k][e] / sum;
+          if (c + e == tgt) pr -= 1.0f;
+          o[e] = pr * invT;
+        }
+        store8<AT>(dl + c, o);
+      }
+    }
+  } else {
+    for (int c = threadIdx.x; c < V; c += blockDim.x) {
+      float pr = expf(lg[c] - mx) / sum;
+      if (c == tgt) pr -= 1.0f;
+      dl[c] = from_f<AT>(pr * invT);
+    }
   }
   float* rowloss = ws_at<float>(t, t.rowloss_off);
   unsigned int* counter = reinterpret_cast<unsigned int*>(ws_at<float>(t, t.lossred_off) + 64);
@@ -335,12 +418,22 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
     last = atomicAdd(counter, 1u) == gridDim.x - 1;
   }
   __syncthreads();
-  if (last && threadIdx.x == 0) {
+  if (last) {
+    // the last block adds the per-token losses in a fixed order: strided per-thread partials, then a fixed tree
     __threadfence();
+    __shared__ float tree[256];
     float a = 0.f;
-    for (int r = 0; r < t.T; ++r) a += reinterpret_cast<volatile float*>(rowloss)[r];
-    ws_at<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = a / (float)t.T;
-    *counter = 0;
+    for (int r = threadIdx.x; r < t.T; r += 256) a += reinterpret_cast<volatile float*>(rowloss)[r];
+    tree[threadIdx.x] = a;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+      if ((int)threadIdx.x < off) tree[threadIdx.x] += tree[threadIdx.x + off];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      ws_at<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = tree[0] / (float)t.T;
+      *counter = 0;
+    }
   }
 }
 
@@ -381,7 +474,40 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
   const float* dl = t.a.delta + s.g_off;
   const float gapf = (float)s.gap;
   const bool corr = d.use_delta != 0;
+  AT* out = gin_write_prev<AT>(t, p, d) + ro;
   float s1 = 0.f, s2 = 0.f;
+  if ((dm & 7) == 0 && dm <= 2048) {                         // 8 columns per lane per pass, values kept in registers
+    float dxh[8][8], xh[8][8];
+    int np = 0;
+    for (int c = lane * 8; c < dm; c += 256, ++np) {
+      float xv[8], dv[8], gv[8];
+      load8<AT>(x + c, xv);
+      load8<AT>(du + ro + c, dv);
+      load8<float>(g + c, gv);
+      if (gs) { float sv[8]; load8<AT>(gs + ro + c, sv);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) dv[k] = __fadd_rn(dv[k], sv[k]); }
+      if (corr) { float cv[8]; load8<float>(dl + c, cv);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) gv[k] = __fsub_rn(gv[k], __fmul_rn(gapf, cv[k])); }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        xh[np][k] = (xv[k] - mu) * rstd;
+        dxh[np][k] = dv[k] * gv[k];
+        s1 += dxh[np][k]; s2 += dxh[np][k] * xh[np][k];
+      }
+    }
+    s1 = warp_sum(s1) / (float)dm;
+    s2 = warp_sum(s2) / (float)dm;
+    np = 0;
+    for (int c = lane * 8; c < dm; c += 256, ++np) {
+      float o[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) o[k] = rstd * (dxh[np][k] - s1 - xh[np][k] * s2);
+      store8<AT>(out + c, o);
+    }
+    return;
+  }
   for (int c = lane; c < dm; c += 32) {
     float gb = g[c];
     if (corr) gb = __fsub_rn(gb, __fmul_rn(gapf, dl[c]));
@@ -391,7 +517,6 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
   }
   s1 = warp_sum(s1) / (float)dm;
   s2 = warp_sum(s2) / (float)dm;
-  AT* out = gin_write_prev<AT>(t, p, d) + ro;
   for (int c = lane; c < dm; c += 32) {
     float gb = g[c];
     if (corr) gb = __fsub_rn(gb, __fmul_rn(gapf, dl[c]));
@@ -402,8 +527,10 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
 }
 
 // LayerNorm parameter gradients: dgain[c] = sum_rows du_total * xhat, dbias[c] = sum_rows du_total.
-// A block owns 32 columns and 256 rows; warp w takes rows w, w+8, ... ascending; per-warp partials are added in
+// A block owns 256 columns (8 per lane) and 256 rows; warp w takes rows w, w+8, ... ascending; per-warp partials are added in
 // warp order, per-block partials in block order by ln_param_finish_kernel.
+constexpr int kLnCols = 256;                         // columns per block: 8 per lane
+
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
   const int p = blockIdx.z;
@@ -411,41 +538,63 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
   const int dm = s.d_in;
-  const int c = blockIdx.x * 32 + (threadIdx.x & 31);
-  if (blockIdx.x * 32 >= dm) return;
+  const int c0 = blockIdx.x * kLnCols;
+  if (c0 >= dm) return;
   const int chunk = blockIdx.y;
   const int r0 = chunk * 256, r1 = min(t.T, r0 + 256);
   if (r0 >= t.T) return;
-  const int warp = threadIdx.x >> 5;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint64_t n = (uint64_t)t.T * dm;
   const AT* du = ws_at<AT>(t, s.dh);
   const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
   const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n);
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
-  float ag = 0.f, ab = 0.f;
-  if (c < dm)
-    for (int r = r0 + warp; r < r1; r += 8) {
-      const uint64_t i = (uint64_t)r * dm + c;
-      const float v = du_total<AT>(du, gs, i);
-      const float xh = (to_f<AT>(x[i]) - st[2 * r]) * st[2 * r + 1];
-      ag = __fadd_rn(ag, __fmul_rn(v, xh));
-      ab = __fadd_rn(ab, v);
+  const bool vec = (dm & 7) == 0;
+  const int c = c0 + lane * 8;
+  float ag[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, ab[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int r = r0 + warp; r < r1; r += 8) {
+    const float mu = st[2 * r], rstd = st[2 * r + 1];
+    const uint64_t i = (uint64_t)r * dm + c;
+    if (vec) {
+      if (c < dm) {
+        float dv[8], xv[8];
+        load8<AT>(du + i, dv);
+        load8<AT>(x + i, xv);
+        if (gs) { float sv[8]; load8<AT>(gs + i, sv);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) dv[k] = __fadd_rn(dv[k], sv[k]); }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          ag[k] = __fadd_rn(ag[k], __fmul_rn(dv[k], (xv[k] - mu) * rstd));
+          ab[k] = __fadd_rn(ab[k], dv[k]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (c + k < dm) {
+          const float v = du_total<AT>(du, gs, i + k);
+          ag[k] = __fadd_rn(ag[k], __fmul_rn(v, (to_f<AT>(x[i + k]) - mu) * rstd));
+          ab[k] = __fadd_rn(ab[k], v);
+        }
     }
-  __shared__ float rg[8][32], rb[8][32];
-  rg[warp][threadIdx.x & 31] = ag;
-  rb[warp][threadIdx.x & 31] = ab;
+  }
+  __shared__ float rg[8][kLnCols], rb[8][kLnCols];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) { rg[warp][lane * 8 + k] = ag[k]; rb[warp][lane * 8 + k] = ab[k]; }
   __syncthreads();
-  if (threadIdx.x < 32 && c < dm) {
+  const int cc = c0 + threadIdx.x;
+  if (cc < dm) {
     float a = 0.f, b2 = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, rg[w][threadIdx.x]); b2 = __fadd_rn(b2, rb[w][threadIdx.x]); }
     if (t.row_chunks == 1) {
-      t.a.grad[s.g_off + c] = a;
-      t.a.grad[s.beta_off + c] = b2;
+      t.a.grad[s.g_off + cc] = a;
+      t.a.grad[s.beta_off + cc] = b2;
     } else {
       float* part = ws_at<float>(t, t.colred_off) + ((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim);
-      part[c] = a;
-      part[t.max_dim + c] = b2;
+      part[cc] = a;
+      part[t.max_dim + cc] = b2;
     }
   }
 }
@@ -475,20 +624,24 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_EMBED) return;
+  extern __shared__ int32_t sid[];                           // the microbatch's token ids
+  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
+  for (int i = threadIdx.x; i < t.T; i += blockDim.x) sid[i] = ids[i];
+  __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int v = blockIdx.x * 8 + warp;
   if (v >= s.vocab) return;
   const int dm = s.d_in;
-  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
   const AT* du = ws_at<AT>(t, s.dh);
   const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
   float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
   const float sc = sqrtf((float)dm);
+  // which tokens carry this id (ascending): at most a handful; collect them once, then stream the columns
   for (int c0 = 0; c0 < dm; c0 += 32 * 8) {                 // up to 8 columns per lane per pass
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     for (int tb = 0; tb < t.T; tb += 32) {
       const int tok = tb + lane;
-      unsigned hit = __ballot_sync(0xffffffffu, tok < t.T && ids[tok] == v);
+      unsigned hit = __ballot_sync(0xffffffffu, tok < t.T && sid[tok] == v);
       while (hit) {
         const int j = __ffs(hit) - 1;
         hit &= hit - 1;
@@ -513,7 +666,7 @@ int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.row_chunks == 1 
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
   if (t.any_ln) {
-    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + 31) / 32, t.row_chunks, t.P);
+    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + kLnCols - 1) / kLnCols, t.row_chunks, t.P);
     if (dtype == PM_F32) { ln_bwd_dx_kernel<float><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<float><<<g2, 256, 0, stream>>>(t); }
     else { ln_bwd_dx_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(t); }
     e = cudaGetLastError();
@@ -527,8 +680,9 @@ cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   }
   if (t.any_embed) {
     dim3 g((t.max_vocab + 7) / 8, t.P);
-    if (dtype == PM_F32) embed_bwd_kernel<float><<<g, 256, 0, stream>>>(t);
-    else embed_bwd_kernel<__nv_bfloat16><<<g, 256, 0, stream>>>(t);
+    const size_t smem = sizeof(int32_t) * (size_t)t.T;
+    if (dtype == PM_F32) embed_bwd_kernel<float><<<g, 256, smem, stream>>>(t);
+    else embed_bwd_kernel<__nv_bfloat16><<<g, 256, smem, stream>>>(t);
     e = cudaGetLastError();
   }
   return e;
