@@ -121,7 +121,6 @@ template <> struct Pair<__nv_bfloat16> {
   static __device__ __forceinline__ void st(__nv_bfloat16* p, float2 v) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v.x, v.y); }
 };
 
-constexpr int kRowChunk = 256;                        // rows per block: 8 warps x 32 rows
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 
 template <typename AT>
@@ -134,7 +133,7 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   const int c0 = blockIdx.x * kActColsV;
   if (c0 >= L.n_out) return;
   const int chunk = blockIdx.y;
-  const int r0 = chunk * kRowChunk, r1 = min(t.T, r0 + kRowChunk);
+  const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + t.chunk_rows);
   if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = c0 + 8 * lane;

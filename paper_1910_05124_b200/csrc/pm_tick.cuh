@@ -18,7 +18,8 @@ struct TickArgs {
   uint64_t pe_off;        // ws: sinusoidal positions [seq_len][d] float (0 if no embedding stage)
   uint64_t rowloss_off;   // ws: per-token losses [T] float (cross-entropy)
   uint64_t colred_off;    // ws: per-row-chunk partial column sums [P][row_chunks][2*max_dim] float
-  int32_t row_chunks;     // ceil(T / 256)
+  int32_t row_chunks;     // ceil(T / chunk_rows)
+  int32_t chunk_rows;     // rows of a microbatch one block of a column reduction covers (256, or 32 for short microbatches)
   int32_t loss_kind;      // PM_LOSS_*
   int32_t any_pre, any_ln, any_embed, any_residual;   // which grouped launches this pipeline needs
   int32_t att_S, att_dk, att_blocks;                   // attention: sequence length, head width, (sequences x heads); 0 = none

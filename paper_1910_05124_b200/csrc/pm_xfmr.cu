@@ -541,7 +541,7 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
   const int c0 = blockIdx.x * kLnCols;
   if (c0 >= dm) return;
   const int chunk = blockIdx.y;
-  const int r0 = chunk * 256, r1 = min(t.T, r0 + 256);
+  const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + t.chunk_rows);
   if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint64_t n = (uint64_t)t.T * dm;
