@@ -137,6 +137,8 @@ def barrier(world):
 # ---- the CUDA arm ---------------------------------------------------------------------------------
 
 WORKLOADS = {
+    "cfg1": "cfg1: 4-stage MLP, 1 Linear(256,256)+ReLU per stage, fp32 (SIMT GEMMs), microbatch 32, SGD momentum 0.9, "
+            "T1 (K=32) + T2 (D=0.5), tau=(7,5,3,1)",
     "cfg3": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master weights, microbatch 128, "
             "SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
     "cfg4": "cfg4: Transformer encoder, 6 layers, d_model 512, 8 heads, FFN 2048, 32 sequences x 128 tokens per "
@@ -157,6 +159,10 @@ def build_workload(args):
         params0 = I.init_encoder_params(wl)
         n_params = sum(int(a.size) for st in params0 for a in st)
         return wl, params0, wl.microbatch // wl.seq_len, n_params
+    if args.workload == "cfg1":
+        wl = I.cfg1()
+        params0 = I.init_stage_params(wl)
+        return wl, params0, wl.microbatch, sum(sp.n_in * sp.n_out + sp.n_out for st in wl.stages for sp in st)
     wl = I.cfg3()
     if args.stages:          # profiler captures only: fewer stages of the same shape, not a bench result
         wl = I.mlp_workload(wl.name + f"_first{args.stages}", args.stages, 1024, 2, "gelu", wl.microbatch, compute="bf16",
@@ -311,9 +317,38 @@ def gemm_flops(wl):
     return {"gemm_fwd": full, "wgrad": full, "dgrad": dgrad}
 
 
+def gemm_bytes(wl):
+    """Algorithmic HBM bytes of one tick per GEMM class on the bf16 path: every operand read once, every result
+    written once (bf16 activations, fp32 weights / discrepancy / gradient, fp32 logits under cross-entropy)."""
+    T = wl.microbatch
+    if wl.kind == "encoder":
+        lin = [(sp.n_in, sp.n_out, sp.act) for sp in wl.stage_specs]
+        gaps = [f - b for f, b in zip(wl.tau_fwd, wl.tau_bkwd)]
+        logits_f32 = True
+    else:
+        lin = [(sp.n_in, sp.n_out, sp.act) for st in wl.stages for sp in st]
+        gaps = [f - b for st, f, b in zip(wl.stages, wl.tau_fwd, wl.tau_bkwd) for _ in st]
+        logits_f32 = False
+    fwd = wgrad = dgrad = 0.0
+    for j, ((a, b, act), gap) in enumerate(zip(lin, gaps)):
+        last = j == len(lin) - 1
+        out_b = 4 if (last and logits_f32) else 2 * (2 if act != "none" else 1)    # z stash and activation y
+        fwd += 2.0 * T * a + 2.0 * a * b + out_b * T * b
+        wgrad += 2.0 * T * a + 2.0 * T * b + 4.0 * a * b
+        if j > 0 or wl.kind == "encoder":
+            dgrad += 2.0 * T * b + (8.0 if (wl.t2 and gap > 0) else 4.0) * a * b + 2.0 * T * a
+    return {"gemm_fwd": fwd, "wgrad": wgrad, "dgrad": dgrad}
+
+
 # DRAM traffic per launch from ncu captures summarised under profiles/ (bytes); scaled to the benchmark workload by
 # the stated unit counts because the full-size workloads hold more device memory than a multi-pass capture may.
 NCU_TRAFFIC = {
+    # GEMM kernels: measured DRAM bytes / algorithmic bytes on the 2-layer cut of cfg4
+    # (profiles/gemm_and_attention_kernels_cfg4_2layer_cut.md); every operand crosses HBM once, so traffic grows
+    # with the algorithmic bytes of the launch
+    "gemm_fwd_ratio": (84.1 + 183.3) / (83.9 + 243.0),
+    "wgrad_ratio": (211.5 + 24.6) / (205.5 + 42.0),
+    "dgrad_ratio": (232.4 + 45.9) / (226.5 + 33.6),
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
@@ -413,13 +448,26 @@ def rooflines(res, hbm_peak, tf_peak, peak_kind, steps):
     if dominant == "update":
         return update, update
     flops = gemm_flops(wl)
+    if dominant in flops and wl.compute == "f32":
+        # fp32 path: plain FFMA on the CUDA cores; peak derived from unit counts and clocks:
+        # 148 SMs x 128 lanes x 2 flop x 1.965 GHz = 74.4 TFLOP/s
+        tfs = flops[dominant] / (per_tick[dominant] * 1e-3) / 1e12
+        dom = {"kernel": "simt_gemm_kernel (" + dominant + ")", "bound": "alu", "achieved": round(tfs, 3), "peak": 74.4,
+               "unit": "TFLOP/s", "frac": round(tfs / 74.4, 5), "of": "derived (148 SMs x 128 FFMA lanes x 1.965 GHz)",
+               "traffic": None, "avg_ms_per_step": round(per_tick[dominant], 5),
+               "share_of_step": round(per_tick[dominant] / res["total_prof"], 4),
+               "note": "46 MFLOP per step: launch-latency bound, not arithmetic bound"}
+        return dom, update
     if dominant in flops:
         launches = res["prof"][dominant][1] / steps
         tfs = flops[dominant] / (per_tick[dominant] * 1e-3) / 1e12
         names = {"gemm_fwd": "umma_gemm_kernel<0> (forward GEMMs)", "wgrad": "umma_gemm_kernel<2> (wgrad GEMMs)",
                  "dgrad": "umma_dgrad_kernel (dgrad GEMMs, weights corrected while loading)"}
         dom = {"kernel": names[dominant], "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
-               "frac": round(tfs / tf_peak, 4), "of": peak_kind + " (sustained bf16 matmul)", "traffic": None,
+               "frac": round(tfs / tf_peak, 4), "of": peak_kind + " (sustained bf16 matmul)",
+               "traffic": int(NCU_TRAFFIC[dominant + "_ratio"] * gemm_bytes(wl)[dominant] / launches),
+               "traffic_note": "DRAM bytes per launch, scaled from the ncu capture of the 2-layer cut by algorithmic bytes",
+               "algorithmic_bytes_per_step": gemm_bytes(wl)[dominant],
                "algorithmic_flops_per_step": flops[dominant], "launches_per_step": launches,
                "avg_ms_per_step": round(per_tick[dominant], 5), "frac_of_nominal_2250TFs": round(tfs / 2250.0, 4),
                "share_of_step": round(per_tick[dominant] / res["total_prof"], 4)}
@@ -439,10 +487,11 @@ def run_cuda(args):
     if sampler is not None:
         sampler.start()
     res = measure(args, args.workload, world, rank, local, device, sampler)
-    other = None
+    others = []
     if world == 1 and not args.no_other and not args.stages:
-        other_name = "cfg3" if args.workload == "cfg4" else "cfg4"
-        other = measure(args, other_name, world, rank, local, device, None, with_e2e=False)
+        for name in ("cfg4", "cfg3", "cfg1"):
+            if name != args.workload:
+                others.append((name, measure(args, name, world, rank, local, device, None, with_e2e=False)))
     if rank != 0:
         return
     wl, P = res["wl"], res["P"]
@@ -453,7 +502,7 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(res["t_ms"] / args.steps, 5), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if wl.compute == "f32" else "bf16", "data": "synthetic",
         "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
                    "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
                    "samples_per_step": res["samples_per_step"], "pipeline_fill_ticks": res["fill"],
@@ -470,12 +519,13 @@ def run_cuda(args):
                      "ms_per_step": round(gemm_ms, 5)},
         "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(res["per_tick_ms"].items(), key=lambda kv: -kv[1])},
     }
-    if other is not None:
+    line["other_workloads"] = []
+    for name, other in others:
         od, ou = rooflines(other, hbm_peak, tf_peak, peak_kind, args.steps)
-        line["other_workload"] = {"workload": WORKLOADS["cfg3" if args.workload == "cfg4" else "cfg4"],
-                                  "value": round(other["units"] / (other["t_ms"] * 1e-3), 2), "unit": UNIT,
-                                  "ms_per_step": round(other["t_ms"] / args.steps, 5), "roofline": od, "roofline_update": ou,
-                                  "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(other["per_tick_ms"].items(), key=lambda kv: -kv[1])}}
+        line["other_workloads"].append({
+            "workload": WORKLOADS[name], "value": round(other["units"] / (other["t_ms"] * 1e-3), 2), "unit": UNIT,
+            "ms_per_step": round(other["t_ms"] / args.steps, 5), "roofline": od, "roofline_update": ou,
+            "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(other["per_tick_ms"].items(), key=lambda kv: -kv[1])}})
     if world == 1:
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, res["samples_per_step"])
