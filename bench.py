@@ -1,14 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the PipeMare hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg3]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg3|cfg1]
 
 A step is one pipeline tick in steady state: every stage runs one forward with the weights it holds, one
 backward against the discrepancy-corrected weights for the microbatch that entered it tau_i updates ago, and
 the fused PipeMare update; one microbatch leaves the pipeline per tick.  The default workload is the largest
 one built: the 6-layer Transformer encoder (config 4; 25 stages; a sample is one sequence of 128 tokens, 32 per
 tick), which exercises every kind of stage.  The 32-stage bf16 MLP (config 3; a sample is one row, 128 per
-tick) is measured briefly in the same run and reported under `other_workload`.
+tick) and the 4-stage fp32 MLP (config 1) are measured in the same run and reported under `other_workloads`.
 
 `roofline` describes the kernel class with the largest share of the step, timed live with CUDA events on
 the launch stream; `roofline_update` is the fused PipeMare update against the HBM peak (the second half of the

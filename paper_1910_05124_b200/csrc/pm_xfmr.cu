@@ -137,7 +137,17 @@ __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
   const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)((d.tick + 1) & 1) * n;     // written by the previous stage last tick
   const AT* y = ws_at<AT>(t, s.ytmp);
   AT* out = ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
+  // buffers start on 256-byte boundaries and slots are n elements apart: groups of eight are aligned when 8 | n
+  const uint64_t n8 = (n % 8 == 0) ? n / 8 : 0;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
+    float a[8], b[8];
+    load8<AT>(skip + 8 * i, a);
+    load8<AT>(y + 8 * i, b);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) a[j] = __fadd_rn(a[j], b[j]);
+    store8<AT>(out + 8 * i, a);
+  }
+  for (uint64_t i = 8 * n8 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
     out[i] = from_f<AT>(__fadd_rn(to_f<AT>(skip[i]), to_f<AT>(y[i])));
 }
 
