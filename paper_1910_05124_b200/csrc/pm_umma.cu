@@ -37,14 +37,12 @@ constexpr int STG_BYTES = 2 * STG_HALF_BYTES;              // w tile + delta til
 constexpr int ACC_COLS = 128, TMEM_COLS = 2 * ACC_COLS;
 constexpr int N_EPI_WARPS = 8;
 
-template <int MODE> struct Cfg {
-  static constexpr int kTransformWarps = MODE == 1 ? 4 : 0;
-  static constexpr int kStages = MODE == 1 ? 2 : 4;        // operand ring depth
-  static constexpr int kStaging = MODE == 1 ? 2 : 0;       // fp32 staging ring depth (dgrad only)
-  static constexpr int kThreads = 32 * (2 + kTransformWarps + N_EPI_WARPS);
-  static constexpr int kOutWarpBytes = MODE == 1 ? 4096 : 8192;   // per epilogue warp: 32 rows x 128 B per output box
+template <int MODE> struct Cfg {                           // MODE 0 forward, 2 wgrad (dgrad has its own kernel)
+  static constexpr int kStages = 4;                        // operand ring depth
+  static constexpr int kThreads = 32 * (2 + N_EPI_WARPS);
+  static constexpr int kOutWarpBytes = 8192;               // per epilogue warp: two boxes of 32 rows x 128 B
   static constexpr int kOutBytes = N_EPI_WARPS * kOutWarpBytes;
-  static constexpr int kTileBytes = kStages * STAGE_BYTES + kStaging * STG_BYTES + kOutBytes;
+  static constexpr int kTileBytes = kStages * STAGE_BYTES + kOutBytes;
   static constexpr int kSmemBytes = kTileBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
@@ -71,6 +69,72 @@ __device__ __forceinline__ void epi_zy8(const float (&pf)[8], uint8_t* zdst, uin
   *reinterpret_cast<uint4*>(ydst) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
 }
 
+// One epilogue block of the forward (MODE 0) or wgrad (MODE 2) GEMM: 32 rows x 64 accumulator columns held in
+// r0, r1 go through this warp's swizzled staging buffer to one or two TMA stores (full 128-byte rows; rows and
+// columns beyond the tensor are clipped).  Called by a whole warp; lane = row within the block.
+template <int MODE>
+__device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* lm, const StageDev& s, const StageDyn& d, const LinDev& L,
+                                          int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
+                                          uint8_t* obuf, uint32_t obuf_s, int lane) {
+  const uint32_t row_off = (uint32_t)lane * 128;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  if (MODE == 0) {
+    const float* bias = t.a.w + L.b_off;
+    const bool f32out = (L.flags & LF_OUT_F32) != 0;
+    const int act = L.act;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const int n = nb + g * 8;
+      float bb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (n < N) {
+        const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
+        bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
+      }
+      float pf[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) pf[e] = __fadd_rn(__uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]), bb[e]);
+      if (f32out) {
+        // fp32 logits: two 32-column boxes per warp, eight 16-byte chunks per row each
+        uint8_t* box = obuf + (g >> 2) * 4096;
+        *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2) ^ sw) << 4)) = make_float4(pf[0], pf[1], pf[2], pf[3]);
+        *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
+      } else {
+        const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
+        if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
+        else if (act == PM_ACT_RELU) epi_zy8<PM_ACT_RELU>(pf, obuf + off, obuf + 4096 + off);
+        else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {                                 // two boxes of 32 fp32 columns
+      *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r0[g * 4], r0[g * 4 + 1], r0[g * 4 + 2], r0[g * 4 + 3]);
+      *reinterpret_cast<uint4*>(obuf + 4096 + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r1[g * 4], r1[g * 4 + 1], r1[g * 4 + 2], r1[g * 4 + 3]);
+    }
+  }
+  fence_async_smem();                                             // staging writes -> visible to the TMA engine
+  __syncwarp();
+  if (lane == 0) {
+    if (MODE == 0) {
+      if (L.flags & LF_OUT_F32) {
+        tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
+        if (nb + 32 < N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
+      } else {
+        if (L.flags & LF_WRITE_Z) tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
+        if (L.flags & LF_WRITE_Y) {
+          const int yslot = lvl < s.n_lin - 1 ? d.f_slot
+                            : (s.post == POST_RESIDUAL ? 0 : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
+          tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
+        }
+      }
+    } else {
+      tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
+      if (nb + 32 < N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
+    }
+    tma_store_commit();
+  }
+}
+
 // ---- tile walk ---------------------------------------------------------------------------------------
 // tile_start[p] .. tile_start[p+1] are the flattened tile ids of stage p for this (mode, level).
 struct Tile { int p, m0, n0, M, N, K, n_kb; bool valid; };
@@ -83,10 +147,9 @@ __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __rest
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
-  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0);
   const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
-  else if (MODE == 1) { r.M = t.T; r.N = L.n_in; r.K = L.n_out; }
   else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
   const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
   const int local = tile - tile_start[lo];
@@ -106,27 +169,23 @@ template <int MODE>
 __global__ void __launch_bounds__(Cfg<MODE>::kThreads, 1)
 umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
   using C = Cfg<MODE>;
-  constexpr int NS = C::kStages, NG = C::kStaging, NT = C::kTransformWarps;
+  constexpr int NS = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
   uint8_t* tiles_ptr = smem_raw + (tiles - raw);
-  const uint32_t stg = tiles + NS * STAGE_BYTES;                      // fp32 staging ring (dgrad)
-  uint8_t* stg_ptr = tiles_ptr + NS * STAGE_BYTES;
-  const uint32_t outs = stg + NG * STG_BYTES;                         // epilogue staging for TMA stores
-  uint8_t* outs_ptr = stg_ptr + NG * STG_BYTES;
+  const uint32_t outs = tiles + NS * STAGE_BYTES;                     // epilogue staging for TMA stores
+  uint8_t* outs_ptr = tiles_ptr + NS * STAGE_BYTES;
   const uint32_t bars = tiles + C::kTileBytes;
-  // barrier block: full[NS] empty[NS] sfull[NG] sempty[NG] tfull[2] tempty[2], then tmem base word and abort flag
-  const uint32_t bar_full = bars, bar_empty = bar_full + 8 * NS, bar_sfull = bar_empty + 8 * NS,
-                 bar_sempty = bar_sfull + 8 * NG, bar_tfull = bar_sempty + 8 * NG, bar_tempty = bar_tfull + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + C::kTileBytes + 8 * (2 * NS + 2 * NG + 4));
+  // barrier block: full[NS] empty[NS] tfull[2] tempty[2], then tmem base word and abort flag
+  const uint32_t bar_full = bars, bar_empty = bar_full + 8 * NS, bar_tfull = bar_empty + 8 * NS, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + C::kTileBytes + 8 * (2 * NS + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, MODE == 1 ? 1 + NT : 1); mbar_init(bar_empty + 8 * i, 1); }
-    for (int i = 0; i < NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, NT); }
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, N_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -144,8 +203,8 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      Ring op{0, 0}, sg{0, 0};
-      int issued_op = 0, issued_sg = 0;
+      Ring op{0, 0};
+      int issued_op = 0;
       bool ok = true;
       for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
         const int tile = order[slot];
@@ -159,28 +218,15 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         const StageDev& sd_ = t.st[tl.p];
         const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
-        else if (MODE == 1) { tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_F32); tma_prefetch_desc(lm + MAP_D_F32); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         for (int kb = 0; kb < tl.n_kb; ++kb) {
           const int k0 = kb * TILE_K;
-          if (MODE == 1) {
-            if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 5)) { ok = false; break; }
-            const uint32_t sw = stg + sg.idx * STG_BYTES, fb = bar_sfull + 8 * sg.idx;
-            const bool corr = d.use_delta != 0;
-            mbar_arrive_expect_tx(fb, corr ? STG_BYTES : STG_HALF_BYTES);
-            tma_load_2d(sw, lm + MAP_W_F32, fb, tl.n0, k0);
-            if (corr) tma_load_2d(sw + STG_HALF_BYTES, lm + MAP_D_F32, fb, tl.n0, k0);
-            sg.advance(NG); ++issued_sg;
-          }
           if (!mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 1)) { ok = false; break; }
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES, fb = bar_full + 8 * op.idx;
           if (MODE == 0) {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.f_xslot : d.f_slot);
             tma_load_2d(sb, lm + MAP_W_K, fb, k0, tl.n0);
-          } else if (MODE == 1) {
-            mbar_arrive_expect_tx(fb, A_BYTES);
-            tma_load_3d(sa, lm + MAP_DZ_K, fb, k0, tl.m0, dz_slot);
           } else {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             const int slot = (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.b_xslot : d.b_slot;
@@ -198,11 +244,6 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
           const int it = issued_op - back;
           const long long t0 = clock64();
           while (!mbar_try_wait(bar_full + 8 * (it % NS), (uint32_t)(it / NS) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
-        }
-        for (int back = 1; back <= NG && back <= issued_sg; ++back) {
-          const int it = issued_sg - back;
-          const long long t0 = clock64();
-          while (!mbar_try_wait(bar_sfull + 8 * (it % (NG > 0 ? NG : 1)), (uint32_t)(it / (NG > 0 ? NG : 1)) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
       }
     }
@@ -238,57 +279,12 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         acc.advance(2);
       }
     }
-  } else if (warp < 2 + NT) {
-    // ---------------- operand transform (dgrad): fp32 w, delta in staging -> bf16(w - gap*delta), MN-major ----------------
-    if (MODE == 1) {
-      const int tt = threadIdx.x - 64;                                // 0..127
-      const int c = tt & 15, rb = tt >> 4;                            // 8-column chunk and row within each 8-row group
-      const uint32_t dst_in_tile = (uint32_t)(c >> 3) * (B_BYTES / 2) + (uint32_t)rb * 128 + (uint32_t)(((c & 7) ^ rb) << 4);
-      const uint32_t src_in_tile = (uint32_t)rb * (TILE_N * 4) + (uint32_t)c * 32;
-      Ring op{0, 0}, sg{0, 0};
-      bool ok = true;
-      for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-        const int tile = order[slot];
-        if (tile < 0) continue;
-        const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
-        if (!tl.valid) continue;
-        const float gapf = (float)t.st[tl.p].gap;
-        const bool corr = t.dyn[tl.p].use_delta != 0;
-        for (int kb = 0; kb < tl.n_kb; ++kb) {
-          bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 7);
-          go = go && mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 3);
-          go = __all_sync(0xffffffffu, go);                           // leave the loops as a whole warp
-          if (!go) { ok = false; break; }
-          const uint8_t* src = stg_ptr + sg.idx * STG_BYTES + src_in_tile;
-          uint8_t* dst = tiles_ptr + op.idx * STAGE_BYTES + A_BYTES + dst_in_tile;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float4 w0 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4);
-            const float4 w1 = *reinterpret_cast<const float4*>(src + j * 8 * TILE_N * 4 + 16);
-            float v[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-            if (corr) {
-              const float4 d0 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4);
-              const float4 d1 = *reinterpret_cast<const float4*>(src + STG_HALF_BYTES + j * 8 * TILE_N * 4 + 16);
-              const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-#pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = __fsub_rn(v[e], __fmul_rn(gapf, dd[e]));   // w - (tau_fwd - tau_bkwd) * delta
-            }
-            *reinterpret_cast<uint4*>(dst + j * 1024) =
-                make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-          }
-          fence_async_smem();                                         // generic-proxy stores -> visible to the tensor core
-          __syncwarp();
-          if (lane == 0) { mbar_arrive(bar_full + 8 * op.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
-          op.advance(NS); sg.advance(NG > 0 ? NG : 1);
-        }
-      }
-    }
   } else {
     // ---------------- epilogue: 8 warps, warp%4 = TMEM lane group, two warps per group split the columns ----------------
     // Each warp drains a 32-row x 64-column block, writes it into its own swizzled staging buffer and lets
     // the TMA engine store it (full 128-byte rows; rows and columns beyond the tensor are clipped).
     const int q = warp & 3;
-    const int ew = warp - 2 - NT;                                     // 0..7
+    const int ew = warp - 2;                                          // 0..7
     const int half = ew >> 2;                                         // 0: columns 0..63, 1: columns 64..127
     uint8_t* obuf = outs_ptr + ew * C::kOutWarpBytes;
     const uint32_t obuf_s = outs + ew * C::kOutWarpBytes;
@@ -326,72 +322,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       __syncwarp();
       acc.advance(2);
       if (mrow >= tl.M || nb >= tl.N) continue;                       // nothing of this block is inside the tensor
-      if (MODE == 0) {
-        const float* bias = t.a.w + L.b_off;
-        const bool f32out = (L.flags & LF_OUT_F32) != 0;
-        const int act = L.act;
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const int n = nb + g * 8;
-          float bb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          if (n < tl.N) {
-            const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
-            bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
-          }
-          float pf[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) pf[e] = __fadd_rn(__uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]), bb[e]);
-          if (f32out) {
-            // fp32 logits: two 32-column boxes per warp, eight 16-byte chunks per row each
-            uint8_t* box = obuf + (g >> 2) * 4096;
-            *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2) ^ sw) << 4)) = make_float4(pf[0], pf[1], pf[2], pf[3]);
-            *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
-          } else {
-            const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
-            if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
-            else if (act == PM_ACT_RELU) epi_zy8<PM_ACT_RELU>(pf, obuf + off, obuf + 4096 + off);
-            else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);
-          }
-        }
-      } else if (MODE == 1) {
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          float f[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
-          *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
-              make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-        }
-      } else {
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {                                 // two boxes of 32 fp32 columns
-          *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r0[g * 4], r0[g * 4 + 1], r0[g * 4 + 2], r0[g * 4 + 3]);
-          *reinterpret_cast<uint4*>(obuf + 4096 + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r1[g * 4], r1[g * 4 + 1], r1[g * 4 + 2], r1[g * 4 + 3]);
-        }
-      }
-      fence_async_smem();                                             // staging writes -> visible to the TMA engine
-      __syncwarp();
-      if (lane == 0) {
-        if (MODE == 0) {
-          if (L.flags & LF_OUT_F32) {
-            tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
-            if (nb + 32 < tl.N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
-          } else {
-            if (L.flags & LF_WRITE_Z) tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
-            if (L.flags & LF_WRITE_Y) {
-              const int yslot = lvl < s.n_lin - 1 ? d.f_slot
-                                : (s.post == POST_RESIDUAL ? 0 : (tl.p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
-              tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
-            }
-          }
-        } else if (MODE == 1) {
-          tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0);
-        } else {
-          tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
-          if (nb + 32 < tl.N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
-        }
-        tma_store_commit();
-      }
+      epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane);
       stored = true;
     }
     if (lane == 0 && stored) tma_store_wait_all();                    // global writes complete before the CTA retires
@@ -402,6 +333,217 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---- CTA-pair GEMM: 256 x 256 output tiles ---------------------------------------------------------------
+// The same forward / wgrad products on tiles of 256 x 256 computed by two CTAs of a cluster with one
+// tcgen05.mma.cta_group::2 per 16 k-columns.  Each CTA loads its 128 rows of A and its 128 of the 256
+// columns of B, so a CTA ingests 32 KB per 128x256x64 product: half the shared-memory fill per FLOP of the
+// single-CTA kernel, whose tensor pipe waits on that fill.  Roles per CTA: warp 0 = TMA producer (loads
+// land in its own shared memory and are counted on the leader's `full` barrier), warp 1 = TMEM owner and,
+// in the leader (cluster rank 0), MMA issuer; eight epilogue warps drain the CTA's own 128 accumulator
+// rows (two warps per lane group, 128 columns each, in two blocks of 64).  tcgen05.commit arrives on the
+// `empty` / `tfull` barriers of both CTAs; the epilogue warps of both arrive on the leader's `tempty`.
+// Used when every GEMM of the launch has at least 256 rows and columns; smaller shapes keep the kernel above.
+constexpr int P2_TILE = 256;
+constexpr int P2_STAGES = 5;
+constexpr int P2_ACC_COLS = 256;                                      // two accumulators fill the 512 TMEM columns
+constexpr int P2_THREADS = 32 * (2 + N_EPI_WARPS);
+constexpr int P2_TILE_BYTES = P2_STAGES * STAGE_BYTES + N_EPI_WARPS * 8192;
+constexpr int P2_SMEM_BYTES = P2_TILE_BYTES + 1024 + 512;
+
+template <int MODE>
+__device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
+  Tile r;
+  int lo = 0, hi = t.P - 1;
+  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  r.p = lo;
+  const StageDyn& d = t.dyn[lo];
+  const StageDev& s = t.st[lo];
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0);
+  const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
+  if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
+  else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
+  const int tiles_n = (r.N + P2_TILE - 1) / P2_TILE;
+  const int local = tile - tile_start[lo];
+  r.m0 = (local / tiles_n) * P2_TILE;
+  r.n0 = (local % tiles_n) * P2_TILE;
+  r.n_kb = (r.K + TILE_K - 1) / TILE_K;
+  return r;
+}
+
+template <int MODE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P2_THREADS, 1)
+umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
+  constexpr int NS = P2_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                      // same offset in both CTAs of the pair
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  const uint32_t outs = tiles + NS * STAGE_BYTES;
+  uint8_t* outs_ptr = tiles_ptr + NS * STAGE_BYTES;
+  const uint32_t bars = tiles + P2_TILE_BYTES;
+  // barrier block: full[NS] (used in the leader) empty[NS] tfull[2] tempty[2] (leader), tmem base word, abort flag
+  const uint32_t bar_full = bars, bar_empty = bar_full + 8 * NS, bar_tfull = bar_empty + 8 * NS, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tiles_ptr + P2_TILE_BYTES + 8 * (2 * NS + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();                            // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 2 * N_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc_pair(smem_u32(tmem_slot), 2 * P2_ACC_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();                                                 // barriers of both CTAs are initialised
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    if (lane == 0) {
+      Ring op{0, 0};
+      int issued_op = 0;
+      bool ok = true;
+      for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
+        const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        const StageDyn& d = t.dyn[tl.p];
+        const StageDev& sd_ = t.st[tl.p];
+        const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
+        else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
+        const int ma = tl.m0 + rank * TILE_M, nbh = tl.n0 + rank * TILE_N;   // this CTA's rows of A and of B
+        for (int kb = 0; kb < tl.n_kb; ++kb) {
+          const int k0 = kb * TILE_K;
+          if (!mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 31)) { ok = false; break; }
+          const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
+          if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * op.idx, 2 * (A_BYTES + B_BYTES));   // the bytes of both CTAs
+          const uint32_t fb = mapa_shared(bar_full + 8 * op.idx, 0);
+          if (MODE == 0) {
+            tma_load_3d_pair(sa, lm + MAP_ACT_K, fb, k0, ma, (lvl == 0 && sd_.pre == PRE_NONE) ? d.f_xslot : d.f_slot);
+            tma_load_2d_pair(sb, lm + MAP_W_K, fb, k0, nbh);
+          } else {
+            const int xslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.b_xslot : d.b_slot;
+            tma_load_3d_pair(sa, lm + MAP_DZ_MN, fb, ma, k0, dz_slot);
+            tma_load_3d_pair(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, ma + 64, k0, dz_slot);
+            tma_load_3d_pair(sb, lm + MAP_ACT_MN, fb, nbh, k0, xslot);
+            tma_load_3d_pair(sb + B_BYTES / 2, lm + MAP_ACT_MN, fb, nbh + 64, k0, xslot);
+          }
+          op.advance(NS); ++issued_op;
+        }
+      }
+      if (*abort_flag) {
+        // copies already issued still land in this CTA's shared memory: give them time (bounded) before leaving
+        if (rank == 0) {
+          for (int back = 1; back <= NS && back <= issued_op; ++back) {
+            const int it = issued_op - back;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_full + 8 * (it % NS), (uint32_t)(it / NS) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+          }
+        } else {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc_mn(P2_TILE, P2_TILE, MODE == 2, MODE != 0);
+      const uint64_t dba = MODE == 2 ? desc_base(A_BYTES / 2, 1024) : desc_base(16, 1024);
+      const uint64_t dbb = MODE == 0 ? desc_base(16, 1024) : desc_base(B_BYTES / 2, 1024);
+      const uint32_t ka = MODE == 2 ? 2048 : 32, kb_ = MODE == 0 ? 32 : 2048;
+      Ring op{0, 0}, acc{0, 0};
+      bool ok = true;
+      for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
+        const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 36)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * P2_ACC_COLS);
+        for (int kb = 0; kb < tl.n_kb; ++kb) {
+          if (!mbar_wait(bar_full + 8 * op.idx, op.phase, abort_flag, status, 32)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+            tc_mma_bf16_pair(tmem_acc, desc_at(dba, sa + k16 * ka), desc_at(dbb, sb + k16 * kb_), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          tc_commit_pair(bar_empty + 8 * op.idx, 3);                  // frees the operand slot in both CTAs
+          op.advance(NS);
+        }
+        if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);           // accumulator complete, both CTAs
+        acc.advance(2);
+      }
+    }
+  } else {
+    // ---------------- epilogue: 8 warps per CTA, warp%4 = TMEM lane group, two warps per group split the 256 columns ----------------
+    const int q = warp & 3;
+    const int ew = warp - 2;                                          // 0..7
+    const int half = ew >> 2;                                         // 0: columns 0..127, 1: columns 128..255
+    uint8_t* obuf = outs_ptr + ew * 8192;
+    const uint32_t obuf_s = outs + ew * 8192;
+    Ring acc{0, 0};
+    bool ok = true;
+    bool stored = false;
+    for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
+      const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const StageDyn& d = t.dyn[tl.p];
+      const StageDev& s = t.st[tl.p];
+      const LinDev& L = s.lin[lvl];
+      const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+      const int mrow = tl.m0 + rank * TILE_M + q * 32;                // first row of this warp's blocks
+      bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 34);
+      ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
+      if (!ready) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < 2; ++c) {
+        const int nb = tl.n0 + half * 128 + c * 64;
+        uint32_t r0[32], r1[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * P2_ACC_COLS + half * 128 + c * 64);
+        tmem_ld32(taddr, r0);
+        tmem_ld32(taddr + 32, r1);
+        tmem_ld_wait();
+        if (c == 1) tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (c == 1) mbar_arrive_cluster(mapa_shared(bar_tempty + 8 * acc.idx, 0));   // this warp has read its part of the accumulator
+          if (stored) tma_store_wait_read();                          // previous stores have finished reading the staging buffer
+        }
+        __syncwarp();
+        if (mrow >= tl.M || nb >= tl.N) continue;                     // nothing of this block is inside the tensor
+        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane);
+        stored = true;
+      }
+      acc.advance(2);
+    }
+    if (lane == 0 && stored) tma_store_wait_all();                    // global writes complete before the CTA retires
+  }
+  tc_fence_before();
+  cluster_sync_all();                                                 // no barrier or shared memory of a CTA is touched after this
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 2 * P2_ACC_COLS);
   }
 }
 
@@ -702,6 +844,7 @@ struct UmmaPlan {
   int* d_status = nullptr;
   int n_slots[3][PM_MAX_LINEARS] = {};
   int grid[3][PM_MAX_LINEARS] = {};
+  bool pair[3][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
   size_t order_off[3][PM_MAX_LINEARS] = {};
   int P = 0;
 };
@@ -715,6 +858,7 @@ struct TileTables {
   std::vector<int> orders;
   int n_slots[3][PM_MAX_LINEARS] = {};
   int grid[3][PM_MAX_LINEARS] = {};
+  bool pair[3][PM_MAX_LINEARS] = {};
   size_t order_off[3][PM_MAX_LINEARS] = {};
 };
 
@@ -727,8 +871,15 @@ static int device_sms() {
   return sms;
 }
 
+// PM_UMMA_PAIR=0 in the environment keeps every launch on the single-CTA kernels (for comparisons).
+static bool pair_kernels_allowed() {
+  const char* v = getenv("PM_UMMA_PAIR");
+  return !(v && v[0] == '0');
+}
+
 static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int sms) {
   const int P = (int)st.size();
+  const bool allow_pair = pair_kernels_allowed();
   TileTables tt;
   tt.tile_start.assign((size_t)3 * PM_MAX_LINEARS * (P + 1), 0);
   auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
@@ -736,13 +887,25 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       int* ts = tt.tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
       std::vector<std::pair<long long, int>> work;          // (weight, tile id)
+      // forward and wgrad launches whose GEMMs all have at least 256 rows and columns run on CTA pairs
+      bool pair = allow_pair && mode != 1 && sms >= 2;
+      int n_lin_here = 0;
+      for (int p = 0; p < P && pair; ++p)
+        if (l < st[p].n_lin) {
+          const LinDev& L = st[p].lin[l];
+          ++n_lin_here;
+          if ((mode == 2 ? L.n_out : T) < P2_TILE || (mode == 0 ? L.n_out : L.n_in) < P2_TILE) pair = false;
+        }
+      pair = pair && n_lin_here > 0;
+      tt.pair[mode][l] = pair;
+      const int tile_m = pair ? P2_TILE : TILE_M, tile_n = pair ? P2_TILE : TILE_N;
       int acc = 0;
       for (int p = 0; p < P; ++p) {
         ts[p] = acc;
         if (l < st[p].n_lin) {
           const LinDev& L = st[p].lin[l];
           const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (mode == 1 ? L.n_out : T);
-          const int tm = cdiv(M, TILE_M), tn = cdiv(N, TILE_N), n_kb = cdiv(K, TILE_K);
+          const int tm = cdiv(M, tile_m), tn = cdiv(N, tile_n), n_kb = cdiv(K, TILE_K);
           const int groups = mode == 1 ? cdiv(tm, DG_MG) : tm;
           for (int g = 0; g < groups; ++g) {
             const int n_m = mode == 1 ? std::min(DG_MG, tm - g * DG_MG) : 1;
@@ -752,8 +915,8 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
         }
       }
       ts[P] = acc;
-      const int G = std::max(1, std::min(acc, sms));
-      tt.grid[mode][l] = G;
+      const int G = std::max(1, std::min(acc, pair ? sms / 2 : sms));     // persistent CTAs, or CTA pairs
+      tt.grid[mode][l] = pair ? 2 * G : G;
       tt.order_off[mode][l] = tt.orders.size();
       if (acc == 0) { tt.n_slots[mode][l] = 0; continue; }
       std::stable_sort(work.begin(), work.end(), [](const std::pair<long long, int>& a, const std::pair<long long, int>& b) { return a.first > b.first; });
@@ -880,6 +1043,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       plan->n_slots[mode][l] = tt.n_slots[mode][l];
       plan->grid[mode][l] = tt.grid[mode][l];
+      plan->pair[mode][l] = tt.pair[mode][l];
       plan->order_off[mode][l] = tt.order_off[mode][l];
     }
   char* region = (char*)ws_region;
@@ -894,6 +1058,8 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<0>::kSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
@@ -913,6 +1079,11 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   const int grid = plan->grid[mode][lvl];                             // one persistent CTA per SM
   const int* ts = plan->d_tile_start + ((size_t)mode * PM_MAX_LINEARS + lvl) * (plan->P + 1);
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
+  if (plan->pair[mode][lvl]) {
+    if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    return cudaGetLastError();
+  }
   if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);

@@ -79,6 +79,22 @@ def test_bf16_small(cuda_device, opt):
     assert torch.equal(pipe.w_lp, pipe.w.to(torch.bfloat16))
 
 
+@pytest.mark.parametrize("width,T", [(320, 384), (512, 256)])
+def test_bf16_cta_pair_tiles(cuda_device, width, T):
+    """Every GEMM has at least 256 rows and columns, so the forward and wgrad launches run on CTA pairs with
+    256 x 256 tiles; 320 and 384 leave ragged tails in rows, columns and the reduction dimension."""
+    wl = I.mlp_workload("pair_tiles", 4, width, 2, "gelu", T, compute="bf16", optimizer="sgdm", alpha=0.01, beta1=0.9,
+                        K=5, D=0.5, steps=20, seed=191005124 + 71)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("pair tiles loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_LOSS_TOL)
+    worst = compare_params(pipe, res, BF16_W_TOL)
+    print("pair tiles worst relative weight error", worst)
+
+
 def test_phase_order_and_drain_rules(cuda_device):
     import torch
     import paper_1910_05124_b200 as pm
