@@ -69,26 +69,44 @@ __device__ __forceinline__ void epi_zy8(const float (&pf)[8], uint8_t* zdst, uin
   *reinterpret_cast<uint4*>(ydst) = make_uint4(pack_bf16(yf[0], yf[1]), pack_bf16(yf[2], yf[3]), pack_bf16(yf[4], yf[5]), pack_bf16(yf[6], yf[7]));
 }
 
+// State of one epilogue warp's staging buffer (two slots of 4 KB) across blocks.
+struct EpiState {
+  bool stored = false;        // a TMA store of this warp may still be reading the staging buffer
+  bool prev_both = false;     // the previous block used both slots
+  uint32_t slot = 0;          // slot the next single-output block writes
+};
+
 // One epilogue block of the forward (MODE 0) or wgrad (MODE 2) GEMM: 32 rows x 64 accumulator columns held in
 // r0, r1 go through this warp's swizzled staging buffer to one or two TMA stores (full 128-byte rows; rows and
 // columns beyond the tensor are clipped).  Called by a whole warp; lane = row within the block.
+// A block with one bf16 output (a Linear without activation) fills one 4 KB slot and alternates slots, so it
+// only waits for the store issued two blocks ago; blocks with two outputs (z and y, or 64 fp32 columns) use both.
+// bias4: the bias of columns 4*l .. 4*l+3 of the warp's column range in lane l (MODE 0), fetched before the
+// accumulator was awaited; bias_lane0: the lane holding this block's first four columns.
 template <int MODE>
 __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* lm, const StageDev& s, const StageDyn& d, const LinDev& L,
                                           int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
-                                          uint8_t* obuf, uint32_t obuf_s, int lane) {
+                                          uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es) {
   const uint32_t row_off = (uint32_t)lane * 128;
   const uint32_t sw = (uint32_t)(lane & 7);
+  const bool f32out = MODE == 0 && (L.flags & LF_OUT_F32) != 0;
+  const bool both = MODE == 2 || f32out || ((L.flags & LF_WRITE_Z) && (L.flags & LF_WRITE_Y));
+  if (lane == 0 && es.stored) {                                   // earlier stores must have finished reading what is overwritten
+    if (both || es.prev_both) tma_store_wait_read(); else tma_store_wait_read_1();
+  }
+  __syncwarp();
+  const uint32_t so = both ? 0u : es.slot * 4096u;                // slot of a single-output block
   if (MODE == 0) {
-    const float* bias = t.a.w + L.b_off;
-    const bool f32out = (L.flags & LF_OUT_F32) != 0;
     const int act = L.act;
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-      const int n = nb + g * 8;
-      float bb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      if (n < N) {
-        const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
-        bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
+      float bb[8];
+      {
+        const int src = bias_lane0 + 2 * g;
+        bb[0] = __shfl_sync(0xffffffffu, bias4.x, src); bb[1] = __shfl_sync(0xffffffffu, bias4.y, src);
+        bb[2] = __shfl_sync(0xffffffffu, bias4.z, src); bb[3] = __shfl_sync(0xffffffffu, bias4.w, src);
+        bb[4] = __shfl_sync(0xffffffffu, bias4.x, src + 1); bb[5] = __shfl_sync(0xffffffffu, bias4.y, src + 1);
+        bb[6] = __shfl_sync(0xffffffffu, bias4.z, src + 1); bb[7] = __shfl_sync(0xffffffffu, bias4.w, src + 1);
       }
       float pf[8];
 #pragma unroll
@@ -100,7 +118,9 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
       } else {
         const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
-        if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
+        if (!both)                                                  // no activation: z = y = bf16(acc + b), one output
+          *reinterpret_cast<uint4*>(obuf + so + off) = make_uint4(pack_bf16(pf[0], pf[1]), pack_bf16(pf[2], pf[3]), pack_bf16(pf[4], pf[5]), pack_bf16(pf[6], pf[7]));
+        else if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
         else if (act == PM_ACT_RELU) epi_zy8<PM_ACT_RELU>(pf, obuf + off, obuf + 4096 + off);
         else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);
       }
@@ -116,16 +136,17 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
   __syncwarp();
   if (lane == 0) {
     if (MODE == 0) {
-      if (L.flags & LF_OUT_F32) {
+      const int yslot = lvl < s.n_lin - 1 ? d.f_slot
+                        : (s.post == POST_RESIDUAL ? 0 : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
+      if (f32out) {
         tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
         if (nb + 32 < N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
+      } else if (!both) {
+        if (L.flags & LF_WRITE_Z) tma_store_3d(lm + MAP_Z_OUT, obuf_s + so, nb, mrow, d.f_slot);
+        else if (L.flags & LF_WRITE_Y) tma_store_3d(lm + MAP_Y_OUT, obuf_s + so, nb, mrow, yslot);
       } else {
-        if (L.flags & LF_WRITE_Z) tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
-        if (L.flags & LF_WRITE_Y) {
-          const int yslot = lvl < s.n_lin - 1 ? d.f_slot
-                            : (s.post == POST_RESIDUAL ? 0 : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
-          tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
-        }
+        tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
+        tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
       }
     } else {
       tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
@@ -133,6 +154,14 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
     }
     tma_store_commit();
   }
+  es.stored = true;
+  es.prev_both = both;
+  if (!both) es.slot ^= 1u;
+}
+
+// bias of columns n .. n+3 (zero beyond the tensor); n is a multiple of four
+__device__ __forceinline__ float4 load_bias4(const float* bias, int n, int N) {
+  return n < N ? __ldg(reinterpret_cast<const float4*>(bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 // ---- tile walk ---------------------------------------------------------------------------------------
@@ -292,7 +321,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     const uint32_t sw = (uint32_t)(lane & 7);
     Ring acc{0, 0};
     bool ok = true;
-    bool stored = false;
+    EpiState es;
     for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
       const int tile = order[slot];
       if (tile < 0) continue;
@@ -304,6 +333,8 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
       const int mrow = tl.m0 + q * 32;                                // first row of this warp's block
       const int nb = tl.n0 + half * 64;
+      // bias of this warp's 64 columns, four per lane in lanes 0..15, on its way while the accumulator completes
+      const float4 bias4 = (MODE == 0 && lane < 16) ? load_bias4(t.a.w + L.b_off, nb + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -315,17 +346,13 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar_tempty + 8 * acc.idx);                        // the accumulator buffer may be overwritten now
-        if (stored) tma_store_wait_read();                            // previous stores have finished reading the staging buffer
-      }
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc.idx);           // the accumulator buffer may be overwritten now
       __syncwarp();
       acc.advance(2);
       if (mrow >= tl.M || nb >= tl.N) continue;                       // nothing of this block is inside the tensor
-      epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane);
-      stored = true;
+      epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, 0, es);
     }
-    if (lane == 0 && stored) tma_store_wait_all();                    // global writes complete before the CTA retires
+    if (lane == 0 && es.stored) tma_store_wait_all();                    // global writes complete before the CTA retires
   }
   tc_fence_before();
   __syncthreads();
@@ -500,7 +527,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
     const uint32_t obuf_s = outs + ew * 8192;
     Ring acc{0, 0};
     bool ok = true;
-    bool stored = false;
+    EpiState es;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
       const int tile = order[slot];
       if (tile < 0) continue;
@@ -511,6 +538,8 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       const LinDev& L = s.lin[lvl];
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
       const int mrow = tl.m0 + rank * TILE_M + q * 32;                // first row of this warp's blocks
+      // bias of this warp's 128 columns, four per lane, on its way while the accumulator completes
+      const float4 bias4 = MODE == 0 ? load_bias4(t.a.w + L.b_off, tl.n0 + half * 128 + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 34);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -525,18 +554,14 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         tmem_ld_wait();
         if (c == 1) tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
-          if (c == 1) mbar_arrive_cluster(mapa_shared(bar_tempty + 8 * acc.idx, 0));   // this warp has read its part of the accumulator
-          if (stored) tma_store_wait_read();                          // previous stores have finished reading the staging buffer
-        }
+        if (c == 1 && lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty + 8 * acc.idx, 0));   // this warp has read its part of the accumulator
         __syncwarp();
         if (mrow >= tl.M || nb >= tl.N) continue;                     // nothing of this block is inside the tensor
-        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane);
-        stored = true;
+        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es);
       }
       acc.advance(2);
     }
-    if (lane == 0 && stored) tma_store_wait_all();                    // global writes complete before the CTA retires
+    if (lane == 0 && es.stored) tma_store_wait_all();                    // global writes complete before the CTA retires
   }
   tc_fence_before();
   cluster_sync_all();                                                 // no barrier or shared memory of a CTA is touched after this
