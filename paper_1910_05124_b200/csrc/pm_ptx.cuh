@@ -153,8 +153,11 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
+// Arrive on a barrier of another CTA of the cluster.  Release at CTA scope (the default): the arrival only says
+// that this thread's tcgen05.ld have completed (tcgen05.wait::ld came before), it publishes no memory, and a
+// cluster-scope release was measured to stall the epilogue warp for microseconds behind its stores in flight.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // every thread of both CTAs
 __device__ __forceinline__ void cluster_sync_all() {
