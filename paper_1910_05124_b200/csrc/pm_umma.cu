@@ -47,7 +47,7 @@ template <int MODE> struct Cfg {                           // MODE 0 forward, 2 
 };
 
 enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6,
-       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAPS_PER_LINEAR = 11 };
+       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAP_W_F32H = 11, MAP_D_F32H = 12, MAPS_PER_LINEAR = 13 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, operand majors as given.
 __device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
@@ -856,6 +856,298 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
   }
 }
 
+// ---- dgrad on CTA pairs ------------------------------------------------------------------------------------
+// The same product and the same on-the-fly correction on tiles of 256 rows x 128 columns per CTA pair
+// (tcgen05.mma.cta_group::2, M = 256, N = 128).  Each CTA stages the fp32 w and delta of ITS 64 columns
+// (2 x 16 KB per k-block), converts them to bf16(w - gap*delta) in its own shared memory, and loads its 128
+// rows of dz; two 256-row tiles share one converted tile, so a CTA ingests 64 KB per 2 x (128x128x64) of its
+// own products, as the single-CTA kernel does, but the accumulators (2 x 128 columns) are double-buffered and
+// the eight epilogue warps drain one group while the next is computed.  Barriers: staging (sfull / sempty)
+// is local to a CTA; the converted tile (bfull) and the dz tiles (afull) are counted in the leader, which
+// issues the MMAs; tcgen05.commit releases slots (bempty, aempty) and publishes accumulators (tfull) in both
+// CTAs; the epilogue warps of both arrive on the leader's tempty.
+constexpr int DP_TILE_M = 256, DP_TILE_N = 128, DP_HALF_N = 64;
+constexpr int DP_MG = 2;                                   // 256-row tiles per converted tile
+constexpr int DP_NG = 3, DP_NB = 2, DP_NA = 4;             // fp32 staging ring, converted ring, dz ring
+constexpr int DP_STG_HALF = TILE_K * DP_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
+constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;
+constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
+constexpr int DP_ACC_COLS = DP_MG * DP_TILE_N;             // 256 columns per accumulator buffer
+constexpr int DP_XF_WARPS = 8, DP_EPI_WARPS = 8;
+constexpr int DP_THREADS = 32 * (2 + DP_XF_WARPS + DP_EPI_WARPS);
+constexpr int DP_TILE_BYTES = DP_NG * DP_STG_BYTES + DP_NB * DP_B_BYTES + DP_NA * A_BYTES + DP_EPI_WARPS * 4096;
+constexpr int DP_SMEM_BYTES = DP_TILE_BYTES + 1024 + 512;
+
+__device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
+  DgTile r;
+  int lo = 0, hi = t.P - 1;
+  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  r.p = lo;
+  const StageDyn& d = t.dyn[lo];
+  const StageDev& s = t.st[lo];
+  r.valid = lvl < s.n_lin && d.b_mb >= 0 && !(lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
+  const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
+  r.M = t.T; r.N = L.n_in; r.K = L.n_out;
+  const int tiles_n = (r.N + DP_TILE_N - 1) / DP_TILE_N;
+  const int tiles_m = (r.M + DP_TILE_M - 1) / DP_TILE_M;
+  const int local = tile - tile_start[lo];
+  const int mg = local / tiles_n;
+  r.m0 = mg * DP_MG * DP_TILE_M;
+  r.n0 = (local % tiles_n) * DP_TILE_N;
+  r.n_m = min(DP_MG, tiles_m - mg * DP_MG);
+  r.n_kb = (r.K + TILE_K - 1) / TILE_K;
+  return r;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(DP_THREADS, 1)
+umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t stg = base;                                          // [DP_NG][w 16 KB | delta 16 KB]
+  const uint32_t sB = stg + DP_NG * DP_STG_BYTES;                     // [DP_NB][8 KB] converted operand (this CTA's 64 columns)
+  const uint32_t sA = sB + DP_NB * DP_B_BYTES;                        // [DP_NA][16 KB] dz tiles (this CTA's 128 rows)
+  const uint32_t sO = sA + DP_NA * A_BYTES;                           // [8][4 KB] epilogue staging
+  uint8_t* stg_ptr = base_ptr;
+  uint8_t* sB_ptr = base_ptr + DP_NG * DP_STG_BYTES;
+  uint8_t* sO_ptr = sB_ptr + DP_NB * DP_B_BYTES + DP_NA * A_BYTES;
+  const uint32_t bars = base + DP_TILE_BYTES;
+  const uint32_t bar_sfull = bars, bar_sempty = bar_sfull + 8 * DP_NG, bar_bfull = bar_sempty + 8 * DP_NG,
+                 bar_bempty = bar_bfull + 8 * DP_NB, bar_afull = bar_bempty + 8 * DP_NB, bar_aempty = bar_afull + 8 * DP_NA,
+                 bar_tfull = bar_aempty + 8 * DP_NA, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + DP_TILE_BYTES + 8 * (2 * DP_NG + 2 * DP_NB + 2 * DP_NA + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();                            // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < DP_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, DP_XF_WARPS); }
+    for (int i = 0; i < DP_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * DP_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < DP_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 2 * DP_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc_pair(smem_u32(tmem_slot), 2 * DP_ACC_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs): the fp32 staging loads run one k-block ahead of the dz loads ----------------
+    if (lane == 0) {
+      struct Cursor { int tile, kb; DgTile tl; bool done; };
+      auto seek = [&](Cursor& c) {
+        for (; c.tile < n_slots; c.tile += n_pairs) {
+          const int tile = order[c.tile];
+          if (tile < 0) continue;
+          c.tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+          if (c.tl.valid) { c.kb = 0; c.done = false; return; }
+        }
+        c.done = true;
+      };
+      auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += n_pairs; seek(c); } };
+      Cursor cs{pair, 0, DgTile{}, false}, ca{pair, 0, DgTile{}, false};
+      seek(cs); seek(ca);
+      Ring sg{0, 0}, ar{0, 0};
+      int issued_sg = 0, issued_a = 0;
+      bool ok = true;
+      auto issue_staging = [&](const Cursor& c) {
+        const StageDyn& d = t.dyn[c.tl.p];
+        const CUtensorMap* lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) { ok = false; return; }
+        const uint32_t sw = stg + sg.idx * DP_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+        const bool corr = d.use_delta != 0;
+        mbar_arrive_expect_tx(fb, corr ? DP_STG_BYTES : DP_STG_HALF);
+        tma_load_2d(sw, lm + MAP_W_F32H, fb, c.tl.n0 + rank * DP_HALF_N, c.kb * TILE_K);
+        if (corr) tma_load_2d(sw + DP_STG_HALF, lm + MAP_D_F32H, fb, c.tl.n0 + rank * DP_HALF_N, c.kb * TILE_K);
+        sg.advance(DP_NG); ++issued_sg;
+      };
+      if (!cs.done) { issue_staging(cs); step(cs); }
+      while (!ca.done && ok) {
+        if (!cs.done) { issue_staging(cs); step(cs); if (!ok) break; }
+        const StageDyn& d = t.dyn[ca.tl.p];
+        const StageDev& sd_ = t.st[ca.tl.p];
+        const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        for (int mi = 0; mi < ca.tl.n_m; ++mi) {
+          if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 42)) { ok = false; break; }
+          if (rank == 0) mbar_arrive_expect_tx(bar_afull + 8 * ar.idx, 2 * A_BYTES);       // the rows of both CTAs
+          tma_load_3d_pair(sA + ar.idx * A_BYTES, lm + MAP_DZ_K, mapa_shared(bar_afull + 8 * ar.idx, 0),
+                           ca.kb * TILE_K, ca.tl.m0 + mi * DP_TILE_M + rank * TILE_M, dz_slot);
+          ar.advance(DP_NA); ++issued_a;
+        }
+        step(ca);
+      }
+      if (*abort_flag) {
+        for (int back = 1; back <= DP_NG && back <= issued_sg; ++back) {
+          const int it = issued_sg - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_sfull + 8 * (it % DP_NG), (uint32_t)(it / DP_NG) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+        if (rank == 0) {
+          for (int back = 1; back <= DP_NA && back <= issued_a; ++back) {
+            const int it = issued_a - back;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_afull + 8 * (it % DP_NA), (uint32_t)(it / DP_NA) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+          }
+        } else {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc_mn(DP_TILE_M, DP_TILE_N, 0, 1);
+      const uint64_t dba = desc_base(16, 1024), dbb = desc_base(DP_B_BYTES, 1024);   // B: one 64-column run per CTA
+      Ring br{0, 0}, ar{0, 0}, acc{0, 0};
+      bool ok = true;
+      for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
+        const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 43)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * DP_ACC_COLS);
+        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+          if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 44)) { ok = false; break; }
+          const uint32_t sb = sB + br.idx * DP_B_BYTES;
+          for (int mi = 0; mi < tl.n_m; ++mi) {
+            if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 45)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = sA + ar.idx * A_BYTES;
+#pragma unroll
+            for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * DP_TILE_N), desc_at(dba, sa + k16 * 32), desc_at(dbb, sb + k16 * 2048),
+                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            tc_commit_pair(bar_aempty + 8 * ar.idx, 3);
+            ar.advance(DP_NA);
+          }
+          if (ok) tc_commit_pair(bar_bempty + 8 * br.idx, 3);
+          br.advance(DP_NB);
+        }
+        if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);
+        acc.advance(2);
+      }
+    }
+  } else if (warp < 2 + DP_XF_WARPS) {
+    // ---------------- operand transform (both CTAs): fp32 w, delta [64 k][64 n] -> bf16(w - gap*delta), MN-major ----------------
+    // thread: four consecutive columns (c4) of rows r0 + 16 j; reads are contiguous float4, stores 8 bytes into the swizzled atom
+    const int tt = threadIdx.x - 64;                                  // 0..255
+    const int c4 = tt & 15, rbase = tt >> 4;                          // 0..15, 0..15
+    const uint32_t leader_bfull = mapa_shared(bar_bfull, 0);
+    Ring br{0, 0}, sg{0, 0};
+    bool ok = true;
+    for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
+      const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const float gapf = (float)t.st[tl.p].gap;
+      const bool corr = t.dyn[tl.p].use_delta != 0;
+      for (int kb = 0; kb < tl.n_kb; ++kb) {
+        bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 46);
+        go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 47);
+        go = __all_sync(0xffffffffu, go);
+        if (!go) { ok = false; break; }
+        const uint8_t* src = stg_ptr + sg.idx * DP_STG_BYTES;
+        uint8_t* dst = sB_ptr + br.idx * DP_B_BYTES;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int r = rbase + 16 * j;                               // k-row
+          const float4 w = *reinterpret_cast<const float4*>(src + r * (DP_HALF_N * 4) + c4 * 16);
+          float v[4] = {w.x, w.y, w.z, w.w};
+          if (corr) {
+            const float4 dl = *reinterpret_cast<const float4*>(src + DP_STG_HALF + r * (DP_HALF_N * 4) + c4 * 16);
+            v[0] = __fsub_rn(v[0], __fmul_rn(gapf, dl.x)); v[1] = __fsub_rn(v[1], __fmul_rn(gapf, dl.y));   // w - (tau_fwd - tau_bkwd) * delta
+            v[2] = __fsub_rn(v[2], __fmul_rn(gapf, dl.z)); v[3] = __fsub_rn(v[3], __fmul_rn(gapf, dl.w));
+          }
+          const uint32_t off = (uint32_t)(r >> 3) * 1024 + (uint32_t)(r & 7) * 128 + ((((uint32_t)c4 >> 1) ^ (uint32_t)(r & 7)) << 4) + ((uint32_t)c4 & 1) * 8;
+          *reinterpret_cast<uint2*>(dst + off) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive_cluster(leader_bfull + 8 * br.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
+        br.advance(DP_NB); sg.advance(DP_NG);
+      }
+    }
+  } else {
+    // ---------------- epilogue (both CTAs): 8 warps, warp%4 = TMEM lane group, two warps per group split the 128 columns ----------------
+    const int q = warp & 3;
+    const int ew = warp - 2 - DP_XF_WARPS;                            // 0..7
+    const int half = ew >> 2;
+    uint8_t* obuf = sO_ptr + ew * 4096;
+    const uint32_t obuf_s = sO + ew * 4096;
+    const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
+    const uint32_t leader_tempty = mapa_shared(bar_tempty, 0);
+    Ring acc{0, 0};
+    bool ok = true, stored = false;
+    for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
+      const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const StageDyn& d = t.dyn[tl.p];
+      const StageDev& s = t.st[tl.p];
+      const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+      bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 48);
+      ready = __all_sync(0xffffffffu, ready);
+      if (!ready) { ok = false; break; }
+      tc_fence_after();
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0;
+      const int nb = tl.n0 + half * 64;
+#pragma unroll 1
+      for (int mi = 0; mi < tl.n_m; ++mi) {
+        const int mrow = tl.m0 + mi * DP_TILE_M + rank * TILE_M + q * 32;
+        uint32_t r0[32], r1[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * DP_ACC_COLS + mi * DP_TILE_N + half * 64);
+        tmem_ld32(taddr, r0);
+        tmem_ld32(taddr + 32, r1);
+        tmem_ld_wait();
+        if (mi == tl.n_m - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc.idx);   // this warp has read its part of both accumulators
+        }
+        if (mrow >= tl.M || nb >= tl.N) continue;
+        if (lane == 0 && stored) tma_store_wait_read();
+        __syncwarp();
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+          *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
+              make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) { tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, dslot); tma_store_commit(); }
+        stored = true;
+      }
+      acc.advance(2);
+    }
+    if (lane == 0 && stored) tma_store_wait_all();
+  }
+  tc_fence_before();
+  cluster_sync_all();                                                 // no barrier or shared memory of a CTA is touched after this
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 2 * DP_ACC_COLS);
+  }
+}
+
 // ---- host side -----------------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -913,17 +1205,19 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
       int* ts = tt.tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
       std::vector<std::pair<long long, int>> work;          // (weight, tile id)
       // forward and wgrad launches whose GEMMs all have at least 256 rows and columns run on CTA pairs
-      bool pair = allow_pair && mode != 1 && sms >= 2;
+      bool pair = allow_pair && sms >= 2;
       int n_lin_here = 0;
       for (int p = 0; p < P && pair; ++p)
         if (l < st[p].n_lin) {
           const LinDev& L = st[p].lin[l];
           ++n_lin_here;
           if ((mode == 2 ? L.n_out : T) < P2_TILE || (mode == 0 ? L.n_out : L.n_in) < P2_TILE) pair = false;
+          if (mode == 1 && p == 0 && l == 0 && st[p].pre != PRE_EMBED) --n_lin_here;   // the first Linear of the network has no input gradient
         }
       pair = pair && n_lin_here > 0;
       tt.pair[mode][l] = pair;
-      const int tile_m = pair ? P2_TILE : TILE_M, tile_n = pair ? P2_TILE : TILE_N;
+      const int tile_m = pair ? P2_TILE : TILE_M, tile_n = pair ? (mode == 1 ? DP_TILE_N : P2_TILE) : TILE_N;
+      const int mg_rows = pair ? DP_MG : DG_MG;                     // dgrad: row tiles sharing one converted weight tile
       int acc = 0;
       for (int p = 0; p < P; ++p) {
         ts[p] = acc;
@@ -931,9 +1225,9 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
           const LinDev& L = st[p].lin[l];
           const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (mode == 1 ? L.n_out : T);
           const int tm = cdiv(M, tile_m), tn = cdiv(N, tile_n), n_kb = cdiv(K, TILE_K);
-          const int groups = mode == 1 ? cdiv(tm, DG_MG) : tm;
+          const int groups = mode == 1 ? cdiv(tm, mg_rows) : tm;
           for (int g = 0; g < groups; ++g) {
-            const int n_m = mode == 1 ? std::min(DG_MG, tm - g * DG_MG) : 1;
+            const int n_m = mode == 1 ? std::min(mg_rows, tm - g * mg_rows) : 1;
             for (int n = 0; n < tn; ++n) work.push_back({(long long)n_kb * n_m + 3 * n_m, acc + g * tn + n});
           }
           acc += groups * tn;
@@ -1020,6 +1314,9 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         okm = okm && encode(fn, m + MAP_W_K, 0, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err);
         okm = okm && encode(fn, m + MAP_W_F32, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
         okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
+        uint32_t box4h[2] = {64, TILE_K};                               // CTA-pair dgrad: 64 columns per CTA
+        okm = okm && encode(fn, m + MAP_W_F32H, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4h, err);
+        okm = okm && encode(fn, m + MAP_D_F32H, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4h, err);
       }
       {
         // dz operand (same rule as dz_src): dz scratch | dh scratch | attention's dy | rotating incoming-gradient mailbox
@@ -1085,6 +1382,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DP_SMEM_BYTES);
   if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
@@ -1106,6 +1404,7 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
   if (plan->pair[mode][lvl]) {
     if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     return cudaGetLastError();
   }
