@@ -1022,17 +1022,23 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
         for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
           if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 44)) { ok = false; break; }
           const uint32_t sb = sB + br.idx * DP_B_BYTES;
+          // both dz tiles first, then the products of the two row tiles interleaved: consecutive MMAs write
+          // different accumulators
+          uint32_t sa[DP_MG], abar[DP_MG];
           for (int mi = 0; mi < tl.n_m; ++mi) {
             if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 45)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t sa = sA + ar.idx * A_BYTES;
-#pragma unroll
-            for (int k16 = 0; k16 < TILE_K / 16; ++k16)
-              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * DP_TILE_N), desc_at(dba, sa + k16 * 32), desc_at(dbb, sb + k16 * 2048),
-                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
-            tc_commit_pair(bar_aempty + 8 * ar.idx, 3);
+            sa[mi] = sA + ar.idx * A_BYTES;
+            abar[mi] = bar_aempty + 8 * ar.idx;
             ar.advance(DP_NA);
           }
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+            for (int mi = 0; mi < tl.n_m; ++mi)
+              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * DP_TILE_N), desc_at(dba, sa[mi] + k16 * 32), desc_at(dbb, sb + k16 * 2048),
+                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          for (int mi = 0; mi < tl.n_m; ++mi) tc_commit_pair(abar[mi], 3);
           if (ok) tc_commit_pair(bar_bempty + 8 * br.idx, 3);
           br.advance(DP_NB);
         }
