@@ -21,7 +21,7 @@ namespace pm {
 constexpr int AT_S = 128, AT_DK = 64;
 constexpr int AT_TILE = AT_S * AT_DK * 2;          // 16 KB: one [128 x 64] bf16 tile
 constexpr int AT_FWD_SMEM = 3 * AT_TILE + 2 * AT_TILE + 1024 + 128;
-constexpr int AT_BWD_SMEM = 7 * AT_TILE + 1024 + 128;   // Q, K, dO, V|P0, P1, dS0, dS1: two CTAs fit on one SM
+constexpr int AT_BWD_SMEM = 5 * AT_TILE + 1024 + 128 + 3 * 2 * AT_S * 4;   // Q, K, dO, V|P0|dS0, P1|dS1, row-statistics exchange: two CTAs per SM
 constexpr int AT_TMEM_COLS = 256;
 
 enum { AMAP_QKV = 0, AMAP_DO = 1, AMAPS_PER_STAGE = 2 };
@@ -90,8 +90,8 @@ __device__ __forceinline__ bool wait_mma(const AttnCommon& c, uint32_t parity, i
   return ok;
 }
 
-__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int causal, int* status) {
-  const int p = blockIdx.y;
+__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int causal, int* status) {
+  const int p = stage_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || s.post != POST_ATTENTION) return;
@@ -179,8 +179,28 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
   attn_teardown(c, tmem_base);
 }
 
-__global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, int causal, int* status) {
-  const int p = blockIdx.y;
+// Backward: 256 threads, two per query row (thread r + 128*hf owns keys 64*hf .. 64*hf+63 of row r), two CTAs per SM.
+// Shared memory holds five tiles: Q, K, dO, and V | X, where P (two 64-key tiles) overwrites V and X once
+// dP = dO V^T is done, and dS overwrites P once dV = P^T dO is done.  The exponentials are computed once and
+// stay in registers; dP is read from tensor memory twice (for D, then for dS).  Row statistics of the two halves
+// meet in a small exchange buffer.  Accumulators: S at columns 0..127, dP at 128..255; then dV at 0..63,
+// dQ at 64..127, dK at 128..191.
+constexpr int AT_BWD_THREADS = 256;
+constexpr int AT_BWD_TILES = 5;
+constexpr int AT_XCH_BYTES = 3 * 2 * AT_S * 4;
+
+__device__ __forceinline__ void attn_store32(__nv_bfloat16* dst, const uint32_t (&o)[32], float sc) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    float f[8];
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(o[g * 8 + e2]) * sc;
+    *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+  }
+}
+
+__global__ void __launch_bounds__(AT_BWD_THREADS, 2) attn_bwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int causal, int* status) {
+  const int p = stage_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.post != POST_ATTENTION) return;
@@ -188,17 +208,17 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
   if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
   extern __shared__ uint8_t smem_raw[];
-  const AttnCommon c = attn_setup(smem_raw, 7 * AT_TILE);
+  const AttnCommon c = attn_setup(smem_raw, AT_BWD_TILES * AT_TILE);
   const uint32_t tmem_base = *c.tmem_slot;
-  // V is dead once dP = dO V^T has completed, so the P tiles take its place (plus one more tile)
-  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sdO = sK + AT_TILE, sV = sdO + AT_TILE, sP = sV, sdS = sP + 2 * AT_TILE;
+  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sdO = sK + AT_TILE, sV = sdO + AT_TILE, sP = sV;   // P and dS: tiles 3 and 4
   uint8_t* pP = c.sptr + 3 * AT_TILE;
-  uint8_t* pdS = c.sptr + 5 * AT_TILE;
+  float* xch = reinterpret_cast<float*>(c.sptr + AT_BWD_TILES * AT_TILE + 128);                      // [3][2][128]
   const CUtensorMap* lm = maps + (size_t)p * AMAPS_PER_STAGE;
-  const int r = threadIdx.x;
-  const int warp = r >> 5;
+  const int tid = threadIdx.x;
+  const int r = tid & 127, hf = tid >> 7;                    // query row (TMEM lane), key half
+  const int warp = tid >> 5;
 
-  if (r == 0) {
+  if (tid == 0) {
     mbar_arrive_expect_tx(c.bar_load, 4 * AT_TILE);
     tma_load_3d(sQ, lm + AMAP_QKV, c.bar_load, h * AT_DK, b * AT_S, d.b_slot);
     tma_load_3d(sK, lm + AMAP_QKV, c.bar_load, dm + h * AT_DK, b * AT_S, d.b_slot);
@@ -214,94 +234,104 @@ __global__ void __launch_bounds__(128) attn_bwd_tc_kernel(TickArgs t, const CUte
   }
   if (wait_mma(c, 0, status, 15)) {
     const float scale = 0.125f;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t colS = (uint32_t)(hf * 64), colP = 128u + (uint32_t)(hf * 64);
+    float e[64];
     float mx = -INFINITY;
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
       uint32_t v[32];
-      tmem_ld32(lane_addr + cc * 32, v);
+      tmem_ld32(lane_addr + colS + cc * 32, v);
       tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (!causal || cc * 32 + j <= r) mx = fmaxf(mx, __uint_as_float(v[j]) * scale);
-    }
-    float l = 0.f;
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-      uint32_t v[32];
-      tmem_ld32(lane_addr + cc * 32, v);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (!causal || cc * 32 + j <= r) l += __expf(__uint_as_float(v[j]) * scale - mx);
-    }
-    const float inv = 1.0f / l;
-    float D = 0.f;
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-      uint32_t v[32], g[32];
-      tmem_ld32(lane_addr + cc * 32, v);
-      tmem_ld32(lane_addr + 128 + cc * 32, g);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (!causal || cc * 32 + j <= r) D += __uint_as_float(g[j]) * (__expf(__uint_as_float(v[j]) * scale - mx) * inv);
-    }
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-      uint32_t v[32], g[32];
-      tmem_ld32(lane_addr + cc * 32, v);
-      tmem_ld32(lane_addr + 128 + cc * 32, g);
-      tmem_ld_wait();
-      float pr[32], ds[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        pr[j] = (!causal || cc * 32 + j <= r) ? __expf(__uint_as_float(v[j]) * scale - mx) * inv : 0.f;
-        ds[j] = pr[j] * (__uint_as_float(g[j]) - D);
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        put_chunk(pP, r, cc * 4 + q, make_uint4(pack_bf16(pr[q * 8], pr[q * 8 + 1]), pack_bf16(pr[q * 8 + 2], pr[q * 8 + 3]),
-                                                 pack_bf16(pr[q * 8 + 4], pr[q * 8 + 5]), pack_bf16(pr[q * 8 + 6], pr[q * 8 + 7])));
-        put_chunk(pdS, r, cc * 4 + q, make_uint4(pack_bf16(ds[q * 8], ds[q * 8 + 1]), pack_bf16(ds[q * 8 + 2], ds[q * 8 + 3]),
-                                                  pack_bf16(ds[q * 8 + 4], ds[q * 8 + 5]), pack_bf16(ds[q * 8 + 6], ds[q * 8 + 7])));
+        e[cc * 32 + j] = (!causal || hf * 64 + cc * 32 + j <= r) ? __uint_as_float(v[j]) * scale : -INFINITY;
+        mx = fmaxf(mx, e[cc * 32 + j]);
       }
     }
+    xch[hf * AT_S + r] = mx;
+    __syncthreads();
+    mx = fmaxf(xch[r], xch[AT_S + r]);
+    float l = 0.f;
+#pragma unroll
+    for (int j = 0; j < 64; ++j) { e[j] = __expf(e[j] - mx); l += e[j]; }
+    xch[2 * AT_S + hf * AT_S + r] = l;
+    __syncthreads();
+    l = xch[2 * AT_S + r] + xch[3 * AT_S + r];
+    const float inv = 1.0f / l;
+#pragma unroll
+    for (int j = 0; j < 64; ++j) e[j] *= inv;                // P (unrounded)
+    float D = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      uint32_t g[32];
+      tmem_ld32(lane_addr + colP + cc * 32, g);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) D += __uint_as_float(g[j]) * e[cc * 32 + j];
+    }
+    xch[4 * AT_S + hf * AT_S + r] = D;
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      put_chunk(pP, r, hf * 8 + q, make_uint4(pack_bf16(e[q * 8], e[q * 8 + 1]), pack_bf16(e[q * 8 + 2], e[q * 8 + 3]),
+                                               pack_bf16(e[q * 8 + 4], e[q * 8 + 5]), pack_bf16(e[q * 8 + 6], e[q * 8 + 7])));
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
-    if (r == 0) {
+    D = xch[4 * AT_S + r] + xch[5 * AT_S + r];
+    const uint32_t i_mm = make_idesc_mn(128, 64, 1, 1), i_km = make_idesc_mn(128, 64, 0, 1);
+    if (tid == 0) {
       tc_fence_after();
       // dV = P^T dO : A = P read MN-major (m = key, k = query row; the second 64-key group one tile on), B = dO MN-major
-      const uint32_t i_mm = make_idesc_mn(128, 64, 1, 1), i_km = make_idesc_mn(128, 64, 0, 1);
       issue_k64(tmem_base, sP, sdO, i_mm, false, false, AT_TILE, 8192, false);
       issue_k64(tmem_base, sP + 4 * 2048, sdO + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
-      // dQ = dS K : A = dS K-major (k = key), B = K MN-major (k = key rows)
-      issue_k64(tmem_base + 64, sdS, sK, i_km, true, false, 0, 8192, false);
-      issue_k64(tmem_base + 64, sdS + AT_TILE, sK + 4 * 2048, i_km, true, false, 0, 8192, true);
-      // dK = dS^T Q : A = dS read MN-major (m = key, k = query row), B = Q MN-major
-      issue_k64(tmem_base + 128, sdS, sQ, i_mm, false, false, AT_TILE, 8192, false);
-      issue_k64(tmem_base + 128, sdS + 4 * 2048, sQ + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
       tc_commit(c.bar_mma);
     }
     if (wait_mma(c, 1, status, 16)) {
-      __nv_bfloat16* dy = reinterpret_cast<__nv_bfloat16*>(t.ws + s.dy) + (size_t)(b * AT_S + r) * 3 * dm + h * AT_DK;
-#pragma unroll 1
-      for (int which = 0; which < 3; ++which) {              // TMEM columns: dV at 0, dQ at 64, dK at 128
-        uint32_t o0[32], o1[32];
-        tmem_ld32(lane_addr + which * 64, o0);
-        tmem_ld32(lane_addr + which * 64 + 32, o1);
+      // dS = bf16(P * (dP - D)) over the P tiles (dV has finished reading them)
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        uint32_t g[32];
+        tmem_ld32(lane_addr + colP + cc * 32, g);
         tmem_ld_wait();
-        const float sc = which == 0 ? 1.0f : scale;
-        __nv_bfloat16* dst = dy + (which == 0 ? 2 * dm : (which == 1 ? 0 : dm));
+        float ds[32];
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint32_t* src = g < 4 ? o0 + (g & 3) * 8 : o1 + (g & 3) * 8;
-          float f[8];
+        for (int j = 0; j < 32; ++j) ds[j] = e[cc * 32 + j] * (__uint_as_float(g[j]) - D);
 #pragma unroll
-          for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(src[e2]) * sc;
-          *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-        }
+        for (int q = 0; q < 4; ++q)
+          put_chunk(pP, r, hf * 8 + cc * 4 + q, make_uint4(pack_bf16(ds[q * 8], ds[q * 8 + 1]), pack_bf16(ds[q * 8 + 2], ds[q * 8 + 3]),
+                                                            pack_bf16(ds[q * 8 + 4], ds[q * 8 + 5]), pack_bf16(ds[q * 8 + 6], ds[q * 8 + 7])));
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == 0) {
+        tc_fence_after();
+        // dQ = dS K : A = dS K-major (k = key), B = K MN-major (k = key rows)
+        issue_k64(tmem_base + 64, sP, sK, i_km, true, false, 0, 8192, false);
+        issue_k64(tmem_base + 64, sP + AT_TILE, sK + 4 * 2048, i_km, true, false, 0, 8192, true);
+        // dK = dS^T Q : A = dS read MN-major (m = key, k = query row), B = Q MN-major
+        issue_k64(tmem_base + 128, sP, sQ, i_mm, false, false, AT_TILE, 8192, false);
+        issue_k64(tmem_base + 128, sP + 4 * 2048, sQ + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
+        tc_commit(c.bar_mma);
+      }
+      // results go to the stage's dy buffer as [dq | dk | dv]; this thread stores 32 of the 64 head columns
+      __nv_bfloat16* dy = reinterpret_cast<__nv_bfloat16*>(t.ws + s.dy) + (size_t)(b * AT_S + r) * 3 * dm + h * AT_DK + hf * 32;
+      {
+        uint32_t o[32];
+        tc_fence_after();
+        tmem_ld32(lane_addr + hf * 32, o);                   // dV while dQ and dK are being computed
+        tmem_ld_wait();
+        attn_store32(dy + 2 * dm, o, 1.0f);
+      }
+      if (wait_mma(c, 0, status, 17)) {
+        uint32_t o[32];
+        tmem_ld32(lane_addr + 64 + hf * 32, o);
+        tmem_ld_wait();
+        attn_store32(dy, o, scale);
+        tmem_ld32(lane_addr + 128 + hf * 32, o);
+        tmem_ld_wait();
+        attn_store32(dy + dm, o, scale);
       }
     }
   }
@@ -316,10 +346,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct AttnPlan {
   const CUtensorMap* d_maps = nullptr;
+  const int* d_stage_ids = nullptr;      // the stages that end in attention, in pipeline order
+  int n_att = 0;
   int* d_status = nullptr;
 };
 
-uint64_t attn_workspace_bytes(int n_stages) { return 256 + (uint64_t)n_stages * AMAPS_PER_STAGE * sizeof(CUtensorMap); }
+static uint64_t attn_maps_bytes(int n_stages) { return (uint64_t)n_stages * AMAPS_PER_STAGE * sizeof(CUtensorMap); }
+uint64_t attn_workspace_bytes(int n_stages) { return 256 + attn_maps_bytes(n_stages) + ((uint64_t)n_stages * sizeof(int) + 255) / 256 * 256; }
 
 bool attn_tc_supported(int dtype, int S, int dk) { return dtype == PM_BF16 && S == AT_S && dk == AT_DK; }
 
@@ -332,6 +365,8 @@ pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<
   EncodeTiledFn fn = (EncodeTiledFn)fnp;
   std::vector<CUtensorMap> maps((size_t)t.P * AMAPS_PER_STAGE);
   memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+  std::vector<int> ids;
+  for (int p = 0; p < t.P; ++p) if (st[p].post == POST_ATTENTION) ids.push_back(p);
   const cuuint64_t T = (cuuint64_t)t.T;
   for (int p = 0; p < t.P; ++p) {
     const StageDev& s = st[p];
@@ -353,6 +388,7 @@ pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<
   }
   char* region = (char*)ws_region;
   cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess && !ids.empty()) e = cudaMemcpyAsync(region + 256 + attn_maps_bytes(t.P), ids.data(), ids.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_FWD_SMEM);
@@ -361,6 +397,8 @@ pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<
   AttnPlan* plan = new AttnPlan();
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
+  plan->d_stage_ids = (const int*)(region + 256 + attn_maps_bytes(t.P));
+  plan->n_att = (int)ids.size();
   *out = plan;
   return PM_OK;
 }
@@ -369,9 +407,10 @@ void attn_plan_destroy(AttnPlan* plan) { delete plan; }
 int* attn_status_word(AttnPlan* plan) { return plan ? plan->d_status : nullptr; }
 
 cudaError_t attn_tc_launch(AttnPlan* plan, const TickArgs& t, bool forward, cudaStream_t stream) {
-  dim3 grid(t.att_blocks, t.P);
-  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, 0, plan->d_status);
-  else attn_bwd_tc_kernel<<<grid, 128, AT_BWD_SMEM, stream>>>(t, plan->d_maps, 0, plan->d_status);
+  if (plan->n_att == 0) return cudaSuccess;
+  dim3 grid(t.att_blocks, plan->n_att);
+  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, 0, plan->d_status);
+  else attn_bwd_tc_kernel<<<grid, AT_BWD_THREADS, AT_BWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, 0, plan->d_status);
   return cudaGetLastError();
 }
 
