@@ -29,6 +29,9 @@ struct Layout {
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
   uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0, off_colred = 0;
+  uint64_t off_ids = 0, off_lnred = 0;
+  std::vector<int32_t> ids;             // [pre | ln | embed | residual] stage lists, P entries each
+  int32_t n_pre = 0, n_ln = 0, n_embed = 0, n_res = 0, ln_chunks = 0, ln_chunk_rows = 0, max_ln_dim = 0, ln_fused = 1;
   int32_t row_chunks = 1, chunk_rows = 256;
   bool att_tc = false;
   int32_t any_pre = 0, any_ln = 0, any_embed = 0, any_residual = 0, att_S = 0, att_dk = 0, att_blocks = 0, max_vocab = 0;
@@ -209,6 +212,21 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.row_chunks = (int32_t)((T + L.chunk_rows - 1) / L.chunk_rows);
   L.off_colred = w; w = align_up(w + (L.row_chunks > 1 ? (uint64_t)P * L.row_chunks * 2 * L.max_dim * 4 : 0), 256);
   L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
+  L.ids.assign((size_t)4 * P, 0);
+  for (int p = 0; p < P; ++p) {
+    const StageDev& s = L.st[p];
+    if (s.pre != PRE_NONE) L.ids[(size_t)0 * P + L.n_pre++] = p;
+    if (s.pre == PRE_LN) {
+      L.ids[(size_t)1 * P + L.n_ln++] = p; L.max_ln_dim = std::max(L.max_ln_dim, s.d_in);
+      if ((s.d_in & 7) != 0 || s.d_in > 1024) L.ln_fused = 0;
+    }
+    if (s.pre == PRE_EMBED) L.ids[(size_t)2 * P + L.n_embed++] = p;
+    if (s.post == POST_RESIDUAL) L.ids[(size_t)3 * P + L.n_res++] = p;
+  }
+  L.off_ids = w; w = align_up(w + sizeof(int32_t) * 4 * P, 256);
+  L.ln_chunk_rows = 64;
+  L.ln_chunks = (int32_t)((T + L.ln_chunk_rows - 1) / L.ln_chunk_rows);
+  L.off_lnred = w; w = align_up(w + (uint64_t)L.n_ln * L.ln_chunks * 2 * L.max_ln_dim * 4, 256);
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
   L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes((int)T, L.st) : 0), 256);
@@ -366,6 +384,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   UP(L.off_sched, c->L.sched);
   UP(L.off_b64, c->L.begin64);
   UP(L.off_e64, c->L.end64);
+  UP(L.off_ids, c->L.ids);
 #undef UP
   if (cfg->alpha_by_step) {
     if (cfg->alpha_len < 1) { delete c; return fail(nullptr, PM_ERR_INVALID_ARG, "alpha_len must be >= 1 with alpha_by_step"); }
@@ -396,6 +415,13 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
   t.any_pre = L.any_pre; t.any_ln = L.any_ln; t.any_embed = L.any_embed; t.any_residual = L.any_residual;
   t.att_S = L.att_S; t.att_dk = L.att_dk; t.att_blocks = L.att_blocks; t.max_vocab = L.max_vocab;
+  {
+    const int32_t* ids = (const int32_t*)(c->ws + L.off_ids);
+    t.pre_ids = ids; t.ln_ids = ids + P; t.embed_ids = ids + 2 * P; t.res_ids = ids + 3 * P;
+    t.n_pre = L.n_pre; t.n_ln = L.n_ln; t.n_embed = L.n_embed; t.n_res = L.n_res;
+    t.lnred_off = L.off_lnred; t.ln_chunks = L.ln_chunks; t.ln_chunk_rows = L.ln_chunk_rows; t.max_ln_dim = L.max_ln_dim;
+    t.ln_fused = L.ln_fused;
+  }
   if (L.pe_seq > 0) {
     // sinusoidal positions: PE[pos, 2i] = sin(pos / 10000^(2i/d)), PE[pos, 2i+1] = cos(same); double, rounded once to float
     std::vector<float> pe((size_t)L.pe_seq * L.pe_d);

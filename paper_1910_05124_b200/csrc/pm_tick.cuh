@@ -27,6 +27,13 @@ struct TickArgs {
   uint64_t loss_off;      // ws: loss log [loss_cap] float
   uint64_t lossred_off;   // ws: per-block loss partials [64] float + completion counter
   int64_t loss_cap;
+  // stage lists of the grouped launches (device, in pipeline order): stages with a pre-op, with LayerNorm, with an
+  // embedding, with a residual add; grids have one block row per list entry
+  const int32_t* pre_ids; const int32_t* ln_ids; const int32_t* embed_ids; const int32_t* res_ids;
+  int32_t n_pre, n_ln, n_embed, n_res;
+  uint64_t lnred_off;     // ws: LayerNorm parameter-gradient partials [n_ln][ln_chunks][2*max_ln_dim] float
+  int32_t ln_chunks, ln_chunk_rows, max_ln_dim;
+  int32_t ln_fused;       // every LayerNorm width is a multiple of 8 and at most 1024: one fused backward kernel
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages
 };

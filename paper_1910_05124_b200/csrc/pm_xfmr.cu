@@ -32,7 +32,7 @@ template <> __device__ __forceinline__ const __nv_bfloat16* table_ptr<__nv_bfloa
 // If the stage emits a skip tensor (attention / skip_out) u is also written to the next stage's skip buffer.
 template <typename AT>
 __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = t.pre_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || s.pre == PRE_NONE) return;
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
 }
 
 cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
-  dim3 grid((t.T + 7) / 8, t.P);
+  dim3 grid((t.T + 7) / 8, t.n_pre);
   if (dtype == PM_F32) pre_fwd_kernel<float><<<grid, 256, 0, stream>>>(t);
   else pre_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
   return cudaGetLastError();
@@ -129,7 +129,7 @@ cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream) {
 // ---- residual add: next stage's input = skip + y --------------------------------------------------------------
 template <typename AT>
 __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = t.res_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || s.post != POST_RESIDUAL) return;
@@ -235,7 +235,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
     if (e != cudaSuccess) return e;
   }
   if (any_res) {
-    dim3 grid(296, t.P);
+    dim3 grid(296, t.n_res);
     if (dtype == PM_F32) residual_kernel<float><<<grid, 256, 0, stream>>>(t);
     else residual_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
     e = cudaGetLastError();
@@ -466,7 +466,7 @@ __device__ __forceinline__ float du_total(const AT* du, const AT* gs, uint64_t i
 //   dxhat = du_total * gain_b (gain_b = gain - gap*delta: T2);  dx = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat*xhat))
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = t.ln_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN || p == 0) return;
@@ -543,7 +543,7 @@ constexpr int kLnCols = 256;                         // columns per block: 8 per
 
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
-  const int p = blockIdx.z;
+  const int p = t.ln_ids[blockIdx.z];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
@@ -610,7 +610,7 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
 }
 
 __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = t.ln_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
@@ -626,70 +626,237 @@ __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
   t.a.grad[s.beta_off + c] = b2;
 }
 
-// Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
-// One warp per vocabulary row, so the order of the additions is fixed and every row is written (zeros included).
-template <typename AT>
-__global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+// Fused LayerNorm backward (widths that are multiples of 8, at most NP*256): one pass over du, x and the skip
+// gradient produces dx and the partial column sums of dgain, dbias.  A block owns ln_chunk_rows rows; warp w takes
+// rows w, w+8, ... in ascending order, a lane owns 8 consecutive columns per 256-column group; per-warp partials are
+// added in warp order, per-block partials in block order by ln_fused_finish_kernel.
+template <typename AT, int NP>
+__global__ void __launch_bounds__(256) ln_bwd_fused_kernel(TickArgs t) {
+  const int li = blockIdx.y, p = t.ln_ids[li];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
-  if (d.b_mb < 0 || s.pre != PRE_EMBED) return;
-  extern __shared__ int32_t sid[];                           // the microbatch's token ids
-  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
-  for (int i = threadIdx.x; i < t.T; i += blockDim.x) sid[i] = ids[i];
-  __syncthreads();
+  if (d.b_mb < 0) return;
+  const int chunk = blockIdx.x;
+  const int r0 = chunk * t.ln_chunk_rows, r1 = min(t.T, r0 + t.ln_chunk_rows);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int v = blockIdx.x * 8 + warp;
-  if (v >= s.vocab) return;
   const int dm = s.d_in;
+  const uint64_t n = (uint64_t)t.T * dm;
   const AT* du = ws_at<AT>(t, s.dh);
   const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
-  float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
-  const float sc = sqrtf((float)dm);
-  // which tokens carry this id (ascending): at most a handful; collect them once, then stream the columns
-  for (int c0 = 0; c0 < dm; c0 += 32 * 8) {                 // up to 8 columns per lane per pass
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int tb = 0; tb < t.T; tb += 32) {
-      const int tok = tb + lane;
-      unsigned hit = __ballot_sync(0xffffffffu, tok < t.T && sid[tok] == v);
-      while (hit) {
-        const int j = __ffs(hit) - 1;
-        hit &= hit - 1;
-        const uint64_t ro = (uint64_t)(tb + j) * dm;
+  const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n);
+  const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
+  AT* out = p > 0 ? gin_write_prev<AT>(t, p, d) : nullptr;          // the first stage has no predecessor to hand dx to
+  const float gapf = (float)s.gap;
+  const bool corr = d.use_delta != 0;
+  float gb[NP][8], ag[NP][8], ab[NP][8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int c = c0 + e * 32 + lane;
-          if (c < dm) acc[e] = __fadd_rn(acc[e], __fmul_rn(du_total<AT>(du, gs, ro + c), sc));
+  for (int q = 0; q < NP; ++q) {
+    const int c = q * 256 + lane * 8;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { gb[q][k] = 0.f; ag[q][k] = 0.f; ab[q][k] = 0.f; }
+    if (c < dm) {
+      load8<float>(t.a.w + s.g_off + c, gb[q]);
+      if (corr) { float cv[8]; load8<float>(t.a.delta + s.g_off + c, cv);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) gb[q][k] = __fsub_rn(gb[q][k], __fmul_rn(gapf, cv[k])); }     // gain - (tau_fwd - tau_bkwd) * delta
+    }
+  }
+  for (int r = r0 + warp; r < r1; r += 8) {
+    const float mu = st[2 * r], rstd = st[2 * r + 1];
+    const uint64_t ro = (uint64_t)r * dm;
+    float xh[NP][8], dxh[NP][8];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int q = 0; q < NP; ++q) {
+      const int c = q * 256 + lane * 8;
+      if (c < dm) {
+        float xv[8], dv[8];
+        load8<AT>(x + ro + c, xv);
+        load8<AT>(du + ro + c, dv);
+        if (gs) { float sv[8]; load8<AT>(gs + ro + c, sv);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) dv[k] = __fadd_rn(dv[k], sv[k]); }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          xh[q][k] = (xv[k] - mu) * rstd;
+          dxh[q][k] = dv[k] * gb[q][k];
+          s1 += dxh[q][k]; s2 += dxh[q][k] * xh[q][k];
+          ag[q][k] = __fadd_rn(ag[q][k], __fmul_rn(dv[k], xh[q][k]));
+          ab[q][k] = __fadd_rn(ab[q][k], dv[k]);
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { xh[q][k] = 0.f; dxh[q][k] = 0.f; }
+      }
+    }
+    s1 = warp_sum(s1) / (float)dm;
+    s2 = warp_sum(s2) / (float)dm;
+    if (out) {
+#pragma unroll
+      for (int q = 0; q < NP; ++q) {
+        const int c = q * 256 + lane * 8;
+        if (c < dm) {
+          float o[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) o[k] = rstd * (dxh[q][k] - s1 - xh[q][k] * s2);
+          store8<AT>(out + ro + c, o);
         }
       }
     }
+  }
+  extern __shared__ float lnred[];                           // [8 warps][2][NP*256]
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int c = c0 + e * 32 + lane;
-      if (c < dm) out[c] = acc[e];
+  for (int q = 0; q < NP; ++q)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      lnred[(warp * 2 + 0) * (NP * 256) + q * 256 + lane * 8 + k] = ag[q][k];
+      lnred[(warp * 2 + 1) * (NP * 256) + q * 256 + lane * 8 + k] = ab[q][k];
+    }
+  __syncthreads();
+  float* part = ws_at<float>(t, t.lnred_off) + ((uint64_t)li * t.ln_chunks + chunk) * (2 * (uint64_t)t.max_ln_dim);
+  for (int c = threadIdx.x; c < dm; c += 256) {
+    float a = 0.f, b2 = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, lnred[(w * 2 + 0) * (NP * 256) + c]); b2 = __fadd_rn(b2, lnred[(w * 2 + 1) * (NP * 256) + c]); }
+    part[c] = a;
+    part[t.max_ln_dim + c] = b2;
+  }
+}
+
+__global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
+  const int li = blockIdx.y, p = t.ln_ids[li];
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0) return;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= s.d_in) return;
+  const float* part = ws_at<float>(t, t.lnred_off) + (uint64_t)li * t.ln_chunks * (2 * (uint64_t)t.max_ln_dim);
+  float a = 0.f, b2 = 0.f;
+  for (int k = 0; k < t.ln_chunks; ++k) {
+    a = __fadd_rn(a, part[(uint64_t)k * 2 * t.max_ln_dim + c]);
+    b2 = __fadd_rn(b2, part[(uint64_t)k * 2 * t.max_ln_dim + t.max_ln_dim + c]);
+  }
+  t.a.grad[s.g_off + c] = a;
+  t.a.grad[s.beta_off + c] = b2;
+}
+
+template <typename AT, int NP>
+static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
+  const size_t smem = (size_t)8 * 2 * NP * 256 * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set && smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute((const void*)ln_bwd_fused_kernel<AT, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  ln_bwd_fused_kernel<AT, NP><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(t);
+  ln_fused_finish_kernel<<<dim3((t.max_ln_dim + 255) / 256, t.n_ln), 256, 0, stream>>>(t);
+  return cudaGetLastError();
+}
+
+// Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
+// A block owns kEmbRows consecutive vocabulary rows.  It walks the microbatch's token ids once, in order, and
+// compacts the tokens that fall into its rows into a list (ballot + prefix over the warps, so the list is in
+// ascending token order); each warp then takes kEmbRows / 8 rows, picks its tokens from the list in order and
+// streams the columns.  Every row is written (zeros included) and the order of the additions is fixed.
+constexpr int kEmbRows = 32;
+
+template <typename AT>
+__global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
+  const int p = t.embed_ids[blockIdx.y];
+  const StageDyn& d = t.dyn[p];
+  const StageDev& s = t.st[p];
+  if (d.b_mb < 0) return;
+  const int v0 = blockIdx.x * kEmbRows;
+  if (v0 >= s.vocab) return;
+  extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
+  __shared__ int warp_cnt[2][8];
+  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int nh = 0;                                                // hits so far (the same value in every thread)
+  for (int tb0 = 0; tb0 < t.T; tb0 += 16 * 256) {            // 16 rounds of 256 tokens; the ids of all rounds are fetched first
+    int rel[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int tok = tb0 + k * 256 + threadIdx.x;
+      rel[k] = tok < t.T ? __ldg(ids + tok) - v0 : -1;
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if (tb0 + k * 256 >= t.T) break;
+      const bool hit = rel[k] >= 0 && rel[k] < kEmbRows;
+      const unsigned bal = __ballot_sync(0xffffffffu, hit);
+      if (lane == 0) warp_cnt[k & 1][warp] = __popc(bal);
+      __syncthreads();                                       // one barrier per round: the counters are double-buffered
+      int base = nh, tot = 0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) { const int cw = warp_cnt[k & 1][w]; if (w < warp) base += cw; tot += cw; }
+      if (hit) hits[base + __popc(bal & ((1u << lane) - 1u))] = ((tb0 + k * 256 + (int)threadIdx.x) << 8) | rel[k];
+      nh += tot;
+    }
+  }
+  __syncthreads();
+  const int dm = s.d_in;
+  const AT* du = ws_at<AT>(t, s.dh);
+  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const float sc = sqrtf((float)dm);
+  for (int rr = warp; rr < kEmbRows; rr += 8) {
+    const int v = v0 + rr;
+    if (v >= s.vocab) break;
+    float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
+    for (int c0 = 0; c0 < dm; c0 += 32 * 16) {               // up to 16 columns per lane per pass
+      float acc[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+      for (int hb = 0; hb < nh; hb += 32) {
+        const int hv = hb + lane < nh ? hits[hb + lane] : -1;
+        unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
+        while (mine) {
+          const int j = __ffs(mine) - 1;
+          mine &= mine - 1;
+          const uint64_t ro = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm;
+          float val[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {                     // all loads of this token first, then the ordered additions
+            const int c = c0 + e * 32 + lane;
+            val[e] = c < dm ? du_total<AT>(du, gs, ro + c) : 0.f;
+          }
+#pragma unroll
+          for (int e = 0; e < 16; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[e], sc));
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int c = c0 + e * 32 + lane;
+        if (c < dm) out[c] = acc[e];
+      }
     }
   }
 }
 
-int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.row_chunks == 1 ? 2 : 3) : 0) + (t.any_embed ? 1 : 0); }
+int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.ln_fused ? 2 : (t.row_chunks == 1 ? 2 : 3)) : 0) + (t.any_embed ? 1 : 0); }
 
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
-  if (t.any_ln) {
-    dim3 g1((t.T + 7) / 8, t.P), g2((t.max_dim + kLnCols - 1) / kLnCols, t.row_chunks, t.P);
+  if (t.any_ln && t.ln_fused) {
+    if (dtype == PM_F32) e = t.max_ln_dim <= 256 ? launch_ln_fused<float, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<float, 2>(t, stream) : launch_ln_fused<float, 4>(t, stream));
+    else e = t.max_ln_dim <= 256 ? launch_ln_fused<__nv_bfloat16, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<__nv_bfloat16, 2>(t, stream) : launch_ln_fused<__nv_bfloat16, 4>(t, stream));
+    if (e != cudaSuccess) return e;
+  } else if (t.any_ln) {
+    dim3 g1((t.T + 7) / 8, t.n_ln), g2((t.max_ln_dim + kLnCols - 1) / kLnCols, t.row_chunks, t.n_ln);
     if (dtype == PM_F32) { ln_bwd_dx_kernel<float><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<float><<<g2, 256, 0, stream>>>(t); }
     else { ln_bwd_dx_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(t); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (t.row_chunks > 1) {
-      dim3 g3((t.max_dim + 255) / 256, t.P);
+      dim3 g3((t.max_ln_dim + 255) / 256, t.n_ln);
       ln_param_finish_kernel<<<g3, 256, 0, stream>>>(t);
       e = cudaGetLastError();
       if (e != cudaSuccess) return e;
     }
   }
   if (t.any_embed) {
-    dim3 g((t.max_vocab + 7) / 8, t.P);
+    dim3 g((t.max_vocab + kEmbRows - 1) / kEmbRows, t.n_embed);
     const size_t smem = sizeof(int32_t) * (size_t)t.T;
     if (dtype == PM_F32) embed_bwd_kernel<float><<<g, 256, smem, stream>>>(t);
     else embed_bwd_kernel<__nv_bfloat16><<<g, 256, smem, stream>>>(t);
