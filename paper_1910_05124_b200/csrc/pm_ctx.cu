@@ -30,7 +30,8 @@ struct Layout {
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
   uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0, off_colred = 0;
   uint64_t off_ids = 0, off_lnred = 0;
-  std::vector<int32_t> ids;             // [pre | ln | embed | residual] stage lists, P entries each
+  std::vector<int32_t> ids;             // [pre | ln | embed | residual] stage lists, P entries each; then act_start[PM_MAX_LINEARS][P+1]
+  int32_t act_blocks[PM_MAX_LINEARS] = {};
   int32_t n_pre = 0, n_ln = 0, n_embed = 0, n_res = 0, ln_chunks = 0, ln_chunk_rows = 0, max_ln_dim = 0, ln_fused = 1;
   int32_t row_chunks = 1, chunk_rows = 256;
   bool att_tc = false;
@@ -223,7 +224,16 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (s.pre == PRE_EMBED) L.ids[(size_t)2 * P + L.n_embed++] = p;
     if (s.post == POST_RESIDUAL) L.ids[(size_t)3 * P + L.n_res++] = p;
   }
-  L.off_ids = w; w = align_up(w + sizeof(int32_t) * 4 * P, 256);
+  for (int l = 0; l < PM_MAX_LINEARS; ++l) {
+    int32_t acc = 0;
+    for (int p = 0; p < P; ++p) {
+      L.ids.push_back(acc);
+      if (l < L.st[p].n_lin) acc += (L.st[p].lin[l].n_out + 255) / 256;
+    }
+    L.ids.push_back(acc);
+    L.act_blocks[l] = acc;
+  }
+  L.off_ids = w; w = align_up(w + sizeof(int32_t) * L.ids.size(), 256);
   L.ln_chunk_rows = 64;
   L.ln_chunks = (int32_t)((T + L.ln_chunk_rows - 1) / L.ln_chunk_rows);
   L.off_lnred = w; w = align_up(w + (uint64_t)L.n_ln * L.ln_chunks * 2 * L.max_ln_dim * 4, 256);
@@ -421,6 +431,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     t.n_pre = L.n_pre; t.n_ln = L.n_ln; t.n_embed = L.n_embed; t.n_res = L.n_res;
     t.lnred_off = L.off_lnred; t.ln_chunks = L.ln_chunks; t.ln_chunk_rows = L.ln_chunk_rows; t.max_ln_dim = L.max_ln_dim;
     t.ln_fused = L.ln_fused;
+    t.act_start = ids + 4 * P;
+    for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_blocks[l] = L.act_blocks[l];
   }
   if (L.pe_seq > 0) {
     // sinusoidal positions: PE[pos, 2i] = sin(pos / 10000^(2i/d)), PE[pos, 2i+1] = cos(same); double, rounded once to float

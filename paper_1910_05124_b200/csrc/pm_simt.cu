@@ -123,14 +123,56 @@ template <> struct Pair<__nv_bfloat16> {
 
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 
+// rows r, r + 8, ... < r1 of 8 columns: four rows are loaded before the first is used
+template <typename AT, int ACT>
+__device__ __forceinline__ void actbwd_rows(const AT* __restrict__ dy, const AT* __restrict__ z, AT* __restrict__ dz, int n_out, int c,
+                                            int r, int r1, float (&sum)[8]) {
+  for (; r + 3 * kActWarps < r1; r += 4 * kActWarps) {
+    float g[4][8], zz[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = (uint64_t)(r + u * kActWarps) * n_out + c;
+      load8<AT>(dy + i, g[u]);
+      if (ACT != PM_ACT_NONE) load8<AT>(z + i, zz[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (ACT != PM_ACT_NONE) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) g[u][k] = round_as<AT>(__fmul_rn(g[u][k], act_grad(zz[u][k], ACT)));
+        store8<AT>(dz + (uint64_t)(r + u * kActWarps) * n_out + c, g[u]);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) sum[k] = __fadd_rn(sum[k], g[u][k]);
+    }
+  }
+  for (; r < r1; r += kActWarps) {
+    const uint64_t i = (uint64_t)r * n_out + c;
+    float g[8];
+    load8<AT>(dy + i, g);
+    if (ACT != PM_ACT_NONE) {
+      float zz[8];
+      load8<AT>(z + i, zz);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) g[k] = round_as<AT>(__fmul_rn(g[k], act_grad(zz[k], ACT)));
+      store8<AT>(dz + i, g);
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sum[k] = __fadd_rn(sum[k], g[k]);
+  }
+}
+
 template <typename AT>
 __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
-  const int p = blockIdx.z;
+  const int* start = t.act_start + (size_t)lvl * (t.P + 1);
+  int lo = 0, hi = t.P - 1;                                 // stage of this column block: largest p with start[p] <= blockIdx.x
+  while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (start[mid] <= (int)blockIdx.x) lo = mid; else hi = mid - 1; }
+  const int p = lo;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
-  const int c0 = blockIdx.x * kActColsV;
+  const int c0 = ((int)blockIdx.x - start[p]) * kActColsV;
   if (c0 >= L.n_out) return;
   const int chunk = blockIdx.y;
   const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + t.chunk_rows);
@@ -145,23 +187,15 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   AT* dz = ws_ptr<AT>(t, s.dz);
   const bool vec = (L.n_out & 7) == 0;                      // vector path needs 8-element alignment of every row
   float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int r = r0 + warp; r < r1; r += kActWarps) {
-    const uint64_t i = (uint64_t)r * L.n_out + c;
-    if (vec) {
-      if (c < L.n_out) {
-        float g[8];
-        load8<AT>(dy + i, g);
-        if (has_act) {
-          float zz[8];
-          load8<AT>(z + i, zz);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) g[k] = round_as<AT>(__fmul_rn(g[k], act_grad(zz[k], L.act)));
-          store8<AT>(dz + i, g);
-        }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) sum[k] = __fadd_rn(sum[k], g[k]);
-      }
-    } else {
+  if (vec) {
+    if (c < L.n_out) {
+      if (L.act == PM_ACT_NONE) actbwd_rows<AT, PM_ACT_NONE>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      else if (L.act == PM_ACT_RELU) actbwd_rows<AT, PM_ACT_RELU>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      else actbwd_rows<AT, PM_ACT_GELU>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+    }
+  } else {
+    for (int r = r0 + warp; r < r1; r += kActWarps) {
+      const uint64_t i = (uint64_t)r * L.n_out + c;
 #pragma unroll
       for (int k = 0; k < 8; ++k)
         if (c + k < L.n_out) {
@@ -203,7 +237,8 @@ __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
 int actbwd_launches(const TickArgs& t) { return t.row_chunks == 1 ? 1 : 2; }
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
-  dim3 grid((t.max_dim + kActColsV - 1) / kActColsV, t.row_chunks, t.P);
+  if (t.act_blocks[lvl] == 0) return cudaSuccess;
+  dim3 grid(t.act_blocks[lvl], t.row_chunks);
   if (dtype == PM_F32) actbwd_kernel<float><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   cudaError_t e = cudaGetLastError();

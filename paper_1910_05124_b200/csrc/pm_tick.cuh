@@ -33,6 +33,10 @@ struct TickArgs {
   int32_t n_pre, n_ln, n_embed, n_res;
   uint64_t lnred_off;     // ws: LayerNorm parameter-gradient partials [n_ln][ln_chunks][2*max_ln_dim] float
   int32_t ln_chunks, ln_chunk_rows, max_ln_dim;
+  // activation-backward launches: column blocks (256 columns) of Linear `lvl` over all stages, flattened;
+  // act_start[lvl * (P + 1) + p] is the first block of stage p, act_blocks[lvl] the total
+  const int32_t* act_start;
+  int32_t act_blocks[PM_MAX_LINEARS];
   int32_t ln_fused;       // every LayerNorm width is a multiple of 8 and at most 1024: one fused backward kernel
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages

@@ -661,21 +661,31 @@ __global__ void __launch_bounds__(256) ln_bwd_fused_kernel(TickArgs t) {
         for (int k = 0; k < 8; ++k) gb[q][k] = __fsub_rn(gb[q][k], __fmul_rn(gapf, cv[k])); }     // gain - (tau_fwd - tau_bkwd) * delta
     }
   }
+  const bool has_gs = gs != nullptr;
+  if (!has_gs) gs = du;                                      // keeps the loads below free of branches; the value is not used
   for (int r = r0 + warp; r < r1; r += 8) {
     const float mu = st[2 * r], rstd = st[2 * r + 1];
     const uint64_t ro = (uint64_t)r * dm;
     float xh[NP][8], dxh[NP][8];
     float s1 = 0.f, s2 = 0.f;
+    // every load of the row is issued before the first use
+    float xa[NP][8], da[NP][8], sa[NP][8];
+#pragma unroll
+    for (int q = 0; q < NP; ++q) {
+      const int c = min(q * 256 + lane * 8, dm - 8);
+      load8<AT>(x + ro + c, xa[q]);
+      load8<AT>(du + ro + c, da[q]);
+      load8<AT>(gs + ro + c, sa[q]);
+    }
 #pragma unroll
     for (int q = 0; q < NP; ++q) {
       const int c = q * 256 + lane * 8;
       if (c < dm) {
-        float xv[8], dv[8];
-        load8<AT>(x + ro + c, xv);
-        load8<AT>(du + ro + c, dv);
-        if (gs) { float sv[8]; load8<AT>(gs + ro + c, sv);
+        float (&xv)[8] = xa[q];
+        float (&dv)[8] = da[q];
+        if (has_gs) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) dv[k] = __fadd_rn(dv[k], sv[k]); }
+          for (int k = 0; k < 8; ++k) dv[k] = __fadd_rn(dv[k], sa[q][k]); }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           xh[q][k] = (xv[k] - mu) * rstd;
@@ -815,11 +825,18 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
           const int j = __ffs(mine) - 1;
           mine &= mine - 1;
           const uint64_t ro = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm;
-          float val[16];
+          // all loads of this token first (no branch between them), then the ordered additions
+          float val[16], sv[16];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {                     // all loads of this token first, then the ordered additions
-            const int c = c0 + e * 32 + lane;
-            val[e] = c < dm ? du_total<AT>(du, gs, ro + c) : 0.f;
+          for (int e = 0; e < 16; ++e) {
+            const int c = min(c0 + e * 32 + lane, dm - 1);
+            val[e] = to_f<AT>(du[ro + c]);
+          }
+          if (gs) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) sv[e] = to_f<AT>(gs[ro + min(c0 + e * 32 + lane, dm - 1)]);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) val[e] = __fadd_rn(val[e], sv[e]);
           }
 #pragma unroll
           for (int e = 0; e < 16; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[e], sc));
