@@ -230,7 +230,15 @@ __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
   if (c >= L.n_out) return;
   const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * (2 * (uint64_t)t.max_dim) + c;
   float sum = 0.f;
-  for (int k = 0; k < t.row_chunks; ++k) sum = __fadd_rn(sum, part[(uint64_t)k * 2 * t.max_dim]);
+  int k = 0;
+  for (; k + 8 <= t.row_chunks; k += 8) {                   // eight partials in flight, added in chunk order
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = part[(uint64_t)(k + u) * 2 * t.max_dim];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
+  }
+  for (; k < t.row_chunks; ++k) sum = __fadd_rn(sum, part[(uint64_t)k * 2 * t.max_dim]);
   t.a.grad[L.b_off + c] = sum;
 }
 

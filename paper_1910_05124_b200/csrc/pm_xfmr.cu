@@ -139,7 +139,20 @@ __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
   AT* out = ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
   // buffers start on 256-byte boundaries and slots are n elements apart: groups of eight are aligned when 8 | n
   const uint64_t n8 = (n % 8 == 0) ? n / 8 : 0;
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < n8; i += 4 * stride) {            // four groups of eight in flight per thread
+    float a[4][8], b[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { load8<AT>(skip + 8 * (i + u * stride), a[u]); load8<AT>(y + 8 * (i + u * stride), b[u]); }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) a[u][j] = __fadd_rn(a[u][j], b[u][j]);
+      store8<AT>(out + 8 * (i + u * stride), a[u]);
+    }
+  }
+  for (; i < n8; i += stride) {
     float a[8], b[8];
     load8<AT>(skip + 8 * i, a);
     load8<AT>(y + 8 * i, b);
@@ -742,9 +755,18 @@ __global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
   if (c >= s.d_in) return;
   const float* part = ws_at<float>(t, t.lnred_off) + (uint64_t)li * t.ln_chunks * (2 * (uint64_t)t.max_ln_dim);
   float a = 0.f, b2 = 0.f;
-  for (int k = 0; k < t.ln_chunks; ++k) {
-    a = __fadd_rn(a, part[(uint64_t)k * 2 * t.max_ln_dim + c]);
-    b2 = __fadd_rn(b2, part[(uint64_t)k * 2 * t.max_ln_dim + t.max_ln_dim + c]);
+  const uint64_t ps = 2 * (uint64_t)t.max_ln_dim;
+  int k = 0;
+  for (; k + 8 <= t.ln_chunks; k += 8) {                    // eight partials in flight, added in chunk order
+    float va[8], vb[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { va[u] = part[(uint64_t)(k + u) * ps + c]; vb[u] = part[(uint64_t)(k + u) * ps + t.max_ln_dim + c]; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { a = __fadd_rn(a, va[u]); b2 = __fadd_rn(b2, vb[u]); }
+  }
+  for (; k < t.ln_chunks; ++k) {
+    a = __fadd_rn(a, part[(uint64_t)k * ps + c]);
+    b2 = __fadd_rn(b2, part[(uint64_t)k * ps + t.max_ln_dim + c]);
   }
   t.a.grad[s.g_off + c] = a;
   t.a.grad[s.beta_off + c] = b2;
