@@ -1,22 +1,32 @@
-"""Pipeline of Transformer-encoder stages with a cross-entropy loss: grad f_t(u_fwd, u_bkwd).
+"""Pipeline of Transformer stages (encoder, or encoder-decoder) with a cross-entropy loss: grad f_t(u_fwd, u_bkwd).
 
 TEST INFRASTRUCTURE (see package docstring).
 
 Every stage holds exactly one weight matrix ("one stage per weight GEMM") and has the shape
 
-    pre   : 'embed' (token embedding * sqrt(d) + sinusoidal positions) | 'ln' (LayerNorm) | 'none'
-    linear: z = u W^T + b ;  y = act(z)
-    post  : 'attention' (split y into q, k, v; multi-head self-attention; also hands u on as a skip tensor)
+    pre   : 'embed' (token embedding * sqrt(d) + sinusoidal positions; source ids)
+            'embed_dec' (the same with the decoder's input ids) | 'ln' (LayerNorm) | 'none'
+    linear: z = u W^T + b ;  y = act(z);  u comes from the main stream, or (src == 'memory') from the
+            encoder output, which every such stage normalises with its own LayerNorm
+    post  : 'attention' (split y into q, k, v; multi-head self-attention, causal if spec.causal; also hands u
+                         on as a skip tensor)
+            'cross_attention' (the main input is q; y is split into k, v; attention of q over k, v)
             'skip_out'  (hands u on as a skip tensor next to y)
-            'residual'  (adds the skip tensor received from the previous stage to y)
+            'residual'  (adds the skip tensor it was sent to y)
             'none'
+    A skip tensor goes to the stage spec.skip_hop (default 1) positions on.  The stage with spec.emit_memory
+    (the last encoder stage) also publishes its output as the memory the decoder's cross-attention stages read.
 
 A post-LN encoder layer is four stages: [ln|embed, W_qkv, attention] [W_o, residual] [ln, W_1 + ReLU, skip_out]
+[W_2, residual]; a decoder layer is seven: [ln|embed_dec, W_qkv, causal attention] [W_o, residual]
+[ln, W_q, skip_out over two] [ln(memory), W_kv, cross_attention] [W_o, residual] [ln, W_1 + ReLU, skip_out]
 [W_2, residual]; the last stage is [ln, W_vocab] followed by the loss.  Parameters of a stage in order:
 [table] (embed), [gain, bias] (ln), W, b.
 
 The backward pass reads u_bkwd in exactly two places (Section 2.1: the weights "used in the backward pass"):
-the Linear matrix of the input-gradient product and the LayerNorm gain of dx_hat = dy * gain.
+the Linear matrix of the input-gradient product and the LayerNorm gain of dx_hat = dy * gain.  The gradients
+the cross-attention stages send to the encoder output are added in descending stage order (the order in which a
+pipeline produces them), each partial sum in operand precision.
 
 Parity of whole training trajectories is unpinned by the paper; this module is pinned through finite
 differences of the complete model (u_fwd = u_bkwd) and the layer-level library cross-checks.
@@ -36,7 +46,7 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
     def unpack(spec, tensors):
         i = 0
         out = {}
-        if spec.pre == "embed":
+        if spec.pre in ("embed", "embed_dec"):
             out["table"] = f64(tensors[i]); i += 1
         if spec.pre == "ln":
             out["gain"], out["beta"] = f64(tensors[i]), f64(tensors[i + 1]); i += 2
@@ -44,20 +54,27 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
         return out
 
     def grad_fn(t, u_fwd, u_bkwd):
-        ids, targets = data_fn(t)
+        data = data_fn(t)
+        ids, targets = data[0], data[-1]
+        dec_ids = data[1] if len(data) == 3 else None
         P = len(stage_specs)
-        main, skip = None, None
+        main, memory = None, None
+        skip_for = {}                                          # receiving stage -> (skip tensor, emitting stage)
         stash = []
         logits = None
         for i, spec in enumerate(stage_specs):
             pf = unpack(spec, u_fwd[i])
             st = {}
+            from_memory = getattr(spec, "src", "main") == "memory"
+            x_in = memory if from_memory else main
             if spec.pre == "embed":
                 u = L.embed_fwd(ids, pf["table"], seq_len, rnd)
+            elif spec.pre == "embed_dec":
+                u = L.embed_fwd(dec_ids, pf["table"], seq_len, rnd)
             elif spec.pre == "ln":
-                u, st["xhat"], st["rstd"] = L.layernorm_fwd(main, pf["gain"], pf["beta"], rnd)
+                u, st["xhat"], st["rstd"] = L.layernorm_fwd(x_in, pf["gain"], pf["beta"], rnd)
             else:
-                u = main
+                u = x_in
             st["u"] = u
             acc = u @ rnd(pf["W"]).T + pf["b"]
             if i == P - 1:
@@ -67,46 +84,63 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
             z = rnd(acc)
             y = rnd(L.act_fwd(z, spec.act))
             st["z"] = z
+            hop = getattr(spec, "skip_hop", 1)
             if spec.post == "attention":
                 d = y.shape[1] // 3
                 st["q"], st["k"], st["v"] = y[:, :d], y[:, d:2 * d], y[:, 2 * d:]
-                main, skip = L.attention_fwd(st["q"], st["k"], st["v"], n_heads, seq_len, False, rnd), u
+                main = L.attention_fwd(st["q"], st["k"], st["v"], n_heads, seq_len, getattr(spec, "causal", False), rnd)
+                skip_for[i + hop] = (u, i)
+            elif spec.post == "cross_attention":
+                d = y.shape[1] // 2
+                st["q"], st["k"], st["v"] = main, y[:, :d], y[:, d:]
+                main = L.attention_fwd(st["q"], st["k"], st["v"], n_heads, seq_len, False, rnd)
             elif spec.post == "skip_out":
-                main, skip = y, u
+                main = y
+                skip_for[i + hop] = (u, i)
             elif spec.post == "residual":
-                main, skip = rnd(skip + y), None
+                sk, st["skip_src"] = skip_for.pop(i)
+                main = rnd(sk + y)
             else:
-                main, skip = y, None
+                main = y
+            if getattr(spec, "emit_memory", False):
+                memory = main
             stash.append(st)
 
         loss, d_main = L.cross_entropy(logits, targets, rnd)
-        d_skip = None
+        d_skip_for = {}                                        # emitting stage -> gradient of the skip tensor it sent
+        d_memory = None
         grads = [[None] * len(u_fwd[i]) for i in range(P)]
         for i in reversed(range(P)):
             spec, st = stage_specs[i], stash[i]
             pb = unpack(spec, u_bkwd[i])
-            du_extra, d_in_skip = None, None
+            from_memory = getattr(spec, "src", "main") == "memory"
+            if getattr(spec, "emit_memory", False):
+                d_main = d_memory                              # the following stage embeds its own ids: no gradient from it
+            d_prev_main = None                                 # gradient handed to the previous stage besides d_in
             if i == P - 1:
                 dz = d_main                                     # dlogits, already in operand precision
             else:
                 if spec.post == "attention":
+                    dq, dk, dv = L.attention_bwd(d_main, st["q"], st["k"], st["v"], n_heads, seq_len,
+                                                 getattr(spec, "causal", False), rnd)
+                    dy = np.concatenate([dq, dk, dv], axis=1)
+                elif spec.post == "cross_attention":
                     dq, dk, dv = L.attention_bwd(d_main, st["q"], st["k"], st["v"], n_heads, seq_len, False, rnd)
-                    dy, du_extra = np.concatenate([dq, dk, dv], axis=1), d_skip
-                elif spec.post == "skip_out":
-                    dy, du_extra = d_main, d_skip
+                    dy, d_prev_main = np.concatenate([dk, dv], axis=1), dq
                 elif spec.post == "residual":
-                    dy, d_in_skip = d_main, d_main
+                    dy = d_main
+                    d_skip_for[st["skip_src"]] = d_main
                 else:
                     dy = d_main
                 dz = rnd(dy * L.act_grad(st["z"], spec.act))
             dW = dz.T @ st["u"]
             db = dz.sum(axis=0)
             du = rnd(dz @ rnd(pb["W"]))
-            if du_extra is not None:
-                du = du + du_extra
+            if i in d_skip_for:
+                du = du + d_skip_for.pop(i)
             g = []
-            if spec.pre == "embed":
-                g.append(L.embed_bwd(du, ids, vocab))
+            if spec.pre in ("embed", "embed_dec"):
+                g.append(L.embed_bwd(du, ids if spec.pre == "embed" else dec_ids, vocab))
                 d_in = None
             elif spec.pre == "ln":
                 d_in, dgain, dbeta = L.layernorm_bwd(du, st["xhat"], st["rstd"], pb["gain"], rnd)
@@ -115,7 +149,11 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
                 d_in = du
             g += [dW, db]
             grads[i] = g
-            d_main, d_skip = d_in, d_in_skip
+            if from_memory:
+                d_memory = d_in if d_memory is None else rnd(d_memory + d_in)
+                d_main = d_prev_main
+            else:
+                d_main = d_in
         return loss, grads
 
     return grad_fn

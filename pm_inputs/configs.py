@@ -32,11 +32,15 @@ class LinearSpec:
 @dataclass
 class StageSpec:
     """One Transformer stage: pre-op, one Linear, post-op (see the encoder workload below)."""
-    pre: str        # 'embed' | 'ln' | 'none'
+    pre: str        # 'embed' | 'embed_dec' | 'ln' | 'none'
     n_in: int
     n_out: int
     act: str        # 'relu' | 'gelu' | 'none'
-    post: str       # 'attention' | 'skip_out' | 'residual' | 'none'
+    post: str       # 'attention' | 'cross_attention' | 'skip_out' | 'residual' | 'none'
+    src: str = "main"           # the Linear reads the main stream, or 'memory' (the encoder output)
+    causal: bool = False        # 'attention': keys after the query are masked
+    skip_hop: int = 1           # the skip tensor this stage emits goes to the stage skip_hop positions on
+    emit_memory: bool = False   # the stage's output is also the memory of the cross-attention stages
 
 
 @dataclass
@@ -243,14 +247,69 @@ def cfg4_small(compute="bf16", n_layers=2, d_model=64, n_heads=2, d_ff=128, seq_
                             steps=steps, seed=191005124 + 44)
 
 
+def encdec_workload(name, n_enc, n_dec, d_model, n_heads, d_ff, seq_len, batch, vocab, **kw):
+    """Post-LN encoder-decoder, one stage per weight matrix.  Encoder layers as in encoder_workload; the last
+    encoder stage also publishes the memory.  A decoder layer is seven stages: [W_qkv + causal attention]
+    [W_o + residual] [LN, W_q, skip over two stages] [LN(memory), W_kv + cross-attention] [W_o + residual]
+    [LN, W_1 + ReLU] [W_2 + residual]; the decoder's first stage embeds the decoder input (the target shifted
+    right behind a begin-of-sequence id 0); the vocabulary projection with the final LayerNorm is the last stage.
+    Source and target sequences have the same length."""
+    specs = []
+    for layer in range(n_enc):
+        specs.append(StageSpec("embed" if layer == 0 else "ln", d_model, 3 * d_model, "none", "attention"))
+        specs.append(StageSpec("none", d_model, d_model, "none", "residual"))
+        specs.append(StageSpec("ln", d_model, d_ff, "relu", "skip_out"))
+        specs.append(StageSpec("none", d_ff, d_model, "none", "residual", emit_memory=(layer == n_enc - 1)))
+    for layer in range(n_dec):
+        specs.append(StageSpec("embed_dec" if layer == 0 else "ln", d_model, 3 * d_model, "none", "attention", causal=True))
+        specs.append(StageSpec("none", d_model, d_model, "none", "residual"))
+        specs.append(StageSpec("ln", d_model, d_model, "none", "skip_out", skip_hop=2))
+        specs.append(StageSpec("ln", d_model, 2 * d_model, "none", "cross_attention", src="memory"))
+        specs.append(StageSpec("none", d_model, d_model, "none", "residual"))
+        specs.append(StageSpec("ln", d_model, d_ff, "relu", "skip_out"))
+        specs.append(StageSpec("none", d_ff, d_model, "none", "residual"))
+    specs.append(StageSpec("ln", d_model, vocab, "none", "none"))
+    P = len(specs)
+    fwd, bkwd = pipemare_delays(P)
+    return Workload(name=name, stages=[], tau_fwd=fwd, tau_bkwd=bkwd, microbatch=batch * seq_len, kind="encoder",
+                    stage_specs=specs, n_heads=n_heads, seq_len=seq_len, vocab=vocab, d_model=d_model, **kw)
+
+
+def cfg5():
+    """Encoder-decoder, 12 + 12 layers, d_model 1024, 16 heads, FFN 4096, sequence 256, microbatch 16 sequences,
+    vocabulary 32000, bf16 GEMMs; source ids Zipf(1.1), target = a fixed seeded permutation of the source ids;
+    Adam(0.9, 0.98), alpha 7e-4, K = 1000, D = 0.1; 48 + 84 + 1 = 133 stages."""
+    return encdec_workload("cfg5_encdec12_bf16", 12, 12, 1024, 16, 4096, 256, 16, 32000, compute="bf16", optimizer="adam",
+                           alpha=7e-4, beta1=0.9, beta2=0.98, eps=1e-8, K=1000, D=0.1, steps=1200, seed=191005124 + 5)
+
+
+def cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=64, n_heads=2, d_ff=128, seq_len=16, batch=3, vocab=96, steps=24):
+    """Same structure as cfg5 at a size the oracle runs in seconds."""
+    return encdec_workload("cfg5_small", n_enc, n_dec, d_model, n_heads, d_ff, seq_len, batch, vocab, compute=compute,
+                           optimizer="adam", alpha=7e-4, beta1=0.9, beta2=0.98, eps=1e-8, K=max(steps // 3, 1), D=0.1,
+                           steps=steps, seed=191005124 + 55)
+
+
+def seq2seq_batch(wl, t):
+    """Microbatch t of an encoder-decoder workload: (source ids, decoder input ids, target ids), each [batch*seq_len].
+    Source ids are Zipf(1.1)-distributed ranks; the target is pi(source) for a permutation pi of the vocabulary fixed
+    by the workload's seed; the decoder input is the target shifted right by one position behind id 0."""
+    n_seq = wl.microbatch // wl.seq_len
+    src = rng.zipf_ranks(wl.seed, _S_TOKENS + 16 * t, wl.microbatch, wl.vocab, 1.1).reshape(n_seq, wl.seq_len)
+    order = np.argsort(rng.uniform01(wl.seed, _S_TOKENS + 5, wl.vocab), kind="stable")   # the permutation pi
+    tgt = order[src]
+    dec_in = np.concatenate([np.zeros((n_seq, 1), dtype=np.int64), tgt[:, :-1]], axis=1)
+    return src.reshape(-1).astype(np.int64), dec_in.reshape(-1).astype(np.int64), tgt.reshape(-1).astype(np.int64)
+
+
 def init_encoder_params(wl):
     """Per stage the tensors [table] [gain, bias] W b (float32): W ~ N(0, 1/fan_in), table ~ N(0, 1/d_model),
     biases 0, LayerNorm gain 1 and bias 0."""
     out = []
     for i, sp in enumerate(wl.stage_specs):
         tensors = []
-        if sp.pre == "embed":
-            e = rng.normal(wl.seed, _S_ENC_INIT + 7, wl.vocab * wl.d_model) / np.sqrt(wl.d_model)
+        if sp.pre in ("embed", "embed_dec"):
+            e = rng.normal(wl.seed, _S_ENC_INIT + (7 if sp.pre == "embed" else 8), wl.vocab * wl.d_model) / np.sqrt(wl.d_model)
             tensors.append(e.reshape(wl.vocab, wl.d_model).astype(np.float32))
         if sp.pre == "ln":
             tensors += [np.ones(sp.n_in, dtype=np.float32), np.zeros(sp.n_in, dtype=np.float32)]
