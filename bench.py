@@ -346,9 +346,9 @@ NCU_TRAFFIC = {
     # GEMM kernels: measured DRAM bytes / algorithmic bytes on the 2-layer cut of cfg4
     # (profiles/gemm_and_attention_kernels_cfg4_2layer_cut.md); every operand crosses HBM once, so traffic grows
     # with the algorithmic bytes of the launch
-    "gemm_fwd_ratio": (84.1 + 183.3) / (83.9 + 243.0),
-    "wgrad_ratio": (211.5 + 24.6) / (205.5 + 42.0),
-    "dgrad_ratio": (232.4 + 45.9) / (226.5 + 33.6),
+    "gemm_fwd_ratio": (84.3 + 182.4) / (83.9 + 243.0),
+    "wgrad_ratio": (210.9 + 23.0) / (205.5 + 42.0),
+    "dgrad_ratio": (232.3 + 30.4) / (226.5 + 33.6),
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
@@ -461,8 +461,9 @@ def rooflines(res, hbm_peak, tf_peak, peak_kind, steps):
     if dominant in flops:
         launches = res["prof"][dominant][1] / steps
         tfs = flops[dominant] / (per_tick[dominant] * 1e-3) / 1e12
-        names = {"gemm_fwd": "umma_gemm_kernel<0> (forward GEMMs)", "wgrad": "umma_gemm_kernel<2> (wgrad GEMMs)",
-                 "dgrad": "umma_dgrad_kernel (dgrad GEMMs, weights corrected while loading)"}
+        names = {"gemm_fwd": "umma_pair_gemm_kernel<0> / umma_gemm_kernel<0> (forward GEMMs)",
+                 "wgrad": "umma_pair_gemm_kernel<2> / umma_gemm_kernel<2> (wgrad GEMMs)",
+                 "dgrad": "umma_dgrad_pair_kernel / umma_dgrad_kernel (dgrad GEMMs, weights corrected while loading)"}
         dom = {"kernel": names[dominant], "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
                "frac": round(tfs / tf_peak, 4), "of": peak_kind + " (sustained bf16 matmul)",
                "traffic": int(NCU_TRAFFIC[dominant + "_ratio"] * gemm_bytes(wl)[dominant] / launches),
