@@ -47,7 +47,15 @@ enum { PM_F32 = 0, PM_BF16 = 1 };                 /* GEMM operand type; state is
 enum { PM_SGDM = 0, PM_ADAM = 1 };
 enum { PM_ACT_NONE = 0, PM_ACT_RELU = 1, PM_ACT_GELU = 2 };   /* GELU = exact erf form      */
 enum { PM_OP_LINEAR = 0, PM_OP_EMBED = 1, PM_OP_LAYERNORM = 2, PM_OP_ATTENTION = 3, PM_OP_SKIP_OUT = 4,
-       PM_OP_RESIDUAL = 5 };
+       PM_OP_RESIDUAL = 5, PM_OP_CROSS_ATTENTION = 6 };
+/* pm_op_desc.flags */
+enum { PM_OPF_CAUSAL = 1,          /* ATTENTION: keys after the query position are masked                        */
+       PM_OPF_FROM_MEMORY = 2,     /* LAYERNORM: normalises the memory (see RESIDUAL) instead of the main input; the
+                                      stage's Linear reads that, the main input goes to the post-op               */
+       PM_OPF_SECOND_STREAM = 4,   /* EMBED: embeds the second token stream (the decoder input)                   */
+       PM_OPF_EMIT_MEMORY = 8,     /* RESIDUAL: the stage's output is the memory (the encoder output); the next
+                                      stage must start with EMBED | PM_OPF_SECOND_STREAM                          */
+       PM_OPF_SKIP_TWO = 16 };     /* SKIP_OUT: the skip tensor goes to the stage two positions on                */
 enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
 
 /* Alignment, in elements, of every stage slice and of every tensor inside it. */
@@ -59,21 +67,29 @@ enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
  * RESIDUAL]  (with a pre- or post-op exactly one LINEAR).
  *   LINEAR     y = act(x W^T + b), W is [n_out, n_in] row-major, b is [n_out].
  *   EMBED      x = table[id] * sqrt(n_out) + sinusoidal position; table is [n_in = vocabulary, n_out = width];
- *              first stage only; the stage's input is then int32 token ids.  seq_len gives the position period.
+ *              the stage's input is int32 token ids: the first stage embeds the first stream; a later stage with
+ *              PM_OPF_SECOND_STREAM (the first stage of a decoder) embeds the second and ignores the previous
+ *              stage's output.  seq_len gives the position period.
  *   LAYERNORM  over the last dimension (n_in = n_out = width), eps 1e-5, biased variance; parameters gain, bias.
  *   ATTENTION  splits the Linear's output [T, 3d] into q, k, v; softmax(q k^T / sqrt(d / n_heads)) v per head and
  *              per sequence of seq_len rows (T a multiple of seq_len, seq_len <= 128); the stage hands o [T, d]
  *              and, as a skip tensor, the Linear's input to the next stage, which must end in RESIDUAL.
  *   SKIP_OUT   hands the Linear's input on as a skip tensor next to its output; next stage must end in RESIDUAL.
- *   RESIDUAL   adds the skip tensor received from the previous stage to the Linear's output.
+ *   RESIDUAL   adds the skip tensor it was sent to the Linear's output.
+ *   CROSS_ATTENTION  the stage starts with LAYERNORM | PM_OPF_FROM_MEMORY; the Linear's output [T, 2d] is k, v, the
+ *              stage's main input [T, d] is q; attention of q over k, v per head and sequence (source and target
+ *              sequences have the same length seq_len); o [T, d] goes to the next stage.  A skip tensor sent with
+ *              PM_OPF_SKIP_TWO by the previous stage passes over this one.  The gradients the memory receives
+ *              from the cross-attention stages are added in descending stage order (Section 2.1 fixes no order).
  * Where the backward pass reads a parameter value it reads the T2-corrected one (Section 3.2): the Linear
  * matrix in the input-gradient product and the LayerNorm gain.  Nothing else is read in the backward pass. */
 typedef struct {
   int32_t kind;            /* PM_OP_* */
   int32_t n_in, n_out;
   int32_t act;             /* PM_ACT_* (LINEAR) */
-  int32_t n_heads;         /* ATTENTION */
-  int32_t seq_len;         /* ATTENTION, EMBED */
+  int32_t n_heads;         /* ATTENTION, CROSS_ATTENTION */
+  int32_t seq_len;         /* ATTENTION, CROSS_ATTENTION, EMBED */
+  int32_t flags;           /* PM_OPF_* */
 } pm_op_desc;
 
 /* One pipeline stage (Section 2.1).  Copied during pm_init_stages.
@@ -165,7 +181,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
 /* One tick = pm_forward, pm_backward, pm_update in this order (pm_step does all three).
  * inputs/targets (device) belong to the microbatch that enters the pipeline at this tick:
  * inputs is [T, n_in of stage 1] (float for PM_F32, bfloat16 for PM_BF16), or [T] int32 token ids when
- * stage 1 starts with EMBED; targets is [T, n_out of stage P] float (PM_LOSS_MSE) or [T] int32 class ids
+ * stage 1 starts with EMBED ([2][T]: first stream, then second stream, when a stage embeds the second
+ * stream); targets is [T, n_out of stage P] float (PM_LOSS_MSE) or [T] int32 class ids
  * (PM_LOSS_CE).  Both are copied before the call returns control to the
  * stream order, so the caller may overwrite them after any later call on the same stream.
  * Pass NULL for both to drain: N microbatches need N + 2P - 1 ticks.

@@ -14,6 +14,8 @@ PM_F32, PM_BF16 = 0, 1
 PM_SGDM, PM_ADAM = 0, 1
 PM_ACT_NONE, PM_ACT_RELU, PM_ACT_GELU = 0, 1, 2
 PM_OP_LINEAR, PM_OP_EMBED, PM_OP_LAYERNORM, PM_OP_ATTENTION, PM_OP_SKIP_OUT, PM_OP_RESIDUAL = 0, 1, 2, 3, 4, 5
+PM_OP_CROSS_ATTENTION = 6
+PM_OPF_CAUSAL, PM_OPF_FROM_MEMORY, PM_OPF_SECOND_STREAM, PM_OPF_EMIT_MEMORY, PM_OPF_SKIP_TWO = 1, 2, 4, 8, 16
 PM_LOSS_MSE, PM_LOSS_CE = 0, 1
 PM_ALIGN_ELEMS = 64
 
@@ -24,7 +26,7 @@ LIB_PATH = os.path.join(_HERE, "libpipemare.so")
 
 class pm_op_desc(C.Structure):
     _fields_ = [("kind", C.c_int32), ("n_in", C.c_int32), ("n_out", C.c_int32), ("act", C.c_int32),
-                ("n_heads", C.c_int32), ("seq_len", C.c_int32)]
+                ("n_heads", C.c_int32), ("seq_len", C.c_int32), ("flags", C.c_int32)]
 
 
 class pm_stage_desc(C.Structure):
@@ -134,6 +136,7 @@ def _ops_from_dicts(ops):
     for j, o in enumerate(ops):
         arr[j].kind, arr[j].n_in, arr[j].n_out = o["kind"], o.get("n_in", 0), o.get("n_out", 0)
         arr[j].act, arr[j].n_heads, arr[j].seq_len = o.get("act", 0), o.get("n_heads", 0), o.get("seq_len", 0)
+        arr[j].flags = o.get("flags", 0)
     return arr
 
 
@@ -142,21 +145,26 @@ def stage_ops(wl, p):
     if getattr(wl, "kind", "mlp") == "encoder":
         sp = wl.stage_specs[p]
         ops, tensors = [], []
-        if sp.pre == "embed":
-            ops.append(dict(kind=PM_OP_EMBED, n_in=wl.vocab, n_out=wl.d_model, seq_len=wl.seq_len))
+        if sp.pre in ("embed", "embed_dec"):
+            ops.append(dict(kind=PM_OP_EMBED, n_in=wl.vocab, n_out=wl.d_model, seq_len=wl.seq_len,
+                            flags=PM_OPF_SECOND_STREAM if sp.pre == "embed_dec" else 0))
             tensors.append((0, 0, (wl.vocab, wl.d_model)))
         elif sp.pre == "ln":
-            ops.append(dict(kind=PM_OP_LAYERNORM, n_in=sp.n_in, n_out=sp.n_in))
+            ops.append(dict(kind=PM_OP_LAYERNORM, n_in=sp.n_in, n_out=sp.n_in,
+                            flags=PM_OPF_FROM_MEMORY if getattr(sp, "src", "main") == "memory" else 0))
             tensors += [(0, 0, (sp.n_in,)), (0, 1, (sp.n_in,))]
         li = len(ops)
         ops.append(dict(kind=PM_OP_LINEAR, n_in=sp.n_in, n_out=sp.n_out, act=_ACT[sp.act]))
         tensors += [(li, 0, (sp.n_out, sp.n_in)), (li, 1, (sp.n_out,))]
         if sp.post == "attention":
-            ops.append(dict(kind=PM_OP_ATTENTION, n_in=sp.n_out, n_out=sp.n_out // 3, n_heads=wl.n_heads, seq_len=wl.seq_len))
+            ops.append(dict(kind=PM_OP_ATTENTION, n_in=sp.n_out, n_out=sp.n_out // 3, n_heads=wl.n_heads, seq_len=wl.seq_len,
+                            flags=PM_OPF_CAUSAL if getattr(sp, "causal", False) else 0))
+        elif sp.post == "cross_attention":
+            ops.append(dict(kind=PM_OP_CROSS_ATTENTION, n_in=sp.n_out, n_out=sp.n_out // 2, n_heads=wl.n_heads, seq_len=wl.seq_len))
         elif sp.post == "skip_out":
-            ops.append(dict(kind=PM_OP_SKIP_OUT))
+            ops.append(dict(kind=PM_OP_SKIP_OUT, flags=PM_OPF_SKIP_TWO if getattr(sp, "skip_hop", 1) == 2 else 0))
         elif sp.post == "residual":
-            ops.append(dict(kind=PM_OP_RESIDUAL))
+            ops.append(dict(kind=PM_OP_RESIDUAL, flags=PM_OPF_EMIT_MEMORY if getattr(sp, "emit_memory", False) else 0))
         return ops, tensors
     ops, tensors = [], []
     for j, sp in enumerate(wl.stages[p]):

@@ -8,7 +8,7 @@
 namespace pm {
 
 enum { PRE_NONE = 0, PRE_EMBED = 1, PRE_LN = 2 };
-enum { POST_NONE = 0, POST_ATTENTION = 1, POST_SKIP_OUT = 2, POST_RESIDUAL = 3 };
+enum { POST_NONE = 0, POST_ATTENTION = 1, POST_SKIP_OUT = 2, POST_RESIDUAL = 3, POST_CROSS_ATTENTION = 4 };
 enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4 };
 
 // Static description of one Linear inside a stage (device copy).
@@ -32,6 +32,15 @@ struct StageDev {
   int32_t n_heads, seq_len, vocab;
   int32_t d_in;               // width of the main input (= width of u, the first Linear's input)
   int32_t d_out_main;         // width of the main output handed to the next stage
+  int32_t causal;             // attention: keys after the query are masked
+  int32_t skip_hop;           // emitting stage: the skip tensor goes to stage p + skip_hop (0: emits none)
+  int32_t skip_depth;         // receiving stage: slots of skip_in = hop + 1, slot = writer's tick % skip_depth
+  int32_t gin_depth;          // slots of gin: 3, or 4 when a stage two positions back reads it as its skip gradient
+  int32_t from_memory;        // LayerNorm input (and its backward output) is the memory, not the main stream
+  int32_t emit_memory;        // residual stage whose output is the memory; its incoming gradient is the memory gradient
+  int32_t mem_first;          // from_memory stage that runs its backward first (the last one): it stores, the others add
+  int32_t ids_stream;         // embedding: which input stream (0, 1)
+  int32_t ids_depth;          // embedding: slots of ids_ring, slot = microbatch % ids_depth
   int32_t _pad;
   uint64_t begin, end;        // padded element range of the stage's parameters in the arenas
   uint64_t tab_off, g_off, beta_off;   // arena offsets: embedding table / LayerNorm gain / LayerNorm bias
@@ -89,6 +98,9 @@ __device__ __forceinline__ float act_grad(float z, int act) {
     return 0.5f * (1.0f + erff(z * 0.70710678118654752440f)) + z * expf(-0.5f * z * z) * 0.39894228040143267794f;
   return 1.0f;
 }
+
+// the stage's last Linear feeds an attention op (its output is the q, k, v stash; its gradient comes from s.dy)
+__host__ __device__ __forceinline__ bool feeds_attention(int post) { return post == POST_ATTENTION || post == POST_CROSS_ATTENTION; }
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }

@@ -29,7 +29,9 @@ struct Layout {
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
   uint64_t off_loss = 0, off_tgt = 0, off_yout = 0, off_umma = 0, off_lossred = 0, off_pe = 0, off_rowloss = 0, off_attn = 0, off_colred = 0;
-  uint64_t off_ids = 0, off_lnred = 0;
+  uint64_t off_ids = 0, off_lnred = 0, mem_ring = 0, off_gmem = 0;
+  int32_t mem_stage = -1, last_mem_reader = -1, mem_dim = 0, mem_depth = 0, gmem_depth = 0, n_streams = 1;
+  bool att_plain = true;
   std::vector<int32_t> ids;             // [pre | ln | embed | residual] stage lists, P entries each; then act_start[PM_MAX_LINEARS][P+1]
   int32_t act_blocks[PM_MAX_LINEARS] = {};
   int32_t n_pre = 0, n_ln = 0, n_embed = 0, n_res = 0, ln_chunks = 0, ln_chunk_rows = 0, max_ln_dim = 0, ln_fused = 1;
@@ -96,8 +98,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     s.pre = PRE_NONE; s.post = POST_NONE; s.n_lin = 0;
     auto offsets = [&](int op, uint64_t* a, uint64_t* b) { pm_op_param_offsets(sd.ops, sd.n_ops, op, a, b); *a += s.begin; *b += s.begin; };
     if (sd.ops[0].kind == PM_OP_EMBED) {
-      if (p != 0) { stage_err(p, "EMBED belongs to the first stage"); return PM_ERR_UNSUPPORTED; }
       const pm_op_desc& op = sd.ops[0];
+      const bool second = (op.flags & PM_OPF_SECOND_STREAM) != 0;
+      if ((p == 0) == second) { stage_err(p, "EMBED belongs to the first stage (first stream) or, with PM_OPF_SECOND_STREAM, to a later one"); return PM_ERR_UNSUPPORTED; }
+      if (second && !L.st[p - 1].emit_memory) { stage_err(p, "a second-stream EMBED must follow the stage that emits the memory"); return PM_ERR_UNSUPPORTED; }
+      if (L.pe_seq > 0 && (L.pe_seq != op.seq_len || L.pe_d != op.n_out)) { stage_err(p, "all EMBED ops share seq_len and width"); return PM_ERR_UNSUPPORTED; }
+      s.ids_stream = second ? 1 : 0;
+      s.ids_depth = 2 * P - p;
+      if (second) L.n_streams = 2;
       if (op.n_in < 1 || op.n_out < 2 || (op.n_out & 1) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (even width, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
       s.pre = PRE_EMBED; s.vocab = op.n_in; s.seq_len = op.seq_len;
       uint64_t dummy; offsets(0, &s.tab_off, &dummy);
@@ -106,6 +114,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     } else if (sd.ops[0].kind == PM_OP_LAYERNORM) {
       if (sd.ops[0].n_in < 1 || sd.ops[0].n_in != sd.ops[0].n_out) { stage_err(p, "LAYERNORM needs n_in = n_out"); return PM_ERR_INVALID_ARG; }
       s.pre = PRE_LN;
+      s.from_memory = (sd.ops[0].flags & PM_OPF_FROM_MEMORY) ? 1 : 0;
       offsets(0, &s.g_off, &s.beta_off);
       idx = 1;
     }
@@ -133,8 +142,16 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
         if (n_out % 3 || op.n_heads < 1 || (n_out / 3) % op.n_heads || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad ATTENTION description"); return PM_ERR_INVALID_ARG; }
         if (op.seq_len > 128) { stage_err(p, "ATTENTION is built for seq_len <= 128"); return PM_ERR_UNSUPPORTED; }
         s.post = POST_ATTENTION; s.n_heads = op.n_heads; s.seq_len = op.seq_len;
-      } else if (op.kind == PM_OP_SKIP_OUT) s.post = POST_SKIP_OUT;
-      else if (op.kind == PM_OP_RESIDUAL) s.post = POST_RESIDUAL;
+        s.causal = (op.flags & PM_OPF_CAUSAL) ? 1 : 0;
+        s.skip_hop = 1;
+      } else if (op.kind == PM_OP_CROSS_ATTENTION) {
+        const int n_out = s.lin[s.n_lin - 1].n_out;
+        if (n_out % 2 || op.n_heads < 1 || (n_out / 2) % op.n_heads || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad CROSS_ATTENTION description"); return PM_ERR_INVALID_ARG; }
+        if (op.seq_len > 128) { stage_err(p, "attention is built for seq_len <= 128"); return PM_ERR_UNSUPPORTED; }
+        if (!s.from_memory || n_out / 2 != s.lin[0].n_in) { stage_err(p, "CROSS_ATTENTION needs LAYERNORM | PM_OPF_FROM_MEMORY and a memory as wide as the queries"); return PM_ERR_UNSUPPORTED; }
+        s.post = POST_CROSS_ATTENTION; s.n_heads = op.n_heads; s.seq_len = op.seq_len;
+      } else if (op.kind == PM_OP_SKIP_OUT) { s.post = POST_SKIP_OUT; s.skip_hop = (op.flags & PM_OPF_SKIP_TWO) ? 2 : 1; }
+      else if (op.kind == PM_OP_RESIDUAL) { s.post = POST_RESIDUAL; s.emit_memory = (op.flags & PM_OPF_EMIT_MEMORY) ? 1 : 0; }
       else { stage_err(p, "unexpected op after the Linear ops"); return PM_ERR_INVALID_ARG; }
       ++idx;
     }
@@ -142,18 +159,36 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if ((s.pre != PRE_NONE || s.post != POST_NONE) && s.n_lin != 1) { stage_err(p, "a stage with a pre- or post-op holds exactly one LINEAR"); return PM_ERR_UNSUPPORTED; }
     s.d_in = s.lin[0].n_in;
     const int n_out_last = s.lin[s.n_lin - 1].n_out;
-    s.d_out_main = s.post == POST_ATTENTION ? n_out_last / 3 : n_out_last;
+    s.d_out_main = s.post == POST_ATTENTION ? n_out_last / 3 : (s.post == POST_CROSS_ATTENTION ? n_out_last / 2 : n_out_last);
+    s.gin_depth = 3;
+    if (s.from_memory && s.post != POST_CROSS_ATTENTION) { stage_err(p, "PM_OPF_FROM_MEMORY belongs to a stage ending in CROSS_ATTENTION"); return PM_ERR_UNSUPPORTED; }
+    if (s.emit_memory) {
+      if (L.mem_stage >= 0) { stage_err(p, "one stage emits the memory"); return PM_ERR_UNSUPPORTED; }
+      L.mem_stage = p; L.mem_dim = n_out_last;
+    }
+    if (s.from_memory) {
+      if (L.mem_stage < 0 || L.mem_dim != s.lin[0].n_in) { stage_err(p, "no memory of this width was emitted before this stage"); return PM_ERR_UNSUPPORTED; }
+      L.last_mem_reader = p;
+    }
     s.max_dim = std::max(std::max(max_in, max_out), s.d_in);
     // ---- chaining
     if (p > 0) {
       const StageDev& q = L.st[p - 1];
-      if (s.pre == PRE_EMBED) { stage_err(p, "EMBED belongs to the first stage"); return PM_ERR_UNSUPPORTED; }
-      if (s.d_in != q.d_out_main) { stage_err(p, "input width does not match the previous stage's output"); return PM_ERR_SHAPE; }
-      const bool emits = q.post == POST_ATTENTION || q.post == POST_SKIP_OUT;
-      if (emits != (s.post == POST_RESIDUAL)) { stage_err(p, "RESIDUAL must directly follow a stage ending in ATTENTION or SKIP_OUT, and only then"); return PM_ERR_UNSUPPORTED; }
-      if (s.post == POST_RESIDUAL && q.d_in != n_out_last) { stage_err(p, "skip tensor width does not match the Linear's output"); return PM_ERR_SHAPE; }
+      const int main_in = s.post == POST_CROSS_ATTENTION ? s.d_out_main : s.d_in;        // width of the main input
+      if (s.pre != PRE_EMBED && main_in != q.d_out_main) { stage_err(p, "input width does not match the previous stage's output"); return PM_ERR_SHAPE; }
+      if (q.emit_memory && s.pre != PRE_EMBED) { stage_err(p, "the stage after the one that emits the memory starts with a second-stream EMBED"); return PM_ERR_UNSUPPORTED; }
+      // skip tensors: an emitter hop positions back must exist for a RESIDUAL, and only then
+      int src = -1;
+      if (q.skip_hop == 1) src = p - 1;
+      if (p >= 2 && L.st[p - 2].skip_hop == 2) { if (src >= 0 || q.post != POST_CROSS_ATTENTION) { stage_err(p, "a skip over two stages passes over a CROSS_ATTENTION stage only"); return PM_ERR_UNSUPPORTED; } src = p - 2; }
+      if ((src >= 0) != (s.post == POST_RESIDUAL)) { stage_err(p, "RESIDUAL must follow the stage that sends it a skip tensor, and only then"); return PM_ERR_UNSUPPORTED; }
+      if (s.post == POST_RESIDUAL) {
+        if (L.st[src].d_in != n_out_last) { stage_err(p, "skip tensor width does not match the Linear's output"); return PM_ERR_SHAPE; }
+        s.skip_depth = (p - src) + 1;
+        s.gin_depth = (p - src) + 2;
+      }
     } else if (s.post == POST_RESIDUAL) { stage_err(p, "the first stage has no skip tensor to add"); return PM_ERR_UNSUPPORTED; }
-    if (p == P - 1 && (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT)) { stage_err(p, "the last stage cannot emit a skip tensor"); return PM_ERR_UNSUPPORTED; }
+    if (p + s.skip_hop > P - 1 && s.skip_hop > 0) { stage_err(p, "a skip tensor needs its RESIDUAL stage"); return PM_ERR_UNSUPPORTED; }
     if (p == P - 1 && ce && (s.n_lin != 1 || s.post != POST_NONE || s.lin[0].act != PM_ACT_NONE)) { stage_err(p, "PM_LOSS_CE needs a last stage of one Linear without activation or post-op"); return PM_ERR_UNSUPPORTED; }
     // ---- what each Linear's forward writes
     for (int l = 0; l < s.n_lin; ++l) {
@@ -161,15 +196,16 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       const bool last = l == s.n_lin - 1;
       const bool logits = last && p == P - 1 && ce;
       ld.flags = 0;
-      if (ld.act != PM_ACT_NONE || (last && s.post == POST_ATTENTION)) ld.flags |= LF_WRITE_Z;
-      if (!(last && s.post == POST_ATTENTION) && !logits) ld.flags |= LF_WRITE_Y;
+      const bool to_attention = last && (s.post == POST_ATTENTION || s.post == POST_CROSS_ATTENTION);   // q, k, v stash
+      if (ld.act != PM_ACT_NONE || to_attention) ld.flags |= LF_WRITE_Z;
+      if (!to_attention && !logits) ld.flags |= LF_WRITE_Y;
       if (logits) ld.flags |= LF_OUT_F32;
     }
     // ---- rings
     if (s.pre != PRE_EMBED) { s.x_ring = ring; ring = align_up(ring + (uint64_t)s.xdepth * T * s.d_in * esz, 256); }
     if (s.pre != PRE_NONE) { s.u_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.d_in * esz, 256); }
     if (s.pre == PRE_LN) { s.stat_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * 2 * 4, 256); }
-    if (s.pre == PRE_EMBED) { s.ids_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * 4, 256); }
+    if (s.pre == PRE_EMBED) { s.ids_ring = ring; ring = align_up(ring + (uint64_t)s.ids_depth * T * 4, 256); }
     for (int l = 0; l < s.n_lin; ++l) {
       if (s.lin[l].flags & LF_WRITE_Z) { s.lin[l].z_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
       if (l < s.n_lin - 1) { s.lin[l].h_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
@@ -180,7 +216,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (s.pre == PRE_LN) L.any_ln = 1;
     if (s.pre == PRE_EMBED) { L.any_embed = 1; L.max_vocab = std::max(L.max_vocab, s.vocab); }
     if (s.post == POST_RESIDUAL) L.any_residual = 1;
-    if (s.post == POST_ATTENTION) {
+    if (s.post == POST_ATTENTION || s.post == POST_CROSS_ATTENTION) {
+      if (s.causal || s.post == POST_CROSS_ATTENTION) L.att_plain = false;
       const int dk = s.d_out_main / s.n_heads;
       L.att_S = std::max(L.att_S, s.seq_len); L.att_dk = std::max(L.att_dk, dk);
       L.att_blocks = std::max(L.att_blocks, (int)(T / s.seq_len) * s.n_heads);
@@ -188,7 +225,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
   }
   for (int p = 0; p < P; ++p) L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
-  L.att_tc = L.att_blocks > 0;
+  if (L.mem_stage >= 0) {
+    if (L.last_mem_reader < 0) { err = "a memory is emitted but no CROSS_ATTENTION stage reads it"; return PM_ERR_UNSUPPORTED; }
+    L.st[L.last_mem_reader].mem_first = 1;
+    L.mem_depth = 2 * P - 2 * L.mem_stage;
+    L.gmem_depth = P - L.mem_stage + 2;
+    L.mem_ring = ring; ring = align_up(ring + (uint64_t)L.mem_depth * T * L.mem_dim * esz, 256);
+  }
+  L.att_tc = L.att_blocks > 0 && L.att_plain;      // the tensor-core kernels cover plain self-attention
   for (int p = 0; p < P; ++p)
     if (L.st[p].post == POST_ATTENTION && !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads)) L.att_tc = false;
   if (L.att_blocks > 0 && !L.att_tc && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
@@ -234,6 +278,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.act_blocks[l] = acc;
   }
   L.off_ids = w; w = align_up(w + sizeof(int32_t) * L.ids.size(), 256);
+  if (L.mem_stage >= 0 && !L.ln_fused) { err = "stages that read the memory need LayerNorm widths that are multiples of 8 and at most 1024"; return PM_ERR_UNSUPPORTED; }
   L.ln_chunk_rows = 64;
   L.ln_chunks = (int32_t)((T + L.ln_chunk_rows - 1) / L.ln_chunk_rows);
   L.off_lnred = w; w = align_up(w + (uint64_t)L.n_ln * L.ln_chunks * 2 * L.max_ln_dim * 4, 256);
@@ -241,17 +286,18 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
   L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes((int)T, L.st) : 0), 256);
   L.off_attn = w; w = align_up(w + (L.att_tc ? attn_workspace_bytes(P) : 0), 256);
+  L.off_gmem = w; w = align_up(w + (uint64_t)L.gmem_depth * T * L.mem_dim * esz, 256);
   for (int p = 0; p < P; ++p) {
     StageDev& s = L.st[p];
     const uint64_t n_out_last = s.lin[s.n_lin - 1].n_out;
     uint64_t mo = 0, mi = 0;
     for (int l = 0; l < s.n_lin; ++l) { mo = std::max<uint64_t>(mo, s.lin[l].n_out); mi = std::max<uint64_t>(mi, s.lin[l].n_in); }
-    s.gin = w; w = align_up(w + 3 * T * s.d_out_main * esz, 256);
+    s.gin = w; w = align_up(w + (uint64_t)s.gin_depth * T * s.d_out_main * esz, 256);
     if (s.post == POST_RESIDUAL) {
-      s.skip_in = w; w = align_up(w + 2 * T * n_out_last * esz, 256);
+      s.skip_in = w; w = align_up(w + (uint64_t)s.skip_depth * T * n_out_last * esz, 256);
       s.ytmp = w; w = align_up(w + T * n_out_last * esz, 256);
     }
-    if (s.post == POST_ATTENTION) { s.dy = w; w = align_up(w + T * n_out_last * esz, 256); }
+    if (s.post == POST_ATTENTION || s.post == POST_CROSS_ATTENTION) { s.dy = w; w = align_up(w + T * n_out_last * esz, 256); }
     s.dz = w; w = align_up(w + T * mo * esz, 256);
     s.dh = w; w = align_up(w + T * mi * esz, 256);
   }
@@ -315,7 +361,7 @@ pm_status pm_stage_param_count(const pm_op_desc* ops, int32_t n_ops, uint64_t* c
   if (!ops || !count || n_ops < 1) return PM_ERR_INVALID_ARG;
   uint64_t c = 0;
   for (int l = 0; l < n_ops; ++l) {
-    if (ops[l].kind < PM_OP_LINEAR || ops[l].kind > PM_OP_RESIDUAL) return PM_ERR_INVALID_ARG;
+    if (ops[l].kind < PM_OP_LINEAR || ops[l].kind > PM_OP_CROSS_ATTENTION) return PM_ERR_INVALID_ARG;
     if (ops[l].kind <= PM_OP_LAYERNORM && (ops[l].n_in < 1 || ops[l].n_out < 1)) return PM_ERR_INVALID_ARG;
     uint64_t n0, n1;
     const int k = op_params(ops[l], &n0, &n1);
@@ -432,6 +478,10 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     t.lnred_off = L.off_lnred; t.ln_chunks = L.ln_chunks; t.ln_chunk_rows = L.ln_chunk_rows; t.max_ln_dim = L.max_ln_dim;
     t.ln_fused = L.ln_fused;
     t.act_start = ids + 4 * P;
+    t.mem_ring = L.mem_ring; t.gmem_off = L.off_gmem; t.mem_depth = L.mem_depth; t.gmem_depth = L.gmem_depth;
+    t.mem_dim = L.mem_dim; t.n_streams = L.n_streams;
+    t.second_embed_stage = 0;
+    for (int p = 0; p < P; ++p) if (L.st[p].pre == PRE_EMBED && L.st[p].ids_stream == 1) t.second_embed_stage = p;
     for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_blocks[l] = L.act_blocks[l];
   }
   if (L.pe_seq > 0) {

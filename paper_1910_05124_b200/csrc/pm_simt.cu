@@ -20,8 +20,13 @@ __global__ void ingest_kernel(TickArgs t, const void* __restrict__ inputs, const
   const StageDev& s0 = t.st[0];
   const uint64_t gid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (uint64_t)gridDim.x * blockDim.x;
   if (s0.pre == PRE_EMBED) {
-    int32_t* idst = ring_ptr<int32_t>(t, s0.ids_ring, (int)(mb % s0.depth), (uint64_t)t.T);
+    int32_t* idst = ring_ptr<int32_t>(t, s0.ids_ring, (int)(mb % s0.ids_depth), (uint64_t)t.T);
     for (uint64_t i = gid; i < (uint64_t)t.T; i += stride) idst[i] = reinterpret_cast<const int32_t*>(inputs)[i];
+    if (t.n_streams > 1) {                                    // second token stream -> the stage that embeds it
+      const StageDev& s1 = t.st[t.second_embed_stage];
+      int32_t* d1 = ring_ptr<int32_t>(t, s1.ids_ring, (int)(mb % s1.ids_depth), (uint64_t)t.T);
+      for (uint64_t i = gid; i < (uint64_t)t.T; i += stride) d1[i] = reinterpret_cast<const int32_t*>(inputs)[(uint64_t)t.T + i];
+    }
   } else {
     const uint64_t n_x = (uint64_t)t.T * t.n_in_first;
     AT* xdst = ring_ptr<AT>(t, s0.x_ring, (int)(mb % s0.xdepth), n_x);
@@ -181,7 +186,7 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   const int c = c0 + 8 * lane;
   const uint64_t n = (uint64_t)t.T * L.n_out;
   const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
-                 : (s.post == POST_ATTENTION ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
+                 : (feeds_attention(s.post) ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
   const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy: nothing is stored
   const AT* z = has_act ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n) : dy;
   AT* dz = ws_ptr<AT>(t, s.dz);

@@ -38,6 +38,11 @@ struct TickArgs {
   const int32_t* act_start;
   int32_t act_blocks[PM_MAX_LINEARS];
   int32_t ln_fused;       // every LayerNorm width is a multiple of 8 and at most 1024: one fused backward kernel
+  // encoder memory (ring arena) [mem_depth][T*mem_dim], slot = microbatch % mem_depth, and its gradient
+  // (workspace) [gmem_depth][T*mem_dim], slot = microbatch % gmem_depth; mem_dim = 0 when there is none
+  uint64_t mem_ring, gmem_off;
+  int32_t mem_depth, gmem_depth, mem_dim, n_streams;
+  int32_t second_embed_stage;   // the stage that embeds the second token stream (when n_streams == 2)
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages
 };
@@ -56,26 +61,48 @@ template <typename AT> __device__ __forceinline__ const AT* lin_input(const Tick
   if (s.pre != PRE_NONE) return ring_at<AT>(t, s.u_ring, fwd ? d.f_slot : d.b_slot, n);
   return ring_at<AT>(t, s.x_ring, fwd ? d.f_xslot : d.b_xslot, n);
 }
-// gradient w.r.t. this stage's main output: written by the next stage during the previous tick
+// slot of a stage's gradient mailbox that holds what was written during the previous tick
+__device__ __forceinline__ int gin_slot_read(const StageDev& s, const StageDyn& d) { return (int)((d.tick + s.gin_depth - 1) % s.gin_depth); }
+// slot of the dz operand of a stage's last Linear when that operand is the incoming gradient itself (no activation,
+// no attention): the rotating mailbox slot written during the previous tick, or the memory-gradient ring slot of the
+// microbatch for the stage that emits the memory
+__device__ __forceinline__ int dz_mailbox_slot(const TickArgs& t, const StageDev& s, const StageDyn& d) {
+  return s.emit_memory ? (int)(d.b_mb % t.gmem_depth) : gin_slot_read(s, d);
+}
+// gradient of the memory for the microbatch in backward at a stage
+template <typename AT> __device__ __forceinline__ AT* gmem_at(const TickArgs& t, const StageDyn& d) {
+  return ws_at<AT>(t, t.gmem_off) + (uint64_t)(d.b_mb % t.gmem_depth) * ((uint64_t)t.T * t.mem_dim);
+}
+// gradient w.r.t. this stage's main output: written by the next stage during the previous tick; the stage that
+// emits the memory receives the sum the cross-attention stages left in the memory-gradient ring
 template <typename AT> __device__ __forceinline__ AT* gin_read(const TickArgs& t, const StageDev& s, const StageDyn& d) {
-  return ws_at<AT>(t, s.gin) + (uint64_t)((d.tick + 2) % 3) * ((uint64_t)t.T * s.d_out_main);
+  if (s.emit_memory) return gmem_at<AT>(t, d);
+  return ws_at<AT>(t, s.gin) + (uint64_t)gin_slot_read(s, d) * ((uint64_t)t.T * s.d_out_main);
 }
 // where stage p writes the gradient w.r.t. its main input (= stage p-1's main output)
 template <typename AT> __device__ __forceinline__ AT* gin_write_prev(const TickArgs& t, int p, const StageDyn& d) {
   const StageDev& sp = t.st[p - 1];
-  return ws_at<AT>(t, sp.gin) + (uint64_t)(d.tick % 3) * ((uint64_t)t.T * sp.d_out_main);
+  return ws_at<AT>(t, sp.gin) + (uint64_t)(d.tick % sp.gin_depth) * ((uint64_t)t.T * sp.d_out_main);
 }
-// gradient w.r.t. the skip tensor stage p emitted: it equals the gradient the next (residual) stage received
-// one tick ago for the same microbatch, i.e. what the stage after it wrote two ticks ago
+// gradient w.r.t. the skip tensor stage p emitted: it equals the gradient the receiving (residual) stage took in
+// skip_hop ticks ago for the same microbatch, i.e. what the stage after that one wrote skip_hop + 1 ticks ago
 template <typename AT> __device__ __forceinline__ const AT* gskip_read(const TickArgs& t, int p, const StageDyn& d) {
-  const StageDev& sn = t.st[p + 1];
-  return ws_at<AT>(t, sn.gin) + (uint64_t)((d.tick + 1) % 3) * ((uint64_t)t.T * sn.d_out_main);
+  const StageDev& sn = t.st[p + t.st[p].skip_hop];
+  if (sn.emit_memory) return gmem_at<AT>(t, d);
+  const int slot = (int)((d.tick + 2 * sn.gin_depth - t.st[p].skip_hop - 1) % sn.gin_depth);
+  return ws_at<AT>(t, sn.gin) + (uint64_t)slot * ((uint64_t)t.T * sn.d_out_main);
+}
+// does stage p emit a skip tensor
+__device__ __forceinline__ bool emits_skip(const StageDev& s) { return s.skip_hop > 0; }
+// the memory of the microbatch a stage processes (forward or backward)
+template <typename AT> __device__ __forceinline__ AT* mem_at(const TickArgs& t, int64_t mb) {
+  return ring_at<AT>(t, t.mem_ring, (int)(mb % t.mem_depth), (uint64_t)t.T * t.mem_dim);
 }
 // dz = dy * act'(z) of Linear lvl as the wgrad / dgrad operand: without an activation it IS the incoming gradient
 template <typename AT> __device__ __forceinline__ const AT* dz_src(const TickArgs& t, const StageDev& s, const StageDyn& d, int lvl) {
   if (s.lin[lvl].act != PM_ACT_NONE) return ws_at<AT>(t, s.dz);
   if (lvl < s.n_lin - 1) return ws_at<AT>(t, s.dh);
-  if (s.post == POST_ATTENTION) return ws_at<AT>(t, s.dy);
+  if (feeds_attention(s.post)) return ws_at<AT>(t, s.dy);
   return gin_read<AT>(t, s, d);
 }
 // destination of Linear lvl's activation y in the forward pass (nullptr: not written)

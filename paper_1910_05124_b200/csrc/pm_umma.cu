@@ -245,7 +245,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         // dz operand: the dz scratch, or (no activation) the incoming gradient itself, which for the last Linear of a
         // stage without attention is the rotating mailbox slot written during the previous tick
         const StageDev& sd_ = t.st[tl.p];
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         for (int kb = 0; kb < tl.n_kb; ++kb) {
@@ -450,7 +450,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         const StageDyn& d = t.dyn[tl.p];
         const StageDev& sd_ = t.st[tl.p];
         const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         const int ma = tl.m0 + rank * TILE_M, nbh = tl.n0 + rank * TILE_N;   // this CTA's rows of A and of B
@@ -687,7 +687,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
         const StageDyn& d = t.dyn[ca.tl.p];
         const StageDev& sd_ = t.st[ca.tl.p];
         const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         for (int mi = 0; mi < ca.tl.n_m; ++mi) {
           if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 22)) { ok = false; break; }
           const uint32_t fa = bar_afull + 8 * ar.idx;
@@ -812,7 +812,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       ready = __all_sync(0xffffffffu, ready);
       if (!ready) { ok = false; break; }
       tc_fence_after();
-      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0;
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % t.st[tl.p - 1].gin_depth) : 0;
       for (int mi = 0; mi < tl.n_m; ++mi) {
         const int mrow = tl.m0 + mi * TILE_M + q * 32;
 #pragma unroll 1
@@ -976,7 +976,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
         const StageDyn& d = t.dyn[ca.tl.p];
         const StageDev& sd_ = t.st[ca.tl.p];
         const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && sd_.post != POST_ATTENTION) ? (int)((d.tick + 2) % 3) : 0;
+        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         for (int mi = 0; mi < ca.tl.n_m; ++mi) {
           if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 42)) { ok = false; break; }
           if (rank == 0) mbar_arrive_expect_tx(bar_afull + 8 * ar.idx, 2 * A_BYTES);       // the rows of both CTAs
@@ -1110,7 +1110,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       ready = __all_sync(0xffffffffu, ready);
       if (!ready) { ok = false; break; }
       tc_fence_after();
-      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % 3) : 0;
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % t.st[tl.p - 1].gin_depth) : 0;
       const int nb = tl.n0 + half * 64;
 #pragma unroll 1
       for (int mi = 0; mi < tl.n_m; ++mi) {
@@ -1329,8 +1329,9 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         char* dzb; uint64_t dz_slots = 1;
         if (L.act != PM_ACT_NONE) dzb = t.ws + s.dz;
         else if (l < s.n_lin - 1) dzb = t.ws + s.dh;
-        else if (s.post == POST_ATTENTION) dzb = t.ws + s.dy;
-        else { dzb = t.ws + s.gin; dz_slots = 3; }
+        else if (feeds_attention(s.post)) dzb = t.ws + s.dy;
+        else if (s.emit_memory) { dzb = t.ws + t.gmem_off; dz_slots = (uint64_t)t.gmem_depth; }
+        else { dzb = t.ws + s.gin; dz_slots = (uint64_t)s.gin_depth; }
         uint64_t dims[3] = {n_out, T, dz_slots}, strides[2] = {n_out * 2, T * n_out * 2};
         uint32_t box_k[3] = {TILE_K, TILE_M, 1}, box_mn[3] = {64, TILE_K, 1};
         okm = okm && encode(fn, m + MAP_DZ_K, 0, dzb, 3, dims, strides, box_k, err);
@@ -1357,7 +1358,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         if (!(p == 0 && l == 0 && s.pre != PRE_EMBED)) {
           const bool to_prev = l == 0 && s.pre == PRE_NONE;
           char* xbase = to_prev ? t.ws + st[p - 1].gin : t.ws + s.dh;
-          uint64_t xd[3] = {n_in, T, (uint64_t)(to_prev ? 3 : 1)}, xs[2] = {n_in * 2, T * n_in * 2};
+          uint64_t xd[3] = {n_in, T, (uint64_t)(to_prev ? st[p - 1].gin_depth : 1)}, xs[2] = {n_in * 2, T * n_in * 2};
           okm = okm && encode(fn, m + MAP_DX_OUT, 1, xbase, 3, xd, xs, box_bf, err);
         }
         uint64_t wd[2] = {n_in, n_out}, wst[1] = {n_in * 4};

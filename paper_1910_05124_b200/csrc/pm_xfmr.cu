@@ -42,11 +42,11 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   const int dm = s.d_in;
   const uint64_t n = (uint64_t)t.T * dm;
   AT* u = ring_at<AT>(t, s.u_ring, d.f_slot, n) + (uint64_t)row * dm;
-  AT* skip = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT)
-                 ? ws_at<AT>(t, t.st[p + 1].skip_in) + (uint64_t)(d.tick & 1) * n + (uint64_t)row * dm : nullptr;
+  const StageDev& sk_dst = t.st[p + s.skip_hop];             // the residual stage that will add this stage's input
+  AT* skip = emits_skip(s) ? ws_at<AT>(t, sk_dst.skip_in) + (uint64_t)(d.tick % sk_dst.skip_depth) * n + (uint64_t)row * dm : nullptr;
   const bool vec = (dm & 7) == 0;                            // 8 consecutive columns per lane, 256 per pass
   if (s.pre == PRE_EMBED) {
-    const int32_t id = ring_at<int32_t>(t, s.ids_ring, d.f_slot, (uint64_t)t.T)[row];
+    const int32_t id = ring_at<int32_t>(t, s.ids_ring, (int)(d.f_mb % s.ids_depth), (uint64_t)t.T)[row];
     const AT* e = table_ptr<AT>(t) + s.tab_off + (uint64_t)id * dm;
     const float* pe = ws_at<float>(t, t.pe_off) + (uint64_t)(row % s.seq_len) * dm;
     const float sc = sqrtf((float)dm);
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
     }
     return;
   }
-  const AT* x = ring_at<AT>(t, s.x_ring, d.f_xslot, n) + (uint64_t)row * dm;
+  const AT* x = (s.from_memory ? mem_at<AT>(t, d.f_mb) : ring_at<AT>(t, s.x_ring, d.f_xslot, n)) + (uint64_t)row * dm;
   const float* g = t.a.w + s.g_off;
   const float* b = t.a.w + s.beta_off;
   float sum = 0.f, sq = 0.f;
@@ -134,9 +134,10 @@ __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || s.post != POST_RESIDUAL) return;
   const uint64_t n = (uint64_t)t.T * s.d_out_main;
-  const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)((d.tick + 1) & 1) * n;     // written by the previous stage last tick
+  const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)((d.tick + 1) % s.skip_depth) * n;   // written skip_depth - 1 ticks ago
   const AT* y = ws_at<AT>(t, s.ytmp);
-  AT* out = ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
+  // the stage that emits the memory writes only there: the next stage embeds its own token stream
+  AT* out = s.emit_memory ? mem_at<AT>(t, d.f_mb) : ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
   // buffers start on 256-byte boundaries and slots are n elements apart: groups of eight are aligned when 8 | n
   const uint64_t n8 = (n % 8 == 0) ? n / 8 : 0;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -170,11 +171,13 @@ __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
 struct AttnShape { int S, dk, d; };
 
 template <typename AT>
-__global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t, int causal) {
+__global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t) {
   const int p = blockIdx.y;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
-  if (d.f_mb < 0 || s.post != POST_ATTENTION) return;
+  if (d.f_mb < 0 || (s.post != POST_ATTENTION && s.post != POST_CROSS_ATTENTION)) return;
+  const bool cross = s.post == POST_CROSS_ATTENTION;        // q = the stage's main input, the Linear gave [k | v]
+  const int causal = s.causal;
   const int S = s.seq_len, H = s.n_heads, dm = s.d_out_main, dk = dm / H;
   const int n_seq = t.T / S;
   if ((int)blockIdx.x >= n_seq * H) return;
@@ -186,14 +189,16 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t, int caus
   AT* Q = reinterpret_cast<AT*>(Ls + S);   // [S][dk+2]
   AT* K = Q + S * ld;
   AT* V = K + S * ld;
-  const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
-  const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.f_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
+  const int wz = cross ? 2 * dm : 3 * dm;                    // row length of the Linear's output
+  const AT* zb = ring_at<AT>(t, s.lin[0].z_ring, d.f_slot, (uint64_t)t.T * wz) + (uint64_t)b * S * wz + h * dk;
+  const AT* qb = cross ? ring_at<AT>(t, s.x_ring, d.f_xslot, (uint64_t)t.T * dm) + (uint64_t)b * S * dm + h * dk : zb;
+  const int wq = cross ? dm : wz, ko = cross ? 0 : dm;
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
-    const AT* row = qkv + (uint64_t)r * 3 * dm;
-    Q[r * ld + c] = row[c];
-    K[r * ld + c] = row[dm + c];
-    V[r * ld + c] = row[2 * dm + c];
+    const AT* row = zb + (uint64_t)r * wz;
+    Q[r * ld + c] = qb[(uint64_t)r * wq + c];
+    K[r * ld + c] = row[ko + c];
+    V[r * ld + c] = row[ko + dm + c];
   }
   __syncthreads();
   const float scale = 1.0f / sqrtf((float)dk);
@@ -242,8 +247,8 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
   cudaError_t e = cudaSuccess;
   if (any_att) {
     dim3 grid(nblk, t.P);
-    if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, attn_fwd_smem(S, dk, 4), stream>>>(t, 0);
-    else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, attn_fwd_smem(S, dk, 2), stream>>>(t, 0);
+    if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, attn_fwd_smem(S, dk, 4), stream>>>(t);
+    else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, attn_fwd_smem(S, dk, 2), stream>>>(t);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -260,11 +265,13 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
 // P recomputed as in the forward pass.  dV = round(P)^T dO; dP = dO V^T; dS = round(P * (dP - rowsum(dP * P)));
 // dQ = dS K / sqrt(d_k); dK = dS^T Q / sqrt(d_k).  Results go to the stage's dy buffer as [dq | dk | dv].
 template <typename AT>
-__global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int causal) {
+__global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t) {
   const int p = blockIdx.y;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
-  if (d.b_mb < 0 || s.post != POST_ATTENTION) return;
+  if (d.b_mb < 0 || (s.post != POST_ATTENTION && s.post != POST_CROSS_ATTENTION)) return;
+  const bool cross = s.post == POST_CROSS_ATTENTION;
+  const int causal = s.causal;
   const int S = s.seq_len, H = s.n_heads, dm = s.d_out_main, dk = dm / H;
   const int n_seq = t.T / S;
   if ((int)blockIdx.x >= n_seq * H) return;
@@ -278,15 +285,17 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
   AT* K = Q + S * ld;
   AT* V = K + S * ld;
   AT* dO = V + S * ld;
-  const uint64_t nqkv = (uint64_t)t.T * 3 * dm;
-  const AT* qkv = ring_at<AT>(t, s.lin[0].z_ring, d.b_slot, nqkv) + (uint64_t)b * S * 3 * dm + h * dk;
+  const int wz = cross ? 2 * dm : 3 * dm;
+  const AT* zb = ring_at<AT>(t, s.lin[0].z_ring, d.b_slot, (uint64_t)t.T * wz) + (uint64_t)b * S * wz + h * dk;
+  const AT* qb = cross ? ring_at<AT>(t, s.x_ring, d.b_xslot, (uint64_t)t.T * dm) + (uint64_t)b * S * dm + h * dk : zb;
+  const int wq = cross ? dm : wz, ko = cross ? 0 : dm;
   const AT* go = gin_read<AT>(t, s, d) + (uint64_t)b * S * dm + h * dk;
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
-    const AT* row = qkv + (uint64_t)r * 3 * dm;
-    Q[r * ld + c] = row[c];
-    K[r * ld + c] = row[dm + c];
-    V[r * ld + c] = row[2 * dm + c];
+    const AT* row = zb + (uint64_t)r * wz;
+    Q[r * ld + c] = qb[(uint64_t)r * wq + c];
+    K[r * ld + c] = row[ko + c];
+    V[r * ld + c] = row[ko + dm + c];
     dO[r * ld + c] = go[(uint64_t)r * dm + c];
   }
   __syncthreads();
@@ -316,7 +325,9 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
     for (int c = lane; c < S; c += 32) Dm[r * lp + c] = round_as<AT>(Pm[r * lp + c] * (Dm[r * lp + c] - dsum));   // dS
   }
   __syncthreads();
-  AT* dy = ws_at<AT>(t, s.dy) + (uint64_t)b * S * 3 * dm + h * dk;
+  // self-attention: dy = [dq | dk | dv]; cross-attention: dy = [dk | dv] and dq goes to the previous stage's mailbox
+  AT* dy = ws_at<AT>(t, s.dy) + (uint64_t)b * S * wz + h * dk;
+  AT* dqb = cross ? gin_write_prev<AT>(t, p, d) + (uint64_t)b * S * dm + h * dk : dy;
   for (int i = threadIdx.x; i < S * dk; i += blockDim.x) {
     const int r = i / dk, c = i % dk;
     float aq = 0.f, ak = 0.f, av = 0.f;
@@ -325,18 +336,18 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t, int caus
       ak = fmaf(Dm[j * lp + r], to_f<AT>(Q[j * ld + c]), ak);            // dK[r] = sum_j dS[j][r] Q[j]
       av = fmaf(round_as<AT>(Pm[j * lp + r]), to_f<AT>(dO[j * ld + c]), av);   // dV[r] = sum_j P[j][r] dO[j]
     }
-    AT* row = dy + (uint64_t)r * 3 * dm;
-    row[c] = from_f<AT>(aq * scale);
-    row[dm + c] = from_f<AT>(ak * scale);
-    row[2 * dm + c] = from_f<AT>(av);
+    AT* row = dy + (uint64_t)r * wz;
+    dqb[(uint64_t)r * wq + c] = from_f<AT>(aq * scale);
+    row[ko + c] = from_f<AT>(ak * scale);
+    row[ko + dm + c] = from_f<AT>(av);
   }
 }
 
 cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   if (t.att_blocks <= 0) return cudaSuccess;
   dim3 grid(t.att_blocks, t.P);
-  if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 4), stream>>>(t, 0);
-  else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 2), stream>>>(t, 0);
+  if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 4), stream>>>(t);
+  else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 2), stream>>>(t);
   return cudaGetLastError();
 }
 
@@ -488,8 +499,9 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
   if (row >= t.T) return;
   const int dm = s.d_in;
   const uint64_t n = (uint64_t)t.T * dm, ro = (uint64_t)row * dm;
+  if (s.from_memory) return;                                 // memory stages take the fused kernel (widths are multiples of 8)
   const AT* du = ws_at<AT>(t, s.dh);
-  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
   const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n) + ro;
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
   const float mu = st[0], rstd = st[1];
@@ -569,7 +581,7 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint64_t n = (uint64_t)t.T * dm;
   const AT* du = ws_at<AT>(t, s.dh);
-  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
   const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n);
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
   const bool vec = (dm & 7) == 0;
@@ -655,10 +667,13 @@ __global__ void __launch_bounds__(256) ln_bwd_fused_kernel(TickArgs t) {
   const int dm = s.d_in;
   const uint64_t n = (uint64_t)t.T * dm;
   const AT* du = ws_at<AT>(t, s.dh);
-  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
-  const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n);
+  const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* x = s.from_memory ? mem_at<AT>(t, d.b_mb) : ring_at<AT>(t, s.x_ring, d.b_xslot, n);
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2);
-  AT* out = p > 0 ? gin_write_prev<AT>(t, p, d) : nullptr;          // the first stage has no predecessor to hand dx to
+  // dx goes to the previous stage's mailbox; a stage that normalises the memory adds it to the memory gradient of
+  // its microbatch (the last such stage runs first and stores); the first stage has no predecessor
+  AT* out = s.from_memory ? gmem_at<AT>(t, d) : (p > 0 ? gin_write_prev<AT>(t, p, d) : nullptr);
+  const bool accumulate = s.from_memory && !s.mem_first;
   const float gapf = (float)s.gap;
   const bool corr = d.use_delta != 0;
   float gb[NP][8], ag[NP][8], ab[NP][8];
@@ -722,6 +737,12 @@ __global__ void __launch_bounds__(256) ln_bwd_fused_kernel(TickArgs t) {
           float o[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) o[k] = rstd * (dxh[q][k] - s1 - xh[q][k] * s2);
+          if (accumulate) {
+            float prev[8];
+            load8<AT>(out + ro + c, prev);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = __fadd_rn(prev[k], round_as<AT>(o[k]));
+          }
           store8<AT>(out + ro + c, o);
         }
       }
@@ -803,7 +824,7 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   if (v0 >= s.vocab) return;
   extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
   __shared__ int warp_cnt[2][8];
-  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, d.b_slot, (uint64_t)t.T);
+  const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, (int)(d.b_mb % s.ids_depth), (uint64_t)t.T);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int nh = 0;                                                // hits so far (the same value in every thread)
   for (int tb0 = 0; tb0 < t.T; tb0 += 16 * 256) {            // 16 rounds of 256 tokens; the ids of all rounds are fetched first
@@ -830,7 +851,7 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   __syncthreads();
   const int dm = s.d_in;
   const AT* du = ws_at<AT>(t, s.dh);
-  const AT* gs = (s.post == POST_ATTENTION || s.post == POST_SKIP_OUT) ? gskip_read<AT>(t, p, d) : nullptr;
+  const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
   const float sc = sqrtf((float)dm);
   for (int rr = warp; rr < kEmbRows; rr += 8) {
     const int v = v0 + rr;

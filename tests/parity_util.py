@@ -20,7 +20,11 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
     in_dtype = torch.bfloat16 if wl.compute == "bf16" else torch.float32
     for s in range(n_steps + 2 * P - 1):
         if s < n_steps:
-            if encoder:
+            if encoder and is_encdec(wl):
+                src, dec_in, tg = I.seq2seq_batch(wl, s)               # two token streams: [source | decoder input]
+                xd = torch.from_numpy(np.concatenate([src, dec_in]).astype(np.int32)).to(pipe.device)
+                yd = torch.from_numpy(tg.astype(np.int32)).to(pipe.device)
+            elif encoder:
                 ids, tg = I.token_batch(wl, s)
                 xd = torch.from_numpy(ids.astype(np.int32)).to(pipe.device)
                 yd = torch.from_numpy(tg.astype(np.int32)).to(pipe.device)
@@ -44,10 +48,15 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
     return pipe, losses, book
 
 
+def is_encdec(wl):
+    return any(sp.pre == "embed_dec" for sp in wl.stage_specs)
+
+
 def run_oracle(wl, params0, n_steps, teacher=None):
     if wl.kind == "encoder":
         from oracle import transformer
-        return transformer.run_workload(wl, params0, lambda t: I.token_batch(wl, t), n_steps=n_steps)
+        data = (lambda t: I.seq2seq_batch(wl, t)) if is_encdec(wl) else (lambda t: I.token_batch(wl, t))
+        return transformer.run_workload(wl, params0, data, n_steps=n_steps)
     from oracle.mlp import run_workload
     teacher = I.teacher_params(wl) if teacher is None else teacher
     return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps)
@@ -83,6 +92,11 @@ def compare_params(pipe, res, tol, per_stage=False):
                     assert np.abs(a[d:2 * d]).max() <= bound and np.abs(ref[d:2 * d]).max() <= bound
                     keep = np.r_[0:d, 2 * d:3 * d]
                     a, ref = a[keep], ref[keep]
+                if sp.post == "cross_attention" and j == len(stage) - 1:
+                    d = sp.n_out // 2                            # [k | v]: the same gauge direction, first half
+                    bound = wl.alpha * len(res.losses) * 1.01 + 1e-12
+                    assert np.abs(a[:d]).max() <= bound and np.abs(ref[:d]).max() <= bound
+                    a, ref = a[d:], ref[d:]
                 scale = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p]) if per_stage else None
                 e = max_rel_err(a, ref) if scale is None else float(np.abs(a - ref).max() / scale)
                 worst = max(worst, e)

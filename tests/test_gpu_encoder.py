@@ -69,3 +69,17 @@ def test_encoder_tensor_core_attention_shape(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("tc attention worst relative weight error (per stage vector)", worst)
+
+
+# ---- encoder-decoder stages: causal self-attention, cross-attention over the encoder memory, two-stage skips ----------
+
+@pytest.mark.parametrize("kw", [dict(n_enc=1, n_dec=1), dict(n_enc=2, n_dec=2, d_model=32, d_ff=64, seq_len=8, batch=2, vocab=40, steps=14)])
+def test_encoder_decoder_fp32(cuda_device, kw):
+    wl = I.cfg5_small(compute="f32", **kw)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
+    worst = compare_params(pipe, res, 2e-5)
+    print("encoder-decoder fp32 worst relative weight error", worst)
