@@ -24,7 +24,9 @@ constexpr int AT_FWD_SMEM = 3 * AT_TILE + 2 * AT_TILE + 1024 + 128;
 constexpr int AT_BWD_SMEM = 5 * AT_TILE + 1024 + 128 + 3 * 2 * AT_S * 4;   // Q, K, dO, V|P0|dS0, P1|dS1, row-statistics exchange: two CTAs per SM
 constexpr int AT_TMEM_COLS = 256;
 
-enum { AMAP_QKV = 0, AMAP_DO = 1, AMAPS_PER_STAGE = 2 };
+// per attention stage: the tensor holding q (the Linear's [q | k | v] output, or for cross-attention the stage's main
+// input ring), the tensor holding k, v (the Linear's output), and the incoming-gradient mailbox
+enum { AMAP_Q = 0, AMAP_KV = 1, AMAP_DO = 2, AMAPS_PER_STAGE = 3 };
 
 __device__ __forceinline__ void issue_k64(uint32_t tmem_d, uint32_t a, uint32_t b, uint32_t idesc, bool a_kmajor, bool b_kmajor,
                                           uint32_t a_lbo, uint32_t b_lbo, bool acc_first) {
@@ -90,11 +92,13 @@ __device__ __forceinline__ bool wait_mma(const AttnCommon& c, uint32_t parity, i
   return ok;
 }
 
-__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int causal, int* status) {
+__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int* status) {
   const int p = stage_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
-  if (d.f_mb < 0 || s.post != POST_ATTENTION) return;
+  if (d.f_mb < 0 || !feeds_attention(s.post)) return;
+  const bool cross = s.post == POST_CROSS_ATTENTION;         // q = the stage's main input; the Linear gave [k | v]
+  const int causal = s.causal;
   const int H = s.n_heads, dm = s.d_out_main;
   if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
@@ -108,10 +112,11 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
   const int warp = r >> 5;
 
   if (r == 0) {
+    const int ko = cross ? 0 : dm;                           // column of k inside the Linear's output
     mbar_arrive_expect_tx(c.bar_load, 3 * AT_TILE);
-    tma_load_3d(sQ, lm + AMAP_QKV, c.bar_load, h * AT_DK, b * AT_S, d.f_slot);
-    tma_load_3d(sK, lm + AMAP_QKV, c.bar_load, dm + h * AT_DK, b * AT_S, d.f_slot);
-    tma_load_3d(sV, lm + AMAP_QKV, c.bar_load, 2 * dm + h * AT_DK, b * AT_S, d.f_slot);
+    tma_load_3d(sQ, lm + AMAP_Q, c.bar_load, h * AT_DK, b * AT_S, cross ? d.f_xslot : d.f_slot);
+    tma_load_3d(sK, lm + AMAP_KV, c.bar_load, ko + h * AT_DK, b * AT_S, d.f_slot);
+    tma_load_3d(sV, lm + AMAP_KV, c.bar_load, ko + dm + h * AT_DK, b * AT_S, d.f_slot);
     if (mbar_wait(c.bar_load, 0, c.abort_flag, status, 11)) {
       tc_fence_after();
       issue_k64(tmem_base, sQ, sK, make_idesc_mn(128, 128, 0, 0), true, true, 0, 0, false);   // S = Q K^T
@@ -199,11 +204,13 @@ __device__ __forceinline__ void attn_store32(__nv_bfloat16* dst, const uint32_t 
   }
 }
 
-__global__ void __launch_bounds__(AT_BWD_THREADS, 2) attn_bwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int causal, int* status) {
+__global__ void __launch_bounds__(AT_BWD_THREADS, 2) attn_bwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int* status) {
   const int p = stage_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
-  if (d.b_mb < 0 || s.post != POST_ATTENTION) return;
+  if (d.b_mb < 0 || !feeds_attention(s.post)) return;
+  const bool cross = s.post == POST_CROSS_ATTENTION;
+  const int causal = s.causal;
   const int H = s.n_heads, dm = s.d_out_main;
   if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
@@ -219,11 +226,12 @@ __global__ void __launch_bounds__(AT_BWD_THREADS, 2) attn_bwd_tc_kernel(TickArgs
   const int warp = tid >> 5;
 
   if (tid == 0) {
+    const int ko = cross ? 0 : dm;
     mbar_arrive_expect_tx(c.bar_load, 4 * AT_TILE);
-    tma_load_3d(sQ, lm + AMAP_QKV, c.bar_load, h * AT_DK, b * AT_S, d.b_slot);
-    tma_load_3d(sK, lm + AMAP_QKV, c.bar_load, dm + h * AT_DK, b * AT_S, d.b_slot);
-    tma_load_3d(sV, lm + AMAP_QKV, c.bar_load, 2 * dm + h * AT_DK, b * AT_S, d.b_slot);
-    tma_load_3d(sdO, lm + AMAP_DO, c.bar_load, h * AT_DK, b * AT_S, (int)((d.tick + 2) % 3));
+    tma_load_3d(sQ, lm + AMAP_Q, c.bar_load, h * AT_DK, b * AT_S, cross ? d.b_xslot : d.b_slot);
+    tma_load_3d(sK, lm + AMAP_KV, c.bar_load, ko + h * AT_DK, b * AT_S, d.b_slot);
+    tma_load_3d(sV, lm + AMAP_KV, c.bar_load, ko + dm + h * AT_DK, b * AT_S, d.b_slot);
+    tma_load_3d(sdO, lm + AMAP_DO, c.bar_load, h * AT_DK, b * AT_S, gin_slot_read(s, d));
     if (mbar_wait(c.bar_load, 0, c.abort_flag, status, 14)) {
       tc_fence_after();
       const uint32_t idesc = make_idesc_mn(128, 128, 0, 0);
@@ -315,23 +323,26 @@ __global__ void __launch_bounds__(AT_BWD_THREADS, 2) attn_bwd_tc_kernel(TickArgs
         issue_k64(tmem_base + 128, sP + 4 * 2048, sQ + 4 * 2048, i_mm, false, false, AT_TILE, 8192, true);
         tc_commit(c.bar_mma);
       }
-      // results go to the stage's dy buffer as [dq | dk | dv]; this thread stores 32 of the 64 head columns
-      __nv_bfloat16* dy = reinterpret_cast<__nv_bfloat16*>(t.ws + s.dy) + (size_t)(b * AT_S + r) * 3 * dm + h * AT_DK + hf * 32;
+      // self-attention: the stage's dy buffer receives [dq | dk | dv]; cross-attention: dy = [dk | dv] and dq goes
+      // to the previous stage's gradient mailbox.  This thread stores 32 of the 64 head columns.
+      const int wz = cross ? 2 * dm : 3 * dm, ko = cross ? 0 : dm;
+      __nv_bfloat16* dy = reinterpret_cast<__nv_bfloat16*>(t.ws + s.dy) + (size_t)(b * AT_S + r) * wz + h * AT_DK + hf * 32;
+      __nv_bfloat16* dq = cross ? gin_write_prev<__nv_bfloat16>(t, p, d) + (size_t)(b * AT_S + r) * dm + h * AT_DK + hf * 32 : dy;
       {
         uint32_t o[32];
         tc_fence_after();
         tmem_ld32(lane_addr + hf * 32, o);                   // dV while dQ and dK are being computed
         tmem_ld_wait();
-        attn_store32(dy + 2 * dm, o, 1.0f);
+        attn_store32(dy + ko + dm, o, 1.0f);
       }
       if (wait_mma(c, 0, status, 17)) {
         uint32_t o[32];
         tmem_ld32(lane_addr + 64 + hf * 32, o);
         tmem_ld_wait();
-        attn_store32(dy, o, scale);
+        attn_store32(dq, o, scale);
         tmem_ld32(lane_addr + 128 + hf * 32, o);
         tmem_ld_wait();
-        attn_store32(dy + dm, o, scale);
+        attn_store32(dy + ko, o, scale);
       }
     }
   }
@@ -366,25 +377,25 @@ pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<
   std::vector<CUtensorMap> maps((size_t)t.P * AMAPS_PER_STAGE);
   memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
   std::vector<int> ids;
-  for (int p = 0; p < t.P; ++p) if (st[p].post == POST_ATTENTION) ids.push_back(p);
+  for (int p = 0; p < t.P; ++p) if (feeds_attention(st[p].post)) ids.push_back(p);
   const cuuint64_t T = (cuuint64_t)t.T;
   for (int p = 0; p < t.P; ++p) {
     const StageDev& s = st[p];
-    if (s.post != POST_ATTENTION) continue;
-    const cuuint64_t d3 = (cuuint64_t)s.lin[0].n_out, dm = (cuuint64_t)s.d_out_main;
+    if (!feeds_attention(s.post)) continue;
+    const bool cross = s.post == POST_CROSS_ATTENTION;
+    const cuuint64_t dz = (cuuint64_t)s.lin[0].n_out, dm = (cuuint64_t)s.d_out_main;
     cuuint32_t box[3] = {AT_DK, AT_S, 1}, es[3] = {1, 1, 1};
-    {
-      cuuint64_t dims[3] = {d3, T, (cuuint64_t)s.depth}, strides[2] = {d3 * 2, T * d3 * 2};
-      CUresult r = fn(&maps[(size_t)p * AMAPS_PER_STAGE + AMAP_QKV], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, t.ring + s.lin[0].z_ring, dims, strides,
+    auto enc = [&](int which, void* base, cuuint64_t width, cuuint64_t slots, const char* what) -> bool {
+      cuuint64_t dims[3] = {width, T, slots}, strides[2] = {width * 2, T * width * 2};
+      CUresult r = fn(&maps[(size_t)p * AMAPS_PER_STAGE + which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides,
                       box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-      if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled (attention qkv) failed with code " + std::to_string((int)r); return PM_ERR_CUDA; }
-    }
-    {
-      cuuint64_t dims[3] = {dm, T, 3}, strides[2] = {dm * 2, T * dm * 2};
-      CUresult r = fn(&maps[(size_t)p * AMAPS_PER_STAGE + AMAP_DO], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, t.ws + s.gin, dims, strides,
-                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-      if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled (attention dO) failed with code " + std::to_string((int)r); return PM_ERR_CUDA; }
-    }
+      if (r != CUDA_SUCCESS) { err = std::string("cuTensorMapEncodeTiled (attention ") + what + ") failed with code " + std::to_string((int)r); return false; }
+      return true;
+    };
+    if (!enc(AMAP_KV, t.ring + s.lin[0].z_ring, dz, (cuuint64_t)s.depth, "k, v")) return PM_ERR_CUDA;
+    if (cross) { if (!enc(AMAP_Q, t.ring + s.x_ring, dm, (cuuint64_t)s.xdepth, "q")) return PM_ERR_CUDA; }
+    else if (!enc(AMAP_Q, t.ring + s.lin[0].z_ring, dz, (cuuint64_t)s.depth, "q")) return PM_ERR_CUDA;
+    if (!enc(AMAP_DO, t.ws + s.gin, dm, (cuuint64_t)s.gin_depth, "dO")) return PM_ERR_CUDA;
   }
   char* region = (char*)ws_region;
   cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream);
@@ -409,8 +420,8 @@ int* attn_status_word(AttnPlan* plan) { return plan ? plan->d_status : nullptr; 
 cudaError_t attn_tc_launch(AttnPlan* plan, const TickArgs& t, bool forward, cudaStream_t stream) {
   if (plan->n_att == 0) return cudaSuccess;
   dim3 grid(t.att_blocks, plan->n_att);
-  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, 0, plan->d_status);
-  else attn_bwd_tc_kernel<<<grid, AT_BWD_THREADS, AT_BWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, 0, plan->d_status);
+  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
+  else attn_bwd_tc_kernel<<<grid, AT_BWD_THREADS, AT_BWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
   return cudaGetLastError();
 }
 

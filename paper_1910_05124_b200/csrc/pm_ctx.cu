@@ -232,9 +232,9 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.gmem_depth = P - L.mem_stage + 2;
     L.mem_ring = ring; ring = align_up(ring + (uint64_t)L.mem_depth * T * L.mem_dim * esz, 256);
   }
-  L.att_tc = L.att_blocks > 0 && L.att_plain;      // the tensor-core kernels cover plain self-attention
+  L.att_tc = L.att_blocks > 0;
   for (int p = 0; p < P; ++p)
-    if (L.st[p].post == POST_ATTENTION && !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads)) L.att_tc = false;
+    if (feeds_attention(L.st[p].post) && !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads)) L.att_tc = false;
   if (L.att_blocks > 0 && !L.att_tc && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
   L.ring_bytes = ring;
   L.total = L.st[P - 1].end;

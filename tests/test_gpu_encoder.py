@@ -83,3 +83,29 @@ def test_encoder_decoder_fp32(cuda_device, kw):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
     worst = compare_params(pipe, res, 2e-5)
     print("encoder-decoder fp32 worst relative weight error", worst)
+
+
+def test_encoder_decoder_bf16_small(cuda_device):
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=2)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("encoder-decoder bf16 loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("encoder-decoder bf16 worst relative weight error (per stage vector)", worst)
+
+
+def test_encoder_decoder_tensor_core_attention_shape(cuda_device):
+    """Sequences of 128 tokens and heads of width 64: causal self-attention and cross-attention run on the
+    tensor-core kernels."""
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=128, n_heads=2, d_ff=256, seq_len=128, batch=2, vocab=200, steps=10)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("enc-dec tc attention loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("enc-dec tc attention worst relative weight error (per stage vector)", worst)
