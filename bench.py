@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the PipeMare hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg3|cfg1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg5|cfg3|cfg1]
 
 A step is one pipeline tick in steady state: every stage runs one forward with the weights it holds, one
 backward against the discrepancy-corrected weights for the microbatch that entered it tau_i updates ago, and
@@ -141,6 +141,10 @@ WORKLOADS = {
             "T1 (K=32) + T2 (D=0.5), tau=(7,5,3,1)",
     "cfg3": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master weights, microbatch 128, "
             "SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
+    "cfg5": "cfg5 cut to 4 + 4 layers: Transformer encoder-decoder, d_model 1024, 16 heads, FFN 4096, 32 sequences x 128 "
+            "tokens per microbatch, vocabulary 32000 (Zipf ids), bf16 GEMMs, fp32 master weights, one stage per weight GEMM "
+            "(45 stages), Adam(0.9, 0.98), T1 (K=1000) + T2 (D=0.1), tau_i=2(45-i)+1; the full 12 + 12 layers (133 stages) "
+            "need 553 GB of activation rings and sequences of 256 tokens need attention kernels that are not built",
     "cfg4": "cfg4: Transformer encoder, 6 layers, d_model 512, 8 heads, FFN 2048, 32 sequences x 128 tokens per "
             "microbatch, vocabulary 8192, bf16 GEMMs, fp32 master weights, one stage per weight GEMM (25 stages), "
             "Adam(0.9, 0.98), T1 (K=100) + T2 (D=0.1), tau_i=2(25-i)+1",
@@ -156,6 +160,11 @@ def build_workload(args):
             wl = I.encoder_workload(wl.name + f"_{args.stages}layers", args.stages, 512, 8, 2048, 128, 32, 8192, compute="bf16",
                                     optimizer="adam", alpha=wl.alpha, beta1=0.9, beta2=0.98, eps=1e-8, K=wl.K, D=wl.D,
                                     steps=wl.steps, seed=wl.seed)
+        params0 = I.init_encoder_params(wl)
+        n_params = sum(int(a.size) for st in params0 for a in st)
+        return wl, params0, wl.microbatch // wl.seq_len, n_params
+    if args.workload == "cfg5":
+        wl = I.cfg5_cut(args.stages, args.stages) if args.stages else I.cfg5_cut()
         params0 = I.init_encoder_params(wl)
         n_params = sum(int(a.size) for st in params0 for a in st)
         return wl, params0, wl.microbatch // wl.seq_len, n_params
@@ -179,8 +188,13 @@ def make_batches(wl, n, device):
     if wl.kind == "encoder":
         import numpy as np
         host = []
+        encdec = any(sp.pre == "embed_dec" for sp in wl.stage_specs)
         for t in range(n):
-            ids, tg = I.token_batch(wl, t)
+            if encdec:                                         # two token streams: [source | decoder input]
+                src, dec_in, tg = I.seq2seq_batch(wl, t)
+                ids = np.concatenate([src, dec_in])
+            else:
+                ids, tg = I.token_batch(wl, t)
             host.append((torch.from_numpy(ids.astype(np.int32)).pin_memory(), torch.from_numpy(tg.astype(np.int32)).pin_memory()))
         return host, [(x.to(device), y.to(device)) for x, y in host]
     teacher = I.teacher_params(wl)
@@ -201,7 +215,8 @@ def cpu_baseline(wl, n_steps, samples_per_step):
     if wl.kind == "encoder":
         from oracle.transformer import run_workload
         params0 = I.init_encoder_params(wl)
-        batches = [I.token_batch(wl, t) for t in range(n_steps)]
+        encdec = any(sp.pre == "embed_dec" for sp in wl.stage_specs)
+        batches = [I.seq2seq_batch(wl, t) if encdec else I.token_batch(wl, t) for t in range(n_steps)]
     else:
         from oracle.mlp import run_workload
         params0 = I.init_stage_params(wl)
@@ -490,7 +505,7 @@ def run_cuda(args):
     res = measure(args, args.workload, world, rank, local, device, sampler)
     others = []
     if world == 1 and not args.no_other and not args.stages:
-        for name in ("cfg4", "cfg3", "cfg1"):
+        for name in ("cfg5", "cfg4", "cfg3", "cfg1"):
             if name != args.workload:
                 others.append((name, measure(args, name, world, rank, local, device, None, with_e2e=False)))
     if rank != 0:
@@ -529,7 +544,8 @@ def run_cuda(args):
             "kernel_ms_per_step": {k: round(v, 5) for k, v in sorted(other["per_tick_ms"].items(), key=lambda kv: -kv[1])}})
     if world == 1:
         if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, res["samples_per_step"])
+            line["cpu_baseline"] = cpu_baseline(wl, 2 if args.workload == "cfg3" else 1, res["samples_per_step"]) \
+                if args.workload != "cfg5" else None         # one full-width cfg5 step takes minutes on the host: see --impl reference
         if not args.no_sweep:
             line["update_sweep"] = update_sweep(device, hbm_peak)
     print(json.dumps(line), flush=True)
@@ -577,6 +593,38 @@ def run_reference(args):
         samples_per_step = full.microbatch
         sample = (f"each step: one microbatch of 128 through {n_stages} of the {full.n_stages} stages "
                   f"(forward, backward, update); samples/s scaled by {n_stages}/{full.n_stages}")
+    elif args.workload == "cfg5":
+        from oracle.transformer import run_workload
+        full = I.cfg5_cut()
+
+        def sub(layers, seqs):
+            wl_ = I.cfg5_cut(layers, layers, batch=seqs)
+            wl_.steps = total_steps
+            return wl_
+
+        def mm_flops(layers, seqs):
+            enc = 1024 * (3072 + 1024 + 4096 + 4096)
+            dec = 1024 * (3072 + 1024 + 1024 + 2048 + 1024 + 4096 + 4096)
+            return 6.0 * seqs * 128 * (layers * (enc + dec) + 1024 * 32000)
+        wl1 = sub(1, 1)
+        p1 = I.init_encoder_params(wl1)
+        b1 = I.seq2seq_batch(wl1, 0)
+        t0 = time.perf_counter()
+        run_workload(wl1, p1, lambda t: b1, n_steps=1)
+        per_flop = (time.perf_counter() - t0) / mm_flops(1, 1)
+        layers, seqs = 4, 32
+        while layers > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
+            layers -= 1
+        while seqs > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
+            seqs //= 2
+        wl = sub(layers, seqs)
+        params0 = I.init_encoder_params(wl)
+        batches = [I.seq2seq_batch(wl, t) for t in range(min(total_steps, 4))]
+        scale = mm_flops(layers, seqs) / mm_flops(4, 32)
+        samples_per_step = 32
+        sample = (f"each step: {seqs} of the 32 sequences through {layers} + {layers} of the 4 + 4 layers plus embedding and "
+                  f"vocabulary stages (forward, backward, update); samples/s scaled by the sampled fraction "
+                  f"{scale:.5f} of the workload's matrix-product FLOPs")
     else:
         from oracle.transformer import run_workload
         full = I.cfg4()

@@ -109,3 +109,19 @@ def test_encoder_decoder_tensor_core_attention_shape(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("enc-dec tc attention worst relative weight error (per stage vector)", worst)
+
+
+def test_cfg5_widths_first_microbatches(cuda_device):
+    """Config 5's widths (d_model 1024, 16 heads, FFN 4096, 32 sequences of 128 tokens) on one encoder and one
+    decoder layer with a vocabulary of 4096: two microbatches fed and drained.  Every GEMM runs on the CTA-pair
+    kernels, attention (self, causal, cross) on the tensor-core kernels."""
+    wl = I.cfg5_cut(1, 1, vocab=4096)
+    n = 2
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, n)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, n)
+    check_book(book, res, n, wl.n_stages)
+    print("cfg5 widths loss relative errors", np.abs(losses / np.array(res.losses) - 1))
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("cfg5 widths worst relative weight error (per stage vector)", worst)
