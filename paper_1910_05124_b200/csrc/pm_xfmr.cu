@@ -393,6 +393,11 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
         for (int e = 0; e < 8; ++e) mx = fmaxf(mx, v[k][e]);
       }
     }
+  } else if ((V & 3) == 0) {                                 // long rows: three vectorised passes, the re-reads hit L2
+    for (int c = threadIdx.x * 4; c < V; c += 4 * blockDim.x) {
+      const float4 q = *reinterpret_cast<const float4*>(lg + c);
+      mx = fmaxf(fmaxf(mx, fmaxf(q.x, q.y)), fmaxf(q.z, q.w));
+    }
   } else {
     for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, lg[c]);
   }
@@ -410,6 +415,11 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) { v[k][e] = expf(v[k][e] - mx); sum += v[k][e]; }
       }
+  } else if ((V & 3) == 0) {
+    for (int c = threadIdx.x * 4; c < V; c += 4 * blockDim.x) {
+      const float4 q = *reinterpret_cast<const float4*>(lg + c);
+      sum += expf(q.x - mx); sum += expf(q.y - mx); sum += expf(q.z - mx); sum += expf(q.w - mx);
+    }
   } else {
     for (int c = threadIdx.x; c < V; c += blockDim.x) sum += expf(lg[c] - mx);
   }
@@ -435,6 +445,17 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
         }
         store8<AT>(dl + c, o);
       }
+    }
+  } else if ((V & 3) == 0) {
+    for (int c = threadIdx.x * 4; c < V; c += 4 * blockDim.x) {
+      const float4 q = *reinterpret_cast<const float4*>(lg + c);
+      float p0 = expf(q.x - mx) / sum, p1 = expf(q.y - mx) / sum, p2 = expf(q.z - mx) / sum, p3 = expf(q.w - mx) / sum;
+      if (tgt == c) p0 -= 1.0f;
+      if (tgt == c + 1) p1 -= 1.0f;
+      if (tgt == c + 2) p2 -= 1.0f;
+      if (tgt == c + 3) p3 -= 1.0f;
+      dl[c] = from_f<AT>(p0 * invT); dl[c + 1] = from_f<AT>(p1 * invT);
+      dl[c + 2] = from_f<AT>(p2 * invT); dl[c + 3] = from_f<AT>(p3 * invT);
     }
   } else {
     for (int c = threadIdx.x; c < V; c += blockDim.x) {
@@ -811,8 +832,11 @@ static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
 // A block owns kEmbRows consecutive vocabulary rows.  It walks the microbatch's token ids once, in order, and
 // compacts the tokens that fall into its rows into a list (ballot + prefix over the warps, so the list is in
 // ascending token order); each warp then takes kEmbRows / 8 rows, picks its tokens from the list in order and
-// streams the columns.  Every row is written (zeros included) and the order of the additions is fixed.
+// streams the columns.  A row with many tokens (frequent ids under a Zipf distribution) is shared by the eight
+// warps: each adds a contiguous segment of the row's tokens in order, and the eight partial sums are added in warp
+// order.  Every row is written (zeros included) and the order of the additions is fixed.
 constexpr int kEmbRows = 32;
+constexpr int kEmbHeavy = 24;                         // tokens per row from which the block shares the row
 
 template <typename AT>
 __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
@@ -824,6 +848,10 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   if (v0 >= s.vocab) return;
   extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
   __shared__ int warp_cnt[2][8];
+  __shared__ int row_cnt[kEmbRows];
+  __shared__ float part[8][512];                             // heavy rows: per-warp partial sums of one 512-column pass
+  if (threadIdx.x < kEmbRows) row_cnt[threadIdx.x] = 0;
+  __syncthreads();
   const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, (int)(d.b_mb % s.ids_depth), (uint64_t)t.T);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int nh = 0;                                                // hits so far (the same value in every thread)
@@ -844,7 +872,7 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
       int base = nh, tot = 0;
 #pragma unroll
       for (int w = 0; w < 8; ++w) { const int cw = warp_cnt[k & 1][w]; if (w < warp) base += cw; tot += cw; }
-      if (hit) hits[base + __popc(bal & ((1u << lane) - 1u))] = ((tb0 + k * 256 + (int)threadIdx.x) << 8) | rel[k];
+      if (hit) { hits[base + __popc(bal & ((1u << lane) - 1u))] = ((tb0 + k * 256 + (int)threadIdx.x) << 8) | rel[k]; atomicAdd(&row_cnt[rel[k]], 1); }
       nh += tot;
     }
   }
@@ -853,9 +881,60 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   const AT* du = ws_at<AT>(t, s.dh);
   const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
   const float sc = sqrtf((float)dm);
+  // ---- rows with many tokens: the whole block per row
+  for (int rr = 0; rr < kEmbRows; ++rr) {
+    const int cnt = row_cnt[rr];
+    if (cnt < kEmbHeavy || v0 + rr >= s.vocab) continue;     // uniform over the block
+    const int k_lo = (int)((long long)cnt * warp / 8), k_hi = (int)((long long)cnt * (warp + 1) / 8);   // this warp's tokens of the row
+    float* out = t.a.grad + s.tab_off + (uint64_t)(v0 + rr) * dm;
+    for (int c0 = 0; c0 < dm; c0 += 32 * 16) {
+      float acc[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+      int seen = 0;                                          // tokens of this row before the current group of 32 list entries
+      for (int hb = 0; hb < nh && seen < k_hi; hb += 32) {
+        const int hv = hb + lane < nh ? hits[hb + lane] : -1;
+        unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
+        const int n_here = __popc(mine);
+        int idx = seen;
+        seen += n_here;
+        if (seen <= k_lo) continue;
+        while (mine) {
+          const int j = __ffs(mine) - 1;
+          mine &= mine - 1;
+          const int my = idx++;
+          if (my < k_lo || my >= k_hi) continue;
+          const uint64_t ro = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm;
+          float val[16], sv[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) val[e] = to_f<AT>(du[ro + min(c0 + e * 32 + lane, dm - 1)]);
+          if (gs) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) sv[e] = to_f<AT>(gs[ro + min(c0 + e * 32 + lane, dm - 1)]);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) val[e] = __fadd_rn(val[e], sv[e]);
+          }
+#pragma unroll
+          for (int e = 0; e < 16; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[e], sc));
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) part[warp][e * 32 + lane] = acc[e];
+      __syncthreads();
+      for (int c = threadIdx.x; c < 512 && c0 + c < dm; c += 256) {
+        float a = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) a = __fadd_rn(a, part[w][c]);
+        out[c0 + c] = a;
+      }
+      __syncthreads();
+    }
+  }
+  // ---- the other rows: one warp per row
   for (int rr = warp; rr < kEmbRows; rr += 8) {
     const int v = v0 + rr;
     if (v >= s.vocab) break;
+    if (row_cnt[rr] >= kEmbHeavy) continue;
     float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
     for (int c0 = 0; c0 < dm; c0 += 32 * 16) {               // up to 16 columns per lane per pass
       float acc[16];
