@@ -66,7 +66,8 @@ enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
 /* One operator of a stage.  A stage is  [EMBED | LAYERNORM]  LINEAR{1..PM_MAX_LINEARS}  [ATTENTION | SKIP_OUT |
  * RESIDUAL]  (with a pre- or post-op exactly one LINEAR).
  *   LINEAR     y = act(x W^T + b), W is [n_out, n_in] row-major, b is [n_out].
- *   EMBED      x = table[id] * sqrt(n_out) + sinusoidal position; table is [n_in = vocabulary, n_out = width];
+ *   EMBED      x = table[id] * sqrt(n_out) + sinusoidal position; table is [n_in = vocabulary, n_out = width, a
+ *              multiple of four];
  *              the stage's input is int32 token ids: the first stage embeds the first stream; a later stage with
  *              PM_OPF_SECOND_STREAM (the first stage of a decoder) embeds the second and ignores the previous
  *              stage's output.  seq_len gives the position period.

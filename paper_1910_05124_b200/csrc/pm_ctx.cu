@@ -106,7 +106,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       s.ids_stream = second ? 1 : 0;
       s.ids_depth = 2 * P - p;
       if (second) L.n_streams = 2;
-      if (op.n_in < 1 || op.n_out < 2 || (op.n_out & 1) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (even width, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
+      if (op.n_in < 1 || op.n_out < 4 || (op.n_out & 3) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (width a multiple of four, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
       s.pre = PRE_EMBED; s.vocab = op.n_in; s.seq_len = op.seq_len;
       uint64_t dummy; offsets(0, &s.tab_off, &dummy);
       L.pe_seq = op.seq_len; L.pe_d = op.n_out;
@@ -470,7 +470,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
   t.any_pre = L.any_pre; t.any_ln = L.any_ln; t.any_embed = L.any_embed; t.any_residual = L.any_residual;
-  t.att_S = L.att_S; t.att_dk = L.att_dk; t.att_blocks = L.att_blocks; t.max_vocab = L.max_vocab;
+  t.att_S = L.att_S; t.att_dk = L.att_dk; t.att_blocks = L.att_blocks; t.max_vocab = L.max_vocab; t.max_embed_dim = L.pe_d;
   {
     const int32_t* ids = (const int32_t*)(c->ws + L.off_ids);
     t.pre_ids = ids; t.ln_ids = ids + P; t.embed_ids = ids + 2 * P; t.res_ids = ids + 3 * P;

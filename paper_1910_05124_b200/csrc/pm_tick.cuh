@@ -23,7 +23,7 @@ struct TickArgs {
   int32_t loss_kind;      // PM_LOSS_*
   int32_t any_pre, any_ln, any_embed, any_residual;   // which grouped launches this pipeline needs
   int32_t att_S, att_dk, att_blocks;                   // attention: sequence length, head width, (sequences x heads); 0 = none
-  int32_t max_vocab;
+  int32_t max_vocab, max_embed_dim;
   uint64_t loss_off;      // ws: loss log [loss_cap] float
   uint64_t lossred_off;   // ws: per-block loss partials [64] float + completion counter
   int64_t loss_cap;

@@ -677,7 +677,7 @@ __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
 // rows w, w+8, ... in ascending order, a lane owns 8 consecutive columns per 256-column group; per-warp partials are
 // added in warp order, per-block partials in block order by ln_fused_finish_kernel.
 template <typename AT, int NP>
-__global__ void __launch_bounds__(256) ln_bwd_fused_kernel(TickArgs t) {
+__global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(TickArgs t) {
   const int li = blockIdx.y, p = t.ln_ids[li];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
@@ -829,31 +829,108 @@ static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
 }
 
 // Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
-// A block owns kEmbRows consecutive vocabulary rows.  It walks the microbatch's token ids once, in order, and
-// compacts the tokens that fall into its rows into a list (ballot + prefix over the warps, so the list is in
-// ascending token order); each warp then takes kEmbRows / 8 rows, picks its tokens from the list in order and
-// streams the columns.  A row with many tokens (frequent ids under a Zipf distribution) is shared by the eight
-// warps: each adds a contiguous segment of the row's tokens in order, and the eight partial sums are added in warp
-// order.  Every row is written (zeros included) and the order of the additions is fixed.
-constexpr int kEmbRows = 32;
+// A block owns kEmbRows consecutive vocabulary rows and kEmbCols columns.  It walks the microbatch's token ids
+// once, in order, and compacts the tokens that fall into its rows into a list (ballot + prefix over the warps, so
+// the list is in ascending token order).  A row with few tokens is summed by one warp; a row with many (frequent
+// ids under a Zipf distribution) by all eight, each adding a contiguous segment of the row's tokens in order, the
+// eight partial sums then added in warp order.  Tokens are gathered eight at a time so that their loads are in
+// flight together.  Every row is written (zeros included) and the order of the additions is fixed.
+constexpr int kEmbRows = 32;                          // a block's columns: 32 lanes x CPL (4, 8 or 16) columns per lane
 constexpr int kEmbHeavy = 24;                         // tokens per row from which the block shares the row
 
-template <typename AT>
+template <typename AT> __device__ __forceinline__ void load4(const AT* p, float (&v)[4]);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float (&v)[4]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[4]) {
+  const uint2 q = *reinterpret_cast<const uint2*>(p);
+  const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&q.x));
+  const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&q.y));
+  v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+
+template <typename AT, int CPL> __device__ __forceinline__ void load_cols(const AT* p, float (&v)[CPL]) {
+  if constexpr (CPL == 4) load4<AT>(p, v);
+  else {
+#pragma unroll
+    for (int h = 0; h < CPL / 8; ++h) {
+      float w[8];
+      load8<AT>(p + 8 * h, w);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[8 * h + e] = w[e];
+    }
+  }
+}
+
+// adds, in list order, the rows of the tokens number k_lo .. k_hi-1 (counted among the list entries of row rr) to acc;
+// 32 / CPL tokens are gathered at a time
+template <typename AT, int CPL>
+__device__ __forceinline__ void embed_gather(const int32_t* hits, int nh, int rr, int k_lo, int k_hi, const AT* du, const AT* gs,
+                                             int dm, int col, float sc, int lane, float (&acc)[CPL]) {
+  constexpr int NB = 32 / CPL;
+  int seen = 0;
+  for (int hb = 0; hb < nh && seen < k_hi; hb += 32) {
+    const int hv = hb + lane < nh ? hits[hb + lane] : -1;
+    unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
+    int idx = seen;
+    seen += __popc(mine);
+    if (seen <= k_lo) continue;
+    while (mine) {                                           // NB tokens at a time: loads first, ordered additions after
+      uint64_t ro[NB];
+      bool use[NB];
+#pragma unroll
+      for (int u = 0; u < NB; ++u) {                         // no loads inside these branches (they would be serialised)
+        use[u] = false;
+        ro[u] = (uint64_t)col;                               // a valid address for the slots that stay empty
+        if (mine) {
+          const int j = __ffs(mine) - 1;
+          mine &= mine - 1;
+          const int my = idx++;
+          use[u] = my >= k_lo && my < k_hi;
+          ro[u] = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm + col;
+        }
+      }
+      float val[NB][CPL], sv[NB][CPL];
+#pragma unroll
+      for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(du + ro[u], val[u]);
+      if (gs) {
+#pragma unroll
+        for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(gs + ro[u], sv[u]);
+#pragma unroll
+        for (int u = 0; u < NB; ++u)
+#pragma unroll
+          for (int e = 0; e < CPL; ++e) val[u][e] = __fadd_rn(val[u][e], sv[u][e]);
+      }
+#pragma unroll
+      for (int u = 0; u < NB; ++u)
+        if (use[u]) {
+#pragma unroll
+          for (int e = 0; e < CPL; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[u][e], sc));
+        }
+    }
+  }
+}
+
+template <typename AT, int CPL>
 __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
+  constexpr int kEmbCols = 32 * CPL;
   const int p = t.embed_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0) return;
   const int v0 = blockIdx.x * kEmbRows;
-  if (v0 >= s.vocab) return;
+  const int dm = s.d_in;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col = blockIdx.z * kEmbCols + lane * CPL;        // this lane's columns
+  if (v0 >= s.vocab || blockIdx.z * kEmbCols >= dm) return;
   extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
   __shared__ int warp_cnt[2][8];
   __shared__ int row_cnt[kEmbRows];
-  __shared__ float part[8][512];                             // heavy rows: per-warp partial sums of one 512-column pass
+  __shared__ float part[8][kEmbCols];                        // shared rows: per-warp partial sums
   if (threadIdx.x < kEmbRows) row_cnt[threadIdx.x] = 0;
   __syncthreads();
   const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, (int)(d.b_mb % s.ids_depth), (uint64_t)t.T);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int nh = 0;                                                // hits so far (the same value in every thread)
   for (int tb0 = 0; tb0 < t.T; tb0 += 16 * 256) {            // 16 rounds of 256 tokens; the ids of all rounds are fetched first
     int rel[16];
@@ -877,98 +954,45 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
     }
   }
   __syncthreads();
-  const int dm = s.d_in;
   const AT* du = ws_at<AT>(t, s.dh);
   const AT* gs = emits_skip(s) ? gskip_read<AT>(t, p, d) : nullptr;
   const float sc = sqrtf((float)dm);
+  const bool col_ok = col < dm;                              // widths are multiples of CPL
+  const int col_ld = col_ok ? col : dm - CPL;                  // every lane takes part in the warp-wide steps; lanes beyond the width load a valid address
   // ---- rows with many tokens: the whole block per row
   for (int rr = 0; rr < kEmbRows; ++rr) {
     const int cnt = row_cnt[rr];
     if (cnt < kEmbHeavy || v0 + rr >= s.vocab) continue;     // uniform over the block
-    const int k_lo = (int)((long long)cnt * warp / 8), k_hi = (int)((long long)cnt * (warp + 1) / 8);   // this warp's tokens of the row
-    float* out = t.a.grad + s.tab_off + (uint64_t)(v0 + rr) * dm;
-    for (int c0 = 0; c0 < dm; c0 += 32 * 16) {
-      float acc[16];
+    const int k_lo = (int)((long long)cnt * warp / 8), k_hi = (int)((long long)cnt * (warp + 1) / 8);
+    float acc[CPL];
 #pragma unroll
-      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-      int seen = 0;                                          // tokens of this row before the current group of 32 list entries
-      for (int hb = 0; hb < nh && seen < k_hi; hb += 32) {
-        const int hv = hb + lane < nh ? hits[hb + lane] : -1;
-        unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
-        const int n_here = __popc(mine);
-        int idx = seen;
-        seen += n_here;
-        if (seen <= k_lo) continue;
-        while (mine) {
-          const int j = __ffs(mine) - 1;
-          mine &= mine - 1;
-          const int my = idx++;
-          if (my < k_lo || my >= k_hi) continue;
-          const uint64_t ro = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm;
-          float val[16], sv[16];
+    for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
+    embed_gather<AT, CPL>(hits, nh, rr, k_lo, k_hi, du, gs, dm, col_ld, sc, lane, acc);
 #pragma unroll
-          for (int e = 0; e < 16; ++e) val[e] = to_f<AT>(du[ro + min(c0 + e * 32 + lane, dm - 1)]);
-          if (gs) {
+    for (int e = 0; e < CPL; ++e) part[warp][lane * CPL + e] = acc[e];
+    __syncthreads();
+    for (int c = threadIdx.x; c < kEmbCols && blockIdx.z * kEmbCols + c < dm; c += 256) {
+      float a = 0.f;
 #pragma unroll
-            for (int e = 0; e < 16; ++e) sv[e] = to_f<AT>(gs[ro + min(c0 + e * 32 + lane, dm - 1)]);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) val[e] = __fadd_rn(val[e], sv[e]);
-          }
-#pragma unroll
-          for (int e = 0; e < 16; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[e], sc));
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 16; ++e) part[warp][e * 32 + lane] = acc[e];
-      __syncthreads();
-      for (int c = threadIdx.x; c < 512 && c0 + c < dm; c += 256) {
-        float a = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) a = __fadd_rn(a, part[w][c]);
-        out[c0 + c] = a;
-      }
-      __syncthreads();
+      for (int w = 0; w < 8; ++w) a = __fadd_rn(a, part[w][c]);
+      t.a.grad[s.tab_off + (uint64_t)(v0 + rr) * dm + blockIdx.z * kEmbCols + c] = a;
     }
+    __syncthreads();
   }
   // ---- the other rows: one warp per row
   for (int rr = warp; rr < kEmbRows; rr += 8) {
     const int v = v0 + rr;
     if (v >= s.vocab) break;
-    if (row_cnt[rr] >= kEmbHeavy) continue;
-    float* out = t.a.grad + s.tab_off + (uint64_t)v * dm;
-    for (int c0 = 0; c0 < dm; c0 += 32 * 16) {               // up to 16 columns per lane per pass
-      float acc[16];
+    const int cnt = row_cnt[rr];
+    if (cnt >= kEmbHeavy) continue;
+    float acc[CPL];
 #pragma unroll
-      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-      for (int hb = 0; hb < nh; hb += 32) {
-        const int hv = hb + lane < nh ? hits[hb + lane] : -1;
-        unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
-        while (mine) {
-          const int j = __ffs(mine) - 1;
-          mine &= mine - 1;
-          const uint64_t ro = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm;
-          // all loads of this token first (no branch between them), then the ordered additions
-          float val[16], sv[16];
+    for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
+    if (cnt > 0) embed_gather<AT, CPL>(hits, nh, rr, 0, cnt, du, gs, dm, col_ld, sc, lane, acc);
+    if (col_ok) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int c = min(c0 + e * 32 + lane, dm - 1);
-            val[e] = to_f<AT>(du[ro + c]);
-          }
-          if (gs) {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) sv[e] = to_f<AT>(gs[ro + min(c0 + e * 32 + lane, dm - 1)]);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) val[e] = __fadd_rn(val[e], sv[e]);
-          }
-#pragma unroll
-          for (int e = 0; e < 16; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[e], sc));
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const int c = c0 + e * 32 + lane;
-        if (c < dm) out[c] = acc[e];
-      }
+      for (int e = 0; e < CPL; e += 4)
+        *reinterpret_cast<float4*>(t.a.grad + s.tab_off + (uint64_t)v * dm + col + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
     }
   }
 }
@@ -995,10 +1019,20 @@ cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
     }
   }
   if (t.any_embed) {
-    dim3 g((t.max_vocab + kEmbRows - 1) / kEmbRows, t.n_embed);
+    // columns per lane: wide models are cut into column slices so that a row with many tokens is spread over blocks
+    const int dm = t.max_embed_dim;
+    const int cpl = (dm % 16 == 0 && dm <= 512) ? 16 : (dm % 8 == 0 ? 8 : 4);
+    dim3 g((t.max_vocab + kEmbRows - 1) / kEmbRows, t.n_embed, (dm + 32 * cpl - 1) / (32 * cpl));
     const size_t smem = sizeof(int32_t) * (size_t)t.T;
-    if (dtype == PM_F32) embed_bwd_kernel<float><<<g, 256, smem, stream>>>(t);
-    else embed_bwd_kernel<__nv_bfloat16><<<g, 256, smem, stream>>>(t);
+    if (dtype == PM_F32) {
+      if (cpl == 16) embed_bwd_kernel<float, 16><<<g, 256, smem, stream>>>(t);
+      else if (cpl == 8) embed_bwd_kernel<float, 8><<<g, 256, smem, stream>>>(t);
+      else embed_bwd_kernel<float, 4><<<g, 256, smem, stream>>>(t);
+    } else {
+      if (cpl == 16) embed_bwd_kernel<__nv_bfloat16, 16><<<g, 256, smem, stream>>>(t);
+      else if (cpl == 8) embed_bwd_kernel<__nv_bfloat16, 8><<<g, 256, smem, stream>>>(t);
+      else embed_bwd_kernel<__nv_bfloat16, 4><<<g, 256, smem, stream>>>(t);
+    }
     e = cudaGetLastError();
   }
   return e;
