@@ -69,6 +69,10 @@ struct StageDyn {
   int32_t active_update;
   float alpha, gamma, one_minus_gamma, bc1, bc2;
   int32_t use_delta;          // T2 on and gap > 0
+  int32_t gin_rslot;          // slot of this stage's gradient mailbox written during the previous tick
+  int32_t prev_wslot;         // slot of the previous stage's gradient mailbox this tick's backward writes
+  int32_t gmem_slot;          // slot of the memory-gradient ring of the microbatch in backward
+  int32_t _pad2;
 };
 
 // Hyper-parameters the schedule kernel needs.

@@ -224,12 +224,17 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     }
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
   }
-  for (int p = 0; p < P; ++p) L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
+  for (int p = 0; p < P; ++p) {
+    L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
+    L.sched[p].gin_depth = L.st[p].gin_depth;
+    L.sched[p].prev_gin_depth = p > 0 ? L.st[p - 1].gin_depth : 0;
+  }
   if (L.mem_stage >= 0) {
     if (L.last_mem_reader < 0) { err = "a memory is emitted but no CROSS_ATTENTION stage reads it"; return PM_ERR_UNSUPPORTED; }
     L.st[L.last_mem_reader].mem_first = 1;
     L.mem_depth = 2 * P - 2 * L.mem_stage;
     L.gmem_depth = P - L.mem_stage + 2;
+    for (int p = 0; p < P; ++p) L.sched[p].gmem_depth = L.gmem_depth;
     L.mem_ring = ring; ring = align_up(ring + (uint64_t)L.mem_depth * T * L.mem_dim * esz, 256);
   }
   L.att_tc = L.att_blocks > 0;

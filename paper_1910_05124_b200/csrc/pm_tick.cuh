@@ -62,16 +62,16 @@ template <typename AT> __device__ __forceinline__ const AT* lin_input(const Tick
   return ring_at<AT>(t, s.x_ring, fwd ? d.f_xslot : d.b_xslot, n);
 }
 // slot of a stage's gradient mailbox that holds what was written during the previous tick
-__device__ __forceinline__ int gin_slot_read(const StageDev& s, const StageDyn& d) { return (int)((d.tick + s.gin_depth - 1) % s.gin_depth); }
+__device__ __forceinline__ int gin_slot_read(const StageDev& s, const StageDyn& d) { (void)s; return d.gin_rslot; }
 // slot of the dz operand of a stage's last Linear when that operand is the incoming gradient itself (no activation,
 // no attention): the rotating mailbox slot written during the previous tick, or the memory-gradient ring slot of the
 // microbatch for the stage that emits the memory
 __device__ __forceinline__ int dz_mailbox_slot(const TickArgs& t, const StageDev& s, const StageDyn& d) {
-  return s.emit_memory ? (int)(d.b_mb % t.gmem_depth) : gin_slot_read(s, d);
+  (void)t; return s.emit_memory ? d.gmem_slot : d.gin_rslot;
 }
 // gradient of the memory for the microbatch in backward at a stage
 template <typename AT> __device__ __forceinline__ AT* gmem_at(const TickArgs& t, const StageDyn& d) {
-  return ws_at<AT>(t, t.gmem_off) + (uint64_t)(d.b_mb % t.gmem_depth) * ((uint64_t)t.T * t.mem_dim);
+  return ws_at<AT>(t, t.gmem_off) + (uint64_t)d.gmem_slot * ((uint64_t)t.T * t.mem_dim);
 }
 // gradient w.r.t. this stage's main output: written by the next stage during the previous tick; the stage that
 // emits the memory receives the sum the cross-attention stages left in the memory-gradient ring
@@ -82,7 +82,7 @@ template <typename AT> __device__ __forceinline__ AT* gin_read(const TickArgs& t
 // where stage p writes the gradient w.r.t. its main input (= stage p-1's main output)
 template <typename AT> __device__ __forceinline__ AT* gin_write_prev(const TickArgs& t, int p, const StageDyn& d) {
   const StageDev& sp = t.st[p - 1];
-  return ws_at<AT>(t, sp.gin) + (uint64_t)(d.tick % sp.gin_depth) * ((uint64_t)t.T * sp.d_out_main);
+  return ws_at<AT>(t, sp.gin) + (uint64_t)d.prev_wslot * ((uint64_t)t.T * sp.d_out_main);
 }
 // gradient w.r.t. the skip tensor stage p emitted: it equals the gradient the receiving (residual) stage took in
 // skip_hop ticks ago for the same microbatch, i.e. what the stage after that one wrote skip_hop + 1 ticks ago

@@ -812,7 +812,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       ready = __all_sync(0xffffffffu, ready);
       if (!ready) { ok = false; break; }
       tc_fence_after();
-      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % t.st[tl.p - 1].gin_depth) : 0;
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
       for (int mi = 0; mi < tl.n_m; ++mi) {
         const int mrow = tl.m0 + mi * TILE_M + q * 32;
 #pragma unroll 1
@@ -1110,7 +1110,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       ready = __all_sync(0xffffffffu, ready);
       if (!ready) { ok = false; break; }
       tc_fence_after();
-      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? (int)(d.tick % t.st[tl.p - 1].gin_depth) : 0;
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
       const int nb = tl.n0 + half * 64;
 #pragma unroll 1
       for (int mi = 0; mi < tl.n_m; ++mi) {

@@ -50,6 +50,10 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
     d.b_slot = ba ? (int32_t)(b % s.depth) : 0;
     d.b_xslot = ba ? (int32_t)(b % s.xdepth) : 0;
   }
+  d.gin_rslot = s.gin_depth > 0 ? (int32_t)((tick + s.gin_depth - 1) % s.gin_depth) : 0;
+  d.prev_wslot = s.prev_gin_depth > 0 ? (int32_t)(tick % s.prev_gin_depth) : 0;
+  d.gmem_slot = (s.gmem_depth > 0 && d.b_mb >= 0) ? (int32_t)(d.b_mb % s.gmem_depth) : 0;
+  d._pad2 = 0;
   d.f_ver = ver;
   d.b_ver = ver;
   d.active_update = d.k >= 0 ? 1 : 0;

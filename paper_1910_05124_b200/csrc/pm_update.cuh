@@ -6,7 +6,7 @@ namespace pm {
 
 // What the scheduler needs to know about a stage (device table, constant over the run).
 struct StageSched {
-  int32_t tau_f, gap, depth, xdepth, next_xdepth, _pad;
+  int32_t tau_f, gap, depth, xdepth, next_xdepth, gin_depth, prev_gin_depth, gmem_depth;
 };
 
 // Launches the scheduler for pipeline tick `tick` with `n_fed` microbatches fed so far.

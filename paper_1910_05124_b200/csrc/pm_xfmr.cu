@@ -829,13 +829,13 @@ static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
 }
 
 // Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
-// A block owns kEmbRows consecutive vocabulary rows and kEmbCols columns.  It walks the microbatch's token ids
-// once, in order, and compacts the tokens that fall into its rows into a list (ballot + prefix over the warps, so
-// the list is in ascending token order).  A row with few tokens is summed by one warp; a row with many (frequent
+// A block owns kEmbRows consecutive vocabulary rows and a slice of the columns.  It reads the microbatch's token
+// ids once (16 consecutive tokens per thread) and compacts the tokens that fall into its rows into a list in
+// ascending token order (a prefix sum over the per-thread counts).  A row with few tokens is summed by one warp; a row with many (frequent
 // ids under a Zipf distribution) by all eight, each adding a contiguous segment of the row's tokens in order, the
 // eight partial sums then added in warp order.  Tokens are gathered eight at a time so that their loads are in
 // flight together.  Every row is written (zeros included) and the order of the additions is fixed.
-constexpr int kEmbRows = 32;                          // a block's columns: 32 lanes x CPL (4, 8 or 16) columns per lane
+constexpr int kEmbRows = 64;                          // a block's columns: 32 lanes x CPL (4, 8 or 16) columns per lane
 constexpr int kEmbHeavy = 24;                         // tokens per row from which the block shares the row
 
 template <typename AT> __device__ __forceinline__ void load4(const AT* p, float (&v)[4]);
@@ -863,52 +863,32 @@ template <typename AT, int CPL> __device__ __forceinline__ void load_cols(const 
   }
 }
 
-// adds, in list order, the rows of the tokens number k_lo .. k_hi-1 (counted among the list entries of row rr) to acc;
-// 32 / CPL tokens are gathered at a time
+// adds the rows of the tokens sub[k_lo .. k_hi-1] (ascending token order) to acc; 32 / CPL tokens are gathered at a time
 template <typename AT, int CPL>
-__device__ __forceinline__ void embed_gather(const int32_t* hits, int nh, int rr, int k_lo, int k_hi, const AT* du, const AT* gs,
-                                             int dm, int col, float sc, int lane, float (&acc)[CPL]) {
+__device__ __forceinline__ void embed_gather(const int32_t* sub, int k_lo, int k_hi, const AT* du, const AT* gs,
+                                             int dm, int col, float sc, float (&acc)[CPL]) {
   constexpr int NB = 32 / CPL;
-  int seen = 0;
-  for (int hb = 0; hb < nh && seen < k_hi; hb += 32) {
-    const int hv = hb + lane < nh ? hits[hb + lane] : -1;
-    unsigned mine = __ballot_sync(0xffffffffu, hv >= 0 && (hv & 255) == rr);
-    int idx = seen;
-    seen += __popc(mine);
-    if (seen <= k_lo) continue;
-    while (mine) {                                           // NB tokens at a time: loads first, ordered additions after
-      uint64_t ro[NB];
-      bool use[NB];
+  for (int k = k_lo; k < k_hi; k += NB) {
+    uint64_t ro[NB];
 #pragma unroll
-      for (int u = 0; u < NB; ++u) {                         // no loads inside these branches (they would be serialised)
-        use[u] = false;
-        ro[u] = (uint64_t)col;                               // a valid address for the slots that stay empty
-        if (mine) {
-          const int j = __ffs(mine) - 1;
-          mine &= mine - 1;
-          const int my = idx++;
-          use[u] = my >= k_lo && my < k_hi;
-          ro[u] = (uint64_t)(__shfl_sync(0xffffffffu, hv, j) >> 8) * dm + col;
-        }
-      }
-      float val[NB][CPL], sv[NB][CPL];
+    for (int u = 0; u < NB; ++u) ro[u] = (uint64_t)sub[min(k + u, k_hi - 1)] * dm + col;   // slots past the end repeat the last token (not added)
+    float val[NB][CPL], sv[NB][CPL];
 #pragma unroll
-      for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(du + ro[u], val[u]);
-      if (gs) {
+    for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(du + ro[u], val[u]);                 // all loads first (no branch between them)
+    if (gs) {
 #pragma unroll
-        for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(gs + ro[u], sv[u]);
-#pragma unroll
-        for (int u = 0; u < NB; ++u)
-#pragma unroll
-          for (int e = 0; e < CPL; ++e) val[u][e] = __fadd_rn(val[u][e], sv[u][e]);
-      }
+      for (int u = 0; u < NB; ++u) load_cols<AT, CPL>(gs + ro[u], sv[u]);
 #pragma unroll
       for (int u = 0; u < NB; ++u)
-        if (use[u]) {
 #pragma unroll
-          for (int e = 0; e < CPL; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[u][e], sc));
-        }
+        for (int e = 0; e < CPL; ++e) val[u][e] = __fadd_rn(val[u][e], sv[u][e]);
     }
+#pragma unroll
+    for (int u = 0; u < NB; ++u)
+      if (k + u < k_hi) {
+#pragma unroll
+        for (int e = 0; e < CPL; ++e) acc[e] = __fadd_rn(acc[e], __fmul_rn(val[u][e], sc));
+      }
   }
 }
 
@@ -926,31 +906,58 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   if (v0 >= s.vocab || blockIdx.z * kEmbCols >= dm) return;
   extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
   __shared__ int warp_cnt[2][8];
-  __shared__ int row_cnt[kEmbRows];
-  __shared__ float part[8][kEmbCols];                        // shared rows: per-warp partial sums
+  __shared__ int row_cnt[kEmbRows], row_start[kEmbRows];
+  int32_t* sub = hits + t.T;                                 // [T] token indices grouped by row, ascending inside a row
+  float (*part)[kEmbCols] = reinterpret_cast<float (*)[kEmbCols]>(sub + t.T);   // [8][kEmbCols] shared rows: per-warp partial sums
   if (threadIdx.x < kEmbRows) row_cnt[threadIdx.x] = 0;
   __syncthreads();
   const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, (int)(d.b_mb % s.ids_depth), (uint64_t)t.T);
   int nh = 0;                                                // hits so far (the same value in every thread)
-  for (int tb0 = 0; tb0 < t.T; tb0 += 16 * 256) {            // 16 rounds of 256 tokens; the ids of all rounds are fetched first
+  for (int tb0 = 0; tb0 < t.T; tb0 += 16 * 256) {            // 4096 tokens per pass: thread i takes tokens 16 i .. 16 i + 15
     int rel[16];
+    const int tok0 = tb0 + 16 * (int)threadIdx.x;
+    if (tok0 + 16 <= t.T && (t.T & 3) == 0) {
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const int tok = tb0 + k * 256 + threadIdx.x;
-      rel[k] = tok < t.T ? __ldg(ids + tok) - v0 : -1;
+      for (int k = 0; k < 4; ++k) {
+        const int4 q = __ldg(reinterpret_cast<const int4*>(ids + tok0) + k);
+        rel[4 * k] = q.x - v0; rel[4 * k + 1] = q.y - v0; rel[4 * k + 2] = q.z - v0; rel[4 * k + 3] = q.w - v0;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) rel[k] = tok0 + k < t.T ? __ldg(ids + tok0 + k) - v0 : -1;
     }
+    int mine = 0;
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      if (tb0 + k * 256 >= t.T) break;
-      const bool hit = rel[k] >= 0 && rel[k] < kEmbRows;
-      const unsigned bal = __ballot_sync(0xffffffffu, hit);
-      if (lane == 0) warp_cnt[k & 1][warp] = __popc(bal);
-      __syncthreads();                                       // one barrier per round: the counters are double-buffered
-      int base = nh, tot = 0;
+    for (int k = 0; k < 16; ++k) mine += (rel[k] >= 0 && rel[k] < kEmbRows) ? 1 : 0;
+    // exclusive prefix of the per-thread counts over the block: shuffle scan per warp, then the warp totals
+    int incl = mine;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) { const int cw = warp_cnt[k & 1][w]; if (w < warp) base += cw; tot += cw; }
-      if (hit) { hits[base + __popc(bal & ((1u << lane) - 1u))] = ((tb0 + k * 256 + (int)threadIdx.x) << 8) | rel[k]; atomicAdd(&row_cnt[rel[k]], 1); }
-      nh += tot;
+    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+    if (lane == 31) warp_cnt[0][warp] = incl;
+    __syncthreads();
+    int base = nh, tot = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { const int cw = warp_cnt[0][w]; if (w < warp) base += cw; tot += cw; }
+    int pos = base + incl - mine;
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+      if (rel[k] >= 0 && rel[k] < kEmbRows) { hits[pos++] = ((tok0 + k) << 8) | rel[k]; atomicAdd(&row_cnt[rel[k]], 1); }
+    nh += tot;
+    __syncthreads();                                         // warp_cnt is reused by the next pass
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) { int a = 0; for (int r = 0; r < kEmbRows; ++r) { row_start[r] = a; a += row_cnt[r]; } }
+  __syncthreads();
+  // the list, grouped by row: warp w scans it once for each of its rows and copies the matching tokens in order
+  for (int rr = warp; rr < kEmbRows; rr += 8) {
+    if (row_cnt[rr] == 0) continue;
+    int seen = row_start[rr];
+    for (int hb = 0; hb < nh; hb += 32) {
+      const int hv = hb + lane < nh ? hits[hb + lane] : -1;
+      const bool m = hv >= 0 && (hv & 255) == rr;
+      const unsigned bal = __ballot_sync(0xffffffffu, m);
+      if (m) sub[seen + __popc(bal & ((1u << lane) - 1u))] = hv >> 8;
+      seen += __popc(bal);
     }
   }
   __syncthreads();
@@ -967,7 +974,7 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
     float acc[CPL];
 #pragma unroll
     for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
-    embed_gather<AT, CPL>(hits, nh, rr, k_lo, k_hi, du, gs, dm, col_ld, sc, lane, acc);
+    embed_gather<AT, CPL>(sub + row_start[rr], k_lo, k_hi, du, gs, dm, col_ld, sc, acc);
 #pragma unroll
     for (int e = 0; e < CPL; ++e) part[warp][lane * CPL + e] = acc[e];
     __syncthreads();
@@ -988,7 +995,7 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
     float acc[CPL];
 #pragma unroll
     for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
-    if (cnt > 0) embed_gather<AT, CPL>(hits, nh, rr, 0, cnt, du, gs, dm, col_ld, sc, lane, acc);
+    if (cnt > 0) embed_gather<AT, CPL>(sub + row_start[rr], 0, cnt, du, gs, dm, col_ld, sc, acc);
     if (col_ok) {
 #pragma unroll
       for (int e = 0; e < CPL; e += 4)
@@ -1023,17 +1030,18 @@ cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
     const int dm = t.max_embed_dim;
     const int cpl = (dm % 16 == 0 && dm <= 512) ? 16 : (dm % 8 == 0 ? 8 : 4);
     dim3 g((t.max_vocab + kEmbRows - 1) / kEmbRows, t.n_embed, (dm + 32 * cpl - 1) / (32 * cpl));
-    const size_t smem = sizeof(int32_t) * (size_t)t.T;
-    if (dtype == PM_F32) {
-      if (cpl == 16) embed_bwd_kernel<float, 16><<<g, 256, smem, stream>>>(t);
-      else if (cpl == 8) embed_bwd_kernel<float, 8><<<g, 256, smem, stream>>>(t);
-      else embed_bwd_kernel<float, 4><<<g, 256, smem, stream>>>(t);
-    } else {
-      if (cpl == 16) embed_bwd_kernel<__nv_bfloat16, 16><<<g, 256, smem, stream>>>(t);
-      else if (cpl == 8) embed_bwd_kernel<__nv_bfloat16, 8><<<g, 256, smem, stream>>>(t);
-      else embed_bwd_kernel<__nv_bfloat16, 4><<<g, 256, smem, stream>>>(t);
-    }
-    e = cudaGetLastError();
+    // the hit list, the same tokens grouped by row, and the per-warp partial sums of a shared row
+    const size_t smem = 2 * sizeof(int32_t) * (size_t)t.T + sizeof(float) * 8 * 32 * (size_t)cpl;
+    auto go = [&](auto kernel) -> cudaError_t {
+      if (smem + 1024 > 48 * 1024) {                         // static shared memory counts towards the default limit
+        cudaError_t ea = cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (ea != cudaSuccess) return ea;
+      }
+      kernel<<<g, 256, smem, stream>>>(t);
+      return cudaGetLastError();
+    };
+    if (dtype == PM_F32) e = cpl == 16 ? go(embed_bwd_kernel<float, 16>) : (cpl == 8 ? go(embed_bwd_kernel<float, 8>) : go(embed_bwd_kernel<float, 4>));
+    else e = cpl == 16 ? go(embed_bwd_kernel<__nv_bfloat16, 16>) : (cpl == 8 ? go(embed_bwd_kernel<__nv_bfloat16, 8>) : go(embed_bwd_kernel<__nv_bfloat16, 4>));
   }
   return e;
 }
