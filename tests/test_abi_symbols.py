@@ -102,3 +102,70 @@ def test_bad_arguments_are_rejected_without_a_gpu(built_lib):
     st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), None, None)
     assert L.pm_status_string(st) == b"PM_ERR_SHAPE"
     assert L.pm_status_string(L.pm_forward(None, None, None)) == b"PM_ERR_INVALID_ARG"
+
+
+def _describe(wl, mutate=None):
+    """Stage descriptors of a Transformer workload as the binding builds them; mutate(p, ops) may edit a stage's op list."""
+    import ctypes as C
+    from paper_1910_05124_b200 import binding as B
+    P = wl.n_stages
+    sd = (B.pm_stage_desc * P)()
+    keep, off = [], 0
+    for p in range(P):
+        ops, tensors = B.stage_ops(wl, p)
+        if mutate:
+            mutate(p, ops)
+        arr = B._ops_from_dicts(ops)
+        keep.append(arr)
+        cnt, _ = B.ops_layout(arr, len(ops), tensors)
+        sd[p].tau_fwd, sd[p].tau_bkwd, sd[p].n_ops = wl.tau_fwd[p], 0, len(ops)
+        sd[p].ops = C.cast(arr, C.POINTER(B.pm_op_desc))
+        sd[p].param_offset, sd[p].param_count = off, cnt
+        off += cnt
+    cfg, _ = B.make_config(n_stages=P, microbatch=wl.microbatch, compute=wl.compute, optimizer=wl.optimizer, alpha=wl.alpha,
+                           beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, K=wl.K, D=wl.D, loss=B.PM_LOSS_CE)
+    return cfg, sd, keep
+
+
+def test_encoder_decoder_layout_and_its_checks(built_lib):
+    """Footprints of the encoder-decoder workloads (host arithmetic only) and the chaining rules of their stages."""
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+
+    def query(wl, mutate=None):
+        cfg, sd, keep = _describe(wl, mutate)
+        sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+        st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+        return L.pm_status_string(st), L.pm_last_error(None), sb.value, rb.value, wb.value
+
+    # config 5 as given: sequences of 256 tokens are refused (attention is built for up to 128)
+    st, msg = query(I.cfg5())[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"seq_len <= 128" in msg
+    # its 12 + 12 layers with 128-token sequences do not fit one GPU in the tick-major stash plan; the 4 + 4 layer cut does
+    st, _, sb, rb, wb = query(I.cfg5_cut(12, 12))
+    assert st == b"PM_OK" and rb > 500e9 and sb < 12e9
+    st, _, sb, rb, wb = query(I.cfg5_cut())
+    assert st == b"PM_OK" and 60e9 < rb < 70e9 and sb + rb + wb < 90e9
+    small = I.cfg5_small()
+    assert query(small)[0] == b"PM_OK"
+    dec0 = [i for i, s in enumerate(small.stage_specs) if s.pre == "embed_dec"][0]
+
+    def drop_flag(stage, kind, flag):
+        def m(p, ops):
+            if p == stage:
+                for o in ops:
+                    if o["kind"] == kind:
+                        o["flags"] = o.get("flags", 0) & ~flag
+        return m
+    # the decoder's embedding without the second-stream flag, the memory stage without its flag, a two-stage skip
+    # declared as a one-stage skip, a cross-attention stage whose LayerNorm reads the main stream
+    st, msg = query(small, drop_flag(dec0, B.PM_OP_EMBED, B.PM_OPF_SECOND_STREAM))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"EMBED" in msg
+    st, msg = query(small, drop_flag(dec0 - 1, B.PM_OP_RESIDUAL, B.PM_OPF_EMIT_MEMORY))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"memory" in msg
+    st, msg = query(small, drop_flag(dec0 + 2, B.PM_OP_SKIP_OUT, B.PM_OPF_SKIP_TWO))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"RESIDUAL" in msg
+    st, msg = query(small, drop_flag(dec0 + 3, B.PM_OP_LAYERNORM, B.PM_OPF_FROM_MEMORY))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"CROSS_ATTENTION" in msg
