@@ -72,6 +72,8 @@ struct StageDyn {
   int32_t gin_rslot;          // slot of this stage's gradient mailbox written during the previous tick
   int32_t prev_wslot;         // slot of the previous stage's gradient mailbox this tick's backward writes
   int32_t gmem_slot;          // slot of the memory-gradient ring of the microbatch in backward
+  int32_t skip_wslot;         // emitting stage: slot of the receiving stage's skip buffer this tick's forward writes
+  int32_t skip_rslot;         // receiving stage: slot of its skip buffer this tick's forward reads
   int32_t _pad2;
 };
 

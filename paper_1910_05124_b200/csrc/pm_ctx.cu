@@ -228,6 +228,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
     L.sched[p].gin_depth = L.st[p].gin_depth;
     L.sched[p].prev_gin_depth = p > 0 ? L.st[p - 1].gin_depth : 0;
+    L.sched[p].skip_dst_depth = L.st[p].skip_hop > 0 ? L.st[p + L.st[p].skip_hop].skip_depth : 0;
+    L.sched[p].skip_depth = L.st[p].skip_depth;
   }
   if (L.mem_stage >= 0) {
     if (L.last_mem_reader < 0) { err = "a memory is emitted but no CROSS_ATTENTION stage reads it"; return PM_ERR_UNSUPPORTED; }

@@ -53,6 +53,8 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
   d.gin_rslot = s.gin_depth > 0 ? (int32_t)((tick + s.gin_depth - 1) % s.gin_depth) : 0;
   d.prev_wslot = s.prev_gin_depth > 0 ? (int32_t)(tick % s.prev_gin_depth) : 0;
   d.gmem_slot = (s.gmem_depth > 0 && d.b_mb >= 0) ? (int32_t)(d.b_mb % s.gmem_depth) : 0;
+  d.skip_wslot = s.skip_dst_depth > 0 ? (int32_t)(tick % s.skip_dst_depth) : 0;
+  d.skip_rslot = s.skip_depth > 0 ? (int32_t)((tick + 1) % s.skip_depth) : 0;
   d._pad2 = 0;
   d.f_ver = ver;
   d.b_ver = ver;

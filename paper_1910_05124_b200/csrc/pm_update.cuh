@@ -7,6 +7,7 @@ namespace pm {
 // What the scheduler needs to know about a stage (device table, constant over the run).
 struct StageSched {
   int32_t tau_f, gap, depth, xdepth, next_xdepth, gin_depth, prev_gin_depth, gmem_depth;
+  int32_t skip_dst_depth, skip_depth;   // slots of the skip buffer this stage writes into / reads from (0: none)
 };
 
 // Launches the scheduler for pipeline tick `tick` with `n_fed` microbatches fed so far.

@@ -30,6 +30,42 @@ template <> __device__ __forceinline__ const __nv_bfloat16* table_ptr<__nv_bfloa
 //   embedding: u = table[id] * sqrt(d) + PE[position]     (table in the GEMM operand type)
 //   LayerNorm: mean, biased variance, rstd = 1/sqrt(var + eps) in fp32; u = xhat * gain + bias (fp32 master values)
 // If the stage emits a skip tensor (attention / skip_out) u is also written to the next stage's skip buffer.
+// LayerNorm of one row of exactly NP * 256 columns by one warp: the row is read once and stays in registers
+template <typename AT, int NP>
+__device__ __forceinline__ void ln_fwd_row(const TickArgs& t, const StageDev& s, const StageDyn& d, const AT* x, const float* g,
+                                           const float* b, AT* u, AT* skip, int row, int lane) {
+  constexpr int dm = NP * 256;
+  float xr[NP][8];
+#pragma unroll
+  for (int q = 0; q < NP; ++q) load8<AT>(x + q * 256 + lane * 8, xr[q]);
+  float sum = 0.f, sq = 0.f;
+#pragma unroll
+  for (int q = 0; q < NP; ++q)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sum += xr[q][k];
+  const float mu = warp_sum(sum) / (float)dm;
+#pragma unroll
+  for (int q = 0; q < NP; ++q)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { const float v = xr[q][k] - mu; sq += v * v; }
+  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)dm + LN_EPS);
+#pragma unroll
+  for (int q = 0; q < NP; ++q) {
+    const int c = q * 256 + lane * 8;
+    float gv[8], bv[8], o[8];
+    load8<float>(g + c, gv);
+    load8<float>(b + c, bv);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o[k] = __fadd_rn(__fmul_rn(__fmul_rn(xr[q][k] - mu, rstd), gv[k]), bv[k]);
+    store8<AT>(u + c, o);
+    if (skip) store8<AT>(skip + c, o);
+  }
+  if (lane == 0) {
+    float* st = ring_at<float>(t, s.stat_ring, d.f_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
+    st[0] = mu; st[1] = rstd;
+  }
+}
+
 template <typename AT>
 __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   const int p = t.pre_ids[blockIdx.y];
@@ -43,7 +79,7 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   const uint64_t n = (uint64_t)t.T * dm;
   AT* u = ring_at<AT>(t, s.u_ring, d.f_slot, n) + (uint64_t)row * dm;
   const StageDev& sk_dst = t.st[p + s.skip_hop];             // the residual stage that will add this stage's input
-  AT* skip = emits_skip(s) ? ws_at<AT>(t, sk_dst.skip_in) + (uint64_t)(d.tick % sk_dst.skip_depth) * n + (uint64_t)row * dm : nullptr;
+  AT* skip = emits_skip(s) ? ws_at<AT>(t, sk_dst.skip_in) + (uint64_t)d.skip_wslot * n + (uint64_t)row * dm : nullptr;
   const bool vec = (dm & 7) == 0;                            // 8 consecutive columns per lane, 256 per pass
   if (s.pre == PRE_EMBED) {
     const int32_t id = ring_at<int32_t>(t, s.ids_ring, (int)(d.f_mb % s.ids_depth), (uint64_t)t.T)[row];
@@ -73,6 +109,9 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   const float* g = t.a.w + s.g_off;
   const float* b = t.a.w + s.beta_off;
   float sum = 0.f, sq = 0.f;
+  if (vec && dm == 512) { ln_fwd_row<AT, 2>(t, s, d, x, g, b, u, skip, row, lane); return; }
+  if (vec && dm == 1024) { ln_fwd_row<AT, 4>(t, s, d, x, g, b, u, skip, row, lane); return; }
+  if (vec && dm == 256) { ln_fwd_row<AT, 1>(t, s, d, x, g, b, u, skip, row, lane); return; }
   if (vec) {
     for (int c = lane * 8; c < dm; c += 256) {
       float xv[8];
@@ -134,32 +173,30 @@ __global__ void __launch_bounds__(256) residual_kernel(TickArgs t) {
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || s.post != POST_RESIDUAL) return;
   const uint64_t n = (uint64_t)t.T * s.d_out_main;
-  const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)((d.tick + 1) % s.skip_depth) * n;   // written skip_depth - 1 ticks ago
+  const AT* skip = ws_at<AT>(t, s.skip_in) + (uint64_t)d.skip_rslot * n;   // written skip_depth - 1 ticks ago
   const AT* y = ws_at<AT>(t, s.ytmp);
   // the stage that emits the memory writes only there: the next stage embeds its own token stream
   AT* out = s.emit_memory ? mem_at<AT>(t, d.f_mb) : ring_at<AT>(t, t.st[p + 1].x_ring, d.f_next_xslot, n);
   // buffers start on 256-byte boundaries and slots are n elements apart: groups of eight are aligned when 8 | n
   const uint64_t n8 = (n % 8 == 0) ? n / 8 : 0;
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  for (; i + 3 * stride < n8; i += 4 * stride) {            // four groups of eight in flight per thread
+  // a block takes runs of 4 x 256 groups of eight: thread t the groups base + t, + 256, + 512, + 768, all loads first
+  for (uint64_t base = (uint64_t)blockIdx.x * 1024; base < n8; base += (uint64_t)gridDim.x * 1024) {
     float a[4][8], b[4][8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) { load8<AT>(skip + 8 * (i + u * stride), a[u]); load8<AT>(y + 8 * (i + u * stride), b[u]); }
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = min(base + u * 256 + threadIdx.x, n8 - 1);
+      load8<AT>(skip + 8 * i, a[u]);
+      load8<AT>(y + 8 * i, b[u]);
+    }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
+      const uint64_t i = base + u * 256 + threadIdx.x;
+      if (i < n8) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) a[u][j] = __fadd_rn(a[u][j], b[u][j]);
-      store8<AT>(out + 8 * (i + u * stride), a[u]);
+        for (int j = 0; j < 8; ++j) a[u][j] = __fadd_rn(a[u][j], b[u][j]);
+        store8<AT>(out + 8 * i, a[u]);
+      }
     }
-  }
-  for (; i < n8; i += stride) {
-    float a[8], b[8];
-    load8<AT>(skip + 8 * i, a);
-    load8<AT>(y + 8 * i, b);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) a[j] = __fadd_rn(a[j], b[j]);
-    store8<AT>(out + 8 * i, a);
   }
   for (uint64_t i = 8 * n8 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
     out[i] = from_f<AT>(__fadd_rn(to_f<AT>(skip[i]), to_f<AT>(y[i])));
@@ -253,7 +290,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
     if (e != cudaSuccess) return e;
   }
   if (any_res) {
-    dim3 grid(296, t.n_res);
+    dim3 grid(64, t.n_res);
     if (dtype == PM_F32) residual_kernel<float><<<grid, 256, 0, stream>>>(t);
     else residual_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
     e = cudaGetLastError();
