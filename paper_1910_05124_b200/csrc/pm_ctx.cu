@@ -1,4 +1,5 @@
 // Host side of the C ABI: layout arithmetic, context set-up, and the launch sequence of a tick.
+#include <functional>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -329,6 +330,20 @@ struct pm_ctx {
   UmmaPlan* umma = nullptr;
   AttnPlan* attn = nullptr;
   uint64_t launches = 0;
+  // The kernel sequence of a phase is the same in every steady-state tick (what differs sits in the device-side
+  // schedule table), so each phase is captured once into a CUDA graph and replayed: one launch instead of up to a
+  // dozen.  Captured on a private stream (the caller's may be the legacy default stream, which cannot capture),
+  // replayed on the caller's.  PM_CUDA_GRAPHS=0 in the environment, profiling, or a failed capture keep the
+  // phase on plain launches.
+  struct PhaseGraph { cudaGraphExec_t exec = nullptr; int eager_runs = 0; uint64_t launches = 0; bool failed = false; };
+  PhaseGraph g_fwd, g_bwd, g_upd;
+  bool graphs = true;
+  cudaStream_t cap_stream = nullptr;
+  cudaStream_t ls = nullptr;            // the stream the phase bodies launch on: `stream`, or `cap_stream` while capturing
+  ~pm_ctx() {
+    for (PhaseGraph* g : {&g_fwd, &g_bwd, &g_upd}) if (g->exec) cudaGraphExecDestroy(g->exec);
+    if (cap_stream) cudaStreamDestroy(cap_stream);
+  }
   // optional per-kernel-class timing with CUDA events on the context's stream
   bool prof_on = false;
   int prof_cls = 0;
@@ -436,6 +451,9 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->cfg.alpha_by_step = nullptr;
   c->L = L;
   c->stream = (cudaStream_t)stream;
+  c->ls = c->stream;
+  { const char* v = getenv("PM_CUDA_GRAPHS"); c->graphs = !(v && v[0] == '0'); }
+  if (c->graphs && cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->cap_stream = nullptr; }
   c->ws = (char*)workspace;
   const int P = cfg->n_stages;
   c->a = ArenasDev{arenas->w, arenas->m, arenas->s, arenas->delta, arenas->grad, (__nv_bfloat16*)arenas->w_lp, arenas->count};
@@ -541,6 +559,39 @@ static inline void prof_begin(pm_ctx* ctx, int cls) {
 }
 #define TIMED(cls, call) (prof_begin(ctx, cls), call)
 
+// Runs the kernel launches of one phase (`body` launches on ctx->ls): plainly the first times and whenever graphs
+// are off, then once under stream capture to build the phase's graph, then by replaying that graph.
+static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::function<pm_status()>& body) {
+  ctx->ls = ctx->stream;
+  if (!ctx->graphs || ctx->prof_on || g.failed || !ctx->cap_stream) return body();
+  if (g.exec) {
+    ctx->launches += g.launches;
+    cudaError_t e = cudaGraphLaunch(g.exec, ctx->stream);
+    return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, "graph launch");
+  }
+  if (g.eager_runs < 2) { ++g.eager_runs; return body(); }      // modules loaded, function attributes set
+  const uint64_t l0 = ctx->launches;
+  if (cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) { cudaGetLastError(); g.failed = true; return body(); }
+  ctx->ls = ctx->cap_stream;
+  const pm_status sb = body();
+  ctx->ls = ctx->stream;
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
+  if (sb == PM_OK && e == cudaSuccess && graph) {
+    g.launches = ctx->launches - l0;
+    e = cudaGraphInstantiate(&g.exec, graph, 0);
+  } else if (e == cudaSuccess) e = cudaErrorUnknown;
+  if (graph) cudaGraphDestroy(graph);
+  if (e != cudaSuccess) {                                        // nothing has run yet: do the phase with plain launches
+    cudaGetLastError();
+    g.failed = true; g.exec = nullptr;
+    ctx->launches = l0;
+    return body();
+  }
+  e = cudaGraphLaunch(g.exec, ctx->stream);
+  return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, "graph launch");
+}
+
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "pm_forward called out of order (expected pm_backward or pm_update)");
@@ -558,16 +609,21 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   }
   // forward of every stage whose microbatch exists: s - (i-1) in [0, n_fed)
   if (ctx->tick - (ctx->cfg.n_stages - 1) < ctx->n_fed) {
-    if (ctx->L.any_pre && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->stream), "embedding / LayerNorm forward"))) != PM_OK) return s;
-    for (int l = 0; l < ctx->L.max_lin; ++l) {
-      prof_begin(ctx, PM_PROF_GEMM_FWD);
-      cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 0, l, ctx->stream)
-                                   : umma_launch(ctx->umma, ctx->ta, 0, l, ctx->stream);
-      if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
-    }
-    if (ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->stream), "attention forward"))) != PM_OK) return s;
-    const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
-    if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ctx->ta, dt, ctx->stream, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
+    s = run_phase(ctx, ctx->g_fwd, [&]() -> pm_status {
+      pm_status s;
+      if (ctx->L.any_pre && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->ls), "embedding / LayerNorm forward"))) != PM_OK) return s;
+      for (int l = 0; l < ctx->L.max_lin; ++l) {
+        prof_begin(ctx, PM_PROF_GEMM_FWD);
+        cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 0, l, ctx->ls)
+                                     : umma_launch(ctx->umma, ctx->ta, 0, l, ctx->ls);
+        if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
+      }
+      if (ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
+      const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
+      if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ctx->ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
+      return PM_OK;
+    });
+    if (s != PM_OK) return s;
   }
   ctx->phase = 1;
   return PM_OK;
@@ -582,22 +638,27 @@ pm_status pm_backward(pm_ctx* ctx) {
   // any backward this tick?  stage P runs microbatch tick-P, stage 1 runs tick-(2P-1)
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
-    if ((s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ctx->ta, dt, ctx->stream), "loss"))) != PM_OK) return s;
-    if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->stream), "attention backward"))) != PM_OK) return s; }
-    else if (ctx->L.att_blocks > 0 && (s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ctx->ta, dt, ctx->stream), "attention backward"))) != PM_OK) return s;
-    for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
-      if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->stream), "activation backward", actbwd_launches(ctx->ta)))) != PM_OK) return s;
-      prof_begin(ctx, PM_PROF_WGRAD);
-      cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->stream)
-                                   : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->stream);
-      if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
-      prof_begin(ctx, PM_PROF_DGRAD);
-      e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 1, l, ctx->stream)
-                       : umma_launch(ctx->umma, ctx->ta, 1, l, ctx->stream);
-      if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
-    }
-    const int n_pre = pre_bwd_launches(ctx->ta);
-    if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ctx->ta, dt, ctx->stream), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
+    s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
+      pm_status s;
+      if ((s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ctx->ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
+      if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, false, ctx->ls), "attention backward"))) != PM_OK) return s; }
+      else if (ctx->L.att_blocks > 0 && (s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ctx->ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
+      for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
+        if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ctx->ta)))) != PM_OK) return s;
+        prof_begin(ctx, PM_PROF_WGRAD);
+        cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->ls)
+                                     : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->ls);
+        if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+        prof_begin(ctx, PM_PROF_DGRAD);
+        e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 1, l, ctx->ls)
+                         : umma_launch(ctx->umma, ctx->ta, 1, l, ctx->ls);
+        if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
+      }
+      const int n_pre = pre_bwd_launches(ctx->ta);
+      if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ctx->ta, dt, ctx->ls), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
+      return PM_OK;
+    });
+    if (s != PM_OK) return s;
   }
   ctx->phase = 2;
   return PM_OK;
@@ -609,11 +670,13 @@ pm_status pm_update(pm_ctx* ctx) {
   const int P = ctx->cfg.n_stages;
   const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
   if (any) {
-    prof_begin(ctx, PM_PROF_UPDATE);
-    cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
-                                  (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
-                                  ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->stream);
-    pm_status s = check(ctx, e, "update");
+    pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
+      prof_begin(ctx, PM_PROF_UPDATE);
+      cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
+                                    (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
+                                    ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls);
+      return check(ctx, e, "update");
+    });
     if (s != PM_OK) return s;
   }
   ctx->tick += 1;
