@@ -868,7 +868,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
 // CTAs; the epilogue warps of both arrive on the leader's tempty.
 constexpr int DP_TILE_M = 256, DP_TILE_N = 128, DP_HALF_N = 64;
 constexpr int DP_MG = 2;                                   // 256-row tiles per converted tile
-constexpr int DP_NG = 3, DP_NB = 2, DP_NA = 4;             // fp32 staging ring, converted ring, dz ring
+constexpr int DP_NG = 3, DP_NB = 3, DP_NA = 4;             // fp32 staging ring, converted ring, dz ring
 constexpr int DP_STG_HALF = TILE_K * DP_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
 constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;
 constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
