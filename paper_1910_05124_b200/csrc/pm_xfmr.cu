@@ -422,14 +422,13 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   float mx = -INFINITY;
   if (in_regs) {
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int c = (k * 256 + threadIdx.x) * 8;
-      if (c < V) {
-        load8<float>(lg + c, v[k]);
+    for (int k = 0; k < 4; ++k) load8<float>(lg + min((k * 256 + (int)threadIdx.x) * 8, V - 8), v[k]);   // all loads first
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if ((k * 256 + (int)threadIdx.x) * 8 < V) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) mx = fmaxf(mx, v[k][e]);
       }
-    }
   } else if ((V & 3) == 0) {                                 // long rows: three vectorised passes, the re-reads hit L2
     for (int c = threadIdx.x * 4; c < V; c += 4 * blockDim.x) {
       const float4 q = *reinterpret_cast<const float4*>(lg + c);
