@@ -361,9 +361,9 @@ NCU_TRAFFIC = {
     # GEMM kernels: measured DRAM bytes / algorithmic bytes on the 2-layer cut of cfg4
     # (profiles/gemm_and_attention_kernels_cfg4_2layer_cut.md); every operand crosses HBM once, so traffic grows
     # with the algorithmic bytes of the launch
-    "gemm_fwd_ratio": (84.3 + 182.4) / (83.9 + 243.0),
-    "wgrad_ratio": (210.9 + 23.0) / (205.5 + 42.0),
-    "dgrad_ratio": (232.3 + 30.4) / (226.5 + 33.6),
+    "gemm_fwd_ratio": (84.3 + 182.8) / (83.9 + 243.0),
+    "wgrad_ratio": (211.4 + 23.2) / (205.5 + 42.0),
+    "dgrad_ratio": (234.6 + 30.2) / (226.5 + 33.6),
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
