@@ -125,3 +125,23 @@ def test_cfg5_widths_first_microbatches(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("cfg5 widths worst relative weight error (per stage vector)", worst)
+
+
+def _final_weights(wl, params0, n):
+    pipe, losses, _ = run_gpu_pipeline(wl, params0, n, collect_book=False)
+    import torch
+    return pipe.w.clone(), torch.tensor(losses)
+
+
+def test_runs_are_bit_reproducible_and_graph_replay_changes_nothing(cuda_device, monkeypatch):
+    """Every reduction on the path has a fixed order (no floating-point atomics), so two runs of the same workload
+    give the same bits; replaying the phases as CUDA graphs launches the same kernels and must give those bits too."""
+    import torch
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, steps=12)
+    params0 = I.init_encoder_params(wl)
+    w_a, l_a = _final_weights(wl, params0, wl.steps)
+    w_b, l_b = _final_weights(wl, params0, wl.steps)
+    assert torch.equal(w_a, w_b) and torch.equal(l_a, l_b)
+    monkeypatch.setenv("PM_CUDA_GRAPHS", "0")
+    w_c, l_c = _final_weights(wl, params0, wl.steps)
+    assert torch.equal(w_a, w_c) and torch.equal(l_a, l_c)
