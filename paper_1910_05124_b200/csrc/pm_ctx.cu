@@ -141,14 +141,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (op.kind == PM_OP_ATTENTION) {
         const int n_out = s.lin[s.n_lin - 1].n_out;
         if (n_out % 3 || op.n_heads < 1 || (n_out / 3) % op.n_heads || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad ATTENTION description"); return PM_ERR_INVALID_ARG; }
-        if (op.seq_len > 128) { stage_err(p, "ATTENTION is built for seq_len <= 128"); return PM_ERR_UNSUPPORTED; }
+        if (op.seq_len > 128 && !attn_tc_supported(cfg->compute_dtype, op.seq_len, (n_out / 3) / op.n_heads)) { stage_err(p, "ATTENTION beyond 128 tokens is built for 256 tokens, bf16 and heads of width 64"); return PM_ERR_UNSUPPORTED; }
         s.post = POST_ATTENTION; s.n_heads = op.n_heads; s.seq_len = op.seq_len;
         s.causal = (op.flags & PM_OPF_CAUSAL) ? 1 : 0;
         s.skip_hop = 1;
       } else if (op.kind == PM_OP_CROSS_ATTENTION) {
         const int n_out = s.lin[s.n_lin - 1].n_out;
         if (n_out % 2 || op.n_heads < 1 || (n_out / 2) % op.n_heads || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad CROSS_ATTENTION description"); return PM_ERR_INVALID_ARG; }
-        if (op.seq_len > 128) { stage_err(p, "attention is built for seq_len <= 128"); return PM_ERR_UNSUPPORTED; }
+        if (op.seq_len > 128 && !attn_tc_supported(cfg->compute_dtype, op.seq_len, (n_out / 2) / op.n_heads)) { stage_err(p, "attention beyond 128 tokens is built for 256 tokens, bf16 and heads of width 64"); return PM_ERR_UNSUPPORTED; }
         if (!s.from_memory || n_out / 2 != s.lin[0].n_in) { stage_err(p, "CROSS_ATTENTION needs LAYERNORM | PM_OPF_FROM_MEMORY and a memory as wide as the queries"); return PM_ERR_UNSUPPORTED; }
         s.post = POST_CROSS_ATTENTION; s.n_heads = op.n_heads; s.seq_len = op.seq_len;
       } else if (op.kind == PM_OP_SKIP_OUT) { s.post = POST_SKIP_OUT; s.skip_hop = (op.flags & PM_OPF_SKIP_TWO) ? 2 : 1; }
@@ -242,7 +242,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   }
   L.att_tc = L.att_blocks > 0;
   for (int p = 0; p < P; ++p)
-    if (feeds_attention(L.st[p].post) && !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads)) L.att_tc = false;
+    if (feeds_attention(L.st[p].post) && (L.st[p].seq_len != L.att_S || !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads))) L.att_tc = false;
   if (L.att_blocks > 0 && !L.att_tc && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
   L.ring_bytes = ring;
   L.total = L.st[P - 1].end;

@@ -140,9 +140,17 @@ def test_encoder_decoder_layout_and_its_checks(built_lib):
         st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
         return L.pm_status_string(st), L.pm_last_error(None), sb.value, rb.value, wb.value
 
-    # config 5 as given: sequences of 256 tokens are refused (attention is built for up to 128)
-    st, msg = query(I.cfg5())[:2]
-    assert st == b"PM_ERR_UNSUPPORTED" and b"seq_len <= 128" in msg
+    # config 5 as given (133 stages, sequences of 256 tokens) is laid out, but its rings do not fit one GPU
+    st, _, sb, rb, wb = query(I.cfg5())
+    assert st == b"PM_OK" and rb > 500e9
+    # beyond 128 tokens attention exists for 256 tokens, bf16 and heads of width 64 only
+    st, msg = query(I.cfg5_small(compute="f32", d_model=128, n_heads=2, seq_len=256, batch=1))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
+    st, msg = query(I.cfg5_small(compute="bf16", d_model=128, n_heads=2, seq_len=512, batch=1))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
+    st, msg = query(I.cfg5_small(compute="bf16", d_model=128, n_heads=4, seq_len=256, batch=1))[:2]
+    assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
+    assert query(I.cfg5_small(compute="bf16", d_model=128, n_heads=2, seq_len=256, batch=1))[0] == b"PM_OK"
     # its 12 + 12 layers with 128-token sequences do not fit one GPU in the tick-major stash plan; the 4 + 4 layer cut does
     st, _, sb, rb, wb = query(I.cfg5_cut(12, 12))
     assert st == b"PM_OK" and rb > 500e9 and sb < 12e9

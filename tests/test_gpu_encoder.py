@@ -111,6 +111,32 @@ def test_encoder_decoder_tensor_core_attention_shape(cuda_device):
     print("enc-dec tc attention worst relative weight error (per stage vector)", worst)
 
 
+def test_encoder_256_token_attention(cuda_device):
+    """Sequences of 256 tokens (two blocks of 128 query rows per head) on the tensor-core attention kernels."""
+    wl = I.cfg4_small(compute="bf16", n_layers=2, d_model=128, n_heads=2, d_ff=256, seq_len=256, batch=2, vocab=200, steps=10)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("256-token attention loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("256-token attention worst relative weight error (per stage vector)", worst)
+
+
+def test_encoder_decoder_256_token_attention(cuda_device):
+    """Config 5's own sequence length: causal self-attention and cross-attention over 256 tokens."""
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=128, n_heads=2, d_ff=256, seq_len=256, batch=2, vocab=200, steps=8)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("enc-dec 256-token attention loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("enc-dec 256-token attention worst relative weight error (per stage vector)", worst)
+
+
 def test_cfg5_widths_first_microbatches(cuda_device):
     """Config 5's widths (d_model 1024, 16 heads, FFN 4096, 32 sequences of 128 tokens) on one encoder and one
     decoder layer with a vocabulary of 4096: two microbatches fed and drained.  Every GEMM runs on the CTA-pair
