@@ -137,11 +137,12 @@ def test_encoder_decoder_256_token_attention(cuda_device):
     print("enc-dec 256-token attention worst relative weight error (per stage vector)", worst)
 
 
-def test_cfg5_widths_first_microbatches(cuda_device):
-    """Config 5's widths (d_model 1024, 16 heads, FFN 4096, 32 sequences of 128 tokens) on one encoder and one
-    decoder layer with a vocabulary of 4096: two microbatches fed and drained.  Every GEMM runs on the CTA-pair
-    kernels, attention (self, causal, cross) on the tensor-core kernels."""
-    wl = I.cfg5_cut(1, 1, vocab=4096)
+@pytest.mark.parametrize("shape", [dict(seq_len=256, batch=16), dict(seq_len=128, batch=32)])
+def test_cfg5_widths_first_microbatches(cuda_device, shape):
+    """Config 5's widths (d_model 1024, 16 heads, FFN 4096; 16 sequences of 256 tokens as the config has them, and
+    32 of 128) on one encoder and one decoder layer with a vocabulary of 4096: two microbatches fed and drained.
+    Every GEMM runs on the CTA-pair kernels, attention (self, causal, cross) on the tensor-core kernels."""
+    wl = I.cfg5_cut(1, 1, vocab=4096, **shape)
     n = 2
     params0 = I.init_encoder_params(wl)
     res = run_oracle(wl, params0, n)

@@ -79,6 +79,39 @@ def test_update_variants_match_oracle(cuda_device, optimizer, kw):
             np.testing.assert_array_equal(got[name].view(np.uint32), ref[name].view(np.uint32), err_msg=f"{name} k={k}")
 
 
+@pytest.mark.parametrize("k", [3, 2000])
+def test_adam_on_zero_and_denormal_state_matches_oracle_bitwise(cuda_device, k):
+    """Parameters that have seen no gradient yet (g = m = s = 0: untouched embedding rows), negative zeros, moments
+    that have decayed into the denormal range and zero weights: the kernel keeps the zeros out of its division and
+    square-root sequences, and the bits must still be those of the plain formula.  At k = 2000 both bias corrections
+    have rounded to 1."""
+    case = I.update_sweep_case(40000, 4, "adam")
+    n = case["total"]
+    idx = np.arange(n)
+    valid = np.zeros(n, dtype=bool)                          # the padding behind each stage stays zero
+    for o, c in zip(case["offsets"], case["counts"]):
+        valid[o:o + c] = True
+    zero = ((idx // 512) % 3 == 0) & valid                   # whole rows of zeros
+    for name in ("g", "m", "s"):
+        case[name][zero] = 0.0
+    case["m"][(idx % 512 == 7) & zero] = -0.0
+    case["g"][(idx % 512 == 9) & zero] = -0.0
+    den = ((idx // 512) % 3 == 1) & valid
+    tiny = np.float32(1e-45)
+    case["m"][den & (idx % 4 == 0)] = tiny                   # smallest denormal, both signs
+    case["m"][den & (idx % 4 == 1)] = -tiny
+    case["s"][den & (idx % 4 < 2)] = tiny
+    case["g"][den & (idx % 4 < 2)] = 0.0
+    case["s"][den & (idx % 4 == 2)] = np.float32(3e-39)      # denormal second moment under a normal first moment
+    case["w"][(idx % 64 == 5)] = 0.0                         # zero weights (biases) take the step as it is
+    hp = hp_("adam")
+    with np.errstate(all="ignore"):
+        ref = oracle_update(case, hp, k)
+    got = gpu_update(case, hp, k)
+    for name in ref:
+        np.testing.assert_array_equal(got[name].view(np.uint32), ref[name].view(np.uint32), err_msg=name)
+
+
 def test_update_with_equal_delays_leaves_delta_alone(cuda_device):
     # tau_fwd = tau_bkwd (weight-stashing style delays): no gap, so no correction state is kept
     case = I.update_sweep_case(20000, 4, "sgdm")
