@@ -865,13 +865,14 @@ static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
 }
 
 // Embedding gradient: dTable[v] = sqrt(d) * sum over tokens t with id[t] == v (ascending t) of du_total[t].
-// A block owns kEmbRows consecutive vocabulary rows and a slice of the columns.  It reads the microbatch's token
-// ids once (16 consecutive tokens per thread) and compacts the tokens that fall into its rows into a list in
-// ascending token order (a prefix sum over the per-thread counts).  A row with few tokens is summed by one warp; a row with many (frequent
-// ids under a Zipf distribution) by all eight, each adding a contiguous segment of the row's tokens in order, the
-// eight partial sums then added in warp order.  Tokens are gathered eight at a time so that their loads are in
+// A block owns up to kEmbRows vocabulary rows (row v belongs to block v mod the number of blocks, so that the
+// frequent ids of a Zipf distribution are spread over the blocks) and a slice of the columns.  It reads the
+// microbatch's token ids once (16 consecutive tokens per thread) and compacts the tokens that fall into its rows
+// into a list in ascending token order (a prefix sum over the per-thread counts).  A row with few tokens is summed
+// by one warp; a row with many by all eight, each adding a contiguous segment of the row's tokens in order, the
+// eight partial sums then added in warp order.  Several tokens are gathered at a time so that their loads are in
 // flight together.  Every row is written (zeros included) and the order of the additions is fixed.
-constexpr int kEmbRows = 64;                          // a block's columns: 32 lanes x CPL (4, 8 or 16) columns per lane
+constexpr int kEmbRows = 256;                         // a block's columns: 32 lanes x CPL (4, 8 or 16) columns per lane
 constexpr int kEmbHeavy = 24;                         // tokens per row from which the block shares the row
 
 template <typename AT> __device__ __forceinline__ void load4(const AT* p, float (&v)[4]);
@@ -935,17 +936,20 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0) return;
-  const int v0 = blockIdx.x * kEmbRows;
+  // rows are dealt to the blocks round-robin (row v belongs to block v mod gridDim.x, a power of two): the frequent
+  // ids of a Zipf distribution, which sit next to each other at the start of the vocabulary, land in different blocks
+  const int nb_shift = __ffs((int)gridDim.x) - 1, nb_mask = (int)gridDim.x - 1, blk = (int)blockIdx.x;
   const int dm = s.d_in;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int col = blockIdx.z * kEmbCols + lane * CPL;        // this lane's columns
-  if (v0 >= s.vocab || blockIdx.z * kEmbCols >= dm) return;
+  if (blk >= s.vocab || blockIdx.z * kEmbCols >= dm) return;
+  const int n_rows = (s.vocab - blk + nb_mask) >> nb_shift;  // rows blk, blk + gridDim.x, ... (at most kEmbRows)
   extern __shared__ int32_t hits[];                          // [T] (token << 8 | row within the block), ascending token
   __shared__ int warp_cnt[2][8];
   __shared__ int row_cnt[kEmbRows], row_start[kEmbRows];
   int32_t* sub = hits + t.T;                                 // [T] token indices grouped by row, ascending inside a row
   float (*part)[kEmbCols] = reinterpret_cast<float (*)[kEmbCols]>(sub + t.T);   // [8][kEmbCols] shared rows: per-warp partial sums
-  if (threadIdx.x < kEmbRows) row_cnt[threadIdx.x] = 0;
+  for (int i = threadIdx.x; i < kEmbRows; i += 256) row_cnt[i] = 0;
   __syncthreads();
   const int32_t* ids = ring_at<int32_t>(t, s.ids_ring, (int)(d.b_mb % s.ids_depth), (uint64_t)t.T);
   int nh = 0;                                                // hits so far (the same value in every thread)
@@ -956,12 +960,14 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int4 q = __ldg(reinterpret_cast<const int4*>(ids + tok0) + k);
-        rel[4 * k] = q.x - v0; rel[4 * k + 1] = q.y - v0; rel[4 * k + 2] = q.z - v0; rel[4 * k + 3] = q.w - v0;
+        rel[4 * k] = q.x; rel[4 * k + 1] = q.y; rel[4 * k + 2] = q.z; rel[4 * k + 3] = q.w;
       }
     } else {
 #pragma unroll
-      for (int k = 0; k < 16; ++k) rel[k] = tok0 + k < t.T ? __ldg(ids + tok0 + k) - v0 : -1;
+      for (int k = 0; k < 16; ++k) rel[k] = tok0 + k < t.T ? __ldg(ids + tok0 + k) : -1;
     }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) rel[k] = (rel[k] >= 0 && (rel[k] & nb_mask) == blk) ? (rel[k] >> nb_shift) : -1;   // row inside this block
     int mine = 0;
 #pragma unroll
     for (int k = 0; k < 16; ++k) mine += (rel[k] >= 0 && rel[k] < kEmbRows) ? 1 : 0;
@@ -982,10 +988,21 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
     __syncthreads();                                         // warp_cnt is reused by the next pass
   }
   __syncthreads();
-  if (threadIdx.x == 0) { int a = 0; for (int r = 0; r < kEmbRows; ++r) { row_start[r] = a; a += row_cnt[r]; } }
+  {                                                          // exclusive prefix of the row counts (kEmbRows = 256 = one per thread)
+    const int mine = row_cnt[threadIdx.x];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+    if (lane == 31) warp_cnt[1][warp] = incl;
+    __syncthreads();
+    int base = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) if (w < warp) base += warp_cnt[1][w];
+    row_start[threadIdx.x] = base + incl - mine;
+  }
   __syncthreads();
   // the list, grouped by row: warp w scans it once for each of its rows and copies the matching tokens in order
-  for (int rr = warp; rr < kEmbRows; rr += 8) {
+  for (int rr = warp; rr < n_rows; rr += 8) {
     if (row_cnt[rr] == 0) continue;
     int seen = row_start[rr];
     for (int hb = 0; hb < nh; hb += 32) {
@@ -1003,9 +1020,9 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   const bool col_ok = col < dm;                              // widths are multiples of CPL
   const int col_ld = col_ok ? col : dm - CPL;                  // every lane takes part in the warp-wide steps; lanes beyond the width load a valid address
   // ---- rows with many tokens: the whole block per row
-  for (int rr = 0; rr < kEmbRows; ++rr) {
+  for (int rr = 0; rr < n_rows; ++rr) {
     const int cnt = row_cnt[rr];
-    if (cnt < kEmbHeavy || v0 + rr >= s.vocab) continue;     // uniform over the block
+    if (cnt < kEmbHeavy) continue;                           // uniform over the block
     const int k_lo = (int)((long long)cnt * warp / 8), k_hi = (int)((long long)cnt * (warp + 1) / 8);
     float acc[CPL];
 #pragma unroll
@@ -1018,14 +1035,13 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
       float a = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) a = __fadd_rn(a, part[w][c]);
-      t.a.grad[s.tab_off + (uint64_t)(v0 + rr) * dm + blockIdx.z * kEmbCols + c] = a;
+      t.a.grad[s.tab_off + (uint64_t)((rr << nb_shift) + blk) * dm + blockIdx.z * kEmbCols + c] = a;
     }
     __syncthreads();
   }
   // ---- the other rows: one warp per row
-  for (int rr = warp; rr < kEmbRows; rr += 8) {
-    const int v = v0 + rr;
-    if (v >= s.vocab) break;
+  for (int rr = warp; rr < n_rows; rr += 8) {
+    const int v = (rr << nb_shift) + blk;
     const int cnt = row_cnt[rr];
     if (cnt >= kEmbHeavy) continue;
     float acc[CPL];
@@ -1065,7 +1081,11 @@ cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
     // columns per lane: wide models are cut into column slices so that a row with many tokens is spread over blocks
     const int dm = t.max_embed_dim;
     const int cpl = (dm % 16 == 0 && dm <= 512) ? 16 : (dm % 8 == 0 ? 8 : 4);
-    dim3 g((t.max_vocab + kEmbRows - 1) / kEmbRows, t.n_embed, (dm + 32 * cpl - 1) / (32 * cpl));
+    const int slices = (dm + 32 * cpl - 1) / (32 * cpl);
+    int n_blk = 1;                                           // a power of two with at most kEmbRows rows per block ...
+    while (n_blk * kEmbRows < t.max_vocab) n_blk <<= 1;
+    while (n_blk * slices * t.n_embed < 2 * 148 && t.max_vocab / n_blk > 32) n_blk <<= 1;   // ... and enough blocks for a small vocabulary
+    dim3 g(n_blk, t.n_embed, slices);
     // the hit list, the same tokens grouped by row, and the per-warp partial sums of a shared row
     const size_t smem = 2 * sizeof(int32_t) * (size_t)t.T + sizeof(float) * 8 * 32 * (size_t)cpl;
     auto go = [&](auto kernel) -> cudaError_t {
