@@ -708,11 +708,13 @@ __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
   t.a.grad[s.beta_off + c] = b2;
 }
 
-// Fused LayerNorm backward (widths that are multiples of 8, at most NP*256): one pass over du, x and the skip
-// gradient produces dx and the partial column sums of dgain, dbias.  A block owns ln_chunk_rows rows; warp w takes
-// rows w, w+8, ... in ascending order, a lane owns 8 consecutive columns per 256-column group; per-warp partials are
-// added in warp order, per-block partials in block order by ln_fused_finish_kernel.
-template <typename AT, int NP>
+// Fused LayerNorm backward (widths that are multiples of 8, at most WPR*NP*256): one pass over du, x and the skip
+// gradient produces dx and the partial column sums of dgain, dbias.  A block owns ln_chunk_rows rows; WPR warps
+// share a row (each NP*256 of its columns; with WPR = 2 the two row sums meet in shared memory behind a 64-thread
+// named barrier, first half + second half), the 8 / WPR warp groups take rows g, g + 8 / WPR, ... in ascending
+// order; a lane owns 8 consecutive columns per 256-column group; per-warp partials are added in warp order,
+// per-block partials in block order by ln_fused_finish_kernel.
+template <typename AT, int NP, int WPR>
 __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(TickArgs t) {
   const int li = blockIdx.y, p = t.ln_ids[li];
   const StageDyn& d = t.dyn[p];
@@ -733,10 +735,13 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   const bool accumulate = s.from_memory && !s.mem_first;
   const float gapf = (float)s.gap;
   const bool corr = d.use_delta != 0;
+  const int half = WPR == 2 ? (warp & 1) : 0, rw = WPR == 2 ? (warp >> 1) : warp;
+  const int cbase = half * NP * 256;                         // first column of this warp's share of a row
+  __shared__ float xs[2][4][2][2];                           // [row parity][warp pair][half][s1, s2]
   float gb[NP][8], ag[NP][8], ab[NP][8];
 #pragma unroll
   for (int q = 0; q < NP; ++q) {
-    const int c = q * 256 + lane * 8;
+    const int c = cbase + q * 256 + lane * 8;
 #pragma unroll
     for (int k = 0; k < 8; ++k) { gb[q][k] = 0.f; ag[q][k] = 0.f; ab[q][k] = 0.f; }
     if (c < dm) {
@@ -748,7 +753,8 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   }
   const bool has_gs = gs != nullptr;
   if (!has_gs) gs = du;                                      // keeps the loads below free of branches; the value is not used
-  for (int r = r0 + warp; r < r1; r += 8) {
+  int par = 0;
+  for (int r = r0 + rw; r < r1; r += 8 / WPR, par ^= 1) {
     const float mu = st[2 * r], rstd = st[2 * r + 1];
     const uint64_t ro = (uint64_t)r * dm;
     float xh[NP][8], dxh[NP][8];
@@ -757,14 +763,14 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
     float xa[NP][8], da[NP][8], sa[NP][8];
 #pragma unroll
     for (int q = 0; q < NP; ++q) {
-      const int c = min(q * 256 + lane * 8, dm - 8);
+      const int c = min(cbase + q * 256 + lane * 8, dm - 8);
       load8<AT>(x + ro + c, xa[q]);
       load8<AT>(du + ro + c, da[q]);
       load8<AT>(gs + ro + c, sa[q]);
     }
 #pragma unroll
     for (int q = 0; q < NP; ++q) {
-      const int c = q * 256 + lane * 8;
+      const int c = cbase + q * 256 + lane * 8;
       if (c < dm) {
         float (&xv)[8] = xa[q];
         float (&dv)[8] = da[q];
@@ -784,12 +790,27 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
         for (int k = 0; k < 8; ++k) { xh[q][k] = 0.f; dxh[q][k] = 0.f; }
       }
     }
-    s1 = warp_sum(s1) / (float)dm;
-    s2 = warp_sum(s2) / (float)dm;
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    if (WPR == 2) {
+      // the slot alternates with the row: a warp that runs ahead writes the other slot, and cannot come back to
+      // this one before its partner has passed the next row's barrier
+      if (lane == 0) { xs[par][rw][half][0] = s1; xs[par][rw][half][1] = s2; }
+      switch (rw) {                                          // barrier numbers as immediates: the kernel reserves five, not all sixteen
+        case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
+        case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
+        case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
+        default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+      }
+      s1 = xs[par][rw][0][0] + xs[par][rw][1][0];
+      s2 = xs[par][rw][0][1] + xs[par][rw][1][1];
+    }
+    s1 /= (float)dm;
+    s2 /= (float)dm;
     if (out) {
 #pragma unroll
       for (int q = 0; q < NP; ++q) {
-        const int c = q * 256 + lane * 8;
+        const int c = cbase + q * 256 + lane * 8;
         if (c < dm) {
           float o[8];
 #pragma unroll
@@ -817,8 +838,10 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   float* part = ws_at<float>(t, t.lnred_off) + ((uint64_t)li * t.ln_chunks + chunk) * (2 * (uint64_t)t.max_ln_dim);
   for (int c = threadIdx.x; c < dm; c += 256) {
     float a = 0.f, b2 = 0.f;
+    const int hf = WPR == 2 ? c / (NP * 256) : 0, lc = c - hf * (NP * 256);   // the warps that hold this column, in warp order
 #pragma unroll
-    for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, lnred[(w * 2 + 0) * (NP * 256) + c]); b2 = __fadd_rn(b2, lnred[(w * 2 + 1) * (NP * 256) + c]); }
+    for (int w = 0; w < 8; ++w)
+      if (WPR == 1 || (w & 1) == hf) { a = __fadd_rn(a, lnred[(w * 2 + 0) * (NP * 256) + lc]); b2 = __fadd_rn(b2, lnred[(w * 2 + 1) * (NP * 256) + lc]); }
     part[c] = a;
     part[t.max_ln_dim + c] = b2;
   }
@@ -850,16 +873,16 @@ __global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
   t.a.grad[s.beta_off + c] = b2;
 }
 
-template <typename AT, int NP>
+template <typename AT, int NP, int WPR>
 static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
   const size_t smem = (size_t)8 * 2 * NP * 256 * sizeof(float);
   static bool attr_set = false;
   if (!attr_set && smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute((const void*)ln_bwd_fused_kernel<AT, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute((const void*)ln_bwd_fused_kernel<AT, NP, WPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  ln_bwd_fused_kernel<AT, NP><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(t);
+  ln_bwd_fused_kernel<AT, NP, WPR><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(t);
   ln_fused_finish_kernel<<<dim3((t.max_ln_dim + 255) / 256, t.n_ln), 256, 0, stream>>>(t);
   return cudaGetLastError();
 }
@@ -1061,8 +1084,8 @@ int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.ln_fused ? 2 : (
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
   if (t.any_ln && t.ln_fused) {
-    if (dtype == PM_F32) e = t.max_ln_dim <= 256 ? launch_ln_fused<float, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<float, 2>(t, stream) : launch_ln_fused<float, 4>(t, stream));
-    else e = t.max_ln_dim <= 256 ? launch_ln_fused<__nv_bfloat16, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<__nv_bfloat16, 2>(t, stream) : launch_ln_fused<__nv_bfloat16, 4>(t, stream));
+    if (dtype == PM_F32) e = t.max_ln_dim <= 256 ? launch_ln_fused<float, 1, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<float, 2, 1>(t, stream) : launch_ln_fused<float, 2, 2>(t, stream));
+    else e = t.max_ln_dim <= 256 ? launch_ln_fused<__nv_bfloat16, 1, 1>(t, stream) : (t.max_ln_dim <= 512 ? launch_ln_fused<__nv_bfloat16, 2, 1>(t, stream) : launch_ln_fused<__nv_bfloat16, 2, 2>(t, stream));
     if (e != cudaSuccess) return e;
   } else if (t.any_ln) {
     dim3 g1((t.T + 7) / 8, t.n_ln), g2((t.max_ln_dim + kLnCols - 1) / kLnCols, t.row_chunks, t.n_ln);

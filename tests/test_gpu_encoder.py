@@ -30,6 +30,22 @@ def test_encoder_fp32(cuda_device, kw):
     print("encoder fp32 worst relative weight error", worst)
 
 
+@pytest.mark.parametrize("d_model", [328, 776])
+def test_encoder_fp32_wide_rows(cuda_device, d_model):
+    """LayerNorm rows of two 256-column groups with a ragged last group (328), and rows shared by two warps with a
+    ragged second half (776).  SGD with momentum: with hundreds of thousands of weights some gradient sums cancel
+    to rounding level, and Adam would turn the sign of such a sum into a step of alpha on either side."""
+    wl = I.encoder_workload("wide_rows", 1, d_model, 2, 64, 8, 9, 60, compute="f32", optimizer="sgdm", alpha=0.02,
+                            beta1=0.9, K=3, D=0.1, steps=10, seed=191005124 + 46)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
+    worst = compare_params(pipe, res, 2e-5)
+    print("encoder fp32 wide rows worst relative weight error", worst)
+
+
 def test_encoder_bf16_small(cuda_device):
     wl = I.cfg4_small(compute="bf16")
     params0 = I.init_encoder_params(wl)
