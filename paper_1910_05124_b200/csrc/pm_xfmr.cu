@@ -400,6 +400,39 @@ cudaError_t attention_set_smem_limits(int S, int dk, int dtype) {
   return e;
 }
 
+// ---- loss reduction shared by the cross-entropy kernels ----
+// per-token loss of this block's row; the last block to arrive adds all of them in a fixed order (strided per-thread
+// partials over the first 256 threads, then a fixed tree).  Called by every thread of the block.
+__device__ __forceinline__ void ce_finish(const TickArgs& t, const StageDyn& d, int row, float mx, float sum, float logit_tgt) {
+  float* rowloss = ws_at<float>(t, t.rowloss_off);
+  unsigned int* counter = reinterpret_cast<unsigned int*>(ws_at<float>(t, t.lossred_off) + 64);
+  __shared__ bool last;
+  if (threadIdx.x == 0) {
+    rowloss[row] = (mx + logf(sum)) - logit_tgt;
+    __threadfence();
+    last = atomicAdd(counter, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (last) {
+    __threadfence();
+    __shared__ float tree[256];
+    if (threadIdx.x < 256) {
+      float a = 0.f;
+      for (int r = threadIdx.x; r < t.T; r += 256) a += reinterpret_cast<volatile float*>(rowloss)[r];
+      tree[threadIdx.x] = a;
+    }
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+      if ((int)threadIdx.x < off) tree[threadIdx.x] += tree[threadIdx.x + off];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      ws_at<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = tree[0] / (float)t.T;
+      *counter = 0;
+    }
+  }
+}
+
 // ---- cross-entropy at the last stage -------------------------------------------------------------------------------
 // One block per token: lse = max + log(sum exp(logit - max)); loss_t = lse - logit[target];
 // dlogits = (softmax - onehot) / T in the activation type, written where the last stage reads its incoming
@@ -500,35 +533,113 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
       dl[c] = from_f<AT>(pr * invT);
     }
   }
-  float* rowloss = ws_at<float>(t, t.rowloss_off);
-  unsigned int* counter = reinterpret_cast<unsigned int*>(ws_at<float>(t, t.lossred_off) + 64);
-  __shared__ bool last;
+  ce_finish(t, d, row, mx, sum, lg[tgt]);
+}
+
+// Rows longer than the register path holds (a vocabulary of tens of thousands): 512 threads read the fp32 row once
+// into shared memory (four float4 in flight per thread), the exponentials replace it there, and the gradient is
+// written from them as 8-byte (bf16) or 16-byte (fp32) vectors.
+constexpr int kCeLongThreads = 1024;
+template <typename AT> __device__ __forceinline__ void store4(AT* p, float a, float b, float c, float e);
+template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float e) { *reinterpret_cast<float4*>(p) = make_float4(a, b, c, e); }
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float e) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, e);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
+
+// fp32 activations take the exact exponential and a true division; with bf16 activations the gradient is rounded to 8
+// bits anyway, so the exponential is the hardware base-2 one (relative error ~2^-21 |x|) and the division a product
+// with the reciprocal of the row sum.  The loss itself uses the fp32 sum of these exponentials either way.
+template <typename AT> __device__ __forceinline__ float ce_exp(float x);
+template <> __device__ __forceinline__ float ce_exp<float>(float x) { return expf(x); }
+template <> __device__ __forceinline__ float ce_exp<__nv_bfloat16>(float x) { return __expf(x); }
+template <typename AT> __device__ __forceinline__ float ce_div(float e, float sum, float rsum);
+template <> __device__ __forceinline__ float ce_div<float>(float e, float sum, float) { return e / sum; }
+template <> __device__ __forceinline__ float ce_div<__nv_bfloat16>(float e, float, float rsum) { return e * rsum; }
+
+template <typename AT>
+__global__ void __launch_bounds__(kCeLongThreads) ce_loss_long_kernel(TickArgs t) {
+  const StageDyn& d = t.dyn[t.P - 1];
+  if (d.b_mb < 0) return;
+  const StageDev& sl = t.st[t.P - 1];
+  const int V = t.n_out_last, row = blockIdx.x, n4 = V >> 2;
+  const uint64_t n = (uint64_t)t.T * V;
+  const float* lg = ws_at<float>(t, t.yout_off) + (uint64_t)((d.tick + 1) & 1) * n + (uint64_t)row * V;
+  const float4* lg4 = reinterpret_cast<const float4*>(lg);
+  const int32_t tgt = (ws_at<int32_t>(t, t.tgt_off) + (uint64_t)(d.b_mb % (t.P + 1)) * t.T)[row];
+  AT* dl = gin_read<AT>(t, sl, d) + (uint64_t)row * V;
+  extern __shared__ float4 rowbuf[];                         // [V / 4]
+  __shared__ float red[kCeLongThreads / 32];
+  __shared__ float bc[3];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < n4; i += 4 * kCeLongThreads) {
+    float4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) q[u] = __ldcs(lg4 + min(i + u * kCeLongThreads, n4 - 1));
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (i + u * kCeLongThreads < n4) {
+        rowbuf[i + u * kCeLongThreads] = q[u];
+        mx = fmaxf(fmaxf(mx, fmaxf(q[u].x, q[u].y)), fmaxf(q[u].z, q[u].w));
+      }
+  }
+  mx = warp_max(mx);
+  if (lane == 0) red[warp] = mx;
+  __syncthreads();
   if (threadIdx.x == 0) {
-    rowloss[row] = (mx + logf(sum)) - lg[tgt];
-    __threadfence();
-    last = atomicAdd(counter, 1u) == gridDim.x - 1;
+    float m = red[0];
+    for (int i = 1; i < kCeLongThreads / 32; ++i) m = fmaxf(m, red[i]);
+    bc[0] = m;
+    bc[2] = reinterpret_cast<const float*>(rowbuf)[tgt];      // the target's logit, before the exponentials replace the row
   }
   __syncthreads();
-  if (last) {
-    // the last block adds the per-token losses in a fixed order: strided per-thread partials, then a fixed tree
-    __threadfence();
-    __shared__ float tree[256];
-    float a = 0.f;
-    for (int r = threadIdx.x; r < t.T; r += 256) a += reinterpret_cast<volatile float*>(rowloss)[r];
-    tree[threadIdx.x] = a;
-    __syncthreads();
-    for (int off = 128; off > 0; off >>= 1) {
-      if ((int)threadIdx.x < off) tree[threadIdx.x] += tree[threadIdx.x + off];
-      __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-      ws_at<float>(t, t.loss_off)[d.b_mb % t.loss_cap] = tree[0] / (float)t.T;
-      *counter = 0;
-    }
+  mx = bc[0];
+  const float logit_tgt = bc[2];
+  float sum = 0.f;
+  for (int i = threadIdx.x; i < n4; i += kCeLongThreads) {
+    float4 q = rowbuf[i];
+    q.x = ce_exp<AT>(q.x - mx); q.y = ce_exp<AT>(q.y - mx); q.z = ce_exp<AT>(q.z - mx); q.w = ce_exp<AT>(q.w - mx);
+    sum += q.x; sum += q.y; sum += q.z; sum += q.w;
+    rowbuf[i] = q;
   }
+  sum = warp_sum(sum);
+  if (lane == 0) red[warp] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) { float a = 0.f; for (int i = 0; i < kCeLongThreads / 32; ++i) a += red[i]; bc[1] = a; }
+  __syncthreads();
+  sum = bc[1];
+  const float invT = 1.0f / (float)t.T, rsum = 1.0f / sum;
+  for (int i = threadIdx.x; i < n4; i += kCeLongThreads) {
+    const float4 q = rowbuf[i];
+    const int c = 4 * i;
+    float p0 = ce_div<AT>(q.x, sum, rsum), p1 = ce_div<AT>(q.y, sum, rsum), p2 = ce_div<AT>(q.z, sum, rsum), p3 = ce_div<AT>(q.w, sum, rsum);
+    if (tgt == c) p0 -= 1.0f;
+    if (tgt == c + 1) p1 -= 1.0f;
+    if (tgt == c + 2) p2 -= 1.0f;
+    if (tgt == c + 3) p3 -= 1.0f;
+    store4<AT>(dl + c, p0 * invT, p1 * invT, p2 * invT, p3 * invT);
+  }
+  ce_finish(t, d, row, mx, sum, logit_tgt);
 }
 
 cudaError_t launch_ce_loss(const TickArgs& t, int dtype, cudaStream_t stream) {
+  const int V = t.n_out_last;
+  const size_t row_bytes = sizeof(float) * (size_t)V;
+  if (V > 8192 && (V & 3) == 0 && row_bytes <= 200 * 1024) {
+    static bool attr_set[2] = {false, false};
+    const int which = dtype == PM_F32 ? 0 : 1;
+    if (!attr_set[which]) {
+      cudaError_t e = dtype == PM_F32
+          ? cudaFuncSetAttribute((const void*)ce_loss_long_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+          : cudaFuncSetAttribute((const void*)ce_loss_long_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_set[which] = true;
+    }
+    if (dtype == PM_F32) ce_loss_long_kernel<float><<<t.T, kCeLongThreads, row_bytes, stream>>>(t);
+    else ce_loss_long_kernel<__nv_bfloat16><<<t.T, kCeLongThreads, row_bytes, stream>>>(t);
+    return cudaGetLastError();
+  }
   if (dtype == PM_F32) ce_loss_kernel<float><<<t.T, 256, 0, stream>>>(t);
   else ce_loss_kernel<__nv_bfloat16><<<t.T, 256, 0, stream>>>(t);
   return cudaGetLastError();

@@ -46,6 +46,22 @@ def test_encoder_fp32_wide_rows(cuda_device, d_model):
     print("encoder fp32 wide rows worst relative weight error", worst)
 
 
+@pytest.mark.parametrize("compute,vocab", [("f32", 8200), ("bf16", 8200), ("f32", 8198)])
+def test_long_logit_rows(cuda_device, compute, vocab):
+    """Vocabularies beyond 8192: the cross-entropy kernel that keeps the row of logits in shared memory (row lengths
+    that are multiples of four) and the plain three-pass path (8198).  SGD with momentum, see the wide-row test."""
+    wl = I.encoder_workload("long_rows", 1, 32, 2, 64, 8, 3, vocab, compute=compute, optimizer="sgdm", alpha=0.02,
+                            beta1=0.9, K=3, D=0.1, steps=10, seed=191005124 + 47)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    f32 = compute == "f32"
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    worst = compare_params(pipe, res, 2e-5 if f32 else 2e-2, per_stage=not f32)
+    print("long logit rows", compute, vocab, "worst relative weight error", worst)
+
+
 def test_encoder_bf16_small(cuda_device):
     wl = I.cfg4_small(compute="bf16")
     params0 = I.init_encoder_params(wl)
