@@ -50,7 +50,7 @@ def make_grad_fn(stage_acts, data_fn, compute="f32"):
     return grad_fn
 
 
-def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None):
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0):
     """Run a pm_inputs.Workload-like description through the recurrence.
 
     params0: per stage a list of (W, b) pairs.  Returns recurrence.Result.
@@ -62,4 +62,4 @@ def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=N
               t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
     grad_fn = make_grad_fn(stage_acts, data_fn, wl.compute)
     return recurrence.run(flat0, wl.tau_fwd, wl.tau_bkwd, grad_fn,
-                          wl.steps if n_steps is None else n_steps, hp, dtype=dtype, on_step=on_step)
+                          wl.steps if n_steps is None else n_steps, hp, dtype=dtype, on_step=on_step, warmup=warmup)

@@ -18,6 +18,13 @@ Readings where the paper is silent:
     writes version t+1.
   * One microbatch per update (N = 1): microbatch index = update index.
 
+Warm-up epochs (PipeMareW, Section 4): the first `warmup` microbatches run the synchronous baseline, i.e. the same
+loop with every delay zero (standard step size, no T2 correction, delta left alone); PipeMare then starts from
+those weights and optimiser state.  Readings: the pipeline is empty at the switch, so version indices are clamped
+at `warmup` (the weights the warm-up produced are the only ones the filling pipeline can see); the T1 annealing
+counts steps from the switch; the base step-size schedule and Adam's bias correction keep counting from 0;
+delta starts at 0 at the switch.
+
 Pins: with all tau = 0 the loop is synchronous SGD, bit for bit; with T2 off
 and tau_bkwd = tau_fwd it is plain delayed SGD; on the scalar quadratic its
 iterates follow the roots of the characteristic polynomials of Sections 3.1,
@@ -39,8 +46,8 @@ class Result:
         self.opt = None
 
 
-def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None):
-    """Run n_steps microbatches.
+def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None, warmup=0):
+    """Run n_steps microbatches, the first `warmup` of them synchronously.
 
     params0:   per stage, a list of arrays (that stage's tensors).
     grad_fn:   (t, u_fwd, u_bkwd) -> (loss, grads) with grads shaped like params0.
@@ -57,16 +64,18 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
     res = Result()
 
     def version(i, t, lag):
-        v = max(0, t - lag)
+        v = max(min(warmup, t), t - lag)       # nothing older than the end of the warm-up (or version 0) exists
         return v, hist[i][-1 - (t - v)]
 
     for t in range(n_steps):
+        sync = t < warmup
         u_fwd, u_bkwd = [], []
         for i in range(P):
-            vf, wf = version(i, t, tau_fwd[i])
-            vb, wb = version(i, t, tau_bkwd[i])
+            tf, tb = (0, 0) if sync else (tau_fwd[i], tau_bkwd[i])
+            vf, wf = version(i, t, tf)
+            vb, wb = version(i, t, tb)
             u_fwd.append(wf)
-            u_bkwd.append([U.corrected_backward_weights(a, d, tau_fwd[i], tau_bkwd[i], hp["t2"])
+            u_bkwd.append([U.corrected_backward_weights(a, d, tf, tb, hp["t2"])
                            for a, d in zip(wb, delta[i])])
             res.book.append((t, i + 1, vf, vb))
         loss, grads = grad_fn(t, u_fwd, u_bkwd)
@@ -75,8 +84,9 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
             new_stage = []
             for j, a in enumerate(w[i]):
                 g = np.asarray(grads[i][j], dtype=dtype)
+                tf, tb = (0, 0) if sync else (tau_fwd[i], tau_bkwd[i])
                 a_new, opt[i][j], delta[i][j] = U.pipemare_update(
-                    a, opt[i][j], delta[i][j], g, k=t, tau_fwd=tau_fwd[i], tau_bkwd=tau_bkwd[i], hp=hp)
+                    a, opt[i][j], delta[i][j], g, k=t, tau_fwd=tf, tau_bkwd=tb, hp=hp, k_t1=max(t - warmup, 0))
                 new_stage.append(a_new)
             w[i] = new_stage
             hist[i].append(new_stage)

@@ -159,11 +159,11 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
     return grad_fn
 
 
-def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None):
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0):
     """params0: per stage the list of tensors in the order [table] [gain, bias] W b."""
     from . import recurrence
     hp = dict(optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
               t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
     grad_fn = make_grad_fn(wl.stage_specs, data_fn, wl.n_heads, wl.seq_len, wl.vocab, wl.compute)
     return recurrence.run(params0, wl.tau_fwd, wl.tau_bkwd, grad_fn, wl.steps if n_steps is None else n_steps,
-                          hp, dtype=dtype, on_step=on_step)
+                          hp, dtype=dtype, on_step=on_step, warmup=warmup)

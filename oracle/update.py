@@ -86,14 +86,16 @@ def delta_refresh(delta, w_new, w_old, gamma):
     return g * delta + (dt(1) - g) * (w_new - w_old)
 
 
-def pipemare_update(w, opt_state, delta, g, *, k, tau_fwd, tau_bkwd, hp):
+def pipemare_update(w, opt_state, delta, g, *, k, tau_fwd, tau_bkwd, hp, k_t1=None):
     """One update of one tensor of one stage.  Returns (w', opt_state', delta').
 
     hp: dict with optimizer ('sgdm'|'adam'), alpha (float or callable k -> float),
     beta1, beta2, eps, t1 (bool), K, t2 (bool), D.
+    k indexes the base step size and Adam's bias correction; k_t1 (default k) is the step the T1 annealing counts
+    from (after synchronous warm-up epochs, Section 4, the annealing starts where PipeMare starts).
     """
     alpha_base = hp["alpha"](k) if callable(hp["alpha"]) else hp["alpha"]
-    alpha = t1_step_size(alpha_base, tau_fwd, k, hp["K"], hp["t1"])
+    alpha = t1_step_size(alpha_base, tau_fwd, k if k_t1 is None else k_t1, hp["K"], hp["t1"])
     if hp["optimizer"] == "sgdm":
         w_new, v_new = sgdm_step(w, opt_state["v"], g, alpha, hp["beta1"])
         new_state = {"v": v_new}

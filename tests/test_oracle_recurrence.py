@@ -265,3 +265,70 @@ def test_two_argument_gradient_on_scalar_chain():
     ub2 = [[np.array([[-123.0]]), z], [np.array([[0.25]]), z]]
     _, g2 = grad_fn(0, uf, ub2)
     assert g2[0][0][0, 0] == g[0][0][0, 0] and g2[1][0][0, 0] == g[1][0][0, 0]
+
+
+# ---- warm-up epochs (PipeMareW, Section 4): synchronous steps first, PipeMare from there -------------------------
+
+@pytest.mark.parametrize("optimizer", ["sgdm", "adam"])
+def test_warmup_covering_every_step_is_the_synchronous_run(optimizer):
+    params, grad_fn = tiny_net(seed=3)
+    P = len(params)
+    tf, tb = [2 * (P - i) + 1 for i in range(1, P + 1)], [0] * P
+    hp = hp_(optimizer=optimizer, alpha=0.03, beta1=0.9, t1=True, K=4, t2=True, D=0.5)
+    warm = recurrence.run(params, tf, tb, grad_fn, 10, hp, warmup=10)
+    sync = recurrence.run(params, [0] * P, [0] * P, grad_fn, 10, hp_(optimizer=optimizer, alpha=0.03, beta1=0.9))
+    assert warm.losses == sync.losses
+    for a, b in zip(warm.params, sync.params):
+        for x, y in zip(a, b):
+            np.testing.assert_array_equal(x, y)
+    for st in warm.delta:
+        for dlt in st:
+            assert not dlt.any()                               # the accumulator is left alone during the warm-up
+    assert all(vf == t and vb == t for (t, _, vf, vb) in warm.book)
+
+
+def test_warmup_then_pipemare_equals_pipemare_started_from_the_warmed_weights():
+    """Plain SGD keeps no optimiser state, so 'initialise with E synchronous steps' can be replayed by hand: run
+    the synchronous steps, then start an ordinary PipeMare run (T1 counting from 0, delta = 0, versions clamped at
+    its own start) on the remaining microbatches from those weights."""
+    params, grad_fn = tiny_net(seed=4)
+    P, E, n = len(params), 5, 14
+    tf, tb = [2 * (P - i) + 1 for i in range(1, P + 1)], [0] * P
+    hp = hp_(alpha=0.04, beta1=0.0, t1=True, K=6, t2=True, D=0.5)
+    both = recurrence.run(params, tf, tb, grad_fn, n, hp, warmup=E)
+    first = recurrence.run(params, [0] * P, [0] * P, grad_fn, E, hp_(alpha=0.04, beta1=0.0))
+    rest = recurrence.run(first.params, tf, tb, lambda t, uf, ub: grad_fn(t + E, uf, ub), n - E, hp)
+    assert both.losses == first.losses + rest.losses
+    for a, b in zip(both.params, rest.params):
+        for x, y in zip(a, b):
+            np.testing.assert_array_equal(x, y)
+    for a, b in zip(both.delta, rest.delta):
+        for x, y in zip(a, b):
+            np.testing.assert_array_equal(x, y)
+    # versions: synchronous during the warm-up, then clamped at E while the pipeline fills
+    for (t, i, vf, vb) in both.book:
+        assert vb == t
+        assert vf == (t if t < E else max(E, t - tf[i - 1]))
+
+
+def test_warmup_keeps_adam_bias_correction_and_base_schedule_on_the_global_step():
+    """One scalar parameter, gradient 1 at every step, no delays after the switch (tau = 0 everywhere), so the only
+    effects of the warm-up flag are the ones under test: Adam's step is alpha_base(k) * m_hat / sqrt(s_hat) with the
+    bias corrections at the global k (m_hat = s_hat = 1 for a constant gradient), hence w_k = w_0 - sum alpha_base."""
+    sched = lambda k: 0.1 / (k + 1)
+    hp = hp_(optimizer="adam", alpha=sched, beta1=0.9, eps=0.0, t1=True, K=3)
+    res = recurrence.run([[np.array([1.0])]], [0], [0], lambda t, uf, ub: (0.0, [[np.array([1.0])]]), 9, hp,
+                         dtype=np.float64, warmup=4)
+    assert res.params[0][0][0] == pytest.approx(1.0 - sum(sched(k) for k in range(9)), rel=1e-12)
+
+
+def test_t1_annealing_counts_from_the_switch():
+    """Scalar, plain SGD, gradient 1: the step at global k >= E is alpha / tau^(1 - min((k - E)/K, 1))."""
+    tau, E, K, alpha = 7, 3, 4, 0.01
+    hp = hp_(alpha=alpha, t1=True, K=K)
+    traj = []
+    recurrence.run([[np.array([0.0])]], [tau], [0], lambda t, uf, ub: (0.0, [[np.array([1.0])]]), 10, hp,
+                   dtype=np.float64, warmup=E, on_step=lambda t, w: traj.append(float(w[0][0][0])))
+    steps = -np.diff([0.0] + traj)
+    want = [alpha if k < E else alpha / tau ** (1.0 - min((k - E) / K, 1.0)) for k in range(10)]
+    np.testing.assert_allclose(steps, want, rtol=1e-12)
