@@ -179,6 +179,18 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
                          const pm_arenas* arenas, void* ring, uint64_t ring_bytes,
                          void* workspace, uint64_t workspace_bytes, void* stream);
 
+/* Synchronous warm-up before PipeMare ("PipeMareW", Section 4: a number of epochs of the synchronous baseline with
+ * the standard learning rate, then PipeMare).  Call once, before the first tick; n_microbatches >= 0 (0 = none,
+ * the default).  The first n_microbatches microbatches then enter 2P ticks apart instead of one per tick, so
+ * that the pipeline holds one microbatch at a time: each of them runs forward and backward on the same weights
+ * and is applied before the next one enters, which is synchronous training with one microbatch per update.
+ * Their updates use the base step size as it is (no T1 division), their backward passes no T2 correction, and
+ * delta is left at zero.  For those microbatches pm_forward takes inputs at ticks 0, 2P, 4P, ... and NULL at the
+ * ticks between (PM_ERR_STATE otherwise); from tick 2P * n_microbatches on the pipeline runs as described below,
+ * with the T1 annealing counted from that point and the base step-size table and Adam's bias correction counted
+ * from the first microbatch.  PM_ERR_STATE if a tick has already run. */
+pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches);
+
 /* One tick = pm_forward, pm_backward, pm_update in this order (pm_step does all three).
  * inputs/targets (device) belong to the microbatch that enters the pipeline at this tick:
  * inputs is [T, n_in of stage 1] (float for PM_F32, bfloat16 for PM_BF16), or [T] int32 token ids when
@@ -186,7 +198,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
  * stream); targets is [T, n_out of stage P] float (PM_LOSS_MSE) or [T] int32 class ids
  * (PM_LOSS_CE).  Both are copied before the call returns control to the
  * stream order, so the caller may overwrite them after any later call on the same stream.
- * Pass NULL for both to drain: N microbatches need N + 2P - 1 ticks.
+ * Pass NULL for both to drain: N microbatches need N + 2P - 1 ticks (plus 2P - 1 ticks for each warm-up
+ * microbatch, see pm_set_warmup).
  *
  * Tick s (0-based): stage i (1-based) runs the forward of microbatch s-(i-1) and the
  * backward and update of microbatch s-(2P-i).  Hence its forward for microbatch a reads

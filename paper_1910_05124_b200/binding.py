@@ -76,6 +76,7 @@ def lib():
     L.pm_query_bytes.argtypes = [C.POINTER(pm_config), C.POINTER(pm_stage_desc), u64p, u64p, u64p]
     L.pm_init_stages.argtypes = [C.POINTER(vp), C.POINTER(pm_config), C.POINTER(pm_stage_desc), C.POINTER(pm_arenas),
                                  vp, C.c_uint64, vp, C.c_uint64, vp]
+    L.pm_set_warmup.argtypes = [vp, C.c_int64]
     L.pm_forward.argtypes = [vp, vp, vp]
     L.pm_backward.argtypes = [vp]
     L.pm_update.argtypes = [vp]
@@ -268,6 +269,9 @@ class Pipeline:
     # -- the C entry points, same names -------------------------------------------------------
     def _ptr(self, t):
         return None if t is None else C.c_void_p(t.data_ptr())
+
+    def pm_set_warmup(self, n_microbatches):
+        _check(self.L.pm_set_warmup(self.ctx, int(n_microbatches)), self.ctx)
 
     def pm_forward(self, inputs=None, targets=None):
         _check(self.L.pm_forward(self.ctx, self._ptr(inputs), self._ptr(targets)), self.ctx)

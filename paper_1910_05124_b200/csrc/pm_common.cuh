@@ -86,7 +86,17 @@ struct HyperDev {
   const double* alpha_tab;    // device, may be null
   int64_t alpha_len;
   float beta1, beta2, eps;
+  int64_t warm, period;       // synchronous warm-up (Section 4): the first `warm` microbatches enter `period` = 2P ticks apart
 };
+
+// The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks
+// (the pipeline holds one microbatch at a time, which is synchronous training), afterwards one per tick.
+__host__ __device__ inline int64_t mb_at_tick(int64_t a, int64_t warm, int64_t period) {
+  if (a < 0) return -1;
+  const int64_t t0 = warm * period;
+  if (a < t0) return (a % period == 0) ? a / period : -1;
+  return warm + (a - t0);
+}
 
 struct ArenasDev {
   float* w; float* m; float* s; float* delta; float* grad; __nv_bfloat16* w_lp;

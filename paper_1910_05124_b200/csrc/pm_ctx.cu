@@ -484,6 +484,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.alpha_tab = cfg->alpha_by_step ? (const double*)(c->ws + L.off_alpha) : nullptr;
   c->hp.alpha_len = cfg->alpha_len;
   c->hp.beta1 = cfg->beta1; c->hp.beta2 = cfg->beta2; c->hp.eps = cfg->eps;
+  c->hp.warm = 0; c->hp.period = 2 * (int64_t)cfg->n_stages;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -592,23 +593,42 @@ static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::functi
   return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, "graph launch");
 }
 
+// is a microbatch in flight at any of the stages whose distance from the entry tick lies in [lo, hi]?
+static bool any_stage_active(const pm_ctx* ctx, int64_t lo, int64_t hi) {
+  if (ctx->hp.warm == 0) return ctx->tick - lo >= 0 && ctx->tick - hi < ctx->n_fed;
+  for (int64_t off = lo; off <= hi; ++off) {
+    const int64_t m = mb_at_tick(ctx->tick - off, ctx->hp.warm, ctx->hp.period);
+    if (m >= 0 && m < ctx->n_fed) return true;
+  }
+  return false;
+}
+
+pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches) {
+  if (!ctx || n_microbatches < 0) return fail(ctx, PM_ERR_INVALID_ARG, "bad argument");
+  if (ctx->tick != 0 || ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "the warm-up length is set before the first tick");
+  ctx->hp.warm = n_microbatches;
+  return PM_OK;
+}
+
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "pm_forward called out of order (expected pm_backward or pm_update)");
   if ((inputs == nullptr) != (targets == nullptr)) return fail(ctx, PM_ERR_INVALID_ARG, "inputs and targets must both be given or both be NULL");
   if (inputs && ctx->draining) return fail(ctx, PM_ERR_STATE, "microbatches must be fed on consecutive ticks; the pipeline is already draining");
+  const int64_t mb = mb_at_tick(ctx->tick, ctx->hp.warm, ctx->hp.period);   // the microbatch that may enter now, or -1
+  if (inputs && mb < 0) return fail(ctx, PM_ERR_STATE, "during the synchronous warm-up a microbatch enters every 2 * n_stages ticks; this tick takes none");
   const int dt = ctx->cfg.compute_dtype;
   pm_status s;
-  if (inputs) ctx->n_fed = ctx->tick + 1; else ctx->draining = true;
+  if (inputs) ctx->n_fed = mb + 1; else if (mb >= 0) ctx->draining = true;   // an empty tick between two warm-up microbatches ends nothing
   s = TIMED(PM_PROF_SCHEDULE, check(ctx, launch_schedule((const StageSched*)(ctx->ws + ctx->L.off_sched), (const int64_t*)(ctx->ws + ctx->L.off_nupd),
                                  (StageDyn*)(ctx->ws + ctx->L.off_dyn), ctx->hp, ctx->tick, ctx->n_fed, -1, ctx->stream), "schedule"));
   if (s != PM_OK) return s;
   if (inputs) {
-    s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, ctx->tick, ctx->stream), "ingest"));
+    s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, mb, ctx->stream), "ingest"));
     if (s != PM_OK) return s;
   }
-  // forward of every stage whose microbatch exists: s - (i-1) in [0, n_fed)
-  if (ctx->tick - (ctx->cfg.n_stages - 1) < ctx->n_fed) {
+  // forward of every stage whose microbatch exists
+  if (any_stage_active(ctx, 0, ctx->cfg.n_stages - 1)) {
     s = run_phase(ctx, ctx->g_fwd, [&]() -> pm_status {
       pm_status s;
       if (ctx->L.any_pre && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ctx->ta, dt, ctx->ls), "embedding / LayerNorm forward"))) != PM_OK) return s;
@@ -635,8 +655,8 @@ pm_status pm_backward(pm_ctx* ctx) {
   const int dt = ctx->cfg.compute_dtype;
   const int P = ctx->cfg.n_stages;
   pm_status s;
-  // any backward this tick?  stage P runs microbatch tick-P, stage 1 runs tick-(2P-1)
-  const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
+  // any backward this tick?  stage P runs the microbatch that entered P ticks ago, stage 1 the one from 2P-1 ticks ago
+  const bool any = any_stage_active(ctx, P, 2 * P - 1);
   if (any) {
     s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
       pm_status s;
@@ -668,7 +688,7 @@ pm_status pm_update(pm_ctx* ctx) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 2) return fail(ctx, PM_ERR_STATE, "pm_update must follow pm_backward");
   const int P = ctx->cfg.n_stages;
-  const bool any = ctx->tick - P >= 0 && ctx->tick - (2 * (int64_t)P - 1) < ctx->n_fed;
+  const bool any = any_stage_active(ctx, P, 2 * P - 1);
   if (any) {
     pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
       prof_begin(ctx, PM_PROF_UPDATE);
@@ -722,8 +742,10 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
 pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t n) {
   if (!ctx || !host_out || first_mb < 0 || n < 0) return fail(ctx, PM_ERR_INVALID_ARG, "bad argument");
   const int P = ctx->cfg.n_stages;
-  // microbatch t's loss is computed in tick t+P; ticks completed so far = ctx->tick
-  const int64_t done = std::min<int64_t>(ctx->n_fed, ctx->tick - P);
+  // a microbatch's loss is computed P ticks after it entered; ticks completed so far = ctx->tick
+  const int64_t last = ctx->tick - P - 1, t0 = ctx->hp.warm * ctx->hp.period;   // latest entry tick whose loss exists
+  const int64_t entered = last < 0 ? 0 : (last < t0 ? last / ctx->hp.period + 1 : ctx->hp.warm + (last - t0) + 1);
+  const int64_t done = std::min<int64_t>(ctx->n_fed, entered);
   if (first_mb + n > done) return fail(ctx, PM_ERR_INVALID_ARG, "loss of a microbatch that has not finished was requested");
   if (done - first_mb > ctx->L.loss_cap) return fail(ctx, PM_ERR_INVALID_ARG, "requested losses have left the device log");
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
@@ -832,6 +854,7 @@ pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
   hp.alpha_const = cfg->alpha_by_step ? cfg->alpha_by_step[k < cfg->alpha_len ? k : cfg->alpha_len - 1] : cfg->alpha_const;
   hp.alpha_tab = nullptr; hp.alpha_len = 0;
   hp.beta1 = cfg->beta1; hp.beta2 = cfg->beta2; hp.eps = cfg->eps;
+  hp.warm = 0; hp.period = 1;
   e = launch_schedule((const StageSched*)(ws + off_sched), (const int64_t*)(ws + off_nupd), (StageDyn*)(ws + off_dyn), hp, 0, 0, k, st);
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "schedule");
   ArenasDev a{arenas->w, arenas->m, arenas->s, arenas->delta, arenas->grad, (__nv_bfloat16*)arenas->w_lp, arenas->count};

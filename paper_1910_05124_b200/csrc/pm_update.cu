@@ -19,8 +19,8 @@ namespace pm {
 
 // ---- scheduler -------------------------------------------------------------------------------
 //
-// Tick s, stage i (1-based): forward of microbatch a = s-(i-1); backward and update of
-// microbatch b = s-(2P-i).  T1 (Eq. 2): alpha_i = alpha_base(k) / tau_i^p, p = 1 - min(k/K, 1).
+// Tick s, stage i (1-based): forward of the microbatch that entered at tick s-(i-1); backward and update of
+// the one that entered at tick s-(2P-i) (microbatch = entry tick, except during a synchronous warm-up).  T1 (Eq. 2): alpha_i = alpha_base(k) / tau_i^p, p = 1 - min(k/K, 1).
 // T2: gamma_i = D^(1/(tau_fwd,i - tau_bkwd,i)).  Scalars are evaluated in double and rounded to
 // float once.
 __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int64_t* __restrict__ nupd,
@@ -37,8 +37,8 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
     d.f_mb = -1; d.b_mb = -1; d.k = flat_k;
     d.f_slot = d.f_xslot = d.f_next_xslot = d.b_slot = d.b_xslot = 0;
   } else {
-    int64_t a = tick - i;
-    int64_t b = tick - (2 * (int64_t)P - (i + 1));
+    int64_t a = mb_at_tick(tick - i, hp.warm, hp.period);
+    int64_t b = mb_at_tick(tick - (2 * (int64_t)P - (i + 1)), hp.warm, hp.period);
     bool fa = a >= 0 && a < n_fed;
     bool ba = b >= 0 && b < n_fed;
     d.f_mb = fa ? a : -1;
@@ -65,14 +65,17 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
     double base = hp.alpha_const;
     if (hp.alpha_tab != nullptr) base = hp.alpha_tab[k < hp.alpha_len ? k : hp.alpha_len - 1];
     double alpha = base;
-    if (hp.t1) {
-      double r = (double)k / (double)hp.K;
+    // warm-up microbatches (Section 4) are synchronous: standard step size, no correction, delta left alone; the T1
+    // annealing counts from the first PipeMare step
+    const bool sync = k < hp.warm;
+    if (hp.t1 && !sync) {
+      double r = (double)(k - hp.warm) / (double)hp.K;
       double p = 1.0 - (r < 1.0 ? r : 1.0);
       int tau = s.tau_f > 1 ? s.tau_f : 1;
       alpha = base / pow((double)tau, p);
     }
     d.alpha = (float)alpha;
-    if (hp.t2 && s.gap > 0) {
+    if (hp.t2 && s.gap > 0 && !sync) {
       d.gamma = (float)pow(hp.D, 1.0 / (double)s.gap);
       d.one_minus_gamma = 1.0f - d.gamma;
       d.use_delta = 1;

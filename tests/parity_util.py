@@ -4,10 +4,11 @@ import numpy as np
 import pm_inputs as I
 
 
-def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
+def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
+    The first `warmup` microbatches enter 2P ticks apart (synchronous warm-up), the rest one per tick.
     """
     import torch
     import paper_1910_05124_b200 as pm
@@ -18,18 +19,23 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True):
         teacher = I.teacher_params(wl) if teacher is None else teacher
     book = {}
     in_dtype = torch.bfloat16 if wl.compute == "bf16" else torch.float32
-    for s in range(n_steps + 2 * P - 1):
-        if s < n_steps:
+    warmup = min(warmup, n_steps)
+    if warmup:
+        pipe.pm_set_warmup(warmup)
+    t0 = 2 * P * warmup                                        # first tick of the one-per-tick phase
+    for s in range(t0 + (n_steps - warmup) + 2 * P - 1):
+        mb = (s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0)
+        if 0 <= mb < n_steps:
             if encoder and is_encdec(wl):
-                src, dec_in, tg = I.seq2seq_batch(wl, s)               # two token streams: [source | decoder input]
+                src, dec_in, tg = I.seq2seq_batch(wl, mb)              # two token streams: [source | decoder input]
                 xd = torch.from_numpy(np.concatenate([src, dec_in]).astype(np.int32)).to(pipe.device)
                 yd = torch.from_numpy(tg.astype(np.int32)).to(pipe.device)
             elif encoder:
-                ids, tg = I.token_batch(wl, s)
+                ids, tg = I.token_batch(wl, mb)
                 xd = torch.from_numpy(ids.astype(np.int32)).to(pipe.device)
                 yd = torch.from_numpy(tg.astype(np.int32)).to(pipe.device)
             else:
-                x, y = I.batch(wl, s, teacher)
+                x, y = I.batch(wl, mb, teacher)
                 xd = torch.from_numpy(x).to(pipe.device).to(in_dtype)
                 yd = torch.from_numpy(y).to(pipe.device)
             pipe.pm_step(xd, yd)
@@ -52,14 +58,14 @@ def is_encdec(wl):
     return any(sp.pre == "embed_dec" for sp in wl.stage_specs)
 
 
-def run_oracle(wl, params0, n_steps, teacher=None):
+def run_oracle(wl, params0, n_steps, teacher=None, warmup=0):
     if wl.kind == "encoder":
         from oracle import transformer
         data = (lambda t: I.seq2seq_batch(wl, t)) if is_encdec(wl) else (lambda t: I.token_batch(wl, t))
-        return transformer.run_workload(wl, params0, data, n_steps=n_steps)
+        return transformer.run_workload(wl, params0, data, n_steps=n_steps, warmup=warmup)
     from oracle.mlp import run_workload
     teacher = I.teacher_params(wl) if teacher is None else teacher
-    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps)
+    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps, warmup=warmup)
 
 
 def max_rel_err(a, b):
