@@ -433,6 +433,16 @@ __device__ __forceinline__ void ce_finish(const TickArgs& t, const StageDyn& d, 
   }
 }
 
+// fp32 activations take the exact exponential and a true division; with bf16 activations the gradient is rounded to 8
+// bits anyway, so the exponential is the hardware base-2 one (relative error ~2^-21 |x|) and the division a product
+// with the reciprocal of the row sum.  The loss itself uses the fp32 sum of these exponentials either way.
+template <typename AT> __device__ __forceinline__ float ce_exp(float x);
+template <> __device__ __forceinline__ float ce_exp<float>(float x) { return expf(x); }
+template <> __device__ __forceinline__ float ce_exp<__nv_bfloat16>(float x) { return __expf(x); }
+template <typename AT> __device__ __forceinline__ float ce_div(float e, float sum, float rsum);
+template <> __device__ __forceinline__ float ce_div<float>(float e, float sum, float) { return e / sum; }
+template <> __device__ __forceinline__ float ce_div<__nv_bfloat16>(float e, float, float rsum) { return e * rsum; }
+
 // ---- cross-entropy at the last stage -------------------------------------------------------------------------------
 // One block per token: lse = max + log(sum exp(logit - max)); loss_t = lse - logit[target];
 // dlogits = (softmax - onehot) / T in the activation type, written where the last stage reads its incoming
@@ -482,7 +492,7 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
     for (int k = 0; k < 4; ++k)
       if ((k * 256 + (int)threadIdx.x) * 8 < V) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { v[k][e] = expf(v[k][e] - mx); sum += v[k][e]; }
+        for (int e = 0; e < 8; ++e) { v[k][e] = ce_exp<AT>(v[k][e] - mx); sum += v[k][e]; }
       }
   } else if ((V & 3) == 0) {
     for (int c = threadIdx.x * 4; c < V; c += 4 * blockDim.x) {
@@ -499,7 +509,7 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   if (threadIdx.x == 0) { float a = 0.f; for (int i = 0; i < 8; ++i) a += red[i]; bc = a; }
   __syncthreads();
   sum = bc;
-  const float invT = 1.0f / (float)t.T;
+  const float invT = 1.0f / (float)t.T, rsum = 1.0f / sum;
   if (in_regs) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -508,7 +518,7 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
         float o[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          float pr = v[k][e] / sum;
+          float pr = ce_div<AT>(v[k][e], sum, rsum);
           if (c + e == tgt) pr -= 1.0f;
           o[e] = pr * invT;
         }
@@ -546,16 +556,6 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
   __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, e);
   *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
 }
-
-// fp32 activations take the exact exponential and a true division; with bf16 activations the gradient is rounded to 8
-// bits anyway, so the exponential is the hardware base-2 one (relative error ~2^-21 |x|) and the division a product
-// with the reciprocal of the row sum.  The loss itself uses the fp32 sum of these exponentials either way.
-template <typename AT> __device__ __forceinline__ float ce_exp(float x);
-template <> __device__ __forceinline__ float ce_exp<float>(float x) { return expf(x); }
-template <> __device__ __forceinline__ float ce_exp<__nv_bfloat16>(float x) { return __expf(x); }
-template <typename AT> __device__ __forceinline__ float ce_div(float e, float sum, float rsum);
-template <> __device__ __forceinline__ float ce_div<float>(float e, float sum, float) { return e / sum; }
-template <> __device__ __forceinline__ float ce_div<__nv_bfloat16>(float e, float, float rsum) { return e * rsum; }
 
 template <typename AT>
 __global__ void __launch_bounds__(kCeLongThreads) ce_loss_long_kernel(TickArgs t) {
