@@ -2,7 +2,8 @@
 // sequences of 128 tokens and heads of width 64 (bf16).  One CTA of 128 threads handles one (sequence, head):
 // thread r owns query row r = TMEM lane r, so the softmax needs no cross-thread traffic.
 //
-// forward :  S = Q K^T (128x128x64)  ->  p~ = exp(S/8 - rowmax), l = sum p~  ->  O = (bf16(p~) V) / l  (128x64x128)
+// forward :  S = Q K^T (128x128x64)  ->  p~ = exp(S/8 - rowmax), l = sum p~  ->  O = (bf16(p~) V) / l  (128x64x128);
+//            P overwrites Q and K, O the columns of S: 50 KB and 128 tensor-memory columns, four CTAs per SM
 // backward:  S = Q K^T, dP = dO V^T  ->  P = softmax, D = rowsum(dP*P), dS = bf16(P*(dP - D)), Pb = bf16(P)
 //            dV = Pb^T dO,  dQ = dS K / 8,  dK = dS^T Q / 8   (each 128x64x128)
 // Q, K, V, dO arrive by TMA as 128-byte-swizzled [128 rows x 64] tiles; the same tile serves as a K-major
@@ -20,7 +21,7 @@ namespace pm {
 
 constexpr int AT_S = 128, AT_DK = 64;
 constexpr int AT_TILE = AT_S * AT_DK * 2;          // 16 KB: one [128 x 64] bf16 tile
-constexpr int AT_FWD_SMEM = 3 * AT_TILE + 2 * AT_TILE + 1024 + 128;
+constexpr int AT_FWD_SMEM = 3 * AT_TILE + 1024 + 128;                       // Q|P0, K|P1, V: four CTAs per SM
 constexpr int AT_BWD_SMEM = 5 * AT_TILE + 1024 + 128 + 3 * 2 * AT_S * 4;   // Q, K, dO, V|P0|dS0, P1|dS1, row-statistics exchange: two CTAs per SM
 constexpr int AT_TMEM_COLS = 256;
 
@@ -102,7 +103,7 @@ __device__ __forceinline__ void attn_store32(__nv_bfloat16* dst, const uint32_t 
   }
 }
 
-__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int* status) {
+__global__ void __launch_bounds__(128, 4) attn_fwd_tc_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ stage_ids, int* status) {
   const int p = stage_ids[blockIdx.y];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
@@ -113,10 +114,10 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
   if ((int)blockIdx.x >= (t.T / AT_S) * H) return;
   const int b = blockIdx.x / H, h = blockIdx.x % H;
   extern __shared__ uint8_t smem_raw[];
-  const AttnCommon c = attn_setup(smem_raw, 5 * AT_TILE);
+  const AttnCommon c = attn_setup(smem_raw, 3 * AT_TILE, 128);
   const uint32_t tmem_base = *c.tmem_slot;
-  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sV = sK + AT_TILE, sP = sV + AT_TILE;
-  uint8_t* pP = c.sptr + 3 * AT_TILE;
+  const uint32_t sQ = c.sbase, sK = sQ + AT_TILE, sV = sK + AT_TILE, sP = sQ;   // P overwrites Q and K once S = Q K^T is done
+  uint8_t* pP = c.sptr;
   const CUtensorMap* lm = maps + (size_t)p * AMAPS_PER_STAGE;
   const int r = threadIdx.x;                                 // query row = TMEM lane
   const int warp = r >> 5;
@@ -169,14 +170,14 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
     if (r == 0) {
       tc_fence_after();
       const uint32_t idesc = make_idesc_mn(128, 64, 0, 1);   // O = P V : A = P K-major, B = V MN-major (k = key rows)
-      issue_k64(tmem_base + 128, sP, sV, idesc, true, false, 0, 8192, false);
-      issue_k64(tmem_base + 128, sP + AT_TILE, sV + 4 * 2048, idesc, true, false, 0, 8192, true);
+      issue_k64(tmem_base, sP, sV, idesc, true, false, 0, 8192, false);            // O takes the columns S has left
+      issue_k64(tmem_base, sP + AT_TILE, sV + 4 * 2048, idesc, true, false, 0, 8192, true);
       tc_commit(c.bar_mma);
     }
     if (wait_mma(c, 1, status, 13)) {
       uint32_t o0[32], o1[32];
-      tmem_ld32(lane_addr + 128, o0);
-      tmem_ld32(lane_addr + 160, o1);
+      tmem_ld32(lane_addr, o0);
+      tmem_ld32(lane_addr + 32, o1);
       tmem_ld_wait();
       const float inv = 1.0f / l;
       __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(t.ring + t.st[p + 1].x_ring) + (size_t)d.f_next_xslot * ((size_t)t.T * dm) +
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(TickArgs t, const CUte
       }
     }
   }
-  attn_teardown(c, tmem_base);
+  attn_teardown(c, tmem_base, 128);
 }
 
 // Backward: 256 threads, two per query row (thread r + 128*hf owns keys 64*hf .. 64*hf+63 of row r), two CTAs per SM.
