@@ -73,7 +73,8 @@ enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
  *              stage's output.  seq_len gives the position period.
  *   LAYERNORM  over the last dimension (n_in = n_out = width), eps 1e-5, biased variance; parameters gain, bias.
  *   ATTENTION  splits the Linear's output [T, 3d] into q, k, v; softmax(q k^T / sqrt(d / n_heads)) v per head and
- *              per sequence of seq_len rows (T a multiple of seq_len, seq_len <= 128); the stage hands o [T, d]
+ *              per sequence of seq_len rows (T a multiple of seq_len; seq_len <= 128, or seq_len = 256 with
+ *              PM_BF16 and heads of width 64, else PM_ERR_UNSUPPORTED); the stage hands o [T, d]
  *              and, as a skip tensor, the Linear's input to the next stage, which must end in RESIDUAL.
  *   SKIP_OUT   hands the Linear's input on as a skip tensor next to its output; next stage must end in RESIDUAL.
  *   RESIDUAL   adds the skip tensor it was sent to the Linear's output.
