@@ -151,10 +151,14 @@ def test_encoder_decoder_layout_and_its_checks(built_lib):
     st, msg = query(I.cfg5_small(compute="bf16", d_model=128, n_heads=4, seq_len=256, batch=1))[:2]
     assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
     assert query(I.cfg5_small(compute="bf16", d_model=128, n_heads=2, seq_len=256, batch=1))[0] == b"PM_OK"
-    # its 12 + 12 layers with 128-token sequences do not fit one GPU in the tick-major stash plan; the 4 + 4 layer cut does
+    # its 12 + 12 layers do not fit one GPU in the tick-major stash plan; the 6 + 6 layer cut does, 7 + 7 does not
     st, _, sb, rb, wb = query(I.cfg5_cut(12, 12))
     assert st == b"PM_OK" and rb > 500e9 and sb < 12e9
     st, _, sb, rb, wb = query(I.cfg5_cut())
+    assert st == b"PM_OK" and 135e9 < rb < 145e9 and sb + rb + wb < 160e9
+    st, _, sb, rb, wb = query(I.cfg5_cut(7, 7))
+    assert st == b"PM_OK" and sb + rb + wb > 200e9
+    st, _, sb, rb, wb = query(I.cfg5_cut(4, 4))
     assert st == b"PM_OK" and 60e9 < rb < 70e9 and sb + rb + wb < 90e9
     small = I.cfg5_small()
     assert query(small)[0] == b"PM_OK"
