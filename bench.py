@@ -141,10 +141,10 @@ WORKLOADS = {
             "T1 (K=32) + T2 (D=0.5), tau=(7,5,3,1)",
     "cfg3": "cfg3: 32-stage MLP, 2x Linear(1024,1024)+GELU per stage, bf16 GEMMs, fp32 master weights, microbatch 128, "
             "SGD momentum 0.9, T1 (K=125) + T2 (D=0.5), tau_i=2(32-i)+1",
-    "cfg5": "cfg5 cut to 6 + 6 layers: Transformer encoder-decoder, d_model 1024, 16 heads, FFN 4096, 16 sequences x 256 "
+    "cfg5": "cfg5 cut to 7 + 7 layers: Transformer encoder-decoder, d_model 1024, 16 heads, FFN 4096, 16 sequences x 256 "
             "tokens per microbatch, vocabulary 32000 (Zipf ids), bf16 GEMMs, fp32 master weights, one stage per weight GEMM "
-            "(67 stages), Adam(0.9, 0.98), T1 (K=1000) + T2 (D=0.1), tau_i=2(67-i)+1; 155 GB on the device; the full "
-            "12 + 12 layers (133 stages) need 553 GB of activation rings",
+            "(78 stages), Adam(0.9, 0.98), T1 (K=1000) + T2 (D=0.1), tau_i=2(78-i)+1; 166 GB on the device; the full "
+            "12 + 12 layers (133 stages) need more than 450 GB of activation rings",
     "cfg4": "cfg4: Transformer encoder, 6 layers, d_model 512, 8 heads, FFN 2048, 32 sequences x 128 tokens per "
             "microbatch, vocabulary 8192, bf16 GEMMs, fp32 master weights, one stage per weight GEMM (25 stages), "
             "Adam(0.9, 0.98), T1 (K=100) + T2 (D=0.1), tau_i=2(25-i)+1",
@@ -509,7 +509,7 @@ def run_cuda(args):
             if name != args.workload:
                 try:
                     others.append((name, measure(args, name, world, rank, local, device, None, with_e2e=False)))
-                except RuntimeError as exc:                  # e.g. cfg5's 155 GB on a device that has less free
+                except RuntimeError as exc:                  # e.g. cfg5's 166 GB on a device that has less free
                     import torch
                     torch.cuda.empty_cache()
                     others.append((name, {"error": str(exc).splitlines()[0][:200]}))
@@ -620,7 +620,7 @@ def run_reference(args):
         t0 = time.perf_counter()
         run_workload(wl1, p1, lambda t: b1, n_steps=1)
         per_flop = (time.perf_counter() - t0) / mm_flops(1, 1)
-        layers, seqs = 6, 16
+        layers, seqs = 7, 16
         while layers > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
             layers -= 1
         while seqs > 1 and total_steps * per_flop * mm_flops(layers, seqs) > budget_s:
@@ -628,9 +628,9 @@ def run_reference(args):
         wl = sub(layers, seqs)
         params0 = I.init_encoder_params(wl)
         batches = [I.seq2seq_batch(wl, t) for t in range(min(total_steps, 4))]
-        scale = mm_flops(layers, seqs) / mm_flops(6, 16)
+        scale = mm_flops(layers, seqs) / mm_flops(7, 16)
         samples_per_step = 16
-        sample = (f"each step: {seqs} of the 16 sequences through {layers} + {layers} of the 6 + 6 layers plus embedding and "
+        sample = (f"each step: {seqs} of the 16 sequences through {layers} + {layers} of the 7 + 7 layers plus embedding and "
                   f"vocabulary stages (forward, backward, update); samples/s scaled by the sampled fraction "
                   f"{scale:.5f} of the workload's matrix-product FLOPs")
     else:

@@ -9,7 +9,9 @@ namespace pm {
 
 enum { PRE_NONE = 0, PRE_EMBED = 1, PRE_LN = 2 };
 enum { POST_NONE = 0, POST_ATTENTION = 1, POST_SKIP_OUT = 2, POST_RESIDUAL = 3, POST_CROSS_ATTENTION = 4 };
-enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4 };
+// LF_ACT_FROM_Y: a ReLU whose pre-activation is not stashed: the backward takes the mask from the stashed output
+// (y > 0 exactly where z > 0), which the next Linear keeps for its weight gradient anyway
+enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4, LF_ACT_FROM_Y = 8 };
 
 // Static description of one Linear inside a stage (device copy).
 struct LinDev {
@@ -74,7 +76,7 @@ struct StageDyn {
   int32_t gmem_slot;          // slot of the memory-gradient ring of the microbatch in backward
   int32_t skip_wslot;         // emitting stage: slot of the receiving stage's skip buffer this tick's forward writes
   int32_t skip_rslot;         // receiving stage: slot of its skip buffer this tick's forward reads
-  int32_t _pad2;
+  int32_t b_next_xslot;       // slot of the NEXT stage's x ring that holds the output of the microbatch in backward
 };
 
 // Hyper-parameters the schedule kernel needs.

@@ -91,6 +91,9 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (sd.param_count < need) { stage_err(p, "param_count smaller than its ops need"); return PM_ERR_INVALID_ARG; }
     s.tau_f = sd.tau_fwd; s.gap = sd.tau_fwd - sd.tau_bkwd;
     s.depth = s.tau_f + 1; s.xdepth = s.tau_f + 2;
+    // the previous stage takes its ReLU mask from this stage's stashed input, one tick after this stage's own
+    // backward: one more slot keeps it until then
+    if (p > 0 && (L.st[p - 1].lin[L.st[p - 1].n_lin - 1].flags & LF_ACT_FROM_Y)) s.xdepth = s.tau_f + 3;
     s.begin = sd.param_offset; s.end = sd.param_offset + sd.param_count;
     prev_end = s.end;
     L.begin64[p] = (uint32_t)(s.begin / 64); L.end64[p] = (uint32_t)(s.end / 64);
@@ -198,7 +201,12 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       const bool logits = last && p == P - 1 && ce;
       ld.flags = 0;
       const bool to_attention = last && (s.post == POST_ATTENTION || s.post == POST_CROSS_ATTENTION);   // q, k, v stash
-      if (ld.act != PM_ACT_NONE || to_attention) ld.flags |= LF_WRITE_Z;
+      // a ReLU needs no stash of its own when its output is stashed anyway: between two Linears of a stage, or as
+      // the main input of the next stage (not when a RESIDUAL adds to it first or the next stage embeds tokens)
+      const bool next_takes_y = p + 1 < P && !(stages[p + 1].n_ops > 0 && stages[p + 1].ops[0].kind == PM_OP_EMBED) &&
+                                (s.post == POST_NONE || s.post == POST_SKIP_OUT);
+      if (ld.act == PM_ACT_RELU && (!last || next_takes_y)) ld.flags |= LF_ACT_FROM_Y;
+      if ((ld.act != PM_ACT_NONE && !(ld.flags & LF_ACT_FROM_Y)) || to_attention) ld.flags |= LF_WRITE_Z;
       if (!to_attention && !logits) ld.flags |= LF_WRITE_Y;
       if (logits) ld.flags |= LF_OUT_F32;
     }

@@ -188,7 +188,10 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
                  : (feeds_attention(s.post) ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
   const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy: nothing is stored
-  const AT* z = has_act ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n) : dy;
+  // the pre-activation stash, or for a ReLU without one the stashed output (same sign pattern)
+  const AT* z = !has_act ? dy
+                : !(L.flags & LF_ACT_FROM_Y) ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n)
+                : (lvl < s.n_lin - 1 ? ring_ptr<AT>(t, L.h_ring, d.b_slot, n) : ring_ptr<AT>(t, t.st[p + 1].x_ring, d.b_next_xslot, n));
   AT* dz = ws_ptr<AT>(t, s.dz);
   const bool vec = (L.n_out & 7) == 0;                      // vector path needs 8-element alignment of every row
   float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};

@@ -118,8 +118,13 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         *reinterpret_cast<float4*>(box + row_off + ((((uint32_t)(g & 3) * 2 + 1) ^ sw) << 4)) = make_float4(pf[4], pf[5], pf[6], pf[7]);
       } else {
         const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
-        if (!both)                                                  // no activation: z = y = bf16(acc + b), one output
+        if (!both) {                                                // one output: no activation (z = y = bf16(acc + b)), or a ReLU whose z is not kept
+          if (act == PM_ACT_RELU) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) pf[e] = fmaxf(pf[e], 0.0f);   // bf16(max(x, 0)) = max(bf16(x), 0)
+          }
           *reinterpret_cast<uint4*>(obuf + so + off) = make_uint4(pack_bf16(pf[0], pf[1]), pack_bf16(pf[2], pf[3]), pack_bf16(pf[4], pf[5]), pack_bf16(pf[6], pf[7]));
+        }
         else if (act == PM_ACT_NONE) epi_zy8<PM_ACT_NONE>(pf, obuf + off, obuf + 4096 + off);
         else if (act == PM_ACT_RELU) epi_zy8<PM_ACT_RELU>(pf, obuf + off, obuf + 4096 + off);
         else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);

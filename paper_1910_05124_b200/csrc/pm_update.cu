@@ -55,7 +55,7 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
   d.gmem_slot = (s.gmem_depth > 0 && d.b_mb >= 0) ? (int32_t)(d.b_mb % s.gmem_depth) : 0;
   d.skip_wslot = s.skip_dst_depth > 0 ? (int32_t)(tick % s.skip_dst_depth) : 0;
   d.skip_rslot = s.skip_depth > 0 ? (int32_t)((tick + 1) % s.skip_depth) : 0;
-  d._pad2 = 0;
+  d.b_next_xslot = (d.b_mb >= 0 && s.next_xdepth > 0) ? (int32_t)(d.b_mb % s.next_xdepth) : 0;
   d.f_ver = ver;
   d.b_ver = ver;
   d.active_update = d.k >= 0 ? 1 : 0;

@@ -283,11 +283,11 @@ def cfg5():
                            alpha=7e-4, beta1=0.9, beta2=0.98, eps=1e-8, K=1000, D=0.1, steps=1200, seed=191005124 + 5)
 
 
-def cfg5_cut(n_enc=6, n_dec=6, seq_len=256, batch=16, vocab=32000):
+def cfg5_cut(n_enc=7, n_dec=7, seq_len=256, batch=16, vocab=32000):
     """cfg5's widths and sequence shape (d_model 1024, 16 heads, FFN 4096, vocabulary 32000, 16 sequences of 256
-    tokens per microbatch) with fewer layers: 6 + 6 layers (67 stages, half the depth) is the deepest form whose
-    activation rings fit one GPU's memory (141 GB of rings, 155 GB in all; 7 + 7 layers need 207 GB, the full
-    12 + 12 layers 578 GB)."""
+    tokens per microbatch) with fewer layers: 7 + 7 layers (78 stages) is the deepest form whose activation rings
+    fit one GPU's memory (150 GB of rings, 166 GB in all; 8 + 8 layers need 212 GB, the full 12 + 12 layers
+    more than 450 GB)."""
     full = cfg5()
     return encdec_workload(f"cfg5_cut_{n_enc}+{n_dec}_bf16", n_enc, n_dec, 1024, 16, 4096, seq_len, batch, vocab, compute="bf16",
                            optimizer="adam", alpha=full.alpha, beta1=0.9, beta2=0.98, eps=1e-8, K=full.K, D=full.D,

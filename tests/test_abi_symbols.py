@@ -70,8 +70,9 @@ def test_query_bytes_and_state_copies_ratio(built_lib):
         baseline = 3 if opt == "sgdm" else 4            # w, g, v   |   w, g, m, s
         assert copies == baseline + 1
         assert copies / baseline == pytest.approx(ratio, rel=1e-12)
-        # ring: sum over stages of (tau+2) input slots + (tau+1) pre-activation slots, 32x256 fp32 each
-        slots = sum((t + 2) + (t + 1) for t in wl.tau_fwd)
+        # ring: (tau+2) input slots per stage; a ReLU's mask is read from the next stage's stashed input, which costs
+        # that stage one more slot instead of (tau+1) pre-activation slots; only the last stage keeps pre-activations
+        slots = sum(t + 2 for t in wl.tau_fwd) + (P - 1) + (wl.tau_fwd[-1] + 1)
         assert rb.value == slots * 32 * 256 * 4
 
 
@@ -142,7 +143,7 @@ def test_encoder_decoder_layout_and_its_checks(built_lib):
 
     # config 5 as given (133 stages, sequences of 256 tokens) is laid out, but its rings do not fit one GPU
     st, _, sb, rb, wb = query(I.cfg5())
-    assert st == b"PM_OK" and rb > 500e9
+    assert st == b"PM_OK" and rb > 400e9
     # beyond 128 tokens attention exists for 256 tokens, bf16 and heads of width 64 only
     st, msg = query(I.cfg5_small(compute="f32", d_model=128, n_heads=2, seq_len=256, batch=1))[:2]
     assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
@@ -151,15 +152,15 @@ def test_encoder_decoder_layout_and_its_checks(built_lib):
     st, msg = query(I.cfg5_small(compute="bf16", d_model=128, n_heads=4, seq_len=256, batch=1))[:2]
     assert st == b"PM_ERR_UNSUPPORTED" and b"beyond 128 tokens" in msg
     assert query(I.cfg5_small(compute="bf16", d_model=128, n_heads=2, seq_len=256, batch=1))[0] == b"PM_OK"
-    # its 12 + 12 layers do not fit one GPU in the tick-major stash plan; the 6 + 6 layer cut does, 7 + 7 does not
+    # its 12 + 12 layers do not fit one GPU in the tick-major stash plan; the 7 + 7 layer cut does, 8 + 8 does not
     st, _, sb, rb, wb = query(I.cfg5_cut(12, 12))
-    assert st == b"PM_OK" and rb > 500e9 and sb < 12e9
+    assert st == b"PM_OK" and rb > 400e9 and sb < 12e9
     st, _, sb, rb, wb = query(I.cfg5_cut())
-    assert st == b"PM_OK" and 135e9 < rb < 145e9 and sb + rb + wb < 160e9
-    st, _, sb, rb, wb = query(I.cfg5_cut(7, 7))
+    assert st == b"PM_OK" and 145e9 < rb < 155e9 and sb + rb + wb < 170e9
+    st, _, sb, rb, wb = query(I.cfg5_cut(8, 8))
     assert st == b"PM_OK" and sb + rb + wb > 200e9
     st, _, sb, rb, wb = query(I.cfg5_cut(4, 4))
-    assert st == b"PM_OK" and 60e9 < rb < 70e9 and sb + rb + wb < 90e9
+    assert st == b"PM_OK" and 45e9 < rb < 55e9 and sb + rb + wb < 70e9
     small = I.cfg5_small()
     assert query(small)[0] == b"PM_OK"
     dec0 = [i for i, s in enumerate(small.stage_specs) if s.pre == "embed_dec"][0]
