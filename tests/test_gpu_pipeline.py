@@ -95,6 +95,22 @@ def test_bf16_cta_pair_tiles(cuda_device, width, T):
     print("pair tiles worst relative weight error", worst)
 
 
+@pytest.mark.parametrize("compute,width,T,per_stage", [("f32", 72, 33, 3), ("bf16", 192, 40, 2), ("bf16", 320, 384, 2)])
+def test_relu_mask_from_stashed_output(cuda_device, compute, width, T, per_stage):
+    """ReLU Linears keep no pre-activation: inside a stage the mask comes from the stash between two Linears, at a
+    stage's end from the next stage's input ring (one slot deeper for that), and only the last stage stores z."""
+    wl = I.mlp_workload("relu_y", 4, width, per_stage, "relu", T, compute=compute, optimizer="sgdm", alpha=0.01, beta1=0.9,
+                        K=5, D=0.5, steps=22, seed=191005124 + 91)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps)
+    check_book(book, res, wl.steps, wl.n_stages)
+    f32 = compute == "f32"
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-5 if f32 else BF16_LOSS_TOL)
+    worst = compare_params(pipe, res, F32_TOL if f32 else BF16_W_TOL)
+    print("relu mask from output", compute, width, "worst relative weight error", worst)
+
+
 def test_phase_order_and_drain_rules(cuda_device):
     import torch
     import paper_1910_05124_b200 as pm
