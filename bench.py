@@ -347,7 +347,8 @@ def gemm_bytes(wl):
     fwd = wgrad = dgrad = 0.0
     for j, ((a, b, act), gap) in enumerate(zip(lin, gaps)):
         last = j == len(lin) - 1
-        out_b = 4 if (last and logits_f32) else 2 * (2 if act != "none" else 1)    # z stash and activation y
+        # z stash and activation y; a ReLU that is not the very last Linear stashes only y
+        out_b = 4 if (last and logits_f32) else 2 * (2 if (act == "gelu" or (act == "relu" and last)) else 1)
         fwd += 2.0 * T * a + 2.0 * a * b + out_b * T * b
         wgrad += 2.0 * T * a + 2.0 * T * b + 4.0 * a * b
         if j > 0 or wl.kind == "encoder":
@@ -361,9 +362,9 @@ NCU_TRAFFIC = {
     # GEMM kernels: measured DRAM bytes / algorithmic bytes on the 2-layer cut of cfg4
     # (profiles/gemm_and_attention_kernels_cfg4_2layer_cut.md); every operand crosses HBM once, so traffic grows
     # with the algorithmic bytes of the launch
-    "gemm_fwd_ratio": (84.3 + 182.8) / (83.9 + 243.0),
-    "wgrad_ratio": (211.4 + 23.2) / (205.5 + 42.0),
-    "dgrad_ratio": (234.6 + 30.2) / (226.5 + 33.6),
+    "gemm_fwd_ratio": (84.2 + 149.4) / (83.9 + 209.7),
+    "wgrad_ratio": (211.2 + 23.0) / (205.5 + 42.0),
+    "dgrad_ratio": (232.1 + 32.4) / (226.5 + 33.6),
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
