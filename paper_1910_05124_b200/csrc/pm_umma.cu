@@ -879,7 +879,7 @@ constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;
 constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
 constexpr int DP_ACC_COLS = DP_MG * DP_TILE_N;             // 256 columns per accumulator buffer
 constexpr int DP_XF_WARPS = 8, DP_EPI_WARPS = 8;
-constexpr int DP_THREADS = 32 * (2 + DP_XF_WARPS + DP_EPI_WARPS);
+constexpr int DP_THREADS = 32 * (3 + DP_XF_WARPS + DP_EPI_WARPS);   // staging producer, MMA issuer, transform, epilogue, dz producer
 constexpr int DP_TILE_BYTES = DP_NG * DP_STG_BYTES + DP_NB * DP_B_BYTES + DP_NA * A_BYTES + DP_EPI_WARPS * 4096;
 constexpr int DP_SMEM_BYTES = DP_TILE_BYTES + 1024 + 512;
 
@@ -945,58 +945,73 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ---------------- TMA producer (both CTAs): the fp32 staging loads run one k-block ahead of the dz loads ----------------
-    if (lane == 0) {
-      struct Cursor { int tile, kb; DgTile tl; bool done; };
-      auto seek = [&](Cursor& c) {
-        for (; c.tile < n_slots; c.tile += n_pairs) {
-          const int tile = order[c.tile];
-          if (tile < 0) continue;
-          c.tl = decode_dgrad_pair(t, tile_start, lvl, tile);
-          if (c.tl.valid) { c.kb = 0; c.done = false; return; }
-        }
-        c.done = true;
-      };
-      auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += n_pairs; seek(c); } };
-      Cursor cs{pair, 0, DgTile{}, false}, ca{pair, 0, DgTile{}, false};
-      seek(cs); seek(ca);
-      Ring sg{0, 0}, ar{0, 0};
-      int issued_sg = 0, issued_a = 0;
-      bool ok = true;
-      auto issue_staging = [&](const Cursor& c) {
+  // Two producer threads, each with its own cursor over the same (tile, k-block) sequence: warp 0 feeds the fp32
+  // staging ring (w, delta), the last warp the dz ring.  Their k-block loops are the critical path of the kernel
+  // (a handful of extra loads in them cost 3 %), so everything that is fixed for a tile is read once when the
+  // cursor reaches the tile and the loops hold nothing but barrier waits and copies.
+  struct Cursor { int tile, kb; DgTile tl; bool done; const CUtensorMap* lm; bool corr; int dz_slot; };
+  auto seek = [&](Cursor& c) {
+    for (; c.tile < n_slots; c.tile += n_pairs) {
+      const int tile = order[c.tile];
+      if (tile < 0) continue;
+      c.tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+      if (c.tl.valid) {
         const StageDyn& d = t.dyn[c.tl.p];
-        const CUtensorMap* lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) { ok = false; return; }
-        const uint32_t sw = stg + sg.idx * DP_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
-        const bool corr = d.use_delta != 0;
-        mbar_arrive_expect_tx(fb, corr ? DP_STG_BYTES : DP_STG_HALF);
-        tma_load_2d(sw, lm + MAP_W_F32H, fb, c.tl.n0 + rank * DP_HALF_N, c.kb * TILE_K);
-        if (corr) tma_load_2d(sw + DP_STG_HALF, lm + MAP_D_F32H, fb, c.tl.n0 + rank * DP_HALF_N, c.kb * TILE_K);
-        sg.advance(DP_NG); ++issued_sg;
-      };
-      if (!cs.done) { issue_staging(cs); step(cs); }
-      while (!ca.done && ok) {
-        if (!cs.done) { issue_staging(cs); step(cs); if (!ok) break; }
-        const StageDyn& d = t.dyn[ca.tl.p];
-        const StageDev& sd_ = t.st[ca.tl.p];
-        const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
-        for (int mi = 0; mi < ca.tl.n_m; ++mi) {
-          if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 42)) { ok = false; break; }
-          if (rank == 0) mbar_arrive_expect_tx(bar_afull + 8 * ar.idx, 2 * A_BYTES);       // the rows of both CTAs
-          tma_load_3d_pair(sA + ar.idx * A_BYTES, lm + MAP_DZ_K, mapa_shared(bar_afull + 8 * ar.idx, 0),
-                           ca.kb * TILE_K, ca.tl.m0 + mi * DP_TILE_M + rank * TILE_M, dz_slot);
-          ar.advance(DP_NA); ++issued_a;
-        }
-        step(ca);
+        const StageDev& sd_ = t.st[c.tl.p];
+        c.lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        c.corr = d.use_delta != 0;
+        c.dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        c.kb = 0; c.done = false;
+        return;
       }
-      if (*abort_flag) {
+    }
+    c.done = true;
+  };
+  auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += n_pairs; seek(c); } };
+
+  if (warp == 0) {
+    // ---------------- TMA producer of the fp32 staging ring (both CTAs) ----------------
+    if (lane == 0) {
+      Cursor cs{pair, 0, DgTile{}, false, nullptr, false, 0};
+      seek(cs);
+      Ring sg{0, 0};
+      int issued_sg = 0;
+      while (!cs.done) {
+        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) break;
+        const uint32_t sw = stg + sg.idx * DP_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+        mbar_arrive_expect_tx(fb, cs.corr ? DP_STG_BYTES : DP_STG_HALF);
+        tma_load_2d(sw, cs.lm + MAP_W_F32H, fb, cs.tl.n0 + rank * DP_HALF_N, cs.kb * TILE_K);
+        if (cs.corr) tma_load_2d(sw + DP_STG_HALF, cs.lm + MAP_D_F32H, fb, cs.tl.n0 + rank * DP_HALF_N, cs.kb * TILE_K);
+        sg.advance(DP_NG); ++issued_sg;
+        step(cs);
+      }
+      if (*abort_flag) {                                              // copies already issued still land here: wait (bounded)
         for (int back = 1; back <= DP_NG && back <= issued_sg; ++back) {
           const int it = issued_sg - back;
           const long long t0 = clock64();
           while (!mbar_try_wait(bar_sfull + 8 * (it % DP_NG), (uint32_t)(it / DP_NG) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
+      }
+    }
+  } else if (warp == 2 + DP_XF_WARPS + DP_EPI_WARPS) {
+    // ---------------- TMA producer of the dz ring (both CTAs) ----------------
+    if (lane == 0) {
+      Cursor ca{pair, 0, DgTile{}, false, nullptr, false, 0};
+      seek(ca);
+      Ring ar{0, 0};
+      int issued_a = 0;
+      bool ok = true;
+      while (!ca.done && ok) {
+        for (int mi = 0; mi < ca.tl.n_m; ++mi) {
+          if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 42)) { ok = false; break; }
+          if (rank == 0) mbar_arrive_expect_tx(bar_afull + 8 * ar.idx, 2 * A_BYTES);       // the rows of both CTAs
+          tma_load_3d_pair(sA + ar.idx * A_BYTES, ca.lm + MAP_DZ_K, mapa_shared(bar_afull + 8 * ar.idx, 0),
+                           ca.kb * TILE_K, ca.tl.m0 + mi * DP_TILE_M + rank * TILE_M, ca.dz_slot);
+          ar.advance(DP_NA); ++issued_a;
+        }
+        step(ca);
+      }
+      if (*abort_flag) {
         if (rank == 0) {
           for (int back = 1; back <= DP_NA && back <= issued_a; ++back) {
             const int it = issued_a - back;
