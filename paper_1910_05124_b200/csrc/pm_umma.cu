@@ -459,17 +459,21 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         const int ma = tl.m0 + rank * TILE_M, nbh = tl.n0 + rank * TILE_N;   // this CTA's rows of A and of B
-        for (int kb = 0; kb < tl.n_kb; ++kb) {
+        // ring slots of the operands: read here, once per tile (the k-block loop is the critical path of the kernel and
+        // every wait in it makes the compiler re-read what lives in memory)
+        const int aslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.f_xslot : d.f_slot;
+        const int xslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.b_xslot : d.b_slot;
+        const int n_kb = tl.n_kb;
+        for (int kb = 0; kb < n_kb; ++kb) {
           const int k0 = kb * TILE_K;
           if (!mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 31)) { ok = false; break; }
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
           if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * op.idx, 2 * (A_BYTES + B_BYTES));   // the bytes of both CTAs
           const uint32_t fb = mapa_shared(bar_full + 8 * op.idx, 0);
           if (MODE == 0) {
-            tma_load_3d_pair(sa, lm + MAP_ACT_K, fb, k0, ma, (lvl == 0 && sd_.pre == PRE_NONE) ? d.f_xslot : d.f_slot);
+            tma_load_3d_pair(sa, lm + MAP_ACT_K, fb, k0, ma, aslot);
             tma_load_2d_pair(sb, lm + MAP_W_K, fb, k0, nbh);
           } else {
-            const int xslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.b_xslot : d.b_slot;
             tma_load_3d_pair(sa, lm + MAP_DZ_MN, fb, ma, k0, dz_slot);
             tma_load_3d_pair(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, ma + 64, k0, dz_slot);
             tma_load_3d_pair(sb, lm + MAP_ACT_MN, fb, nbh, k0, xslot);
