@@ -176,8 +176,7 @@ struct Tile { int p, m0, n0, M, N, K, n_kb; bool valid; };
 template <int MODE>
 __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   Tile r;
-  int lo = 0, hi = t.P - 1;                                            // largest p with tile_start[p] <= tile
-  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -388,8 +387,7 @@ constexpr int P2_SMEM_BYTES = P2_TILE_BYTES + 1024 + 512;
 template <int MODE>
 __device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   Tile r;
-  int lo = 0, hi = t.P - 1;
-  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -599,8 +597,7 @@ struct DgTile { int p, m0, n0, n_m, M, N, K, n_kb; bool valid; };
 
 __device__ __forceinline__ DgTile decode_dgrad(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
-  int lo = 0, hi = t.P - 1;
-  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -877,7 +874,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
 // CTAs; the epilogue warps of both arrive on the leader's tempty.
 constexpr int DP_TILE_M = 256, DP_TILE_N = 128, DP_HALF_N = 64;
 constexpr int DP_MG = 2;                                   // 256-row tiles per converted tile
-constexpr int DP_NG = 3, DP_NB = 3, DP_NA = 4;             // fp32 staging ring, converted ring, dz ring
+constexpr int DP_NG = 2, DP_NB = 2, DP_NA = 7;             // fp32 staging ring, converted ring, dz ring (3.5 k-blocks of dz in flight)
 constexpr int DP_STG_HALF = TILE_K * DP_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
 constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;
 constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
@@ -889,8 +886,7 @@ constexpr int DP_SMEM_BYTES = DP_TILE_BYTES + 1024 + 512;
 
 __device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
-  int lo = 0, hi = t.P - 1;
-  while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tile_start[mid] <= tile) lo = mid; else hi = mid - 1; }
+  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -1186,7 +1182,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct UmmaPlan {
   const CUtensorMap* d_maps = nullptr;
-  const int* d_tile_start = nullptr;     // [3 modes][PM_MAX_LINEARS][P+1]
+  const int* d_tile_start = nullptr;     // per (mode, level) at ts_off: [P+1] starts, then the stage of each tile
+  size_t ts_off[3][PM_MAX_LINEARS] = {};
   const int* d_orders = nullptr;         // concatenated order arrays
   int* d_status = nullptr;
   int n_slots[3][PM_MAX_LINEARS] = {};
@@ -1201,7 +1198,8 @@ struct UmmaPlan {
 // assignment (weight = k-blocks x row tiles + a constant per tile), so that one very deep GEMM (a vocabulary
 // projection next to d_model-sized layers) does not leave most SMs idle.  Unused slots hold -1.
 struct TileTables {
-  std::vector<int> tile_start;           // [3][PM_MAX_LINEARS][P+1]
+  std::vector<int> tile_start;           // per (mode, level): [P+1] starts, then the stage of each tile
+  size_t ts_off[3][PM_MAX_LINEARS] = {};
   std::vector<int> orders;
   int n_slots[3][PM_MAX_LINEARS] = {};
   int grid[3][PM_MAX_LINEARS] = {};
@@ -1228,11 +1226,13 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
   const int P = (int)st.size();
   const bool allow_pair = pair_kernels_allowed();
   TileTables tt;
-  tt.tile_start.assign((size_t)3 * PM_MAX_LINEARS * (P + 1), 0);
   auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
   for (int mode = 0; mode < 3; ++mode)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
-      int* ts = tt.tile_start.data() + ((size_t)mode * PM_MAX_LINEARS + l) * (P + 1);
+      // block of this (mode, level): P + 1 tile starts, then the stage of every tile (one load instead of a search)
+      tt.ts_off[mode][l] = tt.tile_start.size();
+      std::vector<int> ts_block((size_t)P + 1, 0);
+      int* ts = ts_block.data();
       std::vector<std::pair<long long, int>> work;          // (weight, tile id)
       // forward and wgrad launches whose GEMMs all have at least 256 rows and columns run on CTA pairs
       bool pair = allow_pair && sms >= 2;
@@ -1264,6 +1264,8 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
         }
       }
       ts[P] = acc;
+      tt.tile_start.insert(tt.tile_start.end(), ts_block.begin(), ts_block.end());
+      for (int p = 0; p < P; ++p) tt.tile_start.insert(tt.tile_start.end(), (size_t)(ts_block[p + 1] - ts_block[p]), p);
       const int G = std::max(1, std::min(acc, pair ? sms / 2 : sms));     // persistent CTAs, or CTA pairs
       tt.grid[mode][l] = pair ? 2 * G : G;
       tt.order_off[mode][l] = tt.orders.size();
@@ -1398,6 +1400,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       plan->grid[mode][l] = tt.grid[mode][l];
       plan->pair[mode][l] = tt.pair[mode][l];
       plan->order_off[mode][l] = tt.order_off[mode][l];
+      plan->ts_off[mode][l] = tt.ts_off[mode][l];
     }
   char* region = (char*)ws_region;
   cudaError_t e = cudaMemcpyAsync(region + 256, maps.data(), maps_bytes(P), cudaMemcpyHostToDevice, stream);
@@ -1431,7 +1434,7 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   const int n_slots = plan->n_slots[mode][lvl];
   if (n_slots == 0) return cudaSuccess;
   const int grid = plan->grid[mode][lvl];                             // one persistent CTA per SM
-  const int* ts = plan->d_tile_start + ((size_t)mode * PM_MAX_LINEARS + lvl) * (plan->P + 1);
+  const int* ts = plan->d_tile_start + plan->ts_off[mode][lvl];
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
   if (plan->pair[mode][lvl]) {
     if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
