@@ -362,9 +362,9 @@ NCU_TRAFFIC = {
     # GEMM kernels: measured DRAM bytes / algorithmic bytes on the 2-layer cut of cfg4
     # (profiles/gemm_and_attention_kernels_cfg4_2layer_cut.md); every operand crosses HBM once, so traffic grows
     # with the algorithmic bytes of the launch
-    "gemm_fwd_ratio": (84.2 + 149.4) / (83.9 + 209.7),
-    "wgrad_ratio": (211.2 + 23.0) / (205.5 + 42.0),
-    "dgrad_ratio": (232.1 + 32.4) / (226.5 + 33.6),
+    "gemm_fwd_ratio": (84.2 + 149.1) / (83.9 + 209.7),
+    "wgrad_ratio": (211.1 + 24.9) / (205.5 + 42.0),
+    "dgrad_ratio": (231.8 + 29.2) / (226.5 + 33.6),
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
