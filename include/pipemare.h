@@ -20,6 +20,17 @@
  *     error pm_last_error(ctx) gives a readable message.
  *   - Stages are numbered 1..P in the paper and 0..P-1 in array arguments here.
  *   - One microbatch per update (N = 1 in the notation of Section 2.1).
+ *
+ * Two loop orders compute the same recurrence (pm_config.loop_order):
+ *   PM_TICK_MAJOR  the pipeline as it would run on P devices: every call of pm_step is one tick in which all
+ *                  stages work side by side on different microbatches; each stage holds ONE version of its
+ *                  weights and a ring of the activations of its microbatches in flight (depth tau_fwd + 1, so
+ *                  the rings grow with P^2: Appendix A.1).
+ *   PM_MB_MAJOR    the form in which Section 2.1 states the method: every call of pm_step takes one microbatch
+ *                  through all stages forward, then backward, then applies the update; each stage keeps a queue
+ *                  of its last tau_fwd + 1 weight versions (the forward operands) and activations of one
+ *                  microbatch only.  Memory grows with sum_i tau_fwd,i * |w_i| instead of P^2 activations, any
+ *                  tau_fwd,i >= 0 is accepted (all zero = synchronous training), and no drain ticks exist.
  */
 #ifndef PIPEMARE_H
 #define PIPEMARE_H
@@ -57,6 +68,7 @@ enum { PM_OPF_CAUSAL = 1,          /* ATTENTION: keys after the query position a
                                       stage must start with EMBED | PM_OPF_SECOND_STREAM                          */
        PM_OPF_SKIP_TWO = 16 };     /* SKIP_OUT: the skip tensor goes to the stage two positions on                */
 enum { PM_LOSS_MSE = 0, PM_LOSS_CE = 1 };
+enum { PM_TICK_MAJOR = 0, PM_MB_MAJOR = 1 };      /* pm_config.loop_order */
 
 /* Alignment, in elements, of every stage slice and of every tensor inside it. */
 #define PM_ALIGN_ELEMS 64
@@ -98,7 +110,8 @@ typedef struct {
  * tau_fwd / tau_bkwd: number of updates between the forward / backward read of this
  * stage's weights and the update that uses the resulting gradient.  PipeMare
  * (Table 1) has tau_fwd = 2(P-i)+1 and tau_bkwd = 0, which is the only delay
- * pattern the tick schedule realises; other values are PM_ERR_UNSUPPORTED.
+ * pattern the tick schedule (PM_TICK_MAJOR) realises; PM_MB_MAJOR takes any
+ * tau_fwd >= 0 with tau_bkwd = 0; other values are PM_ERR_UNSUPPORTED.
  * param_offset / param_count: this stage's slice of the flat arenas, in elements;
  * both multiples of PM_ALIGN_ELEMS.  Inside the slice each op's W and then b start
  * at the next multiple of PM_ALIGN_ELEMS (pm_op_param_offsets gives the numbers). */
@@ -135,6 +148,7 @@ typedef struct {
   const double* alpha_by_step;   /* host, may be NULL */
   int64_t alpha_len;
   int64_t loss_log_capacity;     /* losses kept on the device (a ring); 0 = default 4096 */
+  int32_t loop_order;            /* PM_TICK_MAJOR | PM_MB_MAJOR (see the top of this file) */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /
@@ -165,8 +179,10 @@ pm_status pm_op_param_offsets(const pm_op_desc* ops, int32_t n_ops, int32_t op,
 
 /* Bytes the caller must provide: state_bytes = all arenas together (fp32 w, m, [s,] delta,
  * grad [+ bf16 copy]); ring_bytes = the per-stage delay rings of in-flight activations
- * (Section 2 / Appendix A: depth grows with 2(P-i)+1); workspace_bytes = gradient
- * mailboxes, per-stage scratch, target ring, loss log and tables. */
+ * (Section 2 / Appendix A: depth grows with 2(P-i)+1) or, for PM_MB_MAJOR, the activations of one
+ * microbatch plus the per-stage queues of weight versions ((tau_fwd,i + 1) copies of the stage's
+ * parameters in the GEMM operand type, and of its biases and LayerNorm parameters in fp32);
+ * workspace_bytes = gradient mailboxes, per-stage scratch, target ring, loss log and tables. */
 pm_status pm_query_bytes(const pm_config* cfg, const pm_stage_desc* stages,
                          uint64_t* state_bytes, uint64_t* ring_bytes, uint64_t* workspace_bytes);
 
@@ -189,7 +205,9 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
  * delta is left at zero.  For those microbatches pm_forward takes inputs at ticks 0, 2P, 4P, ... and NULL at the
  * ticks between (PM_ERR_STATE otherwise); from tick 2P * n_microbatches on the pipeline runs as described below,
  * with the T1 annealing counted from that point and the base step-size table and Adam's bias correction counted
- * from the first microbatch.  PM_ERR_STATE if a tick has already run. */
+ * from the first microbatch.  PM_ERR_STATE if a tick has already run.
+ * PM_MB_MAJOR: the first n_microbatches calls of pm_step read the live weights in the forward pass too (the same
+ * synchronous steps, without idle ticks); everything else as above. */
 pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches);
 
 /* One tick = pm_forward, pm_backward, pm_update in this order (pm_step does all three).
@@ -205,7 +223,15 @@ pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches);
  * Tick s (0-based): stage i (1-based) runs the forward of microbatch s-(i-1) and the
  * backward and update of microbatch s-(2P-i).  Hence its forward for microbatch a reads
  * weight version max(0, a - tau_fwd,i) and its backward reads version a (Section 2.1 with
- * PipeMare's delays). */
+ * PipeMare's delays).
+ *
+ * PM_MB_MAJOR: one call of pm_step (or pm_forward, pm_backward, pm_update in this order) processes microbatch t
+ * completely: pm_forward takes it through stages 1..P, stage i reading weight version max(0, t - tau_fwd,i) from
+ * its queue; pm_backward computes the loss and walks stages P..1 against the live weights (version t, T2-corrected)
+ * and forms every weight gradient; pm_update applies update t to all stages and pushes version t + 1 into the
+ * queues.  inputs and targets must be given at every call (there is nothing to drain: NULL is PM_ERR_INVALID_ARG);
+ * after N calls every stage has applied N updates.  In this order the w_lp arena is read once, at
+ * initialisation (version 0); the live bf16 copy is the newest slot of the queue. */
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets);
 pm_status pm_backward(pm_ctx* ctx);
 pm_status pm_update(pm_ctx* ctx);
@@ -214,7 +240,9 @@ pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets);
 /* Per-stage record of the last completed tick, written by the device kernels, for the
  * delay-bookkeeping check.  out[0..7] = forward microbatch (-1 if idle), weight version
  * the forward read, backward microbatch (-1 if idle), weight version the backward read,
- * updates applied so far, forward ring slot, backward ring slot, tick.  Synchronises. */
+ * updates applied so far, forward ring slot, backward ring slot, tick.  Synchronises.
+ * PM_MB_MAJOR: the record of the last completed microbatch (both passes of every stage are active); out[7] is
+ * that microbatch's index, out[5] the slot of the weight-version queue the forward read. */
 pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8);
 
 /* Copy losses of microbatches first_mb .. first_mb+n-1 to host_out.  The loss of microbatch

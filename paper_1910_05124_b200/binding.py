@@ -17,6 +17,7 @@ PM_OP_LINEAR, PM_OP_EMBED, PM_OP_LAYERNORM, PM_OP_ATTENTION, PM_OP_SKIP_OUT, PM_
 PM_OP_CROSS_ATTENTION = 6
 PM_OPF_CAUSAL, PM_OPF_FROM_MEMORY, PM_OPF_SECOND_STREAM, PM_OPF_EMIT_MEMORY, PM_OPF_SKIP_TWO = 1, 2, 4, 8, 16
 PM_LOSS_MSE, PM_LOSS_CE = 0, 1
+PM_TICK_MAJOR, PM_MB_MAJOR = 0, 1
 PM_ALIGN_ELEMS = 64
 
 _ACT = {"none": PM_ACT_NONE, "relu": PM_ACT_RELU, "gelu": PM_ACT_GELU}
@@ -40,7 +41,7 @@ class pm_config(C.Structure):
                 ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("t1_enable", C.c_int32), ("t1_K", C.c_int64), ("t2_enable", C.c_int32), ("t2_D", C.c_double),
                 ("alpha_const", C.c_double), ("alpha_by_step", C.POINTER(C.c_double)), ("alpha_len", C.c_int64),
-                ("loss_log_capacity", C.c_int64)]
+                ("loss_log_capacity", C.c_int64), ("loop_order", C.c_int32)]
 
 
 class pm_arenas(C.Structure):
@@ -108,7 +109,8 @@ def _check(status, ctx=None):
 
 
 def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, beta2=0.98, eps=1e-8,
-                t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0, loss=PM_LOSS_MSE):
+                t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0, loss=PM_LOSS_MSE,
+                loop_order=PM_TICK_MAJOR):
     cfg = pm_config()
     cfg.n_stages, cfg.microbatch = n_stages, microbatch
     cfg.compute_dtype = PM_BF16 if compute in ("bf16", PM_BF16) and compute != 0 else PM_F32
@@ -124,6 +126,7 @@ def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, b
         cfg.alpha_by_step = C.cast(keep, C.POINTER(C.c_double))
         cfg.alpha_len = len(alpha_by_step)
     cfg.loss_log_capacity = loss_log_capacity
+    cfg.loop_order = PM_MB_MAJOR if loop_order in ("mb_major", PM_MB_MAJOR) and loop_order != 0 else PM_TICK_MAJOR
     return cfg, keep
 
 
@@ -203,7 +206,7 @@ class Pipeline:
     params0: per stage a list of (W[out,in], b[out]) float32 numpy arrays.
     """
 
-    def __init__(self, wl, params0, device="cuda:0", stream=None, loss_log_capacity=0):
+    def __init__(self, wl, params0, device="cuda:0", stream=None, loss_log_capacity=0, loop_order=PM_TICK_MAJOR):
         import torch
         self.torch = torch
         self.wl = wl
@@ -232,7 +235,9 @@ class Pipeline:
         self.cfg, self._alpha_keep = make_config(
             n_stages=P, microbatch=wl.microbatch, compute=wl.compute, optimizer=wl.optimizer, alpha=wl.alpha,
             beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D,
-            loss_log_capacity=loss_log_capacity, loss=PM_LOSS_CE if self.is_encoder else PM_LOSS_MSE)
+            loss_log_capacity=loss_log_capacity, loss=PM_LOSS_CE if self.is_encoder else PM_LOSS_MSE,
+            loop_order=loop_order)
+        self.mb_major = self.cfg.loop_order == PM_MB_MAJOR
         sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
         _check(self.L.pm_query_bytes(C.byref(self.cfg), self.stage_desc, C.byref(sb), C.byref(rb), C.byref(wb)))
         self.state_bytes, self.ring_bytes, self.workspace_bytes = sb.value, rb.value, wb.value

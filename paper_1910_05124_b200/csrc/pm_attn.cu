@@ -654,6 +654,7 @@ struct AttnPlan {
   const int* d_stage_ids = nullptr;      // the stages that end in attention, in pipeline order
   int n_att = 0;
   int* d_status = nullptr;
+  std::vector<int> h_ids;                // host copy of the stage list
 };
 
 static uint64_t attn_maps_bytes(int n_stages) { return (uint64_t)n_stages * AMAPS_PER_STAGE * sizeof(CUtensorMap); }
@@ -706,6 +707,7 @@ pm_status attn_plan_create(AttnPlan** out, const TickArgs& t, const std::vector<
   plan->d_maps = (const CUtensorMap*)(region + 256);
   plan->d_stage_ids = (const int*)(region + 256 + attn_maps_bytes(t.P));
   plan->n_att = (int)ids.size();
+  plan->h_ids = ids;
   *out = plan;
   return PM_OK;
 }
@@ -715,14 +717,22 @@ int* attn_status_word(AttnPlan* plan) { return plan ? plan->d_status : nullptr; 
 
 cudaError_t attn_tc_launch(AttnPlan* plan, const TickArgs& t, bool forward, cudaStream_t stream) {
   if (plan->n_att == 0) return cudaSuccess;
-  dim3 grid(t.att_blocks, plan->n_att);               // att_blocks = (sequence, head) pairs
+  int n_att = plan->n_att;
+  const int* ids = plan->d_stage_ids;
+  if (t.sel_p >= 0) {                                 // one stage only: its entry of the stage list
+    int idx = -1;
+    for (int i = 0; i < plan->n_att; ++i) if (plan->h_ids[(size_t)i] == t.sel_p) idx = i;
+    if (idx < 0) return cudaSuccess;
+    ids += idx; n_att = 1;
+  }
+  dim3 grid(t.att_blocks, n_att);                     // att_blocks = (sequence, head) pairs
   if (t.att_S == AT2_S) {
-    if (forward) attn_fwd_tc256_kernel<<<dim3(2 * t.att_blocks, plan->n_att), 256, AT2_FWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
-    else attn_bwd_tc256_kernel<<<grid, AT2_BWD_THREADS, AT2_BWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
+    if (forward) attn_fwd_tc256_kernel<<<dim3(2 * t.att_blocks, n_att), 256, AT2_FWD_SMEM, stream>>>(t, plan->d_maps, ids, plan->d_status);
+    else attn_bwd_tc256_kernel<<<grid, AT2_BWD_THREADS, AT2_BWD_SMEM, stream>>>(t, plan->d_maps, ids, plan->d_status);
     return cudaGetLastError();
   }
-  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
-  else attn_bwd_tc_kernel<<<grid, AT_BWD_THREADS, AT_BWD_SMEM, stream>>>(t, plan->d_maps, plan->d_stage_ids, plan->d_status);
+  if (forward) attn_fwd_tc_kernel<<<grid, 128, AT_FWD_SMEM, stream>>>(t, plan->d_maps, ids, plan->d_status);
+  else attn_bwd_tc_kernel<<<grid, AT_BWD_THREADS, AT_BWD_SMEM, stream>>>(t, plan->d_maps, ids, plan->d_status);
   return cudaGetLastError();
 }
 

@@ -20,6 +20,8 @@ struct LinDev {
   uint64_t w_off, b_off;      // element offsets into the flat arenas
   uint64_t z_ring;            // byte offset in the ring arena of z[depth][T*n_out] (pre-activation / q,k,v stash)
   uint64_t h_ring;            // byte offset of this Linear's output stash h[depth][T*n_out] (unused for the last Linear)
+  uint32_t b_soff;            // offset of the bias inside a slot of the stage's small-tensor version ring
+  uint32_t _pad;
 };
 
 // Static description of one stage (device copy).  A stage is [pre-op] Linear{1..4} [post-op]:
@@ -43,8 +45,17 @@ struct StageDev {
   int32_t mem_first;          // from_memory stage that runs its backward first (the last one): it stores, the others add
   int32_t ids_stream;         // embedding: which input stream (0, 1)
   int32_t ids_depth;          // embedding: slots of ids_ring, slot = microbatch % ids_depth
+  int32_t vdepth;             // weight versions the forward pass can reach: 1 (the live weights, tick-major) or tau_f + 1
+  uint32_t small_count;       // fp32 elements of a slot of s_ring (biases, LayerNorm gain and bias), a multiple of 64
+  uint32_t g_soff, beta_soff; // offsets of LayerNorm gain / bias inside a slot of s_ring
   int32_t _pad;
   uint64_t begin, end;        // padded element range of the stage's parameters in the arenas
+  // Queue of weight versions (Section 2.1: the forward pass of microbatch t reads the weights after t - tau_fwd
+  // updates), microbatch-major order only.  v_ring: [vdepth][end - begin] copies of the stage's slice in the GEMM
+  // operand type (what the forward GEMM and the embedding read); s_ring: [vdepth][small_count] fp32 copies of the
+  // tensors the forward pass reads in fp32 (bf16 operands only; with fp32 operands v_ring holds them).  Version v
+  // sits in slot v % vdepth; the update writes version k + 1 there.
+  uint64_t v_ring, s_ring;
   uint64_t tab_off, g_off, beta_off;   // arena offsets: embedding table / LayerNorm gain / LayerNorm bias
   uint64_t x_ring;            // ring: x[xdepth][T*d_in] main input (not used by an embedding stage)
   uint64_t u_ring;            // ring: u[depth][T*d_in] first Linear's input when a pre-op produces it
@@ -77,6 +88,9 @@ struct StageDyn {
   int32_t skip_wslot;         // emitting stage: slot of the receiving stage's skip buffer this tick's forward writes
   int32_t skip_rslot;         // receiving stage: slot of its skip buffer this tick's forward reads
   int32_t b_next_xslot;       // slot of the NEXT stage's x ring that holds the output of the microbatch in backward
+  int32_t f_vslot;            // slot of the version rings the forward reads (0 in tick-major order)
+  int32_t u_vslot;            // slot of the version rings the update fills with the new weights
+  int64_t lp_shift;           // the update writes the operand-type copy of element e to lp_base[lp_shift + e]
 };
 
 // Hyper-parameters the schedule kernel needs.
@@ -89,6 +103,8 @@ struct HyperDev {
   int64_t alpha_len;
   float beta1, beta2, eps;
   int64_t warm, period;       // synchronous warm-up (Section 4): the first `warm` microbatches enter `period` = 2P ticks apart
+  int32_t mb_major;           // microbatch-major order: one microbatch in flight, forward weights from the version rings
+  int32_t lp_elem;            // bytes of an element of the version rings' operand copy (2 or 4)
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks

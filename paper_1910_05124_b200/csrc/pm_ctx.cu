@@ -42,6 +42,12 @@ struct Layout {
   int32_t pe_seq = 0, pe_d = 0;
   int64_t loss_cap = 0;
   int32_t max_lin = 0, max_dim = 0, n_in_first = 0, n_out_last = 0;
+  // microbatch-major order
+  bool mb = false;
+  int32_t n_tables = 1;                 // per-tick tables: 1, or 2P + 1 (one per sub-tick and one for the grouped launches)
+  std::vector<SmallSeg> segs;           // fp32 tensors the forward pass reads, per version ring slot (bf16 operands)
+  uint64_t off_segs = 0;
+  std::vector<int32_t> pre_idx, ln_idx, embed_idx, res_idx;   // position of a stage in the stage lists (-1: not in it)
 };
 
 pm_status fail(pm_ctx* ctx, pm_status s, const std::string& msg);
@@ -65,6 +71,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   if (cfg->optimizer != PM_SGDM && cfg->optimizer != PM_ADAM) { err = "unknown optimizer"; return PM_ERR_INVALID_ARG; }
   if (cfg->loss != PM_LOSS_MSE && cfg->loss != PM_LOSS_CE) { err = "unknown loss"; return PM_ERR_INVALID_ARG; }
   if (cfg->t1_enable && cfg->t1_K < 1) { err = "t1_K must be >= 1"; return PM_ERR_INVALID_ARG; }
+  if (cfg->loop_order != PM_TICK_MAJOR && cfg->loop_order != PM_MB_MAJOR) { err = "unknown loop_order"; return PM_ERR_INVALID_ARG; }
+  const bool mb = cfg->loop_order == PM_MB_MAJOR;
+  L.mb = mb;
+  L.n_tables = mb ? 2 * P + 1 : 1;
   const uint64_t esz = cfg->compute_dtype == PM_F32 ? 4 : 2;
   const uint64_t T = (uint64_t)cfg->microbatch;
   const bool ce = cfg->loss == PM_LOSS_CE;
@@ -79,9 +89,13 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     const pm_stage_desc& sd = stages[p];
     StageDev& s = L.st[p];
     if (sd.n_ops < 1 || sd.n_ops > PM_MAX_LINEARS + 2 || !sd.ops) { stage_err(p, "bad op count"); return PM_ERR_INVALID_ARG; }
-    if (sd.tau_bkwd != 0 || sd.tau_fwd != 2 * (P - (p + 1)) + 1) {
+    if (!mb && (sd.tau_bkwd != 0 || sd.tau_fwd != 2 * (P - (p + 1)) + 1)) {
       stage_err(p, "the tick schedule realises tau_fwd = 2(P-i)+1, tau_bkwd = 0 only");
       return PM_ERR_UNSUPPORTED;
+    }
+    if (mb && (sd.tau_bkwd != 0 || sd.tau_fwd < 0)) {
+      stage_err(p, "microbatch-major order takes tau_fwd >= 0 with tau_bkwd = 0");
+      return sd.tau_fwd < 0 || sd.tau_bkwd < 0 ? PM_ERR_INVALID_ARG : PM_ERR_UNSUPPORTED;
     }
     if (sd.param_offset % PM_ALIGN_ELEMS || sd.param_count % PM_ALIGN_ELEMS) { stage_err(p, "param_offset/param_count must be multiples of 64"); return PM_ERR_INVALID_ARG; }
     if (sd.param_offset < prev_end) { err = "stage slices must ascend without overlap"; return PM_ERR_INVALID_ARG; }
@@ -94,6 +108,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     // the previous stage takes its ReLU mask from this stage's stashed input, one tick after this stage's own
     // backward: one more slot keeps it until then
     if (p > 0 && (L.st[p - 1].lin[L.st[p - 1].n_lin - 1].flags & LF_ACT_FROM_Y)) s.xdepth = s.tau_f + 3;
+    // microbatch-major order: one microbatch in flight, so every activation ring has one slot; what grows with
+    // the delay is the queue of weight versions
+    s.vdepth = 1;
+    if (mb) { s.depth = 1; s.xdepth = 1; s.vdepth = s.tau_f + 1; }
     s.begin = sd.param_offset; s.end = sd.param_offset + sd.param_count;
     prev_end = s.end;
     L.begin64[p] = (uint32_t)(s.begin / 64); L.end64[p] = (uint32_t)(s.end / 64);
@@ -108,7 +126,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (second && !L.st[p - 1].emit_memory) { stage_err(p, "a second-stream EMBED must follow the stage that emits the memory"); return PM_ERR_UNSUPPORTED; }
       if (L.pe_seq > 0 && (L.pe_seq != op.seq_len || L.pe_d != op.n_out)) { stage_err(p, "all EMBED ops share seq_len and width"); return PM_ERR_UNSUPPORTED; }
       s.ids_stream = second ? 1 : 0;
-      s.ids_depth = 2 * P - p;
+      s.ids_depth = mb ? 1 : 2 * P - p;
       if (second) L.n_streams = 2;
       if (op.n_in < 1 || op.n_out < 4 || (op.n_out & 3) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (width a multiple of four, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
       s.pre = PRE_EMBED; s.vocab = op.n_in; s.seq_len = op.seq_len;
@@ -219,6 +237,25 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (s.lin[l].flags & LF_WRITE_Z) { s.lin[l].z_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
       if (l < s.n_lin - 1) { s.lin[l].h_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
     }
+    if (mb) {
+      // queue of weight versions: the whole slice in the operand type, and (bf16 operands) the fp32 tensors the forward
+      // pass reads -- LayerNorm gain and bias, Linear biases -- packed into slots of small_count floats
+      s.v_ring = ring; ring = align_up(ring + (uint64_t)s.vdepth * (s.end - s.begin) * esz, 256);
+      uint32_t so = 0;
+      auto seg = [&](uint64_t arena_off, uint64_t n, uint32_t* soff) {
+        *soff = so;
+        const uint32_t padded = (uint32_t)align_up(n, PM_ALIGN_ELEMS);
+        L.segs.push_back(SmallSeg{arena_off, 0, padded, 0, p, (int32_t)so});     // ring_off, slot_stride filled below
+        so += padded;
+      };
+      if (esz == 2) {
+        if (s.pre == PRE_LN) { seg(s.g_off, (uint64_t)s.d_in, &s.g_soff); seg(s.beta_off, (uint64_t)s.d_in, &s.beta_soff); }
+        for (int l = 0; l < s.n_lin; ++l) seg(s.lin[l].b_off, (uint64_t)s.lin[l].n_out, &s.lin[l].b_soff);
+        s.small_count = so;
+        s.s_ring = ring; ring = align_up(ring + (uint64_t)s.vdepth * so * 4, 256);
+        for (auto& g : L.segs) if (g.stage == p) { g.ring_off = s.s_ring + 4ull * (uint32_t)g._pad; g.slot_stride = so; g._pad = 0; }
+      }
+    }
     L.max_lin = std::max(L.max_lin, s.n_lin);
     L.max_dim = std::max(L.max_dim, s.max_dim);
     if (s.pre != PRE_NONE) L.any_pre = 1;
@@ -232,6 +269,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       L.att_blocks = std::max(L.att_blocks, (int)(T / s.seq_len) * s.n_heads);
     }
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
+    L.sched[p].vdepth = s.vdepth; L.sched[p].begin = s.begin; L.sched[p].count = s.end - s.begin; L.sched[p].v_ring = s.v_ring;
   }
   for (int p = 0; p < P; ++p) {
     L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
@@ -243,8 +281,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   if (L.mem_stage >= 0) {
     if (L.last_mem_reader < 0) { err = "a memory is emitted but no CROSS_ATTENTION stage reads it"; return PM_ERR_UNSUPPORTED; }
     L.st[L.last_mem_reader].mem_first = 1;
-    L.mem_depth = 2 * P - 2 * L.mem_stage;
-    L.gmem_depth = P - L.mem_stage + 2;
+    L.mem_depth = mb ? 1 : 2 * P - 2 * L.mem_stage;
+    L.gmem_depth = mb ? 1 : P - L.mem_stage + 2;
     for (int p = 0; p < P; ++p) L.sched[p].gmem_depth = L.gmem_depth;
     L.mem_ring = ring; ring = align_up(ring + (uint64_t)L.mem_depth * T * L.mem_dim * esz, 256);
   }
@@ -261,7 +299,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   uint64_t w = 0;
   L.off_st = w; w = align_up(w + sizeof(StageDev) * P, 256);
   L.off_sched = w; w = align_up(w + sizeof(StageSched) * P, 256);
-  L.off_dyn = w; w = align_up(w + sizeof(StageDyn) * P, 256);
+  L.off_dyn = w; w = align_up(w + sizeof(StageDyn) * P * (uint64_t)L.n_tables, 256);
   L.off_nupd = w; w = align_up(w + sizeof(int64_t) * P, 256);
   L.off_b64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_e64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
@@ -274,15 +312,17 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_colred = w; w = align_up(w + (L.row_chunks > 1 ? (uint64_t)P * L.row_chunks * 2 * L.max_dim * 4 : 0), 256);
   L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
   L.ids.assign((size_t)4 * P, 0);
+  L.pre_idx.assign(P, -1); L.ln_idx.assign(P, -1); L.embed_idx.assign(P, -1); L.res_idx.assign(P, -1);
   for (int p = 0; p < P; ++p) {
     const StageDev& s = L.st[p];
-    if (s.pre != PRE_NONE) L.ids[(size_t)0 * P + L.n_pre++] = p;
+    if (s.pre != PRE_NONE) { L.pre_idx[p] = L.n_pre; L.ids[(size_t)0 * P + L.n_pre++] = p; }
     if (s.pre == PRE_LN) {
+      L.ln_idx[p] = L.n_ln;
       L.ids[(size_t)1 * P + L.n_ln++] = p; L.max_ln_dim = std::max(L.max_ln_dim, s.d_in);
       if ((s.d_in & 7) != 0 || s.d_in > 1024) L.ln_fused = 0;
     }
-    if (s.pre == PRE_EMBED) L.ids[(size_t)2 * P + L.n_embed++] = p;
-    if (s.post == POST_RESIDUAL) L.ids[(size_t)3 * P + L.n_res++] = p;
+    if (s.pre == PRE_EMBED) { L.embed_idx[p] = L.n_embed; L.ids[(size_t)2 * P + L.n_embed++] = p; }
+    if (s.post == POST_RESIDUAL) { L.res_idx[p] = L.n_res; L.ids[(size_t)3 * P + L.n_res++] = p; }
   }
   for (int l = 0; l < PM_MAX_LINEARS; ++l) {
     int32_t acc = 0;
@@ -294,6 +334,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.act_blocks[l] = acc;
   }
   L.off_ids = w; w = align_up(w + sizeof(int32_t) * L.ids.size(), 256);
+  L.off_segs = w; w = align_up(w + sizeof(SmallSeg) * L.segs.size(), 256);
   if (L.mem_stage >= 0 && !L.ln_fused) { err = "stages that read the memory need LayerNorm widths that are multiples of 8 and at most 1024"; return PM_ERR_UNSUPPORTED; }
   L.ln_chunk_rows = 64;
   L.ln_chunks = (int32_t)((T + L.ln_chunk_rows - 1) / L.ln_chunk_rows);
@@ -474,6 +515,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   UP(L.off_b64, c->L.begin64);
   UP(L.off_e64, c->L.end64);
   UP(L.off_ids, c->L.ids);
+  if (!c->L.segs.empty()) { UP(L.off_segs, c->L.segs); }
 #undef UP
   if (cfg->alpha_by_step) {
     if (cfg->alpha_len < 1) { delete c; return fail(nullptr, PM_ERR_INVALID_ARG, "alpha_len must be >= 1 with alpha_by_step"); }
@@ -481,7 +523,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "alpha table upload"); delete c; return r; }
   }
   e = cudaMemsetAsync(c->ws + L.off_nupd, 0, sizeof(int64_t) * P, c->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_dyn, 0, sizeof(StageDyn) * P, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_dyn, 0, sizeof(StageDyn) * P * (uint64_t)L.n_tables, c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_lossred, 0, 512, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // host tables may go out of scope after this
   if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "context set-up"); delete c; return r; }
@@ -493,6 +535,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.alpha_len = cfg->alpha_len;
   c->hp.beta1 = cfg->beta1; c->hp.beta2 = cfg->beta2; c->hp.eps = cfg->eps;
   c->hp.warm = 0; c->hp.period = 2 * (int64_t)cfg->n_stages;
+  c->hp.mb_major = L.mb ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -501,6 +544,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.n_in_first = L.n_in_first; t.n_out_last = L.n_out_last;
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
+  t.mb_major = L.mb ? 1 : 0; t.sel_p = -1;
+  for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
   t.any_pre = L.any_pre; t.any_ln = L.any_ln; t.any_embed = L.any_embed; t.any_residual = L.any_residual;
@@ -544,6 +589,18 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     std::string uerr;
     pm_status us = umma_plan_create(&c->umma, t, c->L.st, c->ws + L.off_umma, c->stream, uerr);
     if (us != PM_OK) { delete c; return fail(nullptr, us, uerr); }
+  }
+  if (L.mb) {
+    // version 0 of every stage's queue: the initial weights in the operand type, and the small fp32 tensors
+    const bool f32 = cfg->compute_dtype == PM_F32;
+    for (int p = 0; p < P && e == cudaSuccess; ++p) {
+      const StageDev& s = c->L.st[p];
+      const void* src = f32 ? (const void*)(arenas->w + s.begin) : (const void*)(arenas->w_lp + s.begin);
+      e = cudaMemcpyAsync(t.ring + s.v_ring, src, (s.end - s.begin) * (f32 ? 4 : 2), cudaMemcpyDeviceToDevice, c->stream);
+    }
+    if (e == cudaSuccess) e = launch_push_small(c->a.w, t.ring, (const SmallSeg*)(c->ws + L.off_segs), (int)c->L.segs.size(), t.dyn, 0, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "weight-version queue set-up"); pm_destroy(c); return r; }
   }
   *out = c;
   return PM_OK;
@@ -618,9 +675,143 @@ pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches) {
   return PM_OK;
 }
 
+
+// ---- microbatch-major order -------------------------------------------------------------------------------------
+// One microbatch at a time: stages 1..P forward (stage i reads weight version max(0, t - tau_fwd,i) from its queue),
+// the loss, stages P..1 backward against the live weights, the weight gradients, then the update of every stage,
+// which also writes version t + 1 into the queues.  The kernels are those of the tick schedule: sub-tick v of
+// microbatch t is virtual tick 2P t + v with exactly one stage in forward (v = i) or backward (v = 2P - 1 - i), so
+// mailboxes and skip buffers are addressed as in a pipeline tick; each launch is restricted to its stage.
+
+// Launch arguments of sub-tick table `v`, restricted to stage p (p < 0: all stages).
+static TickArgs mb_args(const pm_ctx* ctx, int v, int p) {
+  TickArgs t = ctx->ta;
+  const Layout& L = ctx->L;
+  const int P = ctx->cfg.n_stages;
+  t.dyn = (const StageDyn*)(ctx->ws + L.off_dyn) + (size_t)v * P;
+  if (p < 0) return t;
+  const StageDev& s = L.st[p];
+  const int32_t* ids = (const int32_t*)(ctx->ws + L.off_ids);
+  t.sel_p = p;
+  t.n_pre = L.pre_idx[p] >= 0 ? 1 : 0;      t.pre_ids = ids + (L.pre_idx[p] >= 0 ? L.pre_idx[p] : 0);
+  t.n_ln = L.ln_idx[p] >= 0 ? 1 : 0;        t.ln_ids = ids + P + (L.ln_idx[p] >= 0 ? L.ln_idx[p] : 0);
+  t.n_embed = L.embed_idx[p] >= 0 ? 1 : 0;  t.embed_ids = ids + 2 * P + (L.embed_idx[p] >= 0 ? L.embed_idx[p] : 0);
+  t.n_res = L.res_idx[p] >= 0 ? 1 : 0;      t.res_ids = ids + 3 * P + (L.res_idx[p] >= 0 ? L.res_idx[p] : 0);
+  t.any_pre = t.n_pre; t.any_ln = t.n_ln; t.any_embed = t.n_embed; t.any_residual = t.n_res;
+  if (!feeds_attention(s.post)) t.att_blocks = 0;
+  for (int l = 0; l < PM_MAX_LINEARS; ++l) {
+    const int32_t* start = L.ids.data() + (size_t)4 * P + (size_t)l * (P + 1);
+    t.act_first[l] = start[p];
+    t.act_blocks[l] = start[p + 1] - start[p];
+  }
+  return t;
+}
+
+static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
+  if (!inputs || !targets) return fail(ctx, PM_ERR_INVALID_ARG, "microbatch-major order takes a microbatch at every step (there is nothing to drain)");
+  const int dt = ctx->cfg.compute_dtype;
+  const int P = ctx->cfg.n_stages;
+  const int64_t mb = ctx->n_fed;
+  pm_status s;
+  s = TIMED(PM_PROF_SCHEDULE, check(ctx, launch_schedule_mb((const StageSched*)(ctx->ws + ctx->L.off_sched), (StageDyn*)(ctx->ws + ctx->L.off_dyn),
+                                                            ctx->hp, mb, ctx->stream), "schedule"));
+  if (s != PM_OK) return s;
+  s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, mb, ctx->stream), "ingest"));
+  if (s != PM_OK) return s;
+  s = run_phase(ctx, ctx->g_fwd, [&]() -> pm_status {
+    pm_status s;
+    for (int p = 0; p < P; ++p) {
+      const StageDev& sd = ctx->L.st[p];
+      const TickArgs ta = mb_args(ctx, p, p);
+      if (sd.pre != PRE_NONE && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ta, dt, ctx->ls), "embedding / LayerNorm forward"))) != PM_OK) return s;
+      for (int l = 0; l < sd.n_lin; ++l) {
+        prof_begin(ctx, PM_PROF_GEMM_FWD);
+        cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 0, l, ctx->ls) : umma_launch(ctx->umma, ta, 0, l, ctx->ls);
+        if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
+      }
+      const bool att = feeds_attention(sd.post);
+      if (att && ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
+      const int n_post = ((att && !ctx->attn) ? 1 : 0) + (sd.post == POST_RESIDUAL ? 1 : 0);
+      if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
+    }
+    return PM_OK;
+  });
+  if (s != PM_OK) return s;
+  ctx->n_fed = mb + 1;
+  ctx->phase = 1;
+  return PM_OK;
+}
+
+static pm_status mb_backward(pm_ctx* ctx) {
+  const int dt = ctx->cfg.compute_dtype;
+  const int P = ctx->cfg.n_stages;
+  // With one Linear per stage nothing overwrites a stage's dz before the end of the backward chain, so the weight
+  // gradients of all stages run as ONE grouped launch (the tick schedule's launch, which fills the GPU); stages
+  // with several Linears reuse their dz scratch from level to level and form each weight gradient on the spot.
+  const bool grouped = ctx->L.max_lin == 1;
+  pm_status s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
+    pm_status s;
+    for (int p = P - 1; p >= 0; --p) {
+      const StageDev& sd = ctx->L.st[p];
+      const TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
+      if (p == P - 1 && (s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
+      if (feeds_attention(sd.post)) {
+        if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ta, false, ctx->ls), "attention backward"))) != PM_OK) return s; }
+        else if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
+      }
+      for (int l = sd.n_lin - 1; l >= 0; --l) {
+        if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ta)))) != PM_OK) return s;
+        cudaError_t e;
+        if (!grouped) {
+          prof_begin(ctx, PM_PROF_WGRAD);
+          e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, l, ctx->ls) : umma_launch(ctx->umma, ta, 2, l, ctx->ls);
+          if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+        }
+        if (p == 0 && l == 0 && sd.pre != PRE_EMBED) continue;          // raw network inputs need no gradient
+        prof_begin(ctx, PM_PROF_DGRAD);
+        e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, 1, l, ctx->ls);
+        if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
+      }
+      const int n_pre = sd.pre != PRE_NONE ? pre_bwd_launches(ta) : 0;
+      if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ta, dt, ctx->ls), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
+    }
+    if (grouped) {
+      const TickArgs ta = mb_args(ctx, 2 * P, -1);
+      prof_begin(ctx, PM_PROF_WGRAD);
+      cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
+      if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+    }
+    return PM_OK;
+  });
+  if (s != PM_OK) return s;
+  ctx->phase = 2;
+  return PM_OK;
+}
+
+static pm_status mb_update(pm_ctx* ctx) {
+  const int P = ctx->cfg.n_stages;
+  const StageDyn* dyn_all = (const StageDyn*)(ctx->ws + ctx->L.off_dyn) + (size_t)2 * P * P;
+  pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
+    prof_begin(ctx, PM_PROF_UPDATE);
+    cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64), dyn_all,
+                                  (int64_t*)(ctx->ws + ctx->L.off_nupd), P, ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1,
+                                  ctx->cfg.beta2, ctx->cfg.eps, ctx->ls, ctx->ta.ring, ctx->hp.lp_elem);
+    pm_status s = check(ctx, e, "update");
+    if (s != PM_OK || ctx->L.segs.empty()) return s;
+    prof_begin(ctx, PM_PROF_UPDATE);
+    e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(), dyn_all, -1, ctx->ls);
+    return check(ctx, e, "weight-version push");
+  });
+  if (s != PM_OK) return s;
+  ctx->tick += 1;
+  ctx->phase = 0;
+  return PM_OK;
+}
+
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "pm_forward called out of order (expected pm_backward or pm_update)");
+  if (ctx->L.mb) return mb_forward(ctx, inputs, targets);
   if ((inputs == nullptr) != (targets == nullptr)) return fail(ctx, PM_ERR_INVALID_ARG, "inputs and targets must both be given or both be NULL");
   if (inputs && ctx->draining) return fail(ctx, PM_ERR_STATE, "microbatches must be fed on consecutive ticks; the pipeline is already draining");
   const int64_t mb = mb_at_tick(ctx->tick, ctx->hp.warm, ctx->hp.period);   // the microbatch that may enter now, or -1
@@ -660,6 +851,7 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
 pm_status pm_backward(pm_ctx* ctx) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 1) return fail(ctx, PM_ERR_STATE, "pm_backward must follow pm_forward");
+  if (ctx->L.mb) return mb_backward(ctx);
   const int dt = ctx->cfg.compute_dtype;
   const int P = ctx->cfg.n_stages;
   pm_status s;
@@ -695,6 +887,7 @@ pm_status pm_backward(pm_ctx* ctx) {
 pm_status pm_update(pm_ctx* ctx) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 2) return fail(ctx, PM_ERR_STATE, "pm_update must follow pm_backward");
+  if (ctx->L.mb) return mb_update(ctx);
   const int P = ctx->cfg.n_stages;
   const bool any = any_stage_active(ctx, P, 2 * P - 1);
   if (any) {
@@ -738,6 +931,20 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
   StageDyn d;
   int64_t n = 0;
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (ctx->L.mb) {
+    // the stage's forward ran in sub-tick `stage`, its backward in sub-tick 2P - 1 - stage of the last microbatch
+    const int P = ctx->cfg.n_stages;
+    StageDyn df, db;
+    const char* tab = ctx->ws + ctx->L.off_dyn;
+    if (e == cudaSuccess) e = cudaMemcpy(&df, tab + sizeof(StageDyn) * ((size_t)stage * P + stage), sizeof(StageDyn), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(&db, tab + sizeof(StageDyn) * ((size_t)(2 * P - 1 - stage) * P + stage), sizeof(StageDyn), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(&n, ctx->ws + ctx->L.off_nupd + sizeof(int64_t) * stage, sizeof(int64_t), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bookkeeping read-back");
+    if (pm_status ds = check_device_status(ctx)) return ds;
+    out8[0] = df.f_mb; out8[1] = df.f_ver; out8[2] = db.b_mb; out8[3] = db.b_ver; out8[4] = n;
+    out8[5] = df.f_vslot; out8[6] = db.b_slot; out8[7] = ctx->n_fed - 1;
+    return PM_OK;
+  }
   if (e == cudaSuccess) e = cudaMemcpy(&d, ctx->ws + ctx->L.off_dyn + sizeof(StageDyn) * stage, sizeof(StageDyn), cudaMemcpyDeviceToHost);
   if (e == cudaSuccess) e = cudaMemcpy(&n, ctx->ws + ctx->L.off_nupd + sizeof(int64_t) * stage, sizeof(int64_t), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "bookkeeping read-back");
@@ -753,7 +960,7 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
   // a microbatch's loss is computed P ticks after it entered; ticks completed so far = ctx->tick
   const int64_t last = ctx->tick - P - 1, t0 = ctx->hp.warm * ctx->hp.period;   // latest entry tick whose loss exists
   const int64_t entered = last < 0 ? 0 : (last < t0 ? last / ctx->hp.period + 1 : ctx->hp.warm + (last - t0) + 1);
-  const int64_t done = std::min<int64_t>(ctx->n_fed, entered);
+  const int64_t done = ctx->L.mb ? ctx->n_fed - (ctx->phase == 1 ? 1 : 0) : std::min<int64_t>(ctx->n_fed, entered);
   if (first_mb + n > done) return fail(ctx, PM_ERR_INVALID_ARG, "loss of a microbatch that has not finished was requested");
   if (done - first_mb > ctx->L.loss_cap) return fail(ctx, PM_ERR_INVALID_ARG, "requested losses have left the device log");
   cudaError_t e = cudaStreamSynchronize(ctx->stream);

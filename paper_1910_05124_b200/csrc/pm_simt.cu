@@ -170,14 +170,15 @@ __device__ __forceinline__ void actbwd_rows(const AT* __restrict__ dy, const AT*
 template <typename AT>
 __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
   const int* start = t.act_start + (size_t)lvl * (t.P + 1);
-  int lo = 0, hi = t.P - 1;                                 // stage of this column block: largest p with start[p] <= blockIdx.x
-  while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (start[mid] <= (int)blockIdx.x) lo = mid; else hi = mid - 1; }
+  int lo = 0, hi = t.P - 1;                                 // stage of this column block: largest p with start[p] <= its index
+  const int blk = (int)blockIdx.x + t.act_first[lvl];
+  while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (start[mid] <= blk) lo = mid; else hi = mid - 1; }
   const int p = lo;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
-  const int c0 = ((int)blockIdx.x - start[p]) * kActColsV;
+  const int c0 = (blk - start[p]) * kActColsV;
   if (c0 >= L.n_out) return;
   const int chunk = blockIdx.y;
   const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + t.chunk_rows);
@@ -229,7 +230,7 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
 
 // adds the per-row-chunk partial column sums in chunk order: db of Linear lvl
 __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
-  const int p = blockIdx.y;
+  const int p = stage_of_block(t, blockIdx.y);
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
@@ -259,7 +260,7 @@ cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t st
   else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || t.row_chunks == 1) return e;
-  dim3 g2((t.max_dim + 255) / 256, t.P);
+  dim3 g2((t.max_dim + 255) / 256, t.sel_p >= 0 ? 1 : t.P);
   bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
   return cudaGetLastError();
 }
@@ -274,7 +275,7 @@ constexpr int BM = 64, BN = 64, BK = 16;
 
 template <typename AT, typename WT, int MODE>
 __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
-  const int p = blockIdx.z;
+  const int p = stage_of_block(t, blockIdx.z);
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (lvl >= s.n_lin) return;
@@ -293,9 +294,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
   // operand sources
   const AT* xin = lin_input<AT>(t, s, d, lvl, MODE == 0);   // this Linear's input activation (forward or backward slot)
   const AT* dz = dz_src<AT>(t, s, d, lvl);
-  const WT* wf;
-  if (sizeof(WT) == 4) wf = reinterpret_cast<const WT*>(t.a.w) + L.w_off;
-  else wf = reinterpret_cast<const WT*>(t.a.w_lp) + L.w_off;
+  const WT* wf = fwd_weights<WT>(t, s, d, L.w_off);       // forward operand: the weights of the version the forward reads
   const float* wm = t.a.w + L.w_off;
   const float* dl = t.a.delta + L.w_off;
   const float gapf = (float)s.gap;
@@ -377,7 +376,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
     AT* zout = (L.flags & LF_WRITE_Z) ? ring_ptr<AT>(t, L.z_ring, d.f_slot, n_xout) : nullptr;
     AT* yout = y_dest<AT>(t, p, s, d, lvl);
     float* lout = (L.flags & LF_OUT_F32) ? ws_ptr<float>(t, t.yout_off) + (uint64_t)(d.tick & 1) * n_xout : nullptr;
-    const float* bias = t.a.w + L.b_off;
+    const float* bias = fwd_small<AT>(t, s, d, L.b_off, L.b_soff);
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -415,7 +414,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
 template <typename AT, typename WT>
 static cudaError_t launch_simt_t(const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
   const int mt = mode == 2 ? t.max_dim : t.T;
-  dim3 grid((t.max_dim + BN - 1) / BN, (mt + BM - 1) / BM, t.P);
+  dim3 grid((t.max_dim + BN - 1) / BN, (mt + BM - 1) / BM, t.sel_p >= 0 ? 1 : t.P);
   if (mode == 0) simt_gemm_kernel<AT, WT, 0><<<grid, 256, 0, stream>>>(t, lvl);
   else if (mode == 1) simt_gemm_kernel<AT, WT, 1><<<grid, 256, 0, stream>>>(t, lvl);
   else simt_gemm_kernel<AT, WT, 2><<<grid, 256, 0, stream>>>(t, lvl);

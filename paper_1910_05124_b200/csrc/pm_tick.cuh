@@ -45,7 +45,29 @@ struct TickArgs {
   int32_t second_embed_stage;   // the stage that embeds the second token stream (when n_streams == 2)
   int32_t max_lin;        // largest n_lin over stages
   int32_t max_dim;        // largest n_in / n_out over stages
+  // microbatch-major order: the forward pass reads its weights from the stages' version rings
+  int32_t mb_major;
+  // launches restricted to one stage (microbatch-major order runs the stages one after the other): kernels that take
+  // the stage from a block coordinate use sel_p instead (-1: all stages, the coordinate); the stage lists above then
+  // point at that stage's entry; act_first[lvl] is added to the block index of the activation-backward walk
+  int32_t sel_p;
+  int32_t act_first[PM_MAX_LINEARS];
 };
+
+// stage of a block in a kernel whose grid has one coordinate per stage
+__device__ __forceinline__ int stage_of_block(const TickArgs& t, unsigned coord) { return t.sel_p >= 0 ? t.sel_p : (int)coord; }
+// the weights the forward pass reads, in the GEMM operand type WT (float | bf16), at element offset `arena_off` of
+// the flat arenas: the live weights (tick-major: the stage holds one version), or the stage's version-ring slot
+template <typename WT> __device__ __forceinline__ const WT* fwd_weights(const TickArgs& t, const StageDev& s, const StageDyn& d, uint64_t arena_off) {
+  if (!t.mb_major) return (sizeof(WT) == 4 ? reinterpret_cast<const WT*>(t.a.w) : reinterpret_cast<const WT*>(t.a.w_lp)) + arena_off;
+  return reinterpret_cast<const WT*>(t.ring + s.v_ring) + (uint64_t)d.f_vslot * (s.end - s.begin) + (arena_off - s.begin);
+}
+// an fp32 tensor the forward pass reads (bias, LayerNorm gain / bias): arena offset and offset inside a small-ring slot
+template <typename AT> __device__ __forceinline__ const float* fwd_small(const TickArgs& t, const StageDev& s, const StageDyn& d, uint64_t arena_off, uint32_t soff) {
+  if (!t.mb_major) return t.a.w + arena_off;
+  if (sizeof(AT) == 4) return fwd_weights<float>(t, s, d, arena_off);
+  return reinterpret_cast<const float*>(t.ring + s.s_ring) + (uint64_t)d.f_vslot * s.small_count + soff;
+}
 
 // ---- where things live (shared by every tick kernel) -----------------------------------------------------
 template <typename AT> __device__ __forceinline__ AT* ring_at(const TickArgs& t, uint64_t off, int slot, uint64_t slot_elems) {

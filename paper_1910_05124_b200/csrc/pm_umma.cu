@@ -259,7 +259,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
           if (MODE == 0) {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.f_xslot : d.f_slot);
-            tma_load_2d(sb, lm + MAP_W_K, fb, k0, tl.n0);
+            tma_load_3d(sb, lm + MAP_W_K, fb, k0, tl.n0, d.f_vslot);
           } else {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             const int slot = (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.b_xslot : d.b_slot;
@@ -338,7 +338,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const int mrow = tl.m0 + q * 32;                                // first row of this warp's block
       const int nb = tl.n0 + half * 64;
       // bias of this warp's 64 columns, four per lane in lanes 0..15, on its way while the accumulator completes
-      const float4 bias4 = (MODE == 0 && lane < 16) ? load_bias4(t.a.w + L.b_off, nb + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 bias4 = (MODE == 0 && lane < 16) ? load_bias4(fwd_small<__nv_bfloat16>(t, s, d, L.b_off, L.b_soff), nb + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -461,6 +461,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         // every wait in it makes the compiler re-read what lives in memory)
         const int aslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.f_xslot : d.f_slot;
         const int xslot = (lvl == 0 && sd_.pre == PRE_NONE) ? d.b_xslot : d.b_slot;
+        const int vslot = d.f_vslot;                                  // weight version the forward reads
         const int n_kb = tl.n_kb;
         for (int kb = 0; kb < n_kb; ++kb) {
           const int k0 = kb * TILE_K;
@@ -470,7 +471,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
           const uint32_t fb = mapa_shared(bar_full + 8 * op.idx, 0);
           if (MODE == 0) {
             tma_load_3d_pair(sa, lm + MAP_ACT_K, fb, k0, ma, aslot);
-            tma_load_2d_pair(sb, lm + MAP_W_K, fb, k0, nbh);
+            tma_load_3d_pair(sb, lm + MAP_W_K, fb, k0, nbh, vslot);
           } else {
             tma_load_3d_pair(sa, lm + MAP_DZ_MN, fb, ma, k0, dz_slot);
             tma_load_3d_pair(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, ma + 64, k0, dz_slot);
@@ -546,7 +547,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
       const int mrow = tl.m0 + rank * TILE_M + q * 32;                // first row of this warp's blocks
       // bias of this warp's 128 columns, four per lane, on its way while the accumulator completes
-      const float4 bias4 = MODE == 0 ? load_bias4(t.a.w + L.b_off, tl.n0 + half * 128 + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 bias4 = MODE == 0 ? load_bias4(fwd_small<__nv_bfloat16>(t, s, d, L.b_off, L.b_soff), tl.n0 + half * 128 + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 34);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -1191,6 +1192,10 @@ struct UmmaPlan {
   bool pair[3][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
   size_t order_off[3][PM_MAX_LINEARS] = {};
   int P = 0;
+  // launches of one stage (microbatch-major order): the stage's tiles in ascending order are a slice of the identity list
+  std::vector<int> h_tile_start;         // host copy of the tile starts
+  const int* d_identity = nullptr;       // 0, 1, 2, ...
+  int max_ctas = 148;
 };
 
 // Tile tables of every (mode, level): the flattened tile ids per stage, and the order in which the persistent
@@ -1205,6 +1210,7 @@ struct TileTables {
   int grid[3][PM_MAX_LINEARS] = {};
   bool pair[3][PM_MAX_LINEARS] = {};
   size_t order_off[3][PM_MAX_LINEARS] = {};
+  int max_tiles = 0;                     // most tiles of any (mode, level)
 };
 
 static int device_sms() {
@@ -1264,6 +1270,7 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
         }
       }
       ts[P] = acc;
+      tt.max_tiles = std::max(tt.max_tiles, acc);
       tt.tile_start.insert(tt.tile_start.end(), ts_block.begin(), ts_block.end());
       for (int p = 0; p < P; ++p) tt.tile_start.insert(tt.tile_start.end(), (size_t)(ts_block[p + 1] - ts_block[p]), p);
       const int G = std::max(1, std::min(acc, pair ? sms / 2 : sms));     // persistent CTAs, or CTA pairs
@@ -1295,7 +1302,7 @@ static uint64_t ints_bytes(size_t n) { return ((uint64_t)n * sizeof(int) + 255) 
 
 uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st) {
   const TileTables tt = build_tile_tables(T, st, device_sms());
-  return 256 + maps_bytes((int)st.size()) + ints_bytes(tt.tile_start.size()) + ints_bytes(tt.orders.size());
+  return 256 + maps_bytes((int)st.size()) + ints_bytes(tt.tile_start.size()) + ints_bytes(tt.orders.size()) + ints_bytes((size_t)tt.max_tiles);
 }
 
 static bool encode(EncodeTiledFn fn, CUtensorMap* m, int kind, void* base, int rank, const uint64_t* dims,
@@ -1343,7 +1350,17 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       {
         uint64_t dims[2] = {n_in, n_out}, strides[1] = {n_in * 2}, strides4[1] = {n_in * 4};
         uint32_t box[2] = {TILE_K, TILE_N}, box4[2] = {TILE_N, TILE_K};
-        okm = okm && encode(fn, m + MAP_W_K, 0, (void*)(t.a.w_lp + L.w_off), 2, dims, strides, box, err);
+        {
+          // forward operand: the bf16 copy of w; in microbatch-major order one copy per version the forward can reach
+          uint64_t dims3[3] = {n_in, n_out, 1}, strides3[2] = {n_in * 2, n_in * n_out * 2};
+          uint32_t box3[3] = {TILE_K, TILE_N, 1};
+          void* wbase = (void*)(t.a.w_lp + L.w_off);
+          if (t.mb_major) {
+            dims3[2] = (uint64_t)s.vdepth; strides3[1] = (s.end - s.begin) * 2;
+            wbase = (void*)(reinterpret_cast<__nv_bfloat16*>(t.ring + s.v_ring) + (L.w_off - s.begin));
+          }
+          okm = okm && encode(fn, m + MAP_W_K, 0, wbase, 3, dims3, strides3, box3, err);
+        }
         okm = okm && encode(fn, m + MAP_W_F32, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
         okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
         uint32_t box4h[2] = {64, TILE_K};                               // CTA-pair dgrad: 64 columns per CTA
@@ -1408,6 +1425,10 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   char* ord_dev = ts_dev + ints_bytes(tt.tile_start.size());
   if (e == cudaSuccess) e = cudaMemcpyAsync(ts_dev, tt.tile_start.data(), tt.tile_start.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess && !tt.orders.empty()) e = cudaMemcpyAsync(ord_dev, tt.orders.data(), tt.orders.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
+  char* id_dev = ord_dev + ints_bytes(tt.orders.size());
+  std::vector<int> identity((size_t)tt.max_tiles);
+  for (int i = 0; i < tt.max_tiles; ++i) identity[(size_t)i] = i;
+  if (e == cudaSuccess && tt.max_tiles > 0) e = cudaMemcpyAsync(id_dev, identity.data(), identity.size() * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(region, 0, 256, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { err = std::string("tensor map upload: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
@@ -1422,6 +1443,9 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   plan->d_maps = (const CUtensorMap*)(region + 256);
   plan->d_tile_start = (const int*)ts_dev;
   plan->d_orders = (const int*)ord_dev;
+  plan->d_identity = (const int*)id_dev;
+  plan->h_tile_start = tt.tile_start;
+  plan->max_ctas = device_sms();
   *out = plan;
   return PM_OK;
 }
@@ -1431,11 +1455,21 @@ void umma_plan_destroy(UmmaPlan* plan) { delete plan; }
 int* umma_status_word(UmmaPlan* plan) { return plan ? plan->d_status : nullptr; }
 
 cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream) {
-  const int n_slots = plan->n_slots[mode][lvl];
+  int n_slots = plan->n_slots[mode][lvl];
   if (n_slots == 0) return cudaSuccess;
-  const int grid = plan->grid[mode][lvl];                             // one persistent CTA per SM
+  int grid = plan->grid[mode][lvl];                                   // one persistent CTA per SM
   const int* ts = plan->d_tile_start + plan->ts_off[mode][lvl];
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
+  if (t.sel_p >= 0) {                                                 // the tiles of one stage, in ascending order
+    const int* hts = plan->h_tile_start.data() + plan->ts_off[mode][lvl];
+    const int first = hts[t.sel_p];
+    n_slots = hts[t.sel_p + 1] - first;
+    if (n_slots == 0) return cudaSuccess;
+    ord = plan->d_identity + first;
+    const bool pr = plan->pair[mode][lvl];
+    const int G = std::max(1, std::min(n_slots, pr ? plan->max_ctas / 2 : plan->max_ctas));
+    grid = pr ? 2 * G : G;
+  }
   if (plan->pair[mode][lvl]) {
     if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);

@@ -23,53 +23,43 @@ namespace pm {
 // the one that entered at tick s-(2P-i) (microbatch = entry tick, except during a synchronous warm-up).  T1 (Eq. 2): alpha_i = alpha_base(k) / tau_i^p, p = 1 - min(k/K, 1).
 // T2: gamma_i = D^(1/(tau_fwd,i - tau_bkwd,i)).  Scalars are evaluated in double and rounded to
 // float once.
-__global__ void schedule_kernel(const StageSched* __restrict__ sched, const int64_t* __restrict__ nupd,
-                                StageDyn* __restrict__ dyn, HyperDev hp, int64_t tick, int64_t n_fed,
-                                int64_t flat_k) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= hp.n_stages) return;
-  StageSched s = sched[i];
+// Per-stage state of one tick: forward microbatch a and backward microbatch b (-1: idle), `ver` updates applied to the
+// stage so far, the version `fver` its forward reads; k >= 0 activates the update with that index.
+__device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t tick, int64_t a, int64_t b, int64_t k,
+                             int64_t ver, int64_t fver, bool slots) {
   StageDyn d;
-  const int P = hp.n_stages;
   d.tick = tick;
-  int64_t ver = nupd[i];
-  if (flat_k >= 0) {
-    d.f_mb = -1; d.b_mb = -1; d.k = flat_k;
-    d.f_slot = d.f_xslot = d.f_next_xslot = d.b_slot = d.b_xslot = 0;
-  } else {
-    int64_t a = mb_at_tick(tick - i, hp.warm, hp.period);
-    int64_t b = mb_at_tick(tick - (2 * (int64_t)P - (i + 1)), hp.warm, hp.period);
-    bool fa = a >= 0 && a < n_fed;
-    bool ba = b >= 0 && b < n_fed;
-    d.f_mb = fa ? a : -1;
-    d.b_mb = ba ? b : -1;
-    d.k = ba ? b : -1;
-    d.f_slot = fa ? (int32_t)(a % s.depth) : 0;
-    d.f_xslot = fa ? (int32_t)(a % s.xdepth) : 0;
-    d.f_next_xslot = (fa && s.next_xdepth > 0) ? (int32_t)(a % s.next_xdepth) : 0;
-    d.b_slot = ba ? (int32_t)(b % s.depth) : 0;
-    d.b_xslot = ba ? (int32_t)(b % s.xdepth) : 0;
-  }
+  const bool fa = a >= 0, ba = b >= 0;
+  d.f_mb = a; d.b_mb = b; d.k = k;
+  d.f_slot = (fa && slots) ? (int32_t)(a % s.depth) : 0;
+  d.f_xslot = (fa && slots) ? (int32_t)(a % s.xdepth) : 0;
+  d.f_next_xslot = (fa && slots && s.next_xdepth > 0) ? (int32_t)(a % s.next_xdepth) : 0;
+  d.b_slot = (ba && slots) ? (int32_t)(b % s.depth) : 0;
+  d.b_xslot = (ba && slots) ? (int32_t)(b % s.xdepth) : 0;
   d.gin_rslot = s.gin_depth > 0 ? (int32_t)((tick + s.gin_depth - 1) % s.gin_depth) : 0;
   d.prev_wslot = s.prev_gin_depth > 0 ? (int32_t)(tick % s.prev_gin_depth) : 0;
-  d.gmem_slot = (s.gmem_depth > 0 && d.b_mb >= 0) ? (int32_t)(d.b_mb % s.gmem_depth) : 0;
+  d.gmem_slot = (s.gmem_depth > 0 && ba) ? (int32_t)(b % s.gmem_depth) : 0;
   d.skip_wslot = s.skip_dst_depth > 0 ? (int32_t)(tick % s.skip_dst_depth) : 0;
   d.skip_rslot = s.skip_depth > 0 ? (int32_t)((tick + 1) % s.skip_depth) : 0;
-  d.b_next_xslot = (d.b_mb >= 0 && s.next_xdepth > 0) ? (int32_t)(d.b_mb % s.next_xdepth) : 0;
-  d.f_ver = ver;
+  d.b_next_xslot = (ba && slots && s.next_xdepth > 0) ? (int32_t)(b % s.next_xdepth) : 0;
+  d.f_ver = fver;
   d.b_ver = ver;
-  d.active_update = d.k >= 0 ? 1 : 0;
+  // version rings (microbatch-major order): version v sits in slot v % vdepth
+  d.f_vslot = s.vdepth > 1 ? (int32_t)(fver % s.vdepth) : 0;
+  d.u_vslot = s.vdepth > 1 ? (int32_t)((ver + 1) % s.vdepth) : 0;
+  d.lp_shift = hp.mb_major ? (int64_t)(s.v_ring / (uint64_t)hp.lp_elem) + (int64_t)d.u_vslot * (int64_t)s.count - (int64_t)s.begin : 0;
+  d.active_update = k >= 0 ? 1 : 0;
   d.alpha = 0.f; d.gamma = 0.f; d.one_minus_gamma = 1.f; d.bc1 = 1.f; d.bc2 = 1.f; d.use_delta = 0;
-  if (d.k >= 0) {
-    int64_t k = d.k;
+  const int64_t kk = k >= 0 ? k : b;                  // the update index of the microbatch in backward
+  if (kk >= 0) {
     double base = hp.alpha_const;
-    if (hp.alpha_tab != nullptr) base = hp.alpha_tab[k < hp.alpha_len ? k : hp.alpha_len - 1];
+    if (hp.alpha_tab != nullptr) base = hp.alpha_tab[kk < hp.alpha_len ? kk : hp.alpha_len - 1];
     double alpha = base;
     // warm-up microbatches (Section 4) are synchronous: standard step size, no correction, delta left alone; the T1
     // annealing counts from the first PipeMare step
-    const bool sync = k < hp.warm;
+    const bool sync = kk < hp.warm;
     if (hp.t1 && !sync) {
-      double r = (double)(k - hp.warm) / (double)hp.K;
+      double r = (double)(kk - hp.warm) / (double)hp.K;
       double p = 1.0 - (r < 1.0 ? r : 1.0);
       int tau = s.tau_f > 1 ? s.tau_f : 1;
       alpha = base / pow((double)tau, p);
@@ -81,11 +71,27 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
       d.use_delta = 1;
     }
     if (hp.optimizer == PM_ADAM) {
-      d.bc1 = (float)(1.0 - pow((double)hp.beta1, (double)(k + 1)));
-      d.bc2 = (float)(1.0 - pow((double)hp.beta2, (double)(k + 1)));
+      d.bc1 = (float)(1.0 - pow((double)hp.beta1, (double)(kk + 1)));
+      d.bc2 = (float)(1.0 - pow((double)hp.beta2, (double)(kk + 1)));
     }
   }
-  dyn[i] = d;
+  return d;
+}
+
+__global__ void schedule_kernel(const StageSched* __restrict__ sched, const int64_t* __restrict__ nupd,
+                                StageDyn* __restrict__ dyn, HyperDev hp, int64_t tick, int64_t n_fed,
+                                int64_t flat_k) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= hp.n_stages) return;
+  const StageSched s = sched[i];
+  const int P = hp.n_stages;
+  const int64_t ver = nupd[i];
+  if (flat_k >= 0) { dyn[i] = make_dyn(s, hp, tick, -1, -1, flat_k, ver, ver, false); return; }
+  int64_t a = mb_at_tick(tick - i, hp.warm, hp.period);
+  int64_t b = mb_at_tick(tick - (2 * (int64_t)P - (i + 1)), hp.warm, hp.period);
+  if (!(a >= 0 && a < n_fed)) a = -1;
+  if (!(b >= 0 && b < n_fed)) b = -1;
+  dyn[i] = make_dyn(s, hp, tick, a, b, b, ver, ver, true);
 }
 
 cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageDyn* dyn, HyperDev hp,
@@ -96,11 +102,41 @@ cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageD
   return cudaGetLastError();
 }
 
+// Microbatch-major order (the paper's own statement of the method, Section 2.1: a queue of weight versions per
+// stage).  Microbatch t runs alone: stage i's forward in sub-tick i, its backward in sub-tick 2P-1-i, on the same
+// mailbox-slot arithmetic as a pipeline tick (virtual tick = 2P t + sub-tick).  The forward reads version
+// max(0, t - tau_fwd,i) from the stage's version ring (during a synchronous warm-up version t, afterwards nothing
+// older than the end of the warm-up), the backward the live weights (version t).  Table v in 0..2P-1 serves the
+// launches of sub-tick v; table 2P marks every stage in backward with its own backward sub-tick's slots and an
+// active update: it serves the grouped weight-gradient launch and the fused update.
+__global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDyn* __restrict__ tables, HyperDev hp, int64_t t) {
+  const int P = hp.n_stages;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x, v = blockIdx.y;
+  if (i >= P) return;
+  const StageSched s = sched[i];
+  const int64_t base = 2 * (int64_t)P * t;
+  int64_t fver = t - s.tau_f;
+  if (t < hp.warm) fver = t; else if (fver < hp.warm) fver = hp.warm;
+  if (fver < 0) fver = 0;
+  StageDyn d;
+  if (v < 2 * P) d = make_dyn(s, hp, base + v, v == i ? t : -1, v == 2 * P - 1 - i ? t : -1, -1, t, fver, true);
+  else d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, t, t, fver, true);
+  tables[(size_t)v * P + i] = d;
+}
+
+cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream) {
+  const int threads = 128;
+  dim3 grid((hp.n_stages + threads - 1) / threads, 2 * hp.n_stages + 1);
+  schedule_mb_kernel<<<grid, threads, 0, stream>>>(sched, tables, hp, t);
+  return cudaGetLastError();
+}
+
 // ---- fused update ------------------------------------------------------------------------------
 
 struct UpdScalars {
   float alpha, gamma, omg, bc1, bc2;
   int use_delta;
+  int64_t lp_shift;
 };
 
 __device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
@@ -137,9 +173,11 @@ __device__ __forceinline__ float upd_one(float g, float w, float& m, float& s, f
 constexpr int kUpdThreads = 256;
 constexpr int kUpdUnroll = 2;      // float4 groups per thread per array in flight
 
-template <int OPT, bool HAS_LP>
+// LP: operand-type copy of the new weights: 0 none, 1 bfloat16, 2 float (a version-ring slot of fp32 operands);
+// element e of the arenas goes to lp_base[lp_shift + e], lp_shift from the stage's table entry (0: the w_lp arena)
+template <int OPT, int LP>
 __global__ void __launch_bounds__(kUpdThreads)
-update_kernel(ArenasDev a, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
+update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
               const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
               float beta1, float beta2, float eps) {
   extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends
@@ -172,6 +210,7 @@ update_kernel(ArenasDev a, const uint32_t* __restrict__ begin64, const uint32_t*
         const StageDyn& d = dyn[stage[u]];
         sc[u].alpha = d.alpha; sc[u].gamma = d.gamma; sc[u].omg = d.one_minus_gamma;
         sc[u].bc1 = d.bc1; sc[u].bc2 = d.bc2; sc[u].use_delta = d.use_delta;
+        if (LP != 0) sc[u].lp_shift = d.lp_shift;
         if (sc[u].use_delta) dl[u] = ld_stream(a.delta + e);
         if (OPT == PM_ADAM) s[u] = ld_stream(a.s + e);
       }
@@ -189,13 +228,15 @@ update_kernel(ArenasDev a, const uint32_t* __restrict__ begin64, const uint32_t*
       st_stream(a.m + e, m[u]);
       if (OPT == PM_ADAM) st_stream(a.s + e, s[u]);
       if (sc[u].use_delta) st_stream(a.delta + e, dl[u]);
-      if (HAS_LP) {
+      if (LP == 1) {
         __nv_bfloat162 lo2 = __floats2bfloat162_rn(wn.x, wn.y);
         __nv_bfloat162 hi2 = __floats2bfloat162_rn(wn.z, wn.w);
         uint2 packed;
         packed.x = *reinterpret_cast<uint32_t*>(&lo2);
         packed.y = *reinterpret_cast<uint32_t*>(&hi2);
-        *reinterpret_cast<uint2*>(a.w_lp + e) = packed;   // re-read by the next forward: default caching
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(lp_base) + (sc[u].lp_shift + (int64_t)e)) = packed;   // re-read by a later forward: default caching
+      } else if (LP == 2) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(lp_base) + (sc[u].lp_shift + (int64_t)e)) = wn;
       }
       if ((uint32_t)(v[u] >> 4) == sb[stage[u]] && (v[u] & 15) == 0) nupd[stage[u]] += 1;
     }
@@ -204,7 +245,7 @@ update_kernel(ArenasDev a, const uint32_t* __restrict__ begin64, const uint32_t*
 
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
-                          float eps, cudaStream_t stream) {
+                          float eps, cudaStream_t stream, void* lp_base, int lp_elem) {
   if (total64 == 0 || n_stages == 0) return cudaSuccess;
   uint64_t total_vec4 = total64 * 16;
   uint64_t per_block = (uint64_t)kUpdThreads * kUpdUnroll;
@@ -215,14 +256,35 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
   uint64_t cap = (uint64_t)sms * 8;                 // whole waves of resident blocks
   int blocks = (int)(need < cap ? need : cap);
   size_t smem = sizeof(uint32_t) * 2 * (size_t)n_stages;
-  bool lp = a.w_lp != nullptr;
-  if (optimizer == PM_SGDM) {
-    if (lp) update_kernel<PM_SGDM, true><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
-    else    update_kernel<PM_SGDM, false><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
-  } else {
-    if (lp) update_kernel<PM_ADAM, true><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
-    else    update_kernel<PM_ADAM, false><<<blocks, kUpdThreads, smem, stream>>>(a, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps);
+  // the operand-type copy: the w_lp arena (bfloat16) unless the caller names a version ring and its element size
+  if (lp_base == nullptr) { lp_base = a.w_lp; lp_elem = 2; }
+  const int lp = lp_base == nullptr ? 0 : (lp_elem == 4 ? 2 : 1);
+#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps)
+  if (optimizer == PM_SGDM) { if (lp == 0) PM_UPD(PM_SGDM, 0); else if (lp == 1) PM_UPD(PM_SGDM, 1); else PM_UPD(PM_SGDM, 2); }
+  else { if (lp == 0) PM_UPD(PM_ADAM, 0); else if (lp == 1) PM_UPD(PM_ADAM, 1); else PM_UPD(PM_ADAM, 2); }
+#undef PM_UPD
+  return cudaGetLastError();
+}
+
+// ---- fp32 copies of the small forward-read tensors into the version rings -------------------------------------
+// With bfloat16 operands the forward pass still reads biases and LayerNorm parameters in fp32; in microbatch-major
+// order their versions sit in a ring of their own, filled here from the master weights after every update.
+__global__ void __launch_bounds__(128) push_small_kernel(const float* __restrict__ w, char* __restrict__ ring, const SmallSeg* __restrict__ segs,
+                                                         int n_segs, const StageDyn* __restrict__ dyn, int slot_override) {
+  for (int sg = blockIdx.x; sg < n_segs; sg += gridDim.x) {
+    const SmallSeg g = segs[sg];
+    const int slot = slot_override >= 0 ? slot_override : dyn[g.stage].u_vslot;
+    float* dst = reinterpret_cast<float*>(ring + g.ring_off) + (uint64_t)slot * g.slot_stride;
+    const float* src = w + g.arena_off;
+    for (uint32_t i = threadIdx.x * 4; i < g.count; i += blockDim.x * 4)
+      *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(src + i);
   }
+}
+
+cudaError_t launch_push_small(const float* w, char* ring, const SmallSeg* segs, int n_segs, const StageDyn* dyn,
+                              int slot_override, cudaStream_t stream) {
+  if (n_segs == 0) return cudaSuccess;
+  push_small_kernel<<<n_segs < 1184 ? n_segs : 1184, 128, 0, stream>>>(w, ring, segs, n_segs, dyn, slot_override);
   return cudaGetLastError();
 }
 

@@ -22,9 +22,6 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
-template <typename AT> __device__ __forceinline__ const AT* table_ptr(const TickArgs& t);
-template <> __device__ __forceinline__ const float* table_ptr<float>(const TickArgs& t) { return t.a.w; }
-template <> __device__ __forceinline__ const __nv_bfloat16* table_ptr<__nv_bfloat16>(const TickArgs& t) { return t.a.w_lp; }
 
 // ---- pre-op forward: embedding or LayerNorm, one warp per row ------------------------------------------------
 //   embedding: u = table[id] * sqrt(d) + PE[position]     (table in the GEMM operand type)
@@ -83,7 +80,7 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
   const bool vec = (dm & 7) == 0;                            // 8 consecutive columns per lane, 256 per pass
   if (s.pre == PRE_EMBED) {
     const int32_t id = ring_at<int32_t>(t, s.ids_ring, (int)(d.f_mb % s.ids_depth), (uint64_t)t.T)[row];
-    const AT* e = table_ptr<AT>(t) + s.tab_off + (uint64_t)id * dm;
+    const AT* e = fwd_weights<AT>(t, s, d, s.tab_off) + (uint64_t)id * dm;
     const float* pe = ws_at<float>(t, t.pe_off) + (uint64_t)(row % s.seq_len) * dm;
     const float sc = sqrtf((float)dm);
     if (vec) {
@@ -106,8 +103,8 @@ __global__ void __launch_bounds__(256) pre_fwd_kernel(TickArgs t) {
     return;
   }
   const AT* x = (s.from_memory ? mem_at<AT>(t, d.f_mb) : ring_at<AT>(t, s.x_ring, d.f_xslot, n)) + (uint64_t)row * dm;
-  const float* g = t.a.w + s.g_off;
-  const float* b = t.a.w + s.beta_off;
+  const float* g = fwd_small<AT>(t, s, d, s.g_off, s.g_soff);
+  const float* b = fwd_small<AT>(t, s, d, s.beta_off, s.beta_soff);
   float sum = 0.f, sq = 0.f;
   if (vec && dm == 512) { ln_fwd_row<AT, 2>(t, s, d, x, g, b, u, skip, row, lane); return; }
   if (vec && dm == 1024) { ln_fwd_row<AT, 4>(t, s, d, x, g, b, u, skip, row, lane); return; }
@@ -209,7 +206,7 @@ struct AttnShape { int S, dk, d; };
 
 template <typename AT>
 __global__ void __launch_bounds__(256) attention_fwd_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = stage_of_block(t, blockIdx.y);
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.f_mb < 0 || (s.post != POST_ATTENTION && s.post != POST_CROSS_ATTENTION)) return;
@@ -283,7 +280,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
   S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0 && !skip_attention; any_res = t.any_residual != 0;
   cudaError_t e = cudaSuccess;
   if (any_att) {
-    dim3 grid(nblk, t.P);
+    dim3 grid(nblk, t.sel_p >= 0 ? 1 : t.P);
     if (dtype == PM_F32) attention_fwd_kernel<float><<<grid, 256, attn_fwd_smem(S, dk, 4), stream>>>(t);
     else attention_fwd_kernel<__nv_bfloat16><<<grid, 256, attn_fwd_smem(S, dk, 2), stream>>>(t);
     e = cudaGetLastError();
@@ -303,7 +300,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
 // dQ = dS K / sqrt(d_k); dK = dS^T Q / sqrt(d_k).  Results go to the stage's dy buffer as [dq | dk | dv].
 template <typename AT>
 __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t) {
-  const int p = blockIdx.y;
+  const int p = stage_of_block(t, blockIdx.y);
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || (s.post != POST_ATTENTION && s.post != POST_CROSS_ATTENTION)) return;
@@ -382,7 +379,7 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(TickArgs t) {
 
 cudaError_t launch_post_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   if (t.att_blocks <= 0) return cudaSuccess;
-  dim3 grid(t.att_blocks, t.P);
+  dim3 grid(t.att_blocks, t.sel_p >= 0 ? 1 : t.P);
   if (dtype == PM_F32) attention_bwd_kernel<float><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 4), stream>>>(t);
   else attention_bwd_kernel<__nv_bfloat16><<<grid, 256, attn_bwd_smem(t.att_S, t.att_dk, 2), stream>>>(t);
   return cudaGetLastError();

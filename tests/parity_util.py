@@ -4,15 +4,16 @@ import numpy as np
 import pm_inputs as I
 
 
-def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0):
+def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major"):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
     The first `warmup` microbatches enter 2P ticks apart (synchronous warm-up), the rest one per tick.
+    loop_order "mb_major": one call of pm_step per microbatch, nothing to drain.
     """
     import torch
     import paper_1910_05124_b200 as pm
-    pipe = pm.Pipeline(wl, params0)
+    pipe = pm.Pipeline(wl, params0, loop_order=loop_order)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
@@ -23,8 +24,9 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
     if warmup:
         pipe.pm_set_warmup(warmup)
     t0 = 2 * P * warmup                                        # first tick of the one-per-tick phase
-    for s in range(t0 + (n_steps - warmup) + 2 * P - 1):
-        mb = (s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0)
+    mb_major = pipe.mb_major
+    for s in range(n_steps if mb_major else t0 + (n_steps - warmup) + 2 * P - 1):
+        mb = s if mb_major else ((s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0))
         if 0 <= mb < n_steps:
             if encoder and is_encdec(wl):
                 src, dec_in, tg = I.seq2seq_batch(wl, mb)              # two token streams: [source | decoder input]

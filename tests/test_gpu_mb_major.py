@@ -1,0 +1,156 @@
+"""GPU parity of the microbatch-major loop order (a queue of weight versions per stage) against the oracle, and
+its agreement with the tick-major order on the same workload."""
+import numpy as np
+import pytest
+
+import pm_inputs as I
+from parity_util import run_gpu_pipeline, run_oracle, compare_params
+
+pytestmark = pytest.mark.gpu
+
+
+def check_book(book, res, n_steps, P):
+    ref = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    assert len(book) == n_steps * P
+    for key, (vf, vb) in book.items():
+        assert (vf, vb) == ref[key], f"microbatch/stage {key}: device ({vf},{vb}) oracle {ref[key]}"
+
+
+@pytest.mark.parametrize("P,width,T,per_stage,act,opt", [
+    (1, 64, 8, 1, "relu", "sgdm"),
+    (3, 40, 7, 2, "gelu", "sgdm"),
+    (5, 130, 33, 1, "relu", "adam"),
+    (2, 72, 65, 3, "none", "adam"),
+])
+def test_mb_major_fp32_mlp(cuda_device, P, width, T, per_stage, act, opt):
+    wl = I.mlp_workload("t", P, width, per_stage, act, T, compute="f32", optimizer=opt,
+                        alpha=0.01 if opt == "sgdm" else 1e-3, K=6, D=0.5, steps=14, seed=77 + P)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, P)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5)
+    compare_params(pipe, res, 2e-5 if opt == "adam" else 1e-5)
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam"])
+def test_mb_major_bf16_mlp_matches_oracle_and_tick_major(cuda_device, opt):
+    import torch
+    wl = I.cfg3_small(optimizer=opt)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2)
+    print("mb-major bf16 MLP worst relative weight error", worst)
+    # the two loop orders launch the same kernels on the same operands: identical results
+    pipe2, losses2, _ = run_gpu_pipeline(wl, params0, wl.steps, collect_book=False)
+    assert np.array_equal(losses, losses2)
+    assert torch.equal(pipe.w, pipe2.w)
+
+
+@pytest.mark.parametrize("tau", [(0, 0, 0, 0), (5, 0, 3, 1), (2, 2, 2, 2), (9, 1, 0, 4)])
+@pytest.mark.parametrize("compute", ["f32", "bf16"])
+def test_mb_major_any_forward_delays(cuda_device, tau, compute):
+    """Delay patterns the tick schedule cannot realise: all zero is synchronous training (no step-size division, no
+    correction, delta stays zero), the others are fixed per-stage forward delays of Section 2.1's model."""
+    import torch
+    f32 = compute == "f32"
+    wl = I.mlp_workload("delays", 4, 64 if f32 else 192, 1, "gelu", 24 if f32 else 40, compute=compute, optimizer="sgdm",
+                        alpha=0.01, K=6, D=0.5, steps=16, seed=191005124 + 61)
+    wl.tau_fwd = list(tau)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, 4)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-5 if f32 else 1e-3)
+    compare_params(pipe, res, 1e-5 if f32 else 2e-2)
+    if not any(tau):
+        assert float(pipe.delta.abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("compute", ["f32", "bf16"])
+def test_mb_major_encoder(cuda_device, compute):
+    import torch
+    f32 = compute == "f32"
+    wl = I.cfg4_small(compute=compute, n_layers=2, d_model=64, n_heads=4, d_ff=136, seq_len=16, batch=3, vocab=96, steps=24)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    worst = compare_params(pipe, res, 2e-5 if f32 else 2e-2, per_stage=not f32)
+    print("mb-major encoder", compute, "worst relative weight error", worst)
+    pipe2, losses2, _ = run_gpu_pipeline(wl, params0, wl.steps, collect_book=False)
+    assert np.array_equal(losses, losses2) and torch.equal(pipe.w, pipe2.w)      # same kernels, same operands
+
+
+@pytest.mark.parametrize("compute", ["f32", "bf16"])
+def test_mb_major_encoder_decoder(cuda_device, compute):
+    import torch
+    f32 = compute == "f32"
+    wl = I.cfg5_small(compute=compute, n_enc=2, n_dec=2, d_model=32 if f32 else 64, d_ff=64 if f32 else 128, seq_len=8 if f32 else 16,
+                      batch=2, vocab=40 if f32 else 96, steps=14)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    worst = compare_params(pipe, res, 2e-5 if f32 else 2e-2, per_stage=not f32)
+    print("mb-major encoder-decoder", compute, "worst relative weight error", worst)
+    pipe2, losses2, _ = run_gpu_pipeline(wl, params0, wl.steps, collect_book=False)
+    assert np.array_equal(losses, losses2) and torch.equal(pipe.w, pipe2.w)
+
+
+def test_mb_major_tensor_core_attention_and_pair_tiles(cuda_device):
+    """Sequences of 128 tokens, heads of width 64 and GEMMs of at least 256 rows and columns: the tensor-core
+    attention kernels and the CTA-pair GEMMs, launched one stage at a time, with the weight gradients of all
+    stages in one grouped launch at the end of the backward pass."""
+    import torch
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=256, n_heads=4, d_ff=512, seq_len=128, batch=2, vocab=264, steps=16)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    check_book(book, res, wl.steps, wl.n_stages)
+    print("mb-major tc loss errors", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    worst = compare_params(pipe, res, 2e-2, per_stage=True)
+    print("mb-major tc worst relative weight error (per stage vector)", worst)
+    pipe2, losses2, _ = run_gpu_pipeline(wl, params0, wl.steps, collect_book=False)
+    assert np.array_equal(losses, losses2) and torch.equal(pipe.w, pipe2.w)
+
+
+@pytest.mark.parametrize("compute,opt", [("f32", "sgdm"), ("f32", "adam"), ("bf16", "adam")])
+def test_mb_major_warmup(cuda_device, compute, opt):
+    """PipeMareW (Section 4): synchronous steps first.  In this order they are ordinary steps whose forward reads
+    the live weights; the switch clamps the version index at the end of the warm-up."""
+    f32 = compute == "f32"
+    wl = I.mlp_workload("warm", 4, 64 if f32 else 192, 2, "gelu", 16 if f32 else 40, compute=compute, optimizer=opt,
+                        alpha=0.01 if opt == "sgdm" else 1e-3, K=5, D=0.5, steps=18, seed=191005124 + 62)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps, warmup=5)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, warmup=5, loop_order="mb_major")
+    check_book(book, res, wl.steps, 4)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    compare_params(pipe, res, 2e-5 if f32 else 2e-2)
+
+
+def test_mb_major_rules(cuda_device):
+    import torch
+    import paper_1910_05124_b200 as pm
+    wl = I.mlp_workload("t", 2, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
+    pipe = pm.Pipeline(wl, I.init_stage_params(wl), loop_order="mb_major")
+    x, y = I.batch(wl, 0)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_INVALID_ARG"):
+        pipe.pm_step(None, None)                              # nothing to drain in this order
+    pipe.pm_forward(xd, yd)
+    with pytest.raises(pm.PipeMareError, match="not finished"):
+        pipe.pm_get_losses(0, 1)
+    pipe.pm_backward()
+    pipe.pm_update()
+    assert pipe.pm_get_losses(0, 1).shape == (1,)
+    wl.tau_bkwd = [1, 0]
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
+        pm.Pipeline(wl, I.init_stage_params(wl), loop_order="mb_major")
