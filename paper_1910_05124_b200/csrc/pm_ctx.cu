@@ -245,7 +245,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       auto seg = [&](uint64_t arena_off, uint64_t n, uint32_t* soff) {
         *soff = so;
         const uint32_t padded = (uint32_t)align_up(n, PM_ALIGN_ELEMS);
-        L.segs.push_back(SmallSeg{arena_off, 0, padded, 0, p, (int32_t)so});     // ring_off, slot_stride filled below
+        for (uint32_t o = 0; o < padded; o += 2048) {                           // pieces of at most 2048 floats: one block copies a piece
+          const uint32_t cnt = std::min<uint32_t>(2048, padded - o);
+          L.segs.push_back(SmallSeg{arena_off + o, 0, cnt, 0, p, (int32_t)(so + o)});   // ring_off, slot_stride filled below
+        }
         so += padded;
       };
       if (esz == 2) {
@@ -307,7 +310,9 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
   L.off_lossred = w; w = align_up(w + 512, 256);
   L.off_rowloss = w; w = align_up(w + (ce ? T * 4 : 0), 256);
-  L.chunk_rows = T > 512 ? 256 : 32;               // short microbatches: more, smaller blocks (the reductions are latency-bound)
+  // short microbatches: more, smaller blocks (the reductions are latency-bound); so do the one-stage launches of
+  // microbatch-major order, whose grids cover a single stage
+  L.chunk_rows = T > 512 ? (mb ? 64 : 256) : 32;
   L.row_chunks = (int32_t)((T + L.chunk_rows - 1) / L.chunk_rows);
   L.off_colred = w; w = align_up(w + (L.row_chunks > 1 ? (uint64_t)P * L.row_chunks * 2 * L.max_dim * 4 : 0), 256);
   L.off_pe = w; w = align_up(w + (uint64_t)L.pe_seq * L.pe_d * 4, 256);
@@ -336,7 +341,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_ids = w; w = align_up(w + sizeof(int32_t) * L.ids.size(), 256);
   L.off_segs = w; w = align_up(w + sizeof(SmallSeg) * L.segs.size(), 256);
   if (L.mem_stage >= 0 && !L.ln_fused) { err = "stages that read the memory need LayerNorm widths that are multiples of 8 and at most 1024"; return PM_ERR_UNSUPPORTED; }
-  L.ln_chunk_rows = 64;
+  L.ln_chunk_rows = mb ? 16 : 64;
   L.ln_chunks = (int32_t)((T + L.ln_chunk_rows - 1) / L.ln_chunk_rows);
   L.off_lnred = w; w = align_up(w + (uint64_t)L.n_ln * L.ln_chunks * 2 * L.max_ln_dim * 4, 256);
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
@@ -545,6 +550,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
   t.mb_major = L.mb ? 1 : 0; t.sel_p = -1;
+  t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
+  t.ln_li0 = 0; t.defer_finish = 0;
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
@@ -694,7 +701,7 @@ static TickArgs mb_args(const pm_ctx* ctx, int v, int p) {
   const int32_t* ids = (const int32_t*)(ctx->ws + L.off_ids);
   t.sel_p = p;
   t.n_pre = L.pre_idx[p] >= 0 ? 1 : 0;      t.pre_ids = ids + (L.pre_idx[p] >= 0 ? L.pre_idx[p] : 0);
-  t.n_ln = L.ln_idx[p] >= 0 ? 1 : 0;        t.ln_ids = ids + P + (L.ln_idx[p] >= 0 ? L.ln_idx[p] : 0);
+  t.n_ln = L.ln_idx[p] >= 0 ? 1 : 0;        t.ln_li0 = L.ln_idx[p] >= 0 ? L.ln_idx[p] : 0;      // the list itself stays whole: partial sums are kept per entry
   t.n_embed = L.embed_idx[p] >= 0 ? 1 : 0;  t.embed_ids = ids + 2 * P + (L.embed_idx[p] >= 0 ? L.embed_idx[p] : 0);
   t.n_res = L.res_idx[p] >= 0 ? 1 : 0;      t.res_ids = ids + 3 * P + (L.res_idx[p] >= 0 ? L.res_idx[p] : 0);
   t.any_pre = t.n_pre; t.any_ln = t.n_ln; t.any_embed = t.n_embed; t.any_residual = t.n_res;
@@ -731,7 +738,7 @@ static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets
       }
       const bool att = feeds_attention(sd.post);
       if (att && ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
-      const int n_post = ((att && !ctx->attn) ? 1 : 0) + (sd.post == POST_RESIDUAL ? 1 : 0);
+      const int n_post = ((att && !ctx->attn) ? 1 : 0) + ((sd.post == POST_RESIDUAL && !ctx->ta.res_fused) ? 1 : 0);
       if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
     }
     return PM_OK;
@@ -753,7 +760,8 @@ static pm_status mb_backward(pm_ctx* ctx) {
     pm_status s;
     for (int p = P - 1; p >= 0; --p) {
       const StageDev& sd = ctx->L.st[p];
-      const TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
+      TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
+      ta.defer_finish = grouped ? 1 : 0;        // the partial sums of bias and LayerNorm gradients are added up once, below
       if (p == P - 1 && (s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
       if (feeds_attention(sd.post)) {
         if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ta, false, ctx->ls), "attention backward"))) != PM_OK) return s; }
@@ -780,6 +788,8 @@ static pm_status mb_backward(pm_ctx* ctx) {
       prof_begin(ctx, PM_PROF_WGRAD);
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
       if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+      const int n_fin = deferred_finish_launches(ta);
+      if (n_fin && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_deferred_finish(ta, dt, ctx->ls), "bias / LayerNorm gradient sums", n_fin))) != PM_OK) return s;
     }
     return PM_OK;
   });
@@ -838,7 +848,7 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
         if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
       }
       if (ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ctx->ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
-      const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + (ctx->L.any_residual ? 1 : 0);
+      const int n_post = ((ctx->L.att_blocks > 0 && !ctx->attn) ? 1 : 0) + ((ctx->L.any_residual && !ctx->ta.res_fused) ? 1 : 0);
       if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ctx->ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
       return PM_OK;
     });

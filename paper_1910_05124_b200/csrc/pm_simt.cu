@@ -128,15 +128,15 @@ template <> struct Pair<__nv_bfloat16> {
 
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 
-// rows r, r + 8, ... < r1 of 8 columns: four rows are loaded before the first is used
-template <typename AT, int ACT>
+// rows r, r + NW, ... < r1 of 8 columns (NW = warps of the block): four rows are loaded before the first is used
+template <typename AT, int ACT, int NW>
 __device__ __forceinline__ void actbwd_rows(const AT* __restrict__ dy, const AT* __restrict__ z, AT* __restrict__ dz, int n_out, int c,
                                             int r, int r1, float (&sum)[8]) {
-  for (; r + 3 * kActWarps < r1; r += 4 * kActWarps) {
+  for (; r + 3 * NW < r1; r += 4 * NW) {
     float g[4][8], zz[4][8];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const uint64_t i = (uint64_t)(r + u * kActWarps) * n_out + c;
+      const uint64_t i = (uint64_t)(r + u * NW) * n_out + c;
       load8<AT>(dy + i, g[u]);
       if (ACT != PM_ACT_NONE) load8<AT>(z + i, zz[u]);
     }
@@ -145,13 +145,13 @@ __device__ __forceinline__ void actbwd_rows(const AT* __restrict__ dy, const AT*
       if (ACT != PM_ACT_NONE) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) g[u][k] = round_as<AT>(__fmul_rn(g[u][k], act_grad(zz[u][k], ACT)));
-        store8<AT>(dz + (uint64_t)(r + u * kActWarps) * n_out + c, g[u]);
+        store8<AT>(dz + (uint64_t)(r + u * NW) * n_out + c, g[u]);
       }
 #pragma unroll
       for (int k = 0; k < 8; ++k) sum[k] = __fadd_rn(sum[k], g[u][k]);
     }
   }
-  for (; r < r1; r += kActWarps) {
+  for (; r < r1; r += NW) {
     const uint64_t i = (uint64_t)r * n_out + c;
     float g[8];
     load8<AT>(dy + i, g);
@@ -167,11 +167,14 @@ __device__ __forceinline__ void actbwd_rows(const AT* __restrict__ dy, const AT*
   }
 }
 
-template <typename AT>
-__global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int lvl) {
+// NW warps per block: 8 in a grouped launch over all stages; 16 in a launch of one stage (microbatch-major order),
+// which has fewer blocks and needs more loads in flight per block
+template <typename AT, int NW>
+__global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   const int* start = t.act_start + (size_t)lvl * (t.P + 1);
   int lo = 0, hi = t.P - 1;                                 // stage of this column block: largest p with start[p] <= its index
   const int blk = (int)blockIdx.x + t.act_first[lvl];
+  if (t.sel_p >= 0) lo = hi = t.sel_p;                     // a launch of one stage: no search
   while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (start[mid] <= blk) lo = mid; else hi = mid - 1; }
   const int p = lo;
   const StageDyn& d = t.dyn[p];
@@ -198,12 +201,12 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
   float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (vec) {
     if (c < L.n_out) {
-      if (L.act == PM_ACT_NONE) actbwd_rows<AT, PM_ACT_NONE>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
-      else if (L.act == PM_ACT_RELU) actbwd_rows<AT, PM_ACT_RELU>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
-      else actbwd_rows<AT, PM_ACT_GELU>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      if (L.act == PM_ACT_NONE) actbwd_rows<AT, PM_ACT_NONE, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      else if (L.act == PM_ACT_RELU) actbwd_rows<AT, PM_ACT_RELU, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      else actbwd_rows<AT, PM_ACT_GELU, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
     }
   } else {
-    for (int r = r0 + warp; r < r1; r += kActWarps) {
+    for (int r = r0 + warp; r < r1; r += NW) {
       const uint64_t i = (uint64_t)r * L.n_out + c;
 #pragma unroll
       for (int k = 0; k < 8; ++k)
@@ -214,53 +217,83 @@ __global__ void __launch_bounds__(kActWarps * 32) actbwd_kernel(TickArgs t, int 
         }
     }
   }
-  __shared__ float red[kActWarps][kActColsV];
+  __shared__ float red[NW][kActColsV];
 #pragma unroll
   for (int k = 0; k < 8; ++k) red[warp][8 * lane + k] = sum[k];
   __syncthreads();
   const int cc = c0 + threadIdx.x;
-  if (cc < L.n_out) {
+  if (threadIdx.x < kActColsV && cc < L.n_out) {
     float a = 0.f;
 #pragma unroll
-    for (int w = 0; w < kActWarps; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
+    for (int w = 0; w < NW; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
     if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = a;
     else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc] = a;
   }
 }
 
-// adds the per-row-chunk partial column sums in chunk order: db of Linear lvl
+// adds the per-row-chunk partial column sums: db of Linear lvl.  A block owns 32 columns; warp w adds the partials of
+// chunks w, w + 8, ... in ascending order (all of its loads are issued before the first addition: the partials sit a
+// row of the buffer apart, so every load is a separate round trip), then the eight per-warp sums are added in warp
+// order.  The order is fixed, so the result is reproducible.
+constexpr int kFinCols = 32, kFinMaxPer = 32;            // columns per block; partials per warp held in registers at a time
+
 __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
   const int p = stage_of_block(t, blockIdx.y);
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= L.n_out) return;
-  const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * (2 * (uint64_t)t.max_dim) + c;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c = blockIdx.x * kFinCols + lane;
+  if (blockIdx.x * kFinCols >= L.n_out) return;
+  const uint64_t ps = 2 * (uint64_t)t.max_dim;
+  const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * ps + (c < L.n_out ? c : 0);
   float sum = 0.f;
-  int k = 0;
-  for (; k + 8 <= t.row_chunks; k += 8) {                   // eight partials in flight, added in chunk order
-    float v[8];
+  for (int k0 = warp; k0 < t.row_chunks; k0 += 8 * kFinMaxPer) {
+    float v[kFinMaxPer];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = part[(uint64_t)(k + u) * 2 * t.max_dim];
+    for (int u = 0; u < kFinMaxPer; ++u) { const int k = k0 + 8 * u; v[u] = k < t.row_chunks ? part[(uint64_t)k * ps] : 0.f; }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
+    for (int u = 0; u < kFinMaxPer; ++u) if (k0 + 8 * u < t.row_chunks) sum = __fadd_rn(sum, v[u]);
   }
-  for (; k < t.row_chunks; ++k) sum = __fadd_rn(sum, part[(uint64_t)k * 2 * t.max_dim]);
-  t.a.grad[L.b_off + c] = sum;
+  __shared__ float red[8][kFinCols];
+  red[warp][lane] = sum;
+  __syncthreads();
+  if (warp == 0 && c < L.n_out) {
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) a = __fadd_rn(a, red[w][lane]);
+    t.a.grad[L.b_off + c] = a;
+  }
 }
 
-int actbwd_launches(const TickArgs& t) { return t.row_chunks == 1 ? 1 : 2; }
+int actbwd_launches(const TickArgs& t) { return (t.row_chunks == 1 || t.defer_finish) ? 1 : 2; }
+
+int deferred_finish_launches(const TickArgs& t) { return (t.row_chunks > 1 ? t.max_lin : 0) + ln_finish_launches(t); }
+cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t stream) {
+  (void)dtype;
+  if (t.row_chunks > 1) {
+    dim3 g2((t.max_dim + kFinCols - 1) / kFinCols, t.P);
+    for (int lvl = 0; lvl < t.max_lin; ++lvl) bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return launch_ln_finish(t, stream);
+}
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
   if (t.act_blocks[lvl] == 0) return cudaSuccess;
   dim3 grid(t.act_blocks[lvl], t.row_chunks);
-  if (dtype == PM_F32) actbwd_kernel<float><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
-  else actbwd_kernel<__nv_bfloat16><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
+  if (t.sel_p >= 0 && t.row_chunks > 1) {
+    if (dtype == PM_F32) actbwd_kernel<float, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
+    else actbwd_kernel<__nv_bfloat16, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
+  } else {
+    if (dtype == PM_F32) actbwd_kernel<float, kActWarps><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
+    else actbwd_kernel<__nv_bfloat16, kActWarps><<<grid, kActWarps * 32, 0, stream>>>(t, lvl);
+  }
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || t.row_chunks == 1) return e;
-  dim3 g2((t.max_dim + 255) / 256, t.sel_p >= 0 ? 1 : t.P);
+  if (e != cudaSuccess || t.row_chunks == 1 || t.defer_finish) return e;
+  dim3 g2((t.max_dim + kFinCols - 1) / kFinCols, t.sel_p >= 0 ? 1 : t.P);
   bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
   return cudaGetLastError();
 }

@@ -52,6 +52,10 @@ struct TickArgs {
   // point at that stage's entry; act_first[lvl] is added to the block index of the activation-backward walk
   int32_t sel_p;
   int32_t act_first[PM_MAX_LINEARS];
+  int32_t res_fused;      // the forward GEMM's epilogue adds the skip tensor (bf16 tensor-core path): no residual kernel
+  int32_t ln_li0;         // first entry of ln_ids a launch covers (its grid counts entries from there)
+  int32_t defer_finish;   // launches of one stage leave the per-chunk partial sums of bias / LayerNorm gradients in place;
+                          // one grouped launch over all stages adds them up at the end of the backward pass
 };
 
 // stage of a block in a kernel whose grid has one coordinate per stage
@@ -146,6 +150,12 @@ cudaError_t launch_loss(const TickArgs& t, int dtype, cudaStream_t stream);
 // dz = dy * act'(z) and db = column sums, level `lvl` of every stage that runs backward this tick.
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream);
 int actbwd_launches(const TickArgs& t);
+// the finishing passes that launches with defer_finish left out, grouped over all stages (bias column sums, LayerNorm
+// parameter gradients)
+cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t stream);
+int deferred_finish_launches(const TickArgs& t);
+cudaError_t launch_ln_finish(const TickArgs& t, cudaStream_t stream);      // pm_xfmr.cu
+int ln_finish_launches(const TickArgs& t);
 
 // Transformer pieces (all grouped over the stages that carry the op this tick).
 cudaError_t launch_pre_fwd(const TickArgs& t, int dtype, cudaStream_t stream);        // embedding / LayerNorm forward (+ skip hand-over)

@@ -86,7 +86,8 @@ struct EpiState {
 template <int MODE>
 __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* lm, const StageDev& s, const StageDyn& d, const LinDev& L,
                                           int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
-                                          uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es) {
+                                          uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es,
+                                          const uint4 (&skq)[8]) {
   const uint32_t row_off = (uint32_t)lane * 128;
   const uint32_t sw = (uint32_t)(lane & 7);
   const bool f32out = MODE == 0 && (L.flags & LF_OUT_F32) != 0;
@@ -98,6 +99,9 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
   const uint32_t so = both ? 0u : es.slot * 4096u;                // slot of a single-output block
   if (MODE == 0) {
     const int act = L.act;
+    // A stage that ends in a residual add writes the sum itself: out = bf16(skip + bf16(acc + b)), straight into the
+    // next stage's input (or the memory ring); the skip tensor was sent by the emitting stage skip_depth - 1 ticks ago.
+    const bool resid = s.post == POST_RESIDUAL;                     // skq: this lane's 64 skip values (see load_skip64)
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       float bb[8];
@@ -119,6 +123,15 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
       } else {
         const uint32_t off = row_off + (((uint32_t)g ^ sw) << 4);
         if (!both) {                                                // one output: no activation (z = y = bf16(acc + b)), or a ReLU whose z is not kept
+          if (resid) {
+            const uint32_t w[4] = {skq[g].x, skq[g].y, skq[g].z, skq[g].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 sk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+              pf[2 * e] = __fadd_rn(sk.x, __bfloat162float(__float2bfloat16_rn(pf[2 * e])));
+              pf[2 * e + 1] = __fadd_rn(sk.y, __bfloat162float(__float2bfloat16_rn(pf[2 * e + 1])));
+            }
+          }
           if (act == PM_ACT_RELU) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) pf[e] = fmaxf(pf[e], 0.0f);   // bf16(max(x, 0)) = max(bf16(x), 0)
@@ -142,7 +155,7 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
   if (lane == 0) {
     if (MODE == 0) {
       const int yslot = lvl < s.n_lin - 1 ? d.f_slot
-                        : (s.post == POST_RESIDUAL ? 0 : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
+                        : (s.emit_memory ? (int)(d.f_mb % t.mem_depth) : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
       if (f32out) {
         tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
         if (nb + 32 < N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
@@ -162,6 +175,16 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
   es.stored = true;
   es.prev_both = both;
   if (!both) es.slot ^= 1u;
+}
+
+// The 64 skip-tensor values of row `row`, columns nb .. nb+63, that a residual stage's epilogue adds (zeros outside
+// the tensor and for other stages).  Issued before the accumulator is awaited, so the loads overlap the main loop.
+__device__ __forceinline__ void load_skip64(const TickArgs& t, const StageDev& s, const StageDyn& d, int N, int row, int nb, uint4 (&skq)[8]) {
+  const bool on = s.post == POST_RESIDUAL && row < t.T;
+  const __nv_bfloat16* skrow = ws_at<__nv_bfloat16>(t, s.skip_in) + (uint64_t)d.skip_rslot * ((uint64_t)t.T * N) + (uint64_t)row * N + nb;
+#pragma unroll
+  for (int g = 0; g < 8; ++g)                                       // columns are multiples of 8
+    skq[g] = (on && nb + 8 * g < N) ? __ldg(reinterpret_cast<const uint4*>(skrow + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
 }
 
 // bias of columns n .. n+3 (zero beyond the tensor); n is a multiple of four
@@ -339,6 +362,8 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       const int nb = tl.n0 + half * 64;
       // bias of this warp's 64 columns, four per lane in lanes 0..15, on its way while the accumulator completes
       const float4 bias4 = (MODE == 0 && lane < 16) ? load_bias4(fwd_small<__nv_bfloat16>(t, s, d, L.b_off, L.b_soff), nb + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
+      uint4 skq[8];
+      if (MODE == 0) load_skip64(t, s, d, tl.N, mrow + lane, nb, skq);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 4);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -354,7 +379,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       __syncwarp();
       acc.advance(2);
       if (mrow >= tl.M || nb >= tl.N) continue;                       // nothing of this block is inside the tensor
-      epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, 0, es);
+      epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, 0, es, skq);
     }
     if (lane == 0 && es.stored) tma_store_wait_all();                    // global writes complete before the CTA retires
   }
@@ -548,6 +573,8 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       const int mrow = tl.m0 + rank * TILE_M + q * 32;                // first row of this warp's blocks
       // bias of this warp's 128 columns, four per lane, on its way while the accumulator completes
       const float4 bias4 = MODE == 0 ? load_bias4(fwd_small<__nv_bfloat16>(t, s, d, L.b_off, L.b_soff), tl.n0 + half * 128 + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
+      uint4 skq[8];                                                   // skip values of the 64-column block in hand (residual stages)
+      if (MODE == 0) load_skip64(t, s, d, tl.N, mrow + lane, tl.n0 + half * 128, skq);
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 34);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -555,6 +582,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
         const int nb = tl.n0 + half * 128 + c * 64;
+        if (MODE == 0 && c == 1) load_skip64(t, s, d, tl.N, mrow + lane, nb, skq);   // the first block's were issued before the wait
         uint32_t r0[32], r1[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * P2_ACC_COLS + half * 128 + c * 64);
         tmem_ld32(taddr, r0);
@@ -565,7 +593,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         if (c == 1 && lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty + 8 * acc.idx, 0));   // this warp has read its part of the accumulator
         __syncwarp();
         if (mrow >= tl.M || nb >= tl.N) continue;                     // nothing of this block is inside the tensor
-        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es);
+        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es, skq);
       }
       acc.advance(2);
     }
@@ -1392,7 +1420,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         } else if (L.flags & LF_WRITE_Y) {
           char* ybase; uint64_t yslots;
           if (l < s.n_lin - 1) { ybase = t.ring + L.h_ring; yslots = (uint64_t)s.depth; }
-          else if (s.post == POST_RESIDUAL) { ybase = t.ws + s.ytmp; yslots = 1; }
+          else if (s.emit_memory) { ybase = t.ring + t.mem_ring; yslots = (uint64_t)t.mem_depth; }   // the residual sum is the memory
           else if (p < P - 1) { ybase = t.ring + st[p + 1].x_ring; yslots = (uint64_t)st[p + 1].xdepth; }
           else { ybase = t.ws + t.yout_off; yslots = 2; }
           uint64_t yd[3] = {n_out, T, yslots};

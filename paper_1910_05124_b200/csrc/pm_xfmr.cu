@@ -277,7 +277,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
   int S = 0, dk = 0, nblk = 0;
   bool any_res = false, any_att = false;
   // the shapes are uniform over stages in the supported workloads; the host keeps the maxima in TickArgs
-  S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0 && !skip_attention; any_res = t.any_residual != 0;
+  S = t.att_S; dk = t.att_dk; nblk = t.att_blocks; any_att = t.att_blocks > 0 && !skip_attention; any_res = t.any_residual != 0 && !t.res_fused;
   cudaError_t e = cudaSuccess;
   if (any_att) {
     dim3 grid(nblk, t.sel_p >= 0 ? 1 : t.P);
@@ -287,7 +287,7 @@ cudaError_t launch_post_fwd(const TickArgs& t, int dtype, cudaStream_t stream, b
     if (e != cudaSuccess) return e;
   }
   if (any_res) {
-    dim3 grid(64, t.n_res);
+    dim3 grid(t.sel_p >= 0 ? 592 : 64, t.n_res);          // a launch of one stage brings all the blocks itself
     if (dtype == PM_F32) residual_kernel<float><<<grid, 256, 0, stream>>>(t);
     else residual_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(t);
     e = cudaGetLastError();
@@ -655,7 +655,7 @@ __device__ __forceinline__ float du_total(const AT* du, const AT* gs, uint64_t i
 //   dxhat = du_total * gain_b (gain_b = gain - gap*delta: T2);  dx = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat*xhat))
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
-  const int p = t.ln_ids[blockIdx.y];
+  const int p = t.ln_ids[blockIdx.y + t.ln_li0];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN || p == 0) return;
@@ -733,7 +733,7 @@ constexpr int kLnCols = 256;                         // columns per block: 8 per
 
 template <typename AT>
 __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
-  const int p = t.ln_ids[blockIdx.z];
+  const int p = t.ln_ids[blockIdx.z + t.ln_li0];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
@@ -800,7 +800,7 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
 }
 
 __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
-  const int p = t.ln_ids[blockIdx.y];
+  const int p = t.ln_ids[blockIdx.y + t.ln_li0];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || s.pre != PRE_LN) return;
@@ -824,7 +824,7 @@ __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
 // per-block partials in block order by ln_fused_finish_kernel.
 template <typename AT, int NP, int WPR>
 __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(TickArgs t) {
-  const int li = blockIdx.y, p = t.ln_ids[li];
+  const int li = blockIdx.y + t.ln_li0, p = t.ln_ids[li];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0) return;
@@ -955,30 +955,43 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   }
 }
 
+// Adds the per-block partials of dgain, dbias.  A block owns 32 columns; warp w adds the partials of chunks w, w + 8, ...
+// in ascending order (its loads are issued before the first addition: partials of one column sit a buffer row apart,
+// so each is a separate round trip), then the eight per-warp sums are added in warp order: a fixed order.
+constexpr int kLnFinCols = 32, kLnFinPer = 16;
+
 __global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
-  const int li = blockIdx.y, p = t.ln_ids[li];
+  const int li = blockIdx.y + t.ln_li0, p = t.ln_ids[li];
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0) return;
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= s.d_in) return;
-  const float* part = ws_at<float>(t, t.lnred_off) + (uint64_t)li * t.ln_chunks * (2 * (uint64_t)t.max_ln_dim);
-  float a = 0.f, b2 = 0.f;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (blockIdx.x * kLnFinCols >= s.d_in) return;
+  const int c = blockIdx.x * kLnFinCols + lane;
   const uint64_t ps = 2 * (uint64_t)t.max_ln_dim;
-  int k = 0;
-  for (; k + 8 <= t.ln_chunks; k += 8) {                    // eight partials in flight, added in chunk order
-    float va[8], vb[8];
+  const float* part = ws_at<float>(t, t.lnred_off) + (uint64_t)li * t.ln_chunks * ps + (c < s.d_in ? c : 0);
+  float a = 0.f, b2 = 0.f;
+  for (int k0 = warp; k0 < t.ln_chunks; k0 += 8 * kLnFinPer) {
+    float va[kLnFinPer], vb[kLnFinPer];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) { va[u] = part[(uint64_t)(k + u) * ps + c]; vb[u] = part[(uint64_t)(k + u) * ps + t.max_ln_dim + c]; }
+    for (int u = 0; u < kLnFinPer; ++u) {
+      const int k = k0 + 8 * u;
+      va[u] = k < t.ln_chunks ? part[(uint64_t)k * ps] : 0.f;
+      vb[u] = k < t.ln_chunks ? part[(uint64_t)k * ps + t.max_ln_dim] : 0.f;
+    }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) { a = __fadd_rn(a, va[u]); b2 = __fadd_rn(b2, vb[u]); }
+    for (int u = 0; u < kLnFinPer; ++u) if (k0 + 8 * u < t.ln_chunks) { a = __fadd_rn(a, va[u]); b2 = __fadd_rn(b2, vb[u]); }
   }
-  for (; k < t.ln_chunks; ++k) {
-    a = __fadd_rn(a, part[(uint64_t)k * ps + c]);
-    b2 = __fadd_rn(b2, part[(uint64_t)k * ps + t.max_ln_dim + c]);
+  __shared__ float red[2][8][kLnFinCols];
+  red[0][warp][lane] = a; red[1][warp][lane] = b2;
+  __syncthreads();
+  if (warp == 0 && c < s.d_in) {
+    float ga = 0.f, gb = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { ga = __fadd_rn(ga, red[0][w][lane]); gb = __fadd_rn(gb, red[1][w][lane]); }
+    t.a.grad[s.g_off + c] = ga;
+    t.a.grad[s.beta_off + c] = gb;
   }
-  t.a.grad[s.g_off + c] = a;
-  t.a.grad[s.beta_off + c] = b2;
 }
 
 template <typename AT, int NP, int WPR>
@@ -991,7 +1004,7 @@ static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
     attr_set = true;
   }
   ln_bwd_fused_kernel<AT, NP, WPR><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(t);
-  ln_fused_finish_kernel<<<dim3((t.max_ln_dim + 255) / 256, t.n_ln), 256, 0, stream>>>(t);
+  if (!t.defer_finish) ln_fused_finish_kernel<<<dim3((t.max_ln_dim + kLnFinCols - 1) / kLnFinCols, t.n_ln), 256, 0, stream>>>(t);
   return cudaGetLastError();
 }
 
@@ -1187,7 +1200,19 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
   }
 }
 
-int pre_bwd_launches(const TickArgs& t) { return (t.any_ln ? (t.ln_fused ? 2 : (t.row_chunks == 1 ? 2 : 3)) : 0) + (t.any_embed ? 1 : 0); }
+int pre_bwd_launches(const TickArgs& t) {
+  const int fin = t.defer_finish ? 0 : 1;
+  return (t.any_ln ? (t.ln_fused ? 1 + fin : (t.row_chunks == 1 ? 2 : 2 + fin)) : 0) + (t.any_embed ? 1 : 0);
+}
+
+// the LayerNorm finishing pass on its own (grouped over the stages of ln_ids)
+int ln_finish_launches(const TickArgs& t) { return t.any_ln && (t.ln_fused || t.row_chunks > 1) ? 1 : 0; }
+cudaError_t launch_ln_finish(const TickArgs& t, cudaStream_t stream) {
+  if (!t.any_ln) return cudaSuccess;
+  if (t.ln_fused) ln_fused_finish_kernel<<<dim3((t.max_ln_dim + kLnFinCols - 1) / kLnFinCols, t.n_ln), 256, 0, stream>>>(t);
+  else if (t.row_chunks > 1) ln_param_finish_kernel<<<dim3((t.max_ln_dim + 255) / 256, t.n_ln), 256, 0, stream>>>(t);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
   cudaError_t e = cudaSuccess;
@@ -1201,7 +1226,7 @@ cudaError_t launch_pre_bwd(const TickArgs& t, int dtype, cudaStream_t stream) {
     else { ln_bwd_dx_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>(t); ln_bwd_param_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(t); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (t.row_chunks > 1) {
+    if (t.row_chunks > 1 && !t.defer_finish) {
       dim3 g3((t.max_ln_dim + 255) / 256, t.n_ln);
       ln_param_finish_kernel<<<g3, 256, 0, stream>>>(t);
       e = cudaGetLastError();

@@ -34,7 +34,8 @@ def test_reduce_over_ranks_two_gloo_ranks(tmp_path):
 
 
 def test_reference_arm_runs_without_a_gpu():
-    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+    # config 4 here: the default workload (config 5) takes the oracle minutes per step on a small host
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg4", "--steps", "1",
                           "--warmup", "0"], capture_output=True, text=True, timeout=600,
                          env=dict(os.environ, CUDA_VISIBLE_DEVICES=""))
     assert out.returncode == 0, out.stderr[-2000:]
@@ -42,3 +43,6 @@ def test_reference_arm_runs_without_a_gpu():
     r = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
     assert r["impl"] == "reference" and r["value"] > 0 and r["cpu_baseline"]["kind"] == "oracle"
     assert r["e2e"]["h2d_bytes_per_step"] == 0
+    sys.path.insert(0, ROOT)
+    import bench
+    assert r["config"]["workload"] == bench.WORKLOADS["cfg4"]      # the same string the CUDA arm prints
