@@ -19,7 +19,7 @@
  *   - Every function returns a pm_status; nothing throws or aborts.  After an
  *     error pm_last_error(ctx) gives a readable message.
  *   - Stages are numbered 1..P in the paper and 0..P-1 in array arguments here.
- *   - One microbatch per update (N = 1 in the notation of Section 2.1).
+ *   - One microbatch per update (N = 1 in the notation of Section 2.1) unless pm_config.n_micro says otherwise.
  *
  * Two loop orders compute the same recurrence (pm_config.loop_order):
  *   PM_TICK_MAJOR  the pipeline as it would run on P devices: every call of pm_step is one tick in which all
@@ -149,6 +149,14 @@ typedef struct {
   int64_t alpha_len;
   int64_t loss_log_capacity;     /* losses kept on the device (a ring); 0 = default 4096 */
   int32_t loop_order;            /* PM_TICK_MAJOR | PM_MB_MAJOR (see the top of this file) */
+  int32_t n_micro;               /* N of Section 2.1: microbatches per update; 0 or 1 = one.  N > 1 needs PM_MB_MAJOR
+                                    (else PM_ERR_UNSUPPORTED): calls t = 0, 1, ... of pm_step belong to update u = t / N;
+                                    tau_fwd counts updates (Table 1: ceil((2(P-i)+1)/N)), every microbatch of a minibatch
+                                    reads weight version max(0, u - tau_fwd,i); the minibatch loss is the mean of its N
+                                    microbatch losses, so dL/dy carries the factor 1/N and the N parameter gradients are
+                                    added in the grad arena in call order; pm_update applies update u after the N-th call
+                                    and is a no-op before.  The step-size schedule, the T1 annealing and Adam's bias
+                                    correction count updates. */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /
@@ -253,6 +261,15 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
 /* Number of CUDA kernels this context has enqueued since pm_init_stages (for launch accounting). */
 uint64_t pm_launch_count(pm_ctx* ctx);
 
+/* Self-test of the failure path of the tensor-core kernels (PM_BF16 contexts).  Every wait of those kernels on a
+ * barrier is bounded (about one second); when one expires the kernel records a code in a status word, stops, and
+ * the next synchronising call returns PM_ERR_TIMEOUT.  This call exercises exactly that path without disturbing
+ * anything: a one-thread kernel (no tensor memory, no copy in flight) waits with the given limit, in SM cycles, on
+ * a barrier on which nothing arrives.  It synchronises the stream, returns PM_ERR_TIMEOUT when the expiry was
+ * recorded and reported as designed (anything else is a defect), and clears the record, so the context stays
+ * usable.  Use a small limit (a few million cycles = milliseconds). */
+pm_status pm_selftest_wait_timeout(pm_ctx* ctx, int64_t limit_cycles);
+
 /* Optional timing of the tick's kernels by class, with CUDA events recorded on the context's stream around each
  * launch (up to 8192 launches between reads; later ones are not recorded).  pm_profile_read synchronises the
  * stream, writes the summed milliseconds and the number of timed launches per class (arrays of PM_PROF_CLASSES
@@ -275,7 +292,8 @@ void pm_destroy(pm_ctx* ctx);
  * and must hold zeros.  tau_fwd / tau_bkwd: host arrays.  From cfg the optimiser,
  * betas, eps, T1/T2 settings and alpha are read.  `workspace` is a device buffer of at
  * least pm_update_flat_workspace_bytes(n_stages) bytes that receives the stage table.
- * Asynchronous on `stream`. */
+ * Asynchronous on `stream`.  PM_ERR_INVALID_ARG for alpha_by_step with alpha_len < 1;
+ * PM_ERR_NOMEM for a slice that does not fit the arenas. */
 uint64_t pm_update_flat_workspace_bytes(int32_t n_stages);
 pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
                          const uint64_t* stage_counts, const int32_t* tau_fwd,

@@ -68,11 +68,12 @@ def linear_bwd(dy, x, z, W_bkwd, act, rnd=identity, need_dx=True):
     return dW, db, dx
 
 
-def mse_loss(y, target, rnd=identity):
-    """loss = mean over all T*out entries of (y - target)^2 ;  dy = 2 (y - target) / (T*out)."""
+def mse_loss(y, target, rnd=identity, grad_scale=1.0):
+    """loss = mean over all T*out entries of (y - target)^2 ;  dy = grad_scale * 2 (y - target) / (T*out).
+    grad_scale = 1/N when the microbatch is one of N whose mean is the minibatch loss (Section 2.1)."""
     r = y - np.asarray(target, dtype=np.float64)
     loss = float(np.mean(r * r))
-    dy = rnd(2.0 * r / r.size)
+    dy = rnd(2.0 * r / r.size * grad_scale)
     return loss, dy
 
 
@@ -184,8 +185,8 @@ def embed_bwd(dx, ids, vocab):
     return g
 
 
-def cross_entropy(logits, targets, rnd=identity):
-    """loss = mean_t (logsumexp(logits_t) - logits_t[target_t]);  dlogits = (softmax - onehot) / T."""
+def cross_entropy(logits, targets, rnd=identity, grad_scale=1.0):
+    """loss = mean_t (logsumexp(logits_t) - logits_t[target_t]);  dlogits = grad_scale * (softmax - onehot) / T."""
     T = logits.shape[0]
     m = logits.max(axis=1, keepdims=True)
     e = np.exp(logits - m)
@@ -194,4 +195,4 @@ def cross_entropy(logits, targets, rnd=identity):
     loss = float(np.mean(lse - logits[np.arange(T), targets]))
     dl = e / ssum
     dl[np.arange(T), targets] -= 1.0
-    return loss, rnd(dl / T)
+    return loss, rnd(dl / T * grad_scale)

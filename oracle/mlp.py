@@ -24,7 +24,7 @@ def make_grad_fn(stage_acts, data_fn, compute="f32"):
     data_fn: t -> (x [T,in], target [T,out]).  compute: 'f32' | 'bf16'."""
     rnd = bf16_round if compute == "bf16" else L.identity
 
-    def grad_fn(t, u_fwd, u_bkwd):
+    def grad_fn(t, u_fwd, u_bkwd, loss_scale=1.0):
         x, target = data_fn(t)
         h = rnd(np.asarray(x, dtype=np.float64))
         stash = []
@@ -35,7 +35,7 @@ def make_grad_fn(stage_acts, data_fn, compute="f32"):
                 y, z = L.linear_fwd(h, W, b, act, rnd)
                 stash.append((h, z))
                 h = y
-        loss, dy = L.mse_loss(h, target, rnd)
+        loss, dy = L.mse_loss(h, target, rnd, loss_scale)
         grads = [[None] * len(wf) for wf in u_fwd]
         flat = len(stash) - 1
         for i in reversed(range(len(stage_acts))):
@@ -50,7 +50,7 @@ def make_grad_fn(stage_acts, data_fn, compute="f32"):
     return grad_fn
 
 
-def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0):
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0, n_micro=1):
     """Run a pm_inputs.Workload-like description through the recurrence.
 
     params0: per stage a list of (W, b) pairs.  Returns recurrence.Result.
@@ -62,4 +62,5 @@ def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=N
               t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
     grad_fn = make_grad_fn(stage_acts, data_fn, wl.compute)
     return recurrence.run(flat0, wl.tau_fwd, wl.tau_bkwd, grad_fn,
-                          wl.steps if n_steps is None else n_steps, hp, dtype=dtype, on_step=on_step, warmup=warmup)
+                          wl.steps if n_steps is None else n_steps, hp, dtype=dtype, on_step=on_step, warmup=warmup,
+                          n_micro=n_micro)

@@ -16,7 +16,13 @@ Readings where the paper is silent:
   * delta_0 = 0.
   * All reads of version t (every stage's backward) happen before any stage
     writes version t+1.
-  * One microbatch per update (N = 1): microbatch index = update index.
+  * N microbatches per update (Section 2.1: "microbatch gradients are accumulated into gradient buffers, and weights
+    are updated only at minibatch boundaries"; Table 1: tau_fwd,i = ceil((2(P-i)+1)/N), passed in by the caller):
+    delays and version indices count UPDATES; microbatch t belongs to update u = t // N and every microbatch of a
+    minibatch reads the same versions; the minibatch loss is the mean of its N microbatch losses, so each microbatch's
+    gradient carries the factor 1/N (applied to dL/dy, where the backward pass starts) and the N gradients are added
+    in microbatch order in the state precision; the update after the N-th uses step index u.  N = 1: microbatch index =
+    update index.
 
 Warm-up epochs (PipeMareW, Section 4): the first `warmup` microbatches run the synchronous baseline, i.e. the same
 loop with every delay zero (standard step size, no T2 correction, delta left alone); PipeMare then starts from
@@ -46,8 +52,8 @@ class Result:
         self.opt = None
 
 
-def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None, warmup=0):
-    """Run n_steps microbatches, the first `warmup` of them synchronously.
+def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None, warmup=0, n_micro=1):
+    """Run n_steps microbatches, the first `warmup` of them synchronously; n_micro microbatches per update.
 
     params0:   per stage, a list of arrays (that stage's tensors).
     grad_fn:   (t, u_fwd, u_bkwd) -> (loss, grads) with grads shaped like params0.
@@ -67,7 +73,10 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
         v = max(min(warmup, t), t - lag)       # nothing older than the end of the warm-up (or version 0) exists
         return v, hist[i][-1 - (t - v)]
 
-    for t in range(n_steps):
+    assert n_micro >= 1 and (n_micro == 1 or warmup == 0), "warm-up epochs are stated for one microbatch per update"
+    gacc = None
+    for mb in range(n_steps):
+        t = mb // n_micro                       # update index: versions, delays and step counters count updates
         sync = t < warmup
         u_fwd, u_bkwd = [], []
         for i in range(P):
@@ -77,13 +86,20 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
             u_fwd.append(wf)
             u_bkwd.append([U.corrected_backward_weights(a, d, tf, tb, hp["t2"])
                            for a, d in zip(wb, delta[i])])
-            res.book.append((t, i + 1, vf, vb))
-        loss, grads = grad_fn(t, u_fwd, u_bkwd)
+            res.book.append((mb, i + 1, vf, vb))
+        if n_micro == 1:
+            loss, grads = grad_fn(mb, u_fwd, u_bkwd)
+        else:
+            loss, grads = grad_fn(mb, u_fwd, u_bkwd, loss_scale=1.0 / n_micro)
         res.losses.append(loss)
+        g_now = [[np.asarray(g, dtype=dtype) for g in stage] for stage in grads]
+        gacc = g_now if mb % n_micro == 0 else [[a + b for a, b in zip(sa, sb)] for sa, sb in zip(gacc, g_now)]
+        if mb % n_micro != n_micro - 1:
+            continue                            # gradients accumulate; weights change at the minibatch boundary only
         for i in range(P):
             new_stage = []
             for j, a in enumerate(w[i]):
-                g = np.asarray(grads[i][j], dtype=dtype)
+                g = gacc[i][j]
                 tf, tb = (0, 0) if sync else (tau_fwd[i], tau_bkwd[i])
                 a_new, opt[i][j], delta[i][j] = U.pipemare_update(
                     a, opt[i][j], delta[i][j], g, k=t, tau_fwd=tf, tau_bkwd=tb, hp=hp, k_t1=max(t - warmup, 0))

@@ -53,7 +53,7 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
         out["W"], out["b"] = f64(tensors[i]), f64(tensors[i + 1])
         return out
 
-    def grad_fn(t, u_fwd, u_bkwd):
+    def grad_fn(t, u_fwd, u_bkwd, loss_scale=1.0):
         data = data_fn(t)
         ids, targets = data[0], data[-1]
         dec_ids = data[1] if len(data) == 3 else None
@@ -106,7 +106,7 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
                 memory = main
             stash.append(st)
 
-        loss, d_main = L.cross_entropy(logits, targets, rnd)
+        loss, d_main = L.cross_entropy(logits, targets, rnd, loss_scale)
         d_skip_for = {}                                        # emitting stage -> gradient of the skip tensor it sent
         d_memory = None
         grads = [[None] * len(u_fwd[i]) for i in range(P)]
@@ -159,11 +159,11 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
     return grad_fn
 
 
-def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0):
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0, n_micro=1):
     """params0: per stage the list of tensors in the order [table] [gain, bias] W b."""
     from . import recurrence
     hp = dict(optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
               t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
     grad_fn = make_grad_fn(wl.stage_specs, data_fn, wl.n_heads, wl.seq_len, wl.vocab, wl.compute)
     return recurrence.run(params0, wl.tau_fwd, wl.tau_bkwd, grad_fn, wl.steps if n_steps is None else n_steps,
-                          hp, dtype=dtype, on_step=on_step, warmup=warmup)
+                          hp, dtype=dtype, on_step=on_step, warmup=warmup, n_micro=n_micro)

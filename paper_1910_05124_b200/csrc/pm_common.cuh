@@ -91,6 +91,9 @@ struct StageDyn {
   int32_t f_vslot;            // slot of the version rings the forward reads (0 in tick-major order)
   int32_t u_vslot;            // slot of the version rings the update fills with the new weights
   int64_t lp_shift;           // the update writes the operand-type copy of element e to lp_base[lp_shift + e]
+  int32_t accum;              // parameter gradients of this backward are ADDED to what the grad arena holds (the second to
+                              // N-th microbatch of a minibatch, Section 2.1); 0: they overwrite it
+  int32_t _pad2;
 };
 
 // Hyper-parameters the schedule kernel needs.
@@ -105,6 +108,8 @@ struct HyperDev {
   int64_t warm, period;       // synchronous warm-up (Section 4): the first `warm` microbatches enter `period` = 2P ticks apart
   int32_t mb_major;           // microbatch-major order: one microbatch in flight, forward weights from the version rings
   int32_t lp_elem;            // bytes of an element of the version rings' operand copy (2 or 4)
+  int32_t n_micro;            // N: microbatches per update (microbatch-major order; 1 elsewhere)
+  int32_t _pad;
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks

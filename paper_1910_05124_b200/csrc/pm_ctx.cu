@@ -73,6 +73,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   if (cfg->t1_enable && cfg->t1_K < 1) { err = "t1_K must be >= 1"; return PM_ERR_INVALID_ARG; }
   if (cfg->loop_order != PM_TICK_MAJOR && cfg->loop_order != PM_MB_MAJOR) { err = "unknown loop_order"; return PM_ERR_INVALID_ARG; }
   const bool mb = cfg->loop_order == PM_MB_MAJOR;
+  if (cfg->n_micro < 0) { err = "n_micro must be >= 0"; return PM_ERR_INVALID_ARG; }
+  if (cfg->n_micro > 1 && !mb) {
+    // in a running pipeline the version a forward pass reads depends on the microbatch's position inside its minibatch
+    // (floor((a - tau)/N) updates have landed), not on the fixed delay ceil(tau/N) of Table 1; the queue of weight
+    // versions realises Table 1's model exactly
+    err = "n_micro > 1 (several microbatches per update) is built for PM_MB_MAJOR order";
+    return PM_ERR_UNSUPPORTED;
+  }
   L.mb = mb;
   L.n_tables = mb ? 2 * P + 1 : 1;
   const uint64_t esz = cfg->compute_dtype == PM_F32 ? 4 : 2;
@@ -541,6 +549,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.beta1 = cfg->beta1; c->hp.beta2 = cfg->beta2; c->hp.eps = cfg->eps;
   c->hp.warm = 0; c->hp.period = 2 * (int64_t)cfg->n_stages;
   c->hp.mb_major = L.mb ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
+  c->hp.n_micro = cfg->n_micro > 1 ? cfg->n_micro : 1;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -552,6 +561,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.mb_major = L.mb ? 1 : 0; t.sel_p = -1;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
   t.ln_li0 = 0; t.defer_finish = 0;
+  t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
@@ -678,6 +688,7 @@ static bool any_stage_active(const pm_ctx* ctx, int64_t lo, int64_t hi) {
 pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches) {
   if (!ctx || n_microbatches < 0) return fail(ctx, PM_ERR_INVALID_ARG, "bad argument");
   if (ctx->tick != 0 || ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "the warm-up length is set before the first tick");
+  if (ctx->hp.n_micro > 1 && n_microbatches > 0) return fail(ctx, PM_ERR_UNSUPPORTED, "warm-up epochs are built for one microbatch per update");
   ctx->hp.warm = n_microbatches;
   return PM_OK;
 }
@@ -800,6 +811,11 @@ static pm_status mb_backward(pm_ctx* ctx) {
 
 static pm_status mb_update(pm_ctx* ctx) {
   const int P = ctx->cfg.n_stages;
+  if (ctx->n_fed % ctx->hp.n_micro != 0) {          // inside a minibatch: the gradients stay in the arena and the next microbatch adds to them
+    ctx->tick += 1;
+    ctx->phase = 0;
+    return PM_OK;
+  }
   const StageDyn* dyn_all = (const StageDyn*)(ctx->ws + ctx->L.off_dyn) + (size_t)2 * P * P;
   pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
     prof_begin(ctx, PM_PROF_UPDATE);
@@ -983,6 +999,24 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
 
 uint64_t pm_launch_count(pm_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+pm_status pm_selftest_wait_timeout(pm_ctx* ctx, int64_t limit_cycles) {
+  if (!ctx || limit_cycles < 1) return fail(ctx, PM_ERR_INVALID_ARG, "bad argument");
+  if (!ctx->umma) return fail(ctx, PM_ERR_UNSUPPORTED, "the bounded waits belong to the tensor-core kernels (PM_BF16 contexts)");
+  int* d_ret = reinterpret_cast<int*>(ctx->ws + ctx->L.off_lossred) + 100;      // a spare word of the loss-reduction block
+  cudaError_t e = cudaMemsetAsync(d_ret, 0, sizeof(int), ctx->stream);
+  if (e == cudaSuccess) e = umma_wait_timeout_probe(ctx->umma, (long long)limit_cycles, d_ret, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  int ret = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&ret, d_ret, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "wait self-test");
+  if (ret != 2) return fail(ctx, PM_ERR_STATE, "the probe's wait did not give up (code " + std::to_string(ret) + ")");
+  const pm_status st = check_device_status(ctx);        // what any synchronising call reports after an expiry
+  e = umma_clear_status(ctx->umma, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "wait self-test");
+  return st;
+}
+
 pm_status pm_profile_enable(pm_ctx* ctx, int32_t on) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (on && ctx->prof_ev.empty()) {
@@ -1046,10 +1080,12 @@ pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
   if (cfg->optimizer != PM_SGDM && cfg->optimizer != PM_ADAM) return fail(nullptr, PM_ERR_INVALID_ARG, "unknown optimizer");
   if (!arenas->w || !arenas->m || !arenas->delta || !arenas->grad || (cfg->optimizer == PM_ADAM && !arenas->s))
     return fail(nullptr, PM_ERR_INVALID_ARG, "missing arena");
+  if (cfg->alpha_by_step && cfg->alpha_len < 1) return fail(nullptr, PM_ERR_INVALID_ARG, "alpha_len must be >= 1 with alpha_by_step");
   const uint64_t need = pm_update_flat_workspace_bytes(n_stages);
   if (!workspace || workspace_bytes < need) return fail(nullptr, PM_ERR_NOMEM, "workspace too small: need " + std::to_string(need) + " bytes");
   const uint64_t P = (uint64_t)n_stages;
-  std::vector<char> host(need, 0);
+  thread_local std::vector<char> host;             // staging for the stage table: no allocation after the first call of a thread
+  host.assign(need, 0);
   uint64_t off_sched = 0, off_dyn = align_up(sizeof(StageSched) * P, 256);
   uint64_t off_nupd = align_up(off_dyn + sizeof(StageDyn) * P, 256);
   uint64_t off_b = align_up(off_nupd + sizeof(int64_t) * P, 256);
@@ -1062,6 +1098,8 @@ pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
     if (stage_offsets[i] % PM_ALIGN_ELEMS) return fail(nullptr, PM_ERR_INVALID_ARG, "stage offsets must be multiples of 64 elements");
     if (stage_offsets[i] < prev_end) return fail(nullptr, PM_ERR_INVALID_ARG, "stage slices must ascend without overlap");
     if (tau_fwd[i] < 0 || tau_bkwd[i] < 0 || tau_bkwd[i] > tau_fwd[i]) return fail(nullptr, PM_ERR_INVALID_ARG, "need 0 <= tau_bkwd <= tau_fwd");
+    if (stage_counts[i] > arenas->count || stage_offsets[i] > arenas->count - stage_counts[i])      // also catches a sum that would wrap
+      return fail(nullptr, PM_ERR_NOMEM, "stage slice exceeds the arenas");
     uint64_t end = align_up(stage_offsets[i] + stage_counts[i], PM_ALIGN_ELEMS);
     if (end > arenas->count) return fail(nullptr, PM_ERR_NOMEM, "stage slice exceeds the arenas");
     prev_end = end;
@@ -1071,7 +1109,7 @@ pm_status pm_update_flat(const pm_arenas* arenas, const uint64_t* stage_offsets,
   }
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
-  cudaError_t e = cudaMemcpyAsync(ws, host.data(), need, cudaMemcpyHostToDevice, st);
+  cudaError_t e = cudaMemcpyAsync(ws, host.data(), need, cudaMemcpyHostToDevice, st);   // pageable source: staged before the call returns
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "stage table upload");
   HyperDev hp{};
   hp.optimizer = cfg->optimizer; hp.t1 = cfg->t1_enable; hp.t2 = cfg->t2_enable; hp.n_stages = n_stages;

@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kLossThreads) mse_loss_kernel(TickArgs t) {
   AT* dy = gin_read<AT>(t, sl, d);
   float* partial = ws_ptr<float>(t, t.lossred_off);
   unsigned int* counter = reinterpret_cast<unsigned int*>(partial + kLossBlocks);
-  const float scale = (float)(2.0 / (double)n);
+  const float scale = (float)(2.0 / (double)n * (double)t.loss_scale);
   const uint64_t chunk = (n + gridDim.x - 1) / gridDim.x;
   const uint64_t lo = (uint64_t)blockIdx.x * chunk, hi = lo + chunk < n ? lo + chunk : n;
   float part = 0.f;
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
     float a = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
-    if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = a;
+    if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = d.accum ? __fadd_rn(t.a.grad[L.b_off + cc], a) : a;
     else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc] = a;
   }
 }
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
     float a = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) a = __fadd_rn(a, red[w][lane]);
-    t.a.grad[L.b_off + c] = a;
+    t.a.grad[L.b_off + c] = d.accum ? __fadd_rn(t.a.grad[L.b_off + c], a) : a;
   }
 }
 
@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
-        if (m < M && n < N) dW[(uint64_t)m * N + n] = acc[i][j];
+        if (m < M && n < N) dW[(uint64_t)m * N + n] = d.accum ? __fadd_rn(dW[(uint64_t)m * N + n], acc[i][j]) : acc[i][j];
       }
   }
 }

@@ -167,8 +167,13 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
       }
     } else {
-      tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
-      if (nb + 32 < N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
+      if (d.accum) {                                                // a later microbatch of the minibatch: dW adds to the arena
+        tma_reduce_add_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
+        if (nb + 32 < N) tma_reduce_add_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
+      } else {
+        tma_store_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
+        if (nb + 32 < N) tma_store_2d(lm + MAP_DW_OUT, obuf_s + 4096, nb + 32, mrow);
+      }
     }
     tma_store_commit();
   }
@@ -1479,6 +1484,27 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
 }
 
 void umma_plan_destroy(UmmaPlan* plan) { delete plan; }
+
+// ---- self-test of the bounded wait ---------------------------------------------------------------------------
+// One CTA, one thread: waits on an mbarrier on which nothing ever arrives, through the same bounded wait the GEMM
+// kernels use, with the cycle limit given as an argument.  No tensor memory is allocated and no copy is in flight, so
+// giving up is safe: the wait returns false, the abort flag and the status word are set, the kernel ends.
+__global__ void wait_timeout_probe_kernel(int* status, long long limit_cycles, int* returned) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  const uint32_t b = smem_u32(&bar);
+  mbar_init(b, 1);
+  abort_flag = 0;
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  const bool ok = mbar_try_wait(b, 0) || mbar_wait_slow(b, 0, &abort_flag, status, 99, limit_cycles);
+  *returned = ok ? 1 : (abort_flag ? 2 : 3);         // 2: gave up and raised the abort flag
+}
+
+cudaError_t umma_wait_timeout_probe(UmmaPlan* plan, long long limit_cycles, int* d_returned, cudaStream_t stream) {
+  wait_timeout_probe_kernel<<<1, 1, 0, stream>>>(plan->d_status, limit_cycles, d_returned);
+  return cudaGetLastError();
+}
+cudaError_t umma_clear_status(UmmaPlan* plan, cudaStream_t stream) { return cudaMemsetAsync(plan->d_status, 0, sizeof(int), stream); }
 
 int* umma_status_word(UmmaPlan* plan) { return plan ? plan->d_status : nullptr; }
 

@@ -16,6 +16,10 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
 void umma_plan_destroy(UmmaPlan* plan);
 // Device word that a CTA sets when one of its bounded waits expired (0 = none).
 int* umma_status_word(UmmaPlan* plan);
+// Self-test: launches a one-thread kernel whose bounded wait (limit in SM cycles) must expire; it sets the plan's status
+// word like a real expiry would and writes 2 to *d_returned.  umma_clear_status resets the status word.
+cudaError_t umma_wait_timeout_probe(UmmaPlan* plan, long long limit_cycles, int* d_returned, cudaStream_t stream);
+cudaError_t umma_clear_status(UmmaPlan* plan, cudaStream_t stream);
 // mode: 0 forward, 1 dgrad (corrected weights formed in the operand-load path), 2 wgrad.
 cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cudaStream_t stream);
 

@@ -26,9 +26,11 @@ namespace pm {
 // Per-stage state of one tick: forward microbatch a and backward microbatch b (-1: idle), `ver` updates applied to the
 // stage so far, the version `fver` its forward reads; k >= 0 activates the update with that index.
 __device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t tick, int64_t a, int64_t b, int64_t k,
-                             int64_t ver, int64_t fver, bool slots) {
+                             int64_t ver, int64_t fver, bool slots, int64_t kb = -2) {
   StageDyn d;
   d.tick = tick;
+  d.accum = 0; d._pad2 = 0;
+  if (kb == -2) kb = b;                               // update index the microbatch in backward belongs to (N = 1: itself)
   const bool fa = a >= 0, ba = b >= 0;
   d.f_mb = a; d.b_mb = b; d.k = k;
   d.f_slot = (fa && slots) ? (int32_t)(a % s.depth) : 0;
@@ -50,7 +52,7 @@ __device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t ti
   d.lp_shift = hp.mb_major ? (int64_t)(s.v_ring / (uint64_t)hp.lp_elem) + (int64_t)d.u_vslot * (int64_t)s.count - (int64_t)s.begin : 0;
   d.active_update = k >= 0 ? 1 : 0;
   d.alpha = 0.f; d.gamma = 0.f; d.one_minus_gamma = 1.f; d.bc1 = 1.f; d.bc2 = 1.f; d.use_delta = 0;
-  const int64_t kk = k >= 0 ? k : b;                  // the update index of the microbatch in backward
+  const int64_t kk = k >= 0 ? k : kb;                 // the update index of the microbatch in backward
   if (kk >= 0) {
     double base = hp.alpha_const;
     if (hp.alpha_tab != nullptr) base = hp.alpha_tab[kk < hp.alpha_len ? kk : hp.alpha_len - 1];
@@ -115,12 +117,17 @@ __global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDy
   if (i >= P) return;
   const StageSched s = sched[i];
   const int64_t base = 2 * (int64_t)P * t;
-  int64_t fver = t - s.tau_f;
-  if (t < hp.warm) fver = t; else if (fver < hp.warm) fver = hp.warm;
+  // N microbatches per update (Section 2.1): versions, delays and step indices count updates; microbatch t belongs to
+  // update u = t / N, every microbatch of a minibatch reads the same versions, the update follows the N-th
+  const int64_t N = hp.n_micro > 1 ? hp.n_micro : 1;
+  const int64_t u = t / N;
+  int64_t fver = u - s.tau_f;
+  if (u < hp.warm) fver = u; else if (fver < hp.warm) fver = hp.warm;
   if (fver < 0) fver = 0;
   StageDyn d;
-  if (v < 2 * P) d = make_dyn(s, hp, base + v, v == i ? t : -1, v == 2 * P - 1 - i ? t : -1, -1, t, fver, true);
-  else d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, t, t, fver, true);
+  if (v < 2 * P) d = make_dyn(s, hp, base + v, v == i ? t : -1, v == 2 * P - 1 - i ? t : -1, -1, u, fver, true, u);
+  else d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, (t % N == N - 1) ? u : -1, u, fver, true, u);
+  d.accum = (t % N != 0) ? 1 : 0;
   tables[(size_t)v * P + i] = d;
 }
 

@@ -65,6 +65,7 @@ pm_status pm_update_flat_static(const pm_arenas* arenas, const uint64_t* stage_o
   if (cfg->optimizer != PM_SGDM && cfg->optimizer != PM_ADAM) return fail(PM_ERR_INVALID_ARG, "unknown optimizer");
   if (!arenas->w || !arenas->m || !arenas->delta || !arenas->grad || (cfg->optimizer == PM_ADAM && !arenas->s))
     return fail(PM_ERR_INVALID_ARG, "missing arena");
+  if (cfg->alpha_by_step && cfg->alpha_len < 1) return fail(PM_ERR_INVALID_ARG, "alpha_len must be >= 1 with alpha_by_step");
 
   // once per device, with that device current: ask the runtime where the array lives on this GPU
   int dev = -1;
@@ -99,6 +100,8 @@ pm_status pm_update_flat_static(const pm_arenas* arenas, const uint64_t* stage_o
     if (stage_offsets[i] % PM_ALIGN_ELEMS) return fail(PM_ERR_INVALID_ARG, "stage offsets must be multiples of 64 elements");
     if (stage_offsets[i] < prev_end) return fail(PM_ERR_INVALID_ARG, "stage slices must ascend without overlap");
     if (tau_fwd[i] < 0 || tau_bkwd[i] < 0 || tau_bkwd[i] > tau_fwd[i]) return fail(PM_ERR_INVALID_ARG, "need 0 <= tau_bkwd <= tau_fwd");
+    if (stage_counts[i] > arenas->count || stage_offsets[i] > arenas->count - stage_counts[i])      // also catches a sum that would wrap
+      return fail(PM_ERR_NOMEM, "stage slice exceeds the arenas");
     uint64_t end = align_up(stage_offsets[i] + stage_counts[i], PM_ALIGN_ELEMS);
     if (end > arenas->count) return fail(PM_ERR_NOMEM, "stage slice exceeds the arenas");
     prev_end = end;

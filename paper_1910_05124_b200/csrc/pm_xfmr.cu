@@ -506,7 +506,7 @@ __global__ void __launch_bounds__(256) ce_loss_kernel(TickArgs t) {
   if (threadIdx.x == 0) { float a = 0.f; for (int i = 0; i < 8; ++i) a += red[i]; bc = a; }
   __syncthreads();
   sum = bc;
-  const float invT = 1.0f / (float)t.T, rsum = 1.0f / sum;
+  const float invT = t.loss_scale / (float)t.T, rsum = 1.0f / sum;
   if (in_regs) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -606,7 +606,7 @@ __global__ void __launch_bounds__(kCeLongThreads) ce_loss_long_kernel(TickArgs t
   if (threadIdx.x == 0) { float a = 0.f; for (int i = 0; i < kCeLongThreads / 32; ++i) a += red[i]; bc[1] = a; }
   __syncthreads();
   sum = bc[1];
-  const float invT = 1.0f / (float)t.T, rsum = 1.0f / sum;
+  const float invT = t.loss_scale / (float)t.T, rsum = 1.0f / sum;
   for (int i = threadIdx.x; i < n4; i += kCeLongThreads) {
     const float4 q = rowbuf[i];
     const int c = 4 * i;
@@ -789,8 +789,8 @@ __global__ void __launch_bounds__(256) ln_bwd_param_kernel(TickArgs t) {
 #pragma unroll
     for (int w = 0; w < 8; ++w) { a = __fadd_rn(a, rg[w][threadIdx.x]); b2 = __fadd_rn(b2, rb[w][threadIdx.x]); }
     if (t.row_chunks == 1) {
-      t.a.grad[s.g_off + cc] = a;
-      t.a.grad[s.beta_off + cc] = b2;
+      t.a.grad[s.g_off + cc] = d.accum ? __fadd_rn(t.a.grad[s.g_off + cc], a) : a;
+      t.a.grad[s.beta_off + cc] = d.accum ? __fadd_rn(t.a.grad[s.beta_off + cc], b2) : b2;
     } else {
       float* part = ws_at<float>(t, t.colred_off) + ((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim);
       part[cc] = a;
@@ -812,8 +812,8 @@ __global__ void __launch_bounds__(256) ln_param_finish_kernel(TickArgs t) {
     a = __fadd_rn(a, part[(uint64_t)k * 2 * t.max_dim + c]);
     b2 = __fadd_rn(b2, part[(uint64_t)k * 2 * t.max_dim + t.max_dim + c]);
   }
-  t.a.grad[s.g_off + c] = a;
-  t.a.grad[s.beta_off + c] = b2;
+  t.a.grad[s.g_off + c] = d.accum ? __fadd_rn(t.a.grad[s.g_off + c], a) : a;
+  t.a.grad[s.beta_off + c] = d.accum ? __fadd_rn(t.a.grad[s.beta_off + c], b2) : b2;
 }
 
 // Fused LayerNorm backward (widths that are multiples of 8, at most WPR*NP*256): one pass over du, x and the skip
@@ -989,8 +989,8 @@ __global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
     float ga = 0.f, gb = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) { ga = __fadd_rn(ga, red[0][w][lane]); gb = __fadd_rn(gb, red[1][w][lane]); }
-    t.a.grad[s.g_off + c] = ga;
-    t.a.grad[s.beta_off + c] = gb;
+    t.a.grad[s.g_off + c] = d.accum ? __fadd_rn(t.a.grad[s.g_off + c], ga) : ga;
+    t.a.grad[s.beta_off + c] = d.accum ? __fadd_rn(t.a.grad[s.beta_off + c], gb) : gb;
   }
 }
 
@@ -1179,7 +1179,8 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
       float a = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) a = __fadd_rn(a, part[w][c]);
-      t.a.grad[s.tab_off + (uint64_t)((rr << nb_shift) + blk) * dm + blockIdx.z * kEmbCols + c] = a;
+      float* gp = t.a.grad + s.tab_off + (uint64_t)((rr << nb_shift) + blk) * dm + blockIdx.z * kEmbCols + c;
+      *gp = d.accum ? __fadd_rn(*gp, a) : a;
     }
     __syncthreads();
   }
@@ -1194,8 +1195,12 @@ __global__ void __launch_bounds__(256) embed_bwd_kernel(TickArgs t) {
     if (cnt > 0) embed_gather<AT, CPL>(sub + row_start[rr], 0, cnt, du, gs, dm, col_ld, sc, acc);
     if (col_ok) {
 #pragma unroll
-      for (int e = 0; e < CPL; e += 4)
-        *reinterpret_cast<float4*>(t.a.grad + s.tab_off + (uint64_t)v * dm + col + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+      for (int e = 0; e < CPL; e += 4) {
+        float4* gp = reinterpret_cast<float4*>(t.a.grad + s.tab_off + (uint64_t)v * dm + col + e);
+        float4 o = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+        if (d.accum) { const float4 q = *gp; o = make_float4(__fadd_rn(q.x, o.x), __fadd_rn(q.y, o.y), __fadd_rn(q.z, o.z), __fadd_rn(q.w, o.w)); }
+        *gp = o;
+      }
     }
   }
 }

@@ -4,7 +4,7 @@ import numpy as np
 import pm_inputs as I
 
 
-def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major"):
+def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
@@ -13,7 +13,7 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
     """
     import torch
     import paper_1910_05124_b200 as pm
-    pipe = pm.Pipeline(wl, params0, loop_order=loop_order)
+    pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
@@ -51,7 +51,7 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
                     book.setdefault((f_mb, p + 1), [None, None])[0] = f_ver
                 if b_mb >= 0:
                     book.setdefault((b_mb, p + 1), [None, None])[1] = b_ver
-                    assert n_upd == b_ver + 1
+                    assert n_upd == b_ver + (1 if (b_mb + 1) % n_micro == 0 else 0)      # the update follows the N-th microbatch
     losses = pipe.pm_get_losses(0, n_steps)
     return pipe, losses, book
 
@@ -60,14 +60,14 @@ def is_encdec(wl):
     return any(sp.pre == "embed_dec" for sp in wl.stage_specs)
 
 
-def run_oracle(wl, params0, n_steps, teacher=None, warmup=0):
+def run_oracle(wl, params0, n_steps, teacher=None, warmup=0, n_micro=1):
     if wl.kind == "encoder":
         from oracle import transformer
         data = (lambda t: I.seq2seq_batch(wl, t)) if is_encdec(wl) else (lambda t: I.token_batch(wl, t))
-        return transformer.run_workload(wl, params0, data, n_steps=n_steps, warmup=warmup)
+        return transformer.run_workload(wl, params0, data, n_steps=n_steps, warmup=warmup, n_micro=n_micro)
     from oracle.mlp import run_workload
     teacher = I.teacher_params(wl) if teacher is None else teacher
-    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps, warmup=warmup)
+    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps, warmup=warmup, n_micro=n_micro)
 
 
 def max_rel_err(a, b):
@@ -77,11 +77,14 @@ def max_rel_err(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
 
 
-def compare_params(pipe, res, tol, per_stage=False):
+def compare_params(pipe, res, tol, per_stage=False, bias_per_stage=False, report=None):
     """per_stage: measure max |dw| against the largest weight of the whole stage vector (w_t)_i instead of the
     tensor's own largest entry.  Used for bf16 + Adam, where the step of an element is about alpha whatever the
     size of its gradient: an element whose gradient sign is decided by bf16 rounding noise moves by +-alpha per
-    step on either side, which is large against a bias vector that is itself only a few alpha in size."""
+    step on either side, which is large against a bias vector that is itself only a few alpha in size.
+    bias_per_stage: the stage norm for bias vectors only (Linear and LayerNorm biases: the tensors that are a few alpha
+    in size); weight matrices, embedding tables and LayerNorm gains are held to their own largest entry.
+    report: optional dict that receives the worst per-tensor and per-stage-vector errors, whichever is asserted."""
     worst = 0.0
     got = pipe.unpack(pipe.w)
     if pipe.is_encoder:
@@ -105,10 +108,19 @@ def compare_params(pipe, res, tol, per_stage=False):
                     bound = wl.alpha * len(res.losses) * 1.01 + 1e-12
                     assert np.abs(a[:d]).max() <= bound and np.abs(ref[:d]).max() <= bound
                     a, ref = a[d:], ref[d:]
-                scale = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p]) if per_stage else None
-                e = max_rel_err(a, ref) if scale is None else float(np.abs(a - ref).max() / scale)
+                stage_scale = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p])
+                e_tensor, e_stage = max_rel_err(a, ref), float(np.abs(a - ref).max() / stage_scale)
+                n_t = len(stage)
+                is_bias = j == n_t - 1 or (sp.pre == "ln" and j == 1)          # Linear bias (last tensor), LayerNorm bias
+                use_stage = per_stage or (bias_per_stage and is_bias)
+                e = e_stage if use_stage else e_tensor
+                if report is not None:
+                    report["per_tensor"] = max(report.get("per_tensor", 0.0), e_tensor)
+                    report["per_stage_vector"] = max(report.get("per_stage_vector", 0.0), e_stage)
+                    if not is_bias:
+                        report["per_tensor_without_biases"] = max(report.get("per_tensor_without_biases", 0.0), e_tensor)
                 worst = max(worst, e)
-                assert e <= tol, f"stage {p} tensor {j}: {e}"
+                assert e <= tol, f"stage {p} tensor {j}: {e} (per tensor {e_tensor}, per stage vector {e_stage})"
         return worst
     for p, stage in enumerate(got):
         for j, (W, b) in enumerate(stage):
@@ -118,5 +130,61 @@ def compare_params(pipe, res, tol, per_stage=False):
             ref_b = res.params[p][2 * j + 1]
             if np.abs(ref_b).max() > 0:
                 eb = max_rel_err(b, ref_b)
-                assert eb <= tol * 4, f"stage {p} b{j}: {eb}"
+                worst = max(worst, eb)
+                assert eb <= tol, f"stage {p} b{j}: {eb}"
+    return worst
+
+
+def adam_tensor_stats(a, ref, alpha, n_updates, tol=2e-2):
+    """Error measures of one tensor under bf16 + Adam.  Adam's step of an element is about alpha whatever the size of
+    its gradient, so an element whose gradient is rounding noise walks +-alpha per update on either side and the
+    max-norm of the difference is bounded by 2 alpha n_updates, not by the operand precision; what the operand
+    precision does bound is the bulk of the elements.  Returns (relative L2 error, fraction of elements beyond
+    tol * max|ref|, max |difference| / (2 alpha n_updates))."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    ref = np.asarray(ref, dtype=np.float64).ravel()
+    d = np.abs(a - ref)
+    l2 = float(np.sqrt((d * d).sum()) / max(np.sqrt((ref * ref).sum()), 1e-30))
+    frac = float((d > tol * max(np.abs(ref).max(), 1e-30)).mean())
+    return l2, frac, float(d.max() / (2.0 * alpha * n_updates))
+
+
+def compare_params_adam(pipe, res, n_updates, tol=2e-2, max_frac=0.01, report=None):
+    """bf16 + Adam over many updates, per tensor: relative L2 error <= tol; at most max_frac of the elements further
+    than tol * max|w| from the oracle; no element further than the two-sided Adam walk 2 alpha n_updates.
+    Bias vectors (Linear and LayerNorm biases), which are themselves only a few alpha in size, are measured against
+    the largest entry of their stage vector (w_t)_i instead of their own, and their L2 error against the stage's.
+    The key-bias gauge direction of attention stages is bounded by alpha n_updates as in compare_params."""
+    wl = pipe.wl
+    got = pipe.unpack(pipe.w)
+    worst = {"l2": 0.0, "frac_beyond_tol": 0.0, "max_over_adam_walk": 0.0}
+    bad = []
+    for p, stage in enumerate(got):
+        sp = wl.stage_specs[p]
+        stage_max = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p])
+        stage_l2 = np.sqrt(sum(float((np.asarray(t_, dtype=np.float64) ** 2).sum()) for t_ in res.params[p]))
+        for j, a in enumerate(stage):
+            ref = np.asarray(res.params[p][j], dtype=np.float64)
+            a = np.asarray(a, dtype=np.float64)
+            is_bias = j == len(stage) - 1 or (sp.pre == "ln" and j == 1)
+            if sp.post in ("attention", "cross_attention") and j == len(stage) - 1:
+                d = sp.n_out // (3 if sp.post == "attention" else 2)
+                lo = d if sp.post == "attention" else 0
+                bound = wl.alpha * n_updates * 1.01 + 1e-12
+                assert np.abs(a[lo:lo + d]).max() <= bound and np.abs(ref[lo:lo + d]).max() <= bound
+                keep = np.r_[0:lo, lo + d:a.shape[0]]
+                a, ref = a[keep], ref[keep]
+            diff = np.abs(a - ref).ravel()
+            walk = float(diff.max() / (2.0 * wl.alpha * n_updates))
+            scale = stage_max if is_bias else max(np.abs(ref).max(), 1e-30)
+            l2 = float(np.sqrt((diff * diff).sum()) / (stage_l2 if is_bias else max(np.sqrt((ref * ref).sum()), 1e-30)))
+            frac = float((diff > tol * scale).mean())
+            worst["l2"] = max(worst["l2"], l2)
+            worst["frac_beyond_tol"] = max(worst["frac_beyond_tol"], frac)
+            worst["max_over_adam_walk"] = max(worst["max_over_adam_walk"], walk)
+            if l2 > tol or frac > max_frac or walk > 1.0:
+                bad.append(f"stage {p} tensor {j}{' (bias)' if is_bias else ''}: L2 {l2:.3g}, beyond tol {frac:.3g}, of the Adam walk {walk:.3g}")
+    if report is not None:
+        report.update(worst)
+    assert not bad, "; ".join(bad)
     return worst

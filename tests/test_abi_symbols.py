@@ -182,3 +182,52 @@ def test_encoder_decoder_layout_and_its_checks(built_lib):
     assert st == b"PM_ERR_UNSUPPORTED" and b"RESIDUAL" in msg
     st, msg = query(small, drop_flag(dec0 + 3, B.PM_OP_LAYERNORM, B.PM_OPF_FROM_MEMORY))[:2]
     assert st == b"PM_ERR_UNSUPPORTED" and b"CROSS_ATTENTION" in msg
+
+
+def test_microbatch_major_footprint_of_config5(built_lib):
+    """The queue of weight versions: (tau_i + 1) bf16 copies of every stage's slice plus fp32 copies of its biases and
+    LayerNorm parameters, and activations of one microbatch.  Config 5 as configured then fits one 180 GB GPU, which
+    its tick-major rings (more than 400 GB) do not."""
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    wl = I.cfg5()
+    cfg, sd, keep = _describe(wl)
+    cfg.loop_order = B.PM_MB_MAJOR
+    sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    P = wl.n_stages
+    queue = sum((wl.tau_fwd[p] + 1) * sd[p].param_count * 2 for p in range(P))     # the bf16 slices alone
+    assert queue < rb.value < queue + 8e9                        # plus fp32 small tensors and one microbatch of activations
+    assert 125e9 < rb.value < 140e9 and sb.value + rb.value + wb.value < 170e9
+    # any forward delays are accepted in this order, a backward delay is not
+    sd[3].tau_fwd = 0
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    sd[3].tau_bkwd = 1
+    st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+    assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED"
+    cfg.loop_order = 7
+    assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
+
+
+def test_flat_update_argument_checks_need_no_gpu(built_lib):
+    """pm_update_flat / pm_update_flat_static reject an empty step-size table and slices that do not fit the arenas
+    (a sum offset + count that wraps included) before anything touches the device."""
+    import ctypes as C
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    fake = 4096                                                         # never dereferenced: every case fails first
+    ar = B.pm_arenas(fake, fake, fake, fake, fake, None, 1 << 20)
+    offs, cnts = (C.c_uint64 * 2)(0, 1024), (C.c_uint64 * 2)(1024, 1024)
+    tf, tb = (C.c_int32 * 2)(3, 1), (C.c_int32 * 2)(0, 0)
+    cfg, keep = B.make_config(n_stages=2, microbatch=1, compute="f32", optimizer="sgdm", alpha=0.01, alpha_by_step=[0.1, 0.2])
+    cfg.alpha_len = 0
+    st = L.pm_update_flat(C.byref(ar), offs, cnts, tf, tb, 2, C.byref(cfg), 0, C.c_void_p(fake), 1 << 20, None)
+    assert L.pm_status_string(st) == b"PM_ERR_INVALID_ARG" and b"alpha_len" in L.pm_last_error(None)
+    st = L.pm_update_flat_static(C.byref(ar), offs, cnts, tf, tb, 2, C.byref(cfg), 0, None)
+    assert L.pm_status_string(st) == b"PM_ERR_INVALID_ARG" and b"alpha_len" in L.pm_update_flat_static_last_error()
+    cfg.alpha_len = 2
+    cnts[1] = (1 << 64) - 512                                            # offset + count wraps around
+    st = L.pm_update_flat(C.byref(ar), offs, cnts, tf, tb, 2, C.byref(cfg), 0, C.c_void_p(fake), 1 << 20, None)
+    assert L.pm_status_string(st) == b"PM_ERR_NOMEM"

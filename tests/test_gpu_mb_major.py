@@ -174,3 +174,44 @@ def test_cfg5_full_depth_first_microbatches(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
     worst = compare_params(pipe, res, 2e-2, per_stage=True)
     print("cfg5 full depth worst relative weight error (per stage vector)", worst)
+
+
+# ---- N microbatches per update (Section 2.1; Table 1: tau_fwd,i = ceil((2(P-i)+1)/N) updates) ------------------------
+
+@pytest.mark.parametrize("N,compute,opt", [(2, "f32", "sgdm"), (4, "f32", "sgdm"), (2, "f32", "adam"), (2, "bf16", "sgdm"), (4, "bf16", "sgdm")])
+def test_n_microbatches_per_update_mlp(cuda_device, N, compute, opt):
+    f32 = compute == "f32"
+    P = 5
+    wl = I.mlp_workload("n_micro", P, 72 if f32 else 192, 2, "gelu", 33 if f32 else 40, compute=compute, optimizer=opt,
+                        alpha=0.02 if opt == "sgdm" else 1e-3, K=4, D=0.5, steps=6 * N + 1, seed=191005124 + 63)
+    wl.tau_fwd = I.pipemare_delays(P, N)[0]
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps, n_micro=N)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major", n_micro=N)
+    check_book(book, res, wl.steps, P)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    compare_params(pipe, res, (2e-5 if opt == "adam" else 1e-5) if f32 else 2e-2)     # six updates applied, one microbatch pending
+
+
+@pytest.mark.parametrize("N", [2, 4])
+@pytest.mark.parametrize("compute", ["f32", "bf16"])
+def test_n_microbatches_per_update_encoder_decoder(cuda_device, N, compute):
+    """Every kind of parameter gradient accumulates: Linear weights (TMA reduce-add in the bf16 path) and biases,
+    LayerNorm gain and bias, both embedding tables."""
+    f32 = compute == "f32"
+    wl = I.cfg5_small(compute=compute, n_enc=1, n_dec=1, d_model=32 if f32 else 64, d_ff=64 if f32 else 128, seq_len=8 if f32 else 16,
+                      batch=2, vocab=40 if f32 else 96, steps=5 * N)
+    wl.tau_fwd = I.pipemare_delays(wl.n_stages, N)[0]
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps, n_micro=N)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major", n_micro=N)
+    check_book(book, res, wl.steps, wl.n_stages)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    compare_params(pipe, res, 2e-5 if f32 else 2e-2, per_stage=not f32)
+
+
+def test_n_microbatches_needs_the_weight_queue_order(cuda_device):
+    import paper_1910_05124_b200 as pm
+    wl = I.mlp_workload("t", 2, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
+        pm.Pipeline(wl, I.init_stage_params(wl), n_micro=2)

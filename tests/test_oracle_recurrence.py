@@ -332,3 +332,68 @@ def test_t1_annealing_counts_from_the_switch():
     steps = -np.diff([0.0] + traj)
     want = [alpha if k < E else alpha / tau ** (1.0 - min((k - E) / K, 1.0)) for k in range(10)]
     np.testing.assert_allclose(steps, want, rtol=1e-12)
+
+
+# ---- N microbatches per update (Section 2.1, Table 1) -----------------------------------------------------------------
+
+def test_n_microbatches_without_delay_equal_one_synchronous_step_on_the_whole_minibatch():
+    """With every tau = 0, N microbatches of M rows whose gradients (each carrying 1/N) are accumulated and applied
+    at the minibatch boundary are one synchronous step on the N*M rows: the mean loss over the minibatch is the mean
+    of the microbatch means.  float64 state, so the two agree to rounding of the sum order."""
+    import pm_inputs as I
+    from oracle.mlp import run_workload
+    N, M = 3, 8
+    small = I.mlp_workload("n_micro", 3, 24, 2, "gelu", M, compute="f32", optimizer="sgdm", alpha=0.05, K=4, D=0.5, steps=4 * N, seed=123)
+    small.tau_fwd = [0, 0, 0]
+    big = I.mlp_workload("n_micro", 3, 24, 2, "gelu", N * M, compute="f32", optimizer="sgdm", alpha=0.05, K=4, D=0.5, steps=4, seed=123)
+    big.tau_fwd = [0, 0, 0]
+    params0 = I.init_stage_params(small)
+    teacher = I.teacher_params(small)
+    micro = lambda t: I.batch(small, t, teacher)
+
+    def mini(u):
+        xs, ys = zip(*[micro(u * N + j) for j in range(N)])
+        return np.concatenate(xs), np.concatenate(ys)
+    a = run_workload(small, params0, micro, n_steps=4 * N, dtype=np.float64, n_micro=N)
+    b = run_workload(big, params0, mini, n_steps=4, dtype=np.float64)
+    for sa, sb in zip(a.params, b.params):
+        for ta, tb in zip(sa, sb):
+            np.testing.assert_allclose(ta, tb, rtol=1e-11, atol=1e-14)
+    # the minibatch loss is the mean of its microbatch losses
+    np.testing.assert_allclose(np.array(a.losses).reshape(4, N).mean(1), np.array(b.losses), rtol=1e-12)
+    # and the weights change at minibatch boundaries only
+    seen = []
+    run_workload(small, params0, micro, n_steps=2 * N, dtype=np.float64, n_micro=N, on_step=lambda u, w: seen.append(u))
+    assert seen == [0, 1]
+
+
+def test_bookkeeping_with_two_microbatches_per_update_by_hand():
+    """P = 3, N = 2: Table 1 gives tau_fwd = ceil((2(P-i)+1)/N) = (3, 2, 1) updates.  Microbatches 2u and 2u+1 belong
+    to update u; both read forward version max(0, u - tau_i) and backward version u."""
+    import pm_inputs as I
+    from oracle.mlp import run_workload
+    wl = I.mlp_workload("book", 3, 8, 1, "relu", 4, compute="f32", steps=10, seed=3)
+    assert I.pipemare_delays(3, 2)[0] == [3, 2, 1]
+    wl.tau_fwd = I.pipemare_delays(3, 2)[0]
+    res = run_workload(wl, I.init_stage_params(wl), lambda t: I.batch(wl, t), n_steps=10, n_micro=2)
+    book = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    expect = {  # (microbatch, stage): (forward version, backward version)
+        (0, 1): (0, 0), (1, 1): (0, 0), (6, 1): (0, 3), (7, 1): (0, 3), (8, 1): (1, 4), (9, 1): (1, 4),
+        (4, 2): (0, 2), (5, 2): (0, 2), (6, 2): (1, 3), (9, 2): (2, 4),
+        (1, 3): (0, 0), (2, 3): (0, 1), (3, 3): (0, 1), (4, 3): (1, 2), (9, 3): (3, 4)}
+    for key, val in expect.items():
+        assert book[key] == val, key
+    assert len(res.losses) == 10
+
+
+def test_accumulation_happens_in_the_state_precision_in_microbatch_order():
+    """The N gradients are rounded to the state type one by one and added in order (what a gradient buffer does)."""
+    from oracle import recurrence
+    g = [np.array([1.0]), np.array([2.0 ** -24]), np.array([2.0 ** -24])]       # the small ones vanish against 1 in fp32
+    hp = dict(optimizer="sgdm", alpha=1.0, beta1=0.0, beta2=0.0, eps=0.0, t1=False, K=1, t2=False, D=0.5)
+    res = recurrence.run([[np.array([0.0])]], [0], [0], lambda t, uf, ub, loss_scale=1.0: (0.0, [[g[t]]]), 3, hp,
+                         dtype=np.float32, n_micro=3)
+    assert res.params[0][0][0] == np.float32(-1.0)                               # (1 + 2^-24) + 2^-24 = 1 in fp32, twice
+    res64 = recurrence.run([[np.array([0.0])]], [0], [0], lambda t, uf, ub, loss_scale=1.0: (0.0, [[g[t]]]), 3, hp,
+                           dtype=np.float64, n_micro=3)
+    assert res64.params[0][0][0] == -(1.0 + 2.0 ** -23)

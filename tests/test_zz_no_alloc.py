@@ -17,7 +17,7 @@ import pm_inputs as I
 pytestmark = pytest.mark.gpu
 
 
-def run_two_calls(case, optimizer, static):
+def run_two_calls(case, optimizer, static, stream=None, check_no_alloc=False):
     import torch
     import paper_1910_05124_b200 as pm
     dev = torch.device("cuda:0")
@@ -28,8 +28,29 @@ def run_two_calls(case, optimizer, static):
                        alpha=0.01 if optimizer == "sgdm" else 5e-4, K=32, D=0.5)
     call = fu.pm_update_flat_static if static else fu.pm_update_flat
     snaps = []
+    if static and check_no_alloc:
+        call(t["w"], t["m"], s, t["delta"], t["g"], lp, 8)          # the first call on a device looks up the array's address
+        torch.cuda.synchronize()
+        fu2 = pm.FlatUpdate(case["offsets"], case["counts"], case["tau_fwd"], case["tau_bkwd"], optimizer=optimizer,
+                            alpha=0.01 if optimizer == "sgdm" else 5e-4, K=32, D=0.5)
+        t2 = {n: torch.from_numpy(case[n]).to(dev) for n in ("w", "m", "delta", "g")}
+        t = t2                                                       # fresh state, so that the results still compare
+        s = torch.from_numpy(case["s"]).to(dev) if optimizer == "adam" else None
+        lp = torch.zeros(case["total"], dtype=torch.bfloat16, device=dev)
+        call = fu2.pm_update_flat_static
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info(dev)[0]                      # the driver's own count of free device memory
+        reserved0 = torch.cuda.memory_reserved(dev)
     for k in (9, 10):
-        call(t["w"], t["m"], s, t["delta"], t["g"], lp, k)
+        if stream is not None:
+            stream.wait_stream(torch.cuda.current_stream(dev))
+            call(t["w"], t["m"], s, t["delta"], t["g"], lp, k, stream=stream)
+            stream.synchronize()
+        else:
+            call(t["w"], t["m"], s, t["delta"], t["g"], lp, k)
+        if static and check_no_alloc:
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info(dev)[0] == free0 and torch.cuda.memory_reserved(dev) == reserved0
         torch.cuda.synchronize()
         snap = {n: t[n].cpu().numpy().copy() for n in ("w", "m", "delta")}
         if s is not None:
@@ -75,3 +96,17 @@ def test_static_variant_rejects_more_stages_than_it_holds(cuda_device):
         fu.pm_update_flat_static(t["w"], t["m"], None, t["delta"], t["g"], None, 0)
     torch.cuda.synchronize()
     assert torch.equal(before, t["w"])
+
+
+def test_static_variant_allocates_nothing_and_takes_any_stream(cuda_device):
+    """Adam at the 256-stage limit, on a stream of the caller's: the driver reports the same free device memory
+    before and after each call (and torch's pool has not grown), and the bits equal the workspace variant's."""
+    import torch
+    case = I.update_sweep_case(260000, 256, "adam")
+    ref = run_two_calls(case, "adam", static=False)
+    side = torch.cuda.Stream()
+    got = run_two_calls(case, "adam", static=True, stream=side, check_no_alloc=True)
+    for call in range(2):
+        for name in ref[call]:
+            np.testing.assert_array_equal(got[call][name].view(np.uint32), ref[call][name].view(np.uint32),
+                                          err_msg=f"call {call} {name}")
