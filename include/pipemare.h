@@ -149,6 +149,13 @@ typedef struct {
   int64_t alpha_len;
   int64_t loss_log_capacity;     /* losses kept on the device (a ring); 0 = default 4096 */
   int32_t loop_order;            /* PM_TICK_MAJOR | PM_MB_MAJOR (see the top of this file) */
+  int32_t entry_period;          /* E, PM_TICK_MAJOR only; 0 or 1: a microbatch enters at every tick.  E > 1: one enters every
+                                    E ticks (pm_forward takes inputs at ticks 0, E, 2E, ... and NULL between, PM_ERR_STATE
+                                    otherwise), so a stage holds floor(tau_fwd / E) + 1 microbatches' activations instead of
+                                    tau_fwd + 1, and reads the weight version Table 1's delay names, max(0, a - tau_fwd), from a
+                                    queue of tau_fwd + 1 versions as in PM_MB_MAJOR: the recurrence is unchanged, only the
+                                    schedule on the GPU is sparser (activation memory / E, weight queues added).  N microbatches
+                                    need (N - 1) E + 2P ticks.  Not combined with pm_set_warmup. */
   int32_t n_micro;               /* N of Section 2.1: microbatches per update; 0 or 1 = one.  N > 1 needs PM_MB_MAJOR
                                     (else PM_ERR_UNSUPPORTED): calls t = 0, 1, ... of pm_step belong to update u = t / N;
                                     tau_fwd counts updates (Table 1: ceil((2(P-i)+1)/N)), every microbatch of a minibatch

@@ -109,13 +109,14 @@ struct HyperDev {
   int32_t mb_major;           // microbatch-major order: one microbatch in flight, forward weights from the version rings
   int32_t lp_elem;            // bytes of an element of the version rings' operand copy (2 or 4)
   int32_t n_micro;            // N: microbatches per update (microbatch-major order; 1 elsewhere)
-  int32_t _pad;
+  int32_t entry_period;       // tick-major order: a microbatch enters every entry_period ticks (1: every tick)
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks
 // (the pipeline holds one microbatch at a time, which is synchronous training), afterwards one per tick.
-__host__ __device__ inline int64_t mb_at_tick(int64_t a, int64_t warm, int64_t period) {
+__host__ __device__ inline int64_t mb_at_tick(int64_t a, int64_t warm, int64_t period, int64_t entry_period = 1) {
   if (a < 0) return -1;
+  if (entry_period > 1) return (a % entry_period == 0) ? a / entry_period : -1;   // a sparser pipeline: one microbatch every E ticks
   const int64_t t0 = warm * period;
   if (a < t0) return (a % period == 0) ? a / period : -1;
   return warm + (a - t0);

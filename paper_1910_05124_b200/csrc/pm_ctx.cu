@@ -44,6 +44,8 @@ struct Layout {
   int32_t max_lin = 0, max_dim = 0, n_in_first = 0, n_out_last = 0;
   // microbatch-major order
   bool mb = false;
+  bool queue = false;                   // the forward pass reads its weights from per-stage version queues (mb, or entry period > 1)
+  int32_t E = 1;                        // tick-major order: ticks between two entering microbatches
   int32_t n_tables = 1;                 // per-tick tables: 1, or 2P + 1 (one per sub-tick and one for the grouped launches)
   std::vector<SmallSeg> segs;           // fp32 tensors the forward pass reads, per version ring slot (bf16 operands)
   uint64_t off_segs = 0;
@@ -82,6 +84,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     return PM_ERR_UNSUPPORTED;
   }
   L.mb = mb;
+  if (cfg->entry_period < 0 || cfg->entry_period > 2 * P) { err = "entry_period must be in [0, 2 * n_stages]"; return PM_ERR_INVALID_ARG; }
+  const int E = (!mb && cfg->entry_period > 1) ? cfg->entry_period : 1;
+  const bool queue = mb || E > 1;
+  L.E = E; L.queue = queue;
   L.n_tables = mb ? 2 * P + 1 : 1;
   const uint64_t esz = cfg->compute_dtype == PM_F32 ? 4 : 2;
   const uint64_t T = (uint64_t)cfg->microbatch;
@@ -120,6 +126,13 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     // the delay is the queue of weight versions
     s.vdepth = 1;
     if (mb) { s.depth = 1; s.xdepth = 1; s.vdepth = s.tau_f + 1; }
+    if (E > 1) {
+      // a microbatch every E ticks: a stash written at tick mE + i is read at tick mE + i + tau, so floor(tau / E) + 1
+      // microbatches are alive in a stage; the input ring keeps one more (it is also the forward mailbox) and another
+      // when the previous stage takes its ReLU mask from it a tick after this stage's backward
+      const int extra = s.xdepth - (s.tau_f + 1);
+      s.depth = s.tau_f / E + 1; s.xdepth = s.depth + extra; s.vdepth = s.tau_f + 1;
+    }
     s.begin = sd.param_offset; s.end = sd.param_offset + sd.param_count;
     prev_end = s.end;
     L.begin64[p] = (uint32_t)(s.begin / 64); L.end64[p] = (uint32_t)(s.end / 64);
@@ -134,7 +147,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (second && !L.st[p - 1].emit_memory) { stage_err(p, "a second-stream EMBED must follow the stage that emits the memory"); return PM_ERR_UNSUPPORTED; }
       if (L.pe_seq > 0 && (L.pe_seq != op.seq_len || L.pe_d != op.n_out)) { stage_err(p, "all EMBED ops share seq_len and width"); return PM_ERR_UNSUPPORTED; }
       s.ids_stream = second ? 1 : 0;
-      s.ids_depth = mb ? 1 : 2 * P - p;
+      s.ids_depth = mb ? 1 : (E > 1 ? (2 * P - p) / E + 2 : 2 * P - p);
       if (second) L.n_streams = 2;
       if (op.n_in < 1 || op.n_out < 4 || (op.n_out & 3) || op.seq_len < 1 || T % op.seq_len) { stage_err(p, "bad EMBED description (width a multiple of four, seq_len dividing the microbatch)"); return PM_ERR_INVALID_ARG; }
       s.pre = PRE_EMBED; s.vocab = op.n_in; s.seq_len = op.seq_len;
@@ -245,7 +258,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (s.lin[l].flags & LF_WRITE_Z) { s.lin[l].z_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
       if (l < s.n_lin - 1) { s.lin[l].h_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.lin[l].n_out * esz, 256); }
     }
-    if (mb) {
+    if (queue) {
       // queue of weight versions: the whole slice in the operand type, and (bf16 operands) the fp32 tensors the forward
       // pass reads -- LayerNorm gain and bias, Linear biases -- packed into slots of small_count floats
       s.v_ring = ring; ring = align_up(ring + (uint64_t)s.vdepth * (s.end - s.begin) * esz, 256);
@@ -292,8 +305,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   if (L.mem_stage >= 0) {
     if (L.last_mem_reader < 0) { err = "a memory is emitted but no CROSS_ATTENTION stage reads it"; return PM_ERR_UNSUPPORTED; }
     L.st[L.last_mem_reader].mem_first = 1;
-    L.mem_depth = mb ? 1 : 2 * P - 2 * L.mem_stage;
-    L.gmem_depth = mb ? 1 : P - L.mem_stage + 2;
+    L.mem_depth = mb ? 1 : (E > 1 ? (2 * P - 2 * L.mem_stage) / E + 2 : 2 * P - 2 * L.mem_stage);
+    L.gmem_depth = mb ? 1 : (E > 1 ? (P - L.mem_stage + 2) / E + 2 : P - L.mem_stage + 2);
     for (int p = 0; p < P; ++p) L.sched[p].gmem_depth = L.gmem_depth;
     L.mem_ring = ring; ring = align_up(ring + (uint64_t)L.mem_depth * T * L.mem_dim * esz, 256);
   }
@@ -548,7 +561,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.alpha_len = cfg->alpha_len;
   c->hp.beta1 = cfg->beta1; c->hp.beta2 = cfg->beta2; c->hp.eps = cfg->eps;
   c->hp.warm = 0; c->hp.period = 2 * (int64_t)cfg->n_stages;
-  c->hp.mb_major = L.mb ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
+  c->hp.entry_period = L.E;
+  c->hp.mb_major = L.queue ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
   c->hp.n_micro = cfg->n_micro > 1 ? cfg->n_micro : 1;
 
   TickArgs& t = c->ta;
@@ -558,7 +572,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.n_in_first = L.n_in_first; t.n_out_last = L.n_out_last;
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
-  t.mb_major = L.mb ? 1 : 0; t.sel_p = -1;
+  t.mb_major = L.queue ? 1 : 0; t.sel_p = -1;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
   t.ln_li0 = 0; t.defer_finish = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
@@ -607,7 +621,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     pm_status us = umma_plan_create(&c->umma, t, c->L.st, c->ws + L.off_umma, c->stream, uerr);
     if (us != PM_OK) { delete c; return fail(nullptr, us, uerr); }
   }
-  if (L.mb) {
+  if (L.queue) {
     // version 0 of every stage's queue: the initial weights in the operand type, and the small fp32 tensors
     const bool f32 = cfg->compute_dtype == PM_F32;
     for (int p = 0; p < P && e == cudaSuccess; ++p) {
@@ -677,9 +691,9 @@ static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::functi
 
 // is a microbatch in flight at any of the stages whose distance from the entry tick lies in [lo, hi]?
 static bool any_stage_active(const pm_ctx* ctx, int64_t lo, int64_t hi) {
-  if (ctx->hp.warm == 0) return ctx->tick - lo >= 0 && ctx->tick - hi < ctx->n_fed;
+  if (ctx->hp.warm == 0 && ctx->hp.entry_period <= 1) return ctx->tick - lo >= 0 && ctx->tick - hi < ctx->n_fed;
   for (int64_t off = lo; off <= hi; ++off) {
-    const int64_t m = mb_at_tick(ctx->tick - off, ctx->hp.warm, ctx->hp.period);
+    const int64_t m = mb_at_tick(ctx->tick - off, ctx->hp.warm, ctx->hp.period, ctx->hp.entry_period);
     if (m >= 0 && m < ctx->n_fed) return true;
   }
   return false;
@@ -688,6 +702,7 @@ static bool any_stage_active(const pm_ctx* ctx, int64_t lo, int64_t hi) {
 pm_status pm_set_warmup(pm_ctx* ctx, int64_t n_microbatches) {
   if (!ctx || n_microbatches < 0) return fail(ctx, PM_ERR_INVALID_ARG, "bad argument");
   if (ctx->tick != 0 || ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "the warm-up length is set before the first tick");
+  if (ctx->hp.entry_period > 1 && n_microbatches > 0) return fail(ctx, PM_ERR_UNSUPPORTED, "warm-up epochs are not combined with an entry period");
   if (ctx->hp.n_micro > 1 && n_microbatches > 0) return fail(ctx, PM_ERR_UNSUPPORTED, "warm-up epochs are built for one microbatch per update");
   ctx->hp.warm = n_microbatches;
   return PM_OK;
@@ -840,8 +855,9 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (ctx->L.mb) return mb_forward(ctx, inputs, targets);
   if ((inputs == nullptr) != (targets == nullptr)) return fail(ctx, PM_ERR_INVALID_ARG, "inputs and targets must both be given or both be NULL");
   if (inputs && ctx->draining) return fail(ctx, PM_ERR_STATE, "microbatches must be fed on consecutive ticks; the pipeline is already draining");
-  const int64_t mb = mb_at_tick(ctx->tick, ctx->hp.warm, ctx->hp.period);   // the microbatch that may enter now, or -1
-  if (inputs && mb < 0) return fail(ctx, PM_ERR_STATE, "during the synchronous warm-up a microbatch enters every 2 * n_stages ticks; this tick takes none");
+  const int64_t mb = mb_at_tick(ctx->tick, ctx->hp.warm, ctx->hp.period, ctx->hp.entry_period);   // the microbatch that may enter now, or -1
+  if (inputs && mb < 0) return fail(ctx, PM_ERR_STATE, ctx->hp.entry_period > 1 ? "a microbatch enters every entry_period ticks; this tick takes none"
+                                                                               : "during the synchronous warm-up a microbatch enters every 2 * n_stages ticks; this tick takes none");
   const int dt = ctx->cfg.compute_dtype;
   pm_status s;
   if (inputs) ctx->n_fed = mb + 1; else if (mb >= 0) ctx->draining = true;   // an empty tick between two warm-up microbatches ends nothing
@@ -921,8 +937,14 @@ pm_status pm_update(pm_ctx* ctx) {
       prof_begin(ctx, PM_PROF_UPDATE);
       cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
                                     (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
-                                    ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls);
-      return check(ctx, e, "update");
+                                    ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls,
+                                    ctx->L.queue ? (void*)ctx->ta.ring : nullptr, ctx->hp.lp_elem);
+      pm_status s = check(ctx, e, "update");
+      if (s != PM_OK || !ctx->L.queue || ctx->L.segs.empty()) return s;
+      prof_begin(ctx, PM_PROF_UPDATE);                                 // fp32 copies of the updated stages' small tensors into their queues
+      e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(),
+                            (const StageDyn*)(ctx->ws + ctx->L.off_dyn), -1, ctx->ls);
+      return check(ctx, e, "weight-version push");
     });
     if (s != PM_OK) return s;
   }
@@ -985,7 +1007,8 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
   const int P = ctx->cfg.n_stages;
   // a microbatch's loss is computed P ticks after it entered; ticks completed so far = ctx->tick
   const int64_t last = ctx->tick - P - 1, t0 = ctx->hp.warm * ctx->hp.period;   // latest entry tick whose loss exists
-  const int64_t entered = last < 0 ? 0 : (last < t0 ? last / ctx->hp.period + 1 : ctx->hp.warm + (last - t0) + 1);
+  const int64_t entered = last < 0 ? 0 : (ctx->hp.entry_period > 1 ? last / ctx->hp.entry_period + 1
+                                          : (last < t0 ? last / ctx->hp.period + 1 : ctx->hp.warm + (last - t0) + 1));
   const int64_t done = ctx->L.mb ? ctx->n_fed - (ctx->phase == 1 ? 1 : 0) : std::min<int64_t>(ctx->n_fed, entered);
   if (first_mb + n > done) return fail(ctx, PM_ERR_INVALID_ARG, "loss of a microbatch that has not finished was requested");
   if (done - first_mb > ctx->L.loss_cap) return fail(ctx, PM_ERR_INVALID_ARG, "requested losses have left the device log");

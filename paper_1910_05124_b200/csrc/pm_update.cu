@@ -89,11 +89,16 @@ __global__ void schedule_kernel(const StageSched* __restrict__ sched, const int6
   const int P = hp.n_stages;
   const int64_t ver = nupd[i];
   if (flat_k >= 0) { dyn[i] = make_dyn(s, hp, tick, -1, -1, flat_k, ver, ver, false); return; }
-  int64_t a = mb_at_tick(tick - i, hp.warm, hp.period);
-  int64_t b = mb_at_tick(tick - (2 * (int64_t)P - (i + 1)), hp.warm, hp.period);
+  int64_t a = mb_at_tick(tick - i, hp.warm, hp.period, hp.entry_period);
+  int64_t b = mb_at_tick(tick - (2 * (int64_t)P - (i + 1)), hp.warm, hp.period, hp.entry_period);
   if (!(a >= 0 && a < n_fed)) a = -1;
   if (!(b >= 0 && b < n_fed)) b = -1;
-  dyn[i] = make_dyn(s, hp, tick, a, b, b, ver, ver, true);
+  // One microbatch per tick: the weights a stage holds ARE version max(0, a - tau).  With a microbatch only every E
+  // ticks more updates have landed by the time a forward runs, and the forward takes the version Table 1's delay
+  // names from the stage's queue.
+  int64_t fver = ver;
+  if (hp.entry_period > 1 && a >= 0) { fver = a - s.tau_f; if (fver < 0) fver = 0; }
+  dyn[i] = make_dyn(s, hp, tick, a, b, b, ver, fver, true);
 }
 
 cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageDyn* dyn, HyperDev hp,
@@ -280,6 +285,7 @@ __global__ void __launch_bounds__(128) push_small_kernel(const float* __restrict
                                                          int n_segs, const StageDyn* __restrict__ dyn, int slot_override) {
   for (int sg = blockIdx.x; sg < n_segs; sg += gridDim.x) {
     const SmallSeg g = segs[sg];
+    if (slot_override < 0 && !dyn[g.stage].active_update) continue;          // the stage was not updated this tick
     const int slot = slot_override >= 0 ? slot_override : dyn[g.stage].u_vslot;
     float* dst = reinterpret_cast<float*>(ring + g.ring_off) + (uint64_t)slot * g.slot_stride;
     const float* src = w + g.arena_off;

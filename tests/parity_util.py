@@ -4,7 +4,7 @@ import numpy as np
 import pm_inputs as I
 
 
-def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1):
+def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1, entry_period=1):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
@@ -13,7 +13,7 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
     """
     import torch
     import paper_1910_05124_b200 as pm
-    pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro)
+    pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro, entry_period=entry_period)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
@@ -25,8 +25,15 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
         pipe.pm_set_warmup(warmup)
     t0 = 2 * P * warmup                                        # first tick of the one-per-tick phase
     mb_major = pipe.mb_major
-    for s in range(n_steps if mb_major else t0 + (n_steps - warmup) + 2 * P - 1):
-        mb = s if mb_major else ((s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0))
+    E = entry_period                                            # tick-major: a microbatch enters every E ticks
+    n_ticks = n_steps if mb_major else ((n_steps - 1) * E + 2 * P if E > 1 else t0 + (n_steps - warmup) + 2 * P - 1)
+    for s in range(n_ticks):
+        if mb_major:
+            mb = s
+        elif E > 1:
+            mb = s // E if s % E == 0 else -1
+        else:
+            mb = (s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0)
         if 0 <= mb < n_steps:
             if encoder and is_encdec(wl):
                 src, dec_in, tg = I.seq2seq_batch(wl, mb)              # two token streams: [source | decoder input]
