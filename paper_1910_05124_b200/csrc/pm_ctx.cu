@@ -367,7 +367,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_lnred = w; w = align_up(w + (uint64_t)L.n_ln * L.ln_chunks * 2 * L.max_ln_dim * 4, 256);
   L.off_tgt = w; w = align_up(w + (uint64_t)(P + 1) * T * (ce ? 4 : (uint64_t)L.n_out_last * 4), 256);
   L.off_yout = w; w = align_up(w + 2 * T * L.n_out_last * (ce ? 4 : esz), 256);
-  L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes((int)T, L.st) : 0), 256);
+  L.off_umma = w; w = align_up(w + (cfg->compute_dtype == PM_BF16 ? umma_workspace_bytes((int)T, L.st, 0) : 0), 256);
   L.off_attn = w; w = align_up(w + (L.att_tc ? attn_workspace_bytes(P) : 0), 256);
   L.off_gmem = w; w = align_up(w + (uint64_t)L.gmem_depth * T * L.mem_dim * esz, 256);
   for (int p = 0; p < P; ++p) {
@@ -575,6 +575,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.mb_major = L.queue ? 1 : 0; t.sel_p = -1;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
   t.ln_li0 = 0; t.defer_finish = 0;
+  t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;

@@ -53,6 +53,8 @@ struct TickArgs {
   int32_t sel_p;
   int32_t act_first[PM_MAX_LINEARS];
   int32_t res_fused;      // the forward GEMM's epilogue adds the skip tensor (bf16 tensor-core path): no residual kernel
+  int32_t dgrad_split_below;   // CTA-pair dgrad: a Linear whose two-row-tile groups number fewer than this takes one row tile per
+                               // group (0: always two); launches of one stage need enough groups for the CTA pairs
   float loss_scale;       // factor on dL/dy: 1/N with N microbatches per update (the minibatch loss is their mean), else 1
   int32_t ln_li0;         // first entry of ln_ids a launch covers (its grid counts entries from there)
   int32_t defer_finish;   // launches of one stage leave the per-chunk partial sums of bias / LayerNorm gradients in place;

@@ -47,7 +47,7 @@ template <int MODE> struct Cfg {                           // MODE 0 forward, 2 
 };
 
 enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6,
-       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAP_W_F32H = 11, MAP_D_F32H = 12, MAPS_PER_LINEAR = 13 };
+       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAP_W_F32Q = 11, MAP_D_F32Q = 12, MAP_W_F32H = 13, MAP_D_F32H = 14, MAPS_PER_LINEAR = 15 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, operand majors as given.
 __device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
@@ -897,26 +897,37 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
 }
 
 // ---- dgrad on CTA pairs ------------------------------------------------------------------------------------
-// The same product and the same on-the-fly correction on tiles of 256 rows x 128 columns per CTA pair
-// (tcgen05.mma.cta_group::2, M = 256, N = 128).  Each CTA stages the fp32 w and delta of ITS 64 columns
-// (2 x 16 KB per k-block), converts them to bf16(w - gap*delta) in its own shared memory, and loads its 128
-// rows of dz; two 256-row tiles share one converted tile, so a CTA ingests 64 KB per 2 x (128x128x64) of its
-// own products, as the single-CTA kernel does, but the accumulators (2 x 128 columns) are double-buffered and
-// the eight epilogue warps drain one group while the next is computed.  Barriers: staging (sfull / sempty)
-// is local to a CTA; the converted tile (bfull) and the dz tiles (afull) are counted in the leader, which
-// issues the MMAs; tcgen05.commit releases slots (bempty, aempty) and publishes accumulators (tfull) in both
-// CTAs; the epilogue warps of both arrive on the leader's tempty.
-constexpr int DP_TILE_M = 256, DP_TILE_N = 128, DP_HALF_N = 64;
-constexpr int DP_MG = 2;                                   // 256-row tiles per converted tile
-constexpr int DP_NG = 2, DP_NB = 2, DP_NA = 7;             // fp32 staging ring, converted ring, dz ring (3.5 k-blocks of dz in flight)
-constexpr int DP_STG_HALF = TILE_K * DP_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
-constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;
-constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
-constexpr int DP_ACC_COLS = DP_MG * DP_TILE_N;             // 256 columns per accumulator buffer
+// The same product and the same on-the-fly correction on tiles of 256 rows x 256 columns per CTA pair
+// (tcgen05.mma.cta_group::2, M = 256, N = 256: the width at which the tensor pipe runs at its full rate; an MMA
+// costs at least ~84 cycles whatever its width, so 128-column tiles cap it at 77 %).  Each CTA stages the fp32 w
+// and delta of ITS 128 columns in slabs of 32 k-rows (2 x 16 KB per slab, three slabs in flight), converts them to
+// bf16(w - gap*delta) in its own shared memory, and loads its 128 rows of dz.  Up to two 256-row tiles share one
+// converted tile (then the two 256-column accumulators fill the tensor memory and the epilogue drains the first
+// while the MMAs of the second finish; the next group's MMAs start on an accumulator as soon as it is drained);
+// a Linear with few tiles takes one row tile per group and alternates between the two accumulators.
+// Barriers: staging (sfull / sempty) is local to a CTA; the converted tile (bfull) and the dz tiles (afull) are
+// counted in the leader, which issues the MMAs; tcgen05.commit releases slots (bempty, aempty) and publishes
+// accumulators (tfull) in both CTAs; the epilogue warps of both arrive on the leader's tempty.
+constexpr int DP_TILE_M = 256, DP_TILE_N = 256, DP_HALF_N = 128;
+constexpr int DP_MG = 2;                                   // 256-row tiles per converted tile (at most)
+constexpr int DP_SLAB_K = 32;                              // k-rows per fp32 staging slab
+constexpr int DP_NG = 3, DP_NB = 2, DP_NA = 4;             // fp32 slab ring, converted ring, dz ring (two k-blocks of dz in flight)
+constexpr int DP_STG_HALF = DP_SLAB_K * DP_HALF_N * 4;     // one fp32 [32 x 128] slab: 16 KB
+constexpr int DP_STG_BYTES = 2 * DP_STG_HALF;              // w slab + delta slab
+constexpr int DP_B_BYTES = TILE_K * DP_HALF_N * 2;         // converted [64 k x 128 n] bf16: 16 KB (two 64-column runs of 8 KB)
+constexpr int DP_ACC_COLS = DP_TILE_N;                     // 256 columns per accumulator; two fill the tensor memory
 constexpr int DP_XF_WARPS = 8, DP_EPI_WARPS = 8;
 constexpr int DP_THREADS = 32 * (3 + DP_XF_WARPS + DP_EPI_WARPS);   // staging producer, MMA issuer, transform, epilogue, dz producer
 constexpr int DP_TILE_BYTES = DP_NG * DP_STG_BYTES + DP_NB * DP_B_BYTES + DP_NA * A_BYTES + DP_EPI_WARPS * 4096;
 constexpr int DP_SMEM_BYTES = DP_TILE_BYTES + 1024 + 512;
+static_assert(DP_SMEM_BYTES <= 227 * 1024, "pair dgrad kernel: shared memory");
+
+// Row tiles per group for a Linear with these dimensions: two, unless that leaves fewer than `split_below` groups
+// (a launch that covers one stage only must still bring a tile group for most CTA pairs).
+__host__ __device__ inline int dgrad_pair_mg(int T, int n_in, int split_below) {
+  const int tiles_n = (n_in + DP_TILE_N - 1) / DP_TILE_N, tiles_m = (T + DP_TILE_M - 1) / DP_TILE_M;
+  return (((tiles_m + DP_MG - 1) / DP_MG) * tiles_n < split_below) ? 1 : DP_MG;
+}
 
 __device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
@@ -927,16 +938,27 @@ __device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int
   r.valid = lvl < s.n_lin && d.b_mb >= 0 && !(lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
   const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
   r.M = t.T; r.N = L.n_in; r.K = L.n_out;
+  const int mgr = dgrad_pair_mg(r.M, r.N, t.dgrad_split_below);
   const int tiles_n = (r.N + DP_TILE_N - 1) / DP_TILE_N;
   const int tiles_m = (r.M + DP_TILE_M - 1) / DP_TILE_M;
   const int local = tile - tile_start[lo];
   const int mg = local / tiles_n;
-  r.m0 = mg * DP_MG * DP_TILE_M;
+  r.m0 = mg * mgr * DP_TILE_M;
   r.n0 = (local % tiles_n) * DP_TILE_N;
-  r.n_m = min(DP_MG, tiles_m - mg * DP_MG);
+  r.n_m = min(mgr, tiles_m - mg * mgr);
   r.n_kb = (r.K + TILE_K - 1) / TILE_K;
   return r;
 }
+
+// Which accumulator (0 | 1: tensor-memory columns 0..255 | 256..511) a row tile of a group uses, and how often each
+// has been used so far (the barrier phases follow from the counts).  The MMA issuer and the epilogue warps walk the
+// same tile sequence and keep identical copies.
+struct DpAcc {
+  uint32_t uses[2];
+  int next1;                                                         // accumulator of the next single-row-tile group
+  __device__ __forceinline__ int buf(int mi, int n_m) const { return n_m == 2 ? mi : next1; }
+  __device__ __forceinline__ void done_group(int n_m) { if (n_m == 2) { ++uses[0]; ++uses[1]; } else { ++uses[next1]; next1 ^= 1; } }
+};
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(DP_THREADS, 1)
 umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
@@ -944,9 +966,9 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t stg = base;                                          // [DP_NG][w 16 KB | delta 16 KB]
-  const uint32_t sB = stg + DP_NG * DP_STG_BYTES;                     // [DP_NB][8 KB] converted operand (this CTA's 64 columns)
-  const uint32_t sA = sB + DP_NB * DP_B_BYTES;                        // [DP_NA][16 KB] dz tiles (this CTA's 128 rows)
+  const uint32_t stg = base;                                          // [DP_NG][w 16 KB | delta 16 KB] fp32 slabs of 32 k-rows x 128 columns
+  const uint32_t sB = stg + DP_NG * DP_STG_BYTES;                     // [DP_NB][16 KB] converted operand (this CTA's 128 columns, 64 k-rows)
+  const uint32_t sA = sB + DP_NB * DP_B_BYTES;                        // [DP_NA][16 KB] dz tiles (this CTA's 128 rows, 64 k-columns)
   const uint32_t sO = sA + DP_NA * A_BYTES;                           // [8][4 KB] epilogue staging
   uint8_t* stg_ptr = base_ptr;
   uint8_t* sB_ptr = base_ptr + DP_NG * DP_STG_BYTES;
@@ -963,7 +985,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < DP_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, DP_XF_WARPS); }
-    for (int i = 0; i < DP_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * DP_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < DP_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * 2 * DP_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }   // two slabs x two CTAs x eight warps
     for (int i = 0; i < DP_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 2 * DP_EPI_WARPS); }
     *abort_flag = 0;
@@ -980,9 +1002,8 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   const uint32_t tmem_base = *tmem_slot;
 
   // Two producer threads, each with its own cursor over the same (tile, k-block) sequence: warp 0 feeds the fp32
-  // staging ring (w, delta), the last warp the dz ring.  Their k-block loops are the critical path of the kernel
-  // (a handful of extra loads in them cost 3 %), so everything that is fixed for a tile is read once when the
-  // cursor reaches the tile and the loops hold nothing but barrier waits and copies.
+  // slab ring (w, delta), the last warp the dz ring.  Everything that is fixed for a tile is read once when the
+  // cursor reaches the tile; the loops hold nothing but barrier waits and copies.
   struct Cursor { int tile, kb; DgTile tl; bool done; const CUtensorMap* lm; bool corr; int dz_slot; };
   auto seek = [&](Cursor& c) {
     for (; c.tile < n_slots; c.tile += n_pairs) {
@@ -1004,19 +1025,23 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += n_pairs; seek(c); } };
 
   if (warp == 0) {
-    // ---------------- TMA producer of the fp32 staging ring (both CTAs) ----------------
+    // ---------------- TMA producer of the fp32 slab ring (both CTAs): two slabs of 32 k-rows per k-block ----------------
     if (lane == 0) {
       Cursor cs{pair, 0, DgTile{}, false, nullptr, false, 0};
       seek(cs);
       Ring sg{0, 0};
       int issued_sg = 0;
-      while (!cs.done) {
-        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) break;
-        const uint32_t sw = stg + sg.idx * DP_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
-        mbar_arrive_expect_tx(fb, cs.corr ? DP_STG_BYTES : DP_STG_HALF);
-        tma_load_2d(sw, cs.lm + MAP_W_F32H, fb, cs.tl.n0 + rank * DP_HALF_N, cs.kb * TILE_K);
-        if (cs.corr) tma_load_2d(sw + DP_STG_HALF, cs.lm + MAP_D_F32H, fb, cs.tl.n0 + rank * DP_HALF_N, cs.kb * TILE_K);
-        sg.advance(DP_NG); ++issued_sg;
+      bool ok = true;
+      while (!cs.done && ok) {
+        const int ncol = cs.tl.n0 + rank * DP_HALF_N;
+        for (int h = 0; h < TILE_K / DP_SLAB_K; ++h) {
+          if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) { ok = false; break; }
+          const uint32_t sw = stg + sg.idx * DP_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+          mbar_arrive_expect_tx(fb, cs.corr ? DP_STG_BYTES : DP_STG_HALF);
+          tma_load_2d(sw, cs.lm + MAP_W_F32Q, fb, ncol, cs.kb * TILE_K + h * DP_SLAB_K);
+          if (cs.corr) tma_load_2d(sw + DP_STG_HALF, cs.lm + MAP_D_F32Q, fb, ncol, cs.kb * TILE_K + h * DP_SLAB_K);
+          sg.advance(DP_NG); ++issued_sg;
+        }
         step(cs);
       }
       if (*abort_flag) {                                              // copies already issued still land here: wait (bounded)
@@ -1058,28 +1083,26 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
         }
       }
     }
-  } else if (warp == 1) {
+  }
+  else if (warp == 1) {
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = make_idesc_mn(DP_TILE_M, DP_TILE_N, 0, 1);
-      const uint64_t dba = desc_base(16, 1024), dbb = desc_base(DP_B_BYTES, 1024);   // B: one 64-column run per CTA
-      Ring br{0, 0}, ar{0, 0}, acc{0, 0};
+      const uint64_t dba = desc_base(16, 1024), dbb = desc_base(DP_B_BYTES / 2, 1024);   // B: two 64-column runs per CTA, 8 KB apart
+      Ring br{0, 0}, ar{0, 0};
+      DpAcc acc{{0u, 0u}, 0};
       bool ok = true;
       for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
         const int tile = order[slot];
         if (tile < 0) continue;
         const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
-        if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 43)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * DP_ACC_COLS);
-        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+        const int n_m = tl.n_m, n_kb = tl.n_kb;
+        for (int kb = 0; kb < n_kb && ok; ++kb) {
           if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 44)) { ok = false; break; }
           const uint32_t sb = sB + br.idx * DP_B_BYTES;
-          // both dz tiles first, then the products of the two row tiles interleaved: consecutive MMAs write
-          // different accumulators
           uint32_t sa[DP_MG], abar[DP_MG];
-          for (int mi = 0; mi < tl.n_m; ++mi) {
+          for (int mi = 0; mi < n_m; ++mi) {
             if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 45)) { ok = false; break; }
             sa[mi] = sA + ar.idx * A_BYTES;
             abar[mi] = bar_aempty + 8 * ar.idx;
@@ -1087,24 +1110,35 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
           }
           if (!ok) break;
           tc_fence_after();
+          // one row tile after the other: the first k-block of a group waits for each accumulator to be drained just
+          // before its first product, and the last k-block publishes the first accumulator while the products of
+          // the second are still running
+          for (int mi = 0; mi < n_m && ok; ++mi) {
+            const int b = acc.buf(mi, n_m);
+            if (kb == 0) {
+              if (!mbar_wait(bar_tempty + 8 * b, (acc.uses[b] & 1u) ^ 1u, abort_flag, status, 43)) { ok = false; break; }
+              tc_fence_after();
+            }
+            const uint32_t tmem_acc = tmem_base + (uint32_t)(b * DP_ACC_COLS);
 #pragma unroll
-          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
-            for (int mi = 0; mi < tl.n_m; ++mi)
-              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * DP_TILE_N), desc_at(dba, sa[mi] + k16 * 32), desc_at(dbb, sb + k16 * 2048),
-                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
-          for (int mi = 0; mi < tl.n_m; ++mi) tc_commit_pair(abar[mi], 3);
+            for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+              tc_mma_bf16_pair(tmem_acc, desc_at(dba, sa[mi] + k16 * 32), desc_at(dbb, sb + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            tc_commit_pair(abar[mi], 3);                              // this dz tile may be overwritten in both CTAs
+            if (kb == n_kb - 1) tc_commit_pair(bar_tfull + 8 * b, 3);  // accumulator complete, both CTAs
+          }
           if (ok) tc_commit_pair(bar_bempty + 8 * br.idx, 3);
           br.advance(DP_NB);
         }
-        if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);
-        acc.advance(2);
+        acc.done_group(n_m);
       }
     }
   } else if (warp < 2 + DP_XF_WARPS) {
-    // ---------------- operand transform (both CTAs): fp32 w, delta [64 k][64 n] -> bf16(w - gap*delta), MN-major ----------------
-    // thread: four consecutive columns (c4) of rows r0 + 16 j; reads are contiguous float4, stores 8 bytes into the swizzled atom
+    // ---------------- operand transform (both CTAs): fp32 w, delta [32 k][128 n] -> bf16(w - gap*delta), MN-major ----------------
+    // thread: four consecutive columns (c4) of rows rbase + 8 j; reads are contiguous float4, stores 8 bytes into the swizzled atom.
+    // Two slabs (k-rows 0..31 and 32..63) fill one converted tile.
     const int tt = threadIdx.x - 64;                                  // 0..255
-    const int c4 = tt & 15, rbase = tt >> 4;                          // 0..15, 0..15
+    const int c4 = tt & 31, rbase = tt >> 5;                          // 0..31 (four columns each), 0..7
+    const int run = c4 >> 4, cc = (c4 & 15);                          // 64-column run of the tile, position inside it (units of four columns)
     const uint32_t leader_bfull = mapa_shared(bar_bfull, 0);
     Ring br{0, 0}, sg{0, 0};
     bool ok = true;
@@ -1115,20 +1149,344 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       if (!tl.valid) continue;
       const float gapf = (float)t.st[tl.p].gap;
       const bool corr = t.dyn[tl.p].use_delta != 0;
+      for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+        for (int h = 0; h < TILE_K / DP_SLAB_K; ++h) {
+          bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 46);
+          if (h == 0) go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 47);
+          go = __all_sync(0xffffffffu, go);
+          if (!go) { ok = false; break; }
+          const uint8_t* src = stg_ptr + sg.idx * DP_STG_BYTES;
+          uint8_t* dst = sB_ptr + br.idx * DP_B_BYTES + run * (DP_B_BYTES / 2);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int rs = rbase + 8 * j;                             // row of the slab
+            const int r = h * DP_SLAB_K + rs;                         // k-row of the tile
+            const float4 w = *reinterpret_cast<const float4*>(src + rs * (DP_HALF_N * 4) + c4 * 16);
+            float v[4] = {w.x, w.y, w.z, w.w};
+            if (corr) {
+              const float4 dl = *reinterpret_cast<const float4*>(src + DP_STG_HALF + rs * (DP_HALF_N * 4) + c4 * 16);
+              v[0] = __fsub_rn(v[0], __fmul_rn(gapf, dl.x)); v[1] = __fsub_rn(v[1], __fmul_rn(gapf, dl.y));   // w - (tau_fwd - tau_bkwd) * delta
+              v[2] = __fsub_rn(v[2], __fmul_rn(gapf, dl.z)); v[3] = __fsub_rn(v[3], __fmul_rn(gapf, dl.w));
+            }
+            const uint32_t off = (uint32_t)(r >> 3) * 1024 + (uint32_t)(r & 7) * 128 + ((((uint32_t)cc >> 1) ^ (uint32_t)(r & 7)) << 4) + ((uint32_t)cc & 1) * 8;
+            *reinterpret_cast<uint2*>(dst + off) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive_cluster(leader_bfull + 8 * br.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
+          sg.advance(DP_NG);
+        }
+        br.advance(DP_NB);
+      }
+    }
+  }
+  else {
+    // ---------------- epilogue (both CTAs): 8 warps, warp%4 = TMEM lane group, two warps per group split the 256 columns ----------------
+    const int q = warp & 3;
+    const int ew = warp - 2 - DP_XF_WARPS;                            // 0..7
+    const int half = ew >> 2;                                         // 0: columns 0..127 of the tile, 1: columns 128..255
+    uint8_t* obuf = sO_ptr + ew * 4096;
+    const uint32_t obuf_s = sO + ew * 4096;
+    const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
+    const uint32_t leader_tempty = mapa_shared(bar_tempty, 0);
+    DpAcc acc{{0u, 0u}, 0};
+    bool ok = true, stored = false;
+    for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
+      const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const StageDyn& d = t.dyn[tl.p];
+      const StageDev& s = t.st[tl.p];
+      const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+      const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
+#pragma unroll 1
+      for (int mi = 0; mi < tl.n_m && ok; ++mi) {
+        const int b = acc.buf(mi, tl.n_m);
+        bool ready = mbar_wait(bar_tfull + 8 * b, acc.uses[b] & 1u, abort_flag, status, 48);
+        ready = __all_sync(0xffffffffu, ready);
+        if (!ready) { ok = false; break; }
+        tc_fence_after();
+        const int mrow = tl.m0 + mi * DP_TILE_M + rank * TILE_M + q * 32;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          const int nb = tl.n0 + half * 128 + c * 64;
+          uint32_t r0[32], r1[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * DP_ACC_COLS + half * 128 + c * 64);
+          tmem_ld32(taddr, r0);
+          tmem_ld32(taddr + 32, r1);
+          tmem_ld_wait();
+          if (c == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * b);   // this warp has read its part of this accumulator
+          }
+          if (mrow >= tl.M || nb >= tl.N) continue;
+          if (lane == 0 && stored) tma_store_wait_read();
+          __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+            *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
+                make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) { tma_store_3d(lm + MAP_DX_OUT, obuf_s, nb, mrow, dslot); tma_store_commit(); }
+          stored = true;
+        }
+      }
+      acc.done_group(tl.n_m);
+    }
+    if (lane == 0 && stored) tma_store_wait_all();
+  }
+  tc_fence_before();
+  cluster_sync_all();                                                 // no barrier or shared memory of a CTA is touched after this
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 2 * DP_ACC_COLS);
+  }
+}
+
+// ---- dgrad on CTA pairs, 128-column tiles ----------------------------------------------------------------------
+// Used where a launch covers ONE stage whose input is narrow (microbatch-major order): with 256-column tiles such a
+// Linear has too few tile groups for the CTA pairs, and a single row tile per group doubles the fp32 traffic per
+// FLOP beyond what L2 delivers.  Here a tile is half as wide, so twice as many groups exist.
+// The same product and the same on-the-fly correction on tiles of 256 rows x 128 columns per CTA pair
+// (tcgen05.mma.cta_group::2, M = 256, N = 128).  Each CTA stages the fp32 w and delta of ITS 64 columns
+// (2 x 16 KB per k-block), converts them to bf16(w - gap*delta) in its own shared memory, and loads its 128
+// rows of dz; two 256-row tiles share one converted tile, so a CTA ingests 64 KB per 2 x (128x128x64) of its
+// own products, as the single-CTA kernel does, but the accumulators (2 x 128 columns) are double-buffered and
+// the eight epilogue warps drain one group while the next is computed.  Barriers: staging (sfull / sempty)
+// is local to a CTA; the converted tile (bfull) and the dz tiles (afull) are counted in the leader, which
+// issues the MMAs; tcgen05.commit releases slots (bempty, aempty) and publishes accumulators (tfull) in both
+// CTAs; the epilogue warps of both arrive on the leader's tempty.
+constexpr int D1_TILE_M = 256, D1_TILE_N = 128, D1_HALF_N = 64;
+constexpr int D1_MG = 2;                                   // 256-row tiles per converted tile
+constexpr int D1_NG = 2, D1_NB = 2, D1_NA = 7;             // fp32 staging ring, converted ring, dz ring (3.5 k-blocks of dz in flight)
+constexpr int D1_STG_HALF = TILE_K * D1_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
+constexpr int D1_STG_BYTES = 2 * D1_STG_HALF;
+constexpr int D1_B_BYTES = TILE_K * D1_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
+constexpr int D1_ACC_COLS = D1_MG * D1_TILE_N;             // 256 columns per accumulator buffer
+constexpr int D1_XF_WARPS = 8, D1_EPI_WARPS = 8;
+constexpr int D1_THREADS = 32 * (3 + D1_XF_WARPS + D1_EPI_WARPS);   // staging producer, MMA issuer, transform, epilogue, dz producer
+constexpr int D1_TILE_BYTES = D1_NG * D1_STG_BYTES + D1_NB * D1_B_BYTES + D1_NA * A_BYTES + D1_EPI_WARPS * 4096;
+constexpr int D1_SMEM_BYTES = D1_TILE_BYTES + 1024 + 512;
+
+__device__ __forceinline__ DgTile decode_dgrad_pair128(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
+  DgTile r;
+  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  r.p = lo;
+  const StageDyn& d = t.dyn[lo];
+  const StageDev& s = t.st[lo];
+  r.valid = lvl < s.n_lin && d.b_mb >= 0 && !(lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
+  const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
+  r.M = t.T; r.N = L.n_in; r.K = L.n_out;
+  const int tiles_n = (r.N + D1_TILE_N - 1) / D1_TILE_N;
+  const int tiles_m = (r.M + D1_TILE_M - 1) / D1_TILE_M;
+  const int local = tile - tile_start[lo];
+  const int mg = local / tiles_n;
+  r.m0 = mg * D1_MG * D1_TILE_M;
+  r.n0 = (local % tiles_n) * D1_TILE_N;
+  r.n_m = min(D1_MG, tiles_m - mg * D1_MG);
+  r.n_kb = (r.K + TILE_K - 1) / TILE_K;
+  return r;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D1_THREADS, 1)
+umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t stg = base;                                          // [D1_NG][w 16 KB | delta 16 KB]
+  const uint32_t sB = stg + D1_NG * D1_STG_BYTES;                     // [D1_NB][8 KB] converted operand (this CTA's 64 columns)
+  const uint32_t sA = sB + D1_NB * D1_B_BYTES;                        // [D1_NA][16 KB] dz tiles (this CTA's 128 rows)
+  const uint32_t sO = sA + D1_NA * A_BYTES;                           // [8][4 KB] epilogue staging
+  uint8_t* stg_ptr = base_ptr;
+  uint8_t* sB_ptr = base_ptr + D1_NG * D1_STG_BYTES;
+  uint8_t* sO_ptr = sB_ptr + D1_NB * D1_B_BYTES + D1_NA * A_BYTES;
+  const uint32_t bars = base + D1_TILE_BYTES;
+  const uint32_t bar_sfull = bars, bar_sempty = bar_sfull + 8 * D1_NG, bar_bfull = bar_sempty + 8 * D1_NG,
+                 bar_bempty = bar_bfull + 8 * D1_NB, bar_afull = bar_bempty + 8 * D1_NB, bar_aempty = bar_afull + 8 * D1_NA,
+                 bar_tfull = bar_aempty + 8 * D1_NA, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + D1_TILE_BYTES + 8 * (2 * D1_NG + 2 * D1_NB + 2 * D1_NA + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();                            // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < D1_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, D1_XF_WARPS); }
+    for (int i = 0; i < D1_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * D1_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < D1_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 2 * D1_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc_pair(smem_u32(tmem_slot), 2 * D1_ACC_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // Two producer threads, each with its own cursor over the same (tile, k-block) sequence: warp 0 feeds the fp32
+  // staging ring (w, delta), the last warp the dz ring.  Their k-block loops are the critical path of the kernel
+  // (a handful of extra loads in them cost 3 %), so everything that is fixed for a tile is read once when the
+  // cursor reaches the tile and the loops hold nothing but barrier waits and copies.
+  struct Cursor { int tile, kb; DgTile tl; bool done; const CUtensorMap* lm; bool corr; int dz_slot; };
+  auto seek = [&](Cursor& c) {
+    for (; c.tile < n_slots; c.tile += n_pairs) {
+      const int tile = order[c.tile];
+      if (tile < 0) continue;
+      c.tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
+      if (c.tl.valid) {
+        const StageDyn& d = t.dyn[c.tl.p];
+        const StageDev& sd_ = t.st[c.tl.p];
+        c.lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
+        c.corr = d.use_delta != 0;
+        c.dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        c.kb = 0; c.done = false;
+        return;
+      }
+    }
+    c.done = true;
+  };
+  auto step = [&](Cursor& c) { if (++c.kb >= c.tl.n_kb) { c.tile += n_pairs; seek(c); } };
+
+  if (warp == 0) {
+    // ---------------- TMA producer of the fp32 staging ring (both CTAs) ----------------
+    if (lane == 0) {
+      Cursor cs{pair, 0, DgTile{}, false, nullptr, false, 0};
+      seek(cs);
+      Ring sg{0, 0};
+      int issued_sg = 0;
+      while (!cs.done) {
+        if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) break;
+        const uint32_t sw = stg + sg.idx * D1_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
+        mbar_arrive_expect_tx(fb, cs.corr ? D1_STG_BYTES : D1_STG_HALF);
+        tma_load_2d(sw, cs.lm + MAP_W_F32H, fb, cs.tl.n0 + rank * D1_HALF_N, cs.kb * TILE_K);
+        if (cs.corr) tma_load_2d(sw + D1_STG_HALF, cs.lm + MAP_D_F32H, fb, cs.tl.n0 + rank * D1_HALF_N, cs.kb * TILE_K);
+        sg.advance(D1_NG); ++issued_sg;
+        step(cs);
+      }
+      if (*abort_flag) {                                              // copies already issued still land here: wait (bounded)
+        for (int back = 1; back <= D1_NG && back <= issued_sg; ++back) {
+          const int it = issued_sg - back;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_sfull + 8 * (it % D1_NG), (uint32_t)(it / D1_NG) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 2 + D1_XF_WARPS + D1_EPI_WARPS) {
+    // ---------------- TMA producer of the dz ring (both CTAs) ----------------
+    if (lane == 0) {
+      Cursor ca{pair, 0, DgTile{}, false, nullptr, false, 0};
+      seek(ca);
+      Ring ar{0, 0};
+      int issued_a = 0;
+      bool ok = true;
+      while (!ca.done && ok) {
+        for (int mi = 0; mi < ca.tl.n_m; ++mi) {
+          if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 42)) { ok = false; break; }
+          if (rank == 0) mbar_arrive_expect_tx(bar_afull + 8 * ar.idx, 2 * A_BYTES);       // the rows of both CTAs
+          tma_load_3d_pair(sA + ar.idx * A_BYTES, ca.lm + MAP_DZ_K, mapa_shared(bar_afull + 8 * ar.idx, 0),
+                           ca.kb * TILE_K, ca.tl.m0 + mi * D1_TILE_M + rank * TILE_M, ca.dz_slot);
+          ar.advance(D1_NA); ++issued_a;
+        }
+        step(ca);
+      }
+      if (*abort_flag) {
+        if (rank == 0) {
+          for (int back = 1; back <= D1_NA && back <= issued_a; ++back) {
+            const int it = issued_a - back;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_afull + 8 * (it % D1_NA), (uint32_t)(it / D1_NA) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+          }
+        } else {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc_mn(D1_TILE_M, D1_TILE_N, 0, 1);
+      const uint64_t dba = desc_base(16, 1024), dbb = desc_base(D1_B_BYTES, 1024);   // B: one 64-column run per CTA
+      Ring br{0, 0}, ar{0, 0}, acc{0, 0};
+      bool ok = true;
+      for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+        const int tile = order[slot];
+        if (tile < 0) continue;
+        const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
+        if (!tl.valid) continue;
+        if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 43)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * D1_ACC_COLS);
+        for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
+          if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 44)) { ok = false; break; }
+          const uint32_t sb = sB + br.idx * D1_B_BYTES;
+          // both dz tiles first, then the products of the two row tiles interleaved: consecutive MMAs write
+          // different accumulators
+          uint32_t sa[D1_MG], abar[D1_MG];
+          for (int mi = 0; mi < tl.n_m; ++mi) {
+            if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 45)) { ok = false; break; }
+            sa[mi] = sA + ar.idx * A_BYTES;
+            abar[mi] = bar_aempty + 8 * ar.idx;
+            ar.advance(D1_NA);
+          }
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+            for (int mi = 0; mi < tl.n_m; ++mi)
+              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * D1_TILE_N), desc_at(dba, sa[mi] + k16 * 32), desc_at(dbb, sb + k16 * 2048),
+                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          for (int mi = 0; mi < tl.n_m; ++mi) tc_commit_pair(abar[mi], 3);
+          if (ok) tc_commit_pair(bar_bempty + 8 * br.idx, 3);
+          br.advance(D1_NB);
+        }
+        if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);
+        acc.advance(2);
+      }
+    }
+  } else if (warp < 2 + D1_XF_WARPS) {
+    // ---------------- operand transform (both CTAs): fp32 w, delta [64 k][64 n] -> bf16(w - gap*delta), MN-major ----------------
+    // thread: four consecutive columns (c4) of rows r0 + 16 j; reads are contiguous float4, stores 8 bytes into the swizzled atom
+    const int tt = threadIdx.x - 64;                                  // 0..255
+    const int c4 = tt & 15, rbase = tt >> 4;                          // 0..15, 0..15
+    const uint32_t leader_bfull = mapa_shared(bar_bfull, 0);
+    Ring br{0, 0}, sg{0, 0};
+    bool ok = true;
+    for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
+      const int tile = order[slot];
+      if (tile < 0) continue;
+      const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
+      if (!tl.valid) continue;
+      const float gapf = (float)t.st[tl.p].gap;
+      const bool corr = t.dyn[tl.p].use_delta != 0;
       for (int kb = 0; kb < tl.n_kb; ++kb) {
         bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 46);
         go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 47);
         go = __all_sync(0xffffffffu, go);
         if (!go) { ok = false; break; }
-        const uint8_t* src = stg_ptr + sg.idx * DP_STG_BYTES;
-        uint8_t* dst = sB_ptr + br.idx * DP_B_BYTES;
+        const uint8_t* src = stg_ptr + sg.idx * D1_STG_BYTES;
+        uint8_t* dst = sB_ptr + br.idx * D1_B_BYTES;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int r = rbase + 16 * j;                               // k-row
-          const float4 w = *reinterpret_cast<const float4*>(src + r * (DP_HALF_N * 4) + c4 * 16);
+          const float4 w = *reinterpret_cast<const float4*>(src + r * (D1_HALF_N * 4) + c4 * 16);
           float v[4] = {w.x, w.y, w.z, w.w};
           if (corr) {
-            const float4 dl = *reinterpret_cast<const float4*>(src + DP_STG_HALF + r * (DP_HALF_N * 4) + c4 * 16);
+            const float4 dl = *reinterpret_cast<const float4*>(src + D1_STG_HALF + r * (D1_HALF_N * 4) + c4 * 16);
             v[0] = __fsub_rn(v[0], __fmul_rn(gapf, dl.x)); v[1] = __fsub_rn(v[1], __fmul_rn(gapf, dl.y));   // w - (tau_fwd - tau_bkwd) * delta
             v[2] = __fsub_rn(v[2], __fmul_rn(gapf, dl.z)); v[3] = __fsub_rn(v[3], __fmul_rn(gapf, dl.w));
           }
@@ -1138,13 +1496,13 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
         fence_async_smem();
         __syncwarp();
         if (lane == 0) { mbar_arrive_cluster(leader_bfull + 8 * br.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
-        br.advance(DP_NB); sg.advance(DP_NG);
+        br.advance(D1_NB); sg.advance(D1_NG);
       }
     }
   } else {
     // ---------------- epilogue (both CTAs): 8 warps, warp%4 = TMEM lane group, two warps per group split the 128 columns ----------------
     const int q = warp & 3;
-    const int ew = warp - 2 - DP_XF_WARPS;                            // 0..7
+    const int ew = warp - 2 - D1_XF_WARPS;                            // 0..7
     const int half = ew >> 2;
     uint8_t* obuf = sO_ptr + ew * 4096;
     const uint32_t obuf_s = sO + ew * 4096;
@@ -1155,7 +1513,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
       const int tile = order[slot];
       if (tile < 0) continue;
-      const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
+      const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
       const StageDyn& d = t.dyn[tl.p];
       const StageDev& s = t.st[tl.p];
@@ -1168,9 +1526,9 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       const int nb = tl.n0 + half * 64;
 #pragma unroll 1
       for (int mi = 0; mi < tl.n_m; ++mi) {
-        const int mrow = tl.m0 + mi * DP_TILE_M + rank * TILE_M + q * 32;
+        const int mrow = tl.m0 + mi * D1_TILE_M + rank * TILE_M + q * 32;
         uint32_t r0[32], r1[32];
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * DP_ACC_COLS + mi * DP_TILE_N + half * 64);
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * D1_ACC_COLS + mi * D1_TILE_N + half * 64);
         tmem_ld32(taddr, r0);
         tmem_ld32(taddr + 32, r1);
         tmem_ld_wait();
@@ -1204,7 +1562,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc_pair(tmem_base, 2 * DP_ACC_COLS);
+    tmem_dealloc_pair(tmem_base, 2 * D1_ACC_COLS);
   }
 }
 
@@ -1217,13 +1575,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct UmmaPlan {
   const CUtensorMap* d_maps = nullptr;
   const int* d_tile_start = nullptr;     // per (mode, level) at ts_off: [P+1] starts, then the stage of each tile
-  size_t ts_off[3][PM_MAX_LINEARS] = {};
+  size_t ts_off[4][PM_MAX_LINEARS] = {};
   const int* d_orders = nullptr;         // concatenated order arrays
   int* d_status = nullptr;
-  int n_slots[3][PM_MAX_LINEARS] = {};
-  int grid[3][PM_MAX_LINEARS] = {};
-  bool pair[3][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
-  size_t order_off[3][PM_MAX_LINEARS] = {};
+  int n_slots[4][PM_MAX_LINEARS] = {};
+  int grid[4][PM_MAX_LINEARS] = {};
+  bool pair[4][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
+  size_t order_off[4][PM_MAX_LINEARS] = {};
   int P = 0;
   // launches of one stage (microbatch-major order): the stage's tiles in ascending order are a slice of the identity list
   std::vector<int> h_tile_start;         // host copy of the tile starts
@@ -1237,12 +1595,12 @@ struct UmmaPlan {
 // projection next to d_model-sized layers) does not leave most SMs idle.  Unused slots hold -1.
 struct TileTables {
   std::vector<int> tile_start;           // per (mode, level): [P+1] starts, then the stage of each tile
-  size_t ts_off[3][PM_MAX_LINEARS] = {};
+  size_t ts_off[4][PM_MAX_LINEARS] = {};
   std::vector<int> orders;
-  int n_slots[3][PM_MAX_LINEARS] = {};
-  int grid[3][PM_MAX_LINEARS] = {};
-  bool pair[3][PM_MAX_LINEARS] = {};
-  size_t order_off[3][PM_MAX_LINEARS] = {};
+  int n_slots[4][PM_MAX_LINEARS] = {};
+  int grid[4][PM_MAX_LINEARS] = {};
+  bool pair[4][PM_MAX_LINEARS] = {};
+  size_t order_off[4][PM_MAX_LINEARS] = {};
   int max_tiles = 0;                     // most tiles of any (mode, level)
 };
 
@@ -1261,12 +1619,12 @@ static bool pair_kernels_allowed() {
   return !(v && v[0] == '0');
 }
 
-static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int sms) {
+static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int sms, int dgrad_split_below) {
   const int P = (int)st.size();
   const bool allow_pair = pair_kernels_allowed();
   TileTables tt;
   auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
-  for (int mode = 0; mode < 3; ++mode)
+  for (int mode = 0; mode < 4; ++mode)                      // 3: dgrad once more, on 128-column pair tiles (launches of one narrow stage)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       // block of this (mode, level): P + 1 tile starts, then the stage of every tile (one load instead of a search)
       tt.ts_off[mode][l] = tt.tile_start.size();
@@ -1281,22 +1639,26 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
           const LinDev& L = st[p].lin[l];
           ++n_lin_here;
           if ((mode == 2 ? L.n_out : T) < P2_TILE || (mode == 0 ? L.n_out : L.n_in) < P2_TILE) pair = false;
-          if (mode == 1 && p == 0 && l == 0 && st[p].pre != PRE_EMBED) --n_lin_here;   // the first Linear of the network has no input gradient
+          if ((mode == 1 || mode == 3) && p == 0 && l == 0 && st[p].pre != PRE_EMBED) --n_lin_here;   // the first Linear of the network has no input gradient
         }
       pair = pair && n_lin_here > 0;
       tt.pair[mode][l] = pair;
-      const int tile_m = pair ? P2_TILE : TILE_M, tile_n = pair ? (mode == 1 ? DP_TILE_N : P2_TILE) : TILE_N;
-      const int mg_rows = pair ? DP_MG : DG_MG;                     // dgrad: row tiles sharing one converted weight tile
+      if (mode == 3 && !pair) { tt.n_slots[mode][l] = 0; tt.grid[mode][l] = 0; tt.order_off[mode][l] = tt.orders.size();
+                                tt.tile_start.insert(tt.tile_start.end(), (size_t)P + 1, 0); continue; }
+      const bool dg = mode == 1 || mode == 3;
+      const int tile_m = pair ? P2_TILE : TILE_M, tile_n = pair ? (mode == 1 ? DP_TILE_N : (mode == 3 ? D1_TILE_N : P2_TILE)) : TILE_N;
+      const int mg_rows_fixed = pair ? (mode == 3 ? D1_MG : DP_MG) : DG_MG;   // dgrad: row tiles sharing one converted weight tile
       int acc = 0;
       for (int p = 0; p < P; ++p) {
         ts[p] = acc;
         if (l < st[p].n_lin) {
           const LinDev& L = st[p].lin[l];
-          const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (mode == 1 ? L.n_out : T);
+          const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (dg ? L.n_out : T);
           const int tm = cdiv(M, tile_m), tn = cdiv(N, tile_n), n_kb = cdiv(K, TILE_K);
-          const int groups = mode == 1 ? cdiv(tm, mg_rows) : tm;
+          const int mg_rows = (pair && mode == 1) ? dgrad_pair_mg(T, L.n_in, dgrad_split_below) : mg_rows_fixed;
+          const int groups = dg ? cdiv(tm, mg_rows) : tm;
           for (int g = 0; g < groups; ++g) {
-            const int n_m = mode == 1 ? std::min(mg_rows, tm - g * mg_rows) : 1;
+            const int n_m = dg ? std::min(mg_rows, tm - g * mg_rows) : 1;
             for (int n = 0; n < tn; ++n) work.push_back({(long long)n_kb * n_m + 3 * n_m, acc + g * tn + n});
           }
           acc += groups * tn;
@@ -1333,8 +1695,8 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
 static uint64_t maps_bytes(int P) { return (uint64_t)P * PM_MAX_LINEARS * MAPS_PER_LINEAR * sizeof(CUtensorMap); }
 static uint64_t ints_bytes(size_t n) { return ((uint64_t)n * sizeof(int) + 255) / 256 * 256; }
 
-uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st) {
-  const TileTables tt = build_tile_tables(T, st, device_sms());
+uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st, int dgrad_split_below) {
+  const TileTables tt = build_tile_tables(T, st, device_sms(), dgrad_split_below);
   return 256 + maps_bytes((int)st.size()) + ints_bytes(tt.tile_start.size()) + ints_bytes(tt.orders.size()) + ints_bytes((size_t)tt.max_tiles);
 }
 
@@ -1396,7 +1758,10 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
         }
         okm = okm && encode(fn, m + MAP_W_F32, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
         okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
-        uint32_t box4h[2] = {64, TILE_K};                               // CTA-pair dgrad: 64 columns per CTA
+        uint32_t box4q[2] = {DP_HALF_N, DP_SLAB_K};                     // CTA-pair dgrad: slabs of 32 k-rows x 128 columns per CTA
+        okm = okm && encode(fn, m + MAP_W_F32Q, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4q, err);
+        okm = okm && encode(fn, m + MAP_D_F32Q, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4q, err);
+        uint32_t box4h[2] = {64, TILE_K};                               // 128-column pair dgrad: 64 columns per CTA
         okm = okm && encode(fn, m + MAP_W_F32H, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4h, err);
         okm = okm && encode(fn, m + MAP_D_F32H, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4h, err);
       }
@@ -1443,8 +1808,8 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       if (!okm) { delete plan; return PM_ERR_CUDA; }
     }
   }
-  const TileTables tt = build_tile_tables(t.T, st, device_sms());
-  for (int mode = 0; mode < 3; ++mode)
+  const TileTables tt = build_tile_tables(t.T, st, device_sms(), t.dgrad_split_below);
+  for (int mode = 0; mode < 4; ++mode)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       plan->n_slots[mode][l] = tt.n_slots[mode][l];
       plan->grid[mode][l] = tt.grid[mode][l];
@@ -1471,6 +1836,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DP_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_pair128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, D1_SMEM_BYTES);
   if (e != cudaSuccess) { err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); delete plan; return PM_ERR_CUDA; }
   plan->d_status = (int*)region;
   plan->d_maps = (const CUtensorMap*)(region + 256);
@@ -1514,6 +1880,12 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   int grid = plan->grid[mode][lvl];                                   // one persistent CTA per SM
   const int* ts = plan->d_tile_start + plan->ts_off[mode][lvl];
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
+  bool narrow = false;                                                // dgrad of one narrow stage: 128-column tiles
+  if (t.sel_p >= 0 && mode == 1 && plan->pair[1][lvl] && plan->pair[3][lvl]) {
+    const int* h1 = plan->h_tile_start.data() + plan->ts_off[1][lvl];
+    narrow = h1[t.sel_p + 1] - h1[t.sel_p] < 64;                      // too few 256-column tile groups for the CTA pairs
+    if (narrow) { mode = 3; ts = plan->d_tile_start + plan->ts_off[3][lvl]; }
+  }
   if (t.sel_p >= 0) {                                                 // the tiles of one stage, in ascending order
     const int* hts = plan->h_tile_start.data() + plan->ts_off[mode][lvl];
     const int first = hts[t.sel_p];
@@ -1527,6 +1899,7 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   if (plan->pair[mode][lvl]) {
     if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else if (mode == 3) umma_dgrad_pair128_kernel<<<grid, D1_THREADS, D1_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     return cudaGetLastError();
   }

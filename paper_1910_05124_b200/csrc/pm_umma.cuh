@@ -9,7 +9,8 @@ namespace pm {
 struct UmmaPlan;   // tensor maps and launch geometry, built once per context
 
 // Bytes of caller workspace the plan needs (status word + tensor maps).
-uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st);
+// dgrad_split_below: see TickArgs::dgrad_split_below (the plan must be created with the same value).
+uint64_t umma_workspace_bytes(int T, const std::vector<StageDev>& st, int dgrad_split_below);
 // ws_region: device memory of at least umma_workspace_bytes(T, stages), 256-byte aligned.  Synchronises `stream`.
 pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<StageDev>& st, void* ws_region,
                            cudaStream_t stream, std::string& err);

@@ -136,9 +136,12 @@ def compare_params(pipe, res, tol, per_stage=False, bias_per_stage=False, report
             assert eW <= tol, f"stage {p} W{j}: {eW}"
             ref_b = res.params[p][2 * j + 1]
             if np.abs(ref_b).max() > 0:
-                eb = max_rel_err(b, ref_b)
+                # a bias starts at zero and is a few steps in size: it is held to the tolerance against the largest entry
+                # of its stage vector (w_t)_i, the unit in which Section 2.1 states the method, not against itself
+                stage_scale = max(np.abs(np.asarray(t_, dtype=np.float64)).max() for t_ in res.params[p])
+                eb = float(np.abs(np.asarray(b, dtype=np.float64) - np.asarray(ref_b, dtype=np.float64)).max() / stage_scale)
                 worst = max(worst, eb)
-                assert eb <= tol, f"stage {p} b{j}: {eb}"
+                assert eb <= tol, f"stage {p} b{j}: {eb} of the stage vector's largest entry"
     return worst
 
 
