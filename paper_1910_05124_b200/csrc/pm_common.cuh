@@ -11,7 +11,10 @@ enum { PRE_NONE = 0, PRE_EMBED = 1, PRE_LN = 2 };
 enum { POST_NONE = 0, POST_ATTENTION = 1, POST_SKIP_OUT = 2, POST_RESIDUAL = 3, POST_CROSS_ATTENTION = 4 };
 // LF_ACT_FROM_Y: a ReLU whose pre-activation is not stashed: the backward takes the mask from the stashed output
 // (y > 0 exactly where z > 0), which the next Linear keeps for its weight gradient anyway
-enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4, LF_ACT_FROM_Y = 8 };
+// LF_DZ_FUSED: a ReLU at the end of a stage whose output is the next stage's stashed input (bf16 tensor-core path): the
+// next stage's dgrad epilogue applies the mask (its own stashed input > 0) to the gradient it sends back, so this
+// Linear receives dz itself and its backward pass treats it as a Linear without activation
+enum { LF_WRITE_Z = 1, LF_WRITE_Y = 2, LF_OUT_F32 = 4, LF_ACT_FROM_Y = 8, LF_DZ_FUSED = 16 };
 
 // Static description of one Linear inside a stage (device copy).
 struct LinDev {
@@ -45,6 +48,8 @@ struct StageDev {
   int32_t mem_first;          // from_memory stage that runs its backward first (the last one): it stores, the others add
   int32_t ids_stream;         // embedding: which input stream (0, 1)
   int32_t ids_depth;          // embedding: slots of ids_ring, slot = microbatch % ids_depth
+  int32_t mask_dx;            // the gradient this stage's first Linear sends to the previous stage is masked with (own input > 0):
+                              // the previous stage ends in a ReLU whose backward is fused here (LF_DZ_FUSED)
   int32_t vdepth;             // weight versions the forward pass can reach: 1 (the live weights, tick-major) or tau_f + 1
   uint32_t small_count;       // fp32 elements of a slot of s_ring (biases, LayerNorm gain and bias), a multiple of 64
   uint32_t g_soff, beta_soff; // offsets of LayerNorm gain / bias inside a slot of s_ring
@@ -139,6 +144,8 @@ __device__ __forceinline__ float act_grad(float z, int act) {
   return 1.0f;
 }
 
+// the activation as the backward pass sees it (a fused ReLU has been applied upstream already)
+__host__ __device__ __forceinline__ int bwd_act(const LinDev& L) { return (L.flags & LF_DZ_FUSED) ? PM_ACT_NONE : L.act; }
 // the stage's last Linear feeds an attention op (its output is the q, k, v stash; its gradient comes from s.dy)
 __host__ __device__ __forceinline__ bool feeds_attention(int post) { return post == POST_ATTENTION || post == POST_CROSS_ATTENTION; }
 

@@ -248,7 +248,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if ((ld.act != PM_ACT_NONE && !(ld.flags & LF_ACT_FROM_Y)) || to_attention) ld.flags |= LF_WRITE_Z;
       if (!to_attention && !logits) ld.flags |= LF_WRITE_Y;
       if (logits) ld.flags |= LF_OUT_F32;
+      // the ReLU's backward is applied by the next stage's dgrad epilogue when that stage takes y as its plain input
+      // (tensor-core path; PM_RELU_FUSE=0 in the environment keeps the separate pass, for comparisons)
+      static const bool fuse_ok = []() { const char* v = getenv("PM_RELU_FUSE"); return !(v && v[0] == '0'); }();
+      if (fuse_ok && cfg->compute_dtype == PM_BF16 && last && (ld.flags & LF_ACT_FROM_Y) && next_takes_y &&
+          stages[p + 1].ops[0].kind == PM_OP_LINEAR)
+        ld.flags |= LF_DZ_FUSED;
     }
+    if (p > 0 && (L.st[p - 1].lin[L.st[p - 1].n_lin - 1].flags & LF_DZ_FUSED)) s.mask_dx = 1;
     // ---- rings
     if (s.pre != PRE_EMBED) { s.x_ring = ring; ring = align_up(ring + (uint64_t)s.xdepth * T * s.d_in * esz, 256); }
     if (s.pre != PRE_NONE) { s.u_ring = ring; ring = align_up(ring + (uint64_t)s.depth * T * s.d_in * esz, 256); }
@@ -574,7 +581,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
   t.mb_major = L.queue ? 1 : 0; t.sel_p = -1;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
-  t.ln_li0 = 0; t.defer_finish = 0;
+  t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0;
   t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
@@ -795,7 +802,10 @@ static pm_status mb_backward(pm_ctx* ctx) {
         else if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
       }
       for (int l = sd.n_lin - 1; l >= 0; --l) {
-        if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ta)))) != PM_OK) return s;
+        // dz = dy * act'(z) must exist before this stage's dgrad; a Linear without activation needs only the column sums
+        // of its incoming gradient (the bias gradient), which wait for one grouped launch at the end
+        if ((!grouped || bwd_act(sd.lin[l]) != PM_ACT_NONE) &&
+            (s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ta)))) != PM_OK) return s;
         cudaError_t e;
         if (!grouped) {
           prof_begin(ctx, PM_PROF_WGRAD);
@@ -811,7 +821,10 @@ static pm_status mb_backward(pm_ctx* ctx) {
       if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ta, dt, ctx->ls), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
     }
     if (grouped) {
-      const TickArgs ta = mb_args(ctx, 2 * P, -1);
+      TickArgs ta = mb_args(ctx, 2 * P, -1);
+      ta.colsum_only = 1; ta.defer_finish = 1;                  // bias gradients of the Linears without activation, all stages at once
+      if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, 0, ctx->ls), "bias gradient column sums", actbwd_launches(ta)))) != PM_OK) return s;
+      ta.colsum_only = 0; ta.defer_finish = 0;
       prof_begin(ctx, PM_PROF_WGRAD);
       cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
       if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;

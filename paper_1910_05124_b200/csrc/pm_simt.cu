@@ -191,7 +191,8 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   const uint64_t n = (uint64_t)t.T * L.n_out;
   const AT* dy = (lvl < s.n_lin - 1) ? ws_ptr<AT>(t, s.dh)
                  : (feeds_attention(s.post) ? ws_ptr<AT>(t, s.dy) : gin_read<AT>(t, s, d));
-  const bool has_act = L.act != PM_ACT_NONE;                // without an activation dz = dy: nothing is stored
+  const bool has_act = bwd_act(L) != PM_ACT_NONE;           // without an activation (or with one applied upstream) dz = dy: nothing is stored
+  if (t.colsum_only && has_act) return;
   // the pre-activation stash, or for a ReLU without one the stashed output (same sign pattern)
   const AT* z = !has_act ? dy
                 : !(L.flags & LF_ACT_FROM_Y) ? ring_ptr<AT>(t, L.z_ring, d.b_slot, n)
@@ -201,7 +202,7 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (vec) {
     if (c < L.n_out) {
-      if (L.act == PM_ACT_NONE) actbwd_rows<AT, PM_ACT_NONE, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
+      if (!has_act) actbwd_rows<AT, PM_ACT_NONE, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
       else if (L.act == PM_ACT_RELU) actbwd_rows<AT, PM_ACT_RELU, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
       else actbwd_rows<AT, PM_ACT_GELU, NW>(dy, z, dz, L.n_out, c, r0 + warp, r1, sum);
     }

@@ -57,6 +57,8 @@ struct TickArgs {
                                // group (0: always two); launches of one stage need enough groups for the CTA pairs
   float loss_scale;       // factor on dL/dy: 1/N with N microbatches per update (the minibatch loss is their mean), else 1
   int32_t ln_li0;         // first entry of ln_ids a launch covers (its grid counts entries from there)
+  int32_t colsum_only;    // activation-backward launch that only sums columns (bias gradients) of Linears WITHOUT activation:
+                          // stages with an activation were handled by their own launch (microbatch-major order)
   int32_t defer_finish;   // launches of one stage leave the per-chunk partial sums of bias / LayerNorm gradients in place;
                           // one grouped launch over all stages adds them up at the end of the backward pass
 };
@@ -129,7 +131,7 @@ template <typename AT> __device__ __forceinline__ AT* mem_at(const TickArgs& t, 
 }
 // dz = dy * act'(z) of Linear lvl as the wgrad / dgrad operand: without an activation it IS the incoming gradient
 template <typename AT> __device__ __forceinline__ const AT* dz_src(const TickArgs& t, const StageDev& s, const StageDyn& d, int lvl) {
-  if (s.lin[lvl].act != PM_ACT_NONE) return ws_at<AT>(t, s.dz);
+  if (bwd_act(s.lin[lvl]) != PM_ACT_NONE) return ws_at<AT>(t, s.dz);
   if (lvl < s.n_lin - 1) return ws_at<AT>(t, s.dh);
   if (feeds_attention(s.post)) return ws_at<AT>(t, s.dy);
   return gin_read<AT>(t, s, d);

@@ -192,6 +192,27 @@ __device__ __forceinline__ void load_skip64(const TickArgs& t, const StageDev& s
     skq[g] = (on && nb + 8 * g < N) ? __ldg(reinterpret_cast<const uint4*>(skrow + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
 }
 
+// dgrad epilogue of a stage whose predecessor's ReLU backward is fused here (StageDev::mask_dx): the 64 values of this
+// stage's own stashed input x (row `row`, columns nb .. nb+63, the slot of the microbatch in backward) whose sign
+// decides which entries of dx survive: dz_prev = dx where x > 0 (x = ReLU(z_prev) > 0 exactly where z_prev > 0), else 0.
+__device__ __forceinline__ void load_mask64(const TickArgs& t, const StageDev& s, const StageDyn& d, int N, int row, int nb, uint4 (&xq)[8]) {
+  const __nv_bfloat16* xrow = ring_at<__nv_bfloat16>(t, s.x_ring, d.b_xslot, (uint64_t)t.T * N) + (uint64_t)row * N + nb;
+  const bool on = row < t.T;
+#pragma unroll
+  for (int g = 0; g < 8; ++g)
+    xq[g] = (on && nb + 8 * g < N) ? __ldg(reinterpret_cast<const uint4*>(xrow + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
+}
+// zeroes f[e] where the e-th bfloat16 of xq is not positive (sign bit set, or zero)
+__device__ __forceinline__ void apply_mask8(float (&f)[8], const uint4& xq) {
+  const uint32_t w[4] = {xq.x, xq.y, xq.z, xq.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint32_t lo = w[e] & 0xFFFFu, hi = w[e] >> 16;
+    if ((lo & 0x8000u) || (lo & 0x7FFFu) == 0u) f[2 * e] = 0.0f;
+    if ((hi & 0x8000u) || (hi & 0x7FFFu) == 0u) f[2 * e + 1] = 0.0f;
+  }
+}
+
 // bias of columns n .. n+3 (zero beyond the tensor); n is a multiple of four
 __device__ __forceinline__ float4 load_bias4(const float* bias, int n, int N) {
   return n < N ? __ldg(reinterpret_cast<const float4*>(bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -277,7 +298,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         // dz operand: the dz scratch, or (no activation) the incoming gradient itself, which for the last Linear of a
         // stage without attention is the rotating mailbox slot written during the previous tick
         const StageDev& sd_ = t.st[tl.p];
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        const int dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         for (int kb = 0; kb < tl.n_kb; ++kb) {
@@ -483,7 +504,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         const StageDyn& d = t.dyn[tl.p];
         const StageDev& sd_ = t.st[tl.p];
         const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        const int dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         const int ma = tl.m0 + rank * TILE_M, nbh = tl.n0 + rank * TILE_N;   // this CTA's rows of A and of B
@@ -727,7 +748,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
         const StageDyn& d = t.dyn[ca.tl.p];
         const StageDev& sd_ = t.st[ca.tl.p];
         const CUtensorMap* lm = maps + ((size_t)ca.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
-        const int dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        const int dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         for (int mi = 0; mi < ca.tl.n_m; ++mi) {
           if (!mbar_wait(bar_aempty + 8 * ar.idx, ar.phase ^ 1, abort_flag, status, 22)) { ok = false; break; }
           const uint32_t fa = bar_afull + 8 * ar.idx;
@@ -853,6 +874,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       if (!ready) { ok = false; break; }
       tc_fence_after();
       const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
+      const bool masked = lvl == 0 && s.mask_dx != 0;              // the previous stage's ReLU backward is applied here
       for (int mi = 0; mi < tl.n_m; ++mi) {
         const int mrow = tl.m0 + mi * TILE_M + q * 32;
 #pragma unroll 1
@@ -862,6 +884,8 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mi * ACC_COLS + half * 64);
           tmem_ld32(taddr, r0);
           tmem_ld32(taddr + 32, r1);
+          uint4 xq[8];
+          if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
           tmem_ld_wait();
           if (mrow >= tl.M || nb >= tl.N) continue;
           if (lane == 0 && stored) tma_store_wait_read();
@@ -871,6 +895,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+            if (masked) apply_mask8(f, xq[g]);
             *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
                 make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
           }
@@ -1015,7 +1040,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
         const StageDev& sd_ = t.st[c.tl.p];
         c.lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
         c.corr = d.use_delta != 0;
-        c.dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        c.dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         c.kb = 0; c.done = false;
         return;
       }
@@ -1200,6 +1225,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       const StageDev& s = t.st[tl.p];
       const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
       const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
+      const bool masked = lvl == 0 && s.mask_dx != 0;              // the previous stage's ReLU backward is applied here
 #pragma unroll 1
       for (int mi = 0; mi < tl.n_m && ok; ++mi) {
         const int b = acc.buf(mi, tl.n_m);
@@ -1215,6 +1241,8 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * DP_ACC_COLS + half * 128 + c * 64);
           tmem_ld32(taddr, r0);
           tmem_ld32(taddr + 32, r1);
+          uint4 xq[8];
+          if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
           tmem_ld_wait();
           if (c == 1) {
             tc_fence_before();
@@ -1229,6 +1257,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+            if (masked) apply_mask8(f, xq[g]);
             *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
                 make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
           }
@@ -1352,7 +1381,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
         const StageDev& sd_ = t.st[c.tl.p];
         c.lm = maps + ((size_t)c.tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
         c.corr = d.use_delta != 0;
-        c.dz_slot = (sd_.lin[lvl].act == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
+        c.dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         c.kb = 0; c.done = false;
         return;
       }
@@ -1523,6 +1552,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
       if (!ready) { ok = false; break; }
       tc_fence_after();
       const int dslot = (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0;
+      const bool masked = lvl == 0 && s.mask_dx != 0;              // the previous stage's ReLU backward is applied here
       const int nb = tl.n0 + half * 64;
 #pragma unroll 1
       for (int mi = 0; mi < tl.n_m; ++mi) {
@@ -1531,6 +1561,8 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * D1_ACC_COLS + mi * D1_TILE_N + half * 64);
         tmem_ld32(taddr, r0);
         tmem_ld32(taddr + 32, r1);
+        uint4 xq[8];
+        if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
         tmem_ld_wait();
         if (mi == tl.n_m - 1) {
           tc_fence_before();
@@ -1545,6 +1577,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
           float f[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+          if (masked) apply_mask8(f, xq[g]);
           *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
               make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
         }
@@ -1768,7 +1801,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
       {
         // dz operand (same rule as dz_src): dz scratch | dh scratch | attention's dy | rotating incoming-gradient mailbox
         char* dzb; uint64_t dz_slots = 1;
-        if (L.act != PM_ACT_NONE) dzb = t.ws + s.dz;
+        if (bwd_act(L) != PM_ACT_NONE) dzb = t.ws + s.dz;
         else if (l < s.n_lin - 1) dzb = t.ws + s.dh;
         else if (feeds_attention(s.post)) dzb = t.ws + s.dy;
         else if (s.emit_memory) { dzb = t.ws + t.gmem_off; dz_slots = (uint64_t)t.gmem_depth; }
