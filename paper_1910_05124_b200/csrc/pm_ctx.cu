@@ -248,9 +248,12 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if ((ld.act != PM_ACT_NONE && !(ld.flags & LF_ACT_FROM_Y)) || to_attention) ld.flags |= LF_WRITE_Z;
       if (!to_attention && !logits) ld.flags |= LF_WRITE_Y;
       if (logits) ld.flags |= LF_OUT_F32;
-      // the ReLU's backward is applied by the next stage's dgrad epilogue when that stage takes y as its plain input
-      // (tensor-core path; PM_RELU_FUSE=0 in the environment keeps the separate pass, for comparisons)
-      static const bool fuse_ok = []() { const char* v = getenv("PM_RELU_FUSE"); return !(v && v[0] == '0'); }();
+      // The ReLU's backward can be applied by the next stage's dgrad epilogue when that stage takes y as its plain input
+      // (tensor-core path).  Off unless PM_RELU_FUSE=1 is in the environment: the mask costs the dgrad epilogue, which is on
+      // that kernel's critical path (single-buffered accumulators), more than the separate pass costs (measured: config 4
+      // dgrad 0.215 -> 0.290 ms per tick against 0.014 ms saved in the activation-backward pass).
+      const char* fuse_env = getenv("PM_RELU_FUSE");
+      const bool fuse_ok = fuse_env && fuse_env[0] == '1';
       if (fuse_ok && cfg->compute_dtype == PM_BF16 && last && (ld.flags & LF_ACT_FROM_Y) && next_takes_y &&
           stages[p + 1].ops[0].kind == PM_OP_LINEAR)
         ld.flags |= LF_DZ_FUSED;

@@ -195,22 +195,34 @@ __device__ __forceinline__ void load_skip64(const TickArgs& t, const StageDev& s
 // dgrad epilogue of a stage whose predecessor's ReLU backward is fused here (StageDev::mask_dx): the 64 values of this
 // stage's own stashed input x (row `row`, columns nb .. nb+63, the slot of the microbatch in backward) whose sign
 // decides which entries of dx survive: dz_prev = dx where x > 0 (x = ReLU(z_prev) > 0 exactly where z_prev > 0), else 0.
-__device__ __forceinline__ void load_mask64(const TickArgs& t, const StageDev& s, const StageDyn& d, int N, int row, int nb, uint4 (&xq)[8]) {
+__device__ __forceinline__ uint64_t load_mask_bits64(const TickArgs& t, const StageDev& s, const StageDyn& d, int N, int row, int nb) {
+  // Bit i is set where x[row, nb + i] > 0.  The 64 values are compressed to bits BEFORE the accumulator is read from
+  // tensor memory, so that they never share the register file with it (the kernel runs at 96 registers per thread).
+  if (row >= t.T) return 0ull;
   const __nv_bfloat16* xrow = ring_at<__nv_bfloat16>(t, s.x_ring, d.b_xslot, (uint64_t)t.T * N) + (uint64_t)row * N + nb;
-  const bool on = row < t.T;
+  uint4 xq[8];
 #pragma unroll
   for (int g = 0; g < 8; ++g)
-    xq[g] = (on && nb + 8 * g < N) ? __ldg(reinterpret_cast<const uint4*>(xrow + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
-}
-// zeroes f[e] where the e-th bfloat16 of xq is not positive (sign bit set, or zero)
-__device__ __forceinline__ void apply_mask8(float (&f)[8], const uint4& xq) {
-  const uint32_t w[4] = {xq.x, xq.y, xq.z, xq.w};
+    xq[g] = (nb + 8 * g < N) ? __ldg(reinterpret_cast<const uint4*>(xrow + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
+  uint64_t mk = 0ull;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const uint32_t lo = w[e] & 0xFFFFu, hi = w[e] >> 16;
-    if ((lo & 0x8000u) || (lo & 0x7FFFu) == 0u) f[2 * e] = 0.0f;
-    if ((hi & 0x8000u) || (hi & 0x7FFFu) == 0u) f[2 * e + 1] = 0.0f;
+  for (int g = 0; g < 8; ++g) {
+    const uint32_t w[4] = {xq[g].x, xq[g].y, xq[g].z, xq[g].w};
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t lo = w[e] & 0xFFFFu, hi = w[e] >> 16;
+      bits |= (uint32_t)(!(lo & 0x8000u) && (lo & 0x7FFFu) != 0u) << (2 * e);
+      bits |= (uint32_t)(!(hi & 0x8000u) && (hi & 0x7FFFu) != 0u) << (2 * e + 1);
+    }
+    mk |= (uint64_t)bits << (8 * g);
   }
+  return mk;
+}
+// zeroes f[e] where bit e of `bits` is clear
+__device__ __forceinline__ void apply_mask8(float (&f)[8], uint32_t bits) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) if (!((bits >> e) & 1u)) f[e] = 0.0f;
 }
 
 // bias of columns n .. n+3 (zero beyond the tensor); n is a multiple of four
@@ -882,10 +894,9 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
           const int nb = tl.n0 + half * 64;
           uint32_t r0[32], r1[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mi * ACC_COLS + half * 64);
+          const uint64_t mk = masked ? load_mask_bits64(t, s, d, tl.N, mrow + lane, nb) : ~0ull;
           tmem_ld32(taddr, r0);
           tmem_ld32(taddr + 32, r1);
-          uint4 xq[8];
-          if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
           tmem_ld_wait();
           if (mrow >= tl.M || nb >= tl.N) continue;
           if (lane == 0 && stored) tma_store_wait_read();
@@ -895,7 +906,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
-            if (masked) apply_mask8(f, xq[g]);
+            if (masked) apply_mask8(f, (uint32_t)(mk >> (8 * g)) & 0xFFu);
             *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
                 make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
           }
@@ -1239,10 +1250,9 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
           const int nb = tl.n0 + half * 128 + c * 64;
           uint32_t r0[32], r1[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * DP_ACC_COLS + half * 128 + c * 64);
+          const uint64_t mk = masked ? load_mask_bits64(t, s, d, tl.N, mrow + lane, nb) : ~0ull;
           tmem_ld32(taddr, r0);
           tmem_ld32(taddr + 32, r1);
-          uint4 xq[8];
-          if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
           tmem_ld_wait();
           if (c == 1) {
             tc_fence_before();
@@ -1257,7 +1267,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
-            if (masked) apply_mask8(f, xq[g]);
+            if (masked) apply_mask8(f, (uint32_t)(mk >> (8 * g)) & 0xFFu);
             *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
                 make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
           }
@@ -1559,10 +1569,9 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
         const int mrow = tl.m0 + mi * D1_TILE_M + rank * TILE_M + q * 32;
         uint32_t r0[32], r1[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * D1_ACC_COLS + mi * D1_TILE_N + half * 64);
+        const uint64_t mk = masked ? load_mask_bits64(t, s, d, tl.N, mrow + lane, nb) : ~0ull;
         tmem_ld32(taddr, r0);
         tmem_ld32(taddr + 32, r1);
-        uint4 xq[8];
-        if (masked) load_mask64(t, s, d, tl.N, mrow + lane, nb, xq);
         tmem_ld_wait();
         if (mi == tl.n_m - 1) {
           tc_fence_before();
@@ -1577,7 +1586,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
           float f[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
-          if (masked) apply_mask8(f, xq[g]);
+          if (masked) apply_mask8(f, (uint32_t)(mk >> (8 * g)) & 0xFFu);
           *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) =
               make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
         }

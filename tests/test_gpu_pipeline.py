@@ -176,3 +176,19 @@ def test_cfg3_shape_many_steps(cuda_device):
     np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_DEEP_LOSS_TOL)
     worst = compare_params(pipe, res, BF16_W_TOL)
     print("cfg3 narrow 200 steps worst relative weight error", worst)
+
+
+@pytest.mark.parametrize("width,T,per_stage", [(192, 40, 2), (320, 384, 1), (512, 512, 2)])
+def test_relu_backward_fused_into_next_dgrad(cuda_device, monkeypatch, width, T, per_stage):
+    """PM_RELU_FUSE=1: a ReLU at the end of a stage is applied to the gradient by the next stage's dgrad epilogue (mask
+    from that stage's own stashed input) in all three dgrad kernels (single CTA, 128- and 256-column pair tiles)."""
+    monkeypatch.setenv("PM_RELU_FUSE", "1")
+    wl = I.mlp_workload("relu_fused", 4, width, per_stage, "relu", T, compute="bf16", optimizer="sgdm", alpha=0.01, beta1=0.9,
+                        K=5, D=0.5, steps=22, seed=191005124 + 92)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    for order in ("tick_major", "mb_major"):
+        pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order=order)
+        check_book(book, res, wl.steps, wl.n_stages)
+        np.testing.assert_allclose(losses, np.array(res.losses), rtol=BF16_LOSS_TOL)
+        compare_params(pipe, res, BF16_W_TOL)
