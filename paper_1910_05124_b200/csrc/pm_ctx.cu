@@ -422,11 +422,23 @@ struct pm_ctx {
   // phase on plain launches.
   struct PhaseGraph { cudaGraphExec_t exec = nullptr; int eager_runs = 0; uint64_t launches = 0; bool failed = false; };
   PhaseGraph g_fwd, g_bwd, g_upd;
+  // Tick-major order with an entry period E > 1 ("sparse ticks"): a tick's launches cover only the stages whose turn it
+  // is (those at distance = tick mod E from a microbatch's entry), one graph per phase and residue; the forward stages
+  // run on a stream of their own, next to the backward and update of the same tick (see sparse_forward).
+  std::vector<PhaseGraph> gs_fwd, gs_bwd, gs_upd;
+  cudaStream_t fwd_stream = nullptr;
+  cudaEvent_t ev_sched = nullptr, ev_fwd = nullptr;
+  bool fwd_pending = false;             // work of the last tick's forward may still be running on fwd_stream
+  std::vector<int> seg_first, seg_count;   // small-tensor segments of a stage: [seg_first[p], + seg_count[p])
   bool graphs = true;
   cudaStream_t cap_stream = nullptr;
   cudaStream_t ls = nullptr;            // the stream the phase bodies launch on: `stream`, or `cap_stream` while capturing
   ~pm_ctx() {
     for (PhaseGraph* g : {&g_fwd, &g_bwd, &g_upd}) if (g->exec) cudaGraphExecDestroy(g->exec);
+    for (auto* v : {&gs_fwd, &gs_bwd, &gs_upd}) for (auto& g : *v) if (g.exec) cudaGraphExecDestroy(g.exec);
+    if (fwd_stream) cudaStreamDestroy(fwd_stream);
+    if (ev_sched) cudaEventDestroy(ev_sched);
+    if (ev_fwd) cudaEventDestroy(ev_fwd);
     if (cap_stream) cudaStreamDestroy(cap_stream);
   }
   // optional per-kernel-class timing with CUDA events on the context's stream
@@ -632,6 +644,24 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     pm_status us = umma_plan_create(&c->umma, t, c->L.st, c->ws + L.off_umma, c->stream, uerr);
     if (us != PM_OK) { delete c; return fail(nullptr, us, uerr); }
   }
+  if (L.E > 1) {
+    const char* v = getenv("PM_SPARSE_TICKS");           // PM_SPARSE_TICKS=0: every tick launches grids over all stages (for comparisons)
+    if (!(v && v[0] == '0')) {
+      c->gs_fwd.assign((size_t)L.E, pm_ctx::PhaseGraph{}); c->gs_bwd.assign((size_t)L.E, pm_ctx::PhaseGraph{}); c->gs_upd.assign((size_t)L.E, pm_ctx::PhaseGraph{});
+      const char* v2 = getenv("PM_FWD_STREAM");          // PM_FWD_STREAM=0: forward and backward of a tick on one stream
+      if (!(v2 && v2[0] == '0')) {
+        if (cudaStreamCreateWithFlags(&c->fwd_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_sched, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_fwd, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); c->fwd_stream = nullptr; }
+      }
+    }
+    c->seg_first.assign(P, 0); c->seg_count.assign(P, 0);
+    for (size_t k = 0; k < c->L.segs.size(); ++k) {
+      const int p = c->L.segs[k].stage;
+      if (c->seg_count[p] == 0) c->seg_first[p] = (int)k;
+      c->seg_count[p] += 1;
+    }
+  }
   if (L.queue) {
     // version 0 of every stage's queue: the initial weights in the operand type, and the small fp32 tensors
     const bool f32 = cfg->compute_dtype == PM_F32;
@@ -669,12 +699,13 @@ static inline void prof_begin(pm_ctx* ctx, int cls) {
 
 // Runs the kernel launches of one phase (`body` launches on ctx->ls): plainly the first times and whenever graphs
 // are off, then once under stream capture to build the phase's graph, then by replaying that graph.
-static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::function<pm_status()>& body) {
-  ctx->ls = ctx->stream;
+static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::function<pm_status()>& body, cudaStream_t run_on = nullptr) {
+  if (!run_on) run_on = ctx->stream;
+  ctx->ls = run_on;
   if (!ctx->graphs || ctx->prof_on || g.failed || !ctx->cap_stream) return body();
   if (g.exec) {
     ctx->launches += g.launches;
-    cudaError_t e = cudaGraphLaunch(g.exec, ctx->stream);
+    cudaError_t e = cudaGraphLaunch(g.exec, run_on);
     return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, "graph launch");
   }
   if (g.eager_runs < 2) { ++g.eager_runs; return body(); }      // modules loaded, function attributes set
@@ -682,7 +713,7 @@ static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::functi
   if (cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) { cudaGetLastError(); g.failed = true; return body(); }
   ctx->ls = ctx->cap_stream;
   const pm_status sb = body();
-  ctx->ls = ctx->stream;
+  ctx->ls = run_on;
   cudaGraph_t graph = nullptr;
   cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
   if (sb == PM_OK && e == cudaSuccess && graph) {
@@ -696,7 +727,7 @@ static pm_status run_phase(pm_ctx* ctx, pm_ctx::PhaseGraph& g, const std::functi
     ctx->launches = l0;
     return body();
   }
-  e = cudaGraphLaunch(g.exec, ctx->stream);
+  e = cudaGraphLaunch(g.exec, run_on);
   return e == cudaSuccess ? PM_OK : cuda_fail(ctx, e, "graph launch");
 }
 
@@ -751,6 +782,57 @@ static TickArgs mb_args(const pm_ctx* ctx, int v, int p) {
   return t;
 }
 
+// The launches of ONE stage's forward pass (ta restricted to it).
+static pm_status stage_forward(pm_ctx* ctx, const TickArgs& ta, int p) {
+  const int dt = ctx->cfg.compute_dtype;
+  const StageDev& sd = ctx->L.st[p];
+  pm_status s;
+  if (sd.pre != PRE_NONE && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ta, dt, ctx->ls), "embedding / LayerNorm forward"))) != PM_OK) return s;
+  for (int l = 0; l < sd.n_lin; ++l) {
+    prof_begin(ctx, PM_PROF_GEMM_FWD);
+    cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 0, l, ctx->ls) : umma_launch(ctx->umma, ta, 0, l, ctx->ls);
+    if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
+  }
+  const bool att = feeds_attention(sd.post);
+  if (att && ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
+  const int n_post = ((att && !ctx->attn) ? 1 : 0) + ((sd.post == POST_RESIDUAL && !ctx->ta.res_fused) ? 1 : 0);
+  if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
+  return PM_OK;
+}
+
+// The launches of ONE stage's backward pass (ta restricted to it).  grouped: the weight gradient, the bias column sums of
+// Linears without activation and the finishing passes are left to grouped launches over all stages (ta.defer_finish set).
+static pm_status stage_backward(pm_ctx* ctx, const TickArgs& ta, int p, bool grouped) {
+  const int dt = ctx->cfg.compute_dtype;
+  const int P = ctx->cfg.n_stages;
+  const StageDev& sd = ctx->L.st[p];
+  pm_status s;
+  if (p == P - 1 && (s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
+  if (feeds_attention(sd.post)) {
+    if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ta, false, ctx->ls), "attention backward"))) != PM_OK) return s; }
+    else if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
+  }
+  for (int l = sd.n_lin - 1; l >= 0; --l) {
+    // dz = dy * act'(z) must exist before this stage's dgrad; a Linear without activation needs only the column sums
+    // of its incoming gradient (the bias gradient), which can wait for one grouped launch
+    if ((!grouped || bwd_act(sd.lin[l]) != PM_ACT_NONE) &&
+        (s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ta)))) != PM_OK) return s;
+    cudaError_t e;
+    if (!grouped) {
+      prof_begin(ctx, PM_PROF_WGRAD);
+      e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, l, ctx->ls) : umma_launch(ctx->umma, ta, 2, l, ctx->ls);
+      if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+    }
+    if (p == 0 && l == 0 && sd.pre != PRE_EMBED) continue;          // raw network inputs need no gradient
+    prof_begin(ctx, PM_PROF_DGRAD);
+    e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, 1, l, ctx->ls);
+    if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
+  }
+  const int n_pre = sd.pre != PRE_NONE ? pre_bwd_launches(ta) : 0;
+  if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ta, dt, ctx->ls), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
+  return PM_OK;
+}
+
 static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!inputs || !targets) return fail(ctx, PM_ERR_INVALID_ARG, "microbatch-major order takes a microbatch at every step (there is nothing to drain)");
   const int dt = ctx->cfg.compute_dtype;
@@ -764,20 +846,8 @@ static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets
   if (s != PM_OK) return s;
   s = run_phase(ctx, ctx->g_fwd, [&]() -> pm_status {
     pm_status s;
-    for (int p = 0; p < P; ++p) {
-      const StageDev& sd = ctx->L.st[p];
-      const TickArgs ta = mb_args(ctx, p, p);
-      if (sd.pre != PRE_NONE && (s = TIMED(PM_PROF_PRE_FWD, check(ctx, launch_pre_fwd(ta, dt, ctx->ls), "embedding / LayerNorm forward"))) != PM_OK) return s;
-      for (int l = 0; l < sd.n_lin; ++l) {
-        prof_begin(ctx, PM_PROF_GEMM_FWD);
-        cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 0, l, ctx->ls) : umma_launch(ctx->umma, ta, 0, l, ctx->ls);
-        if ((s = check(ctx, e, "forward GEMM")) != PM_OK) return s;
-      }
-      const bool att = feeds_attention(sd.post);
-      if (att && ctx->attn && (s = TIMED(PM_PROF_ATTN_FWD, check(ctx, attn_tc_launch(ctx->attn, ta, true, ctx->ls), "attention forward"))) != PM_OK) return s;
-      const int n_post = ((att && !ctx->attn) ? 1 : 0) + ((sd.post == POST_RESIDUAL && !ctx->ta.res_fused) ? 1 : 0);
-      if (n_post && (s = TIMED(PM_PROF_POST_FWD, check(ctx, launch_post_fwd(ta, dt, ctx->ls, ctx->attn != nullptr), "attention / residual forward", n_post))) != PM_OK) return s;
-    }
+    for (int p = 0; p < P; ++p)
+      if ((s = stage_forward(ctx, mb_args(ctx, p, p), p)) != PM_OK) return s;
     return PM_OK;
   });
   if (s != PM_OK) return s;
@@ -796,32 +866,9 @@ static pm_status mb_backward(pm_ctx* ctx) {
   pm_status s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
     pm_status s;
     for (int p = P - 1; p >= 0; --p) {
-      const StageDev& sd = ctx->L.st[p];
       TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
       ta.defer_finish = grouped ? 1 : 0;        // the partial sums of bias and LayerNorm gradients are added up once, below
-      if (p == P - 1 && (s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
-      if (feeds_attention(sd.post)) {
-        if (ctx->attn) { if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, attn_tc_launch(ctx->attn, ta, false, ctx->ls), "attention backward"))) != PM_OK) return s; }
-        else if ((s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
-      }
-      for (int l = sd.n_lin - 1; l >= 0; --l) {
-        // dz = dy * act'(z) must exist before this stage's dgrad; a Linear without activation needs only the column sums
-        // of its incoming gradient (the bias gradient), which wait for one grouped launch at the end
-        if ((!grouped || bwd_act(sd.lin[l]) != PM_ACT_NONE) &&
-            (s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ta)))) != PM_OK) return s;
-        cudaError_t e;
-        if (!grouped) {
-          prof_begin(ctx, PM_PROF_WGRAD);
-          e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, l, ctx->ls) : umma_launch(ctx->umma, ta, 2, l, ctx->ls);
-          if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
-        }
-        if (p == 0 && l == 0 && sd.pre != PRE_EMBED) continue;          // raw network inputs need no gradient
-        prof_begin(ctx, PM_PROF_DGRAD);
-        e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, 1, l, ctx->ls);
-        if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
-      }
-      const int n_pre = sd.pre != PRE_NONE ? pre_bwd_launches(ta) : 0;
-      if (n_pre && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_pre_bwd(ta, dt, ctx->ls), "LayerNorm / embedding backward", n_pre))) != PM_OK) return s;
+      if ((s = stage_backward(ctx, ta, p, grouped)) != PM_OK) return s;
     }
     if (grouped) {
       TickArgs ta = mb_args(ctx, 2 * P, -1);
@@ -866,6 +913,83 @@ static pm_status mb_update(pm_ctx* ctx) {
   return PM_OK;
 }
 
+// ---- sparse ticks (tick-major order with an entry period E > 1) ----------------------------------------------------
+// Only the stages at distance = tick mod E from a microbatch's entry can hold a microbatch in a given tick, so a
+// tick's launches are restricted to them (each stage's kernels as in microbatch-major order), with one CUDA graph per
+// phase and residue.  A tick's forward stages depend on nothing its backward stages or updates produce (their
+// weights come from the version queues, their inputs from the previous tick's forward; the ring depths keep the two
+// apart), so they run on a stream of their own next to the backward and update of the same tick; the tick's
+// schedule waits for the previous tick's forward, and the forward waits for the schedule, which follows the previous
+// tick's update.
+static bool sparse_ticks(const pm_ctx* ctx) { return ctx->L.E > 1 && !ctx->gs_fwd.empty(); }
+
+static void sparse_stages(const pm_ctx* ctx, bool fwd, std::vector<int>& out) {
+  const int P = ctx->cfg.n_stages, E = ctx->L.E;
+  out.clear();
+  for (int p = 0; p < P; ++p) {
+    const int64_t off = fwd ? p : 2 * (int64_t)P - 1 - p;
+    if ((((ctx->tick - off) % E) + E) % E == 0) out.push_back(p);   // whether a microbatch IS there the kernels read from the schedule table
+  }
+}
+
+static pm_status sparse_forward_phase(pm_ctx* ctx) {
+  const bool side = ctx->fwd_stream && !ctx->prof_on;
+  if (side) {
+    cudaError_t e = cudaEventRecord(ctx->ev_sched, ctx->stream);                 // schedule table and inputs of this tick are in place
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->fwd_stream, ctx->ev_sched, 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "forward stream");
+  }
+  std::vector<int> st;
+  sparse_stages(ctx, true, st);
+  pm_status s = run_phase(ctx, ctx->gs_fwd[(size_t)(ctx->tick % ctx->L.E)], [&]() -> pm_status {
+    for (int p : st) { pm_status s = stage_forward(ctx, mb_args(ctx, 0, p), p); if (s != PM_OK) return s; }
+    return PM_OK;
+  }, side ? ctx->fwd_stream : nullptr);
+  if (s != PM_OK) return s;
+  if (side) {
+    cudaError_t e = cudaEventRecord(ctx->ev_fwd, ctx->fwd_stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "forward stream");
+    ctx->fwd_pending = true;
+  }
+  return PM_OK;
+}
+
+static pm_status sparse_backward_phase(pm_ctx* ctx) {
+  std::vector<int> st;
+  sparse_stages(ctx, false, st);
+  return run_phase(ctx, ctx->gs_bwd[(size_t)(ctx->tick % ctx->L.E)], [&]() -> pm_status {
+    for (auto it = st.rbegin(); it != st.rend(); ++it) {                           // later stages first, as everywhere
+      pm_status s = stage_backward(ctx, mb_args(ctx, 0, *it), *it, false);
+      if (s != PM_OK) return s;
+    }
+    return PM_OK;
+  });
+}
+
+static pm_status sparse_update_phase(pm_ctx* ctx) {
+  std::vector<int> st;
+  sparse_stages(ctx, false, st);
+  return run_phase(ctx, ctx->gs_upd[(size_t)(ctx->tick % ctx->L.E)], [&]() -> pm_status {
+    for (int p : st) {
+      prof_begin(ctx, PM_PROF_UPDATE);
+      cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64) + p, (const uint32_t*)(ctx->ws + ctx->L.off_e64) + p,
+                                    (const StageDyn*)(ctx->ws + ctx->L.off_dyn) + p, (int64_t*)(ctx->ws + ctx->L.off_nupd) + p, 1,
+                                    ctx->L.end64[p], ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls,
+                                    (void*)ctx->ta.ring, ctx->hp.lp_elem, ctx->L.begin64[p]);
+      pm_status s = check(ctx, e, "update");
+      if (s != PM_OK) return s;
+      if (ctx->seg_count[p] > 0) {
+        prof_begin(ctx, PM_PROF_UPDATE);
+        // the segments name their stage by its index in the whole table: hand the kernel the table's base
+        e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs) + ctx->seg_first[p], ctx->seg_count[p],
+                              (const StageDyn*)(ctx->ws + ctx->L.off_dyn), -1, ctx->ls);
+        if ((s = check(ctx, e, "weight-version push")) != PM_OK) return s;
+      }
+    }
+    return PM_OK;
+  });
+}
+
 pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   if (!ctx) return fail(nullptr, PM_ERR_INVALID_ARG, "null context");
   if (ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "pm_forward called out of order (expected pm_backward or pm_update)");
@@ -878,12 +1002,22 @@ pm_status pm_forward(pm_ctx* ctx, const void* inputs, const void* targets) {
   const int dt = ctx->cfg.compute_dtype;
   pm_status s;
   if (inputs) ctx->n_fed = mb + 1; else if (mb >= 0) ctx->draining = true;   // an empty tick between two warm-up microbatches ends nothing
+  if (ctx->fwd_pending) {                          // sparse ticks: the previous tick's forward still reads the schedule table
+    cudaError_t ew = cudaStreamWaitEvent(ctx->stream, ctx->ev_fwd, 0);
+    if (ew != cudaSuccess) return cuda_fail(ctx, ew, "forward stream");
+    ctx->fwd_pending = false;
+  }
   s = TIMED(PM_PROF_SCHEDULE, check(ctx, launch_schedule((const StageSched*)(ctx->ws + ctx->L.off_sched), (const int64_t*)(ctx->ws + ctx->L.off_nupd),
                                  (StageDyn*)(ctx->ws + ctx->L.off_dyn), ctx->hp, ctx->tick, ctx->n_fed, -1, ctx->stream), "schedule"));
   if (s != PM_OK) return s;
   if (inputs) {
     s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, mb, ctx->stream), "ingest"));
     if (s != PM_OK) return s;
+  }
+  if (sparse_ticks(ctx)) {
+    if (any_stage_active(ctx, 0, ctx->cfg.n_stages - 1) && (s = sparse_forward_phase(ctx)) != PM_OK) return s;
+    ctx->phase = 1;
+    return PM_OK;
   }
   // forward of every stage whose microbatch exists
   if (any_stage_active(ctx, 0, ctx->cfg.n_stages - 1)) {
@@ -916,7 +1050,9 @@ pm_status pm_backward(pm_ctx* ctx) {
   pm_status s;
   // any backward this tick?  stage P runs the microbatch that entered P ticks ago, stage 1 the one from 2P-1 ticks ago
   const bool any = any_stage_active(ctx, P, 2 * P - 1);
-  if (any) {
+  if (any && sparse_ticks(ctx)) {
+    if ((s = sparse_backward_phase(ctx)) != PM_OK) return s;
+  } else if (any) {
     s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
       pm_status s;
       if ((s = TIMED(PM_PROF_LOSS, check(ctx, launch_loss(ctx->ta, dt, ctx->ls), "loss"))) != PM_OK) return s;
@@ -949,7 +1085,10 @@ pm_status pm_update(pm_ctx* ctx) {
   if (ctx->L.mb) return mb_update(ctx);
   const int P = ctx->cfg.n_stages;
   const bool any = any_stage_active(ctx, P, 2 * P - 1);
-  if (any) {
+  if (any && sparse_ticks(ctx)) {
+    pm_status s = sparse_update_phase(ctx);
+    if (s != PM_OK) return s;
+  } else if (any) {
     pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
       prof_begin(ctx, PM_PROF_UPDATE);
       cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
@@ -996,6 +1135,7 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
   StageDyn d;
   int64_t n = 0;
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess && ctx->fwd_stream) e = cudaStreamSynchronize(ctx->fwd_stream);
   if (ctx->L.mb) {
     // the stage's forward ran in sub-tick `stage`, its backward in sub-tick 2P - 1 - stage of the last microbatch
     const int P = ctx->cfg.n_stages;
@@ -1030,6 +1170,7 @@ pm_status pm_get_losses(pm_ctx* ctx, float* host_out, int64_t first_mb, int64_t 
   if (first_mb + n > done) return fail(ctx, PM_ERR_INVALID_ARG, "loss of a microbatch that has not finished was requested");
   if (done - first_mb > ctx->L.loss_cap) return fail(ctx, PM_ERR_INVALID_ARG, "requested losses have left the device log");
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess && ctx->fwd_stream) e = cudaStreamSynchronize(ctx->fwd_stream);
   for (int64_t i = 0; i < n && e == cudaSuccess; ++i)
     e = cudaMemcpy(host_out + i, ctx->ws + ctx->L.off_loss + sizeof(float) * ((first_mb + i) % ctx->L.loss_cap), sizeof(float), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "loss read-back");
@@ -1075,6 +1216,7 @@ pm_status pm_profile_enable(pm_ctx* ctx, int32_t on) {
 pm_status pm_profile_read(pm_ctx* ctx, float* ms_by_class, int64_t* launches_by_class) {
   if (!ctx || !ms_by_class || !launches_by_class) return fail(ctx, PM_ERR_INVALID_ARG, "null argument");
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess && ctx->fwd_stream) e = cudaStreamSynchronize(ctx->fwd_stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "profile read");
   for (int i = 0; i < PM_PROF_CLASSES; ++i) { ms_by_class[i] = 0.f; launches_by_class[i] = 0; }
   for (size_t i = 0; i < ctx->prof_used; ++i) {
@@ -1092,6 +1234,7 @@ const char* pm_last_error(pm_ctx* ctx) { return ctx ? ctx->err.c_str() : g_error
 
 void pm_destroy(pm_ctx* ctx) {
   if (!ctx) return;
+  if (ctx->fwd_stream) cudaStreamSynchronize(ctx->fwd_stream);
   umma_plan_destroy(ctx->umma);
   attn_plan_destroy(ctx->attn);
   for (auto& ev : ctx->prof_ev) cudaEventDestroy(ev);

@@ -191,7 +191,7 @@ template <int OPT, int LP>
 __global__ void __launch_bounds__(kUpdThreads)
 update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
               const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
-              float beta1, float beta2, float eps) {
+              float beta1, float beta2, float eps, uint64_t first_vec4) {
   extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends
   uint32_t* sb = sm_bounds;
   uint32_t* se = sm_bounds + n_stages;
@@ -199,7 +199,7 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
   __syncthreads();
   const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
   const uint64_t stride = (uint64_t)gridDim.x * kUpdThreads * kUpdUnroll;
-  for (uint64_t base = (uint64_t)blockIdx.x * kUpdThreads * kUpdUnroll; base < total_vec4; base += stride) {
+  for (uint64_t base = first_vec4 + (uint64_t)blockIdx.x * kUpdThreads * kUpdUnroll; base < total_vec4; base += stride) {
     uint64_t v[kUpdUnroll];
     int stage[kUpdUnroll];
     UpdScalars sc[kUpdUnroll];
@@ -257,11 +257,12 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
 
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
-                          float eps, cudaStream_t stream, void* lp_base, int lp_elem) {
-  if (total64 == 0 || n_stages == 0) return cudaSuccess;
+                          float eps, cudaStream_t stream, void* lp_base, int lp_elem, uint64_t first64) {
+  if (total64 == 0 || n_stages == 0 || first64 >= total64) return cudaSuccess;
   uint64_t total_vec4 = total64 * 16;
+  const uint64_t first_vec4 = first64 * 16;
   uint64_t per_block = (uint64_t)kUpdThreads * kUpdUnroll;
-  uint64_t need = (total_vec4 + per_block - 1) / per_block;
+  uint64_t need = (total_vec4 - first_vec4 + per_block - 1) / per_block;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -271,7 +272,7 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
   // the operand-type copy: the w_lp arena (bfloat16) unless the caller names a version ring and its element size
   if (lp_base == nullptr) { lp_base = a.w_lp; lp_elem = 2; }
   const int lp = lp_base == nullptr ? 0 : (lp_elem == 4 ? 2 : 1);
-#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps)
+#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps, first_vec4)
   if (optimizer == PM_SGDM) { if (lp == 0) PM_UPD(PM_SGDM, 0); else if (lp == 1) PM_UPD(PM_SGDM, 1); else PM_UPD(PM_SGDM, 2); }
   else { if (lp == 0) PM_UPD(PM_ADAM, 0); else if (lp == 1) PM_UPD(PM_ADAM, 1); else PM_UPD(PM_ADAM, 2); }
 #undef PM_UPD

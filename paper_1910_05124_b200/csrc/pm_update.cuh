@@ -27,7 +27,8 @@ cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperD
 // begin64/end64: stage bounds in units of 64 elements, ascending; total64 = end64[P-1].
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
-                          float eps, cudaStream_t stream, void* lp_base = nullptr, int lp_elem = 0);
+                          float eps, cudaStream_t stream, void* lp_base = nullptr, int lp_elem = 0, uint64_t first64 = 0);
+// first64: the walk over the arenas starts at this 64-element group (a launch for one stage starts at that stage's slice).
 // lp_base / lp_elem: where the operand-type copy of the new weights goes: by default the bfloat16 arena a.w_lp
 // (if there is one); microbatch-major order passes the ring arena and the operand size (2 or 4 bytes), and the
 // stages' table entries give the slot (StageDyn::lp_shift).

