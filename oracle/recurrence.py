@@ -24,6 +24,20 @@ Readings where the paper is silent:
     in microbatch order in the state precision; the update after the N-th uses step index u.  N = 1: microbatch index =
     update index.
 
+PipeMare Recompute (Appendix A.2, Appendix D): the stages form segments of consecutive stages; only the input of a
+segment's first stage is kept from the forward pass, and the activations inside a segment are computed again, just
+in time for the backward pass, with the weights the stages hold by then:
+    (u_recomp,t)_i = (w_{t - tau_recomp,i})_i  [ - (tau_fwd,i - tau_recomp,i) * delta_{t,i}  with T2 for recompute ]
+The loss of microbatch t still comes from the forward pass (u_fwd); the backward pass takes every stashed activation
+from the recomputation and reads u_bkwd as before.  Readings: tau_recomp,i is passed in by the caller; the same
+accumulator and the same T2 switch serve both corrections; during a synchronous warm-up tau_recomp = 0 as well.
+
+Which delta a correction reads: the accumulator as it stood when the corrected weights were current, i.e.
+delta_{t - tau_bkwd} with w_{t - tau_bkwd} and delta_{t - tau_recomp} with w_{t - tau_recomp}.  That is what a stage
+has at hand when the pass runs (updates t - tau .. t - 1 have not happened yet), and it is what the characteristic
+polynomials of Section 3.2 and Appendix D encode: their correction terms carry the same power of omega as the
+weights they correct.  With tau_bkwd = 0 this is delta_t, as the statement of T2 writes it.
+
 Warm-up epochs (PipeMareW, Section 4): the first `warmup` microbatches run the synchronous baseline, i.e. the same
 loop with every delay zero (standard step size, no T2 correction, delta left alone); PipeMare then starts from
 those weights and optimiser state.  Readings: the pipeline is empty at the switch, so version indices are clamped
@@ -47,13 +61,18 @@ class Result:
     def __init__(self):
         self.losses = []      # loss of microbatch t, computed from its (stale) forward weights
         self.book = []        # (t, stage index (1-based), forward version, backward version)
+        self.book_recomp = [] # (t, stage index (1-based), version the recomputation read), only with tau_recomp
         self.params = None    # final per-stage lists of tensors
         self.delta = None
         self.opt = None
 
 
-def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None, warmup=0, n_micro=1):
+def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_step=None, warmup=0, n_micro=1,
+        tau_recomp=None):
     """Run n_steps microbatches, the first `warmup` of them synchronously; n_micro microbatches per update.
+
+    tau_recomp: per stage, the recomputation delay (None: no recomputation); grad_fn then also receives
+               u_recomp=<per-stage tensors>.
 
     params0:   per stage, a list of arrays (that stage's tensors).
     grad_fn:   (t, u_fwd, u_bkwd) -> (loss, grads) with grads shaped like params0.
@@ -65,13 +84,16 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
     opt = [[U.fresh_opt_state(a, hp["optimizer"]) for a in stage] for stage in w]
     delta = [[np.zeros_like(a) for a in stage] for stage in w]
     depth = [max(tau_fwd[i], tau_bkwd[i]) + 1 for i in range(P)]
+    if tau_recomp is not None:
+        assert all(tau_bkwd[i] <= tau_recomp[i] <= tau_fwd[i] for i in range(P)), "tau_bkwd <= tau_recomp <= tau_fwd"
     # queue of versions per stage: hist[i][-1] is version t, hist[i][-1-d] is version t-d
     hist = [deque([w[i]], maxlen=depth[i]) for i in range(P)]
+    dhist = [deque([list(delta[i])], maxlen=depth[i]) for i in range(P)]      # the accumulator next to each version
     res = Result()
 
     def version(i, t, lag):
         v = max(min(warmup, t), t - lag)       # nothing older than the end of the warm-up (or version 0) exists
-        return v, hist[i][-1 - (t - v)]
+        return v, hist[i][-1 - (t - v)], dhist[i][-1 - (t - v)]
 
     assert n_micro >= 1 and (n_micro == 1 or warmup == 0), "warm-up epochs are stated for one microbatch per update"
     gacc = None
@@ -79,18 +101,25 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
         t = mb // n_micro                       # update index: versions, delays and step counters count updates
         sync = t < warmup
         u_fwd, u_bkwd = [], []
+        u_rec = None if tau_recomp is None else []
         for i in range(P):
             tf, tb = (0, 0) if sync else (tau_fwd[i], tau_bkwd[i])
-            vf, wf = version(i, t, tf)
-            vb, wb = version(i, t, tb)
+            vf, wf, _ = version(i, t, tf)
+            vb, wb, db = version(i, t, tb)
             u_fwd.append(wf)
             u_bkwd.append([U.corrected_backward_weights(a, d, tf, tb, hp["t2"])
-                           for a, d in zip(wb, delta[i])])
+                           for a, d in zip(wb, db)])
             res.book.append((mb, i + 1, vf, vb))
-        if n_micro == 1:
-            loss, grads = grad_fn(mb, u_fwd, u_bkwd)
-        else:
-            loss, grads = grad_fn(mb, u_fwd, u_bkwd, loss_scale=1.0 / n_micro)
+            if u_rec is not None:
+                tr = 0 if sync else tau_recomp[i]
+                vr, wr, dr = version(i, t, tr)
+                # T2 for recompute (Appendix D): the same accumulator, the gap to the forward delay
+                u_rec.append([U.corrected_backward_weights(a, d, tf, tr, hp["t2"]) for a, d in zip(wr, dr)])
+                res.book_recomp.append((mb, i + 1, vr))
+        kw = {} if n_micro == 1 else {"loss_scale": 1.0 / n_micro}
+        if u_rec is not None:
+            kw["u_recomp"] = u_rec
+        loss, grads = grad_fn(mb, u_fwd, u_bkwd, **kw)
         res.losses.append(loss)
         g_now = [[np.asarray(g, dtype=dtype) for g in stage] for stage in grads]
         gacc = g_now if mb % n_micro == 0 else [[a + b for a, b in zip(sa, sb)] for sa, sb in zip(gacc, g_now)]
@@ -106,6 +135,7 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
                 new_stage.append(a_new)
             w[i] = new_stage
             hist[i].append(new_stage)
+            dhist[i].append(list(delta[i]))
         if on_step is not None:
             on_step(t, w)
     res.params, res.delta, res.opt = w, delta, opt

@@ -37,9 +37,10 @@ from . import layers as L
 from .bf16 import bf16_round
 
 
-def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
+def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32", segment=None):
     """stage_specs: per stage an object with fields pre, post, act (strings).
-    data_fn: t -> (ids [T] int, targets [T] int)."""
+    data_fn: t -> (ids [T] int, targets [T] int).  segment: stages per recompute segment (the gradient function
+    then takes u_recomp)."""
     rnd = bf16_round if compute == "bf16" else L.identity
     f64 = lambda a: np.asarray(a, dtype=np.float64)
 
@@ -53,17 +54,16 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
         out["W"], out["b"] = f64(tensors[i]), f64(tensors[i + 1])
         return out
 
-    def grad_fn(t, u_fwd, u_bkwd, loss_scale=1.0):
-        data = data_fn(t)
-        ids, targets = data[0], data[-1]
-        dec_ids = data[1] if len(data) == 3 else None
+    def forward_range(lo, hi, weights, state, ids, dec_ids, stash):
+        """Forward of stages lo..hi-1 with `weights`, starting from `state` = (main, memory, pending skip tensors);
+        fills stash[i] for those stages.  Returns (state after stage hi-1, logits or None)."""
         P = len(stage_specs)
-        main, memory = None, None
-        skip_for = {}                                          # receiving stage -> (skip tensor, emitting stage)
-        stash = []
+        main, memory, skip_for = state
+        skip_for = dict(skip_for)
         logits = None
-        for i, spec in enumerate(stage_specs):
-            pf = unpack(spec, u_fwd[i])
+        for i in range(lo, hi):
+            spec = stage_specs[i]
+            pf = unpack(spec, weights[i])
             st = {}
             from_memory = getattr(spec, "src", "main") == "memory"
             x_in = memory if from_memory else main
@@ -79,7 +79,7 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
             acc = u @ rnd(pf["W"]).T + pf["b"]
             if i == P - 1:
                 logits = acc                                   # fp32 on the device, not rounded
-                stash.append(st)
+                stash[i] = st
                 break
             z = rnd(acc)
             y = rnd(L.act_fwd(z, spec.act))
@@ -104,7 +104,29 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
                 main = y
             if getattr(spec, "emit_memory", False):
                 memory = main
-            stash.append(st)
+            stash[i] = st
+        return (main, memory, skip_for), logits
+
+    def grad_fn(t, u_fwd, u_bkwd, loss_scale=1.0, u_recomp=None):
+        data = data_fn(t)
+        ids, targets = data[0], data[-1]
+        dec_ids = data[1] if len(data) == 3 else None
+        P = len(stage_specs)
+        stash = [None] * P
+        # the forward pass, stage by stage, keeping what every stage found on its inputs (main stream, memory,
+        # skip tensors on their way): the state a recompute segment starts from
+        state, state_at, logits = (None, None, {}), [], None
+        for i in range(P):
+            state_at.append(state)
+            state, lg = forward_range(i, i + 1, u_fwd, state, ids, dec_ids, stash)
+            logits = lg if lg is not None else logits
+        if u_recomp is not None:
+            # PipeMare Recompute (Appendix A.2): everything the backward pass reads is computed again, segment by
+            # segment, from what the forward pass left at the segment's first stage (tensors that cross a segment
+            # boundary -- the main input, a skip tensor, the memory -- are the forward pass's); loss and logits are not
+            starts = list(range(0, P, segment))
+            for a, b in zip(starts, starts[1:] + [P]):
+                forward_range(a, b, u_recomp, state_at[a], ids, dec_ids, stash)
 
         loss, d_main = L.cross_entropy(logits, targets, rnd, loss_scale)
         d_skip_for = {}                                        # emitting stage -> gradient of the skip tensor it sent
@@ -159,11 +181,15 @@ def make_grad_fn(stage_specs, data_fn, n_heads, seq_len, vocab, compute="f32"):
     return grad_fn
 
 
-def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0, n_micro=1):
-    """params0: per stage the list of tensors in the order [table] [gain, bias] W b."""
+def run_workload(wl, params0, data_fn, n_steps=None, dtype=np.float32, on_step=None, warmup=0, n_micro=1, segment=None):
+    """params0: per stage the list of tensors in the order [table] [gain, bias] W b.
+    segment: stages per recompute segment (None: no recomputation)."""
     from . import recurrence
+    from .mlp import recomp_delays
     hp = dict(optimizer=wl.optimizer, alpha=wl.alpha, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
               t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D)
-    grad_fn = make_grad_fn(wl.stage_specs, data_fn, wl.n_heads, wl.seq_len, wl.vocab, wl.compute)
+    grad_fn = make_grad_fn(wl.stage_specs, data_fn, wl.n_heads, wl.seq_len, wl.vocab, wl.compute, segment)
+    tau_recomp = None if segment is None else recomp_delays(wl.tau_fwd, segment, n_micro)
     return recurrence.run(params0, wl.tau_fwd, wl.tau_bkwd, grad_fn, wl.steps if n_steps is None else n_steps,
-                          hp, dtype=dtype, on_step=on_step, warmup=warmup, n_micro=n_micro)
+                          hp, dtype=dtype, on_step=on_step, warmup=warmup, n_micro=n_micro,
+                          tau_recomp=tau_recomp)

@@ -14,6 +14,7 @@
 //          w' = w - (alpha*(m'/bc1)) / (sqrt(s'/bc2) + eps)
 //   T2 (Section 3.2):      delta' = gamma*delta + (1-gamma)*(w' - w)
 #include "pm_update.cuh"
+#include "pm_update_math.cuh"
 
 namespace pm {
 
@@ -145,42 +146,8 @@ cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperD
 
 // ---- fused update ------------------------------------------------------------------------------
 
-struct UpdScalars {
-  float alpha, gamma, omg, bc1, bc2;
-  int use_delta;
-  int64_t lp_shift;
-};
-
 __device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ void st_stream(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
-
-template <int OPT>
-__device__ __forceinline__ float upd_one(float g, float w, float& m, float& s, float& dl, const UpdScalars& c,
-                                         float beta1, float beta2, float omb1, float omb2, float eps) {
-  float wn;
-  if (OPT == PM_SGDM) {
-    m = __fsub_rn(__fmul_rn(beta1, m), __fmul_rn(c.alpha, g));
-    wn = __fadd_rn(w, m);
-  } else {
-    m = __fadd_rn(__fmul_rn(beta1, m), __fmul_rn(omb1, g));
-    s = __fadd_rn(__fmul_rn(beta2, s), __fmul_rn(omb2, __fmul_rn(g, g)));
-    // Correctly rounded division and square root leave their short instruction sequence for a subroutine when an
-    // operand is zero (parameters whose gradient has been zero so far: untouched embedding rows).  Those lanes
-    // divide 1 instead and keep the zero, which is what the operation returns for them (0 / b = 0 with the sign
-    // of the zero for b > 0, sqrt(+-0) = +-0), so the results are the same bits.
-    const bool mz = m == 0.f, sz = s == 0.f;
-    const float mq = __fdiv_rn(mz ? 1.f : m, c.bc1), sq = __fdiv_rn(sz ? 1.f : s, c.bc2);
-    const float mh = mz ? m : mq, sh = sz ? s : sq;
-    const float rt = __fsqrt_rn(sh == 0.f ? 1.f : sh);
-    const float den = __fadd_rn(sh == 0.f ? sh : rt, eps);
-    const float num = __fmul_rn(c.alpha, mh);
-    const bool nz = num == 0.f && den > 0.f;
-    const float q = __fdiv_rn(nz ? 1.f : num, den);
-    wn = __fsub_rn(w, nz ? num : q);
-  }
-  if (c.use_delta) dl = __fadd_rn(__fmul_rn(c.gamma, dl), __fmul_rn(c.omg, __fsub_rn(wn, w)));
-  return wn;
-}
 
 constexpr int kUpdThreads = 256;
 constexpr int kUpdUnroll = 2;      // float4 groups per thread per array in flight

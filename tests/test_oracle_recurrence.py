@@ -397,3 +397,145 @@ def test_accumulation_happens_in_the_state_precision_in_microbatch_order():
     res64 = recurrence.run([[np.array([0.0])]], [0], [0], lambda t, uf, ub, loss_scale=1.0: (0.0, [[g[t]]]), 3, hp,
                            dtype=np.float64, n_micro=3)
     assert res64.params[0][0][0] == -(1.0 + 2.0 ** -23)
+
+
+# ---- PipeMare Recompute (Appendix A.2, Appendix D) ------------------------------------------------
+
+def recomp_char_poly(tf, tb, tr, alpha, lam, Dl, Phi, gamma):
+    """The recompute polynomial of Appendix D, built term by term (ascending powers); gamma = None: no T2 correction,
+    i.e. w_{t+1} = w_t - a(l+D) w_{t-tf} + a(D-Phi) w_{t-tb} + a Phi w_{t-tr} multiplied through by w^tf."""
+    P = np.polynomial.polynomial
+    wm1 = np.array([-1.0, 1.0])
+    wpow = lambda n: np.concatenate([np.zeros(n), [1.0]])
+    if gamma is None:
+        p = P.polymul(wm1, wpow(tf))
+        p = P.polyadd(p, [alpha * (lam + Dl)])
+        p = P.polysub(p, alpha * (Dl - Phi) * wpow(tf - tb))
+        return P.polysub(p, alpha * Phi * wpow(tf - tr))
+    wmg = np.array([-gamma, 1.0])
+    p = P.polymul(P.polymul(wm1, wmg), wpow(tf))
+    p = P.polyadd(p, alpha * (lam + Dl) * wmg)
+    p = P.polysub(p, alpha * (Dl - Phi) * P.polymul(wpow(tf - tb), wmg))
+    p = P.polyadd(p, alpha * (Dl - Phi) * (tf - tb) * (1 - gamma) * P.polymul(wpow(tf - tb), wm1))
+    p = P.polysub(p, alpha * Phi * P.polymul(wpow(tf - tr), wmg))
+    p = P.polyadd(p, alpha * Phi * (tf - tr) * (1 - gamma) * P.polymul(wpow(tf - tr), wm1))
+    return p
+
+
+def scalar_run_recomp(tf, tb, tr, grad_fn, n, hp, w0=1.0):
+    traj = []
+    recurrence.run([[np.array([w0])]], [tf], [tb], grad_fn, n, hp, dtype=np.float64, tau_recomp=[tr],
+                   on_step=lambda t, w: traj.append(float(w[0][0][0])))
+    return np.array([w0] + traj)
+
+
+def test_recompute_poly_reduces_to_the_t2_poly_when_phi_is_zero():
+    tf, tb, tr, alpha, lam, Dl, D = 10, 0, 4, 0.05, 1.0, 5.0, 0.1
+    gamma = D ** (1.0 / (tf - tb))
+    assert np.allclose(recomp_char_poly(tf, tb, tr, alpha, lam, Dl, 0.0, gamma), t2_char_poly(tf, tb, alpha, lam, Dl, gamma))
+    # and at w = 1 every delayed term cancels against the curvature: p(1) = alpha lambda (1 - gamma) for any Phi
+    P = np.polynomial.polynomial
+    assert P.polyval(1.0, recomp_char_poly(tf, tb, tr, alpha, lam, Dl, -5.0, gamma)) == pytest.approx(alpha * lam * (1 - gamma), rel=1e-10)
+
+
+@pytest.mark.filterwarnings("ignore:overflow")
+@pytest.mark.parametrize("t2", [False, True])
+@pytest.mark.parametrize("alpha", [0.02, 0.05])
+def test_recompute_growth_rate_matches_its_char_poly(alpha, t2):
+    # the setting of the appendix's figure: Delta = 10, Phi = -5, tau_fwd = 10, tau_bkwd = 1, tau_recomp = 4, lambda = 1.
+    # The polynomial is printed for the accumulator decay gamma of the pair (tau_fwd, tau_bkwd); the recurrence uses that
+    # same gamma and delta for both corrections.
+    tf, tb, tr, lam, Dl, Phi, D = 10, 1, 4, 1.0, 10.0, -5.0, 0.1
+    gamma = D ** (1.0 / (tf - tb)) if t2 else None
+    radius = np.abs(np.roots(recomp_char_poly(tf, tb, tr, alpha, lam, Dl, Phi, gamma)[::-1])).max()
+    traj = scalar_run_recomp(tf, tb, tr, quadratic_grad(lam, Dl, Phi=Phi), 1200, hp_(alpha=alpha, t2=t2, D=D))
+    assert growth_rate(traj, 400, 1200) == pytest.approx(radius, rel=2e-3)
+
+
+def test_recompute_discrepancy_correction_widens_the_stable_range():
+    # Appendix D's figure: with the correction the largest root stays below one for step sizes at which the
+    # uncorrected recompute model has already left the unit circle
+    tf, tb, tr, lam, Dl, Phi, D = 10, 1, 4, 1.0, 10.0, -5.0, 0.1
+    gamma = D ** (1.0 / (tf - tb))
+    rad = lambda a, g: np.abs(np.roots(recomp_char_poly(tf, tb, tr, a, lam, Dl, Phi, g)[::-1])).max()
+    alphas = np.linspace(0.002, 0.2, 100)
+    stable_plain = max(a for a in alphas if rad(a, None) < 1.0)
+    stable_t2 = max(a for a in alphas if rad(a, gamma) < 1.0)
+    assert stable_t2 > 1.5 * stable_plain
+
+
+def test_recompute_with_the_forward_delay_changes_nothing():
+    # tau_recomp = tau_fwd: the recomputation reads the forward pass's weights and the correction term has gap zero
+    params, grad_plain = tiny_net(seed=4, P=4)
+    rng = np.random.default_rng(4)
+    X, Y = rng.normal(size=(64, 4, 5)), rng.normal(size=(64, 4, 5))
+    g0 = make_grad_fn([["relu"]] * 4, lambda t: (X[t], Y[t]), "f32")
+    g1 = make_grad_fn([["relu"]] * 4, lambda t: (X[t], Y[t]), "f32", segment=2)
+    tf = [7, 5, 3, 1]
+    hp = hp_(alpha=0.05, t2=True, D=0.3, beta1=0.9)
+    a = recurrence.run(params, tf, [0] * 4, g0, 25, hp)
+    b = recurrence.run(params, tf, [0] * 4, g1, 25, hp, tau_recomp=tf)
+    for sa, sb in zip(a.params, b.params):
+        for x, y in zip(sa, sb):
+            assert np.array_equal(x, y)
+    assert a.losses == b.losses
+
+
+def test_recompute_gradient_by_hand_on_a_scalar_chain():
+    # two scalar stages in one segment, y = w2 w1 x, loss (y - target)^2: forward with (w1f, w2f); the recomputation
+    # gives stage 2 the input h' = w1r x; backward: dW2 = dy h', dh = dy w2b, dW1 = dh x, with dy from the forward's y
+    x, target = 0.7, -0.3
+    w1f, w2f, w1r, w2r, w1b, w2b = 1.1, -0.8, 1.3, -0.5, 0.9, -0.6
+    g = make_grad_fn([["none"], ["none"]], lambda t: (np.array([[x]]), np.array([[target]])), "f32", segment=2)
+    z = np.zeros(1)
+    mk = lambda a, b: [[np.array([[a]]), z], [np.array([[b]]), z]]
+    loss, grads = g(0, mk(w1f, w2f), mk(w1b, w2b), u_recomp=mk(w1r, w2r))
+    y = w2f * w1f * x
+    dy = 2 * (y - target)
+    assert loss == pytest.approx((y - target) ** 2)
+    assert grads[1][0][0, 0] == pytest.approx(dy * (w1r * x))
+    assert grads[0][0][0, 0] == pytest.approx(dy * w2b * x)
+    assert grads[1][1][0] == pytest.approx(dy) and grads[0][1][0] == pytest.approx(dy * w2b)
+    # a segment boundary between the stages: stage 2 starts from the forward pass's h = w1f x
+    g2 = make_grad_fn([["none"], ["none"]], lambda t: (np.array([[x]]), np.array([[target]])), "f32", segment=1)
+    _, grads2 = g2(0, mk(w1f, w2f), mk(w1b, w2b), u_recomp=mk(w1r, w2r))
+    assert grads2[1][0][0, 0] == pytest.approx(dy * (w1f * x))
+
+
+def test_recompute_delays_follow_the_segment_pipeline():
+    from oracle.mlp import recomp_delays
+    P = 16
+    tf = [2 * (P - i) + 1 for i in range(1, P + 1)]
+    tr = recomp_delays(tf, 4)
+    # Appendix A.2's example, 16 stages in 4 segments: inside a segment the j-th stage recomputes 2(S-j) steps before
+    # its gradient arrives (+ 1 for the pass itself); the last segment is the forward pass itself
+    assert tr == [7, 5, 3, 1] * 4
+    assert tr[-4:] == tf[-4:]
+    assert all(b <= a for a, b in zip(tf, tr))
+    assert recomp_delays([-(-t // 2) for t in tf], 4, 2) == [4, 3, 2, 1] * 4
+    # versions the recurrence reads: forward t - tau_fwd, recomputation t - tau_recomp, clamped at 0
+    params, _ = tiny_net(seed=1, P=4)
+    rng = np.random.default_rng(1)
+    X, Y = rng.normal(size=(64, 4, 5)), rng.normal(size=(64, 4, 5))
+    g = make_grad_fn([["relu"]] * 4, lambda t: (X[t], Y[t]), "f32", segment=2)
+    tf4 = [7, 5, 3, 1]
+    res = recurrence.run(params, tf4, [0] * 4, g, 9, hp_(), tau_recomp=recomp_delays(tf4, 2))
+    assert recomp_delays(tf4, 2) == [3, 1, 3, 1]
+    assert [r for r in res.book_recomp if r[0] == 8] == [(8, 1, 5), (8, 2, 7), (8, 3, 5), (8, 4, 7)]
+    assert [r for r in res.book_recomp if r[0] == 2] == [(2, 1, 0), (2, 2, 1), (2, 3, 0), (2, 4, 1)]
+
+
+def test_correction_reads_the_accumulator_of_the_corrected_version():
+    # scalar, tau_fwd = 3, tau_recomp = 1, constant gradient 1, SGD alpha = 0.1, D = 0.5: w_t = 1 - 0.1 t,
+    # gamma = 0.5^(1/3); delta_v by its recursion; u_recomp at step t is w_{t-1} - 2 delta_{t-1}
+    seen = []
+    def grad_fn(t, u_fwd, u_bkwd, u_recomp=None):
+        seen.append(float(u_recomp[0][0][0]))
+        return 0.0, [[np.array([1.0])]]
+    recurrence.run([[np.array([1.0])]], [3], [0], grad_fn, 5, hp_(alpha=0.1, t2=True, D=0.5), dtype=np.float64, tau_recomp=[1])
+    gamma = 0.5 ** (1.0 / 3.0)
+    delta = [0.0]
+    for v in range(1, 5):
+        delta.append(gamma * delta[-1] + (1 - gamma) * (-0.1))
+    expect = [1.0] + [(1 - 0.1 * (t - 1)) - 2 * delta[t - 1] for t in range(1, 5)]
+    assert seen == pytest.approx(expect, rel=1e-12)
