@@ -164,6 +164,20 @@ typedef struct {
                                     added in the grad arena in call order; pm_update applies update u after the N-th call
                                     and is a no-op before.  The step-size schedule, the T1 annealing and Adam's bias
                                     correction count updates. */
+  int32_t recompute_segment;     /* S: PipeMare Recompute (Appendix A.2, Appendix D); 0 = none (also when S >= n_stages).  S > 0
+                                    needs PM_MB_MAJOR (else PM_ERR_UNSUPPORTED).  Stages [kS, (k+1)S) form segment k.  The
+                                    forward pass and the loss are unchanged; before a segment's backward pass its stages run
+                                    forward once more from what the forward pass left at the segment's inputs (main input, skip
+                                    tensors and memory that cross the segment's boundary), reading the weights
+                                    w_{u - tau_recomp,i}, and the backward pass takes every stashed activation from that
+                                    recomputation.  tau_recomp,i = min(tau_fwd,i, ceil((2(S - j) + 1) / N)) for the j-th stage
+                                    (1-based) of its segment: inside a segment the recomputation precedes the backward pass
+                                    like the forward pass of an S-stage pipeline.  The last segment's backward follows its
+                                    forward at that very distance and is not recomputed (tau_recomp = tau_fwd).  With
+                                    t2_enable the recomputation reads w_v - (tau_fwd - tau_recomp) delta_v, v = u -
+                                    tau_recomp (T2 for recompute, with the accumulator as it stood with version v): the update
+                                    that produces version v also writes that copy, in the operand type, into tau_recomp + 1
+                                    further slots of the stage's version queue (counted by pm_query_bytes). */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /
@@ -257,7 +271,8 @@ pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets);
  * the forward read, backward microbatch (-1 if idle), weight version the backward read,
  * updates applied so far, forward ring slot, backward ring slot, tick.  Synchronises.
  * PM_MB_MAJOR: the record of the last completed microbatch (both passes of every stage are active); out[7] is
- * that microbatch's index, out[5] the slot of the weight-version queue the forward read. */
+ * that microbatch's index, out[5] the slot of the weight-version queue the forward read; with recompute_segment > 0
+ * out[6] is the weight version the recomputation read. */
 pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8);
 
 /* Copy losses of microbatches first_mb .. first_mb+n-1 to host_out.  The loss of microbatch

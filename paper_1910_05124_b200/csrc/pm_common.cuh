@@ -53,13 +53,18 @@ struct StageDev {
   int32_t vdepth;             // weight versions the forward pass can reach: 1 (the live weights, tick-major) or tau_f + 1
   uint32_t small_count;       // fp32 elements of a slot of s_ring (biases, LayerNorm gain and bias), a multiple of 64
   uint32_t g_soff, beta_soff; // offsets of LayerNorm gain / bias inside a slot of s_ring
+  int32_t tau_r;              // PipeMare Recompute: delay of the weights the recomputation reads (= tau_f: nothing is recomputed)
+  int32_t rdepth;             // slots of the queue of T2-corrected recompute weights behind the vdepth version slots (0: none;
+                              // the recomputation then reads plain versions)
   int32_t _pad;
   uint64_t begin, end;        // padded element range of the stage's parameters in the arenas
   // Queue of weight versions (Section 2.1: the forward pass of microbatch t reads the weights after t - tau_fwd
   // updates), microbatch-major order only.  v_ring: [vdepth][end - begin] copies of the stage's slice in the GEMM
   // operand type (what the forward GEMM and the embedding read); s_ring: [vdepth][small_count] fp32 copies of the
   // tensors the forward pass reads in fp32 (bf16 operands only; with fp32 operands v_ring holds them).  Version v
-  // sits in slot v % vdepth; the update writes version k + 1 there.
+  // sits in slot v % vdepth; the update writes version k + 1 there.  With PipeMare Recompute and T2 (Appendix D) each
+  // ring has rdepth = tau_r + 1 more slots behind those: slot vdepth + v % rdepth holds w_v - (tau_f - tau_r) delta_v,
+  // what the recomputation of microbatch v + tau_r reads, formed by the update that produced version v.
   uint64_t v_ring, s_ring;
   uint64_t tab_off, g_off, beta_off;   // arena offsets: embedding table / LayerNorm gain / LayerNorm bias
   uint64_t x_ring;            // ring: x[xdepth][T*d_in] main input (not used by an embedding stage)
@@ -98,6 +103,10 @@ struct StageDyn {
   int64_t lp_shift;           // the update writes the operand-type copy of element e to lp_base[lp_shift + e]
   int32_t accum;              // parameter gradients of this backward are ADDED to what the grad arena holds (the second to
                               // N-th microbatch of a minibatch, Section 2.1); 0: they overwrite it
+  int32_t rc_uslot;           // slot of the version rings that takes the corrected recompute weights of the new version (-1: none)
+  int64_t rc_shift;           // their operand-type copy of element e goes to lp_base[rc_shift + e]
+  int64_t r_ver;              // weight version the recomputation of the microbatch in backward reads (PipeMare Recompute)
+  float rc_gap;               // tau_fwd - tau_recomp
   int32_t _pad2;
 };
 
@@ -115,6 +124,8 @@ struct HyperDev {
   int32_t lp_elem;            // bytes of an element of the version rings' operand copy (2 or 4)
   int32_t n_micro;            // N: microbatches per update (microbatch-major order; 1 elsewhere)
   int32_t entry_period;       // tick-major order: a microbatch enters every entry_period ticks (1: every tick)
+  int32_t segment;            // PipeMare Recompute: stages per segment (0: no recomputation)
+  int32_t _pad;
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks

@@ -46,7 +46,9 @@ struct Layout {
   bool mb = false;
   bool queue = false;                   // the forward pass reads its weights from per-stage version queues (mb, or entry period > 1)
   int32_t E = 1;                        // tick-major order: ticks between two entering microbatches
-  int32_t n_tables = 1;                 // per-tick tables: 1, or 2P + 1 (one per sub-tick and one for the grouped launches)
+  int32_t n_tables = 1;                 // per-tick tables: 1, or 2P + 1 (one per sub-tick and one for the grouped launches),
+                                        // with PipeMare Recompute one more for the recomputation and one per segment
+  int32_t segment = 0;                  // PipeMare Recompute: stages per segment (0: none)
   std::vector<SmallSeg> segs;           // fp32 tensors the forward pass reads, per version ring slot (bf16 operands)
   uint64_t off_segs = 0;
   std::vector<int32_t> pre_idx, ln_idx, embed_idx, res_idx;   // position of a stage in the stage lists (-1: not in it)
@@ -84,11 +86,20 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     return PM_ERR_UNSUPPORTED;
   }
   L.mb = mb;
+  if (cfg->recompute_segment < 0) { err = "recompute_segment must be >= 0"; return PM_ERR_INVALID_ARG; }
+  if (cfg->recompute_segment > 0 && !mb) {
+    // the recomputation reads weights of its own delay tau_recomp: a third version per stage and microbatch, which the
+    // queue of weight versions has and a tick schedule with one live version does not
+    err = "recompute_segment > 0 (PipeMare Recompute) is built for PM_MB_MAJOR order";
+    return PM_ERR_UNSUPPORTED;
+  }
+  const int S = cfg->recompute_segment >= P ? 0 : cfg->recompute_segment;    // one segment covering everything: the forward pass itself
+  L.segment = S;
   if (cfg->entry_period < 0 || cfg->entry_period > 2 * P) { err = "entry_period must be in [0, 2 * n_stages]"; return PM_ERR_INVALID_ARG; }
   const int E = (!mb && cfg->entry_period > 1) ? cfg->entry_period : 1;
   const bool queue = mb || E > 1;
   L.E = E; L.queue = queue;
-  L.n_tables = mb ? 2 * P + 1 : 1;
+  L.n_tables = mb ? mb_table_count(P, S) : 1;
   const uint64_t esz = cfg->compute_dtype == PM_F32 ? 4 : 2;
   const uint64_t T = (uint64_t)cfg->microbatch;
   const bool ce = cfg->loss == PM_LOSS_CE;
@@ -126,6 +137,18 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     // the delay is the queue of weight versions
     s.vdepth = 1;
     if (mb) { s.depth = 1; s.xdepth = 1; s.vdepth = s.tau_f + 1; }
+    // PipeMare Recompute (Appendix A.2): inside a segment the recomputation runs ahead of the backward pass like the
+    // forward pass of a pipeline of that many stages, tau_recomp = ceil((2(S - j) + 1) / N) for the j-th stage of a
+    // segment of S, never above tau_fwd; the last segment's backward follows its forward at that very distance, so
+    // nothing is recomputed there.  With T2 a stage whose recomputation is younger than its forward keeps a queue of
+    // tau_recomp + 1 corrected versions (Appendix D) behind its version slots.
+    s.tau_r = s.tau_f; s.rdepth = 0;
+    if (S > 0) {
+      const int seg_end = std::min(P, (p / S + 1) * S);
+      const int nm = cfg->n_micro > 1 ? cfg->n_micro : 1;
+      if (seg_end < P) s.tau_r = std::min(s.tau_f, (2 * (seg_end - 1 - p) + 1 + nm - 1) / nm);
+      if (cfg->t2_enable && s.tau_r < s.tau_f) s.rdepth = s.tau_r + 1;
+    }
     if (E > 1) {
       // a microbatch every E ticks: a stash written at tick mE + i is read at tick mE + i + tau, so floor(tau / E) + 1
       // microbatches are alive in a stage; the input ring keeps one more (it is also the forward mailbox) and another
@@ -271,14 +294,14 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (queue) {
       // queue of weight versions: the whole slice in the operand type, and (bf16 operands) the fp32 tensors the forward
       // pass reads -- LayerNorm gain and bias, Linear biases -- packed into slots of small_count floats
-      s.v_ring = ring; ring = align_up(ring + (uint64_t)s.vdepth * (s.end - s.begin) * esz, 256);
+      s.v_ring = ring; ring = align_up(ring + (uint64_t)(s.vdepth + s.rdepth) * (s.end - s.begin) * esz, 256);
       uint32_t so = 0;
       auto seg = [&](uint64_t arena_off, uint64_t n, uint32_t* soff) {
         *soff = so;
         const uint32_t padded = (uint32_t)align_up(n, PM_ALIGN_ELEMS);
         for (uint32_t o = 0; o < padded; o += 2048) {                           // pieces of at most 2048 floats: one block copies a piece
           const uint32_t cnt = std::min<uint32_t>(2048, padded - o);
-          L.segs.push_back(SmallSeg{arena_off + o, 0, cnt, 0, p, (int32_t)(so + o)});   // ring_off, slot_stride filled below
+          L.segs.push_back(SmallSeg{arena_off + o, 0, cnt, 0, p, (int32_t)(so + o)});   // ring_off, slot_stride, rc_base filled below
         }
         so += padded;
       };
@@ -286,8 +309,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
         if (s.pre == PRE_LN) { seg(s.g_off, (uint64_t)s.d_in, &s.g_soff); seg(s.beta_off, (uint64_t)s.d_in, &s.beta_soff); }
         for (int l = 0; l < s.n_lin; ++l) seg(s.lin[l].b_off, (uint64_t)s.lin[l].n_out, &s.lin[l].b_soff);
         s.small_count = so;
-        s.s_ring = ring; ring = align_up(ring + (uint64_t)s.vdepth * so * 4, 256);
-        for (auto& g : L.segs) if (g.stage == p) { g.ring_off = s.s_ring + 4ull * (uint32_t)g._pad; g.slot_stride = so; g._pad = 0; }
+        s.s_ring = ring; ring = align_up(ring + (uint64_t)(s.vdepth + s.rdepth) * so * 4, 256);
+        for (auto& g : L.segs) if (g.stage == p) { g.ring_off = s.s_ring + 4ull * (uint32_t)g.rc_base; g.slot_stride = so; g.rc_base = s.rdepth > 0 ? s.vdepth : -1; }
       }
     }
     L.max_lin = std::max(L.max_lin, s.n_lin);
@@ -304,6 +327,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     }
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
     L.sched[p].vdepth = s.vdepth; L.sched[p].begin = s.begin; L.sched[p].count = s.end - s.begin; L.sched[p].v_ring = s.v_ring;
+    L.sched[p].tau_r = s.tau_r; L.sched[p].rdepth = s.rdepth;
   }
   for (int p = 0; p < P; ++p) {
     L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
@@ -586,6 +610,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.entry_period = L.E;
   c->hp.mb_major = L.queue ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
   c->hp.n_micro = cfg->n_micro > 1 ? cfg->n_micro : 1;
+  c->hp.segment = L.segment;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -668,9 +693,12 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
     for (int p = 0; p < P && e == cudaSuccess; ++p) {
       const StageDev& s = c->L.st[p];
       const void* src = f32 ? (const void*)(arenas->w + s.begin) : (const void*)(arenas->w_lp + s.begin);
-      e = cudaMemcpyAsync(t.ring + s.v_ring, src, (s.end - s.begin) * (f32 ? 4 : 2), cudaMemcpyDeviceToDevice, c->stream);
+      const uint64_t bytes = (s.end - s.begin) * (f32 ? 4 : 2);
+      e = cudaMemcpyAsync(t.ring + s.v_ring, src, bytes, cudaMemcpyDeviceToDevice, c->stream);
+      // corrected recompute weights of version 0: delta_0 = 0, so the initial weights themselves
+      if (e == cudaSuccess && s.rdepth > 0) e = cudaMemcpyAsync(t.ring + s.v_ring + (uint64_t)s.vdepth * bytes, src, bytes, cudaMemcpyDeviceToDevice, c->stream);
     }
-    if (e == cudaSuccess) e = launch_push_small(c->a.w, t.ring, (const SmallSeg*)(c->ws + L.off_segs), (int)c->L.segs.size(), t.dyn, 0, c->stream);
+    if (e == cudaSuccess) e = launch_push_small(c->a.w, c->a.delta, t.ring, (const SmallSeg*)(c->ws + L.off_segs), (int)c->L.segs.size(), t.dyn, 0, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "weight-version queue set-up"); pm_destroy(c); return r; }
   }
@@ -856,6 +884,16 @@ static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets
   return PM_OK;
 }
 
+// The grouped launches that close a backward pass over the stages table `table` marks (all of them, or one recompute
+// segment): the weight gradients as one launch.
+static pm_status grouped_wgrad(pm_ctx* ctx, int table) {
+  const int dt = ctx->cfg.compute_dtype;
+  TickArgs ta = mb_args(ctx, table, -1);
+  prof_begin(ctx, PM_PROF_WGRAD);
+  cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
+  return check(ctx, e, "wgrad GEMM");
+}
+
 static pm_status mb_backward(pm_ctx* ctx) {
   const int dt = ctx->cfg.compute_dtype;
   const int P = ctx->cfg.n_stages;
@@ -863,21 +901,33 @@ static pm_status mb_backward(pm_ctx* ctx) {
   // gradients of all stages run as ONE grouped launch (the tick schedule's launch, which fills the GPU); stages
   // with several Linears reuse their dz scratch from level to level and form each weight gradient on the spot.
   const bool grouped = ctx->L.max_lin == 1;
+  // PipeMare Recompute (Appendix A.2): segments from the last to the first; before a segment's backward its stages run
+  // forward again from the input the forward pass left at the segment's first stage, with the recompute weights
+  // (table 2P + 1), overwriting every stash the backward reads.  The last segment's backward follows its forward
+  // directly: nothing to recompute.  A segment's weight gradients are formed before the next (earlier) segment is
+  // recomputed, because that recomputation overwrites the input of this segment's first stage.
+  const int S = ctx->L.segment;
+  const int n_seg = S > 0 ? (P + S - 1) / S : 1;
   pm_status s = run_phase(ctx, ctx->g_bwd, [&]() -> pm_status {
     pm_status s;
-    for (int p = P - 1; p >= 0; --p) {
-      TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
-      ta.defer_finish = grouped ? 1 : 0;        // the partial sums of bias and LayerNorm gradients are added up once, below
-      if ((s = stage_backward(ctx, ta, p, grouped)) != PM_OK) return s;
+    for (int k = n_seg - 1; k >= 0; --k) {
+      const int lo = S > 0 ? k * S : 0, hi = S > 0 ? std::min(P, lo + S) : P;
+      if (S > 0 && k < n_seg - 1)
+        for (int p = lo; p < hi; ++p)
+          if ((s = stage_forward(ctx, mb_args(ctx, 2 * P + 1, p), p)) != PM_OK) return s;
+      for (int p = hi - 1; p >= lo; --p) {
+        TickArgs ta = mb_args(ctx, 2 * P - 1 - p, p);
+        ta.defer_finish = grouped ? 1 : 0;      // the partial sums of bias and LayerNorm gradients are added up once, below
+        if ((s = stage_backward(ctx, ta, p, grouped)) != PM_OK) return s;
+      }
+      if (grouped && S > 0 && (s = grouped_wgrad(ctx, 2 * P + 2 + k)) != PM_OK) return s;
     }
     if (grouped) {
       TickArgs ta = mb_args(ctx, 2 * P, -1);
       ta.colsum_only = 1; ta.defer_finish = 1;                  // bias gradients of the Linears without activation, all stages at once
       if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, 0, ctx->ls), "bias gradient column sums", actbwd_launches(ta)))) != PM_OK) return s;
       ta.colsum_only = 0; ta.defer_finish = 0;
-      prof_begin(ctx, PM_PROF_WGRAD);
-      cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
-      if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+      if (S == 0 && (s = grouped_wgrad(ctx, 2 * P)) != PM_OK) return s;
       const int n_fin = deferred_finish_launches(ta);
       if (n_fin && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_deferred_finish(ta, dt, ctx->ls), "bias / LayerNorm gradient sums", n_fin))) != PM_OK) return s;
     }
@@ -904,7 +954,7 @@ static pm_status mb_update(pm_ctx* ctx) {
     pm_status s = check(ctx, e, "update");
     if (s != PM_OK || ctx->L.segs.empty()) return s;
     prof_begin(ctx, PM_PROF_UPDATE);
-    e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(), dyn_all, -1, ctx->ls);
+    e = launch_push_small(ctx->a.w, ctx->a.delta, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(), dyn_all, -1, ctx->ls);
     return check(ctx, e, "weight-version push");
   });
   if (s != PM_OK) return s;
@@ -981,7 +1031,7 @@ static pm_status sparse_update_phase(pm_ctx* ctx) {
       if (ctx->seg_count[p] > 0) {
         prof_begin(ctx, PM_PROF_UPDATE);
         // the segments name their stage by its index in the whole table: hand the kernel the table's base
-        e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs) + ctx->seg_first[p], ctx->seg_count[p],
+        e = launch_push_small(ctx->a.w, ctx->a.delta, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs) + ctx->seg_first[p], ctx->seg_count[p],
                               (const StageDyn*)(ctx->ws + ctx->L.off_dyn), -1, ctx->ls);
         if ((s = check(ctx, e, "weight-version push")) != PM_OK) return s;
       }
@@ -1098,7 +1148,7 @@ pm_status pm_update(pm_ctx* ctx) {
       pm_status s = check(ctx, e, "update");
       if (s != PM_OK || !ctx->L.queue || ctx->L.segs.empty()) return s;
       prof_begin(ctx, PM_PROF_UPDATE);                                 // fp32 copies of the updated stages' small tensors into their queues
-      e = launch_push_small(ctx->a.w, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(),
+      e = launch_push_small(ctx->a.w, ctx->a.delta, ctx->ta.ring, (const SmallSeg*)(ctx->ws + ctx->L.off_segs), (int)ctx->L.segs.size(),
                             (const StageDyn*)(ctx->ws + ctx->L.off_dyn), -1, ctx->ls);
       return check(ctx, e, "weight-version push");
     });
@@ -1147,7 +1197,7 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bookkeeping read-back");
     if (pm_status ds = check_device_status(ctx)) return ds;
     out8[0] = df.f_mb; out8[1] = df.f_ver; out8[2] = db.b_mb; out8[3] = db.b_ver; out8[4] = n;
-    out8[5] = df.f_vslot; out8[6] = db.b_slot; out8[7] = ctx->n_fed - 1;
+    out8[5] = df.f_vslot; out8[6] = ctx->L.segment > 0 ? db.r_ver : (int64_t)db.b_slot; out8[7] = ctx->n_fed - 1;
     return PM_OK;
   }
   if (e == cudaSuccess) e = cudaMemcpy(&d, ctx->ws + ctx->L.off_dyn + sizeof(StageDyn) * stage, sizeof(StageDyn), cudaMemcpyDeviceToHost);

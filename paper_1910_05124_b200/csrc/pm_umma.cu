@@ -1793,7 +1793,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
           uint32_t box3[3] = {TILE_K, TILE_N, 1};
           void* wbase = (void*)(t.a.w_lp + L.w_off);
           if (t.mb_major) {
-            dims3[2] = (uint64_t)s.vdepth; strides3[1] = (s.end - s.begin) * 2;
+            dims3[2] = (uint64_t)(s.vdepth + s.rdepth); strides3[1] = (s.end - s.begin) * 2;
             wbase = (void*)(reinterpret_cast<__nv_bfloat16*>(t.ring + s.v_ring) + (L.w_off - s.begin));
           }
           okm = okm && encode(fn, m + MAP_W_K, 0, wbase, 3, dims3, strides3, box3, err);

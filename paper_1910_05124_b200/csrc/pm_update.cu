@@ -31,6 +31,7 @@ __device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t ti
   StageDyn d;
   d.tick = tick;
   d.accum = 0; d._pad2 = 0;
+  d.rc_uslot = -1; d.rc_shift = 0; d.r_ver = fver; d.rc_gap = 0.f;
   if (kb == -2) kb = b;                               // update index the microbatch in backward belongs to (N = 1: itself)
   const bool fa = a >= 0, ba = b >= 0;
   d.f_mb = a; d.b_mb = b; d.k = k;
@@ -51,6 +52,12 @@ __device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t ti
   d.f_vslot = s.vdepth > 1 ? (int32_t)(fver % s.vdepth) : 0;
   d.u_vslot = s.vdepth > 1 ? (int32_t)((ver + 1) % s.vdepth) : 0;
   d.lp_shift = hp.mb_major ? (int64_t)(s.v_ring / (uint64_t)hp.lp_elem) + (int64_t)d.u_vslot * (int64_t)s.count - (int64_t)s.begin : 0;
+  if (hp.mb_major && s.rdepth > 0) {
+    // corrected recompute weights of version ver + 1: slot vdepth + (ver + 1) % rdepth of the same rings
+    d.rc_uslot = s.vdepth + (int32_t)((ver + 1) % s.rdepth);
+    d.rc_shift = (int64_t)(s.v_ring / (uint64_t)hp.lp_elem) + (int64_t)d.rc_uslot * (int64_t)s.count - (int64_t)s.begin;
+    d.rc_gap = (float)(s.tau_f - s.tau_r);
+  }
   d.active_update = k >= 0 ? 1 : 0;
   d.alpha = 0.f; d.gamma = 0.f; d.one_minus_gamma = 1.f; d.bc1 = 1.f; d.bc2 = 1.f; d.use_delta = 0;
   const int64_t kk = k >= 0 ? k : kb;                 // the update index of the microbatch in backward
@@ -131,15 +138,31 @@ __global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDy
   if (u < hp.warm) fver = u; else if (fver < hp.warm) fver = hp.warm;
   if (fver < 0) fver = 0;
   StageDyn d;
+  // PipeMare Recompute (Appendix A.2, Appendix D): the version the recomputation reads, clamped like the forward's
+  int64_t rver = u - s.tau_r;
+  if (u < hp.warm) rver = u; else if (rver < hp.warm) rver = hp.warm;
+  if (rver < 0) rver = 0;
+  const int seg = hp.segment > 0 ? i / hp.segment : 0;
   if (v < 2 * P) d = make_dyn(s, hp, base + v, v == i ? t : -1, v == 2 * P - 1 - i ? t : -1, -1, u, fver, true, u);
-  else d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, (t % N == N - 1) ? u : -1, u, fver, true, u);
+  else if (v == 2 * P) d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, (t % N == N - 1) ? u : -1, u, fver, true, u);
+  else if (v == 2 * P + 1) {
+    // the stage's forward entry again (same virtual tick, so the same mailbox and skip slots), reading the recompute
+    // weights: the corrected queue behind the version slots when the stage keeps one, else the plain version
+    d = make_dyn(s, hp, base + i, t, -1, -1, u, fver, true, u);
+    d.f_vslot = s.rdepth > 0 ? s.vdepth + (int32_t)(rver % s.rdepth) : (s.vdepth > 1 ? (int32_t)(rver % s.vdepth) : 0);
+  } else {
+    // backward entries of one segment alone: the grouped weight-gradient launch that follows the segment's backward
+    const bool mine = seg == v - (2 * P + 2);
+    d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, mine ? t : -1, -1, u, fver, true, u);
+  }
+  d.r_ver = rver;
   d.accum = (t % N != 0) ? 1 : 0;
   tables[(size_t)v * P + i] = d;
 }
 
 cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream) {
   const int threads = 128;
-  dim3 grid((hp.n_stages + threads - 1) / threads, 2 * hp.n_stages + 1);
+  dim3 grid((hp.n_stages + threads - 1) / threads, mb_table_count(hp.n_stages, hp.segment));
   schedule_mb_kernel<<<grid, threads, 0, stream>>>(sched, tables, hp, t);
   return cudaGetLastError();
 }
@@ -189,8 +212,8 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
         const StageDyn& d = dyn[stage[u]];
         sc[u].alpha = d.alpha; sc[u].gamma = d.gamma; sc[u].omg = d.one_minus_gamma;
         sc[u].bc1 = d.bc1; sc[u].bc2 = d.bc2; sc[u].use_delta = d.use_delta;
-        if (LP != 0) sc[u].lp_shift = d.lp_shift;
-        if (sc[u].use_delta) dl[u] = ld_stream(a.delta + e);
+        if (LP != 0) { sc[u].lp_shift = d.lp_shift; sc[u].rc_shift = d.rc_uslot >= 0 ? d.rc_shift : -1; sc[u].rc_gap = d.rc_gap; }
+        if (sc[u].use_delta || (LP != 0 && sc[u].rc_shift >= 0)) dl[u] = ld_stream(a.delta + e);
         if (OPT == PM_ADAM) s[u] = ld_stream(a.s + e);
       }
     }
@@ -216,6 +239,24 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(lp_base) + (sc[u].lp_shift + (int64_t)e)) = packed;   // re-read by a later forward: default caching
       } else if (LP == 2) {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(lp_base) + (sc[u].lp_shift + (int64_t)e)) = wn;
+      }
+      if (LP != 0 && sc[u].rc_shift >= 0) {
+        // T2 for recompute (Appendix D): the weights a recomputation tau_recomp updates from now reads, corrected with the
+        // accumulator as it stands with this version: w' - (tau_fwd - tau_recomp) * delta'
+        const float gp = sc[u].rc_gap;
+        float4 r;
+        r.x = __fsub_rn(wn.x, __fmul_rn(gp, dl[u].x)); r.y = __fsub_rn(wn.y, __fmul_rn(gp, dl[u].y));
+        r.z = __fsub_rn(wn.z, __fmul_rn(gp, dl[u].z)); r.w = __fsub_rn(wn.w, __fmul_rn(gp, dl[u].w));
+        if (LP == 1) {
+          __nv_bfloat162 lo2 = __floats2bfloat162_rn(r.x, r.y);
+          __nv_bfloat162 hi2 = __floats2bfloat162_rn(r.z, r.w);
+          uint2 packed;
+          packed.x = *reinterpret_cast<uint32_t*>(&lo2);
+          packed.y = *reinterpret_cast<uint32_t*>(&hi2);
+          *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(lp_base) + (sc[u].rc_shift + (int64_t)e)) = packed;
+        } else {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(lp_base) + (sc[u].rc_shift + (int64_t)e)) = r;
+        }
       }
       if ((uint32_t)(v[u] >> 4) == sb[stage[u]] && (v[u] & 15) == 0) nupd[stage[u]] += 1;
     }
@@ -249,23 +290,40 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
 // ---- fp32 copies of the small forward-read tensors into the version rings -------------------------------------
 // With bfloat16 operands the forward pass still reads biases and LayerNorm parameters in fp32; in microbatch-major
 // order their versions sit in a ring of their own, filled here from the master weights after every update.
-__global__ void __launch_bounds__(128) push_small_kernel(const float* __restrict__ w, char* __restrict__ ring, const SmallSeg* __restrict__ segs,
-                                                         int n_segs, const StageDyn* __restrict__ dyn, int slot_override) {
+__global__ void __launch_bounds__(128) push_small_kernel(const float* __restrict__ w, const float* __restrict__ delta, char* __restrict__ ring,
+                                                         const SmallSeg* __restrict__ segs, int n_segs, const StageDyn* __restrict__ dyn, int slot_override) {
   for (int sg = blockIdx.x; sg < n_segs; sg += gridDim.x) {
     const SmallSeg g = segs[sg];
     if (slot_override < 0 && !dyn[g.stage].active_update) continue;          // the stage was not updated this tick
     const int slot = slot_override >= 0 ? slot_override : dyn[g.stage].u_vslot;
-    float* dst = reinterpret_cast<float*>(ring + g.ring_off) + (uint64_t)slot * g.slot_stride;
+    float* base = reinterpret_cast<float*>(ring + g.ring_off);
+    float* dst = base + (uint64_t)slot * g.slot_stride;
     const float* src = w + g.arena_off;
-    for (uint32_t i = threadIdx.x * 4; i < g.count; i += blockDim.x * 4)
-      *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(src + i);
+    // corrected recompute weights of the same version (T2 for recompute, Appendix D): w - (tau_fwd - tau_recomp) * delta
+    const int rslot = g.rc_base < 0 ? -1 : (slot_override >= 0 ? g.rc_base + slot_override : dyn[g.stage].rc_uslot);
+    float* rdst = rslot >= 0 ? base + (uint64_t)rslot * g.slot_stride : nullptr;
+    const float gap = (rslot >= 0 && slot_override < 0) ? dyn[g.stage].rc_gap : 0.f;
+    const float* dl = delta + g.arena_off;
+    for (uint32_t i = threadIdx.x * 4; i < g.count; i += blockDim.x * 4) {
+      const float4 v = *reinterpret_cast<const float4*>(src + i);
+      *reinterpret_cast<float4*>(dst + i) = v;
+      if (rdst) {
+        float4 r = v;
+        if (slot_override < 0) {
+          const float4 d4 = *reinterpret_cast<const float4*>(dl + i);
+          r.x = __fsub_rn(v.x, __fmul_rn(gap, d4.x)); r.y = __fsub_rn(v.y, __fmul_rn(gap, d4.y));
+          r.z = __fsub_rn(v.z, __fmul_rn(gap, d4.z)); r.w = __fsub_rn(v.w, __fmul_rn(gap, d4.w));
+        }
+        *reinterpret_cast<float4*>(rdst + i) = r;
+      }
+    }
   }
 }
 
-cudaError_t launch_push_small(const float* w, char* ring, const SmallSeg* segs, int n_segs, const StageDyn* dyn,
+cudaError_t launch_push_small(const float* w, const float* delta, char* ring, const SmallSeg* segs, int n_segs, const StageDyn* dyn,
                               int slot_override, cudaStream_t stream) {
   if (n_segs == 0) return cudaSuccess;
-  push_small_kernel<<<n_segs < 1184 ? n_segs : 1184, 128, 0, stream>>>(w, ring, segs, n_segs, dyn, slot_override);
+  push_small_kernel<<<n_segs < 1184 ? n_segs : 1184, 128, 0, stream>>>(w, delta, ring, segs, n_segs, dyn, slot_override);
   return cudaGetLastError();
 }
 

@@ -12,16 +12,20 @@ struct StageSched {
   // byte offset of its operand-type ring in the ring arena
   int32_t vdepth, _pad;
   uint64_t begin, count, v_ring;
+  int32_t tau_r, rdepth;                // PipeMare Recompute: delay of the recomputation's weights, slots of their corrected queue
 };
 
 // Launches the scheduler for pipeline tick `tick` with `n_fed` microbatches fed so far.
 // flat_k >= 0 selects the stand-alone update mode: every stage is at update index flat_k.
 cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageDyn* dyn, HyperDev hp,
                             int64_t tick, int64_t n_fed, int64_t flat_k, cudaStream_t stream);
-// Microbatch-major order: fills the 2P + 1 tables of microbatch t ([2P + 1][P] entries): table v for the launches of
+// Microbatch-major order: fills the tables of microbatch t ([n_tables][P] entries): table v < 2P for the launches of
 // sub-tick v (stage i forward at v = i, backward at v = 2P - 1 - i), table 2P for the grouped weight-gradient launch
-// and the update.
+// and the update.  With PipeMare Recompute (hp.segment > 0) table 2P + 1 holds every stage's recomputation (its forward
+// entry with the recompute weights' slot) and table 2P + 2 + k the backward entries of segment k alone (the grouped
+// weight-gradient launch of that segment).
 cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream);
+inline int mb_table_count(int P, int segment) { return 2 * P + 1 + (segment > 0 ? 1 + (P + segment - 1) / segment : 0); }
 
 // Launches the fused update over all stages whose dyn[i].active_update is set.
 // begin64/end64: stage bounds in units of 64 elements, ascending; total64 = end64[P-1].
@@ -36,9 +40,12 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
 // One fp32 tensor the forward pass reads (a bias, a LayerNorm gain or bias): `count` elements (a multiple of 64,
 // padding included) at arena_off of the master weights; its versions sit at ring_off (bytes, slot 0) of the ring
 // arena, slot_stride floats apart.
-struct SmallSeg { uint64_t arena_off, ring_off; uint32_t count, slot_stride; int32_t stage, _pad; };
-// Copies every segment from the master weights into slot dyn[stage].u_vslot of its ring (slot_override >= 0: that slot).
-cudaError_t launch_push_small(const float* w, char* ring, const SmallSeg* segs, int n_segs, const StageDyn* dyn,
+// rc_base: first slot of the stage's corrected recompute weights (= its vdepth), -1 when it keeps none.
+struct SmallSeg { uint64_t arena_off, ring_off; uint32_t count, slot_stride; int32_t stage, rc_base; };
+// Copies every segment from the master weights into slot dyn[stage].u_vslot of its ring and, for a stage with a queue of
+// corrected recompute weights, w - dyn[stage].rc_gap * delta into slot dyn[stage].rc_uslot.  slot_override >= 0 (the
+// initial fill, delta = 0): plain copies into that slot and into rc_base + slot_override.
+cudaError_t launch_push_small(const float* w, const float* delta, char* ring, const SmallSeg* segs, int n_segs, const StageDyn* dyn,
                               int slot_override, cudaStream_t stream);
 
 }  // namespace pm

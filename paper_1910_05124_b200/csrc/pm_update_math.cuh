@@ -13,6 +13,8 @@ struct UpdScalars {
   float alpha, gamma, omg, bc1, bc2;
   int use_delta;
   int64_t lp_shift;
+  int64_t rc_shift;     // element shift of the corrected recompute copy of the new weights, -1: none
+  float rc_gap;         // tau_fwd - tau_recomp
 };
 
 

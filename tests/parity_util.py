@@ -4,16 +4,19 @@ import numpy as np
 import pm_inputs as I
 
 
-def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1, entry_period=1):
+def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1, entry_period=1,
+                     segment=0, book_recomp=None):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
     The first `warmup` microbatches enter 2P ticks apart (synchronous warm-up), the rest one per tick.
     loop_order "mb_major": one call of pm_step per microbatch, nothing to drain.
+    segment: stages per recompute segment (PipeMare Recompute); book_recomp, a dict, then receives
+    (microbatch, stage 1-based) -> version the recomputation read.
     """
     import torch
     import paper_1910_05124_b200 as pm
-    pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro, entry_period=entry_period)
+    pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro, entry_period=entry_period, recompute_segment=segment)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
@@ -59,6 +62,8 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
                 if b_mb >= 0:
                     book.setdefault((b_mb, p + 1), [None, None])[1] = b_ver
                     assert n_upd == b_ver + (1 if (b_mb + 1) % n_micro == 0 else 0)      # the update follows the N-th microbatch
+                    if book_recomp is not None:
+                        book_recomp[(b_mb, p + 1)] = b_slot                              # with recompute: the version it read
     losses = pipe.pm_get_losses(0, n_steps)
     return pipe, losses, book
 
@@ -67,14 +72,14 @@ def is_encdec(wl):
     return any(sp.pre == "embed_dec" for sp in wl.stage_specs)
 
 
-def run_oracle(wl, params0, n_steps, teacher=None, warmup=0, n_micro=1):
+def run_oracle(wl, params0, n_steps, teacher=None, warmup=0, n_micro=1, segment=None):
     if wl.kind == "encoder":
         from oracle import transformer
         data = (lambda t: I.seq2seq_batch(wl, t)) if is_encdec(wl) else (lambda t: I.token_batch(wl, t))
-        return transformer.run_workload(wl, params0, data, n_steps=n_steps, warmup=warmup, n_micro=n_micro)
+        return transformer.run_workload(wl, params0, data, n_steps=n_steps, warmup=warmup, n_micro=n_micro, segment=segment)
     from oracle.mlp import run_workload
     teacher = I.teacher_params(wl) if teacher is None else teacher
-    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps, warmup=warmup, n_micro=n_micro)
+    return run_workload(wl, params0, lambda t: I.batch(wl, t, teacher), n_steps=n_steps, warmup=warmup, n_micro=n_micro, segment=segment)
 
 
 def max_rel_err(a, b):
