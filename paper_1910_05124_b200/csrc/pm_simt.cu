@@ -239,14 +239,23 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
 constexpr int kFinCols = 32, kFinMaxPer = 32;            // columns per block; partials per warp held in registers at a time
 
 __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
-  const int p = stage_of_block(t, blockIdx.y);
+  // the grid follows the list of 256-column blocks of the activation-backward launch (kActColsV / kFinCols blocks
+  // here per entry there), so no block falls outside its Linear's columns however unequal the widths are
+  constexpr int kPer = kActColsV / kFinCols;
+  const int* __restrict__ start = t.act_start + (size_t)lvl * (t.P + 1);
+  const int blk = (int)(blockIdx.x / kPer) + t.act_first[lvl];
+  int lo = 0, hi = t.P - 1;
+  if (t.sel_p >= 0) lo = hi = t.sel_p;
+  while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (start[mid] <= blk) lo = mid; else hi = mid - 1; }
+  const int p = lo;
   const StageDyn& d = t.dyn[p];
   const StageDev& s = t.st[p];
   if (d.b_mb < 0 || lvl >= s.n_lin) return;
   const LinDev& L = s.lin[lvl];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c = blockIdx.x * kFinCols + lane;
-  if (blockIdx.x * kFinCols >= L.n_out) return;
+  const int cb = (blk - start[p]) * kActColsV + (int)(blockIdx.x % kPer) * kFinCols;
+  const int c = cb + lane;
+  if (cb >= L.n_out) return;
   const uint64_t ps = 2 * (uint64_t)t.max_dim;
   const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * ps + (c < L.n_out ? c : 0);
   float sum = 0.f;
@@ -274,8 +283,8 @@ int deferred_finish_launches(const TickArgs& t) { return (t.row_chunks > 1 ? t.m
 cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t stream) {
   (void)dtype;
   if (t.row_chunks > 1) {
-    dim3 g2((t.max_dim + kFinCols - 1) / kFinCols, t.P);
-    for (int lvl = 0; lvl < t.max_lin; ++lvl) bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
+    for (int lvl = 0; lvl < t.max_lin; ++lvl)
+      if (t.act_blocks[lvl] > 0) bias_finish_kernel<<<t.act_blocks[lvl] * (kActColsV / kFinCols), 256, 0, stream>>>(t, lvl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -294,8 +303,7 @@ cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t st
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || t.row_chunks == 1 || t.defer_finish) return e;
-  dim3 g2((t.max_dim + kFinCols - 1) / kFinCols, t.sel_p >= 0 ? 1 : t.P);
-  bias_finish_kernel<<<g2, 256, 0, stream>>>(t, lvl);
+  bias_finish_kernel<<<t.act_blocks[lvl] * (kActColsV / kFinCols), 256, 0, stream>>>(t, lvl);
   return cudaGetLastError();
 }
 
