@@ -166,6 +166,10 @@ WORKLOADS = {
                "GPU (166 GB); same widths, sequences and optimiser as cfg5",
 }
 # loop order each workload is measured in: config 5 only fits one GPU with per-stage weight-version queues
+# workloads that can take the update of the Linear matrices in the weight-gradient GEMM's epilogue (bf16, one Linear per
+# stage): measured slower than the separate update kernel with Adam (8 epilogue warps per SM cannot issue the update's
+# arithmetic fast enough), so it is off unless --fuse is given
+FUSE = {"cfg4": 1, "cfg5": 1, "cfg5cut": 1}
 LOOP_ORDER = {"cfg1": "tick_major", "cfg3": "tick_major", "cfg4": "tick_major", "cfg5": "mb_major", "cfg5cut": "tick_major"}
 
 
@@ -481,7 +485,8 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     P = wl.n_stages
     order = LOOP_ORDER[workload]
     mb_major = order == "mb_major"
-    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order)
+    fused = FUSE.get(workload, 0) if getattr(args, "fuse", False) else 0
+    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused)
     del params0
     host_b, dev_b = make_batches(wl, 4, device)
     warm = max(args.warmup, 3)
@@ -532,7 +537,7 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     per_tick = {k: v[0] / args.steps for k, v in prof.items() if v[1] > 0}
     total_prof = sum(per_tick.values())
 
-    res = {"wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
+    res = {"fused": fused, "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
            "t_ms": t_med, "times": times, "units": units, "launches": launches, "clocks": clocks, "per_tick_ms": per_tick,
            "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "workspace_bytes": pipe.workspace_bytes,
            "prof": prof, "total_prof": total_prof}
@@ -784,6 +789,8 @@ def main():
     ap.add_argument("--no-other", action="store_true", help="skip the short run of the other built workload")
     ap.add_argument("--stages", type=int, default=0, help="profiling runs: same workload cut to this many stages")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
+    ap.add_argument("--fuse", action="store_true", help="apply the update of the Linear matrices in the weight-gradient "
+                    "GEMM's epilogue (pm_config.fuse_update) where the workload allows it; default: the update kernel")
     ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",
                     help="run only the stand-alone fused update on N_PARAMS parameters (profiling runs)")
     args = ap.parse_args()

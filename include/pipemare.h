@@ -178,6 +178,12 @@ typedef struct {
                                     tau_recomp (T2 for recompute, with the accumulator as it stood with version v): the update
                                     that produces version v also writes that copy, in the operand type, into tau_recomp + 1
                                     further slots of the stage's version queue (counted by pm_query_bytes). */
+  int32_t fuse_update;           /* 1: the weight-gradient GEMM of a Linear applies the update of its matrix in its epilogue,
+                                    while dW is still on chip (same arithmetic per element, bit for bit; dW of Linear matrices
+                                    is then NOT written to arenas.grad).  The weight-gradient GEMMs move from pm_backward to
+                                    pm_update, whose update kernel covers the remaining parameters (biases, LayerNorm
+                                    parameters, embedding tables).  Needs PM_BF16, one Linear per stage, n_micro <= 1,
+                                    entry_period <= 1 and recompute_segment = 0, else PM_ERR_UNSUPPORTED.  0: off. */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /

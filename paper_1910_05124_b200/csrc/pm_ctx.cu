@@ -26,6 +26,9 @@ struct Layout {
   std::vector<StageDev> st;
   std::vector<StageSched> sched;
   std::vector<uint32_t> begin64, end64;
+  std::vector<uint32_t> skip_b64, skip_e64;   // per stage, the Linear matrix's range in 64-element groups (fused update), else empty
+  uint64_t off_skb = 0, off_ske = 0;
+  int32_t fuse = 0;                     // the weight-gradient GEMM applies the update of the Linear matrices in its epilogue
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
@@ -329,6 +332,25 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].vdepth = s.vdepth; L.sched[p].begin = s.begin; L.sched[p].count = s.end - s.begin; L.sched[p].v_ring = s.v_ring;
     L.sched[p].tau_r = s.tau_r; L.sched[p].rdepth = s.rdepth;
   }
+  // Fused update (pm_config.fuse_update): the weight-gradient GEMM's epilogue updates the Linear matrices, the update
+  // kernel the rest of every stage (biases, LayerNorm parameters, embedding tables, padding).
+  L.fuse = 0;
+  L.skip_b64.assign(P, 0); L.skip_e64.assign(P, 0);
+  if (cfg->fuse_update) {
+    const char* why = nullptr;
+    if (cfg->compute_dtype != PM_BF16) why = "the tensor-core (PM_BF16) path";
+    else if (L.max_lin != 1) why = "one Linear per stage";
+    else if (cfg->n_micro > 1) why = "one microbatch per update (the gradients of a minibatch are summed in the grad arena)";
+    else if (S > 0) why = "no recomputation (a segment's stashes are overwritten before the update phase)";
+    else if (E > 1) why = "an entry period of one tick";
+    if (why) { err = std::string("fuse_update is built for ") + why; return PM_ERR_UNSUPPORTED; }
+    L.fuse = 1;
+    for (int p = 0; p < P; ++p) {
+      const LinDev& l0 = L.st[p].lin[0];
+      L.skip_b64[p] = (uint32_t)(l0.w_off / 64);
+      L.skip_e64[p] = (uint32_t)((l0.w_off + (uint64_t)l0.n_out * l0.n_in) / 64);     // dimensions are multiples of 8: whole groups
+    }
+  }
   for (int p = 0; p < P; ++p) {
     L.sched[p].next_xdepth = p + 1 < P ? L.st[p + 1].xdepth : 0;
     L.sched[p].gin_depth = L.st[p].gin_depth;
@@ -361,6 +383,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_nupd = w; w = align_up(w + sizeof(int64_t) * P, 256);
   L.off_b64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_e64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
+  L.off_skb = w; w = align_up(w + sizeof(uint32_t) * P, 256);
+  L.off_ske = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_alpha = w; w = align_up(w + sizeof(double) * (cfg->alpha_by_step ? (uint64_t)cfg->alpha_len : 0), 256);
   L.off_loss = w; w = align_up(w + sizeof(float) * (uint64_t)L.loss_cap, 256);
   L.off_lossred = w; w = align_up(w + 512, 256);
@@ -586,6 +610,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   UP(L.off_sched, c->L.sched);
   UP(L.off_b64, c->L.begin64);
   UP(L.off_e64, c->L.end64);
+  UP(L.off_skb, c->L.skip_b64);
+  UP(L.off_ske, c->L.skip_e64);
   UP(L.off_ids, c->L.ids);
   if (!c->L.segs.empty()) { UP(L.off_segs, c->L.segs); }
 #undef UP
@@ -624,6 +650,8 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0;
   t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
+  t.fuse_upd = 0; t.upd_opt = cfg->optimizer; t.upd_beta1 = cfg->beta1; t.upd_beta2 = cfg->beta2; t.upd_eps = cfg->eps;
+  t.upd_lp = L.queue ? reinterpret_cast<__nv_bfloat16*>(t.ring) : c->a.w_lp;
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
   t.pe_off = L.off_pe; t.rowloss_off = L.off_rowloss; t.loss_kind = cfg->loss;
   t.colred_off = L.off_colred; t.row_chunks = L.row_chunks; t.chunk_rows = L.chunk_rows;
@@ -886,9 +914,10 @@ static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets
 
 // The grouped launches that close a backward pass over the stages table `table` marks (all of them, or one recompute
 // segment): the weight gradients as one launch.
-static pm_status grouped_wgrad(pm_ctx* ctx, int table) {
+static pm_status grouped_wgrad(pm_ctx* ctx, int table, bool fused = false) {
   const int dt = ctx->cfg.compute_dtype;
   TickArgs ta = mb_args(ctx, table, -1);
+  ta.fuse_upd = fused ? 1 : 0;
   prof_begin(ctx, PM_PROF_WGRAD);
   cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 2, 0, ctx->ls) : umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
   return check(ctx, e, "wgrad GEMM");
@@ -927,7 +956,7 @@ static pm_status mb_backward(pm_ctx* ctx) {
       ta.colsum_only = 1; ta.defer_finish = 1;                  // bias gradients of the Linears without activation, all stages at once
       if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ta, dt, 0, ctx->ls), "bias gradient column sums", actbwd_launches(ta)))) != PM_OK) return s;
       ta.colsum_only = 0; ta.defer_finish = 0;
-      if (S == 0 && (s = grouped_wgrad(ctx, 2 * P)) != PM_OK) return s;
+      if (S == 0 && !ctx->L.fuse && (s = grouped_wgrad(ctx, 2 * P)) != PM_OK) return s;   // fused update: formed in the update phase
       const int n_fin = deferred_finish_launches(ta);
       if (n_fin && (s = TIMED(PM_PROF_PRE_BWD, check(ctx, launch_deferred_finish(ta, dt, ctx->ls), "bias / LayerNorm gradient sums", n_fin))) != PM_OK) return s;
     }
@@ -947,10 +976,14 @@ static pm_status mb_update(pm_ctx* ctx) {
   }
   const StageDyn* dyn_all = (const StageDyn*)(ctx->ws + ctx->L.off_dyn) + (size_t)2 * P * P;
   pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
+    // fused update: the weight gradients of all stages as one launch whose epilogue updates the Linear matrices
+    if (ctx->L.fuse) { pm_status fs = grouped_wgrad(ctx, 2 * P, true); if (fs != PM_OK) return fs; }
     prof_begin(ctx, PM_PROF_UPDATE);
     cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64), dyn_all,
                                   (int64_t*)(ctx->ws + ctx->L.off_nupd), P, ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1,
-                                  ctx->cfg.beta2, ctx->cfg.eps, ctx->ls, ctx->ta.ring, ctx->hp.lp_elem);
+                                  ctx->cfg.beta2, ctx->cfg.eps, ctx->ls, ctx->ta.ring, ctx->hp.lp_elem, 0,
+                                  ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_skb) : nullptr,
+                                  ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_ske) : nullptr);
     pm_status s = check(ctx, e, "update");
     if (s != PM_OK || ctx->L.segs.empty()) return s;
     prof_begin(ctx, PM_PROF_UPDATE);
@@ -1110,10 +1143,13 @@ pm_status pm_backward(pm_ctx* ctx) {
       else if (ctx->L.att_blocks > 0 && (s = TIMED(PM_PROF_ATTN_BWD, check(ctx, launch_post_bwd(ctx->ta, dt, ctx->ls), "attention backward"))) != PM_OK) return s;
       for (int l = ctx->L.max_lin - 1; l >= 0; --l) {
         if ((s = TIMED(PM_PROF_ACT_BWD, check(ctx, launch_actbwd(ctx->ta, dt, l, ctx->ls), "activation backward", actbwd_launches(ctx->ta)))) != PM_OK) return s;
-        prof_begin(ctx, PM_PROF_WGRAD);
-        cudaError_t e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->ls)
-                                     : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->ls);
-        if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+        cudaError_t e = cudaSuccess;
+        if (!ctx->L.fuse) {                                           // fused update: formed in the update phase
+          prof_begin(ctx, PM_PROF_WGRAD);
+          e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 2, l, ctx->ls)
+                           : umma_launch(ctx->umma, ctx->ta, 2, l, ctx->ls);
+          if ((s = check(ctx, e, "wgrad GEMM")) != PM_OK) return s;
+        }
         prof_begin(ctx, PM_PROF_DGRAD);
         e = dt == PM_F32 ? launch_simt_gemm(ctx->ta, dt, 1, l, ctx->ls)
                          : umma_launch(ctx->umma, ctx->ta, 1, l, ctx->ls);
@@ -1140,11 +1176,23 @@ pm_status pm_update(pm_ctx* ctx) {
     if (s != PM_OK) return s;
   } else if (any) {
     pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
+      cudaError_t e;
+      if (ctx->L.fuse) {
+        // the weight gradients of the stages in backward, with the update of their Linear matrices in the epilogue
+        TickArgs ta = ctx->ta;
+        ta.fuse_upd = 1;
+        prof_begin(ctx, PM_PROF_WGRAD);
+        e = umma_launch(ctx->umma, ta, 2, 0, ctx->ls);
+        pm_status fs = check(ctx, e, "wgrad GEMM with fused update");
+        if (fs != PM_OK) return fs;
+      }
       prof_begin(ctx, PM_PROF_UPDATE);
-      cudaError_t e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
-                                    (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
-                                    ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls,
-                                    ctx->L.queue ? (void*)ctx->ta.ring : nullptr, ctx->hp.lp_elem);
+      e = launch_update(ctx->a, (const uint32_t*)(ctx->ws + ctx->L.off_b64), (const uint32_t*)(ctx->ws + ctx->L.off_e64),
+                        (const StageDyn*)(ctx->ws + ctx->L.off_dyn), (int64_t*)(ctx->ws + ctx->L.off_nupd), P,
+                        ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1, ctx->cfg.beta2, ctx->cfg.eps, ctx->ls,
+                        ctx->L.queue ? (void*)ctx->ta.ring : nullptr, ctx->hp.lp_elem, 0,
+                        ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_skb) : nullptr,
+                        ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_ske) : nullptr);
       pm_status s = check(ctx, e, "update");
       if (s != PM_OK || !ctx->L.queue || ctx->L.segs.empty()) return s;
       prof_begin(ctx, PM_PROF_UPDATE);                                 // fp32 copies of the updated stages' small tensors into their queues

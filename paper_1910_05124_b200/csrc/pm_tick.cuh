@@ -61,6 +61,13 @@ struct TickArgs {
                           // stages with an activation were handled by their own launch (microbatch-major order)
   int32_t defer_finish;   // launches of one stage leave the per-chunk partial sums of bias / LayerNorm gradients in place;
                           // one grouped launch over all stages adds them up at the end of the backward pass
+  // weight-gradient launch that applies the PipeMare update to the Linear matrices in its epilogue (bf16 tensor-core
+  // path): dW never reaches the grad arena; the stage's step size, T2 decay and bias corrections come from its table
+  // entry, the optimiser constants from here, and the operand-type copy of the new weights goes to lp_base
+  int32_t fuse_upd;       // 0: dW is stored (or added) to the grad arena
+  int32_t upd_opt;        // PM_SGDM | PM_ADAM
+  float upd_beta1, upd_beta2, upd_eps;
+  __nv_bfloat16* upd_lp;  // base of the bfloat16 copy: the w_lp arena (tick-major order) or the ring arena (version queues)
 };
 
 // stage of a block in a kernel whose grid has one coordinate per stage

@@ -25,6 +25,7 @@
 
 #include "pm_ptx.cuh"
 #include "pm_umma.cuh"
+#include "pm_update_math.cuh"
 
 namespace pm {
 
@@ -76,6 +77,77 @@ struct EpiState {
   uint32_t slot = 0;          // slot the next single-output block writes
 };
 
+// The PipeMare update of one 32-row x 64-column block of a Linear matrix, applied to the weight gradient while it is
+// still on chip (r0, r1: the block's accumulators, lane = row).  The block goes through the warp's staging buffer
+// once, in the layout the dW store uses, and comes back with a lane owning four consecutive columns of a row, so
+// that every access to the master weights, the moments and delta is a full 128-byte line per eight lanes.  Per
+// element the arithmetic is upd_one's, i.e. exactly what the stand-alone update kernel does with a stored gradient.
+template <int OPT>
+__device__ __forceinline__ void epi_update_block(const TickArgs& t, const StageDyn& d, const LinDev& L, int M, int N, int mrow, int nb,
+                                                 const uint32_t (&r0)[32], const uint32_t (&r1)[32], uint8_t* obuf, int lane) {
+  const uint32_t row_off = (uint32_t)lane * 128, sw = (uint32_t)(lane & 7);
+  __syncwarp();                                                   // the previous block's reads of the buffer are done
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {                                   // two boxes of 32 fp32 columns, 16-byte chunks swizzled by row
+    *reinterpret_cast<uint4*>(obuf + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r0[g * 4], r0[g * 4 + 1], r0[g * 4 + 2], r0[g * 4 + 3]);
+    *reinterpret_cast<uint4*>(obuf + 4096 + row_off + (((uint32_t)g ^ sw) << 4)) = make_uint4(r1[g * 4], r1[g * 4 + 1], r1[g * 4 + 2], r1[g * 4 + 3]);
+  }
+  __syncwarp();
+  UpdScalars sc;
+  sc.alpha = d.alpha; sc.gamma = d.gamma; sc.omg = d.one_minus_gamma; sc.bc1 = d.bc1; sc.bc2 = d.bc2; sc.use_delta = d.use_delta;
+  sc.lp_shift = d.lp_shift; sc.rc_shift = d.rc_uslot >= 0 ? d.rc_shift : -1; sc.rc_gap = d.rc_gap;
+  const bool need_dl = sc.use_delta || sc.rc_shift >= 0;
+  const float beta1 = t.upd_beta1, beta2 = t.upd_beta2, eps = t.upd_eps;
+  const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
+  const int rr0 = lane >> 3, ch = lane & 7;                       // row within a group of four, 16-byte chunk of the 32-column box
+  constexpr int NB = 4;                                           // row groups whose loads are in flight together
+#pragma unroll 1
+  for (int it0 = 0; it0 < 16; it0 += NB) {                        // 16 = 2 boxes x 8 groups of four rows
+    float4 g4[NB], w4[NB], m4[NB], s4[NB], d4[NB];
+    uint64_t e[NB];
+    bool on[NB];
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      const int it = it0 + u, box = it >> 3, rr = (it & 7) * 4 + rr0;
+      const int row = mrow + rr, col = nb + box * 32 + ch * 4;
+      on[u] = row < M && col < N;
+      e[u] = L.w_off + (uint64_t)row * (uint64_t)N + (uint64_t)col;
+      g4[u] = *reinterpret_cast<const float4*>(obuf + box * 4096 + rr * 128 + (((uint32_t)ch ^ (uint32_t)(rr & 7)) << 4));
+      if (on[u]) {
+        w4[u] = __ldcs(reinterpret_cast<const float4*>(t.a.w + e[u]));
+        m4[u] = __ldcs(reinterpret_cast<const float4*>(t.a.m + e[u]));
+        if (need_dl) d4[u] = __ldcs(reinterpret_cast<const float4*>(t.a.delta + e[u]));
+        if (OPT == PM_ADAM) s4[u] = __ldcs(reinterpret_cast<const float4*>(t.a.s + e[u]));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      if (!on[u]) continue;
+      float4 wn;
+      wn.x = upd_one<OPT>(g4[u].x, w4[u].x, m4[u].x, s4[u].x, d4[u].x, sc, beta1, beta2, omb1, omb2, eps);
+      wn.y = upd_one<OPT>(g4[u].y, w4[u].y, m4[u].y, s4[u].y, d4[u].y, sc, beta1, beta2, omb1, omb2, eps);
+      wn.z = upd_one<OPT>(g4[u].z, w4[u].z, m4[u].z, s4[u].z, d4[u].z, sc, beta1, beta2, omb1, omb2, eps);
+      wn.w = upd_one<OPT>(g4[u].w, w4[u].w, m4[u].w, s4[u].w, d4[u].w, sc, beta1, beta2, omb1, omb2, eps);
+      __stcs(reinterpret_cast<float4*>(t.a.w + e[u]), wn);
+      __stcs(reinterpret_cast<float4*>(t.a.m + e[u]), m4[u]);
+      if (OPT == PM_ADAM) __stcs(reinterpret_cast<float4*>(t.a.s + e[u]), s4[u]);
+      if (sc.use_delta) __stcs(reinterpret_cast<float4*>(t.a.delta + e[u]), d4[u]);
+      {
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(wn.x, wn.y), hi2 = __floats2bfloat162_rn(wn.z, wn.w);
+        uint2 pk; pk.x = *reinterpret_cast<uint32_t*>(&lo2); pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+        *reinterpret_cast<uint2*>(t.upd_lp + (sc.lp_shift + (int64_t)e[u])) = pk;              // re-read by a later forward: default caching
+      }
+      if (sc.rc_shift >= 0) {                                     // corrected recompute weights of the new version (T2 for recompute)
+        const float gp = sc.rc_gap;
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(__fsub_rn(wn.x, __fmul_rn(gp, d4[u].x)), __fsub_rn(wn.y, __fmul_rn(gp, d4[u].y)));
+        __nv_bfloat162 hi2 = __floats2bfloat162_rn(__fsub_rn(wn.z, __fmul_rn(gp, d4[u].z)), __fsub_rn(wn.w, __fmul_rn(gp, d4[u].w)));
+        uint2 pk; pk.x = *reinterpret_cast<uint32_t*>(&lo2); pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+        *reinterpret_cast<uint2*>(t.upd_lp + (sc.rc_shift + (int64_t)e[u])) = pk;
+      }
+    }
+  }
+}
+
 // One epilogue block of the forward (MODE 0) or wgrad (MODE 2) GEMM: 32 rows x 64 accumulator columns held in
 // r0, r1 go through this warp's swizzled staging buffer to one or two TMA stores (full 128-byte rows; rows and
 // columns beyond the tensor are clipped).  Called by a whole warp; lane = row within the block.
@@ -88,6 +160,11 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
                                           int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
                                           uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es,
                                           const uint4 (&skq)[8]) {
+  if (MODE == 2 && t.fuse_upd) {                                  // the update is applied here; nothing is stored to the grad arena
+    if (t.upd_opt == PM_SGDM) epi_update_block<PM_SGDM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
+    else epi_update_block<PM_ADAM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
+    return;
+  }
   const uint32_t row_off = (uint32_t)lane * 128;
   const uint32_t sw = (uint32_t)(lane & 7);
   const bool f32out = MODE == 0 && (L.flags & LF_OUT_F32) != 0;

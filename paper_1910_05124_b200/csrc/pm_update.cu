@@ -181,15 +181,30 @@ template <int OPT, int LP>
 __global__ void __launch_bounds__(kUpdThreads)
 update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
               const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
-              float beta1, float beta2, float eps, uint64_t first_vec4) {
-  extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends
+              float beta1, float beta2, float eps, uint64_t first_vec4, const uint32_t* __restrict__ skip_b64, const uint32_t* __restrict__ skip_e64) {
+  extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends, then the skipped ranges' begins and ends
   uint32_t* sb = sm_bounds;
   uint32_t* se = sm_bounds + n_stages;
-  for (int i = threadIdx.x; i < n_stages; i += blockDim.x) { sb[i] = begin64[i]; se[i] = end64[i]; }
+  // ranges (one per stage, in 64-element groups) that another kernel has updated already: the Linear matrices, when the
+  // weight-gradient GEMM applies the update in its epilogue
+  uint32_t* kb = sm_bounds + 2 * n_stages;
+  uint32_t* ke = sm_bounds + 3 * n_stages;
+  const bool skip = skip_b64 != nullptr;
+  for (int i = threadIdx.x; i < n_stages; i += blockDim.x) {
+    sb[i] = begin64[i]; se[i] = end64[i];
+    kb[i] = skip ? skip_b64[i] : 0u; ke[i] = skip ? skip_e64[i] : 0u;
+  }
   __syncthreads();
   const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
   const uint64_t stride = (uint64_t)gridDim.x * kUpdThreads * kUpdUnroll;
   for (uint64_t base = first_vec4 + (uint64_t)blockIdx.x * kUpdThreads * kUpdUnroll; base < total_vec4; base += stride) {
+    if (skip) {
+      // the whole span of this block lies inside a skipped range (and past the stage's first group): nothing to do
+      const uint32_t g0 = (uint32_t)(base >> 4), g1 = (uint32_t)((base + (uint64_t)kUpdThreads * kUpdUnroll - 1) >> 4);
+      int lo = 0, hi = n_stages - 1;
+      while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (sb[mid] <= g0) lo = mid; else hi = mid - 1; }
+      if (kb[lo] <= g0 && g1 < ke[lo] && g0 > sb[lo]) continue;
+    }
     uint64_t v[kUpdUnroll];
     int stage[kUpdUnroll];
     UpdScalars sc[kUpdUnroll];
@@ -202,7 +217,11 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
         uint32_t e64 = (uint32_t)(v[u] >> 4);
         int lo = 0, hi = n_stages - 1;               // largest i with sb[i] <= e64
         while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (sb[mid] <= e64) lo = mid; else hi = mid - 1; }
-        if (sb[lo] <= e64 && e64 < se[lo] && dyn[lo].active_update) stage[u] = lo;
+        if (sb[lo] <= e64 && e64 < se[lo] && dyn[lo].active_update) {
+          if (skip && kb[lo] <= e64 && e64 < ke[lo]) {                     // updated elsewhere; the stage's counter is still kept here
+            if (e64 == sb[lo] && (v[u] & 15) == 0) nupd[lo] += 1;
+          } else stage[u] = lo;
+        }
       }
       if (stage[u] >= 0) {
         const uint64_t e = v[u] * 4;
@@ -265,7 +284,8 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
 
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
-                          float eps, cudaStream_t stream, void* lp_base, int lp_elem, uint64_t first64) {
+                          float eps, cudaStream_t stream, void* lp_base, int lp_elem, uint64_t first64,
+                          const uint32_t* skip_b64, const uint32_t* skip_e64) {
   if (total64 == 0 || n_stages == 0 || first64 >= total64) return cudaSuccess;
   uint64_t total_vec4 = total64 * 16;
   const uint64_t first_vec4 = first64 * 16;
@@ -276,11 +296,11 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   uint64_t cap = (uint64_t)sms * 8;                 // whole waves of resident blocks
   int blocks = (int)(need < cap ? need : cap);
-  size_t smem = sizeof(uint32_t) * 2 * (size_t)n_stages;
+  size_t smem = sizeof(uint32_t) * 4 * (size_t)n_stages;
   // the operand-type copy: the w_lp arena (bfloat16) unless the caller names a version ring and its element size
   if (lp_base == nullptr) { lp_base = a.w_lp; lp_elem = 2; }
   const int lp = lp_base == nullptr ? 0 : (lp_elem == 4 ? 2 : 1);
-#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps, first_vec4)
+#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps, first_vec4, skip_b64, skip_e64)
   if (optimizer == PM_SGDM) { if (lp == 0) PM_UPD(PM_SGDM, 0); else if (lp == 1) PM_UPD(PM_SGDM, 1); else PM_UPD(PM_SGDM, 2); }
   else { if (lp == 0) PM_UPD(PM_ADAM, 0); else if (lp == 1) PM_UPD(PM_ADAM, 1); else PM_UPD(PM_ADAM, 2); }
 #undef PM_UPD

@@ -31,7 +31,11 @@ inline int mb_table_count(int P, int segment) { return 2 * P + 1 + (segment > 0 
 // begin64/end64: stage bounds in units of 64 elements, ascending; total64 = end64[P-1].
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
-                          float eps, cudaStream_t stream, void* lp_base = nullptr, int lp_elem = 0, uint64_t first64 = 0);
+                          float eps, cudaStream_t stream, void* lp_base = nullptr, int lp_elem = 0, uint64_t first64 = 0,
+                          const uint32_t* skip_b64 = nullptr, const uint32_t* skip_e64 = nullptr);
+// skip_b64 / skip_e64: per stage, a range of 64-element groups this launch leaves alone (device arrays, or null): the
+// Linear matrices when the weight-gradient GEMM has applied their update in its epilogue.  The stage's update
+// counter is incremented here all the same.
 // first64: the walk over the arenas starts at this 64-element group (a launch for one stage starts at that stage's slice).
 // lp_base / lp_elem: where the operand-type copy of the new weights goes: by default the bfloat16 arena a.w_lp
 // (if there is one); microbatch-major order passes the ring arena and the operand size (2 or 4 bytes), and the
