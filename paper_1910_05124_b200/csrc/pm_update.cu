@@ -178,7 +178,7 @@ constexpr int kUpdUnroll = 2;      // float4 groups per thread per array in flig
 // LP: operand-type copy of the new weights: 0 none, 1 bfloat16, 2 float (a version-ring slot of fp32 operands);
 // element e of the arenas goes to lp_base[lp_shift + e], lp_shift from the stage's table entry (0: the w_lp arena)
 template <int OPT, int LP>
-__global__ void __launch_bounds__(kUpdThreads)
+__global__ void __launch_bounds__(kUpdThreads, 3)
 update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
               const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
               float beta1, float beta2, float eps, uint64_t first_vec4, const uint32_t* __restrict__ skip_b64, const uint32_t* __restrict__ skip_e64) {
