@@ -645,7 +645,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.n_in_first = L.n_in_first; t.n_out_last = L.n_out_last;
   t.yout_off = L.off_yout; t.tgt_off = L.off_tgt; t.loss_off = L.off_loss; t.loss_cap = L.loss_cap; t.lossred_off = L.off_lossred;
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
-  t.mb_major = L.queue ? 1 : 0; t.sel_p = -1;
+  t.mb_major = L.queue ? 1 : 0; t.sel_p = -1; t.sel_tile0 = 0;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
   t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0;
   t.dgrad_split_below = 0;

@@ -51,6 +51,7 @@ struct TickArgs {
   // the stage from a block coordinate use sel_p instead (-1: all stages, the coordinate); the stage lists above then
   // point at that stage's entry; act_first[lvl] is added to the block index of the activation-backward walk
   int32_t sel_p;
+  int32_t sel_tile0;      // GEMM launches of one stage: flattened id of the stage's first tile (set by the launcher)
   int32_t act_first[PM_MAX_LINEARS];
   int32_t res_fused;      // the forward GEMM's epilogue adds the skip tensor (bf16 tensor-core path): no residual kernel
   int32_t dgrad_split_below;   // CTA-pair dgrad: a Linear whose two-row-tile groups number fewer than this takes one row tile per

@@ -310,11 +310,16 @@ __device__ __forceinline__ float4 load_bias4(const float* bias, int n, int N) {
 // ---- tile walk ---------------------------------------------------------------------------------------
 // tile_start[p] .. tile_start[p+1] are the flattened tile ids of stage p for this (mode, level).
 struct Tile { int p, m0, n0, M, N, K, n_kb; bool valid; };
+// the tile a CTA's slot holds: from the launch's order list, or, in a launch of one stage (its tiles in ascending
+// order), from the launch arguments alone, so that no role starts with a chain of dependent global loads
+__device__ __forceinline__ int tile_at(const TickArgs& t, const int* __restrict__ order, int slot) {
+  return t.sel_p >= 0 ? t.sel_tile0 + slot : order[slot];
+}
 
 template <int MODE>
 __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   Tile r;
-  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  const int lo = t.sel_p >= 0 ? t.sel_p : tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -323,7 +328,7 @@ __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __rest
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
   else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
   const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
-  const int local = tile - tile_start[lo];
+  const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
   r.m0 = (local / tiles_n) * TILE_M;
   r.n0 = (local % tiles_n) * TILE_N;
   r.n_kb = (r.K + TILE_K - 1) / TILE_K;
@@ -378,7 +383,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       int issued_op = 0;
       bool ok = true;
       for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -429,7 +434,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
       Ring op{0, 0}, acc{0, 0};
       bool ok = true;
       for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -465,7 +470,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
     bool ok = true;
     EpiState es;
     for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const Tile tl = decode_tile<MODE>(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -527,7 +532,7 @@ constexpr int P2_SMEM_BYTES = P2_TILE_BYTES + 1024 + 512;
 template <int MODE>
 __device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   Tile r;
-  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  const int lo = t.sel_p >= 0 ? t.sel_p : tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -536,7 +541,7 @@ __device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* _
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
   else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
   const int tiles_n = (r.N + P2_TILE - 1) / P2_TILE;
-  const int local = tile - tile_start[lo];
+  const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
   r.m0 = (local / tiles_n) * P2_TILE;
   r.n0 = (local % tiles_n) * P2_TILE;
   r.n_kb = (r.K + TILE_K - 1) / TILE_K;
@@ -597,7 +602,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       int issued_op = 0;
       bool ok = true;
       for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -657,7 +662,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       Ring op{0, 0}, acc{0, 0};
       bool ok = true;
       for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -691,7 +696,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
     bool ok = true;
     EpiState es;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const Tile tl = decode_pair_tile<MODE>(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -762,7 +767,7 @@ struct DgTile { int p, m0, n0, n_m, M, N, K, n_kb; bool valid; };
 
 __device__ __forceinline__ DgTile decode_dgrad(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
-  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  const int lo = t.sel_p >= 0 ? t.sel_p : tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -771,7 +776,7 @@ __device__ __forceinline__ DgTile decode_dgrad(const TickArgs& t, const int* __r
   r.M = t.T; r.N = L.n_in; r.K = L.n_out;
   const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
   const int tiles_m = (r.M + TILE_M - 1) / TILE_M;
-  const int local = tile - tile_start[lo];
+  const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
   const int mg = local / tiles_n;
   r.m0 = mg * DG_MG * TILE_M;
   r.n0 = (local % tiles_n) * TILE_N;
@@ -828,7 +833,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       struct Cursor { int tile, kb; DgTile tl; bool done; };
       auto seek = [&](Cursor& c) {                                    // move to the next valid tile at or after c.tile
         for (; c.tile < n_slots; c.tile += gridDim.x) {              // c.tile walks the slots of the order array
-          const int tile = order[c.tile];
+          const int tile = tile_at(t, order, c.tile);
           if (tile < 0) continue;
           c.tl = decode_dgrad(t, tile_start, lvl, tile);
           if (c.tl.valid) { c.kb = 0; c.done = false; return; }
@@ -890,7 +895,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
       uint32_t tphase = 0;
       bool ok = true;
       for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -927,7 +932,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     Ring br{0, 0}, sg{0, 0};
     bool ok = true;
     for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -972,7 +977,7 @@ umma_dgrad_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* _
     uint32_t tphase = 0;
     bool ok = true, stored = false;
     for (int slot = blockIdx.x; slot < n_slots && ok; slot += gridDim.x) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -1065,7 +1070,7 @@ __host__ __device__ inline int dgrad_pair_mg(int T, int n_in, int split_below) {
 
 __device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
-  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  const int lo = t.sel_p >= 0 ? t.sel_p : tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -1075,7 +1080,7 @@ __device__ __forceinline__ DgTile decode_dgrad_pair(const TickArgs& t, const int
   const int mgr = dgrad_pair_mg(r.M, r.N, t.dgrad_split_below);
   const int tiles_n = (r.N + DP_TILE_N - 1) / DP_TILE_N;
   const int tiles_m = (r.M + DP_TILE_M - 1) / DP_TILE_M;
-  const int local = tile - tile_start[lo];
+  const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
   const int mg = local / tiles_n;
   r.m0 = mg * mgr * DP_TILE_M;
   r.n0 = (local % tiles_n) * DP_TILE_N;
@@ -1141,7 +1146,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
   struct Cursor { int tile, kb; DgTile tl; bool done; const CUtensorMap* lm; bool corr; int dz_slot; };
   auto seek = [&](Cursor& c) {
     for (; c.tile < n_slots; c.tile += n_pairs) {
-      const int tile = order[c.tile];
+      const int tile = tile_at(t, order, c.tile);
       if (tile < 0) continue;
       c.tl = decode_dgrad_pair(t, tile_start, lvl, tile);
       if (c.tl.valid) {
@@ -1227,7 +1232,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
       DpAcc acc{{0u, 0u}, 0};
       bool ok = true;
       for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -1277,7 +1282,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
     Ring br{0, 0}, sg{0, 0};
     bool ok = true;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -1326,7 +1331,7 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
     DpAcc acc{{0u, 0u}, 0};
     bool ok = true, stored = false;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad_pair(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -1415,7 +1420,7 @@ constexpr int D1_SMEM_BYTES = D1_TILE_BYTES + 1024 + 512;
 
 __device__ __forceinline__ DgTile decode_dgrad_pair128(const TickArgs& t, const int* __restrict__ tile_start, int lvl, int tile) {
   DgTile r;
-  const int lo = tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
+  const int lo = t.sel_p >= 0 ? t.sel_p : tile_start[t.P + 1 + tile];                           // the stage of this tile: table behind the P + 1 starts
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
@@ -1424,7 +1429,7 @@ __device__ __forceinline__ DgTile decode_dgrad_pair128(const TickArgs& t, const 
   r.M = t.T; r.N = L.n_in; r.K = L.n_out;
   const int tiles_n = (r.N + D1_TILE_N - 1) / D1_TILE_N;
   const int tiles_m = (r.M + D1_TILE_M - 1) / D1_TILE_M;
-  const int local = tile - tile_start[lo];
+  const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
   const int mg = local / tiles_n;
   r.m0 = mg * D1_MG * D1_TILE_M;
   r.n0 = (local % tiles_n) * D1_TILE_N;
@@ -1481,7 +1486,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
   struct Cursor { int tile, kb; DgTile tl; bool done; const CUtensorMap* lm; bool corr; int dz_slot; };
   auto seek = [&](Cursor& c) {
     for (; c.tile < n_slots; c.tile += n_pairs) {
-      const int tile = order[c.tile];
+      const int tile = tile_at(t, order, c.tile);
       if (tile < 0) continue;
       c.tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
       if (c.tl.valid) {
@@ -1561,7 +1566,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
       Ring br{0, 0}, ar{0, 0}, acc{0, 0};
       bool ok = true;
       for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-        const int tile = order[slot];
+        const int tile = tile_at(t, order, slot);
         if (tile < 0) continue;
         const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
         if (!tl.valid) continue;
@@ -1604,7 +1609,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
     Ring br{0, 0}, sg{0, 0};
     bool ok = true;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -1648,7 +1653,7 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
     Ring acc{0, 0};
     bool ok = true, stored = false;
     for (int slot = pair; slot < n_slots && ok; slot += n_pairs) {
-      const int tile = order[slot];
+      const int tile = tile_at(t, order, slot);
       if (tile < 0) continue;
       const DgTile tl = decode_dgrad_pair128(t, tile_start, lvl, tile);
       if (!tl.valid) continue;
@@ -2020,6 +2025,7 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
   int grid = plan->grid[mode][lvl];                                   // one persistent CTA per SM
   const int* ts = plan->d_tile_start + plan->ts_off[mode][lvl];
   const int* ord = plan->d_orders + plan->order_off[mode][lvl];
+  int tile0 = 0;
   bool narrow = false;                                                // dgrad of one narrow stage: 128-column tiles
   if (t.sel_p >= 0 && mode == 1 && plan->pair[1][lvl] && plan->pair[3][lvl]) {
     const int* h1 = plan->h_tile_start.data() + plan->ts_off[1][lvl];
@@ -2032,20 +2038,23 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
     n_slots = hts[t.sel_p + 1] - first;
     if (n_slots == 0) return cudaSuccess;
     ord = plan->d_identity + first;
+    tile0 = first;
     const bool pr = plan->pair[mode][lvl];
     const int G = std::max(1, std::min(n_slots, pr ? plan->max_ctas / 2 : plan->max_ctas));
     grid = pr ? 2 * G : G;
   }
+  TickArgs ta = t;
+  ta.sel_tile0 = tile0;
   if (plan->pair[mode][lvl]) {
-    if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
-    else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
-    else if (mode == 3) umma_dgrad_pair128_kernel<<<grid, D1_THREADS, D1_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
-    else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else if (mode == 3) umma_dgrad_pair128_kernel<<<grid, D1_THREADS, D1_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     return cudaGetLastError();
   }
-  if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
-  else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
-  else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(t, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   return cudaGetLastError();
 }
 
