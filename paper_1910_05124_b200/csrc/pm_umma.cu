@@ -548,15 +548,6 @@ __device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* _
   return r;
 }
 
-#ifdef PM_TIMELINE
-__device__ unsigned long long pm_tl[64][296][10];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long v; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(v)); return v; }
-#define TL(k) do { if (MODE == 0 && t.sel_p >= 0 && t.sel_p < 64) pm_tl[t.sel_p][blockIdx.x][k] = (unsigned long long)clock64(); } while (0)
-#define TLG(k) do { if (MODE == 0 && t.sel_p >= 0 && t.sel_p < 64) pm_tl[t.sel_p][blockIdx.x][k] = gtime(); } while (0)
-#else
-#define TL(k)
-#define TLG(k)
-#endif
 template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P2_THREADS, 1)
 umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __restrict__ tile_start, const int* __restrict__ order, int n_slots, int lvl, int* status) {
@@ -576,7 +567,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();                            // 0 = leader
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  if (threadIdx.x == 0) { TL(0); TLG(8); }
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
@@ -593,7 +583,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
   cluster_sync_all();                                                 // barriers of both CTAs are initialised
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (threadIdx.x == 0) TL(1);
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
@@ -622,7 +611,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         for (int kb = 0; kb < n_kb; ++kb) {
           const int k0 = kb * TILE_K;
           if (!mbar_wait(bar_empty + 8 * op.idx, op.phase ^ 1, abort_flag, status, 31)) { ok = false; break; }
-          if (issued_op == 0) TL(2);
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
           if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * op.idx, 2 * (A_BYTES + B_BYTES));   // the bytes of both CTAs
           const uint32_t fb = mapa_shared(bar_full + 8 * op.idx, 0);
@@ -672,7 +660,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         for (int kb = 0; kb < tl.n_kb; ++kb) {
           if (!mbar_wait(bar_full + 8 * op.idx, op.phase, abort_flag, status, 32)) { ok = false; break; }
           tc_fence_after();
-          if (kb == 0 && slot == pair) TL(3);
           const uint32_t sa = tiles + op.idx * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
           for (int k16 = 0; k16 < TILE_K / 16; ++k16)
@@ -681,7 +668,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
           op.advance(NS);
         }
         if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);           // accumulator complete, both CTAs
-        TL(4);
         acc.advance(2);
       }
     }
@@ -713,7 +699,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
       tc_fence_after();
-      if (ew == 0 && lane == 0) TL(5);
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
         const int nb = tl.n0 + half * 128 + c * 64;
@@ -732,9 +717,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       }
       acc.advance(2);
     }
-    if (ew == 0 && lane == 0) TL(6);
     if (lane == 0 && es.stored) tma_store_wait_all();                    // global writes complete before the CTA retires
-    if (ew == 0 && lane == 0) TL(7);
   }
   tc_fence_before();
   cluster_sync_all();                                                 // no barrier or shared memory of a CTA is touched after this
@@ -743,11 +726,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 2 * P2_ACC_COLS);
   }
-  if (threadIdx.x == 0) TLG(9);
 }
-#ifdef PM_TIMELINE
-extern "C" int pm_tl_read(unsigned long long* host) { return (int)cudaMemcpyFromSymbol(host, pm_tl, sizeof(pm_tl)); }
-#endif
 
 // ---- dgrad with reuse of the corrected operand -----------------------------------------------------------
 // D[T,in] = dz[T,out] * Wc[out,in].  With thousands of rows the fp32 w and delta tiles (64 KB per k-block) and
