@@ -486,7 +486,8 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     order = LOOP_ORDER[workload]
     mb_major = order == "mb_major"
     fused = FUSE.get(workload, 0) if getattr(args, "fuse", False) else 0
-    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused)
+    segment = getattr(args, "recompute", 0) if mb_major else 0
+    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused, recompute_segment=segment)
     del params0
     host_b, dev_b = make_batches(wl, 4, device)
     warm = max(args.warmup, 3)
@@ -537,7 +538,7 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     per_tick = {k: v[0] / args.steps for k, v in prof.items() if v[1] > 0}
     total_prof = sum(per_tick.values())
 
-    res = {"fused": fused, "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
+    res = {"fused": fused, "segment": segment, "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
            "t_ms": t_med, "times": times, "units": units, "launches": launches, "clocks": clocks, "per_tick_ms": per_tick,
            "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "workspace_bytes": pipe.workspace_bytes,
            "prof": prof, "total_prof": total_prof}
@@ -689,7 +690,7 @@ def run_cuda(args):
         "warmup": max(args.warmup, 3), "ms_per_step": round(res["t_ms"] / steps, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32" if wl.compute == "f32" else "bf16", "data": "synthetic",
         "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
-                   "loop_order": res["order"],
+                   "loop_order": res["order"], "recompute_segment": res["segment"], "fuse_update": res["fused"],
                    "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
                    "samples_per_step": res["samples_per_step"], "pipeline_fill_ticks": res["fill"],
                    "cache": "per-step working set (state, activations, weight-version queues: see the byte counts) far exceeds the 126 MB L2: no flush needed",
@@ -789,6 +790,8 @@ def main():
     ap.add_argument("--no-other", action="store_true", help="skip the short run of the other built workload")
     ap.add_argument("--stages", type=int, default=0, help="profiling runs: same workload cut to this many stages")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
+    ap.add_argument("--recompute", type=int, default=0, metavar="S", help="PipeMare Recompute with segments of S stages "
+                    "(microbatch-major workloads; default 0: none)")
     ap.add_argument("--fuse", action="store_true", help="apply the update of the Linear matrices in the weight-gradient "
                     "GEMM's epilogue (pm_config.fuse_update) where the workload allows it; default: the update kernel")
     ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",

@@ -634,10 +634,10 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_full + 8 * (it % NS), (uint32_t)(it / NS) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
           }
-        } else {
-          const long long t0 = clock64();
-          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
         }
+        // rank 1's copies are counted on the same barriers of the leader (the expected bytes are those of both CTAs), and
+        // no CTA of the pair leaves before the cluster barrier at the end of the kernel, which the leader reaches only
+        // after these waits: rank 1 needs no wait of its own
       }
     }
   } else if (warp == 1) {
@@ -1195,10 +1195,10 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_afull + 8 * (it % DP_NA), (uint32_t)(it / DP_NA) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
           }
-        } else {
-          const long long t0 = clock64();
-          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
         }
+        // rank 1's copies are counted on the same barriers of the leader (the expected bytes are those of both CTAs), and
+        // no CTA of the pair leaves before the cluster barrier at the end of the kernel, which the leader reaches only
+        // after these waits: rank 1 needs no wait of its own
       }
     }
   }
@@ -1531,10 +1531,10 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_afull + 8 * (it % D1_NA), (uint32_t)(it / D1_NA) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
           }
-        } else {
-          const long long t0 = clock64();
-          while (clock64() - t0 < 4000000LL) {}                       // about 2 ms: far beyond any load latency
         }
+        // rank 1's copies are counted on the same barriers of the leader (the expected bytes are those of both CTAs), and
+        // no CTA of the pair leaves before the cluster barrier at the end of the kernel, which the leader reaches only
+        // after these waits: rank 1 needs no wait of its own
       }
     }
   } else if (warp == 1) {

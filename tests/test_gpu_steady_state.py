@@ -61,6 +61,27 @@ def test_cfg5_widths_steady_state_both_orders(cuda_device):
         pipe.close()
 
 
+def test_cfg5_widths_recompute_steady_state(cuda_device):
+    """PipeMare Recompute at config 5's widths on 2 + 2 layers (23 stages), segments of 5 stages (boundaries inside
+    layers: skip tensors, the memory and the main stream cross them), 2 sequences per microbatch, 2P + 4 microbatches:
+    the pair-tile kernels, the 256-token attention, one weight-gradient launch per segment, T2-corrected recompute
+    weights read from the queue."""
+    wl = I.cfg5_cut(2, 2, batch=2)
+    wl.steps = 2 * wl.n_stages + 4
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps, segment=5)
+    book_r = {}
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major", segment=5, book_recomp=book_r)
+    check_book(book, res, wl.steps, wl.n_stages)
+    ref_r = {(t, i): vr for (t, i, vr) in res.book_recomp}
+    assert book_r == ref_r
+    assert max(vr for vr in ref_r.values()) > 0 and any(ref_r[k] != res_v for k, res_v in ((k, v[0]) for k, v in book.items()))
+    print("cfg5 widths recompute: max loss relative error", np.abs(losses / np.array(res.losses) - 1).max())
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    print("cfg5 widths recompute weight errors", compare_params_adam(pipe, res, wl.steps))
+    pipe.close()
+
+
 def test_adam_noise_evidence_at_config4_widths(cuda_device):
     """Oracle arithmetic only (it sits here because it needs the GPU machine's host cores for a minute): the oracle
     against a copy of itself whose gradients carry a relative perturbation of 2^-20, config 4's 25 stages at its
