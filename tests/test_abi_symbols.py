@@ -211,6 +211,45 @@ def test_microbatch_major_footprint_of_config5(built_lib):
     assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
 
 
+def test_recompute_and_fused_update_options_are_checked_without_a_gpu(built_lib):
+    """PipeMare Recompute: the queue of T2-corrected recompute weights is counted by pm_query_bytes (tau_recomp + 1 slots
+    of every stage outside the last segment, tau_recomp = ceil-free 2(S - j) + 1 for one microbatch per update), and
+    the options' preconditions are reported as PM_ERR_UNSUPPORTED."""
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    wl = I.cfg5()
+    P, S = wl.n_stages, 12
+    cfg, sd, keep = _describe(wl)
+    cfg.loop_order = B.PM_MB_MAJOR
+    sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    plain = rb.value
+    cfg.recompute_segment = S
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    last = (P - 1) // S * S                                   # first stage of the last segment: nothing is recomputed from there on
+    extra = sum((2 * (min(P, (p // S + 1) * S) - 1 - p) + 1 + 1) * sd[p].param_count * 2 for p in range(last))
+    assert extra < rb.value - plain < extra * 1.01            # plus the fp32 copies of biases and LayerNorm parameters
+    cfg.recompute_segment = P                                 # one segment: the forward pass itself
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0 and rb.value == plain
+    cfg.recompute_segment = -1
+    assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
+    cfg.recompute_segment = S
+    cfg.loop_order = B.PM_TICK_MAJOR
+    sd_t = sd                                                 # Table 1's delays: the tick schedule accepts them, but not the option
+    assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd_t, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_UNSUPPORTED"
+    # the update in the weight-gradient epilogue: bf16, one Linear per stage, one microbatch per update, no recomputation
+    cfg.loop_order, cfg.recompute_segment, cfg.fuse_update = B.PM_MB_MAJOR, 0, 1
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    for field, value in (("recompute_segment", S), ("n_micro", 2), ("compute_dtype", B.PM_F32)):
+        old = getattr(cfg, field)
+        setattr(cfg, field, value)
+        st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+        assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED", field
+        setattr(cfg, field, old)
+
+
 def test_flat_update_argument_checks_need_no_gpu(built_lib):
     """pm_update_flat / pm_update_flat_static reject an empty step-size table and slices that do not fit the arenas
     (a sum offset + count that wraps included) before anything touches the device."""
