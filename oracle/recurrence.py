@@ -140,3 +140,53 @@ def run(params0, tau_fwd, tau_bkwd, grad_fn, n_steps, hp, dtype=np.float32, on_s
             on_step(t, w)
     res.params, res.delta, res.opt = w, delta, opt
     return res
+
+
+def run_stochastic(params0, delays, tau_mean, grad_fn, n_steps, hp, dtype=np.float32, on_step=None):
+    """Stage-wise stochastic gradient delays (Appendix E, the Hogwild!-style variant):
+
+        w_{i,t+1} = w_{i,t} - alpha [grad f_{t - tau_i}(w_{t - tau_i})]_i
+
+    Every microbatch t is differentiated at ONE consistent set of weights, the current w_t (forward and backward read the
+    same version), and stage i's slice of that gradient is applied tau_{i,t'} steps later: at step t stage i takes its
+    slice of the gradient of microbatch t - delays[t][i].
+
+    delays:   delays[t][i] >= 0, drawn by the caller (the appendix samples exponentials truncated at tau_max, with a
+              different mean per stage).
+    tau_mean: per stage, the delay the step-size rule T1 divides by (the mean of the stage's distribution, as an integer).
+    Readings: while t - delays[t][i] < 0 no gradient has reached stage i yet and it is left alone (its optimiser state and
+    step counters included: a stage's update index -- for the base step-size schedule, the T1 annealing and Adam's bias
+    correction -- counts the updates it has applied); T2 has nothing to correct (forward and backward read the same
+    weights).
+    Returns a Result; book holds (t, stage (1-based), microbatch whose gradient was applied or -1, updates applied so far).
+    """
+    P = len(params0)
+    w = [[np.array(a, dtype=dtype) for a in stage] for stage in params0]
+    opt = [[U.fresh_opt_state(a, hp["optimizer"]) for a in stage] for stage in w]
+    delta = [[np.zeros_like(a) for a in stage] for stage in w]
+    n_applied = [0] * P
+    grads_of = []                                   # grads_of[s][i]: stage i's slice of the gradient of microbatch s
+    res = Result()
+    hp_stage = dict(hp, t2=False)
+    for t in range(n_steps):
+        loss, grads = grad_fn(t, w, w)
+        res.losses.append(loss)
+        grads_of.append([[np.asarray(g, dtype=dtype) for g in stage] for stage in grads])
+        for i in range(P):
+            s = t - int(delays[t][i])
+            if s < 0:
+                res.book.append((t, i + 1, -1, n_applied[i]))
+                continue
+            new_stage = []
+            for j, a in enumerate(w[i]):
+                a_new, opt[i][j], delta[i][j] = U.pipemare_update(
+                    a, opt[i][j], delta[i][j], grads_of[s][i][j], k=n_applied[i], tau_fwd=tau_mean[i], tau_bkwd=tau_mean[i],
+                    hp=hp_stage, k_t1=n_applied[i])
+                new_stage.append(a_new)
+            w[i] = new_stage
+            n_applied[i] += 1
+            res.book.append((t, i + 1, s, n_applied[i]))
+        if on_step is not None:
+            on_step(t, w)
+    res.params, res.delta, res.opt = w, delta, opt
+    return res

@@ -539,3 +539,60 @@ def test_correction_reads_the_accumulator_of_the_corrected_version():
         delta.append(gamma * delta[-1] + (1 - gamma) * (-0.1))
     expect = [1.0] + [(1 - 0.1 * (t - 1)) - 2 * delta[t - 1] for t in range(1, 5)]
     assert seen == pytest.approx(expect, rel=1e-12)
+
+
+# ---- stage-wise stochastic delays (Appendix E) ----------------------------------------------------------------------
+
+def test_stochastic_delays_all_zero_is_synchronous_sgd_bit_for_bit():
+    params, grad_fn = tiny_net(seed=6, P=3)
+    hp = hp_(alpha=0.05, beta1=0.9)
+    a = recurrence.run(params, [0] * 3, [0] * 3, grad_fn, 20, hp)
+    b = recurrence.run_stochastic(params, [[0] * 3] * 20, [0] * 3, grad_fn, 20, hp)
+    for sa, sb in zip(a.params, b.params):
+        for x, y in zip(sa, sb):
+            assert np.array_equal(x, y)
+    assert a.losses == b.losses
+
+
+def test_stochastic_delays_constant_delay_is_delayed_sgd_on_consistent_weights():
+    # one constant delay for every stage: w_{t+1} = w_t - alpha grad f_{t-tau}(w_{t-tau}), written out directly
+    params, grad_fn = tiny_net(seed=7, P=3)
+    tau, n, alpha = 4, 18, 0.05
+    res = recurrence.run_stochastic(params, [[tau] * 3] * n, [tau] * 3, grad_fn, n, hp_(alpha=alpha), dtype=np.float64)
+    w = [[np.array(a, dtype=np.float64) for a in st] for st in params]
+    past = []
+    for t in range(n):
+        past.append(grad_fn(t, w, w)[1])
+        if t - tau >= 0:
+            g = past[t - tau]
+            w = [[a - alpha * np.asarray(gg) for a, gg in zip(st, gs)] for st, gs in zip(w, g)]
+    for sa, sb in zip(res.params, w):
+        for x, y in zip(sa, sb):
+            np.testing.assert_allclose(x, y, rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("tau,alpha", [(10, 0.2), (5, 0.2), (3, 0.3)])
+def test_stochastic_delay_model_follows_section3_polynomial_for_a_fixed_delay(tau, alpha):
+    # the gradient is taken at w_{t-tau}: on the scalar quadratic w_{t+1} = w_t - alpha lambda w_{t-tau}, whose growth rate
+    # is the largest root of w^(tau+1) - w^tau + alpha lambda (Section 3)
+    lam = 1.0
+    traj = []
+    recurrence.run_stochastic([[np.array([1.0])]], [[tau]] * 1200, [tau], quadratic_grad(lam), 1200, hp_(alpha=alpha),
+                              dtype=np.float64, on_step=lambda t, w: traj.append(float(w[0][0][0])))
+    coeffs = np.zeros(tau + 2)
+    coeffs[0], coeffs[1], coeffs[-1] = 1.0, -1.0, alpha * lam
+    assert growth_rate(np.array([1.0] + traj), 400, 1200) == pytest.approx(np.abs(np.roots(coeffs)).max(), rel=2e-3)
+
+
+def test_stochastic_delays_bookkeeping_and_t1_by_hand():
+    # two scalar stages, gradient 1 for both: stage 1 waits two steps, then takes steps of alpha / tau^p
+    def grad_fn(t, u_fwd, u_bkwd):
+        return 0.0, [[np.array([1.0])], [np.array([1.0])]]
+    delays = [[2, 0], [2, 1], [2, 0], [1, 3], [0, 0]]
+    hp = hp_(alpha=0.1, t1=True, K=2)
+    res = recurrence.run_stochastic([[np.array([0.0])], [np.array([0.0])]], delays, [3, 1], grad_fn, 5, hp, dtype=np.float64)
+    assert [b for b in res.book if b[1] == 1] == [(0, 1, -1, 0), (1, 1, -1, 0), (2, 1, 0, 1), (3, 1, 2, 2), (4, 1, 4, 3)]
+    assert [b for b in res.book if b[1] == 2] == [(0, 2, 0, 1), (1, 2, 0, 2), (2, 2, 2, 3), (3, 2, 0, 4), (4, 2, 4, 5)]
+    # stage 1: its k-th update (k = 0, 1, 2) uses alpha / 3^(1 - min(k/2, 1)) = 0.1/3, 0.1/sqrt(3), 0.1
+    assert res.params[0][0][0] == pytest.approx(-(0.1 / 3 + 0.1 / math.sqrt(3) + 0.1), rel=1e-12)
+    assert res.params[1][0][0] == pytest.approx(-0.5, rel=1e-12)
