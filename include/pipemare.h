@@ -184,6 +184,17 @@ typedef struct {
                                     pm_update, whose update kernel covers the remaining parameters (biases, LayerNorm
                                     parameters, embedding tables).  Needs PM_BF16, one Linear per stage, n_micro <= 1,
                                     entry_period <= 1 and recompute_segment = 0, else PM_ERR_UNSUPPORTED.  0: off. */
+  int32_t stochastic_tau_max;    /* > 0: the stage-wise stochastic delay model of Appendix E instead of the pipeline's fixed delays:
+                                      w_{i,t+1} = w_{i,t} - alpha [grad f_{t-tau_i}(w_{t-tau_i})]_i,   tau_i drawn per step and stage.
+                                    Every microbatch runs forward and backward on the current weights of all stages; the
+                                    gradients of the last stochastic_tau_max + 1 microbatches are kept (a ring of that many
+                                    copies of the grad arena, counted by pm_query_bytes), and at step t stage i applies its slice
+                                    of the gradient of microbatch t - tau_i, tau_i from pm_set_delays (0 <= tau_i <=
+                                    stochastic_tau_max); while t - tau_i < 0 the stage is left alone.  A stage's update index
+                                    (step-size schedule, T1 annealing, Adam's bias correction) counts the updates it has applied;
+                                    pm_stage_desc.tau_fwd is the delay T1 divides by (the mean of the stage's distribution),
+                                    tau_bkwd must be 0 and T2 has nothing to correct.  Needs PM_MB_MAJOR, n_micro <= 1,
+                                    recompute_segment = 0, fuse_update = 0, else PM_ERR_UNSUPPORTED.  0: off. */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /
@@ -272,13 +283,19 @@ pm_status pm_backward(pm_ctx* ctx);
 pm_status pm_update(pm_ctx* ctx);
 pm_status pm_step(pm_ctx* ctx, const void* inputs, const void* targets);
 
+/* Stochastic delay model (pm_config.stochastic_tau_max > 0): the delays of the NEXT step, one per stage (host array of
+ * n_stages entries, copied during the call), each in [0, stochastic_tau_max], else PM_ERR_INVALID_ARG.  They stay in force
+ * until the next call; before the first call every delay is 0.  PM_ERR_STATE outside that model. */
+pm_status pm_set_delays(pm_ctx* ctx, const int32_t* delays);
+
 /* Per-stage record of the last completed tick, written by the device kernels, for the
  * delay-bookkeeping check.  out[0..7] = forward microbatch (-1 if idle), weight version
  * the forward read, backward microbatch (-1 if idle), weight version the backward read,
  * updates applied so far, forward ring slot, backward ring slot, tick.  Synchronises.
  * PM_MB_MAJOR: the record of the last completed microbatch (both passes of every stage are active); out[7] is
  * that microbatch's index, out[5] the slot of the weight-version queue the forward read; with recompute_segment > 0
- * out[6] is the weight version the recomputation read. */
+ * out[6] is the weight version the recomputation read; with stochastic_tau_max > 0 out[6] is the microbatch whose gradient
+ * the stage applied in the last step (-1: none) and out[1] = out[3] the updates it had applied when the step began. */
 pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8);
 
 /* Copy losses of microbatches first_mb .. first_mb+n-1 to host_out.  The loss of microbatch

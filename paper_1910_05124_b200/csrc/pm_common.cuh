@@ -108,6 +108,8 @@ struct StageDyn {
   int64_t r_ver;              // weight version the recomputation of the microbatch in backward reads (PipeMare Recompute)
   float rc_gap;               // tau_fwd - tau_recomp
   int32_t _pad2;
+  int64_t g_shift;            // the update reads the gradient of element e at gsrc[g_shift + e] (0: the grad arena itself; stochastic
+                              // delays: the slot of the gradient ring that holds the microbatch this stage applies)
 };
 
 // Hyper-parameters the schedule kernel needs.
@@ -125,7 +127,8 @@ struct HyperDev {
   int32_t n_micro;            // N: microbatches per update (microbatch-major order; 1 elsewhere)
   int32_t entry_period;       // tick-major order: a microbatch enters every entry_period ticks (1: every tick)
   int32_t segment;            // PipeMare Recompute: stages per segment (0: no recomputation)
-  int32_t _pad;
+  int32_t stochastic;         // stage-wise stochastic delays (Appendix E): slots of the gradient ring, tau_max + 1 (0: off)
+  uint64_t total;             // elements of the arenas (one slot of the gradient ring)
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks

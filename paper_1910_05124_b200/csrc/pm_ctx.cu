@@ -29,6 +29,8 @@ struct Layout {
   std::vector<uint32_t> skip_b64, skip_e64;   // per stage, the Linear matrix's range in 64-element groups (fused update), else empty
   uint64_t off_skb = 0, off_ske = 0;
   int32_t fuse = 0;                     // the weight-gradient GEMM applies the update of the Linear matrices in its epilogue
+  int32_t stochastic = 0;               // stage-wise stochastic delays (Appendix E): slots of the gradient ring (tau_max + 1), 0: off
+  uint64_t g_ring = 0, off_delays = 0;  // ring: [stochastic][total] float gradients of the last microbatches; ws: the step's delays [P]
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
   // workspace offsets
   uint64_t off_st = 0, off_sched = 0, off_dyn = 0, off_nupd = 0, off_b64 = 0, off_e64 = 0, off_alpha = 0;
@@ -98,6 +100,17 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   }
   const int S = cfg->recompute_segment >= P ? 0 : cfg->recompute_segment;    // one segment covering everything: the forward pass itself
   L.segment = S;
+  if (cfg->stochastic_tau_max < 0) { err = "stochastic_tau_max must be >= 0"; return PM_ERR_INVALID_ARG; }
+  const bool stoch = cfg->stochastic_tau_max > 0;
+  if (stoch) {
+    const char* why = nullptr;
+    if (!mb) why = "PM_MB_MAJOR order (every microbatch is differentiated on one consistent set of weights)";
+    else if (cfg->n_micro > 1) why = "one microbatch per update";
+    else if (S > 0) why = "no recomputation";
+    else if (cfg->fuse_update) why = "the separate update kernel (gradients wait in a ring before they are applied)";
+    if (why) { err = std::string("stochastic_tau_max > 0 is built for ") + why; return PM_ERR_UNSUPPORTED; }
+  }
+  L.stochastic = stoch ? cfg->stochastic_tau_max + 1 : 0;
   if (cfg->entry_period < 0 || cfg->entry_period > 2 * P) { err = "entry_period must be in [0, 2 * n_stages]"; return PM_ERR_INVALID_ARG; }
   const int E = (!mb && cfg->entry_period > 1) ? cfg->entry_period : 1;
   const bool queue = mb || E > 1;
@@ -132,6 +145,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (ps != PM_OK) { stage_err(p, "bad op list"); return ps; }
     if (sd.param_count < need) { stage_err(p, "param_count smaller than its ops need"); return PM_ERR_INVALID_ARG; }
     s.tau_f = sd.tau_fwd; s.gap = sd.tau_fwd - sd.tau_bkwd;
+    if (stoch) s.gap = 0;                                    // forward and backward read the same weights: nothing for T2 to correct
     s.depth = s.tau_f + 1; s.xdepth = s.tau_f + 2;
     // the previous stage takes its ReLU mask from this stage's stashed input, one tick after this stage's own
     // backward: one more slot keeps it until then
@@ -139,7 +153,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     // microbatch-major order: one microbatch in flight, so every activation ring has one slot; what grows with
     // the delay is the queue of weight versions
     s.vdepth = 1;
-    if (mb) { s.depth = 1; s.xdepth = 1; s.vdepth = s.tau_f + 1; }
+    if (mb) { s.depth = 1; s.xdepth = 1; s.vdepth = stoch ? 1 : s.tau_f + 1; }   // stochastic delays: the live weights only
     // PipeMare Recompute (Appendix A.2): inside a segment the recomputation runs ahead of the backward pass like the
     // forward pass of a pipeline of that many stages, tau_recomp = ceil((2(S - j) + 1) / N) for the j-th stage of a
     // segment of S, never above tau_fwd; the last segment's backward follows its forward at that very distance, so
@@ -370,8 +384,9 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   for (int p = 0; p < P; ++p)
     if (feeds_attention(L.st[p].post) && (L.st[p].seq_len != L.att_S || !attn_tc_supported(cfg->compute_dtype, L.st[p].seq_len, L.st[p].d_out_main / L.st[p].n_heads))) L.att_tc = false;
   if (L.att_blocks > 0 && !L.att_tc && attention_smem_bytes(L.att_S, L.att_dk, cfg->compute_dtype) > 227 * 1024) { err = "attention tile (seq_len x head width) does not fit in shared memory"; return PM_ERR_UNSUPPORTED; }
-  L.ring_bytes = ring;
   L.total = L.st[P - 1].end;
+  if (L.stochastic > 0) { L.g_ring = ring; ring = align_up(ring + (uint64_t)L.stochastic * L.total * 4, 256); }   // gradients of the last tau_max + 1 microbatches
+  L.ring_bytes = ring;
   L.n_in_first = L.st[0].pre == PRE_EMBED ? 0 : L.st[0].lin[0].n_in;
   L.n_out_last = L.st[P - 1].lin[L.st[P - 1].n_lin - 1].n_out;
   L.loss_cap = cfg->loss_log_capacity > 0 ? cfg->loss_log_capacity : 4096;
@@ -383,6 +398,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.off_nupd = w; w = align_up(w + sizeof(int64_t) * P, 256);
   L.off_b64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_e64 = w; w = align_up(w + sizeof(uint32_t) * P, 256);
+  L.off_delays = w; w = align_up(w + sizeof(int32_t) * P, 256);
   L.off_skb = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_ske = w; w = align_up(w + sizeof(uint32_t) * P, 256);
   L.off_alpha = w; w = align_up(w + sizeof(double) * (cfg->alpha_by_step ? (uint64_t)cfg->alpha_len : 0), 256);
@@ -478,6 +494,7 @@ struct pm_ctx {
   cudaEvent_t ev_sched = nullptr, ev_fwd = nullptr;
   bool fwd_pending = false;             // work of the last tick's forward may still be running on fwd_stream
   std::vector<int> seg_first, seg_count;   // small-tensor segments of a stage: [seg_first[p], + seg_count[p])
+  std::vector<int32_t> h_delays;           // stochastic delay model: host copy of the delays in force
   bool graphs = true;
   cudaStream_t cap_stream = nullptr;
   cudaStream_t ls = nullptr;            // the stream the phase bodies launch on: `stream`, or `cap_stream` while capturing
@@ -622,6 +639,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   }
   e = cudaMemsetAsync(c->ws + L.off_nupd, 0, sizeof(int64_t) * P, c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_dyn, 0, sizeof(StageDyn) * P * (uint64_t)L.n_tables, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_delays, 0, sizeof(int32_t) * P, c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.off_lossred, 0, 512, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // host tables may go out of scope after this
   if (e != cudaSuccess) { pm_status r = cuda_fail(nullptr, e, "context set-up"); delete c; return r; }
@@ -637,6 +655,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.mb_major = L.queue ? 1 : 0; c->hp.lp_elem = cfg->compute_dtype == PM_F32 ? 4 : 2;
   c->hp.n_micro = cfg->n_micro > 1 ? cfg->n_micro : 1;
   c->hp.segment = L.segment;
+  c->hp.stochastic = L.stochastic; c->hp.total = L.total;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -895,8 +914,11 @@ static pm_status mb_forward(pm_ctx* ctx, const void* inputs, const void* targets
   const int P = ctx->cfg.n_stages;
   const int64_t mb = ctx->n_fed;
   pm_status s;
+  const bool stoch = ctx->L.stochastic > 0;
   s = TIMED(PM_PROF_SCHEDULE, check(ctx, launch_schedule_mb((const StageSched*)(ctx->ws + ctx->L.off_sched), (StageDyn*)(ctx->ws + ctx->L.off_dyn),
-                                                            ctx->hp, mb, ctx->stream), "schedule"));
+                                                            ctx->hp, mb, ctx->stream,
+                                                            stoch ? (const int32_t*)(ctx->ws + ctx->L.off_delays) : nullptr,
+                                                            stoch ? (const int64_t*)(ctx->ws + ctx->L.off_nupd) : nullptr), "schedule"));
   if (s != PM_OK) return s;
   s = TIMED(PM_PROF_INGEST, check(ctx, launch_ingest(ctx->ta, dt, inputs, (const float*)targets, mb, ctx->stream), "ingest"));
   if (s != PM_OK) return s;
@@ -975,6 +997,17 @@ static pm_status mb_update(pm_ctx* ctx) {
     return PM_OK;
   }
   const StageDyn* dyn_all = (const StageDyn*)(ctx->ws + ctx->L.off_dyn) + (size_t)2 * P * P;
+  const float* gsrc = nullptr;
+  if (ctx->L.stochastic > 0) {
+    // stochastic delays (Appendix E): this microbatch's gradients join the ring of the last tau_max + 1; every stage's update
+    // reads the slot its table entry names (the slot changes from step to step, so the copy stays outside the graph)
+    float* gq = reinterpret_cast<float*>(ctx->ta.ring + ctx->L.g_ring);
+    const int64_t mb = ctx->n_fed - 1;
+    cudaError_t ce = cudaMemcpyAsync(gq + (uint64_t)(mb % ctx->L.stochastic) * ctx->L.total, ctx->a.grad, ctx->L.total * sizeof(float),
+                                     cudaMemcpyDeviceToDevice, ctx->stream);
+    if (ce != cudaSuccess) return cuda_fail(ctx, ce, "gradient ring copy");
+    gsrc = gq;
+  }
   pm_status s = run_phase(ctx, ctx->g_upd, [&]() -> pm_status {
     // fused update: the weight gradients of all stages as one launch whose epilogue updates the Linear matrices
     if (ctx->L.fuse) { pm_status fs = grouped_wgrad(ctx, 2 * P, true); if (fs != PM_OK) return fs; }
@@ -983,7 +1016,7 @@ static pm_status mb_update(pm_ctx* ctx) {
                                   (int64_t*)(ctx->ws + ctx->L.off_nupd), P, ctx->L.total / 64, ctx->cfg.optimizer, ctx->cfg.beta1,
                                   ctx->cfg.beta2, ctx->cfg.eps, ctx->ls, ctx->ta.ring, ctx->hp.lp_elem, 0,
                                   ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_skb) : nullptr,
-                                  ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_ske) : nullptr);
+                                  ctx->L.fuse ? (const uint32_t*)(ctx->ws + ctx->L.off_ske) : nullptr, gsrc);
     pm_status s = check(ctx, e, "update");
     if (s != PM_OK || ctx->L.segs.empty()) return s;
     prof_begin(ctx, PM_PROF_UPDATE);
@@ -1227,6 +1260,20 @@ static pm_status check_device_status(pm_ctx* ctx) {
   return PM_OK;
 }
 
+pm_status pm_set_delays(pm_ctx* ctx, const int32_t* delays) {
+  if (!ctx || !delays) return fail(ctx, PM_ERR_INVALID_ARG, "null argument");
+  if (ctx->L.stochastic == 0) return fail(ctx, PM_ERR_STATE, "pm_set_delays belongs to the stochastic delay model (pm_config.stochastic_tau_max > 0)");
+  if (ctx->phase != 0) return fail(ctx, PM_ERR_STATE, "pm_set_delays between steps only");
+  const int P = ctx->cfg.n_stages;
+  for (int p = 0; p < P; ++p)
+    if (delays[p] < 0 || delays[p] >= ctx->L.stochastic) return fail(ctx, PM_ERR_INVALID_ARG, "delay of stage " + std::to_string(p) + " outside [0, stochastic_tau_max]");
+  ctx->h_delays.assign(delays, delays + P);
+  // ordered on the context's stream behind the previous step's schedule kernel, which read the old values
+  cudaError_t e = cudaMemcpyAsync(ctx->ws + ctx->L.off_delays, ctx->h_delays.data(), sizeof(int32_t) * P, cudaMemcpyHostToDevice, ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "delay upload");
+  return PM_OK;
+}
+
 pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
   if (!ctx || !out8) return fail(ctx, PM_ERR_INVALID_ARG, "null argument");
   if (stage < 0 || stage >= ctx->cfg.n_stages) return fail(ctx, PM_ERR_INVALID_ARG, "stage out of range");
@@ -1246,6 +1293,12 @@ pm_status pm_get_bookkeeping(pm_ctx* ctx, int32_t stage, int64_t* out8) {
     if (pm_status ds = check_device_status(ctx)) return ds;
     out8[0] = df.f_mb; out8[1] = df.f_ver; out8[2] = db.b_mb; out8[3] = db.b_ver; out8[4] = n;
     out8[5] = df.f_vslot; out8[6] = ctx->L.segment > 0 ? db.r_ver : (int64_t)db.b_slot; out8[7] = ctx->n_fed - 1;
+    if (ctx->L.stochastic > 0) {                                  // the update table's entry names the microbatch whose gradient was applied
+      StageDyn du;
+      e = cudaMemcpy(&du, tab + sizeof(StageDyn) * ((size_t)(2 * P) * P + stage), sizeof(StageDyn), cudaMemcpyDeviceToHost);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "bookkeeping read-back");
+      out8[6] = du.r_ver;
+    }
     return PM_OK;
   }
   if (e == cudaSuccess) e = cudaMemcpy(&d, ctx->ws + ctx->L.off_dyn + sizeof(StageDyn) * stage, sizeof(StageDyn), cudaMemcpyDeviceToHost);

@@ -31,7 +31,7 @@ __device__ StageDyn make_dyn(const StageSched& s, const HyperDev& hp, int64_t ti
   StageDyn d;
   d.tick = tick;
   d.accum = 0; d._pad2 = 0;
-  d.rc_uslot = -1; d.rc_shift = 0; d.r_ver = fver; d.rc_gap = 0.f;
+  d.rc_uslot = -1; d.rc_shift = 0; d.r_ver = fver; d.rc_gap = 0.f; d.g_shift = 0;
   if (kb == -2) kb = b;                               // update index the microbatch in backward belongs to (N = 1: itself)
   const bool fa = a >= 0, ba = b >= 0;
   d.f_mb = a; d.b_mb = b; d.k = k;
@@ -124,7 +124,8 @@ cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageD
 // older than the end of the warm-up), the backward the live weights (version t).  Table v in 0..2P-1 serves the
 // launches of sub-tick v; table 2P marks every stage in backward with its own backward sub-tick's slots and an
 // active update: it serves the grouped weight-gradient launch and the fused update.
-__global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDyn* __restrict__ tables, HyperDev hp, int64_t t) {
+__global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDyn* __restrict__ tables, HyperDev hp, int64_t t,
+                                   const int32_t* __restrict__ delays, const int64_t* __restrict__ nupd) {
   const int P = hp.n_stages;
   const int i = blockIdx.x * blockDim.x + threadIdx.x, v = blockIdx.y;
   if (i >= P) return;
@@ -138,6 +139,22 @@ __global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDy
   if (u < hp.warm) fver = u; else if (fver < hp.warm) fver = hp.warm;
   if (fver < 0) fver = 0;
   StageDyn d;
+  if (hp.stochastic > 0) {
+    // Stage-wise stochastic delays (Appendix E): forward and backward of microbatch t on the stage's current weights
+    // (version = updates it has applied); the update table activates the stage when the gradient of microbatch
+    // t - delay exists, points it at that microbatch's slot of the gradient ring and indexes its step-size schedule,
+    // T1 annealing and bias corrections by the stage's own update count
+    const int64_t ver = nupd[i];
+    const int64_t src = t - (int64_t)delays[i];
+    if (v < 2 * P) d = make_dyn(s, hp, base + v, v == i ? t : -1, v == 2 * P - 1 - i ? t : -1, -1, ver, ver, true, ver);
+    else {
+      d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, t, src >= 0 ? ver : -1, ver, ver, true, ver);
+      d.g_shift = src >= 0 ? (src % hp.stochastic) * (int64_t)hp.total : 0;
+    }
+    d.r_ver = src >= 0 ? src : -1;
+    tables[(size_t)v * P + i] = d;
+    return;
+  }
   // PipeMare Recompute (Appendix A.2, Appendix D): the version the recomputation reads, clamped like the forward's
   int64_t rver = u - s.tau_r;
   if (u < hp.warm) rver = u; else if (rver < hp.warm) rver = hp.warm;
@@ -160,10 +177,11 @@ __global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDy
   tables[(size_t)v * P + i] = d;
 }
 
-cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream) {
+cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream,
+                               const int32_t* delays, const int64_t* nupd) {
   const int threads = 128;
   dim3 grid((hp.n_stages + threads - 1) / threads, mb_table_count(hp.n_stages, hp.segment));
-  schedule_mb_kernel<<<grid, threads, 0, stream>>>(sched, tables, hp, t);
+  schedule_mb_kernel<<<grid, threads, 0, stream>>>(sched, tables, hp, t, delays, nupd);
   return cudaGetLastError();
 }
 
@@ -181,7 +199,8 @@ template <int OPT, int LP>
 __global__ void __launch_bounds__(kUpdThreads, 3)
 update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restrict__ begin64, const uint32_t* __restrict__ end64,
               const StageDyn* __restrict__ dyn, int64_t* __restrict__ nupd, int n_stages, uint64_t total_vec4,
-              float beta1, float beta2, float eps, uint64_t first_vec4, const uint32_t* __restrict__ skip_b64, const uint32_t* __restrict__ skip_e64) {
+              float beta1, float beta2, float eps, uint64_t first_vec4, const uint32_t* __restrict__ skip_b64, const uint32_t* __restrict__ skip_e64,
+              const float* __restrict__ gsrc) {
   extern __shared__ uint32_t sm_bounds[];           // [n_stages] begins, then [n_stages] ends, then the skipped ranges' begins and ends
   uint32_t* sb = sm_bounds;
   uint32_t* se = sm_bounds + n_stages;
@@ -225,10 +244,10 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
       }
       if (stage[u] >= 0) {
         const uint64_t e = v[u] * 4;
-        g[u] = ld_stream(a.grad + e);
+        const StageDyn& d = dyn[stage[u]];
+        g[u] = ld_stream(gsrc + (d.g_shift + (int64_t)e));
         w[u] = ld_stream(a.w + e);
         m[u] = ld_stream(a.m + e);
-        const StageDyn& d = dyn[stage[u]];
         sc[u].alpha = d.alpha; sc[u].gamma = d.gamma; sc[u].omg = d.one_minus_gamma;
         sc[u].bc1 = d.bc1; sc[u].bc2 = d.bc2; sc[u].use_delta = d.use_delta;
         if (LP != 0) { sc[u].lp_shift = d.lp_shift; sc[u].rc_shift = d.rc_uslot >= 0 ? d.rc_shift : -1; sc[u].rc_gap = d.rc_gap; }
@@ -285,7 +304,7 @@ update_kernel(ArenasDev a, void* __restrict__ lp_base, const uint32_t* __restric
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
                           float eps, cudaStream_t stream, void* lp_base, int lp_elem, uint64_t first64,
-                          const uint32_t* skip_b64, const uint32_t* skip_e64) {
+                          const uint32_t* skip_b64, const uint32_t* skip_e64, const float* gsrc) {
   if (total64 == 0 || n_stages == 0 || first64 >= total64) return cudaSuccess;
   uint64_t total_vec4 = total64 * 16;
   const uint64_t first_vec4 = first64 * 16;
@@ -299,8 +318,9 @@ cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* 
   size_t smem = sizeof(uint32_t) * 4 * (size_t)n_stages;
   // the operand-type copy: the w_lp arena (bfloat16) unless the caller names a version ring and its element size
   if (lp_base == nullptr) { lp_base = a.w_lp; lp_elem = 2; }
+  if (gsrc == nullptr) gsrc = a.grad;
   const int lp = lp_base == nullptr ? 0 : (lp_elem == 4 ? 2 : 1);
-#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps, first_vec4, skip_b64, skip_e64)
+#define PM_UPD(OPT, LP) update_kernel<OPT, LP><<<blocks, kUpdThreads, smem, stream>>>(a, lp_base, begin64, end64, dyn, nupd, n_stages, total_vec4, beta1, beta2, eps, first_vec4, skip_b64, skip_e64, gsrc)
   if (optimizer == PM_SGDM) { if (lp == 0) PM_UPD(PM_SGDM, 0); else if (lp == 1) PM_UPD(PM_SGDM, 1); else PM_UPD(PM_SGDM, 2); }
   else { if (lp == 0) PM_UPD(PM_ADAM, 0); else if (lp == 1) PM_UPD(PM_ADAM, 1); else PM_UPD(PM_ADAM, 2); }
 #undef PM_UPD

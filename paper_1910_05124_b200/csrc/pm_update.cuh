@@ -24,7 +24,9 @@ cudaError_t launch_schedule(const StageSched* sched, const int64_t* nupd, StageD
 // and the update.  With PipeMare Recompute (hp.segment > 0) table 2P + 1 holds every stage's recomputation (its forward
 // entry with the recompute weights' slot) and table 2P + 2 + k the backward entries of segment k alone (the grouped
 // weight-gradient launch of that segment).
-cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream);
+// delays / nupd (stochastic delay model only, else null): the step's per-stage delays and the stages' update counters.
+cudaError_t launch_schedule_mb(const StageSched* sched, StageDyn* tables, HyperDev hp, int64_t t, cudaStream_t stream,
+                               const int32_t* delays = nullptr, const int64_t* nupd = nullptr);
 inline int mb_table_count(int P, int segment) { return 2 * P + 1 + (segment > 0 ? 1 + (P + segment - 1) / segment : 0); }
 
 // Launches the fused update over all stages whose dyn[i].active_update is set.
@@ -32,7 +34,8 @@ inline int mb_table_count(int P, int segment) { return 2 * P + 1 + (segment > 0 
 cudaError_t launch_update(ArenasDev a, const uint32_t* begin64, const uint32_t* end64, const StageDyn* dyn,
                           int64_t* nupd, int n_stages, uint64_t total64, int optimizer, float beta1, float beta2,
                           float eps, cudaStream_t stream, void* lp_base = nullptr, int lp_elem = 0, uint64_t first64 = 0,
-                          const uint32_t* skip_b64 = nullptr, const uint32_t* skip_e64 = nullptr);
+                          const uint32_t* skip_b64 = nullptr, const uint32_t* skip_e64 = nullptr, const float* gsrc = nullptr);
+// gsrc: where the gradients are read (element e of stage i at gsrc[dyn[i].g_shift + e]); null: the grad arena.
 // skip_b64 / skip_e64: per stage, a range of 64-element groups this launch leaves alone (device arrays, or null): the
 // Linear matrices when the weight-gradient GEMM has applied their update in its epilogue.  The stage's update
 // counter is incremented here all the same.

@@ -12,5 +12,5 @@ from .configs import (  # noqa: F401
     Workload, LinearSpec, pipemare_delays, mlp_workload, cfg1, cfg3, cfg3_small,
     update_sweep_case, init_stage_params, teacher_params, batch, round_to_bf16,
     StageSpec, encoder_workload, cfg4, cfg4_small, init_encoder_params, token_batch,
-    encdec_workload, cfg5, cfg5_cut, cfg5_small, seq2seq_batch,
+    encdec_workload, cfg5, cfg5_cut, cfg5_small, seq2seq_batch, stochastic_delays,
 )

@@ -335,3 +335,17 @@ def token_batch(wl, t):
     n_seq = wl.microbatch // wl.seq_len
     ids = rng.randint(wl.seed, _S_TOKENS + 16 * t, wl.microbatch, wl.vocab).reshape(n_seq, wl.seq_len)
     return ids.reshape(-1).astype(np.int64), ids[:, ::-1].reshape(-1).astype(np.int64)
+
+
+_S_DELAYS = 900000
+
+
+def stochastic_delays(seed, n_steps, means, tau_max):
+    """Integer gradient delays of the stage-wise stochastic delay model (Appendix E): for every step and stage a draw
+    from the exponential distribution with the stage's mean, truncated below tau_max + 1 (inverse CDF on a counter-based
+    uniform) and rounded down.  Returns a list of n_steps lists of len(means) integers in [0, tau_max]."""
+    P = len(means)
+    u = rng.uniform01(seed, _S_DELAYS, n_steps * P).reshape(n_steps, P)
+    mu = np.maximum(np.asarray(means, dtype=np.float64), 1e-9)[None, :]
+    x = -mu * np.log(1.0 - u * (1.0 - np.exp(-float(tau_max + 1) / mu)))
+    return np.minimum(np.floor(x).astype(np.int64), tau_max).tolist()

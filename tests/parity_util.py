@@ -5,7 +5,7 @@ import pm_inputs as I
 
 
 def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1, entry_period=1,
-                     segment=0, book_recomp=None, fuse_update=0):
+                     segment=0, book_recomp=None, fuse_update=0, delays=None, tau_max=0, book_applied=None):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
@@ -13,11 +13,13 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
     loop_order "mb_major": one call of pm_step per microbatch, nothing to drain.
     segment: stages per recompute segment (PipeMare Recompute); book_recomp, a dict, then receives
     (microbatch, stage 1-based) -> version the recomputation read.
+    delays, tau_max: the stage-wise stochastic delay model: delays[t][i] is set before step t; book_applied, a dict, then
+    receives (step, stage 1-based) -> (microbatch whose gradient was applied or -1, updates applied after the step).
     """
     import torch
     import paper_1910_05124_b200 as pm
     pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro, entry_period=entry_period, recompute_segment=segment,
-                       fuse_update=fuse_update)
+                       fuse_update=fuse_update, stochastic_tau_max=tau_max)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
@@ -38,6 +40,8 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
             mb = s // E if s % E == 0 else -1
         else:
             mb = (s // (2 * P) if s % (2 * P) == 0 else -1) if s < t0 else warmup + (s - t0)
+        if delays is not None:
+            pipe.pm_set_delays(delays[s])
         if 0 <= mb < n_steps:
             if encoder and is_encdec(wl):
                 src, dec_in, tg = I.seq2seq_batch(wl, mb)              # two token streams: [source | decoder input]
@@ -60,6 +64,9 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
                 assert tick == s
                 if f_mb >= 0:
                     book.setdefault((f_mb, p + 1), [None, None])[0] = f_ver
+                if book_applied is not None:
+                    book_applied[(s, p + 1)] = (b_slot, n_upd)
+                    continue
                 if b_mb >= 0:
                     book.setdefault((b_mb, p + 1), [None, None])[1] = b_ver
                     assert n_upd == b_ver + (1 if (b_mb + 1) % n_micro == 0 else 0)      # the update follows the N-th microbatch

@@ -250,6 +250,38 @@ def test_recompute_and_fused_update_options_are_checked_without_a_gpu(built_lib)
         setattr(cfg, field, old)
 
 
+def test_stochastic_delay_model_footprint_and_checks_without_a_gpu(built_lib):
+    """Appendix E's model keeps the gradients of the last tau_max + 1 microbatches (copies of the grad arena) and one weight
+    version per stage; its preconditions are reported as PM_ERR_UNSUPPORTED."""
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    wl = I.cfg4()
+    cfg, sd, keep = _describe(wl)
+    cfg.loop_order = B.PM_MB_MAJOR
+    sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    total = sum(sd[p].param_count for p in range(wl.n_stages))
+    sizes = {}
+    for tmax in (1, 5):
+        cfg.stochastic_tau_max = tmax
+        assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+        sizes[tmax] = rb.value
+    assert sizes[5] - sizes[1] == 4 * total * 4
+    cfg.stochastic_tau_max = 0
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    assert rb.value > sizes[1] - 2 * total * 4                # without the model the stages queue tau_i + 1 weight versions instead
+    cfg.stochastic_tau_max = 3
+    for field, value in (("loop_order", B.PM_TICK_MAJOR), ("n_micro", 2), ("recompute_segment", 5), ("fuse_update", 1)):
+        old = getattr(cfg, field)
+        setattr(cfg, field, value)
+        st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+        assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED", field
+        setattr(cfg, field, old)
+    cfg.stochastic_tau_max = -2
+    assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
+
+
 def test_flat_update_argument_checks_need_no_gpu(built_lib):
     """pm_update_flat / pm_update_flat_static reject an empty step-size table and slices that do not fit the arenas
     (a sum offset + count that wraps included) before anything touches the device."""
