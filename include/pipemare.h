@@ -111,7 +111,10 @@ typedef struct {
  * stage's weights and the update that uses the resulting gradient.  PipeMare
  * (Table 1) has tau_fwd = 2(P-i)+1 and tau_bkwd = 0, which is the only delay
  * pattern the tick schedule (PM_TICK_MAJOR) realises; PM_MB_MAJOR takes any
- * tau_fwd >= 0 with tau_bkwd = 0; other values are PM_ERR_UNSUPPORTED.
+ * tau_fwd >= 0 with tau_bkwd = 0, or tau_bkwd = tau_fwd for EVERY stage: weight
+ * stashing (Section 2.2), the backward pass of a microbatch reads the queued version
+ * its forward read (weights in the operand type, LayerNorm gain in fp32), there is no
+ * discrepancy and T2 corrects nothing; other values are PM_ERR_UNSUPPORTED.
  * param_offset / param_count: this stage's slice of the flat arenas, in elements;
  * both multiples of PM_ALIGN_ELEMS.  Inside the slice each op's W and then b start
  * at the next multiple of PM_ALIGN_ELEMS (pm_op_param_offsets gives the numbers). */

@@ -29,6 +29,7 @@ struct Layout {
   std::vector<uint32_t> skip_b64, skip_e64;   // per stage, the Linear matrix's range in 64-element groups (fused update), else empty
   uint64_t off_skb = 0, off_ske = 0;
   int32_t fuse = 0;                     // the weight-gradient GEMM applies the update of the Linear matrices in its epilogue
+  int32_t stash = 0;                    // weight stashing: every stage has tau_bkwd = tau_fwd (microbatch-major order)
   int32_t stochastic = 0;               // stage-wise stochastic delays (Appendix E): slots of the gradient ring (tau_max + 1), 0: off
   uint64_t g_ring = 0, off_delays = 0;  // ring: [stochastic][total] float gradients of the last microbatches; ws: the step's delays [P]
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
@@ -125,6 +126,7 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   L.end64.assign(P, 0);
   uint64_t ring = 0;
   uint64_t prev_end = 0;
+  bool any_stash = false, any_plain = false;                 // stages with tau_bkwd = tau_fwd > 0 / with tau_bkwd = 0 < tau_fwd
   auto stage_err = [&](int p, const std::string& m) { err = "stage " + std::to_string(p) + ": " + m; };
   for (int p = 0; p < P; ++p) {
     const pm_stage_desc& sd = stages[p];
@@ -134,8 +136,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       stage_err(p, "the tick schedule realises tau_fwd = 2(P-i)+1, tau_bkwd = 0 only");
       return PM_ERR_UNSUPPORTED;
     }
-    if (mb && (sd.tau_bkwd != 0 || sd.tau_fwd < 0)) {
-      stage_err(p, "microbatch-major order takes tau_fwd >= 0 with tau_bkwd = 0");
+    if (mb && sd.tau_fwd >= 0 && sd.tau_bkwd == sd.tau_fwd && sd.tau_fwd > 0) any_stash = true;     // weight stashing (Section 2.2)
+    else if (mb && sd.tau_fwd > 0) any_plain = true;
+    if (mb && ((sd.tau_bkwd != 0 && sd.tau_bkwd != sd.tau_fwd) || sd.tau_fwd < 0 || (any_stash && any_plain))) {
+      stage_err(p, "microbatch-major order takes tau_fwd >= 0 with tau_bkwd = 0, or tau_bkwd = tau_fwd for every stage (weight stashing)");
       return sd.tau_fwd < 0 || sd.tau_bkwd < 0 ? PM_ERR_INVALID_ARG : PM_ERR_UNSUPPORTED;
     }
     if (sd.param_offset % PM_ALIGN_ELEMS || sd.param_count % PM_ALIGN_ELEMS) { stage_err(p, "param_offset/param_count must be multiples of 64"); return PM_ERR_INVALID_ARG; }
@@ -294,8 +298,10 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       // dgrad 0.215 -> 0.290 ms per tick against 0.014 ms saved in the activation-backward pass).
       const char* fuse_env = getenv("PM_RELU_FUSE");
       const bool fuse_ok = fuse_env && fuse_env[0] == '1';
+      // (never with weight stashing, whose plain dgrad epilogue applies no mask: a stage with tau_bkwd = tau_fwd > 0)
       if (fuse_ok && cfg->compute_dtype == PM_BF16 && last && (ld.flags & LF_ACT_FROM_Y) && next_takes_y &&
-          stages[p + 1].ops[0].kind == PM_OP_LINEAR)
+          stages[p + 1].ops[0].kind == PM_OP_LINEAR && !(sd.tau_fwd > 0 && sd.tau_bkwd == sd.tau_fwd) &&
+          !(stages[p + 1].tau_fwd > 0 && stages[p + 1].tau_bkwd == stages[p + 1].tau_fwd))
         ld.flags |= LF_DZ_FUSED;
     }
     if (p > 0 && (L.st[p - 1].lin[L.st[p - 1].n_lin - 1].flags & LF_DZ_FUSED)) s.mask_dx = 1;
@@ -345,6 +351,13 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     L.sched[p].tau_f = s.tau_f; L.sched[p].gap = s.gap; L.sched[p].depth = s.depth; L.sched[p].xdepth = s.xdepth;
     L.sched[p].vdepth = s.vdepth; L.sched[p].begin = s.begin; L.sched[p].count = s.end - s.begin; L.sched[p].v_ring = s.v_ring;
     L.sched[p].tau_r = s.tau_r; L.sched[p].rdepth = s.rdepth;
+  }
+  // Weight stashing (Section 2.2, tau_bkwd = tau_fwd): the backward pass of a microbatch reads the queued version its forward
+  // read, in the operand type (the copy the forward used), so dgrad is a plain GEMM and T2 has nothing to correct.
+  L.stash = any_stash ? 1 : 0;
+  if (L.stash && (S > 0 || stoch || cfg->fuse_update)) {
+    err = "weight stashing (tau_bkwd = tau_fwd) is not combined with recompute_segment, stochastic_tau_max or fuse_update";
+    return PM_ERR_UNSUPPORTED;
   }
   // Fused update (pm_config.fuse_update): the weight-gradient GEMM's epilogue updates the Linear matrices, the update
   // kernel the rest of every stage (biases, LayerNorm parameters, embedding tables, padding).
@@ -669,6 +682,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0;
   t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
+  t.stash = L.stash;
   t.fuse_upd = 0; t.upd_opt = cfg->optimizer; t.upd_beta1 = cfg->beta1; t.upd_beta2 = cfg->beta2; t.upd_eps = cfg->eps;
   t.upd_lp = L.queue ? reinterpret_cast<__nv_bfloat16*>(t.ring) : c->a.w_lp;
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
@@ -900,7 +914,7 @@ static pm_status stage_backward(pm_ctx* ctx, const TickArgs& ta, int p, bool gro
     }
     if (p == 0 && l == 0 && sd.pre != PRE_EMBED) continue;          // raw network inputs need no gradient
     prof_begin(ctx, PM_PROF_DGRAD);
-    e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, 1, l, ctx->ls);
+    e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, ctx->L.stash ? 4 : 1, l, ctx->ls);
     if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
   }
   const int n_pre = sd.pre != PRE_NONE ? pre_bwd_launches(ta) : 0;

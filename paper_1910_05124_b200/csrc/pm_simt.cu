@@ -386,7 +386,9 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(TickArgs t, int lvl) {
         float v = 0.f;
         if (n < N && k < K) {
           uint64_t idx = (uint64_t)k * L.n_in + n;
-          if (MODE == 1) {      // T2: w - (tau_fwd - tau_bkwd) * delta, then rounded as the operand type holds it
+          if (MODE == 1 && t.stash) {   // weight stashing: the queued version the forward read, as the operand type holds it
+            v = to_f<WT>(wf[idx]);
+          } else if (MODE == 1) {      // T2: w - (tau_fwd - tau_bkwd) * delta, then rounded as the operand type holds it
             float wv = wm[idx];
             if (corr) wv = __fsub_rn(wv, __fmul_rn(gapf, dl[idx]));
             v = round_as<WT>(wv);

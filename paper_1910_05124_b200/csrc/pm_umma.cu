@@ -38,7 +38,8 @@ constexpr int STG_BYTES = 2 * STG_HALF_BYTES;              // w tile + delta til
 constexpr int ACC_COLS = 128, TMEM_COLS = 2 * ACC_COLS;
 constexpr int N_EPI_WARPS = 8;
 
-template <int MODE> struct Cfg {                           // MODE 0 forward, 2 wgrad (dgrad has its own kernel)
+template <int MODE> struct Cfg {                           // MODE 0 forward, 2 wgrad, 1 dgrad against a QUEUED weight version (weight
+                                                           // stashing, tau_bkwd = tau_fwd: a plain bf16 operand; the corrected dgrad has kernels of its own)
   static constexpr int kStages = 4;                        // operand ring depth
   static constexpr int kThreads = 32 * (2 + N_EPI_WARPS);
   static constexpr int kOutWarpBytes = 8192;               // per epilogue warp: two boxes of 32 rows x 128 B
@@ -48,7 +49,7 @@ template <int MODE> struct Cfg {                           // MODE 0 forward, 2 
 };
 
 enum { MAP_ACT_K = 0, MAP_W_K = 1, MAP_DZ_K = 2, MAP_DZ_MN = 3, MAP_ACT_MN = 4, MAP_W_F32 = 5, MAP_D_F32 = 6,
-       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAP_W_F32Q = 11, MAP_D_F32Q = 12, MAP_W_F32H = 13, MAP_D_F32H = 14, MAPS_PER_LINEAR = 15 };
+       MAP_Z_OUT = 7, MAP_Y_OUT = 8, MAP_DX_OUT = 9, MAP_DW_OUT = 10, MAP_W_F32Q = 11, MAP_D_F32Q = 12, MAP_W_F32H = 13, MAP_D_F32H = 14, MAP_W_MN = 15, MAPS_PER_LINEAR = 16 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, operand majors as given.
 __device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
@@ -220,6 +221,15 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         else epi_zy8<PM_ACT_GELU>(pf, obuf + off, obuf + 4096 + off);
       }
     }
+  } else if (MODE == 1) {
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {                                 // dx: one bf16 output, 64 columns per row
+      float f[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(g < 4 ? r0[(g & 3) * 8 + e] : r1[(g & 3) * 8 + e]);
+      *reinterpret_cast<uint4*>(obuf + so + row_off + (((uint32_t)g ^ sw) << 4)) =
+          make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+    }
   } else {
 #pragma unroll
     for (int g = 0; g < 8; ++g) {                                 // two boxes of 32 fp32 columns
@@ -243,6 +253,9 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         tma_store_3d(lm + MAP_Z_OUT, obuf_s, nb, mrow, d.f_slot);
         tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb, mrow, yslot);
       }
+    } else if (MODE == 1) {
+      // to the previous stage's gradient mailbox, or this stage's own scratch when a pre-op stands before the Linear
+      tma_store_3d(lm + MAP_DX_OUT, obuf_s + so, nb, mrow, (lvl == 0 && s.pre == PRE_NONE) ? d.prev_wslot : 0);
     } else {
       if (d.accum) {                                                // a later microbatch of the minibatch: dW adds to the arena
         tma_reduce_add_2d(lm + MAP_DW_OUT, obuf_s, nb, mrow);
@@ -323,9 +336,10 @@ __device__ __forceinline__ Tile decode_tile(const TickArgs& t, const int* __rest
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
-  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0);
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
   const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
+  else if (MODE == 1) { r.M = t.T; r.N = L.n_in; r.K = L.n_out; }
   else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
   const int tiles_n = (r.N + TILE_N - 1) / TILE_N;
   const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
@@ -394,6 +408,7 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
         const StageDev& sd_ = t.st[tl.p];
         const int dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
+        else if (MODE == 1) { tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_MN); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         for (int kb = 0; kb < tl.n_kb; ++kb) {
           const int k0 = kb * TILE_K;
@@ -403,6 +418,13 @@ umma_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const int* __
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             tma_load_3d(sa, lm + MAP_ACT_K, fb, k0, tl.m0, (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.f_xslot : d.f_slot);
             tma_load_3d(sb, lm + MAP_W_K, fb, k0, tl.n0, d.f_vslot);
+          } else if (MODE == 1) {
+            // dx = dz W_v: dz K-major, the queued version v of the weights (the one the microbatch's forward read) as the
+            // MN-major operand, two 64-column runs
+            mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+            tma_load_3d(sa, lm + MAP_DZ_K, fb, k0, tl.m0, dz_slot);
+            tma_load_3d(sb, lm + MAP_W_MN, fb, tl.n0, k0, d.f_vslot);
+            tma_load_3d(sb + B_BYTES / 2, lm + MAP_W_MN, fb, tl.n0 + 64, k0, d.f_vslot);
           } else {
             mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
             const int slot = (lvl == 0 && t.st[tl.p].pre == PRE_NONE) ? d.b_xslot : d.b_slot;
@@ -536,9 +558,10 @@ __device__ __forceinline__ Tile decode_pair_tile(const TickArgs& t, const int* _
   r.p = lo;
   const StageDyn& d = t.dyn[lo];
   const StageDev& s = t.st[lo];
-  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0);
+  r.valid = lvl < s.n_lin && (MODE == 0 ? d.f_mb >= 0 : d.b_mb >= 0) && !(MODE == 1 && lo == 0 && lvl == 0 && s.pre != PRE_EMBED);
   const LinDev& L = s.lin[lvl < s.n_lin ? lvl : 0];
   if (MODE == 0) { r.M = t.T; r.N = L.n_out; r.K = L.n_in; }
+  else if (MODE == 1) { r.M = t.T; r.N = L.n_in; r.K = L.n_out; }
   else { r.M = L.n_out; r.N = L.n_in; r.K = t.T; }
   const int tiles_n = (r.N + P2_TILE - 1) / P2_TILE;
   const int local = tile - (t.sel_p >= 0 ? t.sel_tile0 : tile_start[lo]);
@@ -600,6 +623,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         const CUtensorMap* lm = maps + ((size_t)tl.p * PM_MAX_LINEARS + lvl) * MAPS_PER_LINEAR;
         const int dz_slot = (bwd_act(sd_.lin[lvl]) == PM_ACT_NONE && lvl == sd_.n_lin - 1 && !feeds_attention(sd_.post)) ? dz_mailbox_slot(t, sd_, d) : 0;
         if (MODE == 0) { tma_prefetch_desc(lm + MAP_ACT_K); tma_prefetch_desc(lm + MAP_W_K); }
+        else if (MODE == 1) { tma_prefetch_desc(lm + MAP_DZ_K); tma_prefetch_desc(lm + MAP_W_MN); }
         else { tma_prefetch_desc(lm + MAP_DZ_MN); tma_prefetch_desc(lm + MAP_ACT_MN); }
         const int ma = tl.m0 + rank * TILE_M, nbh = tl.n0 + rank * TILE_N;   // this CTA's rows of A and of B
         // ring slots of the operands: read here, once per tile (the k-block loop is the critical path of the kernel and
@@ -617,6 +641,10 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
           if (MODE == 0) {
             tma_load_3d_pair(sa, lm + MAP_ACT_K, fb, k0, ma, aslot);
             tma_load_3d_pair(sb, lm + MAP_W_K, fb, k0, nbh, vslot);
+          } else if (MODE == 1) {
+            tma_load_3d_pair(sa, lm + MAP_DZ_K, fb, k0, ma, dz_slot);
+            tma_load_3d_pair(sb, lm + MAP_W_MN, fb, nbh, k0, vslot);
+            tma_load_3d_pair(sb + B_BYTES / 2, lm + MAP_W_MN, fb, nbh + 64, k0, vslot);
           } else {
             tma_load_3d_pair(sa, lm + MAP_DZ_MN, fb, ma, k0, dz_slot);
             tma_load_3d_pair(sa + A_BYTES / 2, lm + MAP_DZ_MN, fb, ma + 64, k0, dz_slot);
@@ -1699,13 +1727,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct UmmaPlan {
   const CUtensorMap* d_maps = nullptr;
   const int* d_tile_start = nullptr;     // per (mode, level) at ts_off: [P+1] starts, then the stage of each tile
-  size_t ts_off[4][PM_MAX_LINEARS] = {};
+  size_t ts_off[5][PM_MAX_LINEARS] = {};
   const int* d_orders = nullptr;         // concatenated order arrays
   int* d_status = nullptr;
-  int n_slots[4][PM_MAX_LINEARS] = {};
-  int grid[4][PM_MAX_LINEARS] = {};
-  bool pair[4][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
-  size_t order_off[4][PM_MAX_LINEARS] = {};
+  int n_slots[5][PM_MAX_LINEARS] = {};
+  int grid[5][PM_MAX_LINEARS] = {};
+  bool pair[5][PM_MAX_LINEARS] = {};     // launch uses the CTA-pair kernel (256 x 256 tiles)
+  size_t order_off[5][PM_MAX_LINEARS] = {};
   int P = 0;
   // launches of one stage (microbatch-major order): the stage's tiles in ascending order are a slice of the identity list
   std::vector<int> h_tile_start;         // host copy of the tile starts
@@ -1719,12 +1747,12 @@ struct UmmaPlan {
 // projection next to d_model-sized layers) does not leave most SMs idle.  Unused slots hold -1.
 struct TileTables {
   std::vector<int> tile_start;           // per (mode, level): [P+1] starts, then the stage of each tile
-  size_t ts_off[4][PM_MAX_LINEARS] = {};
+  size_t ts_off[5][PM_MAX_LINEARS] = {};
   std::vector<int> orders;
-  int n_slots[4][PM_MAX_LINEARS] = {};
-  int grid[4][PM_MAX_LINEARS] = {};
-  bool pair[4][PM_MAX_LINEARS] = {};
-  size_t order_off[4][PM_MAX_LINEARS] = {};
+  int n_slots[5][PM_MAX_LINEARS] = {};
+  int grid[5][PM_MAX_LINEARS] = {};
+  bool pair[5][PM_MAX_LINEARS] = {};
+  size_t order_off[5][PM_MAX_LINEARS] = {};
   int max_tiles = 0;                     // most tiles of any (mode, level)
 };
 
@@ -1748,7 +1776,8 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
   const bool allow_pair = pair_kernels_allowed();
   TileTables tt;
   auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
-  for (int mode = 0; mode < 4; ++mode)                      // 3: dgrad once more, on 128-column pair tiles (launches of one narrow stage)
+  for (int mode = 0; mode < 5; ++mode)                      // 3: dgrad once more, on 128-column pair tiles (launches of one narrow stage);
+                                                            // 4: dgrad as a plain GEMM against a queued weight version (weight stashing)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       // block of this (mode, level): P + 1 tile starts, then the stage of every tile (one load instead of a search)
       tt.ts_off[mode][l] = tt.tile_start.size();
@@ -1763,7 +1792,7 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
           const LinDev& L = st[p].lin[l];
           ++n_lin_here;
           if ((mode == 2 ? L.n_out : T) < P2_TILE || (mode == 0 ? L.n_out : L.n_in) < P2_TILE) pair = false;
-          if ((mode == 1 || mode == 3) && p == 0 && l == 0 && st[p].pre != PRE_EMBED) --n_lin_here;   // the first Linear of the network has no input gradient
+          if ((mode == 1 || mode == 3 || mode == 4) && p == 0 && l == 0 && st[p].pre != PRE_EMBED) --n_lin_here;   // the first Linear of the network has no input gradient
         }
       pair = pair && n_lin_here > 0;
       tt.pair[mode][l] = pair;
@@ -1777,7 +1806,7 @@ static TileTables build_tile_tables(int T, const std::vector<StageDev>& st, int 
         ts[p] = acc;
         if (l < st[p].n_lin) {
           const LinDev& L = st[p].lin[l];
-          const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : (dg ? L.n_out : T);
+          const int M = mode == 2 ? L.n_out : T, N = mode == 0 ? L.n_out : L.n_in, K = mode == 0 ? L.n_in : ((dg || mode == 4) ? L.n_out : T);
           const int tm = cdiv(M, tile_m), tn = cdiv(N, tile_n), n_kb = cdiv(K, TILE_K);
           const int mg_rows = (pair && mode == 1) ? dgrad_pair_mg(T, L.n_in, dgrad_split_below) : mg_rows_fixed;
           const int groups = dg ? cdiv(tm, mg_rows) : tm;
@@ -1879,6 +1908,8 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
             wbase = (void*)(reinterpret_cast<__nv_bfloat16*>(t.ring + s.v_ring) + (L.w_off - s.begin));
           }
           okm = okm && encode(fn, m + MAP_W_K, 0, wbase, 3, dims3, strides3, box3, err);
+          uint32_t box3mn[3] = {64, TILE_K, 1};                         // the same copies as an MN-major operand (dgrad against a queued version)
+          okm = okm && encode(fn, m + MAP_W_MN, 0, wbase, 3, dims3, strides3, box3mn, err);
         }
         okm = okm && encode(fn, m + MAP_W_F32, 3, (void*)(t.a.w + L.w_off), 2, dims, strides4, box4, err);
         okm = okm && encode(fn, m + MAP_D_F32, 3, (void*)(t.a.delta + L.w_off), 2, dims, strides4, box4, err);
@@ -1933,7 +1964,7 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
     }
   }
   const TileTables tt = build_tile_tables(t.T, st, device_sms(), t.dgrad_split_below);
-  for (int mode = 0; mode < 4; ++mode)
+  for (int mode = 0; mode < 5; ++mode)
     for (int l = 0; l < PM_MAX_LINEARS; ++l) {
       plan->n_slots[mode][l] = tt.n_slots[mode][l];
       plan->grid[mode][l] = tt.grid[mode][l];
@@ -1957,6 +1988,8 @@ pm_status umma_plan_create(UmmaPlan** out, const TickArgs& t, const std::vector<
   e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<0>::kSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_pair_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute((const void*)umma_dgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DP_SMEM_BYTES);
@@ -2028,11 +2061,13 @@ cudaError_t umma_launch(UmmaPlan* plan, const TickArgs& t, int mode, int lvl, cu
     if (mode == 0) umma_pair_gemm_kernel<0><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else if (mode == 1) umma_dgrad_pair_kernel<<<grid, DP_THREADS, DP_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else if (mode == 3) umma_dgrad_pair128_kernel<<<grid, D1_THREADS, D1_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+    else if (mode == 4) umma_pair_gemm_kernel<1><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     else umma_pair_gemm_kernel<2><<<grid, P2_THREADS, P2_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
     return cudaGetLastError();
   }
   if (mode == 0) umma_gemm_kernel<0><<<grid, Cfg<0>::kThreads, Cfg<0>::kSmemBytes, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   else if (mode == 1) umma_dgrad_kernel<<<grid, DG_THREADS, DG_SMEM_BYTES, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
+  else if (mode == 4) umma_gemm_kernel<1><<<grid, Cfg<1>::kThreads, Cfg<1>::kSmemBytes, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   else umma_gemm_kernel<2><<<grid, Cfg<2>::kThreads, Cfg<2>::kSmemBytes, stream>>>(ta, plan->d_maps, ts, ord, n_slots, lvl, plan->d_status);
   return cudaGetLastError();
 }

@@ -670,7 +670,7 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
   const AT* x = ring_at<AT>(t, s.x_ring, d.b_xslot, n) + ro;
   const float* st = ring_at<float>(t, s.stat_ring, d.b_slot, (uint64_t)t.T * 2) + (uint64_t)row * 2;
   const float mu = st[0], rstd = st[1];
-  const float* g = t.a.w + s.g_off;
+  const float* g = t.stash ? fwd_small<AT>(t, s, d, s.g_off, s.g_soff) : t.a.w + s.g_off;   // stashing: the gain of the queued version
   const float* dl = t.a.delta + s.g_off;
   const float gapf = (float)s.gap;
   const bool corr = d.use_delta != 0;
@@ -853,7 +853,7 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
 #pragma unroll
     for (int k = 0; k < 8; ++k) { gb[q][k] = 0.f; ag[q][k] = 0.f; ab[q][k] = 0.f; }
     if (c < dm) {
-      load8<float>(t.a.w + s.g_off + c, gb[q]);
+      load8<float>((t.stash ? fwd_small<AT>(t, s, d, s.g_off, s.g_soff) : t.a.w + s.g_off) + c, gb[q]);   // stashing: the queued version's gain
       if (corr) { float cv[8]; load8<float>(t.a.delta + s.g_off + c, cv);
 #pragma unroll
         for (int k = 0; k < 8; ++k) gb[q][k] = __fsub_rn(gb[q][k], __fmul_rn(gapf, cv[k])); }     // gain - (tau_fwd - tau_bkwd) * delta

@@ -207,6 +207,18 @@ def test_microbatch_major_footprint_of_config5(built_lib):
     sd[3].tau_bkwd = 1
     st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
     assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED"
+    # ... unless it equals the forward delay in every stage (weight stashing): the same queues, nothing more to store
+    sd[3].tau_fwd, sd[3].tau_bkwd = wl.tau_fwd[3], 0
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    queues = rb.value
+    for p in range(P):
+        sd[p].tau_bkwd = sd[p].tau_fwd
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0 and rb.value == queues
+    sd[5].tau_bkwd = 0                                            # a mixture of the two patterns is not a mode
+    st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+    assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED"
+    for p in range(P):
+        sd[p].tau_bkwd = 0
     cfg.loop_order = 7
     assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
 

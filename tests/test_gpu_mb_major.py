@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 import pm_inputs as I
-from parity_util import run_gpu_pipeline, run_oracle, compare_params
+from parity_util import run_gpu_pipeline, run_oracle, compare_params, compare_params_adam, max_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -215,3 +215,71 @@ def test_n_microbatches_needs_the_weight_queue_order(cuda_device):
     wl = I.mlp_workload("t", 2, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
     with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
         pm.Pipeline(wl, I.init_stage_params(wl), n_micro=2)
+
+
+# ---- weight stashing: tau_bkwd = tau_fwd (Section 2.2), backward against the queued version the forward read -------------
+
+@pytest.mark.parametrize("compute,opt,per_stage", [("f32", "sgdm", 2), ("f32", "adam", 1), ("bf16", "sgdm", 2), ("bf16", "adam", 1)])
+def test_weight_stashing_mlp(cuda_device, compute, opt, per_stage):
+    f32 = compute == "f32"
+    P = 5
+    wl = I.mlp_workload("stash", P, 72 if f32 else 192, per_stage, "gelu", 33 if f32 else 40, compute=compute, optimizer=opt,
+                        alpha=0.02 if opt == "sgdm" else 1e-3, K=5, D=0.5, steps=2 * P + 6, seed=191005124 + 95)
+    wl.tau_bkwd = list(wl.tau_fwd)
+    params0 = I.init_stage_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    plain = list(wl.tau_bkwd)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    ref = {(t, i): (vf, vb) for (t, i, vf, vb) in res.book}
+    assert all(vf == vb for (vf, vb) in ref.values())                       # the oracle's backward reads the forward's version
+    for key, (vf, vb) in book.items():
+        assert vf == ref[key][0]                                            # (the device reports the live version as b_ver)
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    compare_params(pipe, res, (2e-5 if opt == "adam" else 1e-5) if f32 else 2e-2)
+    assert float(pipe.delta.abs().max()) == 0.0                             # no discrepancy, nothing for T2 to track
+    # and it is another trajectory than PipeMare's on the same delays
+    wl.tau_bkwd = [0] * P
+    other = run_oracle(wl, params0, wl.steps)
+    tol = (2e-5 if opt == "adam" else 1e-5) if f32 else 2e-2
+    moved = max(max_rel_err(a, b) for sa, sb in zip(res.params, other.params) for a, b in zip(sa, sb))
+    print("stashing vs PipeMare delays: largest relative weight difference", moved)
+    assert moved > (50 * tol if f32 else 2 * tol)
+
+
+@pytest.mark.parametrize("compute", ["f32", "bf16"])
+def test_weight_stashing_encoder_decoder(cuda_device, compute):
+    """LayerNorm gains are read from the queued version in the backward pass too."""
+    f32 = compute == "f32"
+    wl = I.cfg5_small(compute=compute, n_enc=1, n_dec=1, d_model=32 if f32 else 64, d_ff=64 if f32 else 128, seq_len=8 if f32 else 16,
+                      batch=2, vocab=40 if f32 else 96, steps=14)
+    wl.tau_bkwd = list(wl.tau_fwd)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=2e-5 if f32 else 1e-3)
+    compare_params(pipe, res, 2e-5 if f32 else 2e-2, per_stage=not f32)
+
+
+def test_weight_stashing_pair_tiles(cuda_device):
+    """The plain dgrad GEMM on CTA pairs (256-wide Linears, 256 rows): the queued bf16 version as the MN-major operand."""
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=256, n_heads=4, d_ff=512, seq_len=128, batch=2, vocab=264, steps=12)
+    wl.tau_bkwd = list(wl.tau_fwd)
+    params0 = I.init_encoder_params(wl)
+    res = run_oracle(wl, params0, wl.steps)
+    pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
+    np.testing.assert_allclose(losses, np.array(res.losses), rtol=1e-3)
+    print("weight stashing pair tiles", compare_params_adam(pipe, res, wl.steps))
+
+
+def test_weight_stashing_rules(cuda_device):
+    import paper_1910_05124_b200 as pm
+    wl = I.mlp_workload("t", 3, 64, 1, "relu", 8, compute="f32", steps=4, seed=9)
+    params0 = I.init_stage_params(wl)
+    wl.tau_bkwd = [wl.tau_fwd[0], 0, 0]                                      # mixed: some stages stash, others do not
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
+        pm.Pipeline(wl, params0, loop_order="mb_major")
+    wl.tau_bkwd = list(wl.tau_fwd)
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
+        pm.Pipeline(wl, params0)                                             # the tick schedule has one live version
+    with pytest.raises(pm.PipeMareError, match="PM_ERR_UNSUPPORTED"):
+        pm.Pipeline(wl, params0, loop_order="mb_major", recompute_segment=2)
