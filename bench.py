@@ -487,7 +487,11 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     mb_major = order == "mb_major"
     fused = FUSE.get(workload, 0) if getattr(args, "fuse", False) else 0
     segment = getattr(args, "recompute", 0) if mb_major else 0
-    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused, recompute_segment=segment)
+    if getattr(args, "stash", False) and mb_major:
+        wl.tau_bkwd = list(wl.tau_fwd)         # weight stashing: the backward pass reads the queued version (plain bf16 dgrad)
+    materialize = 1 if (getattr(args, "materialize", False) and mb_major) else 0
+    pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused, recompute_segment=segment,
+                       materialize_backward=materialize)
     del params0
     host_b, dev_b = make_batches(wl, 4, device)
     warm = max(args.warmup, 3)
@@ -538,7 +542,7 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     per_tick = {k: v[0] / args.steps for k, v in prof.items() if v[1] > 0}
     total_prof = sum(per_tick.values())
 
-    res = {"fused": fused, "segment": segment, "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
+    res = {"fused": fused, "segment": segment, "plain_dgrad": bool(materialize or (getattr(args, "stash", False) and mb_major)), "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
            "t_ms": t_med, "times": times, "units": units, "launches": launches, "clocks": clocks, "per_tick_ms": per_tick,
            "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "workspace_bytes": pipe.workspace_bytes,
            "prof": prof, "total_prof": total_prof}
@@ -609,7 +613,10 @@ def rooflines(res, peaks, steps):
                         "note": "46 MFLOP per step: launch-latency bound, not arithmetic bound"}
             continue
         launches = res["prof"][cls][1] / steps
-        out[cls] = {"kernel": GEMM_KERNELS[cls], "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
+        kname = GEMM_KERNELS[cls]
+        if cls == "dgrad" and res.get("plain_dgrad"):
+            kname = "umma_pair_gemm_kernel<1> / umma_gemm_kernel<1> (dgrad as a plain GEMM against a queued operand copy)"
+        out[cls] = {"kernel": kname, "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
                     "frac": round(tfs / tf_peak, 4), "of": f"{peaks['kind']} ({tf_kind} bf16 matmul; the median SM clock of the timed region decides)",
                     "frac_of_burst": round(tfs / peaks["tf_burst"], 4), "frac_of_sustained": round(tfs / peaks["tf_sustained"], 4),
                     "frac_of_nominal_2250TFs": round(tfs / 2250.0, 4),
@@ -678,6 +685,19 @@ def run_cuda(args):
                 except RuntimeError as exc:                  # e.g. not enough free device memory for config 5's queues
                     torch.cuda.empty_cache()
                     others.append((name, {"error": str(exc).splitlines()[0][:200]}))
+    # the same workload with the corrected backward weights written by the update instead of formed inside dgrad
+    # (pm_config.materialize_backward: same bits, one more operand copy): a measured variant, not the headline
+    variant = None
+    if world == 1 and not args.no_other and not args.stages and LOOP_ORDER[args.workload] == "mb_major" and not getattr(args, "materialize", False):
+        try:
+            a3 = argparse.Namespace(**vars(args))
+            a3.materialize = True
+            s3 = ClockSampler(local)
+            s3.start()
+            variant = measure(a3, args.workload, world, rank, local, device, s3, with_e2e=False, repeats=3)
+        except RuntimeError as exc:
+            torch.cuda.empty_cache()
+            variant = {"error": str(exc).splitlines()[0][:200]}
     if rank != 0:
         return
     wl, P = res["wl"], res["P"]
@@ -691,6 +711,8 @@ def run_cuda(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32" if wl.compute == "f32" else "bf16", "data": "synthetic",
         "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
                    "loop_order": res["order"], "recompute_segment": res["segment"], "fuse_update": res["fused"],
+                   "weight_stashing": bool(getattr(args, "stash", False)) and res["order"] == "mb_major",
+                   "materialize_backward": bool(getattr(args, "materialize", False)) and res["order"] == "mb_major",
                    "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
                    "samples_per_step": res["samples_per_step"], "pipeline_fill_ticks": res["fill"],
                    "cache": "per-step working set (state, activations, weight-version queues: see the byte counts) far exceeds the 126 MB L2: no flush needed",
@@ -720,6 +742,19 @@ def run_cuda(args):
             "ms_per_step": round(other["t_ms"] / steps, 5), "best_ms_per_step": round(min(other["times"]) / steps, 5),
             "clocks": other["clocks"], "roofline": orep["rooflines"][orep["dominant"]], "rooflines": orep["rooflines"],
             "gemm_all": orep["gemm_all"], "elementwise": orep["elementwise"], "kernel_ms_per_step": orep["kernel_ms_per_step"]})
+    if variant is not None:
+        if "error" in variant:
+            line["variants"] = [{"option": "materialize_backward", "error": variant["error"]}]
+        else:
+            vrep = workload_report(variant, peaks, steps)
+            line["variants"] = [{
+                "option": "materialize_backward",
+                "what": "the update writes bf16(w - tau delta) into one more slot of the version queue and dgrad reads it as a plain "
+                        "operand; every result has the same bits as the headline run, which forms the corrected weights inside dgrad",
+                "value": round(variant["units"] / (variant["t_ms"] * 1e-3), 2), "unit": UNIT,
+                "ms_per_step": round(variant["t_ms"] / steps, 5), "best_ms_per_step": round(min(variant["times"]) / steps, 5),
+                "ring_bytes": variant["ring_bytes"], "clocks": variant["clocks"], "rooflines": vrep["rooflines"],
+                "kernel_ms_per_step": vrep["kernel_ms_per_step"]}]
     if world == 1:
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(args.workload, 2 if args.workload in ("cfg3", "cfg1") else 1)
@@ -792,6 +827,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
     ap.add_argument("--recompute", type=int, default=0, metavar="S", help="PipeMare Recompute with segments of S stages "
                     "(microbatch-major workloads; default 0: none)")
+    ap.add_argument("--materialize", action="store_true", help="pm_config.materialize_backward: the update writes the corrected "
+                    "backward weights, dgrad reads them as a plain operand (microbatch-major workloads; same bits, one more copy)")
+    ap.add_argument("--stash", action="store_true", help="weight stashing (tau_bkwd = tau_fwd) instead of PipeMare's delays "
+                    "(microbatch-major workloads): shows what dgrad costs without the on-the-fly correction")
     ap.add_argument("--fuse", action="store_true", help="apply the update of the Linear matrices in the weight-gradient "
                     "GEMM's epilogue (pm_config.fuse_update) where the workload allows it; default: the update kernel")
     ap.add_argument("--update-only", type=int, default=0, metavar="N_PARAMS",

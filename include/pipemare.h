@@ -198,6 +198,15 @@ typedef struct {
                                     pm_stage_desc.tau_fwd is the delay T1 divides by (the mean of the stage's distribution),
                                     tau_bkwd must be 0 and T2 has nothing to correct.  Needs PM_MB_MAJOR, n_micro <= 1,
                                     recompute_segment = 0, fuse_update = 0, else PM_ERR_UNSUPPORTED.  0: off. */
+  int32_t materialize_backward;  /* 0 (default): the T2-corrected backward weights w - tau delta exist only inside the dgrad
+                                    kernel, formed while the operand is loaded; no second copy of the weights is kept.
+                                    1: the update that produces version v also writes bf16(w_v - tau delta_v) (fp32 with
+                                    PM_F32) into one more slot of the stage's version queue, and the backward pass of the next
+                                    step reads that copy: dgrad becomes a plain GEMM.  The same bits in every result (the
+                                    correction is the same fp32 subtraction and product, rounded once), + one operand-type copy
+                                    of the parameters in memory and 2 B per parameter of update traffic, less dgrad time.
+                                    Needs PM_MB_MAJOR, recompute_segment = 0, stochastic_tau_max = 0, fuse_update = 0 and
+                                    tau_bkwd = 0, else PM_ERR_UNSUPPORTED. */
 } pm_config;
 
 /* Flat state arenas, device, `count` elements each.  w: master weights; m: momentum /

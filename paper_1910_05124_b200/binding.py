@@ -43,7 +43,7 @@ class pm_config(C.Structure):
                 ("alpha_const", C.c_double), ("alpha_by_step", C.POINTER(C.c_double)), ("alpha_len", C.c_int64),
                 ("loss_log_capacity", C.c_int64), ("loop_order", C.c_int32), ("entry_period", C.c_int32), ("n_micro", C.c_int32),
                 ("recompute_segment", C.c_int32), ("fuse_update", C.c_int32),
-                ("stochastic_tau_max", C.c_int32)]
+                ("stochastic_tau_max", C.c_int32), ("materialize_backward", C.c_int32)]
 
 
 class pm_arenas(C.Structure):
@@ -114,7 +114,7 @@ def _check(status, ctx=None):
 
 def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, beta2=0.98, eps=1e-8,
                 t1=True, K=1, t2=True, D=0.5, alpha_by_step=None, loss_log_capacity=0, loss=PM_LOSS_MSE,
-                loop_order=PM_TICK_MAJOR, n_micro=1, entry_period=0, recompute_segment=0, fuse_update=0, stochastic_tau_max=0):
+                loop_order=PM_TICK_MAJOR, n_micro=1, entry_period=0, recompute_segment=0, fuse_update=0, stochastic_tau_max=0, materialize_backward=0):
     cfg = pm_config()
     cfg.n_stages, cfg.microbatch = n_stages, microbatch
     cfg.compute_dtype = PM_BF16 if compute in ("bf16", PM_BF16) and compute != 0 else PM_F32
@@ -135,6 +135,7 @@ def make_config(*, n_stages, microbatch, compute, optimizer, alpha, beta1=0.9, b
     cfg.recompute_segment = int(recompute_segment)
     cfg.fuse_update = int(bool(fuse_update))
     cfg.stochastic_tau_max = int(stochastic_tau_max)
+    cfg.materialize_backward = int(bool(materialize_backward))
     cfg.entry_period = int(entry_period)
     return cfg, keep
 
@@ -216,7 +217,7 @@ class Pipeline:
     """
 
     def __init__(self, wl, params0, device="cuda:0", stream=None, loss_log_capacity=0, loop_order=PM_TICK_MAJOR, n_micro=1, entry_period=0,
-                 recompute_segment=0, fuse_update=0, stochastic_tau_max=0):
+                 recompute_segment=0, fuse_update=0, stochastic_tau_max=0, materialize_backward=0):
         import torch
         self.torch = torch
         self.wl = wl
@@ -247,7 +248,8 @@ class Pipeline:
             beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, t1=wl.t1, K=wl.K, t2=wl.t2, D=wl.D,
             loss_log_capacity=loss_log_capacity, loss=PM_LOSS_CE if self.is_encoder else PM_LOSS_MSE,
             loop_order=loop_order, n_micro=n_micro, entry_period=entry_period, recompute_segment=recompute_segment,
-            fuse_update=fuse_update, stochastic_tau_max=stochastic_tau_max)
+            fuse_update=fuse_update, stochastic_tau_max=stochastic_tau_max,
+            materialize_backward=materialize_backward)
         self.mb_major = self.cfg.loop_order == PM_MB_MAJOR
         sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
         _check(self.L.pm_query_bytes(C.byref(self.cfg), self.stage_desc, C.byref(sb), C.byref(rb), C.byref(wb)))

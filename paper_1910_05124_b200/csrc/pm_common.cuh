@@ -129,6 +129,8 @@ struct HyperDev {
   int32_t segment;            // PipeMare Recompute: stages per segment (0: no recomputation)
   int32_t stochastic;         // stage-wise stochastic delays (Appendix E): slots of the gradient ring, tau_max + 1 (0: off)
   uint64_t total;             // elements of the arenas (one slot of the gradient ring)
+  int32_t materialize;        // backward entries point at the slot that holds the materialised corrected weights (or the live version)
+  int32_t _pad3;
 };
 
 // The microbatch that enters the first stage at tick a, or -1: during the warm-up one microbatch every `period` ticks

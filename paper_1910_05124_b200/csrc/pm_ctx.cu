@@ -30,6 +30,7 @@ struct Layout {
   uint64_t off_skb = 0, off_ske = 0;
   int32_t fuse = 0;                     // the weight-gradient GEMM applies the update of the Linear matrices in its epilogue
   int32_t stash = 0;                    // weight stashing: every stage has tau_bkwd = tau_fwd (microbatch-major order)
+  int32_t materialize = 0;              // the corrected backward weights are written by the update into a slot of the version queue
   int32_t stochastic = 0;               // stage-wise stochastic delays (Appendix E): slots of the gradient ring (tau_max + 1), 0: off
   uint64_t g_ring = 0, off_delays = 0;  // ring: [stochastic][total] float gradients of the last microbatches; ws: the step's delays [P]
   uint64_t ring_bytes = 0, ws_bytes = 0, total = 0;
@@ -112,6 +113,12 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
     if (why) { err = std::string("stochastic_tau_max > 0 is built for ") + why; return PM_ERR_UNSUPPORTED; }
   }
   L.stochastic = stoch ? cfg->stochastic_tau_max + 1 : 0;
+  const bool mat = cfg->materialize_backward != 0;
+  if (mat && (!mb || S > 0 || stoch || cfg->fuse_update)) {
+    err = "materialize_backward is built for PM_MB_MAJOR order without recompute_segment, stochastic_tau_max or fuse_update";
+    return PM_ERR_UNSUPPORTED;
+  }
+  L.materialize = mat ? 1 : 0;
   if (cfg->entry_period < 0 || cfg->entry_period > 2 * P) { err = "entry_period must be in [0, 2 * n_stages]"; return PM_ERR_INVALID_ARG; }
   const int E = (!mb && cfg->entry_period > 1) ? cfg->entry_period : 1;
   const bool queue = mb || E > 1;
@@ -170,6 +177,9 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
       if (seg_end < P) s.tau_r = std::min(s.tau_f, (2 * (seg_end - 1 - p) + 1 + nm - 1) / nm);
       if (cfg->t2_enable && s.tau_r < s.tau_f) s.rdepth = s.tau_r + 1;
     }
+    // materialize_backward: the same mechanism with delay 0: one slot holding w_v - (tau_fwd - 0) delta_v of the live version,
+    // which is exactly the T2-corrected operand of the next backward pass
+    if (mat && cfg->t2_enable && s.gap > 0) { s.tau_r = 0; s.rdepth = 1; }
     if (E > 1) {
       // a microbatch every E ticks: a stash written at tick mE + i is read at tick mE + i + tau, so floor(tau / E) + 1
       // microbatches are alive in a stage; the input ring keeps one more (it is also the forward mailbox) and another
@@ -355,8 +365,8 @@ pm_status build_layout(const pm_config* cfg, const pm_stage_desc* stages, Layout
   // Weight stashing (Section 2.2, tau_bkwd = tau_fwd): the backward pass of a microbatch reads the queued version its forward
   // read, in the operand type (the copy the forward used), so dgrad is a plain GEMM and T2 has nothing to correct.
   L.stash = any_stash ? 1 : 0;
-  if (L.stash && (S > 0 || stoch || cfg->fuse_update)) {
-    err = "weight stashing (tau_bkwd = tau_fwd) is not combined with recompute_segment, stochastic_tau_max or fuse_update";
+  if (L.stash && (S > 0 || stoch || cfg->fuse_update || mat)) {
+    err = "weight stashing (tau_bkwd = tau_fwd) is not combined with recompute_segment, stochastic_tau_max, fuse_update or materialize_backward";
     return PM_ERR_UNSUPPORTED;
   }
   // Fused update (pm_config.fuse_update): the weight-gradient GEMM's epilogue updates the Linear matrices, the update
@@ -669,6 +679,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   c->hp.n_micro = cfg->n_micro > 1 ? cfg->n_micro : 1;
   c->hp.segment = L.segment;
   c->hp.stochastic = L.stochastic; c->hp.total = L.total;
+  c->hp.materialize = L.materialize;
 
   TickArgs& t = c->ta;
   t.st = (const StageDev*)(c->ws + L.off_st);
@@ -682,7 +693,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0;
   t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
-  t.stash = L.stash;
+  t.stash = (L.stash || L.materialize) ? 1 : 0;     // the backward pass reads its table entry's version slot
   t.fuse_upd = 0; t.upd_opt = cfg->optimizer; t.upd_beta1 = cfg->beta1; t.upd_beta2 = cfg->beta2; t.upd_eps = cfg->eps;
   t.upd_lp = L.queue ? reinterpret_cast<__nv_bfloat16*>(t.ring) : c->a.w_lp;
   for (int l = 0; l < PM_MAX_LINEARS; ++l) t.act_first[l] = 0;
@@ -914,7 +925,7 @@ static pm_status stage_backward(pm_ctx* ctx, const TickArgs& ta, int p, bool gro
     }
     if (p == 0 && l == 0 && sd.pre != PRE_EMBED) continue;          // raw network inputs need no gradient
     prof_begin(ctx, PM_PROF_DGRAD);
-    e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, ctx->L.stash ? 4 : 1, l, ctx->ls);
+    e = dt == PM_F32 ? launch_simt_gemm(ta, dt, 1, l, ctx->ls) : umma_launch(ctx->umma, ta, (ctx->L.stash || ctx->L.materialize) ? 4 : 1, l, ctx->ls);
     if ((s = check(ctx, e, "dgrad GEMM")) != PM_OK) return s;
   }
   const int n_pre = sd.pre != PRE_NONE ? pre_bwd_launches(ta) : 0;

@@ -173,6 +173,11 @@ __global__ void schedule_mb_kernel(const StageSched* __restrict__ sched, StageDy
     d = make_dyn(s, hp, base + 2 * P - 1 - i, -1, mine ? t : -1, -1, u, fver, true, u);
   }
   d.r_ver = rver;
+  if (hp.materialize && (v >= 2 * P || v == 2 * P - 1 - i)) {
+    // a backward entry: its version slot is the one the update filled with w - tau delta of the live version (stages that
+    // keep none -- no gap, or T2 off -- read the live version itself)
+    d.f_vslot = s.rdepth > 0 ? s.vdepth : (s.vdepth > 1 ? (int32_t)(u % s.vdepth) : 0);
+  }
   d.accum = (t % N != 0) ? 1 : 0;
   tables[(size_t)v * P + i] = d;
 }

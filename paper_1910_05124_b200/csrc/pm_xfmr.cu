@@ -673,7 +673,7 @@ __global__ void __launch_bounds__(256) ln_bwd_dx_kernel(TickArgs t) {
   const float* g = t.stash ? fwd_small<AT>(t, s, d, s.g_off, s.g_soff) : t.a.w + s.g_off;   // stashing: the gain of the queued version
   const float* dl = t.a.delta + s.g_off;
   const float gapf = (float)s.gap;
-  const bool corr = d.use_delta != 0;
+  const bool corr = d.use_delta != 0 && !t.stash;          // a version read from the queue is used as it is
   AT* out = gin_write_prev<AT>(t, p, d) + ro;
   float s1 = 0.f, s2 = 0.f;
   if ((dm & 7) == 0 && dm <= 2048) {                         // 8 columns per lane per pass, values kept in registers
@@ -842,7 +842,7 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   AT* out = s.from_memory ? gmem_at<AT>(t, d) : (p > 0 ? gin_write_prev<AT>(t, p, d) : nullptr);
   const bool accumulate = s.from_memory && !s.mem_first;
   const float gapf = (float)s.gap;
-  const bool corr = d.use_delta != 0;
+  const bool corr = d.use_delta != 0 && !t.stash;          // a version read from the queue is used as it is
   const int half = WPR == 2 ? (warp & 1) : 0, rw = WPR == 2 ? (warp >> 1) : warp;
   const int cbase = half * NP * 256;                         // first column of this warp's share of a row
   __shared__ float xs[2][4][2][2];                           // [row parity][warp pair][half][s1, s2]

@@ -5,7 +5,7 @@ import pm_inputs as I
 
 
 def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warmup=0, loop_order="tick_major", n_micro=1, entry_period=1,
-                     segment=0, book_recomp=None, fuse_update=0, delays=None, tau_max=0, book_applied=None):
+                     segment=0, book_recomp=None, fuse_update=0, delays=None, tau_max=0, book_applied=None, materialize=0):
     """Feed n_steps microbatches through the CUDA pipeline, drain it, return (pipeline, losses, book).
 
     book maps (microbatch, stage 1-based) -> [forward version, backward version] as recorded by the device.
@@ -19,7 +19,7 @@ def run_gpu_pipeline(wl, params0, n_steps, teacher=None, collect_book=True, warm
     import torch
     import paper_1910_05124_b200 as pm
     pipe = pm.Pipeline(wl, params0, loop_order=loop_order, n_micro=n_micro, entry_period=entry_period, recompute_segment=segment,
-                       fuse_update=fuse_update, stochastic_tau_max=tau_max)
+                       fuse_update=fuse_update, stochastic_tau_max=tau_max, materialize_backward=materialize)
     P = wl.n_stages
     encoder = wl.kind == "encoder"
     if not encoder:
