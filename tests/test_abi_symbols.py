@@ -294,6 +294,31 @@ def test_stochastic_delay_model_footprint_and_checks_without_a_gpu(built_lib):
     assert L.pm_status_string(L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))) == b"PM_ERR_INVALID_ARG"
 
 
+def test_materialize_backward_footprint_and_checks_without_a_gpu(built_lib):
+    """The option keeps one more operand-type copy of every stage that has a delay gap (config 5: all of them) and is
+    refused outside microbatch-major order or together with the options it does not combine with."""
+    import ctypes as C
+    import pm_inputs as I
+    from paper_1910_05124_b200 import binding as B
+    L = B.lib()
+    wl = I.cfg5()
+    cfg, sd, keep = _describe(wl)
+    cfg.loop_order = B.PM_MB_MAJOR
+    sb, rb, wb = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    plain = rb.value
+    cfg.materialize_backward = 1
+    assert L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb)) == 0
+    copy = sum(sd[p].param_count * 2 for p in range(wl.n_stages))
+    assert copy <= rb.value - plain < copy * 1.01
+    for field, value in (("loop_order", B.PM_TICK_MAJOR), ("recompute_segment", 12), ("stochastic_tau_max", 3), ("fuse_update", 1)):
+        old = getattr(cfg, field)
+        setattr(cfg, field, value)
+        st = L.pm_query_bytes(C.byref(cfg), sd, C.byref(sb), C.byref(rb), C.byref(wb))
+        assert L.pm_status_string(st) == b"PM_ERR_UNSUPPORTED", field
+        setattr(cfg, field, old)
+
+
 def test_flat_update_argument_checks_need_no_gpu(built_lib):
     """pm_update_flat / pm_update_flat_static reject an empty step-size table and slices that do not fit the arenas
     (a sum offset + count that wraps included) before anything touches the device."""
