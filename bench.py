@@ -483,15 +483,19 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     a2.workload = workload
     wl, params0, samples_per_step, n_params = build_workload(a2)
     P = wl.n_stages
-    order = LOOP_ORDER[workload]
+    order = getattr(args, "order", None) or LOOP_ORDER[workload]
     mb_major = order == "mb_major"
+    n_micro = getattr(args, "n_micro", 1) if mb_major else 1
+    if n_micro > 1:                            # Table 1: delays count updates, tau = ceil((2(P-i)+1)/N)
+        import pm_inputs as I
+        wl.tau_fwd = I.pipemare_delays(P, n_micro)[0]
     fused = FUSE.get(workload, 0) if getattr(args, "fuse", False) else 0
     segment = getattr(args, "recompute", 0) if mb_major else 0
     if getattr(args, "stash", False) and mb_major:
         wl.tau_bkwd = list(wl.tau_fwd)         # weight stashing: the backward pass reads the queued version (plain bf16 dgrad)
     materialize = 1 if (getattr(args, "materialize", False) and mb_major) else 0
     pipe = pm.Pipeline(wl, params0, device=str(device), loop_order=order, fuse_update=fused, recompute_segment=segment,
-                       materialize_backward=materialize)
+                       materialize_backward=materialize, n_micro=n_micro)
     del params0
     host_b, dev_b = make_batches(wl, 4, device)
     warm = max(args.warmup, 3)
@@ -542,7 +546,7 @@ def measure(args, workload, world, rank, local, device, sampler=None, with_e2e=T
     per_tick = {k: v[0] / args.steps for k, v in prof.items() if v[1] > 0}
     total_prof = sum(per_tick.values())
 
-    res = {"fused": fused, "segment": segment, "plain_dgrad": bool(materialize or (getattr(args, "stash", False) and mb_major)), "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
+    res = {"n_micro": n_micro, "fused": fused, "segment": segment, "plain_dgrad": bool(materialize or (getattr(args, "stash", False) and mb_major)), "wl": wl, "P": P, "fill": fill, "samples_per_step": samples_per_step, "n_params": n_params, "order": order,
            "t_ms": t_med, "times": times, "units": units, "launches": launches, "clocks": clocks, "per_tick_ms": per_tick,
            "ring_bytes": pipe.ring_bytes, "state_bytes": pipe.state_bytes, "workspace_bytes": pipe.workspace_bytes,
            "prof": prof, "total_prof": total_prof}
@@ -710,7 +714,7 @@ def run_cuda(args):
         "warmup": max(args.warmup, 3), "ms_per_step": round(res["t_ms"] / steps, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32" if wl.compute == "f32" else "bf16", "data": "synthetic",
         "config": {"workload": WORKLOADS[args.workload] + (f" [cut to {args.stages} for profiling]" if args.stages else ""),
-                   "loop_order": res["order"], "recompute_segment": res["segment"], "fuse_update": res["fused"],
+                   "loop_order": res["order"], "n_micro": res["n_micro"], "recompute_segment": res["segment"], "fuse_update": res["fused"],
                    "weight_stashing": bool(getattr(args, "stash", False)) and res["order"] == "mb_major",
                    "materialize_backward": bool(getattr(args, "materialize", False)) and res["order"] == "mb_major",
                    "parallelism": "replicas only" if world > 1 else f"single GPU, {P} emulated pipeline stages",
@@ -827,6 +831,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (profiling runs)")
     ap.add_argument("--recompute", type=int, default=0, metavar="S", help="PipeMare Recompute with segments of S stages "
                     "(microbatch-major workloads; default 0: none)")
+    ap.add_argument("--order", choices=["tick_major", "mb_major"], default=None, help="loop order (default: the workload's own)")
+    ap.add_argument("--n-micro", type=int, default=1, dest="n_micro", metavar="N", help="microbatches per update (microbatch-major "
+                    "order): a step stays one microbatch, the update runs every N-th step with Table 1's delays for N")
     ap.add_argument("--materialize", action="store_true", help="pm_config.materialize_backward: the update writes the corrected "
                     "backward weights, dgrad reads them as a plain operand (microbatch-major workloads; same bits, one more copy)")
     ap.add_argument("--stash", action="store_true", help="weight stashing (tau_bkwd = tau_fwd) instead of PipeMare's delays "
