@@ -6,7 +6,9 @@
 // backward weights): the embedding table and the LayerNorm gain/bias are read in the forward pass; the
 // backward pass reads only the LayerNorm gain, in dx_hat = dy * gain, and takes it T2-corrected
 // (gain - gap * delta).  Parameter gradients use stashed forward quantities only.
+#include <algorithm>
 #include "pm_tick.cuh"
+#include "pm_ptx.cuh"
 
 namespace pm {
 
@@ -846,6 +848,26 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
   const int half = WPR == 2 ? (warp & 1) : 0, rw = WPR == 2 ? (warp >> 1) : warp;
   const int cbase = half * NP * 256;                         // first column of this warp's share of a row
   __shared__ float xs[2][4][2][2];                           // [row parity][warp pair][half][s1, s2]
+  extern __shared__ float lnred[];                           // [8 warps][2][NP*256] at the end; before that the staged rows
+  // Staging (launches of one stage, which have one block or two per SM and few rows in flight otherwise): every row of
+  // the block's x, du and skip gradient is requested at once with 16-byte asynchronous copies; the row loop then
+  // reads shared memory, so a block pays one round trip to memory instead of one per row.
+  const bool stage = t.ln_stage != 0;
+  AT* stg = reinterpret_cast<AT*>(lnred);
+  const uint64_t rstride = (uint64_t)t.ln_chunk_rows * dm;   // elements of one staged array
+  if (stage) {
+    const int per_row = dm * (int)sizeof(AT) / 16, total = (r1 - r0) * per_row;
+    const bool with_gs = gs != nullptr;
+    for (int i = threadIdx.x; i < total; i += 256) {
+      const int rr = i / per_row, cc = i - rr * per_row;
+      const uint64_t go = ((uint64_t)(r0 + rr) * dm) * sizeof(AT) + (uint64_t)cc * 16, so = ((uint64_t)rr * dm) * sizeof(AT) + (uint64_t)cc * 16;
+      cp_async16(reinterpret_cast<char*>(stg) + so, reinterpret_cast<const char*>(x) + go);
+      cp_async16(reinterpret_cast<char*>(stg + rstride) + so, reinterpret_cast<const char*>(du) + go);
+      if (with_gs) cp_async16(reinterpret_cast<char*>(stg + 2 * rstride) + so, reinterpret_cast<const char*>(gs) + go);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+  }
   float gb[NP][8], ag[NP][8], ab[NP][8];
 #pragma unroll
   for (int q = 0; q < NP; ++q) {
@@ -869,12 +891,16 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
     float s1 = 0.f, s2 = 0.f;
     // every load of the row is issued before the first use
     float xa[NP][8], da[NP][8], sa[NP][8];
+    const uint64_t so = (uint64_t)(r - r0) * dm;
+    const AT* xr = stage ? stg + so : x + ro;
+    const AT* dr = stage ? stg + rstride + so : du + ro;
+    const AT* sr = stage ? (has_gs ? stg + 2 * rstride + so : dr) : gs + ro;
 #pragma unroll
     for (int q = 0; q < NP; ++q) {
       const int c = min(cbase + q * 256 + lane * 8, dm - 8);
-      load8<AT>(x + ro + c, xa[q]);
-      load8<AT>(du + ro + c, da[q]);
-      load8<AT>(gs + ro + c, sa[q]);
+      load8<AT>(xr + c, xa[q]);
+      load8<AT>(dr + c, da[q]);
+      load8<AT>(sr + c, sa[q]);
     }
 #pragma unroll
     for (int q = 0; q < NP; ++q) {
@@ -934,7 +960,7 @@ __global__ void __launch_bounds__(256, NP <= 2 ? 2 : 1) ln_bwd_fused_kernel(Tick
       }
     }
   }
-  extern __shared__ float lnred[];                           // [8 warps][2][NP*256]
+  if (stage) __syncthreads();                                // the staged rows are not read any more: the buffer takes the partial sums
 #pragma unroll
   for (int q = 0; q < NP; ++q)
 #pragma unroll
@@ -996,14 +1022,19 @@ __global__ void __launch_bounds__(256) ln_fused_finish_kernel(TickArgs t) {
 
 template <typename AT, int NP, int WPR>
 static cudaError_t launch_ln_fused(const TickArgs& t, cudaStream_t stream) {
-  const size_t smem = (size_t)8 * 2 * NP * 256 * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set && smem > 48 * 1024) {
+  size_t smem = (size_t)8 * 2 * NP * 256 * sizeof(float);
+  // launches of one stage stage their rows in shared memory when two such blocks fit on an SM
+  const size_t stage_bytes = (size_t)3 * t.ln_chunk_rows * t.max_ln_dim * sizeof(AT);
+  TickArgs ta = t;
+  ta.ln_stage = (t.sel_p >= 0 && stage_bytes <= 100 * 1024 && (t.max_ln_dim * sizeof(AT)) % 16 == 0) ? 1 : 0;
+  if (ta.ln_stage) smem = std::max(smem, stage_bytes);
+  static size_t attr_bytes = 48 * 1024;
+  if (smem > attr_bytes) {
     cudaError_t e = cudaFuncSetAttribute((const void*)ln_bwd_fused_kernel<AT, NP, WPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_bytes = smem;
   }
-  ln_bwd_fused_kernel<AT, NP, WPR><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(t);
+  ln_bwd_fused_kernel<AT, NP, WPR><<<dim3(t.ln_chunks, t.n_ln), 256, smem, stream>>>(ta);
   if (!t.defer_finish) ln_fused_finish_kernel<<<dim3((t.max_ln_dim + kLnFinCols - 1) / kLnFinCols, t.n_ln), 256, 0, stream>>>(t);
   return cudaGetLastError();
 }
