@@ -127,6 +127,7 @@ template <> struct Pair<__nv_bfloat16> {
 };
 
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
+constexpr int kColsumGroup = 8;                       // row chunks per block in a launch that only sums columns
 
 // rows r, r + NW, ... < r1 of 8 columns (NW = warps of the block): four rows are loaded before the first is used
 template <typename AT, int ACT, int NW>
@@ -183,8 +184,11 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   const LinDev& L = s.lin[lvl];
   const int c0 = (blk - start[p]) * kActColsV;
   if (c0 >= L.n_out) return;
-  const int chunk = blockIdx.y;
-  const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + t.chunk_rows);
+  // a launch that only sums columns gives a block kColsumGroup row chunks (fewer, longer-lived blocks); their sum goes
+  // to the first chunk's partial row and zeros to the others, which the finishing pass adds like any partial
+  const int cg = (t.colsum_only && t.row_chunks > 1) ? kColsumGroup : 1;
+  const int chunk = blockIdx.y * cg;
+  const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + cg * t.chunk_rows);
   if (r0 >= t.T) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = c0 + 8 * lane;
@@ -228,7 +232,11 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
 #pragma unroll
     for (int w = 0; w < NW; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
     if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = d.accum ? __fadd_rn(t.a.grad[L.b_off + cc], a) : a;
-    else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc] = a;
+    else {
+      float* part = ws_ptr<float>(t, t.colred_off) + ((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc;
+      part[0] = a;
+      for (int j = 1; j < cg && chunk + j < t.row_chunks; ++j) part[(uint64_t)j * (2 * (uint64_t)t.max_dim)] = 0.f;
+    }
   }
 }
 
@@ -293,7 +301,7 @@ cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t st
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
   if (t.act_blocks[lvl] == 0) return cudaSuccess;
-  dim3 grid(t.act_blocks[lvl], t.row_chunks);
+  dim3 grid(t.act_blocks[lvl], (t.colsum_only && t.row_chunks > 1) ? (t.row_chunks + kColsumGroup - 1) / kColsumGroup : t.row_chunks);
   if (t.sel_p >= 0 && t.row_chunks > 1) {
     if (dtype == PM_F32) actbwd_kernel<float, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
     else actbwd_kernel<__nv_bfloat16, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
