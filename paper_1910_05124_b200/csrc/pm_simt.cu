@@ -128,6 +128,7 @@ template <> struct Pair<__nv_bfloat16> {
 
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 constexpr int kColsumGroup = 8;                       // row chunks per block in a launch that only sums columns
+constexpr int kStageGroup = 4;                        // ... and in a launch of one stage
 
 // rows r, r + NW, ... < r1 of 8 columns (NW = warps of the block): four rows are loaded before the first is used
 template <typename AT, int ACT, int NW>
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   if (c0 >= L.n_out) return;
   // a launch that only sums columns gives a block kColsumGroup row chunks (fewer, longer-lived blocks); their sum goes
   // to the first chunk's partial row and zeros to the others, which the finishing pass adds like any partial
-  const int cg = (t.colsum_only && t.row_chunks > 1) ? kColsumGroup : 1;
+  const int cg = t.row_chunks > 1 ? (t.colsum_only ? kColsumGroup : (t.sel_p >= 0 ? kStageGroup : 1)) : 1;
   const int chunk = blockIdx.y * cg;
   const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + cg * t.chunk_rows);
   if (r0 >= t.T) return;
@@ -301,7 +302,8 @@ cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t st
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
   if (t.act_blocks[lvl] == 0) return cudaSuccess;
-  dim3 grid(t.act_blocks[lvl], (t.colsum_only && t.row_chunks > 1) ? (t.row_chunks + kColsumGroup - 1) / kColsumGroup : t.row_chunks);
+  const int cg = t.row_chunks > 1 ? (t.colsum_only ? kColsumGroup : (t.sel_p >= 0 ? kStageGroup : 1)) : 1;
+  dim3 grid(t.act_blocks[lvl], (t.row_chunks + cg - 1) / cg);
   if (t.sel_p >= 0 && t.row_chunks > 1) {
     if (dtype == PM_F32) actbwd_kernel<float, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
     else actbwd_kernel<__nv_bfloat16, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);
