@@ -160,7 +160,7 @@ template <int MODE>
 __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* lm, const StageDev& s, const StageDyn& d, const LinDev& L,
                                           int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
                                           uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es,
-                                          const uint4 (&skq)[8]) {
+                                          uint4 (&skq)[8], const __nv_bfloat16* next_skip = nullptr, int next_cols = 0) {
   if (MODE == 2 && t.fuse_upd) {                                  // the update is applied here; nothing is stored to the grad arena
     if (t.upd_opt == PM_SGDM) epi_update_block<PM_SGDM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
     else epi_update_block<PM_ADAM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
@@ -203,6 +203,9 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
         if (!both) {                                                // one output: no activation (z = y = bf16(acc + b)), or a ReLU whose z is not kept
           if (resid) {
             const uint32_t w[4] = {skq[g].x, skq[g].y, skq[g].z, skq[g].w};
+            // the registers just read take the NEXT block's skip values (same row, 64 columns on): their latency hides
+            // behind the rest of this block instead of standing in front of the next one
+            if (next_skip) skq[g] = 8 * g < next_cols ? __ldg(reinterpret_cast<const uint4*>(next_skip + 8 * g)) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const float2 sk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
@@ -730,7 +733,6 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
         const int nb = tl.n0 + half * 128 + c * 64;
-        if (MODE == 0 && c == 1) load_skip64(t, s, d, tl.N, mrow + lane, nb, skq);   // the first block's were issued before the wait
         uint32_t r0[32], r1[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc.idx * P2_ACC_COLS + half * 128 + c * 64);
         tmem_ld32(taddr, r0);
@@ -741,7 +743,11 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         if (c == 1 && lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty + 8 * acc.idx, 0));   // this warp has read its part of the accumulator
         __syncwarp();
         if (mrow >= tl.M || nb >= tl.N) continue;                     // nothing of this block is inside the tensor
-        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es, skq);
+        // a residual stage: block 0 refills the skip registers with block 1's values as it consumes them
+        const __nv_bfloat16* nxt = nullptr;
+        if (MODE == 0 && c == 0 && s.post == POST_RESIDUAL && mrow + lane < t.T && nb + 64 < tl.N)
+          nxt = ws_at<__nv_bfloat16>(t, s.skip_in) + (uint64_t)d.skip_rslot * ((uint64_t)t.T * tl.N) + (uint64_t)(mrow + lane) * tl.N + nb + 64;
+        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es, skq, nxt, tl.N - (nb + 64));
       }
       acc.advance(2);
     }
