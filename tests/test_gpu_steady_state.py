@@ -63,11 +63,12 @@ def test_cfg5_widths_steady_state_both_orders(cuda_device):
 
 def test_cfg5_widths_recompute_steady_state(cuda_device):
     """PipeMare Recompute at config 5's widths on 2 + 2 layers (23 stages), segments of 5 stages (boundaries inside
-    layers: skip tensors, the memory and the main stream cross them), 2 sequences per microbatch, 2P + 4 microbatches:
+    layers: skip tensors, the memory and the main stream cross them), 2 sequences per microbatch, 32 microbatches (every
+    recompute delay, at most 9 here, is past its clamp after ten; the forward delays' steady state is the test above):
     the pair-tile kernels, the 256-token attention, one weight-gradient launch per segment, T2-corrected recompute
     weights read from the queue."""
     wl = I.cfg5_cut(2, 2, batch=2)
-    wl.steps = 2 * wl.n_stages + 4
+    wl.steps = 32
     params0 = I.init_encoder_params(wl)
     res = run_oracle(wl, params0, wl.steps, segment=5)
     book_r = {}
