@@ -690,7 +690,7 @@ pm_status pm_init_stages(pm_ctx** out, const pm_config* cfg, const pm_stage_desc
   t.max_lin = L.max_lin; t.max_dim = L.max_dim;
   t.mb_major = L.queue ? 1 : 0; t.sel_p = -1; t.sel_tile0 = 0;
   t.res_fused = cfg->compute_dtype == PM_BF16 ? 1 : 0;
-  t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0; t.ln_stage = 0;
+  t.ln_li0 = 0; t.defer_finish = 0; t.colsum_only = 0; t.ln_stage = 0; t.fin_deferred = 0;
   t.dgrad_split_below = 0;
   t.loss_scale = 1.0f / (float)(cfg->n_micro > 1 ? cfg->n_micro : 1);
   t.stash = (L.stash || L.materialize) ? 1 : 0;     // the backward pass reads its table entry's version slot

@@ -129,6 +129,10 @@ template <> struct Pair<__nv_bfloat16> {
 constexpr int kActColsV = 256;                        // columns per block: 8 per lane
 constexpr int kColsumGroup = 8;                       // row chunks per block in a launch that only sums columns
 constexpr int kStageGroup = 4;                        // ... and in a launch of one stage
+// Row chunks one block of the activation-backward launch covers; its sum is partial row (first chunk / group) of the stage.
+__host__ __device__ inline int act_chunk_group(const TickArgs& t) {
+  return t.row_chunks > 1 ? (t.colsum_only ? kColsumGroup : (t.sel_p >= 0 ? kStageGroup : 1)) : 1;
+}
 
 // rows r, r + NW, ... < r1 of 8 columns (NW = warps of the block): four rows are loaded before the first is used
 template <typename AT, int ACT, int NW>
@@ -185,9 +189,9 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
   const LinDev& L = s.lin[lvl];
   const int c0 = (blk - start[p]) * kActColsV;
   if (c0 >= L.n_out) return;
-  // a launch that only sums columns gives a block kColsumGroup row chunks (fewer, longer-lived blocks); their sum goes
-  // to the first chunk's partial row and zeros to the others, which the finishing pass adds like any partial
-  const int cg = t.row_chunks > 1 ? (t.colsum_only ? kColsumGroup : (t.sel_p >= 0 ? kStageGroup : 1)) : 1;
+  // a launch that only sums columns, or a launch of one stage, gives a block several row chunks (fewer, longer-lived
+  // blocks); a block's sum is one partial row, and the finishing pass adds as many rows as the launch had blocks
+  const int cg = act_chunk_group(t);
   const int chunk = blockIdx.y * cg;
   const int r0 = chunk * t.chunk_rows, r1 = min(t.T, r0 + cg * t.chunk_rows);
   if (r0 >= t.T) return;
@@ -233,11 +237,7 @@ __global__ void __launch_bounds__(NW * 32) actbwd_kernel(TickArgs t, int lvl) {
 #pragma unroll
     for (int w = 0; w < NW; ++w) a = __fadd_rn(a, red[w][threadIdx.x]);
     if (t.row_chunks == 1) t.a.grad[L.b_off + cc] = d.accum ? __fadd_rn(t.a.grad[L.b_off + cc], a) : a;
-    else {
-      float* part = ws_ptr<float>(t, t.colred_off) + ((uint64_t)p * t.row_chunks + chunk) * (2 * (uint64_t)t.max_dim) + cc;
-      part[0] = a;
-      for (int j = 1; j < cg && chunk + j < t.row_chunks; ++j) part[(uint64_t)j * (2 * (uint64_t)t.max_dim)] = 0.f;
-    }
+    else ws_ptr<float>(t, t.colred_off)[((uint64_t)p * t.row_chunks + blockIdx.y) * (2 * (uint64_t)t.max_dim) + cc] = a;   // partial rows are dense: one per block
   }
 }
 
@@ -267,13 +267,16 @@ __global__ void __launch_bounds__(256) bias_finish_kernel(TickArgs t, int lvl) {
   if (cb >= L.n_out) return;
   const uint64_t ps = 2 * (uint64_t)t.max_dim;
   const float* part = ws_ptr<float>(t, t.colred_off) + (uint64_t)p * t.row_chunks * ps + (c < L.n_out ? c : 0);
+  // partial rows the activation-backward launch of this Linear wrote: one per block of that launch
+  const int cg = t.fin_deferred ? (t.row_chunks > 1 ? (bwd_act(L) != PM_ACT_NONE ? kStageGroup : kColsumGroup) : 1) : act_chunk_group(t);
+  const int n_rows = (t.row_chunks + cg - 1) / cg;
   float sum = 0.f;
-  for (int k0 = warp; k0 < t.row_chunks; k0 += 8 * kFinMaxPer) {
+  for (int k0 = warp; k0 < n_rows; k0 += 8 * kFinMaxPer) {
     float v[kFinMaxPer];
 #pragma unroll
-    for (int u = 0; u < kFinMaxPer; ++u) { const int k = k0 + 8 * u; v[u] = k < t.row_chunks ? part[(uint64_t)k * ps] : 0.f; }
+    for (int u = 0; u < kFinMaxPer; ++u) { const int k = k0 + 8 * u; v[u] = k < n_rows ? part[(uint64_t)k * ps] : 0.f; }
 #pragma unroll
-    for (int u = 0; u < kFinMaxPer; ++u) if (k0 + 8 * u < t.row_chunks) sum = __fadd_rn(sum, v[u]);
+    for (int u = 0; u < kFinMaxPer; ++u) if (k0 + 8 * u < n_rows) sum = __fadd_rn(sum, v[u]);
   }
   __shared__ float red[8][kFinCols];
   red[warp][lane] = sum;
@@ -292,8 +295,10 @@ int deferred_finish_launches(const TickArgs& t) { return (t.row_chunks > 1 ? t.m
 cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t stream) {
   (void)dtype;
   if (t.row_chunks > 1) {
+    TickArgs tf = t;
+    tf.fin_deferred = 1;
     for (int lvl = 0; lvl < t.max_lin; ++lvl)
-      if (t.act_blocks[lvl] > 0) bias_finish_kernel<<<t.act_blocks[lvl] * (kActColsV / kFinCols), 256, 0, stream>>>(t, lvl);
+      if (t.act_blocks[lvl] > 0) bias_finish_kernel<<<t.act_blocks[lvl] * (kActColsV / kFinCols), 256, 0, stream>>>(tf, lvl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -302,7 +307,7 @@ cudaError_t launch_deferred_finish(const TickArgs& t, int dtype, cudaStream_t st
 
 cudaError_t launch_actbwd(const TickArgs& t, int dtype, int lvl, cudaStream_t stream) {
   if (t.act_blocks[lvl] == 0) return cudaSuccess;
-  const int cg = t.row_chunks > 1 ? (t.colsum_only ? kColsumGroup : (t.sel_p >= 0 ? kStageGroup : 1)) : 1;
+  const int cg = act_chunk_group(t);
   dim3 grid(t.act_blocks[lvl], (t.row_chunks + cg - 1) / cg);
   if (t.sel_p >= 0 && t.row_chunks > 1) {
     if (dtype == PM_F32) actbwd_kernel<float, 16><<<grid, 16 * 32, 0, stream>>>(t, lvl);

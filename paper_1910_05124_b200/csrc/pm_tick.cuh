@@ -65,6 +65,8 @@ struct TickArgs {
   // weight-gradient launch that applies the PipeMare update to the Linear matrices in its epilogue (bf16 tensor-core
   // path): dW never reaches the grad arena; the stage's step size, T2 decay and bias corrections come from its table
   // entry, the optimiser constants from here, and the operand-type copy of the new weights goes to lp_base
+  int32_t fin_deferred;   // bias finishing pass launched once for all stages at the end of a microbatch-major backward pass: the partial
+                          // rows were written by launches of one stage (Linears with activation) or by the column-sum-only launch
   int32_t ln_stage;       // LayerNorm backward: a block first brings its rows of x, du and the skip gradient into shared memory
                           // with asynchronous copies (all in flight at once), then works from there (set by the launcher)
   int32_t stash;          // weight stashing (tau_bkwd = tau_fwd for every stage): the backward pass reads the queued version the
