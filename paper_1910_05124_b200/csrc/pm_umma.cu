@@ -160,7 +160,7 @@ template <int MODE>
 __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* lm, const StageDev& s, const StageDyn& d, const LinDev& L,
                                           int p, int lvl, int N, int mrow, int nb, const uint32_t (&r0)[32], const uint32_t (&r1)[32],
                                           uint8_t* obuf, uint32_t obuf_s, int lane, const float4 bias4, int bias_lane0, EpiState& es,
-                                          uint4 (&skq)[8], const __nv_bfloat16* next_skip = nullptr, int next_cols = 0) {
+                                          uint4 (&skq)[8], const __nv_bfloat16* next_skip = nullptr, int next_cols = 0, int yslot_pre = -1) {
   if (MODE == 2 && t.fuse_upd) {                                  // the update is applied here; nothing is stored to the grad arena
     if (t.upd_opt == PM_SGDM) epi_update_block<PM_SGDM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
     else epi_update_block<PM_ADAM>(t, d, L, L.n_out, N, mrow, nb, r0, r1, obuf, lane);
@@ -244,8 +244,9 @@ __device__ __forceinline__ void epi_block(const TickArgs& t, const CUtensorMap* 
   __syncwarp();
   if (lane == 0) {
     if (MODE == 0) {
-      const int yslot = lvl < s.n_lin - 1 ? d.f_slot
-                        : (s.emit_memory ? (int)(d.f_mb % t.mem_depth) : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1)));
+      // (the caller may have formed the slot before it waited for the accumulator: it is the same for every block of a tile)
+      const int yslot = yslot_pre >= 0 ? yslot_pre : (lvl < s.n_lin - 1 ? d.f_slot
+                        : (s.emit_memory ? (int)(d.f_mb % t.mem_depth) : (p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1))));
       if (f32out) {
         tma_store_3d(lm + MAP_Y_OUT, obuf_s, nb, mrow, (int)(d.tick & 1));
         if (nb + 32 < N) tma_store_3d(lm + MAP_Y_OUT, obuf_s + 4096, nb + 32, mrow, (int)(d.tick & 1));
@@ -726,6 +727,9 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
       const float4 bias4 = MODE == 0 ? load_bias4(fwd_small<__nv_bfloat16>(t, s, d, L.b_off, L.b_soff), tl.n0 + half * 128 + 4 * lane, tl.N) : make_float4(0.f, 0.f, 0.f, 0.f);
       uint4 skq[8];                                                   // skip values of the 64-column block in hand (residual stages)
       if (MODE == 0) load_skip64(t, s, d, tl.N, mrow + lane, tl.n0 + half * 128, skq);
+      // ring slot of the forward output, formed while the accumulator completes (the elected lane needs it for its stores)
+      const int yslot_pre = MODE != 0 ? -1 : (lvl < s.n_lin - 1 ? d.f_slot
+                            : (s.emit_memory ? (int)(d.f_mb % t.mem_depth) : (tl.p < t.P - 1 ? d.f_next_xslot : (int)(d.tick & 1))));
       bool ready = mbar_wait(bar_tfull + 8 * acc.idx, acc.phase, abort_flag, status, 34);
       ready = __all_sync(0xffffffffu, ready);                         // tcgen05.ld needs the whole warp
       if (!ready) { ok = false; break; }
@@ -747,7 +751,7 @@ umma_pair_gemm_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const in
         const __nv_bfloat16* nxt = nullptr;
         if (MODE == 0 && c == 0 && s.post == POST_RESIDUAL && mrow + lane < t.T && nb + 64 < tl.N)
           nxt = ws_at<__nv_bfloat16>(t, s.skip_in) + (uint64_t)d.skip_rslot * ((uint64_t)t.T * tl.N) + (uint64_t)(mrow + lane) * tl.N + nb + 64;
-        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es, skq, nxt, tl.N - (nb + 64));
+        epi_block<MODE>(t, lm, s, d, L, tl.p, lvl, tl.N, mrow, nb, r0, r1, obuf, obuf_s, lane, bias4, c * 16, es, skq, nxt, tl.N - (nb + 64), yslot_pre);
       }
       acc.advance(2);
     }
