@@ -1425,13 +1425,14 @@ umma_dgrad_pair_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, const i
 // CTAs; the epilogue warps of both arrive on the leader's tempty.
 constexpr int D1_TILE_M = 256, D1_TILE_N = 128, D1_HALF_N = 64;
 constexpr int D1_MG = 2;                                   // 256-row tiles per converted tile
+constexpr int D1_PF = 4;                                   // k-blocks of fp32 w and delta asked of L2 ahead of the staging ring
 constexpr int D1_NG = 2, D1_NB = 2, D1_NA = 7;             // fp32 staging ring, converted ring, dz ring (3.5 k-blocks of dz in flight)
 constexpr int D1_STG_HALF = TILE_K * D1_HALF_N * 4;        // one fp32 [64 x 64] tile: 16 KB
 constexpr int D1_STG_BYTES = 2 * D1_STG_HALF;
 constexpr int D1_B_BYTES = TILE_K * D1_HALF_N * 2;         // converted [64 k x 64 n] bf16: 8 KB
 constexpr int D1_ACC_COLS = D1_MG * D1_TILE_N;             // 256 columns per accumulator buffer
 constexpr int D1_XF_WARPS = 8, D1_EPI_WARPS = 8;
-constexpr int D1_THREADS = 32 * (3 + D1_XF_WARPS + D1_EPI_WARPS);   // staging producer, MMA issuer, transform, epilogue, dz producer
+constexpr int D1_THREADS = 32 * (4 + D1_XF_WARPS + D1_EPI_WARPS);   // staging producer, MMA issuer, transform, epilogue, dz producer, second MMA issuer
 constexpr int D1_TILE_BYTES = D1_NG * D1_STG_BYTES + D1_NB * D1_B_BYTES + D1_NA * A_BYTES + D1_EPI_WARPS * 4096;
 constexpr int D1_SMEM_BYTES = D1_TILE_BYTES + 1024 + 512;
 
@@ -1480,9 +1481,9 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < D1_NG; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, D1_XF_WARPS); }
-    for (int i = 0; i < D1_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * D1_XF_WARPS); mbar_init(bar_bempty + 8 * i, 1); }
+    for (int i = 0; i < D1_NB; ++i) { mbar_init(bar_bfull + 8 * i, 2 * D1_XF_WARPS); mbar_init(bar_bempty + 8 * i, D1_MG); }   // released by both MMA issuers
     for (int i = 0; i < D1_NA; ++i) { mbar_init(bar_afull + 8 * i, 1); mbar_init(bar_aempty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 2 * D1_EPI_WARPS); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, D1_MG); mbar_init(bar_tempty + 8 * i, 2 * D1_EPI_WARPS); }   // published by both MMA issuers
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1525,9 +1526,21 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
     if (lane == 0) {
       Cursor cs{pair, 0, DgTile{}, false, nullptr, false, 0};
       seek(cs);
+      Cursor cp = cs;                                                 // runs D1_PF k-blocks ahead and asks L2 for them
+      auto prefetch = [&]() {
+        if (cp.done) return;
+        if (cp.tl.m0 == 0) {                                          // the pairs of one row group ask for all: the others run beside them
+          tma_prefetch_2d(cp.lm + MAP_W_F32H, cp.tl.n0 + rank * D1_HALF_N, cp.kb * TILE_K);
+          if (cp.corr) tma_prefetch_2d(cp.lm + MAP_D_F32H, cp.tl.n0 + rank * D1_HALF_N, cp.kb * TILE_K);
+        }
+        step(cp);
+      };
+      for (int i = 0; i < D1_NG; ++i) step(cp);                       // the first D1_NG k-blocks are loaded at once
+      for (int i = 0; i < D1_PF; ++i) prefetch();
       Ring sg{0, 0};
       int issued_sg = 0;
       while (!cs.done) {
+        prefetch();
         if (!mbar_wait(bar_sempty + 8 * sg.idx, sg.phase ^ 1, abort_flag, status, 41)) break;
         const uint32_t sw = stg + sg.idx * D1_STG_BYTES, fb = bar_sfull + 8 * sg.idx;
         mbar_arrive_expect_tx(fb, cs.corr ? D1_STG_BYTES : D1_STG_HALF);
@@ -1575,9 +1588,15 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
         // after these waits: rank 1 needs no wait of its own
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer (leader CTA only) ----------------
+  } else if (warp == 1 || warp == 3 + D1_XF_WARPS + D1_EPI_WARPS) {
+    // ---------------- MMA issuers (leader CTA only): one thread per row tile of a group ----------------
+    // Issuing an MMA, its commits and the barrier polls in front of them cost the issuing thread about 1400 cycles per
+    // k-block of two row tiles, of which the tensor pipe works 512: one thread cannot keep the pipe busy.  The two row tiles
+    // of a group have accumulators of their own, so their MMAs need no order between them: thread `me` waits for the
+    // shared converted tile and for ITS dz tile, issues its four MMAs and commits its dz slot; both threads commit the
+    // converted slot and the accumulator buffer (those barriers count two arrivals).
     if (lane == 0 && rank == 0) {
+      const int me = warp == 1 ? 0 : 1;
       const uint32_t idesc = make_idesc_mn(D1_TILE_M, D1_TILE_N, 0, 1);
       const uint64_t dba = desc_base(16, 1024), dbb = desc_base(D1_B_BYTES, 1024);   // B: one 64-column run per CTA
       Ring br{0, 0}, ar{0, 0}, acc{0, 0};
@@ -1589,28 +1608,25 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
         if (!tl.valid) continue;
         if (!mbar_wait(bar_tempty + 8 * acc.idx, acc.phase ^ 1, abort_flag, status, 43)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * D1_ACC_COLS);
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(acc.idx * D1_ACC_COLS + me * D1_TILE_N);
+        const bool mine = me < tl.n_m;                               // a group at the end of the rows may hold one tile only
         for (int kb = 0; kb < tl.n_kb && ok; ++kb) {
           if (!mbar_wait(bar_bfull + 8 * br.idx, br.phase, abort_flag, status, 44)) { ok = false; break; }
           const uint32_t sb = sB + br.idx * D1_B_BYTES;
-          // both dz tiles first, then the products of the two row tiles interleaved: consecutive MMAs write
-          // different accumulators
-          uint32_t sa[D1_MG], abar[D1_MG];
-          for (int mi = 0; mi < tl.n_m; ++mi) {
-            if (!mbar_wait(bar_afull + 8 * ar.idx, ar.phase, abort_flag, status, 45)) { ok = false; break; }
-            sa[mi] = sA + ar.idx * A_BYTES;
-            abar[mi] = bar_aempty + 8 * ar.idx;
-            ar.advance(D1_NA);
-          }
-          if (!ok) break;
-          tc_fence_after();
+          // the dz slots of this k-block sit in ring order, row tile 0 first; this thread's is the me-th
+          Ring mr = ar;
+          if (me == 1) mr.advance(D1_NA);
+          for (int mi = 0; mi < tl.n_m; ++mi) ar.advance(D1_NA);
+          if (mine) {
+            if (!mbar_wait(bar_afull + 8 * mr.idx, mr.phase, abort_flag, status, 45)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = sA + mr.idx * A_BYTES;
 #pragma unroll
-          for (int k16 = 0; k16 < TILE_K / 16; ++k16)
-            for (int mi = 0; mi < tl.n_m; ++mi)
-              tc_mma_bf16_pair(tmem_acc + (uint32_t)(mi * D1_TILE_N), desc_at(dba, sa[mi] + k16 * 32), desc_at(dbb, sb + k16 * 2048),
-                               idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
-          for (int mi = 0; mi < tl.n_m; ++mi) tc_commit_pair(abar[mi], 3);
-          if (ok) tc_commit_pair(bar_bempty + 8 * br.idx, 3);
+            for (int k16 = 0; k16 < TILE_K / 16; ++k16)
+              tc_mma_bf16_pair(tmem_acc, desc_at(dba, sa + k16 * 32), desc_at(dbb, sb + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            tc_commit_pair(bar_aempty + 8 * mr.idx, 3);
+          }
+          tc_commit_pair(bar_bempty + 8 * br.idx, 3);                 // with no MMA of this thread outstanding it arrives at once
           br.advance(D1_NB);
         }
         if (ok) tc_commit_pair(bar_tfull + 8 * acc.idx, 3);
@@ -1634,27 +1650,43 @@ umma_dgrad_pair128_kernel(TickArgs t, const CUtensorMap* __restrict__ maps, cons
       const bool corr = t.dyn[tl.p].use_delta != 0;
       for (int kb = 0; kb < tl.n_kb; ++kb) {
         bool go = mbar_wait(bar_sfull + 8 * sg.idx, sg.phase, abort_flag, status, 46);
-        go = go && mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 47);
         go = __all_sync(0xffffffffu, go);
         if (!go) { ok = false; break; }
+        // the staged fp32 values go to registers and the staging slot back to its producer at once: the wait for a free
+        // converted slot and the stores into it are then off the slot's round trip (copy latency + this read)
         const uint8_t* src = stg_ptr + sg.idx * D1_STG_BYTES;
-        uint8_t* dst = sB_ptr + br.idx * D1_B_BYTES;
+        float4 w[4], dl[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int r = rbase + 16 * j;                               // k-row
-          const float4 w = *reinterpret_cast<const float4*>(src + r * (D1_HALF_N * 4) + c4 * 16);
-          float v[4] = {w.x, w.y, w.z, w.w};
+          w[j] = *reinterpret_cast<const float4*>(src + r * (D1_HALF_N * 4) + c4 * 16);
+          if (corr) dl[j] = *reinterpret_cast<const float4*>(src + D1_STG_HALF + r * (D1_HALF_N * 4) + c4 * 16);
+        }
+        uint2 o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float v[4] = {w[j].x, w[j].y, w[j].z, w[j].w};
           if (corr) {
-            const float4 dl = *reinterpret_cast<const float4*>(src + D1_STG_HALF + r * (D1_HALF_N * 4) + c4 * 16);
-            v[0] = __fsub_rn(v[0], __fmul_rn(gapf, dl.x)); v[1] = __fsub_rn(v[1], __fmul_rn(gapf, dl.y));   // w - (tau_fwd - tau_bkwd) * delta
-            v[2] = __fsub_rn(v[2], __fmul_rn(gapf, dl.z)); v[3] = __fsub_rn(v[3], __fmul_rn(gapf, dl.w));
+            v[0] = __fsub_rn(v[0], __fmul_rn(gapf, dl[j].x)); v[1] = __fsub_rn(v[1], __fmul_rn(gapf, dl[j].y));   // w - (tau_fwd - tau_bkwd) * delta
+            v[2] = __fsub_rn(v[2], __fmul_rn(gapf, dl[j].z)); v[3] = __fsub_rn(v[3], __fmul_rn(gapf, dl[j].w));
           }
+          o[j] = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+        }
+        __syncwarp();                                                 // every lane's values have arrived (they were used above)
+        if (lane == 0) mbar_arrive(bar_sempty + 8 * sg.idx);
+        go = mbar_wait(bar_bempty + 8 * br.idx, br.phase ^ 1, abort_flag, status, 47);
+        go = __all_sync(0xffffffffu, go);
+        if (!go) { ok = false; break; }
+        uint8_t* dst = sB_ptr + br.idx * D1_B_BYTES;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int r = rbase + 16 * j;
           const uint32_t off = (uint32_t)(r >> 3) * 1024 + (uint32_t)(r & 7) * 128 + ((((uint32_t)c4 >> 1) ^ (uint32_t)(r & 7)) << 4) + ((uint32_t)c4 & 1) * 8;
-          *reinterpret_cast<uint2*>(dst + off) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+          *reinterpret_cast<uint2*>(dst + off) = o[j];
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) { mbar_arrive_cluster(leader_bfull + 8 * br.idx); mbar_arrive(bar_sempty + 8 * sg.idx); }
+        if (lane == 0) mbar_arrive_cluster(leader_bfull + 8 * br.idx);
         br.advance(D1_NB); sg.advance(D1_NG);
       }
     }
