@@ -107,12 +107,14 @@ def test_mb_major_encoder_decoder(cuda_device, compute):
     check_orders_agree(wl, params0, pipe, losses, f32)
 
 
-def test_mb_major_tensor_core_attention_and_pair_tiles(cuda_device):
-    """Sequences of 128 tokens, heads of width 64 and GEMMs of at least 256 rows and columns: the tensor-core
+@pytest.mark.parametrize("seq_len,batch", [(128, 2), (256, 3)])
+def test_mb_major_tensor_core_attention_and_pair_tiles(cuda_device, seq_len, batch):
+    """Sequences of 128 or 256 tokens, heads of width 64 and GEMMs of at least 256 rows and columns: the tensor-core
     attention kernels and the CTA-pair GEMMs, launched one stage at a time, with the weight gradients of all
-    stages in one grouped launch at the end of the backward pass."""
+    stages in one grouped launch at the end of the backward pass.  256 rows are one row tile (a dgrad group of one:
+    the second MMA-issuing thread has nothing to issue), 768 rows are a group of two and a group of one."""
     import torch
-    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=256, n_heads=4, d_ff=512, seq_len=128, batch=2, vocab=264, steps=16)
+    wl = I.cfg5_small(compute="bf16", n_enc=1, n_dec=1, d_model=256, n_heads=4, d_ff=512, seq_len=seq_len, batch=batch, vocab=264, steps=16)
     params0 = I.init_encoder_params(wl)
     res = run_oracle(wl, params0, wl.steps)
     pipe, losses, book = run_gpu_pipeline(wl, params0, wl.steps, loop_order="mb_major")
