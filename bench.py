@@ -61,9 +61,9 @@ def tensor_peak(peaks, clocks):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, throttle reasons and board power with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw,power.limit")
 
     def __init__(self, index):
         self.index, self.rows, self.proc, self.first = index, [], None, 0
@@ -98,7 +98,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, mx, reasons, watts, limit, capped = [], None, set(), [], None, 0
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows[self.first:]:
             if len(r) < 6:
@@ -111,9 +111,20 @@ class ClockSampler:
             for name, v in zip(names, r[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
+            capped += r[5].lower().startswith("active")
+            try:
+                watts.append(float(r[6]))
+                limit = float(r[7])
+            except (IndexError, ValueError):
+                pass
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        watts.sort()
+        out = {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+               "samples": len(sm)}
+        if watts:        # how close the timed region ran to the board's power limit: a capped step trades kernel time for clock
+            out.update({"power_w": watts[len(watts) // 2], "power_limit_w": limit,
+                        "power_capped_samples": capped})
+        return out
 
 
 def dist_setup(n_gpus):
