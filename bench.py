@@ -442,6 +442,10 @@ NCU_TRAFFIC = {
     "gemm_fwd_ratio": (84.2 + 149.1) / (83.9 + 209.7),
     "wgrad_ratio": (211.1 + 24.9) / (205.5 + 42.0),
     "dgrad_ratio": (231.8 + 29.2) / (226.5 + 33.6),
+    # dgrad launched one stage at a time on config 5's widths (profiles/narrow_dgrad_and_ln_backward_cfg5_1+1_layers.md):
+    # six launches read 776.4 MB and wrote 16.7 MB of DRAM against 826.2 MB of dz, fp32 w and delta, and dx (the
+    # dx of a launch is still in L2 when it ends)
+    "dgrad_one_stage_ratio": (776.4 + 16.7) / 826.2,
     # fused update: 2.941 GB at 100 M parameters, momentum SGD (profiles/update_kernel_100M_params.md); pure streaming,
     # so it is scaled by the algorithmic bytes of the launch (30 B/param there; 38 B/param with Adam's second moment)
     "update_bytes_per_param": 29.41,
@@ -631,12 +635,16 @@ def rooflines(res, peaks, steps):
         kname = GEMM_KERNELS[cls]
         if cls == "dgrad" and res.get("plain_dgrad"):
             kname = "umma_pair_gemm_kernel<1> / umma_gemm_kernel<1> (dgrad as a plain GEMM against a queued operand copy)"
+        ratio, note = NCU_TRAFFIC[cls + "_ratio"], "DRAM bytes per launch, scaled from the ncu capture of the 2-layer cut of cfg4 by algorithmic bytes"
+        if cls == "dgrad" and res.get("order") == "mb_major" and not res.get("plain_dgrad") and wl.kind == "encoder":
+            kname = "umma_dgrad_pair128_kernel / umma_dgrad_pair_kernel (dgrad of one stage per launch, weights corrected while loading)"
+            ratio, note = NCU_TRAFFIC["dgrad_one_stage_ratio"], "DRAM bytes per launch, scaled from the ncu capture of one-stage launches on config 5's widths (1 + 1 layers) by algorithmic bytes"
         out[cls] = {"kernel": kname, "bound": "tensor", "achieved": round(tfs, 1), "peak": tf_peak, "unit": "TFLOP/s",
                     "frac": round(tfs / tf_peak, 4), "of": f"{peaks['kind']} ({tf_kind} bf16 matmul; the median SM clock of the timed region decides)",
                     "frac_of_burst": round(tfs / peaks["tf_burst"], 4), "frac_of_sustained": round(tfs / peaks["tf_sustained"], 4),
                     "frac_of_nominal_2250TFs": round(tfs / 2250.0, 4),
-                    "traffic": int(NCU_TRAFFIC[cls + "_ratio"] * gemm_bytes(wl)[cls] / launches),
-                    "traffic_note": "DRAM bytes per launch, scaled from the ncu capture of the 2-layer cut of cfg4 by algorithmic bytes",
+                    "traffic": int(ratio * gemm_bytes(wl)[cls] / launches),
+                    "traffic_note": note,
                     "algorithmic_bytes_per_step": gemm_bytes(wl)[cls], "algorithmic_flops_per_step": flops[cls],
                     "launches_per_step": launches, "avg_ms_per_step": round(per_tick[cls], 5), "share_of_step": share}
     dominant = max(out, key=lambda k: out[k].get("share_of_step") or 0.0)
