@@ -46,3 +46,33 @@ def test_reference_arm_runs_without_a_gpu():
     sys.path.insert(0, ROOT)
     import bench
     assert r["config"]["workload"] == bench.WORKLOADS["cfg4"]      # the same string the CUDA arm prints
+
+
+def test_clock_sampler_summary_from_rows():
+    """The summary of the sampled nvidia-smi rows: median clock, reasons seen, board power; rows taken before the
+    mark and malformed rows are left out, and rows without the power columns still give the clock figures."""
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class Done:
+        def terminate(self): pass
+        def wait(self, timeout=None): return 0
+
+    s = bench.ClockSampler(0)
+    s.proc = Done()
+    s.rows = [["300", "1965", "Not Active", "Not Active", "Not Active", "Not Active", "120.0", "1000.00"],   # before the mark
+              ["1965", "1965", "Not Active", "Not Active", "Not Active", "Not Active", "700.5", "1000.00"],
+              ["1905", "1965", "Not Active", "Not Active", "Not Active", "Active", "905.0", "1000.00"],
+              ["1890", "1965", "Not Active", "Not Active", "Not Active", "Active", "990.0", "1000.00"],
+              ["[N/A]", "1965", "Not Active", "Not Active", "Not Active", "Active", "1.0", "1000.00"],
+              ["short", "row"]]
+    s.first = 1
+    out = s.stop()
+    assert out["sm_mhz"] == 1905.0 and out["sm_max_mhz"] == 1965.0 and out["samples"] == 3
+    assert out["reasons"] == ["sw_power_cap"]
+    assert out["power_w"] == 905.0 and out["power_limit_w"] == 1000.0 and out["power_capped_samples"] == 2
+    s = bench.ClockSampler(0)
+    s.proc = Done()
+    s.rows = [["1800", "1965", "Not Active", "Active", "Not Active", "Not Active"]]
+    out = s.stop()
+    assert out["sm_mhz"] == 1800.0 and out["reasons"] == ["hw_thermal_slowdown"] and "power_w" not in out
